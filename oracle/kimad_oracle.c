@@ -1,0 +1,446 @@
+/*
+ * kimad_oracle.c -- plain CPU oracle for the worker-side Kimad+ compression pass.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, by-the-definition reference
+ * that the tests, the smoke check and the benchmark's CPU-baseline leg compare
+ * the CUDA library against.  It shares no code, header, table or constant with
+ * the CUDA library and must never be called from the product path.
+ *
+ * What it computes, per simulated worker and per step (paper notation: u is the
+ * fresh update / gradient, u^ is the EF21 estimator, called g here):
+ *
+ *   O1  d = u - u^                     (Section 3 footnote; Algorithm 1, upload line;
+ *                                       Eq. 6: the compressor is applied to grad - u^)
+ *   O2  TopK order                     (Section 2.2: "K largest absolute value" --
+ *                                       ties: larger |x| first, then lower index)
+ *   O3  k-table from the ratio grid    (Section 3.2: discrete set of ratios per layer;
+ *                                       Omega = {TopK : K > 0}, Section 4.2)
+ *   O4  err_l(k) = ||d_l - TopK_k(d_l)||^2   (Eq. 4; "Errors" matrix of Algorithm 3)
+ *   O5  byte costs, budget c, budget cells   (Eq. 2, Eq. 3; "Costs" matrix of Algorithm 3)
+ *   O6  knapsack DP over the budget axis     (Section 3.2, Algorithm 3)
+ *   O7  TopK select + sparse pack            (Algorithm 1, upload line)
+ *   O8  EF21 estimator update u^ += C(d)     (Algorithm 1 aggregate line, Eq. 6)
+ *
+ * Floating point: the element-wise operations (O1, O8, the DP adds) are single
+ * IEEE binary32 operations in a fixed order, because the compared results must be
+ * bit-identical.  The error curve is accumulated in binary64 from the smallest
+ * magnitude upward and rounded to binary32 once.
+ *
+ * Pins (tests/test_oracle_*.py): numpy float32 re-computation for O1/O8, full
+ * stable sort + math.fsum for O2/O4/O7, closed forms for d_i = i+1, exhaustive
+ * enumeration of all K^L assignments for O6, the 0/1-knapsack special case, a
+ * hand-computed three-layer example (tests/golden/), torch's bfloat16 cast for
+ * the bf16 rounding.  The whole-step composition has no value printed in the
+ * paper to compare with: it is pinned by the identities g_new - g = C(d),
+ * ||d - C(d)||^2 = err and sum(bytes) <= c only.
+ *
+ * Build: gcc -O2 -ffp-contract=off -fopenmp -shared -fPIC (see kimad_oracle.py).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define KO_OK 0
+#define KO_STATUS_INFEASIBLE 1 /* no assignment fits the budget: every layer takes j = 0 */
+#define KO_STATUS_PLATEAU 2    /* budget covers the largest candidate of every layer      */
+#define KO_ERR_ARG (-1)
+#define KO_ERR_NOMEM (-2)
+#define KO_ERR_CAPACITY (-3)
+
+typedef struct {
+    uint32_t key; /* magnitude bit pattern, bits(d) & 0x7fffffff */
+    uint32_t idx; /* layer-local index */
+} ko_pair;
+
+static uint32_t f2u(float f) {
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    return u;
+}
+static float u2f(uint32_t u) {
+    float f;
+    memcpy(&f, &u, 4);
+    return f;
+}
+
+/* O2: descending magnitude, then ascending index.  +0 and -0 share key 0. */
+static int ko_cmp_order(const void* a, const void* b) {
+    const ko_pair* x = (const ko_pair*)a;
+    const ko_pair* y = (const ko_pair*)b;
+    if (x->key != y->key) return x->key > y->key ? -1 : 1;
+    if (x->idx != y->idx) return x->idx < y->idx ? -1 : 1;
+    return 0;
+}
+static int ko_cmp_u32(const void* a, const void* b) {
+    uint32_t x = *(const uint32_t*)a, y = *(const uint32_t*)b;
+    return x < y ? -1 : (x > y ? 1 : 0);
+}
+
+/* round-to-nearest-even binary32 -> bfloat16 bit pattern (finite inputs). */
+uint16_t ko_bf16_rne(float x) {
+    uint32_t u = f2u(x);
+    uint32_t lsb = (u >> 16) & 1u;
+    u += 0x7fffu + lsb;
+    return (uint16_t)(u >> 16);
+}
+float ko_bf16_to_f32(uint16_t h) { return u2f(((uint32_t)h) << 16); }
+
+/* O1 */
+void ko_diff(const float* grad, const float* g, float* d, uint64_t n) {
+    for (uint64_t i = 0; i < n; ++i) d[i] = grad[i] - g[i];
+}
+
+/* O3: k_{l,j} = min(n_l, max(1, ceil(r_j * n_l))) with r_j and the product in binary64. */
+int ko_k_table(const uint64_t* layer_sizes, uint32_t L, const double* ratios, uint32_t K,
+               uint64_t* k_out /* [L][K] */) {
+    if (!layer_sizes || !ratios || !k_out || L == 0 || K == 0) return KO_ERR_ARG;
+    for (uint32_t j = 0; j < K; ++j) {
+        if (!(ratios[j] > 0.0) || ratios[j] > 1.0) return KO_ERR_ARG;
+        if (j > 0 && !(ratios[j] > ratios[j - 1])) return KO_ERR_ARG; /* grid strictly ascending */
+    }
+    for (uint32_t l = 0; l < L; ++l) {
+        uint64_t n = layer_sizes[l];
+        if (n == 0 || n > 0xffffffffull) return KO_ERR_ARG;
+        for (uint32_t j = 0; j < K; ++j) {
+            double x = ceil(ratios[j] * (double)n);
+            uint64_t k = (uint64_t)x;
+            if (k < 1) k = 1;
+            if (k > n) k = n;
+            k_out[(size_t)l * K + j] = k;
+        }
+    }
+    return KO_OK;
+}
+
+/* sorted (key desc, idx asc) copy of a layer */
+static ko_pair* ko_sorted_pairs(const float* d, uint64_t n) {
+    ko_pair* p = (ko_pair*)malloc((size_t)(n ? n : 1) * sizeof(ko_pair));
+    if (!p) return NULL;
+    for (uint64_t i = 0; i < n; ++i) {
+        p[i].key = f2u(d[i]) & 0x7fffffffu;
+        p[i].idx = (uint32_t)i;
+    }
+    qsort(p, (size_t)n, sizeof(ko_pair), ko_cmp_order);
+    return p;
+}
+
+/* O4 on an already sorted layer.  k[] must be non-decreasing, 1 <= k <= n.
+ * err[j]  = sum of squares of the entries ranked >= k[j], added from the last rank
+ *           (smallest magnitude) upward in binary64, rounded to binary32 once
+ * tau[j]  = key of the k[j]-th entry (the selection threshold)
+ * keep_eq[j] = how many entries whose key equals tau[j] are kept (the lowest indices)
+ * n_gt[j], n_eq[j] = entries with key > tau[j], key == tau[j] */
+static int ko_curve_sorted(const ko_pair* p, uint64_t n, const uint64_t* k, uint32_t K, float* err,
+                           uint32_t* tau, uint32_t* keep_eq, uint32_t* n_gt, uint32_t* n_eq) {
+    for (uint32_t j = 0; j < K; ++j) {
+        if (k[j] < 1 || k[j] > n) return KO_ERR_ARG;
+        if (j > 0 && k[j] < k[j - 1]) return KO_ERR_ARG;
+    }
+    double acc = 0.0;
+    uint64_t rank = n;
+    for (uint32_t jj = K; jj-- > 0;) {
+        while (rank > k[jj]) {
+            --rank;
+            double v = (double)u2f(p[rank].key);
+            acc += v * v;
+        }
+        if (err) err[jj] = (float)acc;
+    }
+    for (uint32_t j = 0; j < K; ++j) {
+        uint32_t t = p[k[j] - 1].key;
+        uint64_t lo = k[j] - 1, hi = k[j];
+        while (lo > 0 && p[lo - 1].key == t) --lo;
+        while (hi < n && p[hi].key == t) ++hi;
+        if (tau) tau[j] = t;
+        if (n_gt) n_gt[j] = (uint32_t)lo;
+        if (n_eq) n_eq[j] = (uint32_t)(hi - lo);
+        if (keep_eq) keep_eq[j] = (uint32_t)(k[j] - lo);
+    }
+    return KO_OK;
+}
+
+/* O4 for one layer. */
+int ko_layer_curve(const float* d, uint64_t n, const uint64_t* k, uint32_t K, float* err,
+                   uint32_t* tau, uint32_t* keep_eq, uint32_t* n_gt, uint32_t* n_eq) {
+    if (!d || n == 0 || n > 0xffffffffull || !k || K == 0) return KO_ERR_ARG;
+    ko_pair* p = ko_sorted_pairs(d, n);
+    if (!p) return KO_ERR_NOMEM;
+    int rc = ko_curve_sorted(p, n, k, K, err, tau, keep_eq, n_gt, n_eq);
+    free(p);
+    return rc;
+}
+
+/* O7 on a sorted layer: the first k entries of the order, emitted by ascending index.
+ * value_dtype 0: val is float[k] holding d_i; 1: val is uint16_t[k] holding bf16_rne(d_i). */
+static int ko_pack_sorted(const ko_pair* p, const float* d, uint64_t k, uint32_t value_dtype,
+                          uint32_t* idx_out, void* val_out) {
+    for (uint64_t i = 0; i < k; ++i) idx_out[i] = p[i].idx;
+    qsort(idx_out, (size_t)k, sizeof(uint32_t), ko_cmp_u32);
+    for (uint64_t i = 0; i < k; ++i) {
+        float v = d[idx_out[i]];
+        if (value_dtype == 0)
+            ((float*)val_out)[i] = v;
+        else
+            ((uint16_t*)val_out)[i] = ko_bf16_rne(v);
+    }
+    return KO_OK;
+}
+
+int ko_select_pack(const float* d, uint64_t n, uint64_t k, uint32_t value_dtype, uint32_t* idx_out,
+                   void* val_out) {
+    if (!d || n == 0 || n > 0xffffffffull || k < 1 || k > n || value_dtype > 1 || !idx_out || !val_out)
+        return KO_ERR_ARG;
+    ko_pair* p = ko_sorted_pairs(d, n);
+    if (!p) return KO_ERR_NOMEM;
+    int rc = ko_pack_sorted(p, d, k, value_dtype, idx_out, val_out);
+    free(p);
+    return rc;
+}
+
+/* O8: g_i <- g_i + v_i on the kept entries, v_i the value actually sent. */
+void ko_state_update(float* g, const uint32_t* idx, const void* val, uint64_t k, uint32_t value_dtype) {
+    for (uint64_t i = 0; i < k; ++i) {
+        float v = value_dtype == 0 ? ((const float*)val)[i] : ko_bf16_to_f32(((const uint16_t*)val)[i]);
+        g[idx[i]] = g[idx[i]] + v;
+    }
+}
+
+/* O5: c = floor(B * t) in binary64 (B in bytes/s, t in s). */
+uint64_t ko_budget_bytes(double bandwidth_bytes_per_s, double t_target_s) {
+    double c = floor(bandwidth_bytes_per_s * t_target_s);
+    if (!(c > 0.0)) return 0;
+    if (c >= 18446744073709551615.0) return 0xffffffffffffffffull;
+    return (uint64_t)c;
+}
+
+/* O5: bytes_{l,j} = k_{l,j} * (4 + vb); cells_{l,j} = ceil(bytes * D / c).
+ * Returns KO_STATUS_PLATEAU when c covers the largest candidate of every layer,
+ * KO_STATUS_INFEASIBLE when c == 0 (cells then undefined), else 0. */
+int ko_units(const uint64_t* k_table, uint32_t L, uint32_t K, uint32_t value_dtype, uint64_t c, uint32_t D,
+             uint64_t* units_out /* [L][K] */) {
+    uint64_t bpe = value_dtype == 0 ? 8 : 6;
+    uint64_t full = 0;
+    for (uint32_t l = 0; l < L; ++l) full += k_table[(size_t)l * K + (K - 1)] * bpe;
+    if (c >= full) return KO_STATUS_PLATEAU;
+    if (c == 0) return KO_STATUS_INFEASIBLE;
+    for (uint32_t l = 0; l < L; ++l)
+        for (uint32_t j = 0; j < K; ++j) {
+            uint64_t bytes = k_table[(size_t)l * K + j] * bpe;
+            units_out[(size_t)l * K + j] = (bytes * (uint64_t)D + c - 1) / c;
+        }
+    return KO_OK;
+}
+
+/* O6: Algorithm 3 read with the budget as the knapsack axis (D + 1 cells) and the
+ * un-discretised binary32 error as the value.  Layer 1 is treated like every other
+ * layer, from a virtual row prev = [0, inf, inf, ...].  Candidates in ascending j,
+ * strict '<' (the first candidate that reaches a value keeps the cell), final cell =
+ * the lowest b attaining the minimum, then the backward walk through PD.
+ * Returns 0 or KO_STATUS_INFEASIBLE (then j_out is all zero). */
+int ko_dp(const float* err /* [L][K] */, const uint64_t* units /* [L][K] */, uint32_t L, uint32_t K,
+          uint32_t D, uint32_t* j_out /* [L] */, float* best_value, uint32_t* best_cell) {
+    if (!err || !units || !j_out || L == 0 || K == 0 || D == 0) return KO_ERR_ARG;
+    size_t row = (size_t)D + 1;
+    float* prev = (float*)malloc(row * sizeof(float));
+    float* cur = (float*)malloc(row * sizeof(float));
+    uint32_t* PD = (uint32_t*)malloc(row * L * sizeof(uint32_t));
+    if (!prev || !cur || !PD) {
+        free(prev); free(cur); free(PD);
+        return KO_ERR_NOMEM;
+    }
+    prev[0] = 0.0f;
+    for (size_t b = 1; b < row; ++b) prev[b] = INFINITY;
+    for (uint32_t l = 0; l < L; ++l) {
+        for (size_t b = 0; b < row; ++b) { cur[b] = INFINITY; PD[(size_t)l * row + b] = 0; }
+        for (uint32_t j = 0; j < K; ++j) {
+            uint64_t u = units[(size_t)l * K + j];
+            if (u > D) continue;
+            float e = err[(size_t)l * K + j];
+            for (size_t b = (size_t)u; b < row; ++b) {
+                float t = prev[b - u] + e;
+                if (t < cur[b]) { cur[b] = t; PD[(size_t)l * row + b] = j; }
+            }
+        }
+        float* sw = prev; prev = cur; cur = sw;
+    }
+    size_t bstar = 0;
+    for (size_t b = 1; b < row; ++b)
+        if (prev[b] < prev[bstar]) bstar = b;
+    int status = KO_OK;
+    if (!(prev[bstar] < INFINITY)) {
+        status = KO_STATUS_INFEASIBLE;
+        for (uint32_t l = 0; l < L; ++l) j_out[l] = 0;
+    } else {
+        size_t b = bstar;
+        for (uint32_t l = L; l-- > 0;) {
+            uint32_t j = PD[(size_t)l * row + b];
+            j_out[l] = j;
+            b -= (size_t)units[(size_t)l * K + j];
+        }
+    }
+    if (best_value) *best_value = prev[bstar];
+    if (best_cell) *best_cell = (uint32_t)bstar;
+    free(prev); free(cur); free(PD);
+    return status;
+}
+
+/* Per-worker statistics reported by ko_step. */
+typedef struct {
+    uint64_t budget_bytes; /* c */
+    uint64_t used_bytes;   /* sum_l bytes_{l, j_l} */
+    uint64_t n_selected;   /* sum_l k_l */
+    float total_err;       /* err_{1,j_1} + ... + err_{L,j_L}, added left to right in binary32 */
+    int32_t status;        /* 0, KO_STATUS_INFEASIBLE or KO_STATUS_PLATEAU */
+} ko_stats;
+
+void ko_set_threads(int n) {
+#ifdef _OPENMP
+    if (n > 0) omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}
+int ko_get_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* The whole pass (O1..O8) for W workers.  Layout:
+ *   grads, state : [W][stride] binary32, layers concatenated in list order (stride >= N)
+ *   err/tau/keep_eq out : [W][L][K];  j_out/k_out : [W][L]
+ *   idx_out : [W][cap] layer-local indices; val_out : [W][cap] float or uint16 (bf16)
+ *   offs_out : [W][L+1] running sum of k_l
+ * state is updated in place.  When inject_err != NULL the DP consumes that [W][L][K] table
+ * instead of the curves computed here (the curves are still computed and returned). */
+int ko_step(const uint64_t* layer_sizes, uint32_t L, uint32_t W, const double* ratios, uint32_t K, uint32_t D,
+            uint32_t value_dtype, uint64_t stride, const float* grads, float* state,
+            const double* bandwidth_bytes_per_s, double t_target_s, const float* inject_err, float* err_out,
+            uint32_t* tau_out, uint32_t* keep_eq_out, uint32_t* j_out, uint32_t* k_out, uint32_t* idx_out,
+            void* val_out, uint64_t cap, uint64_t* offs_out, ko_stats* stats_out) {
+    if (!layer_sizes || !ratios || !grads || !state || !bandwidth_bytes_per_s || L == 0 || W == 0 || K == 0 ||
+        value_dtype > 1)
+        return KO_ERR_ARG;
+    uint64_t N = 0;
+    for (uint32_t l = 0; l < L; ++l) N += layer_sizes[l];
+    if (stride < N) return KO_ERR_ARG;
+    uint64_t* ktab = (uint64_t*)malloc((size_t)L * K * sizeof(uint64_t));
+    uint64_t* loff = (uint64_t*)malloc(((size_t)L + 1) * sizeof(uint64_t));
+    float* err = (float*)malloc((size_t)W * L * K * sizeof(float));
+    uint32_t* jsel = (uint32_t*)malloc((size_t)W * L * sizeof(uint32_t));
+    ko_stats* st = (ko_stats*)malloc((size_t)W * sizeof(ko_stats));
+    float* d = (float*)malloc((size_t)W * (N ? N : 1) * sizeof(float));
+    int rc = KO_OK;
+    int fail = 0;
+    const uint64_t bpe = value_dtype == 0 ? 8 : 6; /* bytes per kept entry: u32 index + value */
+    const size_t vsz = value_dtype == 0 ? 4 : 2;
+    if (!ktab || !loff || !err || !jsel || !st || !d) { rc = KO_ERR_NOMEM; goto done; }
+    rc = ko_k_table(layer_sizes, L, ratios, K, ktab);
+    if (rc != KO_OK) goto done;
+    loff[0] = 0;
+    for (uint32_t l = 0; l < L; ++l) loff[l + 1] = loff[l] + layer_sizes[l];
+
+    /* O1 + O4: difference and error curve of every (worker, layer) */
+#pragma omp parallel for schedule(dynamic, 1) collapse(2)
+    for (uint32_t w = 0; w < W; ++w)
+        for (uint32_t l = 0; l < L; ++l) {
+            uint64_t n = layer_sizes[l];
+            float* dl = d + (size_t)w * N + loff[l];
+            ko_diff(grads + (size_t)w * stride + loff[l], state + (size_t)w * stride + loff[l], dl, n);
+            size_t o = ((size_t)w * L + l) * K;
+            int r = ko_layer_curve(dl, n, ktab + (size_t)l * K, K, err + o, tau_out ? tau_out + o : NULL,
+                                   keep_eq_out ? keep_eq_out + o : NULL, NULL, NULL);
+            if (r != KO_OK) {
+#pragma omp atomic write
+                fail = r;
+            }
+        }
+    if (fail) { rc = fail; goto done; }
+    if (err_out) memcpy(err_out, err, (size_t)W * L * K * sizeof(float));
+
+    /* O5 + O6 per worker */
+    for (uint32_t w = 0; w < W; ++w) {
+        const float* e = (inject_err ? inject_err : err) + (size_t)w * L * K;
+        uint64_t c = ko_budget_bytes(bandwidth_bytes_per_s[w], t_target_s);
+        uint64_t* units = (uint64_t*)malloc((size_t)L * K * sizeof(uint64_t));
+        if (!units) { rc = KO_ERR_NOMEM; goto done; }
+        int s = ko_units(ktab, L, K, value_dtype, c, D, units);
+        uint32_t* js = jsel + (size_t)w * L;
+        if (s == KO_STATUS_PLATEAU) {
+            for (uint32_t l = 0; l < L; ++l) js[l] = K - 1;
+        } else if (s == KO_STATUS_INFEASIBLE) {
+            for (uint32_t l = 0; l < L; ++l) js[l] = 0;
+        } else {
+            s = ko_dp(e, units, L, K, D, js, NULL, NULL);
+            if (s < 0) { free(units); rc = s; goto done; }
+        }
+        free(units);
+        st[w].budget_bytes = c;
+        st[w].status = s;
+        st[w].used_bytes = 0;
+        st[w].n_selected = 0;
+        float tot = 0.0f;
+        for (uint32_t l = 0; l < L; ++l) {
+            uint64_t k = ktab[(size_t)l * K + js[l]];
+            st[w].used_bytes += k * bpe;
+            st[w].n_selected += k;
+            tot = tot + e[(size_t)l * K + js[l]];
+        }
+        st[w].total_err = tot;
+        if (st[w].n_selected > cap && idx_out) { rc = KO_ERR_CAPACITY; goto done; }
+    }
+
+    /* O7 + O8 */
+    for (uint32_t w = 0; w < W; ++w) {
+        uint64_t run = 0;
+        for (uint32_t l = 0; l < L; ++l) {
+            if (offs_out) offs_out[(size_t)w * (L + 1) + l] = run;
+            run += ktab[(size_t)l * K + jsel[(size_t)w * L + l]];
+        }
+        if (offs_out) offs_out[(size_t)w * (L + 1) + L] = run;
+    }
+#pragma omp parallel for schedule(dynamic, 1) collapse(2)
+    for (uint32_t w = 0; w < W; ++w)
+        for (uint32_t l = 0; l < L; ++l) {
+            uint64_t n = layer_sizes[l];
+            uint32_t j = jsel[(size_t)w * L + l];
+            uint64_t k = ktab[(size_t)l * K + j];
+            if (j_out) j_out[(size_t)w * L + l] = j;
+            if (k_out) k_out[(size_t)w * L + l] = (uint32_t)k;
+            uint64_t off = 0;
+            for (uint32_t q = 0; q < l; ++q) off += ktab[(size_t)q * K + jsel[(size_t)w * L + q]];
+            const float* dl = d + (size_t)w * N + loff[l];
+            uint32_t* ib;
+            void* vb;
+            uint32_t* itmp = NULL;
+            void* vtmp = NULL;
+            if (idx_out && val_out) {
+                ib = idx_out + (size_t)w * cap + off;
+                vb = (char*)val_out + ((size_t)w * cap + off) * vsz;
+            } else {
+                itmp = (uint32_t*)malloc((size_t)k * sizeof(uint32_t));
+                vtmp = malloc((size_t)k * vsz);
+                ib = itmp;
+                vb = vtmp;
+            }
+            int r = (ib && vb) ? ko_select_pack(dl, n, k, value_dtype, ib, vb) : KO_ERR_NOMEM;
+            if (r == KO_OK) ko_state_update(state + (size_t)w * stride + loff[l], ib, vb, k, value_dtype);
+            else {
+#pragma omp atomic write
+                fail = r;
+            }
+            free(itmp);
+            free(vtmp);
+        }
+    if (fail) { rc = fail; goto done; }
+    if (stats_out) memcpy(stats_out, st, (size_t)W * sizeof(ko_stats));
+done:
+    free(ktab); free(loff); free(err); free(jsel); free(st); free(d);
+    return rc;
+}
