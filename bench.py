@@ -1,0 +1,325 @@
+#!/usr/bin/env python
+"""Benchmark of the Kimad+ compression pass on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 1..5] [--impl kimad|reference]
+
+One "step" is one kimad_step(): the whole hot path (EF21 difference, error curves, knapsack DP,
+Top-K select, pack, EF21 update) for all simulated workers of one GPU on one batch of synthetic
+gradients.  Prints ONE JSON line (rank 0).  With N > 1 (torchrun) every rank runs its own set of
+workers on its own GPU (the path shards by worker: no collective on the data path) and the time is
+the maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2312_08053_b200 import workloads  # noqa: E402
+from paper_2312_08053_b200.dist import max_over_ranks, barrier, init_distributed  # noqa: E402
+
+METRIC = "compressed_gradient_elements_per_second"
+UNIT = "elements/s"
+
+# DRAM traffic of the dominant kernel per input element, from the ncu capture summarised under
+# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum of one launch / elements of that launch).
+NCU_TRAFFIC_BYTES_PER_ELEM = {"diff_hist1": None}
+
+# algorithmic bytes per input element of each stage (what the stage must move at least once)
+STAGE_ALGO_BYTES = {"diff_hist1": 12.0,  # read grad + g, write d
+                    "hist2": 4.0, "hist3": 4.0, "select_count": 4.0, "select_write": 4.0}
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        return float(json.load(open(p))["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_id):
+        self.rows, self.proc, self.gpu_id = [], None, gpu_id
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu_id), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self):
+        if self.proc is None:
+            return
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+
+    def summary(self, t0, t1):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        rows = [r for (t, r) in self.rows if t0 <= t <= t1] or [r for (_, r) in self.rows]
+        for r in rows:
+            f = [x.strip() for x in r.split(",")]
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except Exception:
+                continue
+            for name, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def run_reference(args, rank):
+    """The oracle, as it stands, on the host cores: each step is one oracle pass over a bounded sample
+    (shrunk tensors, same layer list / distributions / budget trace) of the configured workload."""
+    if rank != 0:
+        return
+    from oracle import kimad_oracle as ko
+
+    wl_full = workloads.workload(args.config)
+    target = 3_000_000
+    div = max(1, int(np.ceil(wl_full.N * wl_full.n_workers / target)))
+    wl = workloads.workload(args.config, div)
+    bw = workloads.bandwidth_trace(wl, 64)
+    grads = [workloads.gradients(wl, s).numpy() for s in range(2)]
+    state = np.zeros((wl.n_workers, wl.N), np.float32)
+    times = []
+    for s in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        r = ko.step(wl.layer_sizes, wl.n_workers, wl.ratio_grid, wl.D, wl.value_dtype, grads[s % 2], state,
+                    bw[s % len(bw)], wl.t_target, cap=wl.N)
+        dt = time.perf_counter() - t0
+        state = r.state
+        if s >= args.warmup:
+            times.append(dt)
+    ms = 1e3 * float(np.mean(times))
+    elems = wl.N * wl.n_workers
+    val = elems / (ms * 1e-3)
+    sample = f"{wl.name}: {wl.n_workers} workers x {wl.N} elements per step (tensors shrunk {div}x)"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": wl_full.name, "cfg": args.config, "sample": sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": ko.get_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def cpu_baseline(cfg):
+    """Oracle timed on a bounded sample (about 10-30 s of CPU work) of the same workload."""
+    from oracle import kimad_oracle as ko
+
+    wl_full = workloads.workload(cfg)
+    total = wl_full.N * wl_full.n_workers
+
+    def one(target):
+        div = max(1, int(np.ceil(total / target)))
+        wl = workloads.workload(cfg, div)
+        bw = workloads.bandwidth_trace(wl, 8)
+        grads = workloads.gradients(wl, 0).numpy()
+        state = np.zeros_like(grads)
+        t0 = time.perf_counter()
+        ko.step(wl.layer_sizes, wl.n_workers, wl.ratio_grid, wl.D, wl.value_dtype, grads, state, bw[3], wl.t_target,
+                cap=wl.N)
+        return wl, div, time.perf_counter() - t0
+
+    wl, div, dt = one(8_000_000)              # calibration run, not reported
+    rate = wl.N * wl.n_workers / dt
+    wl, div, dt = one(min(total, max(8_000_000, rate * 15.0)))  # about 15 s of oracle work
+    return {"value": wl.N * wl.n_workers / dt, "unit": UNIT, "cores": ko.get_threads(), "kind": "oracle",
+            "sample": f"1 oracle step on {wl.name}: {wl.n_workers} workers x {wl.N} elements "
+                      f"(tensors shrunk {div}x), {dt:.1f} s"}
+
+
+def run_kimad(args, rank, world):
+    import torch
+
+    from paper_2312_08053_b200 import binding as kb
+
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", 0)))
+    torch.cuda.set_device(dev)
+    wl = workloads.workload(args.config)
+    W, N, L = wl.n_workers, wl.N, wl.L
+    bw = workloads.bandwidth_trace(wl)
+    bpe = 8 if wl.value_dtype == 0 else 6
+    dense_cap = N
+    cap = int(min(dense_cap, np.max(bw) * wl.t_target / bpe + L + 1))
+    ctx = kb.new_context(wl.layer_sizes, W, wl.ratio_grid, device=dev, D=wl.D, value_dtype=wl.value_dtype,
+                         max_packed_elems=cap)
+    out = kb.Packed(ctx, device=dev)
+    n_bufs = 2
+    # fresh gradients per buffer; every rank draws its own streams (seed offset by rank)
+    grads = [workloads.gradients(wl, 1000 * rank + s, device=dev) for s in range(n_bufs)]
+    state = torch.zeros((W, N), dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step(s):
+        kb.kimad_step(ctx, grads[s % n_bufs], state, bw[s % len(bw)], wl.t_target, out, stream)
+
+    for s in range(args.warmup):
+        step(s)
+    torch.cuda.synchronize()
+    props = torch.cuda.get_device_properties(dev)
+    gpu_id = str(getattr(props, "uuid", "")) or str(dev.index)
+    if "-" in gpu_id and not gpu_id.startswith("GPU-"):
+        gpu_id = "GPU-" + gpu_id
+    sampler = ClockSampler(gpu_id)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    launches0 = kb.kimad_launch_count(ctx)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    barrier()
+    torch.cuda.synchronize()
+    t_wall0 = time.time()
+    ev[0].record(stream)
+    for s in range(args.steps):
+        step(args.warmup + s)
+        ev[s + 1].record(stream)
+    torch.cuda.synchronize()
+    barrier()
+    t_wall1 = time.time()
+    total_ms = ev[0].elapsed_time(ev[-1])
+    per_step = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
+    launches = kb.kimad_launch_count(ctx) - launches0
+    total_ms = max_over_ranks(total_ms)
+    ms_per_step = total_ms / args.steps
+    elems_per_step = W * N * world
+    value = elems_per_step / (ms_per_step * 1e-3)
+    status, _ = kb.kimad_get_k(ctx)
+    if status < 0:
+        raise RuntimeError(f"kimad step failed on rank {rank}: {kb.kimad_strerror(status)}")
+
+    # ---- end to end: host buffers in, packed message out, copies inside the timed region
+    host_grads = [g.cpu().pin_memory() for g in grads]
+    dev_in = torch.empty_like(grads[0])
+    h_stats = torch.empty_like(out.stats, device="cpu").pin_memory()
+    h_idx = torch.empty((W, cap), dtype=torch.int32).pin_memory()
+    h_val = torch.empty((W, cap), dtype=out.val.dtype).pin_memory()
+    e2e_steps = max(3, min(args.steps, 10))
+    d2h_bytes = 0
+
+    def e2e_step(s):
+        nonlocal d2h_bytes
+        dev_in.copy_(host_grads[s % n_bufs], non_blocking=True)
+        kb.kimad_step(ctx, dev_in, state, bw[s % len(bw)], wl.t_target, out, stream)
+        h_stats.copy_(out.stats, non_blocking=True)
+        stream.synchronize()
+        st = h_stats.numpy().view(kb.STATS_DTYPE).reshape(-1)
+        moved = h_stats.numel()
+        for w in range(W):
+            n = int(st["n_selected"][w])
+            h_idx[w, :n].copy_(out.idx[w, :n], non_blocking=True)
+            h_val[w, :n].copy_(out.val[w, :n], non_blocking=True)
+            moved += n * bpe
+        stream.synchronize()
+        d2h_bytes += moved
+
+    e2e_step(0)
+    d2h_bytes = 0
+    barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for s in range(e2e_steps):
+        e2e_step(1 + s)
+    torch.cuda.synchronize()
+    e2e_ms = (time.perf_counter() - t0) * 1e3
+    e2e_ms = max_over_ranks(e2e_ms) / e2e_steps
+    e2e = {"value": elems_per_step / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+           "h2d_bytes_per_step": int(W * N * 4), "d2h_bytes_per_step": int(d2h_bytes / e2e_steps)}
+
+    # ---- per-stage device times (CUDA events on the launch stream) for the roofline of the top kernel
+    kb.kimad_debug_enable_stage_timing(ctx, True)
+    acc = np.zeros(len(kb.STAGE_NAMES))
+    n_prof = max(3, min(args.steps, 10))
+    for s in range(n_prof):
+        step(args.warmup + s)
+        acc += kb.kimad_debug_stage_times(ctx)
+    kb.kimad_debug_enable_stage_timing(ctx, False)
+    stage_ms = dict(zip(kb.STAGE_NAMES, (acc / n_prof).tolist()))
+    if rank == 0:
+        sampler.stop()
+    if rank != 0:
+        return
+    peak, peak_kind = peaks()
+    top = max(stage_ms, key=stage_ms.get)
+    algo_b = STAGE_ALGO_BYTES.get(top, 4.0) * W * N
+    achieved = algo_b / (stage_ms[top] * 1e-3) / 1e9
+    tpe = NCU_TRAFFIC_BYTES_PER_ELEM.get(top)
+    roofline = {"bound": "hbm", "kernel": top, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+                "traffic": (tpe * W * N if tpe is not None else None),
+                "algorithmic_bytes_per_launch": algo_b, "kernel_ms": stage_ms[top]}
+    compulsory = 8.0 * W * N  # read grad + g once; packed output and sparse g write-back are < 3 % more
+    step_gbs = compulsory / (ms_per_step * 1e-3) / 1e9  # per GPU: every rank moves its own W * N elements
+    res = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": wl.name, "cfg": wl.cfg, "workers_per_gpu": W, "layers": L, "elements_per_worker": N,
+                   "ratios": len(wl.ratio_grid), "D": wl.D, "value_dtype": "bf16" if wl.value_dtype else "f32",
+                   "l2": "inputs_larger_than_l2" if W * N * 4 > 200e6 else "inputs_fit_l2",
+                   "budget_trace": "cycled", "parallelism": f"worker-sharded x{world}"},
+        "e2e": e2e, "gpu_launches": int(launches),
+        "roofline": roofline,
+        "step_roofline": {"bound": "hbm", "compulsory_bytes_per_step": compulsory, "achieved": step_gbs, "peak": peak,
+                          "unit": "GB/s", "frac": step_gbs / peak, "peak_kind": f"of {peak_kind}"},
+        "stage_ms": stage_ms, "step_ms_minmax": [min(per_step), max(per_step)],
+        "clocks": sampler.summary(t_wall0, t_wall1),
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        res["cpu_baseline"] = cpu_baseline(args.config)
+    print(json.dumps(res))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=4, help="workload 1..5 (default 4: GPT-2-small shape, 4 workers)")
+    ap.add_argument("--impl", default="kimad", choices=["kimad", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "kimad" else args.warmup
+    rank = int(os.environ.get("RANK", 0))
+    world = int(os.environ.get("WORLD_SIZE", 1))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+    init_distributed("nccl")
+    run_kimad(args, rank, world)
+
+
+if __name__ == "__main__":
+    main()

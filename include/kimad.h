@@ -1,0 +1,166 @@
+/*
+ * kimad.h -- C ABI of the B200 (sm_100a) worker-side compression pass of Kimad+.
+ *
+ * One call of kimad_step() runs, for W independent data-parallel workers whose gradients
+ * live on ONE GPU, the part of a Kimad round that sits between "gradient computed" and
+ * "message uploaded" (Algorithm 1, worker lines "Select compressor" and "Upload"):
+ *
+ *   (a) d = grad - g                   EF21 difference (Section 3 footnote; Eq. 6)
+ *   (b) err_l(k_j) = ||d_l - TopK_{k_j}(d_l)||^2 for every layer l and every candidate
+ *       ratio j                        (Eq. 4; the "Errors" matrix of Algorithm 3)
+ *   (c) the Kimad+ knapsack dynamic program choosing one candidate per layer so that the
+ *       summed error is minimal and the summed size fits the budget c = B * t
+ *                                      (Eq. 2, Eq. 3, Section 3.2, Algorithm 3)
+ *   (d) TopK selection at the chosen k_l  (Section 2.2: the K entries largest in magnitude)
+ *   (e) the sparse (index, value) message C(d)  (Algorithm 1, upload line)
+ *   (f) g <- g + C(d)                  EF21 estimator update (Algorithm 1 aggregate line; Eq. 6)
+ *
+ * Conventions
+ *   - L layers of sizes n_l, concatenated in list order into one flat vector of N elements.
+ *     Worker w's vector starts at element w * worker_stride of `grads` and of `state`.
+ *   - "device" pointers are CUDA device memory of the current device; "host" pointers are
+ *     ordinary host memory.  The library never allocates or frees device memory: scratch is
+ *     the caller's (kimad_set_workspace).  All kernels go to the caller's stream.
+ *   - TopK order inside a layer: larger |d| first (compared on the 31 magnitude bits, so +0
+ *     and -0 tie), then lower index.  Inputs must be finite.
+ *   - Size of a layer compressed at k: k * (4 + vb) bytes (u32 index + value of vb = 4 or 2
+ *     bytes).  Budget c = floor(bandwidth * t_target) bytes.  Budget axis of the DP: D cells
+ *     of c / D bytes; a candidate occupies ceil(bytes * D / c) cells.
+ *   - Return values: 0 = ok; > 0 = soft status (the step ran); < 0 = error.
+ */
+#ifndef KIMAD_H
+#define KIMAD_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define KIMAD_OK 0
+#define KIMAD_STATUS_INFEASIBLE 1 /* not even the smallest candidates fit: every layer took candidate 0 */
+#define KIMAD_STATUS_PLATEAU 2    /* budget covers the largest candidate of every layer: all taken      */
+#define KIMAD_ERR_INVALID_ARG (-1)
+#define KIMAD_ERR_WORKSPACE (-2) /* workspace missing, too small or misaligned                        */
+#define KIMAD_ERR_CAPACITY (-3)  /* a worker selected more entries than max_packed_elems             */
+#define KIMAD_ERR_NONFINITE (-4) /* Inf/NaN met in grad - g (only reported when check_finite != 0)   */
+#define KIMAD_ERR_TIMEOUT (-5)   /* reserved: no kernel of this library waits on another             */
+#define KIMAD_ERR_CUDA (-6)      /* a CUDA runtime call failed                                       */
+#define KIMAD_ERR_NOMEM (-7)     /* host allocation failed                                           */
+
+#define KIMAD_MAX_RATIOS 127 /* candidates per layer */
+#define KIMAD_MAX_D 16383    /* budget cells */
+
+typedef struct kimad_ctx kimad_ctx;
+
+typedef struct {
+    uint32_t D;                 /* budget cells of the DP; 0 -> 1000 (Section 4.3: factor 1000); needs D >= L */
+    uint32_t value_dtype;       /* 0: packed values are f32; 1: bf16, round-to-nearest-even          */
+    uint32_t check_finite;      /* != 0: a non-finite d makes that worker's step fail with NONFINITE */
+    uint32_t infeasible_policy; /* 0: take candidate 0 everywhere and report KIMAD_STATUS_INFEASIBLE */
+    uint64_t max_packed_elems;  /* capacity (entries) of each worker's idx/val buffer; 0 -> N        */
+    uint64_t worker_stride;     /* elements between consecutive workers in grads/state; 0 -> N       */
+} kimad_options;
+
+/* Per-worker result record, written by the device. */
+typedef struct {
+    uint64_t budget_bytes; /* c                                                          */
+    uint64_t used_bytes;   /* sum_l k_l * (4 + vb); <= c unless status is INFEASIBLE     */
+    uint64_t n_selected;   /* sum_l k_l                                                  */
+    float total_err;       /* err_1(k_1) + ... + err_L(k_L), added left to right in f32  */
+    int32_t status;        /* 0, a KIMAD_STATUS_* or a KIMAD_ERR_* of this worker        */
+} kimad_stats;
+
+/* Output buffers of one step, all DEVICE memory owned by the caller.
+ *   idx   u32 [W][max_packed_elems]  layer-local indices; layer l of worker w occupies
+ *                                    [offs[w][l], offs[w][l+1]), ascending index inside a layer
+ *   val   f32 or bf16 [W][max_packed_elems]  the kept d values, same positions as idx
+ *   offs  u64 [W][L+1]               running sum of k_l
+ *   k     u32 [W][L]                 chosen k per layer
+ *   j     u32 [W][L]                 chosen candidate (index into the ratio grid) per layer
+ *   stats [W]                                                                                  */
+typedef struct {
+    uint32_t* idx;
+    void* val;
+    uint64_t* offs;
+    uint32_t* k;
+    uint32_t* j;
+    kimad_stats* stats;
+} kimad_packed;
+
+/* Problem statement of Section 3.2: the layers, the workers and the discrete ratio set
+ * {c^1..c^K}.  layer_sizes: host, [n_layers], each in [1, 2^32).  ratio_grid: host,
+ * [n_ratios], strictly ascending in (0, 1]; candidate k_{l,j} = min(n_l, max(1, ceil(r_j n_l))).
+ * opt may be NULL (all defaults).  Host-only: touches no GPU.  *out is owned by the caller
+ * until kimad_destroy.  Errors: INVALID_ARG, NOMEM. */
+int kimad_create(kimad_ctx** out, const uint64_t* layer_sizes, uint32_t n_layers, uint32_t n_workers,
+                 const double* ratio_grid, uint32_t n_ratios, const kimad_options* opt);
+void kimad_destroy(kimad_ctx* ctx);
+
+/* Scratch the kernels need (difference vector, histograms, DP back-pointers, tile counts). */
+size_t kimad_workspace_bytes(const kimad_ctx* ctx);
+/* dev_ptr: device, 256-byte aligned, at least kimad_workspace_bytes(); stays owned by the
+ * caller and must outlive the context's steps.  Uploads the static tables and zeroes the
+ * histograms with synchronous copies on the current device.  Errors: WORKSPACE, CUDA. */
+int kimad_set_workspace(kimad_ctx* ctx, void* dev_ptr, size_t bytes);
+
+/* One compression pass (a)-(f) for all W workers, asynchronous on cuda_stream (a cudaStream_t,
+ * NULL = default stream).
+ *   grads_dev  device, f32 [W][worker_stride], read only
+ *   state_dev  device, f32 [W][worker_stride], the EF21 estimators g; updated in place
+ *   bandwidth_bytes_per_s  host, [W]: monitored bandwidth B_m^k of each worker (Section 2.4)
+ *   t_target_s one-direction communication time; budget c_w = floor(B_w * t) bytes.  A caller
+ *              following Eq. 2 passes (t - T_comp) / 2; a fixed byte budget is (B = bytes, t = 1)
+ *   out        host struct of device pointers (see kimad_packed)
+ * Returns 0 or a CUDA/argument error; per-worker outcomes land in out->stats[w].status. */
+int kimad_step(kimad_ctx* ctx, const float* grads_dev, float* state_dev, const double* bandwidth_bytes_per_s,
+               double t_target_s, const kimad_packed* out, void* cuda_stream);
+
+/* Copies the last step's chosen k to host_k (host, u32 [W][L]; may be NULL) after synchronising
+ * cuda_stream.  Returns the most severe per-worker status of that step: the lowest negative
+ * error if any worker failed, else the largest soft status, else 0. */
+int kimad_get_k(kimad_ctx* ctx, uint32_t* host_k, void* cuda_stream);
+
+/* Static tables (host-only calls).  host_k_table: u64 [L][K] candidates k_{l,j}. */
+int kimad_get_k_table(const kimad_ctx* ctx, uint64_t* host_k_table);
+/* Budget arithmetic of one worker exactly as the device applies it: c = floor(B * t); cells
+ * (u64 [L][K], may be NULL) = ceil(k_{l,j} (4+vb) D / c).  Returns 0, KIMAD_STATUS_PLATEAU
+ * (c covers every layer's largest candidate; cells not written) or KIMAD_STATUS_INFEASIBLE
+ * (c == 0; cells not written). */
+int kimad_plan_budget(const kimad_ctx* ctx, double bandwidth_bytes_per_s, double t_target_s,
+                      uint64_t* budget_bytes, uint64_t* cells);
+
+/* Stage isolation for tests.  All synchronise the device.
+ * kimad_debug_get_curve: results of stage (b) of the last step; each pointer is host
+ *   [W][L][K] or NULL: err (f32), tau (31-bit magnitude key of the k-th largest entry),
+ *   keep_eq (how many entries equal to tau are kept). */
+int kimad_debug_get_curve(kimad_ctx* ctx, float* host_err, uint32_t* host_tau, uint32_t* host_keep_eq);
+/* kimad_step whose DP (c) consumes err_dev (device, f32 [W][L][K]) instead of the curves it
+ * computed; stages (a), (b), (d)-(f) unchanged. */
+int kimad_debug_step_with_err(kimad_ctx* ctx, const float* grads_dev, float* state_dev,
+                              const double* bandwidth_bytes_per_s, double t_target_s, const kimad_packed* out,
+                              void* cuda_stream, const float* err_dev);
+/* kimad_step without stage (c): candidate j_dev[w][l] (device, u32 [W][L]) is taken as given. */
+int kimad_debug_step_with_j(kimad_ctx* ctx, const float* grads_dev, float* state_dev,
+                            const double* bandwidth_bytes_per_s, double t_target_s, const kimad_packed* out,
+                            void* cuda_stream, const uint32_t* j_dev);
+
+/* Per-stage device timing for benchmarks.  enable != 0: every following step records CUDA events
+ * around its stages on the step's stream (first use creates the events).  kimad_debug_stage_times
+ * synchronises the device and writes the last step's stage durations in milliseconds to host_ms
+ * (host, f32 [KIMAD_N_STAGES]), stage order: diff+hist1, resolve1, hist2, resolve2, hist3, resolve3,
+ * dp, select_count, select_scan, select_write. */
+#define KIMAD_N_STAGES 10
+int kimad_debug_enable_stage_timing(kimad_ctx* ctx, int enable);
+int kimad_debug_stage_times(kimad_ctx* ctx, float* host_ms);
+
+/* Kernels launched by this context so far (for launch accounting in benchmarks). */
+uint64_t kimad_launch_count(const kimad_ctx* ctx);
+/* Static description of a code returned by this library. */
+const char* kimad_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KIMAD_H */

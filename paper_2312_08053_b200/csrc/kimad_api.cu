@@ -1,0 +1,365 @@
+// Host side of the C ABI declared in include/kimad.h: context, static planner (candidate table,
+// chunk table, workspace layout) and the per-step launch sequence.  No device memory is allocated
+// here; the caller's workspace is carved into the regions listed in `Layout`.
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "kimad_kernels.cuh"
+
+using namespace kimad;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+struct Layout {
+    size_t dbuf, chunks, layers, ktab, h1_cnt, h1_ss, h23_cnt, h23_ss, cands, slots, err, tau, keep_eq, sel, chunk_cnt,
+        flags, pd, total;
+};
+
+} // namespace
+
+struct kimad_ctx {
+    uint32_t L = 0, W = 0, K = 0, D = 1000;
+    uint32_t value_dtype = 0, check_finite = 0;
+    uint64_t N = 0, stride = 0, dstride = 0, cap = 0, full_bytes = 0;
+    uint32_t bpe = 8;
+    std::vector<uint64_t> layer_sizes, ktab;
+    std::vector<double> grid;
+    std::vector<Chunk> chunks;
+    std::vector<LayerDesc> layers;
+    Layout lay{};
+    unsigned char* ws = nullptr;
+    bool pd_in_smem = false;
+    size_t dp_smem = 0;
+    uint64_t launches = 0;
+    kimad_packed last_out{};
+    bool have_last = false;
+    bool timing = false;
+    cudaEvent_t ev[KIMAD_N_STAGES + 1] = {};
+    bool have_ev = false;
+    template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
+};
+
+namespace {
+
+void plan_layout(kimad_ctx* c) {
+    Layout& y = c->lay;
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes); return at; };
+    const size_t WL = (size_t)c->W * c->L, WLK = WL * c->K;
+    y.dbuf = take((size_t)c->W * c->dstride * sizeof(float));
+    y.chunks = take(c->chunks.size() * sizeof(Chunk));
+    y.layers = take(c->layers.size() * sizeof(LayerDesc));
+    y.ktab = take(c->ktab.size() * sizeof(uint64_t));
+    y.h1_cnt = take(WL * kL1Bins * sizeof(uint32_t));
+    y.h1_ss = take(WL * kL1Bins * sizeof(double));
+    y.h23_cnt = take(WLK * kL23Bins * sizeof(uint32_t));
+    y.h23_ss = take(WLK * kL23Bins * sizeof(double));
+    y.cands = take(WLK * sizeof(Cand));
+    y.slots = take(WL * sizeof(SlotTab));
+    y.err = take(WLK * sizeof(float));
+    y.tau = take(WLK * sizeof(uint32_t));
+    y.keep_eq = take(WLK * sizeof(uint32_t));
+    y.sel = take(WL * sizeof(Sel));
+    y.chunk_cnt = take((size_t)c->W * c->chunks.size() * sizeof(uint2));
+    y.flags = take((size_t)c->W * sizeof(uint32_t));
+    y.pd = take(c->pd_in_smem ? 0 : (size_t)c->W * c->L * (c->D + 1));
+    y.total = o;
+}
+
+#define CUDA_TRY(x)                                  \
+    do {                                             \
+        if ((x) != cudaSuccess) return KIMAD_ERR_CUDA; \
+    } while (0)
+
+enum StepMode { kNormal = 0, kInjectErr = 1, kGivenJ = 2 };
+
+int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, double t, const kimad_packed* out,
+             void* stream_v, StepMode mode, const float* err_dev, const uint32_t* j_dev) {
+    if (!c || !grads || !state || !bw || !out || !out->idx || !out->val || !out->offs || !out->k || !out->j ||
+        !out->stats)
+        return KIMAD_ERR_INVALID_ARG;
+    if (!c->ws) return KIMAD_ERR_WORKSPACE;
+    if (!(t >= 0.0)) return KIMAD_ERR_INVALID_ARG;
+    if (mode == kInjectErr && !err_dev) return KIMAD_ERR_INVALID_ARG;
+    if (mode == kGivenJ && !j_dev) return KIMAD_ERR_INVALID_ARG;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream_v);
+    const uint32_t L = c->L, W = c->W, K = c->K;
+    const uint32_t nch = (uint32_t)c->chunks.size();
+    const bool vec = ((uintptr_t)grads % 16 == 0) && ((uintptr_t)state % 16 == 0) && (c->stride % 4 == 0);
+
+    float* dbuf = c->at<float>(c->lay.dbuf);
+    const Chunk* chunks = c->at<Chunk>(c->lay.chunks);
+    const LayerDesc* layers = c->at<LayerDesc>(c->lay.layers);
+    const uint64_t* ktab = c->at<uint64_t>(c->lay.ktab);
+    uint32_t* h1c = c->at<uint32_t>(c->lay.h1_cnt);
+    unsigned long long* h1s = c->at<unsigned long long>(c->lay.h1_ss);
+    uint32_t* h23c = c->at<uint32_t>(c->lay.h23_cnt);
+    unsigned long long* h23s = c->at<unsigned long long>(c->lay.h23_ss);
+    Cand* cands = c->at<Cand>(c->lay.cands);
+    SlotTab* slots = c->at<SlotTab>(c->lay.slots);
+    float* err = c->at<float>(c->lay.err);
+    uint32_t* tau = c->at<uint32_t>(c->lay.tau);
+    uint32_t* keq = c->at<uint32_t>(c->lay.keep_eq);
+    Sel* sel = c->at<Sel>(c->lay.sel);
+    uint2* ccnt = c->at<uint2>(c->lay.chunk_cnt);
+    uint32_t* flags = c->at<uint32_t>(c->lay.flags);
+    uint8_t* pd = c->at<uint8_t>(c->lay.pd);
+
+    const dim3 gch(nch, W), glw(L, W), blk(kThreads);
+    int stage = 0;
+    auto mark = [&]() { if (c->timing) cudaEventRecord(c->ev[stage++], s); };
+    mark();
+
+    // (a) + first digit
+    if (vec)
+        k_diff_hist1<true><<<gch, blk, 0, s>>>(grads, state, dbuf, chunks, c->stride, c->dstride, L, h1c, h1s, flags);
+    else
+        k_diff_hist1<false><<<gch, blk, 0, s>>>(grads, state, dbuf, chunks, c->stride, c->dstride, L, h1c, h1s, flags);
+    mark();
+    // (b) remaining digits
+    k_resolve1<<<glw, blk, 0, s>>>(h1c, h1s, ktab, L, K, cands, slots);
+    mark();
+    k_hist23<2, true><<<gch, blk, 0, s>>>(dbuf, chunks, c->dstride, L, K, slots, h23c, h23s);
+    mark();
+    k_resolve23<2><<<glw, blk, 0, s>>>(h23c, h23s, L, K, cands, slots, err, tau, keq);
+    mark();
+    k_hist23<3, true><<<gch, blk, 0, s>>>(dbuf, chunks, c->dstride, L, K, slots, h23c, h23s);
+    mark();
+    k_resolve23<3><<<glw, blk, 0, s>>>(h23c, h23s, L, K, cands, slots, err, tau, keq);
+    mark();
+    c->launches += 6;
+    // (c)
+    for (uint32_t w0 = 0; w0 < W; w0 += kDpWorkersPerLaunch) {
+        DpBudgets b{};
+        const uint32_t nw = std::min<uint32_t>(kDpWorkersPerLaunch, W - w0);
+        for (uint32_t i = 0; i < nw; ++i) {
+            double cb = std::floor(bw[w0 + i] * t);
+            b.c[i] = !(cb > 0.0) ? 0ull : (cb >= 18446744073709551615.0 ? ~0ull : (uint64_t)cb);
+        }
+        k_dp<<<nw, kDpThreads, c->dp_smem, s>>>(b, w0, W, L, K, c->D, c->bpe, c->full_bytes, c->cap, c->check_finite,
+                                                mode == kGivenJ ? 1 : 0, ktab, mode == kInjectErr ? err_dev : err, tau,
+                                                keq, j_dev, flags, pd, c->pd_in_smem ? 1 : 0, sel, out->k, out->j,
+                                                out->offs, out->stats);
+        c->launches += 1;
+    }
+    mark();
+    // (d), (e), (f)
+    k_select_count<true><<<gch, blk, 0, s>>>(dbuf, chunks, nch, c->dstride, L, sel, layers, ccnt);
+    mark();
+    k_select_scan<<<glw, blk, 0, s>>>(layers, nch, ccnt);
+    mark();
+    if (c->value_dtype == 1)
+        k_select_write<true><<<gch, blk, 0, s>>>(dbuf, state, chunks, nch, c->dstride, c->stride, L, sel, layers, ccnt,
+                                                 c->cap, out->idx, out->val);
+    else
+        k_select_write<false><<<gch, blk, 0, s>>>(dbuf, state, chunks, nch, c->dstride, c->stride, L, sel, layers, ccnt,
+                                                  c->cap, out->idx, out->val);
+    mark();
+    c->launches += 3;
+    CUDA_TRY(cudaGetLastError());
+    c->last_out = *out;
+    c->have_last = true;
+    return KIMAD_OK;
+}
+
+} // namespace
+
+extern "C" {
+
+int kimad_create(kimad_ctx** out, const uint64_t* layer_sizes, uint32_t n_layers, uint32_t n_workers,
+                 const double* ratio_grid, uint32_t n_ratios, const kimad_options* opt) {
+    if (!out) return KIMAD_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!layer_sizes || !ratio_grid || n_layers == 0 || n_workers == 0 || n_ratios == 0 ||
+        n_ratios > KIMAD_MAX_RATIOS)
+        return KIMAD_ERR_INVALID_ARG;
+    kimad_options o{};
+    if (opt) o = *opt;
+    if (o.D == 0) o.D = 1000;
+    if (o.D > KIMAD_MAX_D || o.D < n_layers || o.value_dtype > 1 || o.infeasible_policy != 0)
+        return KIMAD_ERR_INVALID_ARG;
+    for (uint32_t j = 0; j < n_ratios; ++j) {
+        if (!(ratio_grid[j] > 0.0) || ratio_grid[j] > 1.0) return KIMAD_ERR_INVALID_ARG;
+        if (j && !(ratio_grid[j] > ratio_grid[j - 1])) return KIMAD_ERR_INVALID_ARG;
+    }
+    kimad_ctx* c = new (std::nothrow) kimad_ctx();
+    if (!c) return KIMAD_ERR_NOMEM;
+    try {
+        c->L = n_layers; c->W = n_workers; c->K = n_ratios; c->D = o.D;
+        c->value_dtype = o.value_dtype; c->check_finite = o.check_finite;
+        c->bpe = o.value_dtype == 0 ? 8 : 6;
+        c->layer_sizes.assign(layer_sizes, layer_sizes + n_layers);
+        c->grid.assign(ratio_grid, ratio_grid + n_ratios);
+        c->ktab.resize((size_t)n_layers * n_ratios);
+        uint64_t N = 0;
+        for (uint32_t l = 0; l < n_layers; ++l) {
+            const uint64_t n = layer_sizes[l];
+            if (n == 0 || n > 0xffffffffull) { delete c; return KIMAD_ERR_INVALID_ARG; }
+            for (uint32_t j = 0; j < n_ratios; ++j) { // candidate k: ratio of the layer, at least one entry
+                uint64_t k = (uint64_t)std::ceil(ratio_grid[j] * (double)n);
+                if (k < 1) k = 1;
+                if (k > n) k = n;
+                c->ktab[(size_t)l * n_ratios + j] = k;
+            }
+            c->full_bytes += c->ktab[(size_t)l * n_ratios + n_ratios - 1] * c->bpe;
+            // chunk table: aligned windows of the flat vector intersected with this layer
+            LayerDesc ld{N, n, (uint32_t)c->chunks.size(), 0};
+            for (uint64_t p = N; p < N + n;) {
+                const uint64_t e = std::min(N + n, (p / kChunkElems + 1) * kChunkElems);
+                c->chunks.push_back(Chunk{l, 0, p, e});
+                p = e;
+            }
+            ld.n_chunks = (uint32_t)c->chunks.size() - ld.first_chunk;
+            c->layers.push_back(ld);
+            N += n;
+        }
+        c->N = N;
+        c->stride = o.worker_stride ? o.worker_stride : N;
+        c->cap = o.max_packed_elems ? o.max_packed_elems : N;
+        if (c->stride < N || c->chunks.size() > 0x7fffffffull) { delete c; return KIMAD_ERR_INVALID_ARG; }
+        c->dstride = (N + 3) / 4 * 4;
+        const size_t dp_rows = ((size_t)2 * (c->D + 1) + 2 * c->K + c->L) * 4;
+        const size_t pd_bytes = (size_t)c->L * (c->D + 1);
+        c->pd_in_smem = dp_rows + pd_bytes <= 225 * 1024;
+        c->dp_smem = dp_rows + (c->pd_in_smem ? pd_bytes : 0);
+        if (dp_rows > 200 * 1024) { delete c; return KIMAD_ERR_INVALID_ARG; }
+        plan_layout(c);
+    } catch (const std::bad_alloc&) {
+        delete c;
+        return KIMAD_ERR_NOMEM;
+    }
+    *out = c;
+    return KIMAD_OK;
+}
+
+void kimad_destroy(kimad_ctx* ctx) {
+    if (ctx && ctx->have_ev)
+        for (cudaEvent_t e : ctx->ev) cudaEventDestroy(e);
+    delete ctx;
+}
+
+int kimad_debug_enable_stage_timing(kimad_ctx* c, int enable) {
+    if (!c) return KIMAD_ERR_INVALID_ARG;
+    if (enable && !c->have_ev) {
+        for (cudaEvent_t& e : c->ev) CUDA_TRY(cudaEventCreate(&e));
+        c->have_ev = true;
+    }
+    c->timing = enable != 0;
+    return KIMAD_OK;
+}
+
+int kimad_debug_stage_times(kimad_ctx* c, float* host_ms) {
+    if (!c || !host_ms || !c->have_ev || !c->have_last) return KIMAD_ERR_INVALID_ARG;
+    CUDA_TRY(cudaDeviceSynchronize());
+    for (int i = 0; i < KIMAD_N_STAGES; ++i) CUDA_TRY(cudaEventElapsedTime(&host_ms[i], c->ev[i], c->ev[i + 1]));
+    return KIMAD_OK;
+}
+
+size_t kimad_workspace_bytes(const kimad_ctx* ctx) { return ctx ? ctx->lay.total : 0; }
+
+int kimad_set_workspace(kimad_ctx* c, void* dev_ptr, size_t bytes) {
+    if (!c) return KIMAD_ERR_INVALID_ARG;
+    if (!dev_ptr || bytes < c->lay.total || (uintptr_t)dev_ptr % kAlign) return KIMAD_ERR_WORKSPACE;
+    c->ws = static_cast<unsigned char*>(dev_ptr);
+    const Layout& y = c->lay;
+    CUDA_TRY(cudaMemcpy(c->ws + y.chunks, c->chunks.data(), c->chunks.size() * sizeof(Chunk), cudaMemcpyHostToDevice));
+    CUDA_TRY(cudaMemcpy(c->ws + y.layers, c->layers.data(), c->layers.size() * sizeof(LayerDesc), cudaMemcpyHostToDevice));
+    CUDA_TRY(cudaMemcpy(c->ws + y.ktab, c->ktab.data(), c->ktab.size() * sizeof(uint64_t), cudaMemcpyHostToDevice));
+    // everything after the static tables starts at zero: the histograms are kept clean by the kernels
+    CUDA_TRY(cudaMemset(c->ws + y.h1_cnt, 0, y.total - y.h1_cnt));
+    CUDA_TRY(cudaFuncSetAttribute(k_dp, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->dp_smem));
+    CUDA_TRY(cudaDeviceSynchronize());
+    return KIMAD_OK;
+}
+
+int kimad_step(kimad_ctx* ctx, const float* grads_dev, float* state_dev, const double* bandwidth_bytes_per_s,
+               double t_target_s, const kimad_packed* out, void* cuda_stream) {
+    return run_step(ctx, grads_dev, state_dev, bandwidth_bytes_per_s, t_target_s, out, cuda_stream, kNormal, nullptr,
+                    nullptr);
+}
+
+int kimad_debug_step_with_err(kimad_ctx* ctx, const float* grads_dev, float* state_dev,
+                              const double* bandwidth_bytes_per_s, double t_target_s, const kimad_packed* out,
+                              void* cuda_stream, const float* err_dev) {
+    return run_step(ctx, grads_dev, state_dev, bandwidth_bytes_per_s, t_target_s, out, cuda_stream, kInjectErr, err_dev,
+                    nullptr);
+}
+
+int kimad_debug_step_with_j(kimad_ctx* ctx, const float* grads_dev, float* state_dev,
+                            const double* bandwidth_bytes_per_s, double t_target_s, const kimad_packed* out,
+                            void* cuda_stream, const uint32_t* j_dev) {
+    return run_step(ctx, grads_dev, state_dev, bandwidth_bytes_per_s, t_target_s, out, cuda_stream, kGivenJ, nullptr,
+                    j_dev);
+}
+
+int kimad_get_k(kimad_ctx* c, uint32_t* host_k, void* cuda_stream) {
+    if (!c || !c->have_last) return KIMAD_ERR_INVALID_ARG;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+    std::vector<kimad_stats> st(c->W);
+    if (host_k)
+        CUDA_TRY(cudaMemcpyAsync(host_k, c->last_out.k, (size_t)c->W * c->L * sizeof(uint32_t), cudaMemcpyDeviceToHost, s));
+    CUDA_TRY(cudaMemcpyAsync(st.data(), c->last_out.stats, c->W * sizeof(kimad_stats), cudaMemcpyDeviceToHost, s));
+    CUDA_TRY(cudaStreamSynchronize(s));
+    int worst_err = 0, worst_soft = 0;
+    for (const kimad_stats& x : st) {
+        if (x.status < worst_err) worst_err = x.status;
+        if (x.status > worst_soft) worst_soft = x.status;
+    }
+    return worst_err < 0 ? worst_err : worst_soft;
+}
+
+int kimad_get_k_table(const kimad_ctx* c, uint64_t* host_k_table) {
+    if (!c || !host_k_table) return KIMAD_ERR_INVALID_ARG;
+    std::memcpy(host_k_table, c->ktab.data(), c->ktab.size() * sizeof(uint64_t));
+    return KIMAD_OK;
+}
+
+int kimad_plan_budget(const kimad_ctx* c, double bandwidth_bytes_per_s, double t_target_s, uint64_t* budget_bytes,
+                      uint64_t* cells) {
+    if (!c) return KIMAD_ERR_INVALID_ARG;
+    const double cb = std::floor(bandwidth_bytes_per_s * t_target_s);
+    const uint64_t cc = !(cb > 0.0) ? 0ull : (cb >= 18446744073709551615.0 ? ~0ull : (uint64_t)cb);
+    if (budget_bytes) *budget_bytes = cc;
+    if (cc >= c->full_bytes) return KIMAD_STATUS_PLATEAU;
+    if (cc == 0) return KIMAD_STATUS_INFEASIBLE;
+    if (cells)
+        for (size_t i = 0; i < c->ktab.size(); ++i) cells[i] = budget_cells(c->ktab[i] * c->bpe, c->D, cc);
+    return KIMAD_OK;
+}
+
+int kimad_debug_get_curve(kimad_ctx* c, float* host_err, uint32_t* host_tau, uint32_t* host_keep_eq) {
+    if (!c) return KIMAD_ERR_INVALID_ARG;
+    if (!c->ws) return KIMAD_ERR_WORKSPACE;
+    const size_t n = (size_t)c->W * c->L * c->K;
+    CUDA_TRY(cudaDeviceSynchronize());
+    if (host_err) CUDA_TRY(cudaMemcpy(host_err, c->ws + c->lay.err, n * 4, cudaMemcpyDeviceToHost));
+    if (host_tau) CUDA_TRY(cudaMemcpy(host_tau, c->ws + c->lay.tau, n * 4, cudaMemcpyDeviceToHost));
+    if (host_keep_eq) CUDA_TRY(cudaMemcpy(host_keep_eq, c->ws + c->lay.keep_eq, n * 4, cudaMemcpyDeviceToHost));
+    return KIMAD_OK;
+}
+
+uint64_t kimad_launch_count(const kimad_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+const char* kimad_strerror(int code) {
+    switch (code) {
+        case KIMAD_OK: return "ok";
+        case KIMAD_STATUS_INFEASIBLE: return "budget below the smallest candidates: candidate 0 taken everywhere";
+        case KIMAD_STATUS_PLATEAU: return "budget covers the largest candidate of every layer";
+        case KIMAD_ERR_INVALID_ARG: return "invalid argument";
+        case KIMAD_ERR_WORKSPACE: return "workspace missing, too small or misaligned";
+        case KIMAD_ERR_CAPACITY: return "selected entries exceed max_packed_elems";
+        case KIMAD_ERR_NONFINITE: return "non-finite value in grad - state";
+        case KIMAD_ERR_TIMEOUT: return "device wait timed out";
+        case KIMAD_ERR_CUDA: return "CUDA runtime error";
+        case KIMAD_ERR_NOMEM: return "host allocation failed";
+        default: return "unknown code";
+    }
+}
+
+} // extern "C"

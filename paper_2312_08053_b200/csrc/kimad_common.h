@@ -1,0 +1,61 @@
+// Plain structs and integer helpers shared by the host planner and the kernels of the CUDA library.
+#pragma once
+#include <stdint.h>
+
+#include "kimad.h"
+
+#if defined(__CUDACC__)
+#define KIMAD_HD __host__ __device__ __forceinline__
+#else
+#define KIMAD_HD inline
+#endif
+
+namespace kimad {
+
+// A chunk is the part of one layer that falls inside one aligned window of kChunkElems elements of
+// the flat per-worker vector.  One CTA streams one chunk.
+constexpr uint64_t kChunkElems = 32768;
+constexpr int kDpWorkersPerLaunch = 32;
+
+struct Chunk {
+    uint32_t layer;
+    uint32_t _pad;
+    uint64_t begin; // flat element index inside the worker's vector
+    uint64_t end;
+};
+
+struct LayerDesc {
+    uint64_t begin;
+    uint64_t n;
+    uint32_t first_chunk;
+    uint32_t n_chunks;
+};
+
+// Radix-select state of one (worker, layer, candidate) between digit passes.
+struct Cand {
+    double err_low;  // sum of squares of everything known to lie below the current bin
+    uint32_t rank;   // 1-based rank of the wanted key inside the current bin, counted from the top
+    uint32_t gt;     // keys known to be larger than everything in the current bin
+    uint32_t slot;   // which histogram slot of this (worker, layer) refines the current bin
+    uint32_t prefix; // the bin: top 11 / 21 / 31 bits of the key after digit 1 / 2 / 3
+};
+
+struct SlotTab {
+    uint32_t n;
+    uint32_t prefix[KIMAD_MAX_RATIOS];
+};
+
+// What the select kernels need to know about one (worker, layer) after the DP.
+struct Sel {
+    uint32_t tau;     // threshold key
+    uint32_t keep_eq; // entries equal to tau that are kept (lowest indices first)
+    uint32_t k;       // 0: nothing to pack for this layer (the worker failed)
+    uint32_t _pad;
+    uint64_t base;    // first output position of the layer in the worker's packed buffers
+};
+
+// Budget cells a candidate of `bytes` occupies when c bytes are split into D cells (rounded up, so
+// the byte constraint of Eq. 3 can never be exceeded).  c > 0.
+KIMAD_HD uint64_t budget_cells(uint64_t bytes, uint32_t D, uint64_t c) { return (bytes * (uint64_t)D + c - 1) / c; }
+
+} // namespace kimad

@@ -1,0 +1,688 @@
+// Device code of the Kimad+ compression pass for sm_100a.
+//
+// Stage map (letters as in include/kimad.h):
+//   k_diff_hist1          (a) d = grad - g, written to scratch, fused with the first digit
+//                             (11 bits) of a 3-digit radix histogram of the magnitude key
+//   k_resolve1/2/3        (b) locate, for every candidate k_j of every layer, the bin that holds
+//   k_hist2, k_hist3          the k_j-th largest key, digit by digit (11 + 10 + 10 bits), while
+//                             summing the squares of everything below it -> err, tau, keep_eq
+//   k_dp                  (c) Algorithm 3 on the budget axis, one CTA per worker
+//   k_select_count/scan   (d) per-chunk counts of entries above / equal to the chosen threshold
+//   k_select_write        (e)+(f) ordered compaction into (idx, val) and g += C(d)
+//
+// Everything is HBM- or latency-bound; there is no dense contraction, so no tensor-core path.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "kimad_common.h"
+
+namespace kimad {
+
+constexpr int kThreads = 256;
+constexpr int kL1Bins = 2048;  // 8 exponent bits + 3 mantissa bits
+constexpr int kL23Bins = 1024; // 10 bits each
+
+__device__ __forceinline__ uint32_t key_of(float d) { return __float_as_uint(d) & 0x7fffffffu; }
+
+// ------------------------------------------------------------------------------------------------
+// block-wide exclusive scans (256 threads), result valid in every thread; `total` optional
+// ------------------------------------------------------------------------------------------------
+template <typename T>
+__device__ __forceinline__ T block_excl_scan(T v, T* s_warp /* [8] */, T* total) {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    T x = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        T y = __shfl_up_sync(0xffffffffu, x, o);
+        if (lane >= o) x += y;
+    }
+    __syncthreads(); // s_warp may still be read from a previous call
+    if (lane == 31) s_warp[wid] = x;
+    __syncthreads();
+    T base = 0, tot = 0;
+#pragma unroll
+    for (int i = 0; i < kThreads / 32; ++i) {
+        T t = s_warp[i];
+        if (i < wid) base += t;
+        tot += t;
+    }
+    if (total) *total = tot;
+    return base + x - v;
+}
+
+// ------------------------------------------------------------------------------------------------
+// (a) difference + level-1 histogram
+// ------------------------------------------------------------------------------------------------
+// Squares are accumulated as exact integers.  Every histogram bin holds keys of one exponent e, so
+// value^2 = M^2 * 4^(max(e,1)-150) with M the 24-bit significand (no hidden bit for subnormals);
+// bins sum (M^2 >> 16), a 32-bit quantity (truncation <= 2^-30 relative).  Integer adds commute, so
+// the sums -- and with them the error curve -- do not depend on the order the atomics land in.
+__device__ __forceinline__ uint64_t sq_fixed(uint32_t key) {
+    const uint32_t e = key >> 23, mant = key & 0x7fffffu;
+    const uint32_t M = e ? (mant | 0x800000u) : mant;
+    return ((uint64_t)M * (uint64_t)M) >> 16;
+}
+// scale that turns a bin's integer sum back into a sum of squared values; e = exponent field of the bin
+__device__ __forceinline__ double sq_scale(uint32_t e) { return ldexp(1.0, 2 * ((int)(e ? e : 1u) - 150) + 16); }
+
+// One shared-memory word per level-1 bin: count in the top 17 bits, sum of sq_fixed in the low 47
+// (a chunk has at most 2^15 elements, each adding < 2^32).
+constexpr int kL1CountShift = 47;
+
+struct L1Acc {
+    unsigned long long* acc;
+    uint32_t nonfinite;
+    __device__ __forceinline__ void add(float dv) {
+        const uint32_t key = key_of(dv);
+        atomicAdd(&acc[key >> 20], (1ull << kL1CountShift) | sq_fixed(key));
+        nonfinite |= ((key >> 23) == 255u);
+    }
+};
+
+template <bool VEC>
+__global__ void __launch_bounds__(kThreads)
+k_diff_hist1(const float* __restrict__ grads, const float* __restrict__ state, float* __restrict__ dbuf,
+             const Chunk* __restrict__ chunks, uint64_t stride, uint64_t dstride, uint32_t L,
+             uint32_t* __restrict__ g_cnt, unsigned long long* __restrict__ g_ss, uint32_t* __restrict__ flags) {
+    __shared__ unsigned long long s_acc[kL1Bins];
+    const Chunk ch = chunks[blockIdx.x];
+    const uint32_t w = blockIdx.y;
+    for (int b = threadIdx.x; b < kL1Bins; b += kThreads) s_acc[b] = 0ull;
+    __syncthreads();
+    const float* gr = grads + (size_t)w * stride;
+    const float* st = state + (size_t)w * stride;
+    float* dd = dbuf + (size_t)w * dstride;
+    L1Acc acc{s_acc, 0u};
+
+    const uint64_t q0 = ch.begin & ~3ull;
+    constexpr int U = 4;
+    for (uint64_t base = q0; base < ch.end; base += (uint64_t)4 * kThreads * U) {
+        float4 a[U], b[U];
+        bool full[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint64_t q = base + 4ull * (threadIdx.x + (uint64_t)u * kThreads);
+            full[u] = VEC && q >= ch.begin && q + 4 <= ch.end;
+            if (full[u]) {
+                a[u] = __ldcs(reinterpret_cast<const float4*>(gr + q));
+                b[u] = __ldcs(reinterpret_cast<const float4*>(st + q));
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint64_t q = base + 4ull * (threadIdx.x + (uint64_t)u * kThreads);
+            if (full[u]) {
+                float4 r;
+                r.x = __fsub_rn(a[u].x, b[u].x);
+                r.y = __fsub_rn(a[u].y, b[u].y);
+                r.z = __fsub_rn(a[u].z, b[u].z);
+                r.w = __fsub_rn(a[u].w, b[u].w);
+                *reinterpret_cast<float4*>(dd + q) = r;
+                acc.add(r.x); acc.add(r.y); acc.add(r.z); acc.add(r.w);
+            } else if (q < ch.end) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const uint64_t p = q + i;
+                    if (p >= ch.begin && p < ch.end) {
+                        const float r = __fsub_rn(gr[p], st[p]);
+                        dd[p] = r;
+                        acc.add(r);
+                    }
+                }
+            }
+        }
+    }
+    if (acc.nonfinite) atomicOr(&flags[w], 1u);
+    __syncthreads();
+    uint32_t* gc = g_cnt + ((size_t)w * L + ch.layer) * kL1Bins;
+    unsigned long long* gs = g_ss + ((size_t)w * L + ch.layer) * kL1Bins;
+    for (int b = threadIdx.x; b < kL1Bins; b += kThreads) {
+        const unsigned long long v = s_acc[b];
+        if (v) {
+            atomicAdd(&gc[b], (uint32_t)(v >> kL1CountShift));
+            atomicAdd(&gs[b], v & ((1ull << kL1CountShift) - 1));
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// (b) resolve: candidates -> bins.  One CTA per (worker, layer).
+// ------------------------------------------------------------------------------------------------
+// In-place: on return s_incl[p] (p = position counted from the TOP bin, p = NB-1-bin) holds the
+// inclusive count of keys in bins >= that bin; s_below[bin] holds the sum of ss over bins < bin.
+template <int NB>
+__device__ __forceinline__ void scan_bins(uint32_t* s_incl /* in: counts by position */, double* s_below /* in: ss by bin */,
+                                          uint32_t* s_w32, double* s_w64) {
+    constexpr int PER = NB / kThreads;
+    uint32_t loc[PER];
+    uint32_t sum = 0;
+#pragma unroll
+    for (int i = 0; i < PER; ++i) { loc[i] = s_incl[threadIdx.x * PER + i]; sum += loc[i]; }
+    uint32_t ex = block_excl_scan<uint32_t>(sum, s_w32, nullptr);
+#pragma unroll
+    for (int i = 0; i < PER; ++i) { ex += loc[i]; s_incl[threadIdx.x * PER + i] = ex; }
+    if (s_below) {
+        double dl[PER];
+        double ds = 0.0;
+#pragma unroll
+        for (int i = 0; i < PER; ++i) { dl[i] = s_below[threadIdx.x * PER + i]; ds += dl[i]; }
+        double de = block_excl_scan<double>(ds, s_w64, nullptr);
+#pragma unroll
+        for (int i = 0; i < PER; ++i) { s_below[threadIdx.x * PER + i] = de; de += dl[i]; }
+    }
+    __syncthreads();
+}
+
+// first position p (0 = top bin) whose inclusive count reaches `rank` (1-based)
+template <int NB>
+__device__ __forceinline__ int find_pos(const uint32_t* s_incl, uint32_t rank) {
+    int lo = 0, hi = NB - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (s_incl[mid] >= rank) hi = mid; else lo = mid + 1;
+    }
+    return lo;
+}
+
+__global__ void __launch_bounds__(kThreads)
+k_resolve1(uint32_t* __restrict__ g_cnt, unsigned long long* __restrict__ g_ss, const uint64_t* __restrict__ ktab,
+           uint32_t L, uint32_t K, Cand* __restrict__ cands, SlotTab* __restrict__ slots) {
+    __shared__ uint32_t s_incl[kL1Bins];
+    __shared__ double s_below[kL1Bins];
+    __shared__ uint32_t s_w32[8];
+    __shared__ double s_w64[8];
+    const uint32_t l = blockIdx.x, w = blockIdx.y;
+    const size_t wl = (size_t)w * L + l;
+    uint32_t* gc = g_cnt + wl * kL1Bins;
+    unsigned long long* gs = g_ss + wl * kL1Bins;
+    for (int b = threadIdx.x; b < kL1Bins; b += kThreads) {
+        s_incl[kL1Bins - 1 - b] = gc[b];
+        s_below[b] = (double)gs[b] * sq_scale((uint32_t)b >> 3);
+        gc[b] = 0; // leave the histogram clean for the next step
+        gs[b] = 0ull;
+    }
+    __syncthreads();
+    scan_bins<kL1Bins>(s_incl, s_below, s_w32, s_w64);
+    Cand* cd = cands + wl * K;
+    for (uint32_t j = threadIdx.x; j < K; j += kThreads) {
+        const uint32_t k = (uint32_t)ktab[(size_t)l * K + j];
+        const int p = find_pos<kL1Bins>(s_incl, k);
+        const uint32_t above = p ? s_incl[p - 1] : 0u;
+        Cand c;
+        c.prefix = (uint32_t)(kL1Bins - 1 - p);
+        c.rank = k - above;
+        c.gt = above;
+        c.err_low = s_below[kL1Bins - 1 - p];
+        c.slot = 0;
+        cd[j] = c;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) { // distinct prefixes, in candidate order (prefix is non-increasing in j)
+        SlotTab& stab = slots[wl];
+        uint32_t ns = 0;
+        for (uint32_t j = 0; j < K; ++j) {
+            if (ns == 0 || stab.prefix[ns - 1] != cd[j].prefix) stab.prefix[ns++] = cd[j].prefix;
+            cd[j].slot = ns - 1;
+        }
+        stab.n = ns;
+    }
+}
+
+// LEVEL 2: refine inside a level-1 bin; LEVEL 3: inside a (level-1, level-2) bin.
+template <int LEVEL>
+__global__ void __launch_bounds__(kThreads)
+k_resolve23(uint32_t* __restrict__ g_cnt, unsigned long long* __restrict__ g_ss, uint32_t L, uint32_t K,
+            Cand* __restrict__ cands, SlotTab* __restrict__ slots, float* __restrict__ err_out,
+            uint32_t* __restrict__ tau_out, uint32_t* __restrict__ keep_eq_out) {
+    __shared__ uint32_t s_incl[kL23Bins];
+    __shared__ double s_below[kL23Bins];
+    __shared__ uint32_t s_w32[8];
+    __shared__ double s_w64[8];
+    const uint32_t l = blockIdx.x, w = blockIdx.y;
+    const size_t wl = (size_t)w * L + l;
+    Cand* cd = cands + wl * K;
+    SlotTab& stab = slots[wl];
+    const uint32_t ns = stab.n;
+    for (uint32_t s = 0; s < ns; ++s) {
+        uint32_t* gc = g_cnt + (wl * K + s) * kL23Bins;
+        unsigned long long* gs = g_ss + (wl * K + s) * kL23Bins;
+        const uint32_t prefix = stab.prefix[s];
+        for (int b = threadIdx.x; b < kL23Bins; b += kThreads) {
+            const uint32_t c = gc[b];
+            s_incl[kL23Bins - 1 - b] = c;
+            gc[b] = 0;
+            if (LEVEL == 2) { // prefix = level-1 bin: 8 exponent bits + 3 mantissa bits
+                s_below[b] = (double)gs[b] * sq_scale(prefix >> 3);
+                gs[b] = 0ull;
+            } else { // all 31 bits known: the bin's sum of squares is count * value^2
+                const double v = (double)__uint_as_float((prefix << 10) | (uint32_t)b);
+                s_below[b] = (double)c * v * v;
+            }
+        }
+        __syncthreads();
+        scan_bins<kL23Bins>(s_incl, s_below, s_w32, s_w64);
+        for (uint32_t j = threadIdx.x; j < K; j += kThreads) {
+            Cand c = cd[j];
+            if (c.slot != s) continue;
+            const int p = find_pos<kL23Bins>(s_incl, c.rank);
+            const uint32_t above = p ? s_incl[p - 1] : 0u;
+            const uint32_t bin = (uint32_t)(kL23Bins - 1 - p);
+            c.prefix = (prefix << 10) | bin;
+            c.gt += above;
+            c.err_low += s_below[bin];
+            if (LEVEL == 2) {
+                c.rank -= above;
+                cd[j] = c;
+            } else {
+                const uint32_t eq = s_incl[p] - above;
+                const uint32_t keep = c.rank - above; // 1 <= keep <= eq
+                const double v = (double)__uint_as_float(c.prefix);
+                const double e = c.err_low + (double)(eq - keep) * v * v;
+                err_out[wl * K + j] = (float)e;
+                tau_out[wl * K + j] = c.prefix;
+                keep_eq_out[wl * K + j] = keep;
+            }
+        }
+        __syncthreads();
+    }
+    if (LEVEL == 2 && threadIdx.x == 0) { // new slots: distinct 21-bit prefixes (non-increasing in j)
+        uint32_t n2 = 0;
+        for (uint32_t j = 0; j < K; ++j) {
+            if (n2 == 0 || stab.prefix[n2 - 1] != cd[j].prefix) stab.prefix[n2++] = cd[j].prefix;
+            cd[j].slot = n2 - 1;
+        }
+        stab.n = n2;
+    }
+}
+
+// level-2 / level-3 histograms over the materialised difference
+template <int LEVEL, bool VEC>
+__global__ void __launch_bounds__(kThreads)
+k_hist23(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks, uint64_t dstride, uint32_t L,
+         uint32_t K, const SlotTab* __restrict__ slots, uint32_t* __restrict__ g_cnt,
+         unsigned long long* __restrict__ g_ss) {
+    __shared__ uint8_t s_first[kL1Bins]; // level-1 bin -> first slot whose prefix starts with it (0xff: none)
+    __shared__ uint8_t s_num[kL1Bins];   // ... and how many consecutive slots share that bin (level 3)
+    __shared__ uint32_t s_prefix[KIMAD_MAX_RATIOS];
+    const Chunk ch = chunks[blockIdx.x];
+    const uint32_t w = blockIdx.y;
+    const size_t wl = (size_t)w * L + ch.layer;
+    const SlotTab& stab = slots[wl];
+    const uint32_t ns = stab.n;
+    for (int b = threadIdx.x; b < kL1Bins; b += kThreads) { s_first[b] = 0xff; s_num[b] = 0; }
+    for (uint32_t s = threadIdx.x; s < ns; s += kThreads) s_prefix[s] = stab.prefix[s];
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (uint32_t s = 0; s < ns; ++s) {
+            const uint32_t b1 = LEVEL == 2 ? s_prefix[s] : (s_prefix[s] >> 10);
+            if (s_first[b1] == 0xff) s_first[b1] = (uint8_t)s;
+            s_num[b1]++;
+        }
+    }
+    __syncthreads();
+    const float* dd = dbuf + (size_t)w * dstride;
+    uint32_t* gc = g_cnt + wl * K * kL23Bins;
+    unsigned long long* gs = g_ss + wl * K * kL23Bins;
+
+    auto visit = [&](float dv) {
+        const uint32_t key = key_of(dv);
+        const uint32_t f = s_first[key >> 20];
+        if (f == 0xff) return;
+        if (LEVEL == 2) {
+            const uint32_t bin = (key >> 10) & 1023u;
+            atomicAdd(&gc[(size_t)f * kL23Bins + bin], 1u);
+            atomicAdd(&gs[(size_t)f * kL23Bins + bin], (unsigned long long)sq_fixed(key));
+        } else {
+            const uint32_t n = s_num[key >> 20];
+            const uint32_t p21 = key >> 10;
+            for (uint32_t s = f; s < f + n; ++s)
+                if (s_prefix[s] == p21) { atomicAdd(&gc[(size_t)s * kL23Bins + (key & 1023u)], 1u); break; }
+        }
+    };
+
+    const uint64_t q0 = ch.begin & ~3ull;
+    constexpr int U = 4;
+    for (uint64_t base = q0; base < ch.end; base += (uint64_t)4 * kThreads * U) {
+        float4 a[U];
+        bool full[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint64_t q = base + 4ull * (threadIdx.x + (uint64_t)u * kThreads);
+            full[u] = VEC && q >= ch.begin && q + 4 <= ch.end;
+            if (full[u]) a[u] = __ldcs(reinterpret_cast<const float4*>(dd + q));
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint64_t q = base + 4ull * (threadIdx.x + (uint64_t)u * kThreads);
+            if (full[u]) {
+                visit(a[u].x); visit(a[u].y); visit(a[u].z); visit(a[u].w);
+            } else if (q < ch.end) {
+                for (int i = 0; i < 4; ++i) {
+                    const uint64_t p = q + i;
+                    if (p >= ch.begin && p < ch.end) visit(dd[p]);
+                }
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// (c) knapsack DP over the budget axis, one CTA per worker
+// ------------------------------------------------------------------------------------------------
+struct DpBudgets { uint64_t c[kDpWorkersPerLaunch]; };
+
+constexpr int kDpThreads = 1024;
+
+// mode 0: DP; mode 1: candidates given (j_in)
+__global__ void __launch_bounds__(kDpThreads)
+k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uint32_t D, uint32_t bpe,
+     uint64_t full_bytes, uint64_t cap, uint32_t check_finite, int mode, const uint64_t* __restrict__ ktab,
+     const float* __restrict__ err, const uint32_t* __restrict__ tau, const uint32_t* __restrict__ keep_eq,
+     const uint32_t* __restrict__ j_in, uint32_t* __restrict__ flags, uint8_t* __restrict__ pd_global,
+     int pd_in_smem, Sel* __restrict__ sel, uint32_t* __restrict__ out_k, uint32_t* __restrict__ out_j,
+     uint64_t* __restrict__ out_offs, kimad_stats* __restrict__ out_stats) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const uint32_t w = w_base + blockIdx.x;
+    if (w >= W) return;
+    const uint64_t c = budgets.c[blockIdx.x];
+    const uint32_t row = D + 1;
+    float* prev = reinterpret_cast<float*>(smem_raw);
+    float* cur = prev + row;
+    uint32_t* s_units = reinterpret_cast<uint32_t*>(cur + row);
+    float* s_err = reinterpret_cast<float*>(s_units + K);
+    uint32_t* s_j = reinterpret_cast<uint32_t*>(s_err + K); // [L]
+    uint8_t* pd = pd_in_smem ? reinterpret_cast<uint8_t*>(s_j + L) : pd_global + (size_t)w * L * row;
+    __shared__ float s_redv[32];
+    __shared__ uint32_t s_redb[32];
+    __shared__ int s_status;
+
+    const float* e_w = err + (size_t)w * L * K;
+    const uint32_t fl = flags[w];
+    int status = KIMAD_OK;
+    if (check_finite && (fl & 1u)) status = KIMAD_ERR_NONFINITE;
+
+    if (status == KIMAD_OK) {
+        if (mode == 1) {
+            for (uint32_t l = threadIdx.x; l < L; l += blockDim.x) s_j[l] = min(j_in[(size_t)w * L + l], K - 1);
+        } else if (c >= full_bytes) {
+            status = KIMAD_STATUS_PLATEAU;
+            for (uint32_t l = threadIdx.x; l < L; l += blockDim.x) s_j[l] = K - 1;
+        } else if (c == 0) {
+            status = KIMAD_STATUS_INFEASIBLE;
+            for (uint32_t l = threadIdx.x; l < L; l += blockDim.x) s_j[l] = 0;
+        } else {
+            for (uint32_t b = threadIdx.x; b < row; b += blockDim.x) prev[b] = b ? __int_as_float(0x7f800000) : 0.f;
+            for (uint32_t l = 0; l < L; ++l) {
+                __syncthreads();
+                if (threadIdx.x < K) {
+                    const uint64_t bytes = ktab[(size_t)l * K + threadIdx.x] * bpe;
+                    const uint64_t u = budget_cells(bytes, D, c);
+                    s_units[threadIdx.x] = u > D ? 0xffffffffu : (uint32_t)u;
+                    s_err[threadIdx.x] = e_w[(size_t)l * K + threadIdx.x];
+                }
+                __syncthreads();
+                for (uint32_t b = threadIdx.x; b < row; b += blockDim.x) {
+                    float best = __int_as_float(0x7f800000);
+                    uint32_t bj = 0;
+                    for (uint32_t j = 0; j < K; ++j) {
+                        const uint32_t u = s_units[j];
+                        if (u <= b) {
+                            const float t = __fadd_rn(prev[b - u], s_err[j]);
+                            if (t < best) { best = t; bj = j; }
+                        }
+                    }
+                    cur[b] = best;
+                    pd[(size_t)l * row + b] = (uint8_t)bj;
+                }
+                float* sw = prev; prev = cur; cur = sw;
+            }
+            __syncthreads();
+            // lowest cell attaining the minimum: lexicographic (value, cell) min-reduction
+            float bv = __int_as_float(0x7f800000);
+            uint32_t bb = 0xffffffffu;
+            for (uint32_t b = threadIdx.x; b < row; b += blockDim.x) {
+                const float v = prev[b];
+                if (v < bv || (v == bv && b < bb)) { bv = v; bb = b; }
+            }
+#pragma unroll
+            for (int o = 16; o; o >>= 1) {
+                const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+                const uint32_t ob = __shfl_xor_sync(0xffffffffu, bb, o);
+                if (ov < bv || (ov == bv && ob < bb)) { bv = ov; bb = ob; }
+            }
+            if ((threadIdx.x & 31) == 0) { s_redv[threadIdx.x >> 5] = bv; s_redb[threadIdx.x >> 5] = bb; }
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                for (uint32_t i = 1; i < blockDim.x / 32; ++i) {
+                    const float ov = s_redv[i];
+                    const uint32_t ob = s_redb[i];
+                    if (ov < bv || (ov == bv && ob < bb)) { bv = ov; bb = ob; }
+                }
+                if (!(bv < __int_as_float(0x7f800000))) {
+                    s_status = KIMAD_STATUS_INFEASIBLE;
+                } else {
+                    s_status = KIMAD_OK;
+                    uint32_t b = bb;
+                    for (uint32_t l = L; l-- > 0;) { // walk the back-pointers
+                        const uint32_t j = pd[(size_t)l * row + b];
+                        s_j[l] = j;
+                        const uint64_t bytes = ktab[(size_t)l * K + j] * bpe;
+                        b -= (uint32_t)budget_cells(bytes, D, c);
+                    }
+                }
+            }
+            __syncthreads();
+            status = s_status;
+            if (status == KIMAD_STATUS_INFEASIBLE)
+                for (uint32_t l = threadIdx.x; l < L; l += blockDim.x) s_j[l] = 0;
+        }
+    }
+    __syncthreads();
+
+    // totals, capacity check and outputs
+    if (threadIdx.x == 0) {
+        uint64_t nsel = 0;
+        float tot = 0.f;
+        if (status >= 0)
+            for (uint32_t l = 0; l < L; ++l) {
+                nsel += ktab[(size_t)l * K + s_j[l]];
+                tot = __fadd_rn(tot, e_w[(size_t)l * K + s_j[l]]);
+            }
+        if (status >= 0 && nsel > cap) status = KIMAD_ERR_CAPACITY;
+        kimad_stats s;
+        s.budget_bytes = c;
+        s.n_selected = status >= 0 ? nsel : 0;
+        s.used_bytes = s.n_selected * bpe;
+        s.total_err = status >= 0 ? tot : 0.f;
+        s.status = status;
+        out_stats[w] = s;
+        uint64_t run = 0;
+        for (uint32_t l = 0; l < L; ++l) {
+            out_offs[(size_t)w * (L + 1) + l] = run;
+            if (status >= 0) run += ktab[(size_t)l * K + s_j[l]];
+        }
+        out_offs[(size_t)w * (L + 1) + L] = run;
+        s_status = status;
+        flags[w] = 0; // consumed
+    }
+    __syncthreads();
+    status = s_status;
+    for (uint32_t l = threadIdx.x; l < L; l += blockDim.x) {
+        const size_t wl = (size_t)w * L + l;
+        Sel s;
+        if (status >= 0) {
+            const uint32_t j = s_j[l];
+            const uint64_t k = ktab[(size_t)l * K + j];
+            s.tau = tau[wl * K + j];
+            s.keep_eq = keep_eq[wl * K + j];
+            s.k = (uint32_t)k;
+            s.base = out_offs[(size_t)w * (L + 1) + l];
+            out_k[wl] = (uint32_t)k;
+            out_j[wl] = j;
+        } else {
+            s.tau = 0; s.keep_eq = 0; s.k = 0; s.base = 0;
+            out_k[wl] = 0;
+            out_j[wl] = 0;
+        }
+        sel[wl] = s;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// (d) per-chunk counts at the chosen threshold, then an exclusive scan over each layer's chunks
+// ------------------------------------------------------------------------------------------------
+template <bool VEC>
+__global__ void __launch_bounds__(kThreads)
+k_select_count(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks, uint64_t dstride,
+               uint32_t L, const Sel* __restrict__ sel, const LayerDesc* __restrict__ layers,
+               uint2* __restrict__ chunk_cnt) {
+    __shared__ uint32_t s_w[8];
+    const Chunk ch = chunks[blockIdx.x];
+    const uint32_t w = blockIdx.y;
+    const Sel s = sel[(size_t)w * L + ch.layer];
+    uint2* out = chunk_cnt + (size_t)w * n_chunks + blockIdx.x;
+    if (s.k == 0) { if (threadIdx.x == 0) *out = make_uint2(0, 0); return; }
+    if ((uint64_t)s.k == layers[ch.layer].n) { // everything kept: no need to look at the data
+        if (threadIdx.x == 0) *out = make_uint2((uint32_t)(ch.end - ch.begin), 0);
+        return;
+    }
+    const float* dd = dbuf + (size_t)w * dstride;
+    uint32_t gt = 0, eq = 0;
+    auto visit = [&](float dv) {
+        const uint32_t key = key_of(dv);
+        gt += key > s.tau;
+        eq += key == s.tau;
+    };
+    const uint64_t q0 = ch.begin & ~3ull;
+    constexpr int U = 4;
+    for (uint64_t base = q0; base < ch.end; base += (uint64_t)4 * kThreads * U) {
+        float4 a[U];
+        bool full[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint64_t q = base + 4ull * (threadIdx.x + (uint64_t)u * kThreads);
+            full[u] = VEC && q >= ch.begin && q + 4 <= ch.end;
+            if (full[u]) a[u] = __ldg(reinterpret_cast<const float4*>(dd + q));
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint64_t q = base + 4ull * (threadIdx.x + (uint64_t)u * kThreads);
+            if (full[u]) {
+                visit(a[u].x); visit(a[u].y); visit(a[u].z); visit(a[u].w);
+            } else if (q < ch.end) {
+                for (int i = 0; i < 4; ++i) {
+                    const uint64_t p = q + i;
+                    if (p >= ch.begin && p < ch.end) visit(dd[p]);
+                }
+            }
+        }
+    }
+    uint32_t tg, te;
+    block_excl_scan<uint32_t>(gt, s_w, &tg);
+    block_excl_scan<uint32_t>(eq, s_w, &te);
+    if (threadIdx.x == 0) *out = make_uint2(tg, te);
+}
+
+// in place: chunk_cnt[(w, chunk)] becomes the exclusive prefix (gt, eq) over the layer's earlier chunks
+__global__ void __launch_bounds__(kThreads)
+k_select_scan(const LayerDesc* __restrict__ layers, uint32_t n_chunks, uint2* __restrict__ chunk_cnt) {
+    __shared__ uint32_t s_w[8];
+    const LayerDesc ld = layers[blockIdx.x];
+    uint2* cc = chunk_cnt + (size_t)blockIdx.y * n_chunks + ld.first_chunk;
+    uint32_t run_g = 0, run_e = 0;
+    for (uint32_t base = 0; base < ld.n_chunks; base += kThreads) {
+        const uint32_t i = base + threadIdx.x;
+        uint2 v = i < ld.n_chunks ? cc[i] : make_uint2(0, 0);
+        uint32_t tg, te;
+        const uint32_t eg = block_excl_scan<uint32_t>(v.x, s_w, &tg);
+        const uint32_t ee = block_excl_scan<uint32_t>(v.y, s_w, &te);
+        if (i < ld.n_chunks) cc[i] = make_uint2(run_g + eg, run_e + ee);
+        run_g += tg;
+        run_e += te;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// (e) + (f) ordered compaction and EF21 update
+// ------------------------------------------------------------------------------------------------
+template <bool BF16>
+__global__ void __launch_bounds__(kThreads)
+k_select_write(const float* __restrict__ dbuf, float* __restrict__ state, const Chunk* __restrict__ chunks,
+               uint32_t n_chunks, uint64_t dstride, uint64_t stride, uint32_t L, const Sel* __restrict__ sel,
+               const LayerDesc* __restrict__ layers, const uint2* __restrict__ chunk_pre, uint64_t cap,
+               uint32_t* __restrict__ out_idx, void* __restrict__ out_val) {
+    __shared__ uint32_t s_w[8];
+    const Chunk ch = chunks[blockIdx.x];
+    const uint32_t w = blockIdx.y;
+    const Sel s = sel[(size_t)w * L + ch.layer];
+    if (s.k == 0) return;
+    const LayerDesc ld = layers[ch.layer];
+    const bool all = (uint64_t)s.k == ld.n;
+    const uint2 pre = chunk_pre[(size_t)w * n_chunks + blockIdx.x];
+    // entries equal to tau are kept while their rank among equals (ascending index) is below keep_eq
+    uint32_t eq_seen = pre.y;
+    uint64_t pos = s.base + pre.x + min(pre.y, s.keep_eq);
+    const float* dd = dbuf + (size_t)w * dstride;
+    float* st = state + (size_t)w * stride;
+    uint32_t* oi = out_idx + (size_t)w * cap;
+    float* ov32 = reinterpret_cast<float*>(out_val) + (size_t)w * cap;
+    __nv_bfloat16* ov16 = reinterpret_cast<__nv_bfloat16*>(out_val) + (size_t)w * cap;
+
+    const uint64_t q0 = ch.begin & ~3ull;
+    for (uint64_t base = q0; base < ch.end; base += 4ull * kThreads) {
+        const uint64_t q = base + 4ull * threadIdx.x;
+        float v[4];
+        bool in[4], isgt[4], iseq[4];
+        uint32_t ngt = 0, neq = 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint64_t p = q + i;
+            in[i] = p >= ch.begin && p < ch.end;
+            v[i] = in[i] ? dd[p] : 0.f;
+            const uint32_t key = key_of(v[i]);
+            isgt[i] = in[i] && (all || key > s.tau);
+            iseq[i] = in[i] && !all && key == s.tau;
+            ngt += isgt[i];
+            neq += iseq[i];
+        }
+        uint32_t tot_eq;
+        uint32_t eq_rank = eq_seen + block_excl_scan<uint32_t>(neq, s_w, &tot_eq);
+        uint32_t nkeep = ngt;
+        bool keep[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            keep[i] = isgt[i];
+            if (iseq[i]) {
+                keep[i] = eq_rank < s.keep_eq;
+                nkeep += keep[i];
+                ++eq_rank;
+            }
+        }
+        uint32_t tot_keep;
+        uint64_t o = pos + block_excl_scan<uint32_t>(nkeep, s_w, &tot_keep);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if (keep[i]) {
+                const uint64_t p = q + i;
+                oi[o] = (uint32_t)(p - ld.begin);
+                float sent;
+                if (BF16) {
+                    const __nv_bfloat16 h = __float2bfloat16_rn(v[i]);
+                    ov16[o] = h;
+                    sent = __bfloat162float(h);
+                } else {
+                    ov32[o] = v[i];
+                    sent = v[i];
+                }
+                st[p] = __fadd_rn(st[p], sent);
+                ++o;
+            }
+        }
+        eq_seen += tot_eq;
+        pos += tot_keep;
+    }
+}
+
+} // namespace kimad

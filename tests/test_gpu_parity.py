@@ -1,0 +1,196 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import kimad_oracle as ko
+from paper_2312_08053_b200 import binding as kb
+from paper_2312_08053_b200 import workloads
+from tests._harness import Runner, u32
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_workload(cfg, divisor, steps, grid=None, D=None):
+    wl = workloads.workload(cfg, divisor)
+    grid = grid or wl.ratio_grid
+    r = Runner(wl.layer_sizes, wl.n_workers, grid, D or wl.D, wl.value_dtype)
+    bw = workloads.bandwidth_trace(wl, max(steps, 60))
+    pick = np.linspace(0, len(bw) - 1, steps).astype(int)  # spread over the trace: low and high budgets
+    state = torch.zeros((wl.n_workers, wl.N), dtype=torch.float32, device="cuda")
+    mismatched = 0
+    for s in range(steps):
+        grads = workloads.gradients(wl, s, device="cuda")
+        res = r.compare_step(grads, state, bw[pick[s]], wl.t_target)
+        mismatched += not res["same_k"]
+    # the free-running state after `steps` steps was compared bit for bit at every step
+    assert mismatched == 0, f"{mismatched} steps chose another k than the oracle on its own curve"
+
+
+def test_cfg1_mlp_full_size():
+    _run_workload(1, 1, 3)
+
+
+def test_cfg2_resnet18_shape_scaled():
+    _run_workload(2, 8, 4)
+
+
+def test_cfg3_resnet50_shape_scaled():
+    _run_workload(3, 16, 3)
+
+
+def test_cfg4_gpt2_shape_scaled():
+    _run_workload(4, 64, 3)
+
+
+def test_cfg5_llama_shape_scaled_bf16():
+    _run_workload(5, 512, 4)
+
+
+def test_paper_grid_50_candidates():
+    _run_workload(2, 32, 2, grid=workloads.paper_grid_50())
+
+
+def test_worked_example_on_gpu():
+    a = np.arange(1, 11, dtype=np.float32)
+    b = np.float32([-8, 0.5, 8, -0.5])
+    c = np.float32([3, -3, 3, 0, -0.0, 1])
+    flat = torch.from_numpy(np.concatenate([a, b, c])[None, :]).cuda()
+    for budget, D, want in [(96, 12, [5, 4, 3]), (96, 1000, [5, 2, 3]), (100, 1000, [5, 4, 3]), (95, 12, [5, 2, 2]),
+                            (200, 1000, [10, 4, 6]), (47, 1000, [3, 1, 2])]:
+        r = Runner([10, 4, 6], 1, [0.25, 0.5, 1.0], D=D)
+        state = torch.zeros_like(flat)
+        res = r.compare_step(flat, state, [float(budget)], 1.0)
+        assert u32(r.out.k)[0].tolist() == want
+        assert res["same_k"]
+
+
+def _adversarial_layers(rng):
+    n = 70001
+    layers = []
+    layers.append(np.full(n, 0.5, np.float32) * np.where(rng.uniform(size=n) < 0.5, -1, 1))      # all equal magnitude
+    layers.append(np.zeros(4097, np.float32))                                                      # all zero
+    z = np.zeros(33000, np.float32); z[::2] = -0.0                                                 # +0 / -0 mix
+    layers.append(z)
+    one = np.zeros(40000, np.float32); one[31999] = -3.0                                           # a single nonzero
+    layers.append(one)
+    layers.append(np.float32([7.0]))                                                               # n = 1
+    den = (rng.integers(1, 2 ** 22, 50000).astype(np.uint32)).view(np.float32)                     # denormals
+    layers.append(den * np.where(rng.uniform(size=50000) < 0.5, -1, 1).astype(np.float32))
+    dup = rng.choice(np.float32([1.0, 1.0000001, 0.9999999, 2.0, 1e-3]), 100003).astype(np.float32)  # few distinct values
+    layers.append(dup)
+    emb = np.zeros(64 * 3000, np.float32)                                                          # row-sparse "embedding"
+    rows = rng.choice(3000, 90, replace=False)
+    for r in rows:
+        emb[r * 64:(r + 1) * 64] = rng.standard_normal(64).astype(np.float32) * 1e-2
+    layers.append(emb)
+    layers.append((rng.standard_normal(13) * 1e15).astype(np.float32))                             # huge, squares still finite
+    layers.append((rng.standard_normal(65537) * 1e-30).astype(np.float32))                         # tiny normals
+    return [np.ascontiguousarray(x, np.float32) for x in layers]
+
+
+@pytest.mark.parametrize("value_dtype", [0, 1])
+def test_adversarial_inputs(value_dtype):
+    rng = np.random.default_rng(77)
+    layers = _adversarial_layers(rng)
+    sizes = [x.size for x in layers]
+    N = sum(sizes)
+    grid = [0.001, 0.01, 0.1, 0.5, 0.9, 1.0]
+    r = Runner(sizes, 2, grid, value_dtype=value_dtype)
+    flat = np.concatenate(layers)
+    grads = torch.from_numpy(np.stack([flat, flat[::-1].copy()])).cuda()   # worker 1: same values, other layout
+    bpe = 8 if value_dtype == 0 else 6
+    state = torch.zeros_like(grads)
+    for frac in (0.02, 0.3, 0.95):
+        # several layers here have exactly linear error curves, so many assignments tie up to the last
+        # rounding of the curve: the decision is compared on the SAME curve (inside compare_step) only
+        r.compare_step(grads, state, [frac * N * bpe, 0.5 * frac * N * bpe], 1.0)
+
+
+def test_unaligned_stride_and_offsets_take_scalar_path():
+    rng = np.random.default_rng(5)
+    sizes = [10, 1000, 50257, 3, 40001, 7]            # layer starts not 16-byte aligned
+    N = sum(sizes)
+    stride = N + 3                                     # worker rows not 16-byte aligned either
+    grid = [0.01, 0.1, 0.5, 1.0]
+    r = Runner(sizes, 3, grid, stride=stride)
+    grads = torch.from_numpy((rng.standard_t(3, (3, stride)) * 1e-2).astype(np.float32)).cuda()
+    state = torch.from_numpy((rng.standard_normal((3, stride)) * 1e-3).astype(np.float32)).cuda()
+    pad_before = state[:, N:].clone()
+    res = r.compare_step(grads, state, [0.05 * N * 8, 0.2 * N * 8, 0.6 * N * 8], 1.0)
+    assert res["same_k"]
+    assert torch.equal(state[:, N:], pad_before)       # padding between workers untouched
+
+
+def test_statuses_plateau_infeasible_capacity_nonfinite():
+    rng = np.random.default_rng(6)
+    sizes = [5000, 300, 70000]
+    N = sum(sizes)
+    grid = [0.01, 0.1, 1.0]
+    grads = torch.from_numpy(rng.standard_normal((2, N)).astype(np.float32)).cuda()
+    # plateau on worker 0, infeasible on worker 1
+    r = Runner(sizes, 2, grid)
+    state = torch.zeros_like(grads)
+    res = r.compare_step(grads, state, [8.0 * N, 100.0], 1.0)
+    st = r.out.stats_host()
+    assert st["status"].tolist() == [kb.KIMAD_STATUS_PLATEAU, kb.KIMAD_STATUS_INFEASIBLE]
+    assert res["status"] == kb.KIMAD_STATUS_PLATEAU
+    assert u32(r.out.k)[0].tolist() == sizes and st["total_err"][0] == 0.0
+    assert torch.equal(state[0], grads[0] - torch.zeros_like(grads[0]))  # everything sent: g + (grad - g), g = 0
+    # capacity: worker 0 wants more entries than the packed buffers hold -> error status, state untouched
+    r = Runner(sizes, 2, grid, cap=1000)
+    state = torch.zeros_like(grads)
+    status, k = r.gpu_step(grads, state, [8.0 * N, 8.0 * 900], 1.0)
+    st = r.out.stats_host()
+    assert status == kb.KIMAD_ERR_CAPACITY
+    assert st["status"][0] == kb.KIMAD_ERR_CAPACITY and st["status"][1] == 0
+    assert int(st["n_selected"][0]) == 0 and not state[0].any()
+    assert int(st["n_selected"][1]) <= 900 and state[1].any()
+    # non-finite input with check_finite
+    r = Runner(sizes, 2, grid, check_finite=1)
+    bad = grads.clone()
+    bad[1, 5100] = float("inf")
+    state = torch.zeros_like(grads)
+    status, k = r.gpu_step(bad, state, [8.0 * 800, 8.0 * 800], 1.0)
+    st = r.out.stats_host()
+    assert status == kb.KIMAD_ERR_NONFINITE
+    assert st["status"].tolist() == [0, kb.KIMAD_ERR_NONFINITE]
+    assert not state[1].any() and state[0].any()
+    # the flag does not stick: the next clean step succeeds
+    status, k = r.gpu_step(grads, state, [8.0 * 800, 8.0 * 800], 1.0)
+    assert status == 0
+
+
+def test_given_j_skips_the_dp():
+    rng = np.random.default_rng(8)
+    sizes = [3000, 50, 20000]
+    grid = [0.01, 0.05, 0.25, 1.0]
+    r = Runner(sizes, 1, grid)
+    grads = torch.from_numpy(rng.standard_normal((1, sum(sizes))).astype(np.float32)).cuda()
+    state = torch.zeros_like(grads)
+    j = torch.tensor([[2, 0, 3]], dtype=torch.int32, device="cuda")
+    kb.kimad_debug_step_with_j(r.ctx, grads, state, [1.0], 1.0, r.out, j)
+    status, k = kb.kimad_get_k(r.ctx)
+    assert k[0].tolist() == [750, 1, 20000]
+    d = grads.cpu().numpy()[0]
+    offs = np.concatenate([[0], np.cumsum(sizes)])
+    pos = 0
+    for l, kk in enumerate(k[0]):
+        idx, val = ko.select_pack(d[offs[l]:offs[l + 1]], int(kk))
+        assert np.array_equal(u32(r.out.idx)[0, pos:pos + kk], idx)
+        assert np.array_equal(r.out.val.cpu().numpy()[0, pos:pos + kk], val)
+        pos += int(kk)
+
+
+def test_run_to_run_determinism_of_decisions():
+    wl = workloads.workload(3, 32)
+    bw = workloads.bandwidth_trace(wl, 10)[7]
+    grads = workloads.gradients(wl, 0, device="cuda")
+    outs = []
+    for _ in range(3):
+        r = Runner(wl.layer_sizes, wl.n_workers, wl.ratio_grid)
+        state = torch.zeros_like(grads)
+        r.gpu_step(grads, state, bw, wl.t_target)
+        outs.append((u32(r.out.k).copy(), u32(r.out.idx).copy(), u32(state).copy()))
+    for o in outs[1:]:
+        assert all(np.array_equal(a, b) for a, b in zip(outs[0], o))
