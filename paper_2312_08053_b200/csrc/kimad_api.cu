@@ -18,7 +18,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
     size_t dbuf, chunks, layers, ktab, h1_cnt, h1_ss, h23_cnt, h23_ss, cands, slots, err, tau, keep_eq, sel, chunk_cnt,
-        flags, pd, total;
+        chunk_pre, flags, pd, total;
 };
 
 } // namespace
@@ -34,8 +34,8 @@ struct kimad_ctx {
     std::vector<LayerDesc> layers;
     Layout lay{};
     unsigned char* ws = nullptr;
-    bool pd_in_smem = false;
-    size_t dp_smem = 0;
+    DpPlan dp_plan{};
+    size_t dp_smem = 0, hist2_smem = 0, hist3_smem = 0;
     uint64_t launches = 0;
     kimad_packed last_out{};
     bool have_last = false;
@@ -67,8 +67,9 @@ void plan_layout(kimad_ctx* c) {
     y.keep_eq = take(WLK * sizeof(uint32_t));
     y.sel = take(WL * sizeof(Sel));
     y.chunk_cnt = take((size_t)c->W * c->chunks.size() * sizeof(uint2));
+    y.chunk_pre = take((size_t)c->W * c->chunks.size() * sizeof(uint2));
     y.flags = take((size_t)c->W * sizeof(uint32_t));
-    y.pd = take(c->pd_in_smem ? 0 : (size_t)c->W * c->L * (c->D + 1));
+    y.pd = take(c->dp_plan.pd_in_smem ? 0 : (size_t)c->W * c->L * c->dp_plan.pd_row_bytes);
     y.total = o;
 }
 
@@ -108,6 +109,7 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
     uint32_t* keq = c->at<uint32_t>(c->lay.keep_eq);
     Sel* sel = c->at<Sel>(c->lay.sel);
     uint2* ccnt = c->at<uint2>(c->lay.chunk_cnt);
+    uint2* cpre = c->at<uint2>(c->lay.chunk_pre);
     uint32_t* flags = c->at<uint32_t>(c->lay.flags);
     uint8_t* pd = c->at<uint8_t>(c->lay.pd);
 
@@ -123,17 +125,30 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
         k_diff_hist1<false><<<gch, blk, 0, s>>>(grads, state, dbuf, chunks, c->stride, c->dstride, L, h1c, h1s, flags);
     mark();
     // (b) remaining digits
+    const bool smem_hist = true;
+    const uint32_t skip = smem_hist ? (uint32_t)kSmemSlots : 0u;
+    const uint32_t zslots = std::min<uint32_t>(K, KIMAD_MAX_RATIOS);
+    const dim3 grun((nch + kRunChunks - 1) / kRunChunks, W), gslot(L, W, zslots);
     k_resolve1<<<glw, blk, 0, s>>>(h1c, h1s, ktab, L, K, cands, slots);
     mark();
-    k_hist23<2, true><<<gch, blk, 0, s>>>(dbuf, chunks, c->dstride, L, K, slots, h23c, h23s);
+    k_hist23_smem<2><<<grun, kHThreads, c->hist2_smem, s>>>(dbuf, chunks, nch, c->dstride, L, K, slots, h23c, h23s);
+    if (K > (uint32_t)kSmemSlots) {
+        k_hist23<2, true><<<gch, blk, 0, s>>>(dbuf, chunks, c->dstride, L, K, slots, h23c, h23s, skip);
+        c->launches += 1;
+    }
     mark();
-    k_resolve23<2><<<glw, blk, 0, s>>>(h23c, h23s, L, K, cands, slots, err, tau, keq);
+    k_resolve23<2><<<gslot, blk, 0, s>>>(h23c, h23s, L, K, cands, slots, err, tau, keq);
+    k_rebuild_slots<<<(W * L + kThreads - 1) / kThreads, blk, 0, s>>>(W * L, K, cands, slots);
     mark();
-    k_hist23<3, true><<<gch, blk, 0, s>>>(dbuf, chunks, c->dstride, L, K, slots, h23c, h23s);
+    k_hist23_smem<3><<<grun, kHThreads, c->hist3_smem, s>>>(dbuf, chunks, nch, c->dstride, L, K, slots, h23c, h23s);
+    if (K > (uint32_t)kSmemSlots) {
+        k_hist23<3, true><<<gch, blk, 0, s>>>(dbuf, chunks, c->dstride, L, K, slots, h23c, h23s, skip);
+        c->launches += 1;
+    }
     mark();
-    k_resolve23<3><<<glw, blk, 0, s>>>(h23c, h23s, L, K, cands, slots, err, tau, keq);
+    k_resolve23<3><<<gslot, blk, 0, s>>>(h23c, h23s, L, K, cands, slots, err, tau, keq);
     mark();
-    c->launches += 6;
+    c->launches += 7;
     // (c)
     for (uint32_t w0 = 0; w0 < W; w0 += kDpWorkersPerLaunch) {
         DpBudgets b{};
@@ -143,23 +158,23 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
             b.c[i] = !(cb > 0.0) ? 0ull : (cb >= 18446744073709551615.0 ? ~0ull : (uint64_t)cb);
         }
         k_dp<<<nw, kDpThreads, c->dp_smem, s>>>(b, w0, W, L, K, c->D, c->bpe, c->full_bytes, c->cap, c->check_finite,
-                                                mode == kGivenJ ? 1 : 0, ktab, mode == kInjectErr ? err_dev : err, tau,
-                                                keq, j_dev, flags, pd, c->pd_in_smem ? 1 : 0, sel, out->k, out->j,
-                                                out->offs, out->stats);
+                                                mode == kGivenJ ? 1 : 0, c->dp_plan, ktab,
+                                                mode == kInjectErr ? err_dev : err, tau, keq, j_dev, flags, pd, sel,
+                                                out->k, out->j, out->offs, out->stats);
         c->launches += 1;
     }
     mark();
     // (d), (e), (f)
-    k_select_count<true><<<gch, blk, 0, s>>>(dbuf, chunks, nch, c->dstride, L, sel, layers, ccnt);
+    k_select_count<<<gch, blk, 0, s>>>(dbuf, chunks, nch, c->dstride, L, sel, layers, ccnt);
     mark();
-    k_select_scan<<<glw, blk, 0, s>>>(layers, nch, ccnt);
+    k_select_scan<<<glw, blk, 0, s>>>(layers, nch, ccnt, cpre);
     mark();
     if (c->value_dtype == 1)
         k_select_write<true><<<gch, blk, 0, s>>>(dbuf, state, chunks, nch, c->dstride, c->stride, L, sel, layers, ccnt,
-                                                 c->cap, out->idx, out->val);
+                                                 cpre, c->cap, out->idx, out->val);
     else
         k_select_write<false><<<gch, blk, 0, s>>>(dbuf, state, chunks, nch, c->dstride, c->stride, L, sel, layers, ccnt,
-                                                  c->cap, out->idx, out->val);
+                                                  cpre, c->cap, out->idx, out->val);
     mark();
     c->launches += 3;
     CUDA_TRY(cudaGetLastError());
@@ -224,11 +239,21 @@ int kimad_create(kimad_ctx** out, const uint64_t* layer_sizes, uint32_t n_layers
         c->cap = o.max_packed_elems ? o.max_packed_elems : N;
         if (c->stride < N || c->chunks.size() > 0x7fffffffull) { delete c; return KIMAD_ERR_INVALID_ARG; }
         c->dstride = (N + 3) / 4 * 4;
-        const size_t dp_rows = ((size_t)2 * (c->D + 1) + 2 * c->K + c->L) * 4;
-        const size_t pd_bytes = (size_t)c->L * (c->D + 1);
-        c->pd_in_smem = dp_rows + pd_bytes <= 225 * 1024;
-        c->dp_smem = dp_rows + (c->pd_in_smem ? pd_bytes : 0);
-        if (dp_rows > 200 * 1024) { delete c; return KIMAD_ERR_INVALID_ARG; }
+        // shared-memory plan of the DP kernel
+        const size_t kDpSmemMax = 225 * 1024;
+        const size_t dp_base = ((size_t)2 * (c->D + 1) + c->L) * 4;
+        const size_t tab_all = (size_t)c->L * c->K * 8, tab_one = (size_t)c->K * 8;
+        c->dp_plan.pd_nibble = c->K <= 16 ? 1u : 0u;
+        c->dp_plan.pd_row_bytes = c->dp_plan.pd_nibble ? (c->D + 2) / 2 : (c->D + 1);
+        const size_t pd_bytes = (size_t)c->L * c->dp_plan.pd_row_bytes;
+        if (dp_base + tab_one > kDpSmemMax) { delete c; return KIMAD_ERR_INVALID_ARG; }
+        c->dp_plan.tab_in_smem = dp_base + tab_all <= kDpSmemMax ? 1u : 0u;
+        size_t used = dp_base + (c->dp_plan.tab_in_smem ? tab_all : tab_one);
+        c->dp_plan.pd_in_smem = used + pd_bytes <= kDpSmemMax ? 1u : 0u;
+        if (c->dp_plan.pd_in_smem) used += pd_bytes;
+        c->dp_smem = used;
+        c->hist2_smem = (size_t)3 * kSmemSlots * kL23Bins * 4 + 2 * kL1Bins + kSmemSlots * 4;
+        c->hist3_smem = (size_t)kSmemSlots * kL23Bins * 4 + 2 * kL1Bins + kSmemSlots * 4;
         plan_layout(c);
     } catch (const std::bad_alloc&) {
         delete c;
@@ -274,6 +299,8 @@ int kimad_set_workspace(kimad_ctx* c, void* dev_ptr, size_t bytes) {
     // everything after the static tables starts at zero: the histograms are kept clean by the kernels
     CUDA_TRY(cudaMemset(c->ws + y.h1_cnt, 0, y.total - y.h1_cnt));
     CUDA_TRY(cudaFuncSetAttribute(k_dp, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->dp_smem));
+    CUDA_TRY(cudaFuncSetAttribute(k_hist23_smem<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->hist2_smem));
+    CUDA_TRY(cudaFuncSetAttribute(k_hist23_smem<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->hist3_smem));
     CUDA_TRY(cudaDeviceSynchronize());
     return KIMAD_OK;
 }

@@ -67,16 +67,21 @@ __device__ __forceinline__ uint64_t sq_fixed(uint32_t key) {
 // scale that turns a bin's integer sum back into a sum of squared values; e = exponent field of the bin
 __device__ __forceinline__ double sq_scale(uint32_t e) { return ldexp(1.0, 2 * ((int)(e ? e : 1u) - 150) + 16); }
 
-// One shared-memory word per level-1 bin: count in the top 17 bits, sum of sq_fixed in the low 47
-// (a chunk has at most 2^15 elements, each adding < 2^32).
-constexpr int kL1CountShift = 47;
-
+// Shared-memory histogram words are u32 (native shared atomics): per bin a count, and the sum of
+// sq_fixed split into its high and low 16 bits.  A bin that received at most 2^16 entries since the
+// last flush cannot overflow either sum.
 struct L1Acc {
-    unsigned long long* acc;
+    uint32_t* cnt;
+    uint32_t* hi;
+    uint32_t* lo;
     uint32_t nonfinite;
     __device__ __forceinline__ void add(float dv) {
         const uint32_t key = key_of(dv);
-        atomicAdd(&acc[key >> 20], (1ull << kL1CountShift) | sq_fixed(key));
+        const uint32_t sq = (uint32_t)sq_fixed(key);
+        const uint32_t b = key >> 20;
+        atomicAdd(&cnt[b], 1u);
+        atomicAdd(&hi[b], sq >> 16);
+        atomicAdd(&lo[b], sq & 0xffffu);
         nonfinite |= ((key >> 23) == 255u);
     }
 };
@@ -86,15 +91,15 @@ __global__ void __launch_bounds__(kThreads)
 k_diff_hist1(const float* __restrict__ grads, const float* __restrict__ state, float* __restrict__ dbuf,
              const Chunk* __restrict__ chunks, uint64_t stride, uint64_t dstride, uint32_t L,
              uint32_t* __restrict__ g_cnt, unsigned long long* __restrict__ g_ss, uint32_t* __restrict__ flags) {
-    __shared__ unsigned long long s_acc[kL1Bins];
+    __shared__ uint32_t s_cnt[kL1Bins], s_hi[kL1Bins], s_lo[kL1Bins];
     const Chunk ch = chunks[blockIdx.x];
     const uint32_t w = blockIdx.y;
-    for (int b = threadIdx.x; b < kL1Bins; b += kThreads) s_acc[b] = 0ull;
+    for (int b = threadIdx.x; b < kL1Bins; b += kThreads) { s_cnt[b] = 0; s_hi[b] = 0; s_lo[b] = 0; }
     __syncthreads();
     const float* gr = grads + (size_t)w * stride;
     const float* st = state + (size_t)w * stride;
     float* dd = dbuf + (size_t)w * dstride;
-    L1Acc acc{s_acc, 0u};
+    L1Acc acc{s_cnt, s_hi, s_lo, 0u};
 
     const uint64_t q0 = ch.begin & ~3ull;
     constexpr int U = 4;
@@ -139,10 +144,10 @@ k_diff_hist1(const float* __restrict__ grads, const float* __restrict__ state, f
     uint32_t* gc = g_cnt + ((size_t)w * L + ch.layer) * kL1Bins;
     unsigned long long* gs = g_ss + ((size_t)w * L + ch.layer) * kL1Bins;
     for (int b = threadIdx.x; b < kL1Bins; b += kThreads) {
-        const unsigned long long v = s_acc[b];
-        if (v) {
-            atomicAdd(&gc[b], (uint32_t)(v >> kL1CountShift));
-            atomicAdd(&gs[b], v & ((1ull << kL1CountShift) - 1));
+        const uint32_t c = s_cnt[b];
+        if (c) {
+            atomicAdd(&gc[b], c);
+            atomicAdd(&gs[b], ((unsigned long long)s_hi[b] << 16) + s_lo[b]);
         }
     }
 }
@@ -156,21 +161,35 @@ template <int NB>
 __device__ __forceinline__ void scan_bins(uint32_t* s_incl /* in: counts by position */, double* s_below /* in: ss by bin */,
                                           uint32_t* s_w32, double* s_w64) {
     constexpr int PER = NB / kThreads;
+    static_assert(PER % 4 == 0, "16-byte shared-memory accesses");
     uint32_t loc[PER];
     uint32_t sum = 0;
+    uint4* v4 = reinterpret_cast<uint4*>(s_incl + threadIdx.x * PER);
 #pragma unroll
-    for (int i = 0; i < PER; ++i) { loc[i] = s_incl[threadIdx.x * PER + i]; sum += loc[i]; }
+    for (int i = 0; i < PER / 4; ++i) {
+        const uint4 t = v4[i];
+        loc[4 * i] = t.x; loc[4 * i + 1] = t.y; loc[4 * i + 2] = t.z; loc[4 * i + 3] = t.w;
+    }
+#pragma unroll
+    for (int i = 0; i < PER; ++i) sum += loc[i];
     uint32_t ex = block_excl_scan<uint32_t>(sum, s_w32, nullptr);
 #pragma unroll
-    for (int i = 0; i < PER; ++i) { ex += loc[i]; s_incl[threadIdx.x * PER + i] = ex; }
+    for (int i = 0; i < PER; ++i) { ex += loc[i]; loc[i] = ex; }
+#pragma unroll
+    for (int i = 0; i < PER / 4; ++i) v4[i] = make_uint4(loc[4 * i], loc[4 * i + 1], loc[4 * i + 2], loc[4 * i + 3]);
     if (s_below) {
         double dl[PER];
         double ds = 0.0;
+        double2* d2 = reinterpret_cast<double2*>(s_below + threadIdx.x * PER);
 #pragma unroll
-        for (int i = 0; i < PER; ++i) { dl[i] = s_below[threadIdx.x * PER + i]; ds += dl[i]; }
+        for (int i = 0; i < PER / 2; ++i) { const double2 t = d2[i]; dl[2 * i] = t.x; dl[2 * i + 1] = t.y; }
+#pragma unroll
+        for (int i = 0; i < PER; ++i) ds += dl[i];
         double de = block_excl_scan<double>(ds, s_w64, nullptr);
 #pragma unroll
-        for (int i = 0; i < PER; ++i) { s_below[threadIdx.x * PER + i] = de; de += dl[i]; }
+        for (int i = 0; i < PER; ++i) { const double t = dl[i]; dl[i] = de; de += t; }
+#pragma unroll
+        for (int i = 0; i < PER / 2; ++i) d2[i] = make_double2(dl[2 * i], dl[2 * i + 1]);
     }
     __syncthreads();
 }
@@ -189,8 +208,8 @@ __device__ __forceinline__ int find_pos(const uint32_t* s_incl, uint32_t rank) {
 __global__ void __launch_bounds__(kThreads)
 k_resolve1(uint32_t* __restrict__ g_cnt, unsigned long long* __restrict__ g_ss, const uint64_t* __restrict__ ktab,
            uint32_t L, uint32_t K, Cand* __restrict__ cands, SlotTab* __restrict__ slots) {
-    __shared__ uint32_t s_incl[kL1Bins];
-    __shared__ double s_below[kL1Bins];
+    __shared__ __align__(16) uint32_t s_incl[kL1Bins];
+    __shared__ __align__(16) double s_below[kL1Bins];
     __shared__ uint32_t s_w32[8];
     __shared__ double s_w64[8];
     const uint32_t l = blockIdx.x, w = blockIdx.y;
@@ -231,70 +250,76 @@ k_resolve1(uint32_t* __restrict__ g_cnt, unsigned long long* __restrict__ g_ss, 
 }
 
 // LEVEL 2: refine inside a level-1 bin; LEVEL 3: inside a (level-1, level-2) bin.
+// One CTA per (layer, worker, slot).
 template <int LEVEL>
 __global__ void __launch_bounds__(kThreads)
 k_resolve23(uint32_t* __restrict__ g_cnt, unsigned long long* __restrict__ g_ss, uint32_t L, uint32_t K,
-            Cand* __restrict__ cands, SlotTab* __restrict__ slots, float* __restrict__ err_out,
+            Cand* __restrict__ cands, const SlotTab* __restrict__ slots, float* __restrict__ err_out,
             uint32_t* __restrict__ tau_out, uint32_t* __restrict__ keep_eq_out) {
-    __shared__ uint32_t s_incl[kL23Bins];
-    __shared__ double s_below[kL23Bins];
+    __shared__ __align__(16) uint32_t s_incl[kL23Bins];
+    __shared__ __align__(16) double s_below[kL23Bins];
     __shared__ uint32_t s_w32[8];
     __shared__ double s_w64[8];
-    const uint32_t l = blockIdx.x, w = blockIdx.y;
+    const uint32_t l = blockIdx.x, w = blockIdx.y, s = blockIdx.z;
     const size_t wl = (size_t)w * L + l;
+    const SlotTab& stab = slots[wl];
+    if (s >= stab.n) return;
     Cand* cd = cands + wl * K;
+    uint32_t* gc = g_cnt + (wl * K + s) * kL23Bins;
+    unsigned long long* gs = g_ss + (wl * K + s) * kL23Bins;
+    const uint32_t prefix = stab.prefix[s];
+    for (int b = threadIdx.x; b < kL23Bins; b += kThreads) {
+        const uint32_t c = gc[b];
+        s_incl[kL23Bins - 1 - b] = c;
+        gc[b] = 0;
+        if (LEVEL == 2) { // prefix = level-1 bin: 8 exponent bits + 3 mantissa bits
+            s_below[b] = (double)gs[b] * sq_scale(prefix >> 3);
+            gs[b] = 0ull;
+        } else { // all 31 bits known: the bin's sum of squares is count * value^2
+            const double v = (double)__uint_as_float((prefix << 10) | (uint32_t)b);
+            s_below[b] = (double)c * v * v;
+        }
+    }
+    __syncthreads();
+    scan_bins<kL23Bins>(s_incl, s_below, s_w32, s_w64);
+    for (uint32_t j = threadIdx.x; j < K; j += kThreads) {
+        Cand c = cd[j];
+        if (c.slot != s) continue;
+        const int p = find_pos<kL23Bins>(s_incl, c.rank);
+        const uint32_t above = p ? s_incl[p - 1] : 0u;
+        const uint32_t bin = (uint32_t)(kL23Bins - 1 - p);
+        c.prefix = (prefix << 10) | bin;
+        c.gt += above;
+        c.err_low += s_below[bin];
+        if (LEVEL == 2) {
+            c.rank -= above;
+            cd[j] = c;
+        } else {
+            const uint32_t eq = s_incl[p] - above;
+            const uint32_t keep = c.rank - above; // 1 <= keep <= eq
+            const double v = (double)__uint_as_float(c.prefix);
+            const double e = c.err_low + (double)(eq - keep) * v * v;
+            err_out[wl * K + j] = (float)e;
+            tau_out[wl * K + j] = c.prefix;
+            keep_eq_out[wl * K + j] = keep;
+        }
+    }
+}
+
+// After digit 2: new slots = distinct 21-bit prefixes (non-increasing in j).  One thread per (worker, layer).
+__global__ void __launch_bounds__(kThreads)
+k_rebuild_slots(uint32_t WL, uint32_t K, Cand* __restrict__ cands, SlotTab* __restrict__ slots) {
+    const uint32_t wl = blockIdx.x * kThreads + threadIdx.x;
+    if (wl >= WL) return;
+    Cand* cd = cands + (size_t)wl * K;
     SlotTab& stab = slots[wl];
-    const uint32_t ns = stab.n;
-    for (uint32_t s = 0; s < ns; ++s) {
-        uint32_t* gc = g_cnt + (wl * K + s) * kL23Bins;
-        unsigned long long* gs = g_ss + (wl * K + s) * kL23Bins;
-        const uint32_t prefix = stab.prefix[s];
-        for (int b = threadIdx.x; b < kL23Bins; b += kThreads) {
-            const uint32_t c = gc[b];
-            s_incl[kL23Bins - 1 - b] = c;
-            gc[b] = 0;
-            if (LEVEL == 2) { // prefix = level-1 bin: 8 exponent bits + 3 mantissa bits
-                s_below[b] = (double)gs[b] * sq_scale(prefix >> 3);
-                gs[b] = 0ull;
-            } else { // all 31 bits known: the bin's sum of squares is count * value^2
-                const double v = (double)__uint_as_float((prefix << 10) | (uint32_t)b);
-                s_below[b] = (double)c * v * v;
-            }
-        }
-        __syncthreads();
-        scan_bins<kL23Bins>(s_incl, s_below, s_w32, s_w64);
-        for (uint32_t j = threadIdx.x; j < K; j += kThreads) {
-            Cand c = cd[j];
-            if (c.slot != s) continue;
-            const int p = find_pos<kL23Bins>(s_incl, c.rank);
-            const uint32_t above = p ? s_incl[p - 1] : 0u;
-            const uint32_t bin = (uint32_t)(kL23Bins - 1 - p);
-            c.prefix = (prefix << 10) | bin;
-            c.gt += above;
-            c.err_low += s_below[bin];
-            if (LEVEL == 2) {
-                c.rank -= above;
-                cd[j] = c;
-            } else {
-                const uint32_t eq = s_incl[p] - above;
-                const uint32_t keep = c.rank - above; // 1 <= keep <= eq
-                const double v = (double)__uint_as_float(c.prefix);
-                const double e = c.err_low + (double)(eq - keep) * v * v;
-                err_out[wl * K + j] = (float)e;
-                tau_out[wl * K + j] = c.prefix;
-                keep_eq_out[wl * K + j] = keep;
-            }
-        }
-        __syncthreads();
+    uint32_t n2 = 0;
+    for (uint32_t j = 0; j < K; ++j) {
+        const uint32_t pfx = cd[j].prefix;
+        if (n2 == 0 || stab.prefix[n2 - 1] != pfx) stab.prefix[n2++] = pfx;
+        cd[j].slot = n2 - 1;
     }
-    if (LEVEL == 2 && threadIdx.x == 0) { // new slots: distinct 21-bit prefixes (non-increasing in j)
-        uint32_t n2 = 0;
-        for (uint32_t j = 0; j < K; ++j) {
-            if (n2 == 0 || stab.prefix[n2 - 1] != cd[j].prefix) stab.prefix[n2++] = cd[j].prefix;
-            cd[j].slot = n2 - 1;
-        }
-        stab.n = n2;
-    }
+    stab.n = n2;
 }
 
 // level-2 / level-3 histograms over the materialised difference
@@ -302,7 +327,7 @@ template <int LEVEL, bool VEC>
 __global__ void __launch_bounds__(kThreads)
 k_hist23(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks, uint64_t dstride, uint32_t L,
          uint32_t K, const SlotTab* __restrict__ slots, uint32_t* __restrict__ g_cnt,
-         unsigned long long* __restrict__ g_ss) {
+         unsigned long long* __restrict__ g_ss, uint32_t skip_up_to_slots) {
     __shared__ uint8_t s_first[kL1Bins]; // level-1 bin -> first slot whose prefix starts with it (0xff: none)
     __shared__ uint8_t s_num[kL1Bins];   // ... and how many consecutive slots share that bin (level 3)
     __shared__ uint32_t s_prefix[KIMAD_MAX_RATIOS];
@@ -311,6 +336,7 @@ k_hist23(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks, uint6
     const size_t wl = (size_t)w * L + ch.layer;
     const SlotTab& stab = slots[wl];
     const uint32_t ns = stab.n;
+    if (ns <= skip_up_to_slots) return; // those layers belong to k_hist23_smem
     for (int b = threadIdx.x; b < kL1Bins; b += kThreads) { s_first[b] = 0xff; s_num[b] = 0; }
     for (uint32_t s = threadIdx.x; s < ns; s += kThreads) s_prefix[s] = stab.prefix[s];
     __syncthreads();
@@ -368,32 +394,185 @@ k_hist23(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks, uint6
     }
 }
 
+
+// Same histograms, accumulated in shared memory with u32 atomics by CTAs that own a run of
+// consecutive chunks; used for layers with at most kSmemSlots slots (the usual case, K <= 16).
+constexpr int kHThreads = 1024;
+constexpr int kSmemSlots = 16;
+constexpr int kRunChunks = 8;
+constexpr uint64_t kDirectElems = 2048; // chunks this small go straight to global atomics
+
+template <int LEVEL>
+__global__ void __launch_bounds__(kHThreads, 1)
+k_hist23_smem(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks, uint64_t dstride,
+              uint32_t L, uint32_t K, const SlotTab* __restrict__ slots, uint32_t* __restrict__ g_cnt,
+              unsigned long long* __restrict__ g_ss) {
+    extern __shared__ __align__(16) uint32_t sh[];
+    constexpr int NW = kSmemSlots * kL23Bins;
+    uint32_t* h_cnt = sh;
+    uint32_t* h_hi = sh + NW;     // LEVEL 2 only
+    uint32_t* h_lo = sh + 2 * NW; // LEVEL 2 only
+    uint8_t* s_first = reinterpret_cast<uint8_t*>(sh + (LEVEL == 2 ? 3 : 1) * NW);
+    uint8_t* s_num = s_first + kL1Bins;
+    uint32_t* s_prefix = reinterpret_cast<uint32_t*>(s_num + kL1Bins);
+    __shared__ int s_flag;
+    const uint32_t w = blockIdx.y;
+    const uint32_t c0 = blockIdx.x * kRunChunks, c1 = min(n_chunks, c0 + kRunChunks);
+    for (int i = threadIdx.x; i < (LEVEL == 2 ? 3 : 1) * NW; i += kHThreads) sh[i] = 0;
+    if (threadIdx.x == 0) s_flag = 0;
+    const float* dd = dbuf + (size_t)w * dstride;
+    int cur_layer = -1;
+    uint32_t ns = 0;
+    bool active = false, dirty = false;
+    uint32_t* gc = nullptr;
+    unsigned long long* gs = nullptr;
+
+    auto flush = [&]() {
+        __syncthreads();
+        for (uint32_t i = threadIdx.x; i < ns * kL23Bins; i += kHThreads) {
+            const uint32_t c = h_cnt[i];
+            if (c) {
+                atomicAdd(&gc[i], c);
+                h_cnt[i] = 0;
+                if (LEVEL == 2) {
+                    atomicAdd(&gs[i], ((unsigned long long)h_hi[i] << 16) + h_lo[i]);
+                    h_hi[i] = 0;
+                    h_lo[i] = 0;
+                }
+            }
+        }
+        if (threadIdx.x == 0) s_flag = 0;
+        __syncthreads();
+        dirty = false;
+    };
+
+    for (uint32_t c = c0; c < c1; ++c) {
+        const Chunk ch = chunks[c];
+        if ((int)ch.layer != cur_layer) {
+            if (dirty) flush();
+            cur_layer = (int)ch.layer;
+            const size_t wl = (size_t)w * L + ch.layer;
+            const SlotTab& stab = slots[wl];
+            ns = stab.n;
+            active = ns <= (uint32_t)kSmemSlots;
+            gc = g_cnt + wl * K * kL23Bins;
+            gs = g_ss + wl * K * kL23Bins;
+            if (active) {
+                __syncthreads();
+                for (int b = threadIdx.x; b < kL1Bins; b += kHThreads) { s_first[b] = 0xff; s_num[b] = 0; }
+                if (threadIdx.x < ns) s_prefix[threadIdx.x] = stab.prefix[threadIdx.x];
+                __syncthreads();
+                if (threadIdx.x == 0)
+                    for (uint32_t s = 0; s < ns; ++s) {
+                        const uint32_t b1 = LEVEL == 2 ? s_prefix[s] : (s_prefix[s] >> 10);
+                        if (s_first[b1] == 0xff) s_first[b1] = (uint8_t)s;
+                        s_num[b1]++;
+                    }
+                __syncthreads();
+            }
+        }
+        if (!active) continue;
+        const bool direct = ch.end - ch.begin <= kDirectElems;
+        auto visit = [&](float dv) {
+            const uint32_t key = key_of(dv);
+            const uint32_t f = s_first[key >> 20];
+            if (f == 0xff) return;
+            if (LEVEL == 2) {
+                const uint32_t i = f * kL23Bins + ((key >> 10) & 1023u);
+                const uint32_t sq = (uint32_t)sq_fixed(key);
+                if (direct) {
+                    atomicAdd(&gc[i], 1u);
+                    atomicAdd(&gs[i], (unsigned long long)sq);
+                } else {
+                    const uint32_t old = atomicAdd(&h_cnt[i], 1u);
+                    atomicAdd(&h_hi[i], sq >> 16);
+                    atomicAdd(&h_lo[i], sq & 0xffffu);
+                    if (old >= 32768u) s_flag = 1; // flush at the next chunk boundary, before any sum can overflow
+                }
+            } else {
+                const uint32_t n = s_num[key >> 20];
+                const uint32_t p21 = key >> 10;
+                for (uint32_t s = f; s < f + n; ++s)
+                    if (s_prefix[s] == p21) {
+                        const uint32_t i = s * kL23Bins + (key & 1023u);
+                        if (direct) atomicAdd(&gc[i], 1u); else atomicAdd(&h_cnt[i], 1u);
+                        break;
+                    }
+            }
+        };
+        const uint64_t q0 = ch.begin & ~3ull;
+        constexpr int U = 2;
+        for (uint64_t base = q0; base < ch.end; base += (uint64_t)4 * kHThreads * U) {
+            float4 a[U];
+            bool full[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const uint64_t q = base + 4ull * (threadIdx.x + (uint64_t)u * kHThreads);
+                full[u] = q >= ch.begin && q + 4 <= ch.end;
+                if (full[u]) a[u] = __ldcs(reinterpret_cast<const float4*>(dd + q));
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const uint64_t q = base + 4ull * (threadIdx.x + (uint64_t)u * kHThreads);
+                if (full[u]) {
+                    visit(a[u].x); visit(a[u].y); visit(a[u].z); visit(a[u].w);
+                } else if (q < ch.end) {
+                    for (int i = 0; i < 4; ++i) {
+                        const uint64_t p = q + i;
+                        if (p >= ch.begin && p < ch.end) visit(dd[p]);
+                    }
+                }
+            }
+        }
+        if (!direct) {
+            dirty = true;
+            __syncthreads();
+            if (s_flag) flush();
+        }
+    }
+    if (dirty) flush();
+}
+
 // ------------------------------------------------------------------------------------------------
 // (c) knapsack DP over the budget axis, one CTA per worker
 // ------------------------------------------------------------------------------------------------
 struct DpBudgets { uint64_t c[kDpWorkersPerLaunch]; };
 
-constexpr int kDpThreads = 1024;
+constexpr int kDpThreads = 512;
+
+// Shared-memory plan of k_dp (host computes the same sizes):
+//   prev[D+1], cur[D+1] f32 | j[L] u32 | units[L*K] u32, err[L*K] f32 (if tab_in_smem) | PD
+// PD holds the winning candidate of every (layer, cell): a nibble when K <= 16, else a byte; it lives
+// in shared memory when it fits, else in the caller's workspace.
+struct DpPlan {
+    uint32_t tab_in_smem; // candidate tables preloaded for all layers (else one layer at a time)
+    uint32_t pd_in_smem;
+    uint32_t pd_nibble;
+    uint32_t pd_row_bytes;
+};
 
 // mode 0: DP; mode 1: candidates given (j_in)
 __global__ void __launch_bounds__(kDpThreads)
 k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uint32_t D, uint32_t bpe,
-     uint64_t full_bytes, uint64_t cap, uint32_t check_finite, int mode, const uint64_t* __restrict__ ktab,
-     const float* __restrict__ err, const uint32_t* __restrict__ tau, const uint32_t* __restrict__ keep_eq,
-     const uint32_t* __restrict__ j_in, uint32_t* __restrict__ flags, uint8_t* __restrict__ pd_global,
-     int pd_in_smem, Sel* __restrict__ sel, uint32_t* __restrict__ out_k, uint32_t* __restrict__ out_j,
-     uint64_t* __restrict__ out_offs, kimad_stats* __restrict__ out_stats) {
+     uint64_t full_bytes, uint64_t cap, uint32_t check_finite, int mode, DpPlan plan,
+     const uint64_t* __restrict__ ktab, const float* __restrict__ err, const uint32_t* __restrict__ tau,
+     const uint32_t* __restrict__ keep_eq, const uint32_t* __restrict__ j_in, uint32_t* __restrict__ flags,
+     uint8_t* __restrict__ pd_global, Sel* __restrict__ sel, uint32_t* __restrict__ out_k,
+     uint32_t* __restrict__ out_j, uint64_t* __restrict__ out_offs, kimad_stats* __restrict__ out_stats) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const uint32_t w = w_base + blockIdx.x;
     if (w >= W) return;
     const uint64_t c = budgets.c[blockIdx.x];
     const uint32_t row = D + 1;
+    const float kInf = __int_as_float(0x7f800000);
     float* prev = reinterpret_cast<float*>(smem_raw);
     float* cur = prev + row;
-    uint32_t* s_units = reinterpret_cast<uint32_t*>(cur + row);
-    float* s_err = reinterpret_cast<float*>(s_units + K);
-    uint32_t* s_j = reinterpret_cast<uint32_t*>(s_err + K); // [L]
-    uint8_t* pd = pd_in_smem ? reinterpret_cast<uint8_t*>(s_j + L) : pd_global + (size_t)w * L * row;
+    uint32_t* s_j = reinterpret_cast<uint32_t*>(cur + row); // [L]
+    uint32_t* s_units = s_j + L;                             // [L*K] or [K]
+    const uint32_t ntab = plan.tab_in_smem ? L * K : K;
+    float* s_err = reinterpret_cast<float*>(s_units + ntab);
+    uint8_t* pd = plan.pd_in_smem ? reinterpret_cast<uint8_t*>(s_err + ntab)
+                                  : pd_global + (size_t)w * L * plan.pd_row_bytes;
     __shared__ float s_redv[32];
     __shared__ uint32_t s_redb[32];
     __shared__ int s_status;
@@ -413,34 +592,56 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
             status = KIMAD_STATUS_INFEASIBLE;
             for (uint32_t l = threadIdx.x; l < L; l += blockDim.x) s_j[l] = 0;
         } else {
-            for (uint32_t b = threadIdx.x; b < row; b += blockDim.x) prev[b] = b ? __int_as_float(0x7f800000) : 0.f;
+            auto load_tab = [&](uint32_t src, uint32_t dst) { // candidate src of the [L][K] tables -> smem slot dst
+                const uint64_t u = budget_cells(ktab[src] * bpe, D, c);
+                s_units[dst] = u > D ? 0xffffffffu : (uint32_t)u;
+                s_err[dst] = e_w[src];
+            };
+            if (plan.tab_in_smem)
+                for (uint32_t i = threadIdx.x; i < L * K; i += blockDim.x) load_tab(i, i);
+            for (uint32_t b = threadIdx.x; b < row; b += blockDim.x) prev[b] = b ? kInf : 0.f;
             for (uint32_t l = 0; l < L; ++l) {
                 __syncthreads();
-                if (threadIdx.x < K) {
-                    const uint64_t bytes = ktab[(size_t)l * K + threadIdx.x] * bpe;
-                    const uint64_t u = budget_cells(bytes, D, c);
-                    s_units[threadIdx.x] = u > D ? 0xffffffffu : (uint32_t)u;
-                    s_err[threadIdx.x] = e_w[(size_t)l * K + threadIdx.x];
+                if (!plan.tab_in_smem) {
+                    if (threadIdx.x < K) load_tab(l * K + threadIdx.x, threadIdx.x);
+                    __syncthreads();
                 }
-                __syncthreads();
-                for (uint32_t b = threadIdx.x; b < row; b += blockDim.x) {
-                    float best = __int_as_float(0x7f800000);
-                    uint32_t bj = 0;
+                const uint32_t* un = s_units + (plan.tab_in_smem ? l * K : 0);
+                const float* er = s_err + (plan.tab_in_smem ? l * K : 0);
+                uint8_t* pdl = pd + (size_t)l * plan.pd_row_bytes;
+                // each thread owns the cell pair (2t, 2t+1): one PD byte holds both nibbles
+                for (uint32_t b0 = 2 * threadIdx.x; b0 < row; b0 += 2 * blockDim.x) {
+                    float best0 = kInf, best1 = kInf;
+                    uint32_t bj0 = 0, bj1 = 0;
+                    const uint32_t b1 = b0 + 1;
+#pragma unroll 4
                     for (uint32_t j = 0; j < K; ++j) {
-                        const uint32_t u = s_units[j];
-                        if (u <= b) {
-                            const float t = __fadd_rn(prev[b - u], s_err[j]);
-                            if (t < best) { best = t; bj = j; }
+                        const uint32_t u = un[j];
+                        if (u > b1) continue; // covers the "unusable" marker 0xffffffff too
+                        const float e = er[j];
+                        if (u <= b0) {
+                            const float t = __fadd_rn(prev[b0 - u], e);
+                            if (t < best0) { best0 = t; bj0 = j; }
+                        }
+                        if (b1 < row) {
+                            const float t = __fadd_rn(prev[b1 - u], e);
+                            if (t < best1) { best1 = t; bj1 = j; }
                         }
                     }
-                    cur[b] = best;
-                    pd[(size_t)l * row + b] = (uint8_t)bj;
+                    cur[b0] = best0;
+                    if (b1 < row) cur[b1] = best1;
+                    if (plan.pd_nibble) {
+                        pdl[b0 >> 1] = (uint8_t)(bj0 | (bj1 << 4));
+                    } else {
+                        pdl[b0] = (uint8_t)bj0;
+                        if (b1 < row) pdl[b1] = (uint8_t)bj1;
+                    }
                 }
                 float* sw = prev; prev = cur; cur = sw;
             }
             __syncthreads();
             // lowest cell attaining the minimum: lexicographic (value, cell) min-reduction
-            float bv = __int_as_float(0x7f800000);
+            float bv = kInf;
             uint32_t bb = 0xffffffffu;
             for (uint32_t b = threadIdx.x; b < row; b += blockDim.x) {
                 const float v = prev[b];
@@ -460,16 +661,17 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
                     const uint32_t ob = s_redb[i];
                     if (ov < bv || (ov == bv && ob < bb)) { bv = ov; bb = ob; }
                 }
-                if (!(bv < __int_as_float(0x7f800000))) {
+                if (!(bv < kInf)) {
                     s_status = KIMAD_STATUS_INFEASIBLE;
                 } else {
                     s_status = KIMAD_OK;
                     uint32_t b = bb;
                     for (uint32_t l = L; l-- > 0;) { // walk the back-pointers
-                        const uint32_t j = pd[(size_t)l * row + b];
+                        const uint8_t* pdl = pd + (size_t)l * plan.pd_row_bytes;
+                        const uint32_t j = plan.pd_nibble ? ((pdl[b >> 1] >> (4 * (b & 1))) & 15u) : pdl[b];
                         s_j[l] = j;
-                        const uint64_t bytes = ktab[(size_t)l * K + j] * bpe;
-                        b -= (uint32_t)budget_cells(bytes, D, c);
+                        b -= plan.tab_in_smem ? s_units[l * K + j]
+                                              : (uint32_t)budget_cells(ktab[(size_t)l * K + j] * bpe, D, c);
                     }
                 }
             }
@@ -481,14 +683,23 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
     }
     __syncthreads();
 
-    // totals, capacity check and outputs
+    // totals, capacity check and outputs (prev/cur are free now: stage k_l and err_l there)
+    uint32_t* s_k = reinterpret_cast<uint32_t*>(smem_raw);
+    float* s_e = reinterpret_cast<float*>(smem_raw) + row;
+    const bool staged = L <= row;
+    if (staged && status >= 0)
+        for (uint32_t l = threadIdx.x; l < L; l += blockDim.x) {
+            s_k[l] = (uint32_t)ktab[(size_t)l * K + s_j[l]];
+            s_e[l] = e_w[(size_t)l * K + s_j[l]];
+        }
+    __syncthreads();
     if (threadIdx.x == 0) {
         uint64_t nsel = 0;
         float tot = 0.f;
         if (status >= 0)
             for (uint32_t l = 0; l < L; ++l) {
-                nsel += ktab[(size_t)l * K + s_j[l]];
-                tot = __fadd_rn(tot, e_w[(size_t)l * K + s_j[l]]);
+                nsel += staged ? s_k[l] : ktab[(size_t)l * K + s_j[l]];
+                tot = __fadd_rn(tot, staged ? s_e[l] : e_w[(size_t)l * K + s_j[l]]);
             }
         if (status >= 0 && nsel > cap) status = KIMAD_ERR_CAPACITY;
         kimad_stats s;
@@ -501,7 +712,7 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
         uint64_t run = 0;
         for (uint32_t l = 0; l < L; ++l) {
             out_offs[(size_t)w * (L + 1) + l] = run;
-            if (status >= 0) run += ktab[(size_t)l * K + s_j[l]];
+            if (status >= 0) run += staged ? s_k[l] : ktab[(size_t)l * K + s_j[l]];
         }
         out_offs[(size_t)w * (L + 1) + L] = run;
         s_status = status;
@@ -526,6 +737,7 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
             out_k[wl] = 0;
             out_j[wl] = 0;
         }
+        s._pad = 0;
         sel[wl] = s;
     }
 }
@@ -533,7 +745,6 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
 // ------------------------------------------------------------------------------------------------
 // (d) per-chunk counts at the chosen threshold, then an exclusive scan over each layer's chunks
 // ------------------------------------------------------------------------------------------------
-template <bool VEC>
 __global__ void __launch_bounds__(kThreads)
 k_select_count(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks, uint64_t dstride,
                uint32_t L, const Sel* __restrict__ sel, const LayerDesc* __restrict__ layers,
@@ -563,7 +774,7 @@ k_select_count(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks,
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const uint64_t q = base + 4ull * (threadIdx.x + (uint64_t)u * kThreads);
-            full[u] = VEC && q >= ch.begin && q + 4 <= ch.end;
+            full[u] = q >= ch.begin && q + 4 <= ch.end;
             if (full[u]) a[u] = __ldg(reinterpret_cast<const float4*>(dd + q));
         }
 #pragma unroll
@@ -585,12 +796,14 @@ k_select_count(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks,
     if (threadIdx.x == 0) *out = make_uint2(tg, te);
 }
 
-// in place: chunk_cnt[(w, chunk)] becomes the exclusive prefix (gt, eq) over the layer's earlier chunks
+// chunk_pre[(w, chunk)] = exclusive prefix (gt, eq) over the layer's earlier chunks
 __global__ void __launch_bounds__(kThreads)
-k_select_scan(const LayerDesc* __restrict__ layers, uint32_t n_chunks, uint2* __restrict__ chunk_cnt) {
+k_select_scan(const LayerDesc* __restrict__ layers, uint32_t n_chunks, const uint2* __restrict__ chunk_cnt,
+              uint2* __restrict__ chunk_pre) {
     __shared__ uint32_t s_w[8];
     const LayerDesc ld = layers[blockIdx.x];
-    uint2* cc = chunk_cnt + (size_t)blockIdx.y * n_chunks + ld.first_chunk;
+    const uint2* cc = chunk_cnt + (size_t)blockIdx.y * n_chunks + ld.first_chunk;
+    uint2* cp = chunk_pre + (size_t)blockIdx.y * n_chunks + ld.first_chunk;
     uint32_t run_g = 0, run_e = 0;
     for (uint32_t base = 0; base < ld.n_chunks; base += kThreads) {
         const uint32_t i = base + threadIdx.x;
@@ -598,21 +811,23 @@ k_select_scan(const LayerDesc* __restrict__ layers, uint32_t n_chunks, uint2* __
         uint32_t tg, te;
         const uint32_t eg = block_excl_scan<uint32_t>(v.x, s_w, &tg);
         const uint32_t ee = block_excl_scan<uint32_t>(v.y, s_w, &te);
-        if (i < ld.n_chunks) cc[i] = make_uint2(run_g + eg, run_e + ee);
+        if (i < ld.n_chunks) cp[i] = make_uint2(run_g + eg, run_e + ee);
         run_g += tg;
         run_e += te;
     }
 }
 
 // ------------------------------------------------------------------------------------------------
-// (e) + (f) ordered compaction and EF21 update
+// (e) + (f) ordered compaction and EF21 update.  Every thread owns 16 consecutive elements of a
+// 4096-element round, so that ranks inside a round follow the index order.
 // ------------------------------------------------------------------------------------------------
 template <bool BF16>
 __global__ void __launch_bounds__(kThreads)
 k_select_write(const float* __restrict__ dbuf, float* __restrict__ state, const Chunk* __restrict__ chunks,
                uint32_t n_chunks, uint64_t dstride, uint64_t stride, uint32_t L, const Sel* __restrict__ sel,
-               const LayerDesc* __restrict__ layers, const uint2* __restrict__ chunk_pre, uint64_t cap,
-               uint32_t* __restrict__ out_idx, void* __restrict__ out_val) {
+               const LayerDesc* __restrict__ layers, const uint2* __restrict__ chunk_cnt,
+               const uint2* __restrict__ chunk_pre, uint64_t cap, uint32_t* __restrict__ out_idx,
+               void* __restrict__ out_val) {
     __shared__ uint32_t s_w[8];
     const Chunk ch = chunks[blockIdx.x];
     const uint32_t w = blockIdx.y;
@@ -620,8 +835,12 @@ k_select_write(const float* __restrict__ dbuf, float* __restrict__ state, const 
     if (s.k == 0) return;
     const LayerDesc ld = layers[ch.layer];
     const bool all = (uint64_t)s.k == ld.n;
+    const uint2 cnt = chunk_cnt[(size_t)w * n_chunks + blockIdx.x];
     const uint2 pre = chunk_pre[(size_t)w * n_chunks + blockIdx.x];
+    if (!all && cnt.x == 0 && (cnt.y == 0 || pre.y >= s.keep_eq)) return; // nothing kept in this chunk
     // entries equal to tau are kept while their rank among equals (ascending index) is below keep_eq
+    // eq_mode 0: none of this chunk's equals is kept; 1: all are; 2: ranks must be counted
+    const int eq_mode = (all || cnt.y == 0 || pre.y >= s.keep_eq) ? 0 : (pre.y + cnt.y <= s.keep_eq ? 1 : 2);
     uint32_t eq_seen = pre.y;
     uint64_t pos = s.base + pre.x + min(pre.y, s.keep_eq);
     const float* dd = dbuf + (size_t)w * dstride;
@@ -630,58 +849,76 @@ k_select_write(const float* __restrict__ dbuf, float* __restrict__ state, const 
     float* ov32 = reinterpret_cast<float*>(out_val) + (size_t)w * cap;
     __nv_bfloat16* ov16 = reinterpret_cast<__nv_bfloat16*>(out_val) + (size_t)w * cap;
 
+    constexpr int E = 16; // elements per thread per round
     const uint64_t q0 = ch.begin & ~3ull;
-    for (uint64_t base = q0; base < ch.end; base += 4ull * kThreads) {
-        const uint64_t q = base + 4ull * threadIdx.x;
-        float v[4];
-        bool in[4], isgt[4], iseq[4];
-        uint32_t ngt = 0, neq = 0;
+    auto load_round = [&](uint64_t base, float* v) {
+        const uint64_t t0 = base + (uint64_t)E * threadIdx.x;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const uint64_t p = q + i;
-            in[i] = p >= ch.begin && p < ch.end;
-            v[i] = in[i] ? dd[p] : 0.f;
-            const uint32_t key = key_of(v[i]);
-            isgt[i] = in[i] && (all || key > s.tau);
-            iseq[i] = in[i] && !all && key == s.tau;
-            ngt += isgt[i];
-            neq += iseq[i];
-        }
-        uint32_t tot_eq;
-        uint32_t eq_rank = eq_seen + block_excl_scan<uint32_t>(neq, s_w, &tot_eq);
-        uint32_t nkeep = ngt;
-        bool keep[4];
+        for (int u = 0; u < E / 4; ++u) {
+            const uint64_t q = t0 + 4 * u;
+            if (q >= ch.begin && q + 4 <= ch.end) {
+                const float4 a = __ldg(reinterpret_cast<const float4*>(dd + q));
+                v[4 * u] = a.x; v[4 * u + 1] = a.y; v[4 * u + 2] = a.z; v[4 * u + 3] = a.w;
+            } else {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            keep[i] = isgt[i];
-            if (iseq[i]) {
-                keep[i] = eq_rank < s.keep_eq;
-                nkeep += keep[i];
-                ++eq_rank;
-            }
-        }
-        uint32_t tot_keep;
-        uint64_t o = pos + block_excl_scan<uint32_t>(nkeep, s_w, &tot_keep);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            if (keep[i]) {
-                const uint64_t p = q + i;
-                oi[o] = (uint32_t)(p - ld.begin);
-                float sent;
-                if (BF16) {
-                    const __nv_bfloat16 h = __float2bfloat16_rn(v[i]);
-                    ov16[o] = h;
-                    sent = __bfloat162float(h);
-                } else {
-                    ov32[o] = v[i];
-                    sent = v[i];
+                for (int i = 0; i < 4; ++i) {
+                    const uint64_t p = q + i;
+                    v[4 * u + i] = (p >= ch.begin && p < ch.end) ? dd[p] : 0.f;
                 }
-                st[p] = __fadd_rn(st[p], sent);
-                ++o;
             }
         }
-        eq_seen += tot_eq;
-        pos += tot_keep;
+    };
+    float v[E], nxt[E];
+    load_round(q0, v);
+    for (uint64_t base = q0; base < ch.end; base += (uint64_t)E * kThreads) {
+        const uint64_t t0 = base + (uint64_t)E * threadIdx.x;
+        const uint64_t nbase = base + (uint64_t)E * kThreads;
+        if (nbase < ch.end) load_round(nbase, nxt); // in flight while this round is compacted
+        uint32_t keepm = 0, eqm = 0;
+#pragma unroll
+        for (int i = 0; i < E; ++i) {
+            const uint64_t p = t0 + i;
+            const bool in = p >= ch.begin && p < ch.end;
+            const uint32_t key = key_of(v[i]);
+            if (in && (all || key > s.tau || (eq_mode == 1 && key == s.tau))) keepm |= 1u << i;
+            if (in && eq_mode == 2 && key == s.tau) eqm |= 1u << i;
+        }
+        if (__syncthreads_or((keepm | eqm) != 0)) {
+            if (eq_mode == 2) { // uniform over the CTA
+                uint32_t tot_eq;
+                uint32_t eq_rank = eq_seen + block_excl_scan<uint32_t>(__popc(eqm), s_w, &tot_eq);
+#pragma unroll
+                for (int i = 0; i < E; ++i)
+                    if (eqm & (1u << i)) {
+                        if (eq_rank < s.keep_eq) keepm |= 1u << i;
+                        ++eq_rank;
+                    }
+                eq_seen += tot_eq;
+            }
+            uint32_t tot_keep;
+            uint64_t o = pos + block_excl_scan<uint32_t>(__popc(keepm), s_w, &tot_keep);
+#pragma unroll
+            for (int i = 0; i < E; ++i) {
+                if (keepm & (1u << i)) {
+                    const uint64_t p = t0 + i;
+                    oi[o] = (uint32_t)(p - ld.begin);
+                    float sent;
+                    if (BF16) {
+                        const __nv_bfloat16 h = __float2bfloat16_rn(v[i]);
+                        ov16[o] = h;
+                        sent = __bfloat162float(h);
+                    } else {
+                        ov32[o] = v[i];
+                        sent = v[i];
+                    }
+                    st[p] = __fadd_rn(st[p], sent);
+                    ++o;
+                }
+            }
+            pos += tot_keep;
+        }
+#pragma unroll
+        for (int i = 0; i < E; ++i) v[i] = nxt[i];
     }
 }
 
