@@ -7,7 +7,7 @@
 #include <new>
 #include <vector>
 
-#include "kimad_kernels.cuh"
+#include "kimad_select.cuh"
 
 using namespace kimad;
 
@@ -18,7 +18,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
     size_t dbuf, chunks, layers, ktab, h1_cnt, h1_ss, h23_cnt, h23_ss, cands, slots, err, tau, keep_eq, sel, chunk_cnt,
-        chunk_pre, flags, pd, total;
+        chunk_pre, csel, low_hist, recount, flags, pd, total;
 };
 
 } // namespace
@@ -68,6 +68,9 @@ void plan_layout(kimad_ctx* c) {
     y.sel = take(WL * sizeof(Sel));
     y.chunk_cnt = take((size_t)c->W * c->chunks.size() * sizeof(uint2));
     y.chunk_pre = take((size_t)c->W * c->chunks.size() * sizeof(uint2));
+    y.csel = take((size_t)c->W * c->chunks.size() * sizeof(ChunkSel));
+    y.low_hist = take(WL * kLowBins * sizeof(uint32_t));
+    y.recount = take(256 + (size_t)c->W * c->chunks.size() * sizeof(uint2));
     y.flags = take((size_t)c->W * sizeof(uint32_t));
     y.pd = take(c->dp_plan.pd_in_smem ? 0 : (size_t)c->W * c->L * c->dp_plan.pd_row_bytes);
     y.total = o;
@@ -110,6 +113,10 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
     Sel* sel = c->at<Sel>(c->lay.sel);
     uint2* ccnt = c->at<uint2>(c->lay.chunk_cnt);
     uint2* cpre = c->at<uint2>(c->lay.chunk_pre);
+    ChunkSel* csel = c->at<ChunkSel>(c->lay.csel);
+    uint32_t* lowh = c->at<uint32_t>(c->lay.low_hist);
+    uint32_t* recount_n = c->at<uint32_t>(c->lay.recount);
+    uint2* recount_list = c->at<uint2>(c->lay.recount + 256);
     uint32_t* flags = c->at<uint32_t>(c->lay.flags);
     uint8_t* pd = c->at<uint8_t>(c->lay.pd);
 
@@ -159,24 +166,27 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
         }
         k_dp<<<nw, kDpThreads, c->dp_smem, s>>>(b, w0, W, L, K, c->D, c->bpe, c->full_bytes, c->cap, c->check_finite,
                                                 mode == kGivenJ ? 1 : 0, c->dp_plan, ktab,
-                                                mode == kInjectErr ? err_dev : err, tau, keq, j_dev, flags, pd, sel,
+                                                mode == kInjectErr ? err_dev : err, tau, keq, nullptr, j_dev, flags, pd,
+                                                sel,
                                                 out->k, out->j, out->offs, out->stats);
         c->launches += 1;
     }
     mark();
     // (d), (e), (f)
-    k_select_count<<<gch, blk, 0, s>>>(dbuf, chunks, nch, c->dstride, L, sel, layers, ccnt);
+    k_sel_count<<<gch, blk, 0, s>>>(dbuf, chunks, nch, c->dstride, L, sel, layers, csel, lowh, recount_n, recount_list);
     mark();
-    k_select_scan<<<glw, blk, 0, s>>>(layers, nch, ccnt, cpre);
+    k_sel_resolve<<<glw, blk, 0, s>>>(L, layers, lowh, sel);
+    k_sel_recount<<<2 * 148, blk, 0, s>>>(dbuf, chunks, nch, c->dstride, L, sel, recount_n, recount_list, ccnt);
+    k_sel_scan<<<glw, blk, 0, s>>>(L, layers, nch, sel, csel, ccnt, cpre, recount_n);
     mark();
     if (c->value_dtype == 1)
-        k_select_write<true><<<gch, blk, 0, s>>>(dbuf, state, chunks, nch, c->dstride, c->stride, L, sel, layers, ccnt,
-                                                 cpre, c->cap, out->idx, out->val);
+        k_sel_write<true><<<gch, blk, 0, s>>>(dbuf, state, chunks, nch, c->dstride, c->stride, L, sel, layers, ccnt, cpre,
+                                              c->cap, out->idx, out->val);
     else
-        k_select_write<false><<<gch, blk, 0, s>>>(dbuf, state, chunks, nch, c->dstride, c->stride, L, sel, layers, ccnt,
-                                                  cpre, c->cap, out->idx, out->val);
+        k_sel_write<false><<<gch, blk, 0, s>>>(dbuf, state, chunks, nch, c->dstride, c->stride, L, sel, layers, ccnt, cpre,
+                                               c->cap, out->idx, out->val);
     mark();
-    c->launches += 3;
+    c->launches += 5;
     CUDA_TRY(cudaGetLastError());
     c->last_out = *out;
     c->have_last = true;

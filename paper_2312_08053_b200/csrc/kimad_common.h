@@ -45,11 +45,15 @@ struct SlotTab {
     uint32_t prefix[KIMAD_MAX_RATIOS];
 };
 
-// What the select kernels need to know about one (worker, layer) after the DP.
+// What the select kernels need to know about one (worker, layer) after the DP.  The threshold lies in
+// the key interval [tau, tau + 2^shift) and is the keep_eq-th largest key inside it; k_sel_resolve
+// narrows that to the exact threshold (shift = 0) and to the number of ties kept.
 struct Sel {
-    uint32_t tau;     // threshold key
-    uint32_t keep_eq; // entries equal to tau that are kept (lowest indices first)
+    uint32_t tau;     // lower key of the interval, then the exact threshold key
+    uint32_t keep_eq; // rank inside the interval, then: entries equal to tau that are kept (lowest indices first)
     uint32_t k;       // 0: nothing to pack for this layer (the worker failed)
+    uint32_t shift;   // log2 of the interval width (<= 10)
+    uint32_t tau_low; // exact threshold minus the interval's lower key
     uint32_t _pad;
     uint64_t base;    // first output position of the layer in the worker's packed buffers
 };

@@ -556,7 +556,8 @@ __global__ void __launch_bounds__(kDpThreads)
 k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uint32_t D, uint32_t bpe,
      uint64_t full_bytes, uint64_t cap, uint32_t check_finite, int mode, DpPlan plan,
      const uint64_t* __restrict__ ktab, const float* __restrict__ err, const uint32_t* __restrict__ tau,
-     const uint32_t* __restrict__ keep_eq, const uint32_t* __restrict__ j_in, uint32_t* __restrict__ flags,
+     const uint32_t* __restrict__ keep_eq, const uint32_t* __restrict__ shift /* may be null: all exact */,
+     const uint32_t* __restrict__ j_in, uint32_t* __restrict__ flags,
      uint8_t* __restrict__ pd_global, Sel* __restrict__ sel, uint32_t* __restrict__ out_k,
      uint32_t* __restrict__ out_j, uint64_t* __restrict__ out_offs, kimad_stats* __restrict__ out_stats) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -729,196 +730,18 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
             s.tau = tau[wl * K + j];
             s.keep_eq = keep_eq[wl * K + j];
             s.k = (uint32_t)k;
+            s.shift = shift ? shift[wl * K + j] : 0u;
             s.base = out_offs[(size_t)w * (L + 1) + l];
             out_k[wl] = (uint32_t)k;
             out_j[wl] = j;
         } else {
-            s.tau = 0; s.keep_eq = 0; s.k = 0; s.base = 0;
+            s.tau = 0; s.keep_eq = 0; s.k = 0; s.shift = 0; s.base = 0;
             out_k[wl] = 0;
             out_j[wl] = 0;
         }
+        s.tau_low = 0;
         s._pad = 0;
         sel[wl] = s;
-    }
-}
-
-// ------------------------------------------------------------------------------------------------
-// (d) per-chunk counts at the chosen threshold, then an exclusive scan over each layer's chunks
-// ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kThreads)
-k_select_count(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks, uint64_t dstride,
-               uint32_t L, const Sel* __restrict__ sel, const LayerDesc* __restrict__ layers,
-               uint2* __restrict__ chunk_cnt) {
-    __shared__ uint32_t s_w[8];
-    const Chunk ch = chunks[blockIdx.x];
-    const uint32_t w = blockIdx.y;
-    const Sel s = sel[(size_t)w * L + ch.layer];
-    uint2* out = chunk_cnt + (size_t)w * n_chunks + blockIdx.x;
-    if (s.k == 0) { if (threadIdx.x == 0) *out = make_uint2(0, 0); return; }
-    if ((uint64_t)s.k == layers[ch.layer].n) { // everything kept: no need to look at the data
-        if (threadIdx.x == 0) *out = make_uint2((uint32_t)(ch.end - ch.begin), 0);
-        return;
-    }
-    const float* dd = dbuf + (size_t)w * dstride;
-    uint32_t gt = 0, eq = 0;
-    auto visit = [&](float dv) {
-        const uint32_t key = key_of(dv);
-        gt += key > s.tau;
-        eq += key == s.tau;
-    };
-    const uint64_t q0 = ch.begin & ~3ull;
-    constexpr int U = 4;
-    for (uint64_t base = q0; base < ch.end; base += (uint64_t)4 * kThreads * U) {
-        float4 a[U];
-        bool full[U];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const uint64_t q = base + 4ull * (threadIdx.x + (uint64_t)u * kThreads);
-            full[u] = q >= ch.begin && q + 4 <= ch.end;
-            if (full[u]) a[u] = __ldg(reinterpret_cast<const float4*>(dd + q));
-        }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const uint64_t q = base + 4ull * (threadIdx.x + (uint64_t)u * kThreads);
-            if (full[u]) {
-                visit(a[u].x); visit(a[u].y); visit(a[u].z); visit(a[u].w);
-            } else if (q < ch.end) {
-                for (int i = 0; i < 4; ++i) {
-                    const uint64_t p = q + i;
-                    if (p >= ch.begin && p < ch.end) visit(dd[p]);
-                }
-            }
-        }
-    }
-    uint32_t tg, te;
-    block_excl_scan<uint32_t>(gt, s_w, &tg);
-    block_excl_scan<uint32_t>(eq, s_w, &te);
-    if (threadIdx.x == 0) *out = make_uint2(tg, te);
-}
-
-// chunk_pre[(w, chunk)] = exclusive prefix (gt, eq) over the layer's earlier chunks
-__global__ void __launch_bounds__(kThreads)
-k_select_scan(const LayerDesc* __restrict__ layers, uint32_t n_chunks, const uint2* __restrict__ chunk_cnt,
-              uint2* __restrict__ chunk_pre) {
-    __shared__ uint32_t s_w[8];
-    const LayerDesc ld = layers[blockIdx.x];
-    const uint2* cc = chunk_cnt + (size_t)blockIdx.y * n_chunks + ld.first_chunk;
-    uint2* cp = chunk_pre + (size_t)blockIdx.y * n_chunks + ld.first_chunk;
-    uint32_t run_g = 0, run_e = 0;
-    for (uint32_t base = 0; base < ld.n_chunks; base += kThreads) {
-        const uint32_t i = base + threadIdx.x;
-        uint2 v = i < ld.n_chunks ? cc[i] : make_uint2(0, 0);
-        uint32_t tg, te;
-        const uint32_t eg = block_excl_scan<uint32_t>(v.x, s_w, &tg);
-        const uint32_t ee = block_excl_scan<uint32_t>(v.y, s_w, &te);
-        if (i < ld.n_chunks) cp[i] = make_uint2(run_g + eg, run_e + ee);
-        run_g += tg;
-        run_e += te;
-    }
-}
-
-// ------------------------------------------------------------------------------------------------
-// (e) + (f) ordered compaction and EF21 update.  Every thread owns 16 consecutive elements of a
-// 4096-element round, so that ranks inside a round follow the index order.
-// ------------------------------------------------------------------------------------------------
-template <bool BF16>
-__global__ void __launch_bounds__(kThreads)
-k_select_write(const float* __restrict__ dbuf, float* __restrict__ state, const Chunk* __restrict__ chunks,
-               uint32_t n_chunks, uint64_t dstride, uint64_t stride, uint32_t L, const Sel* __restrict__ sel,
-               const LayerDesc* __restrict__ layers, const uint2* __restrict__ chunk_cnt,
-               const uint2* __restrict__ chunk_pre, uint64_t cap, uint32_t* __restrict__ out_idx,
-               void* __restrict__ out_val) {
-    __shared__ uint32_t s_w[8];
-    const Chunk ch = chunks[blockIdx.x];
-    const uint32_t w = blockIdx.y;
-    const Sel s = sel[(size_t)w * L + ch.layer];
-    if (s.k == 0) return;
-    const LayerDesc ld = layers[ch.layer];
-    const bool all = (uint64_t)s.k == ld.n;
-    const uint2 cnt = chunk_cnt[(size_t)w * n_chunks + blockIdx.x];
-    const uint2 pre = chunk_pre[(size_t)w * n_chunks + blockIdx.x];
-    if (!all && cnt.x == 0 && (cnt.y == 0 || pre.y >= s.keep_eq)) return; // nothing kept in this chunk
-    // entries equal to tau are kept while their rank among equals (ascending index) is below keep_eq
-    // eq_mode 0: none of this chunk's equals is kept; 1: all are; 2: ranks must be counted
-    const int eq_mode = (all || cnt.y == 0 || pre.y >= s.keep_eq) ? 0 : (pre.y + cnt.y <= s.keep_eq ? 1 : 2);
-    uint32_t eq_seen = pre.y;
-    uint64_t pos = s.base + pre.x + min(pre.y, s.keep_eq);
-    const float* dd = dbuf + (size_t)w * dstride;
-    float* st = state + (size_t)w * stride;
-    uint32_t* oi = out_idx + (size_t)w * cap;
-    float* ov32 = reinterpret_cast<float*>(out_val) + (size_t)w * cap;
-    __nv_bfloat16* ov16 = reinterpret_cast<__nv_bfloat16*>(out_val) + (size_t)w * cap;
-
-    constexpr int E = 16; // elements per thread per round
-    const uint64_t q0 = ch.begin & ~3ull;
-    auto load_round = [&](uint64_t base, float* v) {
-        const uint64_t t0 = base + (uint64_t)E * threadIdx.x;
-#pragma unroll
-        for (int u = 0; u < E / 4; ++u) {
-            const uint64_t q = t0 + 4 * u;
-            if (q >= ch.begin && q + 4 <= ch.end) {
-                const float4 a = __ldg(reinterpret_cast<const float4*>(dd + q));
-                v[4 * u] = a.x; v[4 * u + 1] = a.y; v[4 * u + 2] = a.z; v[4 * u + 3] = a.w;
-            } else {
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const uint64_t p = q + i;
-                    v[4 * u + i] = (p >= ch.begin && p < ch.end) ? dd[p] : 0.f;
-                }
-            }
-        }
-    };
-    float v[E], nxt[E];
-    load_round(q0, v);
-    for (uint64_t base = q0; base < ch.end; base += (uint64_t)E * kThreads) {
-        const uint64_t t0 = base + (uint64_t)E * threadIdx.x;
-        const uint64_t nbase = base + (uint64_t)E * kThreads;
-        if (nbase < ch.end) load_round(nbase, nxt); // in flight while this round is compacted
-        uint32_t keepm = 0, eqm = 0;
-#pragma unroll
-        for (int i = 0; i < E; ++i) {
-            const uint64_t p = t0 + i;
-            const bool in = p >= ch.begin && p < ch.end;
-            const uint32_t key = key_of(v[i]);
-            if (in && (all || key > s.tau || (eq_mode == 1 && key == s.tau))) keepm |= 1u << i;
-            if (in && eq_mode == 2 && key == s.tau) eqm |= 1u << i;
-        }
-        if (__syncthreads_or((keepm | eqm) != 0)) {
-            if (eq_mode == 2) { // uniform over the CTA
-                uint32_t tot_eq;
-                uint32_t eq_rank = eq_seen + block_excl_scan<uint32_t>(__popc(eqm), s_w, &tot_eq);
-#pragma unroll
-                for (int i = 0; i < E; ++i)
-                    if (eqm & (1u << i)) {
-                        if (eq_rank < s.keep_eq) keepm |= 1u << i;
-                        ++eq_rank;
-                    }
-                eq_seen += tot_eq;
-            }
-            uint32_t tot_keep;
-            uint64_t o = pos + block_excl_scan<uint32_t>(__popc(keepm), s_w, &tot_keep);
-#pragma unroll
-            for (int i = 0; i < E; ++i) {
-                if (keepm & (1u << i)) {
-                    const uint64_t p = t0 + i;
-                    oi[o] = (uint32_t)(p - ld.begin);
-                    float sent;
-                    if (BF16) {
-                        const __nv_bfloat16 h = __float2bfloat16_rn(v[i]);
-                        ov16[o] = h;
-                        sent = __bfloat162float(h);
-                    } else {
-                        ov32[o] = v[i];
-                        sent = v[i];
-                    }
-                    st[p] = __fadd_rn(st[p], sent);
-                    ++o;
-                }
-            }
-            pos += tot_keep;
-        }
-#pragma unroll
-        for (int i = 0; i < E; ++i) v[i] = nxt[i];
     }
 }
 

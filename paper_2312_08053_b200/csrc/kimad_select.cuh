@@ -1,0 +1,312 @@
+// Stages (d)-(f): Top-K selection at the chosen k, ordered sparse pack, EF21 update.
+//
+// After the DP every (worker, layer) knows a key interval [lo, lo + 2^shift) that contains its
+// threshold and the rank of the threshold inside that interval (shift = 0 when the curve stage already
+// resolved all 31 bits).  One sweep over the difference vector (k_sel_count) counts, per chunk, the
+// entries above the interval and remembers the few entries inside it; k_sel_resolve turns the
+// per-layer histogram of those entries into the exact threshold; k_sel_scan derives every chunk's
+// output offset; k_sel_write compacts in index order and updates the estimator.  No kernel waits on
+// another: offsets come from stored per-chunk counts.
+#pragma once
+#include "kimad_kernels.cuh"
+
+namespace kimad {
+
+constexpr int kListCap = 32;                    // in-interval entries remembered per chunk
+constexpr uint32_t kListOverflow = 0xffffffffu; // more than that: the chunk is recounted exactly
+constexpr int kLowBins = 1024;                  // 2^shift never exceeds this
+
+struct ChunkSel { // per (worker, chunk)
+    uint32_t above;          // entries whose key lies above the interval
+    uint32_t n_in;           // entries inside the interval, or kListOverflow
+    uint16_t low[kListCap];  // key - lo of those entries (any order)
+};
+
+// Aligned view of a chunk for 128-bit loads: quads start at a0 = begin & ~3; only the first and the
+// last quad can be partial.  All offsets are 32-bit and relative to a0.
+struct ChunkView {
+    uint64_t a0;
+    uint32_t first, len; // valid element offsets are [first, len)
+    __device__ __forceinline__ explicit ChunkView(const Chunk& ch)
+        : a0(ch.begin & ~3ull), first((uint32_t)(ch.begin - (ch.begin & ~3ull))), len((uint32_t)(ch.end - (ch.begin & ~3ull))) {}
+    __device__ __forceinline__ uint32_t quads() const { return (len + 3) >> 2; }
+    __device__ __forceinline__ bool quad_full(uint32_t q) const { return 4 * q >= first && 4 * q + 4 <= len; }
+};
+
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads)
+k_sel_count(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks, uint64_t dstride,
+            uint32_t L, const Sel* __restrict__ sel, const LayerDesc* __restrict__ layers, ChunkSel* __restrict__ csel,
+            uint32_t* __restrict__ low_hist, uint32_t* __restrict__ recount_n, uint2* __restrict__ recount_list) {
+    __shared__ uint32_t s_w[8];
+    __shared__ uint32_t s_hist[kLowBins];
+    __shared__ uint32_t s_n;
+    __shared__ uint16_t s_low[kListCap];
+    const Chunk ch = chunks[blockIdx.x];
+    const uint32_t w = blockIdx.y;
+    const size_t wl = (size_t)w * L + ch.layer;
+    const Sel s = sel[wl];
+    ChunkSel* out = csel + (size_t)w * n_chunks + blockIdx.x;
+    if (s.k == 0 || (uint64_t)s.k == layers[ch.layer].n) { // nothing / everything kept: no need to look at the data
+        if (threadIdx.x == 0) { out->above = s.k ? (uint32_t)(ch.end - ch.begin) : 0u; out->n_in = 0; }
+        return;
+    }
+    const uint32_t lo = s.tau, width = 1u << s.shift;
+    for (int i = threadIdx.x; i < kLowBins; i += kThreads) s_hist[i] = 0;
+    if (threadIdx.x == 0) s_n = 0;
+    __syncthreads();
+    const ChunkView cv(ch);
+    const float* dd = dbuf + (size_t)w * dstride + cv.a0;
+    uint32_t above = 0;
+    auto visit = [&](float dv) {
+        const uint32_t d1 = key_of(dv) - lo; // wraps to >= 2^31 for keys below the interval
+        if (d1 < width) {
+            atomicAdd(&s_hist[d1], 1u);
+            const uint32_t p = atomicAdd(&s_n, 1u);
+            if (p < (uint32_t)kListCap) s_low[p] = (uint16_t)d1;
+        } else {
+            above += d1 < 0x80000000u;
+        }
+    };
+    const uint32_t nq = cv.quads();
+    constexpr int U = 4;
+    for (uint32_t qb = 0; qb < nq; qb += kThreads * U) {
+        float4 a[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t q = qb + u * kThreads + threadIdx.x;
+            if (q < nq && cv.quad_full(q)) a[u] = __ldcs(reinterpret_cast<const float4*>(dd) + q);
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t q = qb + u * kThreads + threadIdx.x;
+            if (q >= nq) continue;
+            if (cv.quad_full(q)) {
+                visit(a[u].x); visit(a[u].y); visit(a[u].z); visit(a[u].w);
+            } else {
+                for (uint32_t e = 4 * q; e < 4 * q + 4; ++e)
+                    if (e >= cv.first && e < cv.len) visit(dd[e]);
+            }
+        }
+    }
+    uint32_t tot;
+    block_excl_scan<uint32_t>(above, s_w, &tot);
+    __syncthreads();
+    const uint32_t n_in = s_n;
+    if (n_in) { // rare: publish this chunk's part of the layer's in-interval histogram
+        uint32_t* gh = low_hist + wl * kLowBins;
+        for (uint32_t i = threadIdx.x; i < width; i += kThreads)
+            if (s_hist[i]) atomicAdd(&gh[i], s_hist[i]);
+    }
+    if (threadIdx.x < min(n_in, (uint32_t)kListCap)) out->low[threadIdx.x] = s_low[threadIdx.x];
+    if (threadIdx.x == 0) {
+        out->above = tot;
+        if (n_in <= (uint32_t)kListCap) {
+            out->n_in = n_in;
+        } else {
+            out->n_in = kListOverflow;
+            recount_list[atomicAdd(recount_n, 1u)] = make_uint2(w, blockIdx.x);
+        }
+    }
+}
+
+// Exact threshold of every (worker, layer) from the histogram of the entries inside its interval.
+__global__ void __launch_bounds__(kThreads)
+k_sel_resolve(uint32_t L, const LayerDesc* __restrict__ layers, uint32_t* __restrict__ low_hist, Sel* __restrict__ sel) {
+    __shared__ __align__(16) uint32_t s_incl[kLowBins];
+    __shared__ uint32_t s_w32[8];
+    const uint32_t l = blockIdx.x, w = blockIdx.y;
+    const size_t wl = (size_t)w * L + l;
+    Sel s = sel[wl];
+    if (s.k == 0 || (uint64_t)s.k == layers[l].n) return;
+    const uint32_t width = 1u << s.shift;
+    uint32_t* gh = low_hist + wl * kLowBins;
+    for (int b = threadIdx.x; b < kLowBins; b += kThreads) {
+        uint32_t c = 0;
+        if ((uint32_t)b < width) { c = gh[b]; gh[b] = 0; }
+        s_incl[kLowBins - 1 - b] = c;
+    }
+    __syncthreads();
+    scan_bins<kLowBins>(s_incl, nullptr, s_w32, nullptr);
+    if (threadIdx.x == 0) {
+        const int p = find_pos<kLowBins>(s_incl, s.keep_eq); // keep_eq holds the rank inside the interval
+        const uint32_t above = p ? s_incl[p - 1] : 0u;
+        const uint32_t bin = (uint32_t)(kLowBins - 1 - p);
+        s.tau_low = bin;
+        s.tau += bin;
+        s.keep_eq -= above;
+        sel[wl] = s;
+    }
+}
+
+// Exact (gt, eq) of the chunks whose list overflowed.
+__global__ void __launch_bounds__(kThreads)
+k_sel_recount(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks, uint64_t dstride,
+              uint32_t L, const Sel* __restrict__ sel, const uint32_t* __restrict__ recount_n,
+              const uint2* __restrict__ recount_list, uint2* __restrict__ chunk_cnt) {
+    __shared__ uint32_t s_w[8];
+    const uint32_t n = *recount_n;
+    for (uint32_t it = blockIdx.x; it < n; it += gridDim.x) {
+        const uint2 e = recount_list[it];
+        const Chunk ch = chunks[e.y];
+        const Sel s = sel[(size_t)e.x * L + ch.layer];
+        const ChunkView cv(ch);
+        const float* dd = dbuf + (size_t)e.x * dstride + cv.a0;
+        uint32_t gt = 0, eq = 0;
+        for (uint32_t x = cv.first + threadIdx.x; x < cv.len; x += kThreads) {
+            const uint32_t key = key_of(dd[x]);
+            gt += key > s.tau;
+            eq += key == s.tau;
+        }
+        uint32_t tg, te;
+        block_excl_scan<uint32_t>(gt, s_w, &tg);
+        block_excl_scan<uint32_t>(eq, s_w, &te);
+        if (threadIdx.x == 0) chunk_cnt[(size_t)e.x * n_chunks + e.y] = make_uint2(tg, te);
+        __syncthreads();
+    }
+}
+
+// chunk_cnt[(w, chunk)] = (entries above tau, entries equal to tau); chunk_pre = exclusive prefix of
+// both over the layer's earlier chunks.
+__global__ void __launch_bounds__(kThreads)
+k_sel_scan(uint32_t L, const LayerDesc* __restrict__ layers, uint32_t n_chunks, const Sel* __restrict__ sel,
+           const ChunkSel* __restrict__ csel, uint2* __restrict__ chunk_cnt, uint2* __restrict__ chunk_pre,
+           uint32_t* __restrict__ recount_n) {
+    __shared__ uint32_t s_w[8];
+    const LayerDesc ld = layers[blockIdx.x];
+    const uint32_t w = blockIdx.y;
+    const Sel s = sel[(size_t)w * L + blockIdx.x];
+    const ChunkSel* cs = csel + (size_t)w * n_chunks + ld.first_chunk;
+    uint2* cc = chunk_cnt + (size_t)w * n_chunks + ld.first_chunk;
+    uint2* cp = chunk_pre + (size_t)w * n_chunks + ld.first_chunk;
+    if (blockIdx.x == 0 && w == 0 && threadIdx.x == 0) *recount_n = 0; // consumed by k_sel_recount already
+    uint32_t run_g = 0, run_e = 0;
+    for (uint32_t base = 0; base < ld.n_chunks; base += kThreads) {
+        const uint32_t i = base + threadIdx.x;
+        uint2 v = make_uint2(0, 0);
+        if (i < ld.n_chunks) {
+            const uint32_t n_in = cs[i].n_in;
+            if (n_in == kListOverflow) {
+                v = cc[i];
+            } else {
+                v.x = cs[i].above;
+                for (uint32_t e = 0; e < n_in; ++e) {
+                    const uint32_t low = cs[i].low[e];
+                    v.x += low > s.tau_low;
+                    v.y += low == s.tau_low;
+                }
+                cc[i] = v;
+            }
+        }
+        uint32_t tg, te;
+        const uint32_t eg = block_excl_scan<uint32_t>(v.x, s_w, &tg);
+        const uint32_t ee = block_excl_scan<uint32_t>(v.y, s_w, &te);
+        if (i < ld.n_chunks) cp[i] = make_uint2(run_g + eg, run_e + ee);
+        run_g += tg;
+        run_e += te;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// (e) + (f).  Every thread owns 16 consecutive elements of a 4096-element round, so that ranks inside
+// a round follow the index order.
+// ------------------------------------------------------------------------------------------------
+template <bool BF16>
+__global__ void __launch_bounds__(kThreads)
+k_sel_write(const float* __restrict__ dbuf, float* __restrict__ state, const Chunk* __restrict__ chunks,
+            uint32_t n_chunks, uint64_t dstride, uint64_t stride, uint32_t L, const Sel* __restrict__ sel,
+            const LayerDesc* __restrict__ layers, const uint2* __restrict__ chunk_cnt,
+            const uint2* __restrict__ chunk_pre, uint64_t cap, uint32_t* __restrict__ out_idx,
+            void* __restrict__ out_val) {
+    __shared__ uint32_t s_w[8];
+    const Chunk ch = chunks[blockIdx.x];
+    const uint32_t w = blockIdx.y;
+    const Sel s = sel[(size_t)w * L + ch.layer];
+    if (s.k == 0) return;
+    const LayerDesc ld = layers[ch.layer];
+    const bool all = (uint64_t)s.k == ld.n;
+    const uint2 cnt = chunk_cnt[(size_t)w * n_chunks + blockIdx.x];
+    const uint2 pre = chunk_pre[(size_t)w * n_chunks + blockIdx.x];
+    if (!all && cnt.x == 0 && (cnt.y == 0 || pre.y >= s.keep_eq)) return; // nothing kept in this chunk
+    // entries equal to tau are kept while their rank among equals (ascending index) is below keep_eq
+    // eq_mode 0: none of this chunk's equals is kept; 1: all are; 2: ranks must be counted
+    const int eq_mode = (all || cnt.y == 0 || pre.y >= s.keep_eq) ? 0 : (pre.y + cnt.y <= s.keep_eq ? 1 : 2);
+    // keep <=> key > thr, with thr = tau - 1 when this chunk's equals are all kept (tau >= 1 then, or all)
+    const uint32_t tau = s.tau;
+    uint32_t eq_seen = pre.y;
+    uint32_t pos = 0; // kept so far in this chunk
+    const ChunkView cv(ch);
+    const float* dd = dbuf + (size_t)w * dstride + cv.a0;
+    float* st = state + (size_t)w * stride + cv.a0;
+    const uint64_t obase = (size_t)w * cap + s.base + pre.x + min(pre.y, s.keep_eq);
+    uint32_t* oi = out_idx + obase;
+    float* ov32 = reinterpret_cast<float*>(out_val) + obase;
+    __nv_bfloat16* ov16 = reinterpret_cast<__nv_bfloat16*>(out_val) + obase;
+    const uint32_t idx0 = (uint32_t)(cv.a0 - ld.begin); // layer-local index of offset 0 (may wrap; added back below)
+
+    constexpr int E = 16;
+    for (uint32_t rb = 0; rb < cv.len; rb += E * kThreads) {
+        const uint32_t t0 = rb + E * threadIdx.x;
+        uint32_t keepm = 0, eqm = 0;
+        const bool interior = rb >= cv.first && rb + E * kThreads <= cv.len;
+        if (interior) {
+#pragma unroll
+            float v[E];
+#pragma unroll
+            for (int u = 0; u < E / 4; ++u) {
+                const float4 a = __ldg(reinterpret_cast<const float4*>(dd + t0) + u);
+                v[4 * u] = a.x; v[4 * u + 1] = a.y; v[4 * u + 2] = a.z; v[4 * u + 3] = a.w;
+            }
+#pragma unroll
+            for (int i = 0; i < E; ++i) {
+                const uint32_t key = key_of(v[i]);
+                if (all || key > tau || (eq_mode == 1 && key == tau)) keepm |= 1u << i;
+                if (eq_mode == 2 && key == tau) eqm |= 1u << i;
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < E; ++i) {
+                const uint32_t e = t0 + i;
+                const bool in = e >= cv.first && e < cv.len;
+                const uint32_t key = key_of(in ? __ldg(dd + e) : 0.f);
+                if (in && (all || key > tau || (eq_mode == 1 && key == tau))) keepm |= 1u << i;
+                if (in && eq_mode == 2 && key == tau) eqm |= 1u << i;
+            }
+        }
+        if (!__syncthreads_or((keepm | eqm) != 0)) continue;
+        if (eq_mode == 2) { // uniform over the CTA
+            uint32_t tot_eq;
+            uint32_t eq_rank = eq_seen + block_excl_scan<uint32_t>(__popc(eqm), s_w, &tot_eq);
+#pragma unroll
+            for (int i = 0; i < E; ++i)
+                if (eqm & (1u << i)) {
+                    if (eq_rank < s.keep_eq) keepm |= 1u << i;
+                    ++eq_rank;
+                }
+            eq_seen += tot_eq;
+        }
+        uint32_t tot_keep;
+        uint32_t o = pos + block_excl_scan<uint32_t>(__popc(keepm), s_w, &tot_keep);
+        pos += tot_keep;
+        while (keepm) {
+            const int i = __ffs(keepm) - 1;
+            keepm &= keepm - 1;
+            const uint32_t e = t0 + i;
+            const float val = dd[e]; // loaded a moment ago: an L1 hit
+            oi[o] = idx0 + e;
+            float sent;
+            if (BF16) {
+                const __nv_bfloat16 h = __float2bfloat16_rn(val);
+                ov16[o] = h;
+                sent = __bfloat162float(h);
+            } else {
+                ov32[o] = val;
+                sent = val;
+            }
+            st[e] = __fadd_rn(st[e], sent);
+            ++o;
+        }
+    }
+}
+
+} // namespace kimad
