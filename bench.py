@@ -32,11 +32,11 @@ UNIT = "elements/s"
 
 # DRAM traffic of the dominant kernel per input element, from the ncu capture summarised under
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum of one launch / elements of that launch).
-NCU_TRAFFIC_BYTES_PER_ELEM = {"diff_hist1": None}
+NCU_TRAFFIC_BYTES_PER_ELEM = {"sweep": None}
 
 # algorithmic bytes per input element of each stage (what the stage must move at least once)
-STAGE_ALGO_BYTES = {"diff_hist1": 12.0,  # read grad + g, write d
-                    "hist2": 4.0, "hist3": 4.0, "select_count": 4.0, "select_write": 4.0}
+STAGE_ALGO_BYTES = {"sweep": 12.0,  # read grad + g, write d
+                    "select_count": 4.0, "select_write": 4.0}
 
 
 def peaks():
@@ -177,8 +177,9 @@ def run_kimad(args, rank, world):
     ctx = kb.new_context(wl.layer_sizes, W, wl.ratio_grid, device=dev, D=wl.D, value_dtype=wl.value_dtype,
                          max_packed_elems=cap)
     out = kb.Packed(ctx, device=dev)
-    n_bufs = 2
-    # fresh gradients per buffer; every rank draws its own streams (seed offset by rank)
+    # fresh gradients for every step (as in training), as far as ~70 GB of device memory go; beyond that the
+    # buffers are cycled.  Every rank draws its own streams (seed offset by rank).
+    n_bufs = int(max(2, min(args.warmup + args.steps, 70e9 // (W * N * 4))))
     grads = [workloads.gradients(wl, 1000 * rank + s, device=dev) for s in range(n_bufs)]
     state = torch.zeros((W, N), dtype=torch.float32, device=dev)
     stream = torch.cuda.current_stream()
@@ -221,7 +222,8 @@ def run_kimad(args, rank, world):
         raise RuntimeError(f"kimad step failed on rank {rank}: {kb.kimad_strerror(status)}")
 
     # ---- end to end: host buffers in, packed message out, copies inside the timed region
-    host_grads = [g.cpu().pin_memory() for g in grads]
+    e2e_bufs = min(n_bufs, 3)
+    host_grads = [g.cpu().pin_memory() for g in grads[:e2e_bufs]]
     dev_in = torch.empty_like(grads[0])
     h_stats = torch.empty_like(out.stats, device="cpu").pin_memory()
     h_idx = torch.empty((W, cap), dtype=torch.int32).pin_memory()
@@ -231,7 +233,7 @@ def run_kimad(args, rank, world):
 
     def e2e_step(s):
         nonlocal d2h_bytes
-        dev_in.copy_(host_grads[s % n_bufs], non_blocking=True)
+        dev_in.copy_(host_grads[s % e2e_bufs], non_blocking=True)
         kb.kimad_step(ctx, dev_in, state, bw[s % len(bw)], wl.t_target, out, stream)
         h_stats.copy_(out.stats, non_blocking=True)
         stream.synchronize()
@@ -289,12 +291,13 @@ def run_kimad(args, rank, world):
         "config": {"workload": wl.name, "cfg": wl.cfg, "workers_per_gpu": W, "layers": L, "elements_per_worker": N,
                    "ratios": len(wl.ratio_grid), "D": wl.D, "value_dtype": "bf16" if wl.value_dtype else "f32",
                    "l2": "inputs_larger_than_l2" if W * N * 4 > 200e6 else "inputs_fit_l2",
-                   "budget_trace": "cycled", "parallelism": f"worker-sharded x{world}"},
+                   "budget_trace": "cycled", "gradient_buffers": n_bufs, "parallelism": f"worker-sharded x{world}"},
         "e2e": e2e, "gpu_launches": int(launches),
         "roofline": roofline,
         "step_roofline": {"bound": "hbm", "compulsory_bytes_per_step": compulsory, "achieved": step_gbs, "peak": peak,
                           "unit": "GB/s", "frac": step_gbs / peak, "peak_kind": f"of {peak_kind}"},
         "stage_ms": stage_ms, "step_ms_minmax": [min(per_step), max(per_step)],
+        "exact_path_layers": kb.kimad_debug_exact_path_layers(ctx, detail=True),
         "clocks": sampler.summary(t_wall0, t_wall1),
     }
     if world == 1 and not args.no_cpu_baseline:

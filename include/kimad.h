@@ -61,6 +61,9 @@ typedef struct {
     uint32_t infeasible_policy; /* 0: take candidate 0 everywhere and report KIMAD_STATUS_INFEASIBLE */
     uint64_t max_packed_elems;  /* capacity (entries) of each worker's idx/val buffer; 0 -> N        */
     uint64_t worker_stride;     /* elements between consecutive workers in grads/state; 0 -> N       */
+    uint32_t curve_mode;        /* 0: error curves from one sweep over sampled bands, exact radix select
+                                   only where the certificate fails; 1: exact radix select everywhere   */
+    uint32_t reserved;
 } kimad_options;
 
 /* Per-worker result record, written by the device. */
@@ -133,9 +136,15 @@ int kimad_plan_budget(const kimad_ctx* ctx, double bandwidth_bytes_per_s, double
 
 /* Stage isolation for tests.  All synchronise the device.
  * kimad_debug_get_curve: results of stage (b) of the last step; each pointer is host
- *   [W][L][K] or NULL: err (f32), tau (31-bit magnitude key of the k-th largest entry),
- *   keep_eq (how many entries equal to tau are kept). */
-int kimad_debug_get_curve(kimad_ctx* ctx, float* host_err, uint32_t* host_tau, uint32_t* host_keep_eq);
+ *   [W][L][K] or NULL: err (f32); shift: the threshold of the candidate is known to lie in the
+ *   key interval [tau, tau + 2^shift) and to be the keep_eq-th largest key inside it.  Where
+ *   shift is 0, tau is the 31-bit magnitude key of the k-th largest entry and keep_eq the number
+ *   of entries equal to tau that are kept.
+ * kimad_debug_get_selection: exact threshold key and number of kept ties of the candidate chosen
+ *   for every layer in the last step, host u32 [W][L] each (meaningless where k = n_l or k = 0). */
+int kimad_debug_get_curve(kimad_ctx* ctx, float* host_err, uint32_t* host_tau, uint32_t* host_keep_eq,
+                          uint32_t* host_shift);
+int kimad_debug_get_selection(kimad_ctx* ctx, uint32_t* host_tau, uint32_t* host_keep_eq);
 /* kimad_step whose DP (c) consumes err_dev (device, f32 [W][L][K]) instead of the curves it
  * computed; stages (a), (b), (d)-(f) unchanged. */
 int kimad_debug_step_with_err(kimad_ctx* ctx, const float* grads_dev, float* state_dev,
@@ -146,12 +155,22 @@ int kimad_debug_step_with_j(kimad_ctx* ctx, const float* grads_dev, float* state
                             const double* bandwidth_bytes_per_s, double t_target_s, const kimad_packed* out,
                             void* cuda_stream, const uint32_t* j_dev);
 
+/* How many (worker, layer) pairs took the exact radix path since the workspace was attached.
+ * host_count: host, u64 [5]: total, then by reason: forced by curve_mode 1; bands too wide for
+ * the tables; a threshold outside its sampled band; error bound too loose.  Synchronises the device. */
+int kimad_debug_exact_path_layers(kimad_ctx* ctx, uint64_t* host_count);
+
+/* Band tables of the last step, one record of four u32 per (worker, layer above the tiny size), in
+ * worker-major order: bins used, 11-bit bins split into cells, flag (0: sampled bands in use, 1: exact
+ * path forced, 2: bands did not fit the tables), detail of the misfit.  host_meta: host, u32 [W][R][4]. */
+int kimad_debug_get_band_meta(kimad_ctx* ctx, uint32_t* host_meta);
+
 /* Per-stage device timing for benchmarks.  enable != 0: every following step records CUDA events
  * around its stages on the step's stream (first use creates the events).  kimad_debug_stage_times
  * synchronises the device and writes the last step's stage durations in milliseconds to host_ms
- * (host, f32 [KIMAD_N_STAGES]), stage order: diff+hist1, resolve1, hist2, resolve2, hist3, resolve3,
- * dp, select_count, select_scan, select_write. */
-#define KIMAD_N_STAGES 10
+ * (host, f32 [KIMAD_N_STAGES]), stage order: sample, sweep (difference + banded histogram), curve
+ * (resolve + tiny layers), exact radix fallback, dp, select_count, select_scan, select_write. */
+#define KIMAD_N_STAGES 8
 int kimad_debug_enable_stage_timing(kimad_ctx* ctx, int enable);
 int kimad_debug_stage_times(kimad_ctx* ctx, float* host_ms);
 

@@ -27,7 +27,8 @@ KIMAD_ERR_NOMEM = -7
 
 class kimad_options(C.Structure):
     _fields_ = [("D", C.c_uint32), ("value_dtype", C.c_uint32), ("check_finite", C.c_uint32),
-                ("infeasible_policy", C.c_uint32), ("max_packed_elems", C.c_uint64), ("worker_stride", C.c_uint64)]
+                ("infeasible_policy", C.c_uint32), ("max_packed_elems", C.c_uint64), ("worker_stride", C.c_uint64),
+                ("curve_mode", C.c_uint32), ("reserved", C.c_uint32)]
 
 
 class kimad_stats(C.Structure):
@@ -90,11 +91,17 @@ def load():
     L.kimad_plan_budget.restype = C.c_int
     L.kimad_plan_budget.argtypes = [vp, dbl, dbl, C.POINTER(u64), vp]
     L.kimad_debug_get_curve.restype = C.c_int
-    L.kimad_debug_get_curve.argtypes = [vp, vp, vp, vp]
+    L.kimad_debug_get_curve.argtypes = [vp, vp, vp, vp, vp]
+    L.kimad_debug_get_selection.restype = C.c_int
+    L.kimad_debug_get_selection.argtypes = [vp, vp, vp]
     L.kimad_debug_enable_stage_timing.restype = C.c_int
     L.kimad_debug_enable_stage_timing.argtypes = [vp, C.c_int]
     L.kimad_debug_stage_times.restype = C.c_int
     L.kimad_debug_stage_times.argtypes = [vp, vp]
+    L.kimad_debug_get_band_meta.restype = C.c_int
+    L.kimad_debug_get_band_meta.argtypes = [vp, vp]
+    L.kimad_debug_exact_path_layers.restype = C.c_int
+    L.kimad_debug_exact_path_layers.argtypes = [vp, C.POINTER(u64)]
     L.kimad_launch_count.restype = u64
     L.kimad_launch_count.argtypes = [vp]
     L.kimad_strerror.restype = C.c_char_p
@@ -131,10 +138,10 @@ class Ctx:
 
 
 def kimad_create(layer_sizes, n_workers, ratio_grid, D=0, value_dtype=0, check_finite=0, max_packed_elems=0,
-                 worker_stride=0) -> Ctx:
+                 worker_stride=0, curve_mode=0) -> Ctx:
     ls = np.ascontiguousarray(layer_sizes, dtype=np.uint64)
     rg = np.ascontiguousarray(ratio_grid, dtype=np.float64)
-    opts = kimad_options(D, value_dtype, check_finite, 0, max_packed_elems, worker_stride)
+    opts = kimad_options(D, value_dtype, check_finite, 0, max_packed_elems, worker_stride, curve_mode, 0)
     h = C.c_void_p()
     _check(load().kimad_create(C.byref(h), ls.ctypes.data_as(C.POINTER(C.c_uint64)), ls.size, n_workers,
                                rg.ctypes.data_as(C.POINTER(C.c_double)), rg.size, C.byref(opts)), "kimad_create")
@@ -239,18 +246,27 @@ def kimad_plan_budget(ctx: Ctx, bandwidth_bytes_per_s: float, t_target_s: float)
 
 
 def kimad_debug_get_curve(ctx: Ctx):
-    """Returns (err f32, tau u32, keep_eq u32), each [W][L][K], of the last step."""
+    """Returns (err f32, tau u32, keep_eq u32, shift u32), each [W][L][K], of the last step."""
     shape = (ctx.W, ctx.L, ctx.K)
     err = np.zeros(shape, np.float32)
     tau = np.zeros(shape, np.uint32)
     keq = np.zeros(shape, np.uint32)
-    _check(load().kimad_debug_get_curve(ctx.handle, err.ctypes.data, tau.ctypes.data, keq.ctypes.data),
-           "kimad_debug_get_curve")
-    return err, tau, keq
+    shift = np.zeros(shape, np.uint32)
+    _check(load().kimad_debug_get_curve(ctx.handle, err.ctypes.data, tau.ctypes.data, keq.ctypes.data,
+                                        shift.ctypes.data), "kimad_debug_get_curve")
+    return err, tau, keq, shift
 
 
-STAGE_NAMES = ["diff_hist1", "resolve1", "hist2", "resolve2", "hist3", "resolve3", "dp", "select_count",
-               "select_scan", "select_write"]
+def kimad_debug_get_selection(ctx: Ctx):
+    """Returns (tau u32, keep_eq u32), each [W][L]: exact threshold of the chosen candidate of every layer."""
+    tau = np.zeros((ctx.W, ctx.L), np.uint32)
+    keq = np.zeros((ctx.W, ctx.L), np.uint32)
+    _check(load().kimad_debug_get_selection(ctx.handle, tau.ctypes.data, keq.ctypes.data),
+           "kimad_debug_get_selection")
+    return tau, keq
+
+
+STAGE_NAMES = ["sample", "sweep", "curve", "exact_fallback", "dp", "select_count", "select_scan", "select_write"]
 
 
 def kimad_debug_enable_stage_timing(ctx: Ctx, enable: bool) -> None:
@@ -262,6 +278,21 @@ def kimad_debug_stage_times(ctx: Ctx) -> np.ndarray:
     ms = np.zeros(len(STAGE_NAMES), np.float32)
     _check(load().kimad_debug_stage_times(ctx.handle, ms.ctypes.data), "kimad_debug_stage_times")
     return ms
+
+
+def kimad_debug_get_band_meta(ctx: Ctx, n_regular: int) -> np.ndarray:
+    """u32 [W][n_regular][4]: bins, split 11-bit bins, flag, detail (see kimad.h)."""
+    out = np.zeros((ctx.W, n_regular, 4), np.uint32)
+    _check(load().kimad_debug_get_band_meta(ctx.handle, out.ctypes.data), "kimad_debug_get_band_meta")
+    return out
+
+
+def kimad_debug_exact_path_layers(ctx: Ctx, detail: bool = False):
+    """Layers handed to the exact radix path so far; with detail also the count per reason
+    (forced, bands too wide, threshold outside band, bound too loose)."""
+    n = (C.c_uint64 * 5)()
+    _check(load().kimad_debug_exact_path_layers(ctx.handle, n), "kimad_debug_exact_path_layers")
+    return [int(x) for x in n] if detail else int(n[0])
 
 
 def kimad_launch_count(ctx: Ctx) -> int:

@@ -17,8 +17,13 @@ constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-    size_t dbuf, chunks, layers, ktab, h1_cnt, h1_ss, h23_cnt, h23_ss, cands, slots, err, tau, keep_eq, sel, chunk_cnt,
-        chunk_pre, csel, low_hist, recount, flags, pd, total;
+    // static tables
+    size_t dbuf, chunks, layers, ktab, reg_layers, tiny_layers, reg_index;
+    // zeroed at set_workspace and kept clean by the kernels
+    size_t zero_from, h1_cnt, h1_ss, h23_cnt, h23_ss, bh_cnt, bh_sum, low_hist, recount, fb, r2, flags;
+    // scratch without initial-state requirements
+    size_t lut_t1, lut_t2, bin_lo, meta, cands, slots, err, tau, keep_eq, shift, sel, chunk_cnt, chunk_pre, csel,
+        fb_chunks, fb_layers, r2_chunks, r2_layers, pd, total;
 };
 
 } // namespace
@@ -32,10 +37,13 @@ struct kimad_ctx {
     std::vector<double> grid;
     std::vector<Chunk> chunks;
     std::vector<LayerDesc> layers;
+    std::vector<uint32_t> reg_layers, tiny_layers, reg_index; // layers above / up to kTinyMax elements
+    uint32_t curve_mode = 0;
+    size_t sample_smem = 0, pass_a_smem = 0, tiny_smem = 0;
     Layout lay{};
     unsigned char* ws = nullptr;
     DpPlan dp_plan{};
-    size_t dp_smem = 0, hist2_smem = 0, hist3_smem = 0;
+    size_t dp_smem = 0;
     uint64_t launches = 0;
     kimad_packed last_out{};
     bool have_last = false;
@@ -51,27 +59,45 @@ void plan_layout(kimad_ctx* c) {
     Layout& y = c->lay;
     size_t o = 0;
     auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes); return at; };
-    const size_t WL = (size_t)c->W * c->L, WLK = WL * c->K;
+    const size_t WL = (size_t)c->W * c->L, WLK = WL * c->K, WR = (size_t)c->W * c->reg_layers.size();
+    const size_t nch = c->chunks.size();
     y.dbuf = take((size_t)c->W * c->dstride * sizeof(float));
-    y.chunks = take(c->chunks.size() * sizeof(Chunk));
+    y.chunks = take(nch * sizeof(Chunk));
     y.layers = take(c->layers.size() * sizeof(LayerDesc));
     y.ktab = take(c->ktab.size() * sizeof(uint64_t));
+    y.reg_layers = take(c->reg_layers.size() * sizeof(uint32_t));
+    y.tiny_layers = take(c->tiny_layers.size() * sizeof(uint32_t));
+    y.reg_index = take(c->reg_index.size() * sizeof(uint32_t));
+    y.zero_from = o;
     y.h1_cnt = take(WL * kL1Bins * sizeof(uint32_t));
-    y.h1_ss = take(WL * kL1Bins * sizeof(double));
+    y.h1_ss = take(WL * kL1Bins * sizeof(uint64_t));
     y.h23_cnt = take(WLK * kL23Bins * sizeof(uint32_t));
-    y.h23_ss = take(WLK * kL23Bins * sizeof(double));
+    y.h23_ss = take(WLK * kL23Bins * sizeof(uint64_t));
+    y.bh_cnt = take(WR * kMaxBins * sizeof(uint32_t));
+    y.bh_sum = take(WR * kMaxBins * sizeof(uint64_t));
+    y.low_hist = take(WL * kLowBins * sizeof(uint32_t));
+    y.recount = take(256 + (size_t)2 * c->W * nch * sizeof(uint2));
+    y.fb = take(sizeof(FbList));
+    y.r2 = take(sizeof(Round2));
+    y.flags = take((size_t)c->W * sizeof(uint32_t));
+    y.lut_t1 = take(WR * kL1Bins * sizeof(uint16_t));
+    y.lut_t2 = take(WR * kMaxRows * 32 * sizeof(uint32_t));
+    y.bin_lo = take(WR * (kMaxBins + 1) * sizeof(uint32_t));
+    y.meta = take(WR * sizeof(BandMeta));
     y.cands = take(WLK * sizeof(Cand));
     y.slots = take(WL * sizeof(SlotTab));
     y.err = take(WLK * sizeof(float));
     y.tau = take(WLK * sizeof(uint32_t));
     y.keep_eq = take(WLK * sizeof(uint32_t));
+    y.shift = take(WLK * sizeof(uint32_t));
     y.sel = take(WL * sizeof(Sel));
-    y.chunk_cnt = take((size_t)c->W * c->chunks.size() * sizeof(uint2));
-    y.chunk_pre = take((size_t)c->W * c->chunks.size() * sizeof(uint2));
-    y.csel = take((size_t)c->W * c->chunks.size() * sizeof(ChunkSel));
-    y.low_hist = take(WL * kLowBins * sizeof(uint32_t));
-    y.recount = take(256 + (size_t)c->W * c->chunks.size() * sizeof(uint2));
-    y.flags = take((size_t)c->W * sizeof(uint32_t));
+    y.chunk_cnt = take((size_t)c->W * nch * sizeof(uint2));
+    y.chunk_pre = take((size_t)c->W * nch * sizeof(uint2));
+    y.csel = take((size_t)c->W * nch * sizeof(ChunkSel));
+    y.fb_chunks = take((size_t)c->W * nch * sizeof(uint2));
+    y.fb_layers = take(WL * sizeof(uint2));
+    y.r2_chunks = take((size_t)c->W * nch * sizeof(uint2));
+    y.r2_layers = take(WL * sizeof(uint2));
     y.pd = take(c->dp_plan.pd_in_smem ? 0 : (size_t)c->W * c->L * c->dp_plan.pd_row_bytes);
     y.total = o;
 }
@@ -97,65 +123,92 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
     const uint32_t nch = (uint32_t)c->chunks.size();
     const bool vec = ((uintptr_t)grads % 16 == 0) && ((uintptr_t)state % 16 == 0) && (c->stride % 4 == 0);
 
-    float* dbuf = c->at<float>(c->lay.dbuf);
-    const Chunk* chunks = c->at<Chunk>(c->lay.chunks);
-    const LayerDesc* layers = c->at<LayerDesc>(c->lay.layers);
-    const uint64_t* ktab = c->at<uint64_t>(c->lay.ktab);
-    uint32_t* h1c = c->at<uint32_t>(c->lay.h1_cnt);
-    unsigned long long* h1s = c->at<unsigned long long>(c->lay.h1_ss);
-    uint32_t* h23c = c->at<uint32_t>(c->lay.h23_cnt);
-    unsigned long long* h23s = c->at<unsigned long long>(c->lay.h23_ss);
-    Cand* cands = c->at<Cand>(c->lay.cands);
-    SlotTab* slots = c->at<SlotTab>(c->lay.slots);
-    float* err = c->at<float>(c->lay.err);
-    uint32_t* tau = c->at<uint32_t>(c->lay.tau);
-    uint32_t* keq = c->at<uint32_t>(c->lay.keep_eq);
-    Sel* sel = c->at<Sel>(c->lay.sel);
-    uint2* ccnt = c->at<uint2>(c->lay.chunk_cnt);
-    uint2* cpre = c->at<uint2>(c->lay.chunk_pre);
-    ChunkSel* csel = c->at<ChunkSel>(c->lay.csel);
-    uint32_t* lowh = c->at<uint32_t>(c->lay.low_hist);
-    uint32_t* recount_n = c->at<uint32_t>(c->lay.recount);
-    uint2* recount_list = c->at<uint2>(c->lay.recount + 256);
-    uint32_t* flags = c->at<uint32_t>(c->lay.flags);
-    uint8_t* pd = c->at<uint8_t>(c->lay.pd);
+    const Layout& y = c->lay;
+    float* dbuf = c->at<float>(y.dbuf);
+    const Chunk* chunks = c->at<Chunk>(y.chunks);
+    const LayerDesc* layers = c->at<LayerDesc>(y.layers);
+    const uint64_t* ktab = c->at<uint64_t>(y.ktab);
+    const uint32_t* reg_layers = c->at<uint32_t>(y.reg_layers);
+    const uint32_t* tiny_layers = c->at<uint32_t>(y.tiny_layers);
+    const uint32_t* reg_index = c->at<uint32_t>(y.reg_index);
+    uint32_t* h1c = c->at<uint32_t>(y.h1_cnt);
+    unsigned long long* h1s = c->at<unsigned long long>(y.h1_ss);
+    uint32_t* h23c = c->at<uint32_t>(y.h23_cnt);
+    unsigned long long* h23s = c->at<unsigned long long>(y.h23_ss);
+    uint32_t* bhc = c->at<uint32_t>(y.bh_cnt);
+    unsigned long long* bhs = c->at<unsigned long long>(y.bh_sum);
+    uint16_t* lut1 = c->at<uint16_t>(y.lut_t1);
+    uint32_t* lut2 = c->at<uint32_t>(y.lut_t2);
+    uint32_t* binlo = c->at<uint32_t>(y.bin_lo);
+    BandMeta* meta = c->at<BandMeta>(y.meta);
+    Cand* cands = c->at<Cand>(y.cands);
+    SlotTab* slots = c->at<SlotTab>(y.slots);
+    float* err = c->at<float>(y.err);
+    uint32_t* tau = c->at<uint32_t>(y.tau);
+    uint32_t* keq = c->at<uint32_t>(y.keep_eq);
+    uint32_t* shf = c->at<uint32_t>(y.shift);
+    Sel* sel = c->at<Sel>(y.sel);
+    uint2* ccnt = c->at<uint2>(y.chunk_cnt);
+    uint2* cpre = c->at<uint2>(y.chunk_pre);
+    ChunkSel* csel = c->at<ChunkSel>(y.csel);
+    uint32_t* lowh = c->at<uint32_t>(y.low_hist);
+    uint32_t* recount_n = c->at<uint32_t>(y.recount);
+    uint2* recount_list = c->at<uint2>(y.recount + 256);
+    FbList* fb = c->at<FbList>(y.fb);
+    uint2* fb_chunks = c->at<uint2>(y.fb_chunks);
+    uint2* fb_layers = c->at<uint2>(y.fb_layers);
+    Round2* r2 = c->at<Round2>(y.r2);
+    uint2* r2_chunks = c->at<uint2>(y.r2_chunks);
+    uint2* r2_layers = c->at<uint2>(y.r2_layers);
+    uint32_t* flags = c->at<uint32_t>(y.flags);
+    uint8_t* pd = c->at<uint8_t>(y.pd);
 
+    const uint32_t R = (uint32_t)c->reg_layers.size(), T = (uint32_t)c->tiny_layers.size();
     const dim3 gch(nch, W), glw(L, W), blk(kThreads);
+    const dim3 grun((nch + kRunChunksA - 1) / kRunChunksA, W);
     int stage = 0;
     auto mark = [&]() { if (c->timing) cudaEventRecord(c->ev[stage++], s); };
     mark();
-
-    // (a) + first digit
+    // (a) + (b): sample -> bands -> one sweep -> curves
+    if (R) {
+        k_sample<<<dim3(R, W), kBigThreads, c->sample_smem, s>>>(grads, state, c->stride, layers, reg_layers, R, ktab, K,
+                                                                 c->curve_mode == 1 ? 1u : 0u, lut1, lut2, binlo, meta);
+        c->launches += 1;
+    }
+    mark();
     if (vec)
-        k_diff_hist1<true><<<gch, blk, 0, s>>>(grads, state, dbuf, chunks, c->stride, c->dstride, L, h1c, h1s, flags);
+        k_pass_a<true><<<grun, kBigThreads, c->pass_a_smem, s>>>(grads, state, dbuf, chunks, nch, c->stride, c->dstride,
+                                                                 reg_index, R, lut1, lut2, meta, bhc, bhs);
     else
-        k_diff_hist1<false><<<gch, blk, 0, s>>>(grads, state, dbuf, chunks, c->stride, c->dstride, L, h1c, h1s, flags);
+        k_pass_a<false><<<grun, kBigThreads, c->pass_a_smem, s>>>(grads, state, dbuf, chunks, nch, c->stride, c->dstride,
+                                                                  reg_index, R, lut1, lut2, meta, bhc, bhs);
+    c->launches += 1;
     mark();
-    // (b) remaining digits
-    const bool smem_hist = true;
-    const uint32_t skip = smem_hist ? (uint32_t)kSmemSlots : 0u;
-    const uint32_t zslots = std::min<uint32_t>(K, KIMAD_MAX_RATIOS);
-    const dim3 grun((nch + kRunChunks - 1) / kRunChunks, W), gslot(L, W, zslots);
-    k_resolve1<<<glw, blk, 0, s>>>(h1c, h1s, ktab, L, K, cands, slots);
-    mark();
-    k_hist23_smem<2><<<grun, kHThreads, c->hist2_smem, s>>>(dbuf, chunks, nch, c->dstride, L, K, slots, h23c, h23s);
-    if (K > (uint32_t)kSmemSlots) {
-        k_hist23<2, true><<<gch, blk, 0, s>>>(dbuf, chunks, c->dstride, L, K, slots, h23c, h23s, skip);
+    if (R) {
+        k_resolve_a<<<dim3(R, W), kBigThreads, 0, s>>>(layers, reg_layers, R, L, ktab, K, meta, binlo, bhc, bhs, err, tau,
+                                                       keq, shf, flags, fb, fb_chunks, fb_layers);
+        c->launches += 1;
+    }
+    if (T) {
+        k_tiny_exact<<<dim3(T, W), blk, c->tiny_smem, s>>>(dbuf, c->dstride, layers, tiny_layers, L, ktab, K, err, tau, keq,
+                                                           shf, flags);
         c->launches += 1;
     }
     mark();
-    k_resolve23<2><<<gslot, blk, 0, s>>>(h23c, h23s, L, K, cands, slots, err, tau, keq);
-    k_rebuild_slots<<<(W * L + kThreads - 1) / kThreads, blk, 0, s>>>(W * L, K, cands, slots);
-    mark();
-    k_hist23_smem<3><<<grun, kHThreads, c->hist3_smem, s>>>(dbuf, chunks, nch, c->dstride, L, K, slots, h23c, h23s);
-    if (K > (uint32_t)kSmemSlots) {
-        k_hist23<3, true><<<gch, blk, 0, s>>>(dbuf, chunks, c->dstride, L, K, slots, h23c, h23s, skip);
-        c->launches += 1;
+    // exact radix select for the layers handed over by k_resolve_a (the lists are usually empty)
+    if (R) {
+        const uint32_t gfb = 2 * 148, glay = std::min<uint32_t>(W * R, 128u);
+        const dim3 gslot(glay, 1, K);
+        k_fb_hist1<<<gfb, blk, 0, s>>>(dbuf, chunks, c->dstride, L, fb, fb_chunks, h1c, h1s, flags);
+        k_resolve1<<<glay, blk, 0, s>>>(fb, fb_layers, h1c, h1s, ktab, L, K, cands, slots);
+        k_fb_hist23<2><<<gfb, blk, 0, s>>>(dbuf, chunks, c->dstride, L, K, fb, fb_chunks, slots, h23c, h23s);
+        k_resolve23<2><<<gslot, blk, 0, s>>>(fb, fb_layers, h23c, h23s, L, K, cands, slots, err, tau, keq, shf);
+        k_rebuild_slots<<<(W * R + kThreads - 1) / kThreads, blk, 0, s>>>(fb, fb_layers, L, K, cands, slots);
+        k_fb_hist23<3><<<gfb, blk, 0, s>>>(dbuf, chunks, c->dstride, L, K, fb, fb_chunks, slots, h23c, h23s);
+        k_resolve23<3><<<gslot, blk, 0, s>>>(fb, fb_layers, h23c, h23s, L, K, cands, slots, err, tau, keq, shf);
+        c->launches += 7;
     }
     mark();
-    k_resolve23<3><<<gslot, blk, 0, s>>>(h23c, h23s, L, K, cands, slots, err, tau, keq);
-    mark();
-    c->launches += 7;
     // (c)
     for (uint32_t w0 = 0; w0 < W; w0 += kDpWorkersPerLaunch) {
         DpBudgets b{};
@@ -166,8 +219,7 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
         }
         k_dp<<<nw, kDpThreads, c->dp_smem, s>>>(b, w0, W, L, K, c->D, c->bpe, c->full_bytes, c->cap, c->check_finite,
                                                 mode == kGivenJ ? 1 : 0, c->dp_plan, ktab,
-                                                mode == kInjectErr ? err_dev : err, tau, keq, nullptr, j_dev, flags, pd,
-                                                sel,
+                                                mode == kInjectErr ? err_dev : err, tau, keq, shf, j_dev, flags, pd, sel,
                                                 out->k, out->j, out->offs, out->stats);
         c->launches += 1;
     }
@@ -175,9 +227,13 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
     // (d), (e), (f)
     k_sel_count<<<gch, blk, 0, s>>>(dbuf, chunks, nch, c->dstride, L, sel, layers, csel, lowh, recount_n, recount_list);
     mark();
-    k_sel_resolve<<<glw, blk, 0, s>>>(L, layers, lowh, sel);
+    k_sel_resolve<<<glw, blk, 0, s>>>(L, layers, nch, csel, lowh, sel, r2, r2_layers, r2_chunks);
+    k_sel_count_r2<<<2 * 148, blk, 0, s>>>(dbuf, chunks, nch, c->dstride, L, sel, layers, csel, lowh, recount_n,
+                                          recount_list, r2, r2_chunks);
+    k_sel_resolve_r2<<<std::min<uint32_t>(W * L, 128u), blk, 0, s>>>(L, layers, nch, csel, lowh, sel, r2, r2_layers,
+                                                                   r2_chunks);
     k_sel_recount<<<2 * 148, blk, 0, s>>>(dbuf, chunks, nch, c->dstride, L, sel, recount_n, recount_list, ccnt);
-    k_sel_scan<<<glw, blk, 0, s>>>(L, layers, nch, sel, csel, ccnt, cpre, recount_n);
+    k_sel_scan<<<glw, blk, 0, s>>>(L, layers, nch, sel, csel, ccnt, cpre, recount_n, fb, r2);
     mark();
     if (c->value_dtype == 1)
         k_sel_write<true><<<gch, blk, 0, s>>>(dbuf, state, chunks, nch, c->dstride, c->stride, L, sel, layers, ccnt, cpre,
@@ -186,7 +242,7 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
         k_sel_write<false><<<gch, blk, 0, s>>>(dbuf, state, chunks, nch, c->dstride, c->stride, L, sel, layers, ccnt, cpre,
                                                c->cap, out->idx, out->val);
     mark();
-    c->launches += 5;
+    c->launches += 7;
     CUDA_TRY(cudaGetLastError());
     c->last_out = *out;
     c->have_last = true;
@@ -207,7 +263,7 @@ int kimad_create(kimad_ctx** out, const uint64_t* layer_sizes, uint32_t n_layers
     kimad_options o{};
     if (opt) o = *opt;
     if (o.D == 0) o.D = 1000;
-    if (o.D > KIMAD_MAX_D || o.D < n_layers || o.value_dtype > 1 || o.infeasible_policy != 0)
+    if (o.D > KIMAD_MAX_D || o.D < n_layers || o.value_dtype > 1 || o.infeasible_policy != 0 || o.curve_mode > 1)
         return KIMAD_ERR_INVALID_ARG;
     for (uint32_t j = 0; j < n_ratios; ++j) {
         if (!(ratio_grid[j] > 0.0) || ratio_grid[j] > 1.0) return KIMAD_ERR_INVALID_ARG;
@@ -242,6 +298,13 @@ int kimad_create(kimad_ctx** out, const uint64_t* layer_sizes, uint32_t n_layers
             }
             ld.n_chunks = (uint32_t)c->chunks.size() - ld.first_chunk;
             c->layers.push_back(ld);
+            if (n <= (uint64_t)kTinyMax) {
+                c->reg_index.push_back(0xffffffffu);
+                c->tiny_layers.push_back(l);
+            } else {
+                c->reg_index.push_back((uint32_t)c->reg_layers.size());
+                c->reg_layers.push_back(l);
+            }
             N += n;
         }
         c->N = N;
@@ -262,8 +325,10 @@ int kimad_create(kimad_ctx** out, const uint64_t* layer_sizes, uint32_t n_layers
         c->dp_plan.pd_in_smem = used + pd_bytes <= kDpSmemMax ? 1u : 0u;
         if (c->dp_plan.pd_in_smem) used += pd_bytes;
         c->dp_smem = used;
-        c->hist2_smem = (size_t)3 * kSmemSlots * kL23Bins * 4 + 2 * kL1Bins + kSmemSlots * 4;
-        c->hist3_smem = (size_t)kSmemSlots * kL23Bins * 4 + 2 * kL1Bins + kSmemSlots * 4;
+        c->curve_mode = o.curve_mode;
+        c->sample_smem = (size_t)(2 * (1024 + 32) + 32768 + 2048 + 1024 + 2048 + 2048 + 32 + 3 * 128) * 4;
+        c->pass_a_smem = (size_t)(3 * kMaxBins + kMaxRows * 32) * 4 + kL1Bins * 2;
+        c->tiny_smem = (size_t)kTinyMax * (8 + 4);
         plan_layout(c);
     } catch (const std::bad_alloc&) {
         delete c;
@@ -306,11 +371,18 @@ int kimad_set_workspace(kimad_ctx* c, void* dev_ptr, size_t bytes) {
     CUDA_TRY(cudaMemcpy(c->ws + y.chunks, c->chunks.data(), c->chunks.size() * sizeof(Chunk), cudaMemcpyHostToDevice));
     CUDA_TRY(cudaMemcpy(c->ws + y.layers, c->layers.data(), c->layers.size() * sizeof(LayerDesc), cudaMemcpyHostToDevice));
     CUDA_TRY(cudaMemcpy(c->ws + y.ktab, c->ktab.data(), c->ktab.size() * sizeof(uint64_t), cudaMemcpyHostToDevice));
-    // everything after the static tables starts at zero: the histograms are kept clean by the kernels
-    CUDA_TRY(cudaMemset(c->ws + y.h1_cnt, 0, y.total - y.h1_cnt));
+    if (!c->reg_layers.empty())
+        CUDA_TRY(cudaMemcpy(c->ws + y.reg_layers, c->reg_layers.data(), c->reg_layers.size() * 4, cudaMemcpyHostToDevice));
+    if (!c->tiny_layers.empty())
+        CUDA_TRY(cudaMemcpy(c->ws + y.tiny_layers, c->tiny_layers.data(), c->tiny_layers.size() * 4, cudaMemcpyHostToDevice));
+    CUDA_TRY(cudaMemcpy(c->ws + y.reg_index, c->reg_index.data(), c->reg_index.size() * 4, cudaMemcpyHostToDevice));
+    // histograms, work lists and flags start at zero and are kept clean by the kernels that consume them
+    CUDA_TRY(cudaMemset(c->ws + y.zero_from, 0, y.lut_t1 - y.zero_from));
     CUDA_TRY(cudaFuncSetAttribute(k_dp, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->dp_smem));
-    CUDA_TRY(cudaFuncSetAttribute(k_hist23_smem<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->hist2_smem));
-    CUDA_TRY(cudaFuncSetAttribute(k_hist23_smem<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->hist3_smem));
+    CUDA_TRY(cudaFuncSetAttribute(k_sample, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->sample_smem));
+    CUDA_TRY(cudaFuncSetAttribute(k_pass_a<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->pass_a_smem));
+    CUDA_TRY(cudaFuncSetAttribute(k_pass_a<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->pass_a_smem));
+    CUDA_TRY(cudaFuncSetAttribute(k_tiny_exact, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->tiny_smem));
     CUDA_TRY(cudaDeviceSynchronize());
     return KIMAD_OK;
 }
@@ -370,7 +442,8 @@ int kimad_plan_budget(const kimad_ctx* c, double bandwidth_bytes_per_s, double t
     return KIMAD_OK;
 }
 
-int kimad_debug_get_curve(kimad_ctx* c, float* host_err, uint32_t* host_tau, uint32_t* host_keep_eq) {
+int kimad_debug_get_curve(kimad_ctx* c, float* host_err, uint32_t* host_tau, uint32_t* host_keep_eq,
+                          uint32_t* host_shift) {
     if (!c) return KIMAD_ERR_INVALID_ARG;
     if (!c->ws) return KIMAD_ERR_WORKSPACE;
     const size_t n = (size_t)c->W * c->L * c->K;
@@ -378,6 +451,41 @@ int kimad_debug_get_curve(kimad_ctx* c, float* host_err, uint32_t* host_tau, uin
     if (host_err) CUDA_TRY(cudaMemcpy(host_err, c->ws + c->lay.err, n * 4, cudaMemcpyDeviceToHost));
     if (host_tau) CUDA_TRY(cudaMemcpy(host_tau, c->ws + c->lay.tau, n * 4, cudaMemcpyDeviceToHost));
     if (host_keep_eq) CUDA_TRY(cudaMemcpy(host_keep_eq, c->ws + c->lay.keep_eq, n * 4, cudaMemcpyDeviceToHost));
+    if (host_shift) CUDA_TRY(cudaMemcpy(host_shift, c->ws + c->lay.shift, n * 4, cudaMemcpyDeviceToHost));
+    return KIMAD_OK;
+}
+
+int kimad_debug_get_selection(kimad_ctx* c, uint32_t* host_tau, uint32_t* host_keep_eq) {
+    if (!c) return KIMAD_ERR_INVALID_ARG;
+    if (!c->ws) return KIMAD_ERR_WORKSPACE;
+    const size_t n = (size_t)c->W * c->L;
+    std::vector<Sel> sel(n);
+    CUDA_TRY(cudaDeviceSynchronize());
+    CUDA_TRY(cudaMemcpy(sel.data(), c->ws + c->lay.sel, n * sizeof(Sel), cudaMemcpyDeviceToHost));
+    for (size_t i = 0; i < n; ++i) {
+        if (host_tau) host_tau[i] = sel[i].tau;
+        if (host_keep_eq) host_keep_eq[i] = sel[i].keep_eq;
+    }
+    return KIMAD_OK;
+}
+
+int kimad_debug_get_band_meta(kimad_ctx* c, uint32_t* host_meta) {
+    if (!c || !host_meta) return KIMAD_ERR_INVALID_ARG;
+    if (!c->ws) return KIMAD_ERR_WORKSPACE;
+    CUDA_TRY(cudaDeviceSynchronize());
+    CUDA_TRY(cudaMemcpy(host_meta, c->ws + c->lay.meta, (size_t)c->W * c->reg_layers.size() * sizeof(BandMeta),
+                        cudaMemcpyDeviceToHost));
+    return KIMAD_OK;
+}
+
+int kimad_debug_exact_path_layers(kimad_ctx* c, uint64_t* host_count) {
+    if (!c || !host_count) return KIMAD_ERR_INVALID_ARG;
+    if (!c->ws) return KIMAD_ERR_WORKSPACE;
+    FbList f{};
+    CUDA_TRY(cudaDeviceSynchronize());
+    CUDA_TRY(cudaMemcpy(&f, c->ws + c->lay.fb, sizeof(FbList), cudaMemcpyDeviceToHost));
+    host_count[0] = f.total_layers;
+    for (int i = 0; i < 4; ++i) host_count[1 + i] = f.why[i];
     return KIMAD_OK;
 }
 

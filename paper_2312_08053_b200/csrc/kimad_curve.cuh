@@ -1,0 +1,697 @@
+// Stage (a)+(b), fast path: EF21 difference fused with a banded histogram that yields the error curve of
+// every candidate in ONE sweep over the gradients.
+//
+//   k_sample     per (worker, layer): histogram of a stratified sample of |d| over 16-bit key prefixes
+//                ("cells"); for every candidate k_j the cells that can contain the k_j-th largest key
+//                (sample rank +- 6 sigma) form a band.  Band cells are cut into fine bins of 2^shift
+//                keys, everything else into coarse "gap" bins; the mapping key -> bin is a two-level
+//                table (11-bit bin -> row, row x 5 more bits -> bin base and shift).
+//   k_pass_a     the sweep: d = grad - g (written to scratch), bin = table(key(d)), three u32 shared-
+//                memory atomics per element (count, and the exact integer sum of squares in two halves).
+//   k_resolve_a  per (worker, layer): walks the bins from the top, finds the bin that holds every
+//                candidate's threshold, sums the squares below it.  The candidate's error is certified
+//                to 2^-19 relative from the bin's width; if a threshold fell into a gap bin (the sample
+//                mispredicted) or the bound is too loose, the layer is handed to the exact radix path.
+//   k_tiny_exact layers of at most kTinyMax elements are sorted in shared memory instead.
+//   k_fb_*       exact three-digit radix select over the chunks of the layers handed over (rare).
+#pragma once
+#include "kimad_kernels.cuh"
+
+namespace kimad {
+
+constexpr int kTinyMax = 4096;
+constexpr int kFineBins = 12288;                    // fine bins per (worker, layer)
+constexpr int kMaxBins = kL1Bins + 256 + kFineBins; // + gap bins (one per 11-bit bin, plus pieces around bands)
+constexpr int kMaxRows = 128;                       // 11-bit bins that contain band cells
+constexpr int kMaxShift = 15;                       // a fine bin is 2^shift keys wide, at most a whole cell
+constexpr int kSampleUnits = 4095;                  // sample = units of 16 consecutive elements (<= 65520 elements)
+constexpr int kBigThreads = 1024;
+constexpr uint32_t kGapBit = 1u;                    // bin_lo entries carry this bit when the bin is a gap bin
+
+struct BandMeta { // per (worker, regular layer)
+    uint32_t n_bins;
+    uint32_t n_rows;
+    uint32_t flagged; // 1: this layer takes the exact radix path in this step
+    uint32_t _pad;
+};
+
+__device__ __forceinline__ uint32_t hash_u32(uint32_t x) {
+    x ^= x >> 16; x *= 0x7feb352du; x ^= x >> 15; x *= 0x846ca68bu; x ^= x >> 16;
+    return x;
+}
+
+// ------------------------------------------------------------------------------------------------
+// k_sample: one CTA per (regular layer, worker)
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kBigThreads, 1)
+k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint64_t stride,
+         const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ reg_layers, uint32_t R,
+         const uint64_t* __restrict__ ktab, uint32_t K, uint32_t force_exact, uint16_t* __restrict__ lut_t1,
+         uint32_t* __restrict__ lut_t2, uint32_t* __restrict__ bin_lo, BandMeta* __restrict__ meta) {
+    extern __shared__ __align__(16) uint32_t sh[];
+    double* s_sq = reinterpret_cast<double*>(sh); // [1024] squares (cell midpoints) below each thread segment
+    double* s_wd = s_sq + 1024;                   // [32]
+    uint32_t* h32 = sh + 2 * (1024 + 32);         // [32768] two u16 cell counters per word
+    uint32_t* bitmap = h32 + 32768;               // [2048] bit c of word b: cell (b << 5 | c) belongs to a band
+    uint32_t* s_pre = bitmap + 2048;              // [1024] inclusive sample count of the thread segments, from the top
+    uint32_t* s_base = s_pre + 1024;              // [2048] first bin id of every 11-bit bin
+    uint32_t* s_aux = s_base + 2048;              // [2048] row index of split 11-bit bins
+    uint32_t* s_w = s_aux + 2048;                 // [32]
+    uint32_t* s_cb = s_w + 32;                    // [128] per candidate, then per merged group: lowest cell,
+    uint32_t* s_ct = s_cb + 128;                  // [128] highest cell,
+    uint32_t* s_cs = s_ct + 128;                  // [128] shift
+    __shared__ uint32_t s_m, s_flag, s_ng;
+    const uint32_t r = blockIdx.x, w = blockIdx.y;
+    const uint32_t l = reg_layers[r];
+    const size_t wr = (size_t)w * R + r;
+    BandMeta* mt = meta + wr;
+    if (force_exact) {
+        if (threadIdx.x == 0) *mt = BandMeta{0, 0, 1, 0};
+        return;
+    }
+    const LayerDesc ld = layers[l];
+    const uint32_t n = (uint32_t)ld.n;
+    for (int i = threadIdx.x; i < 32768 + 2048; i += kBigThreads) h32[i] = 0;
+    if (threadIdx.x == 0) { s_m = 0; s_flag = 0; s_ng = 0; }
+    __syncthreads();
+
+    // ---- stratified sample of |grad - g|
+    const float* gr = grads + (size_t)w * stride + ld.begin;
+    const float* st = state + (size_t)w * stride + ld.begin;
+    const uint32_t n_units = (n + 15) / 16;
+    const uint32_t m_units = min(n_units, (uint32_t)kSampleUnits);
+    const bool whole = m_units == n_units;
+    const double stratum = (double)n / (double)m_units;
+    uint32_t mine = 0;
+    for (uint32_t i = threadIdx.x >> 4; i < m_units; i += kBigThreads / 16) { // a half-warp reads one unit
+        uint32_t start;
+        if (whole) {
+            start = 16 * i;
+        } else { // unit i somewhere inside stratum i
+            const uint32_t s0 = (uint32_t)((double)i * stratum), s1 = (uint32_t)((double)(i + 1) * stratum);
+            const uint32_t room = s1 > s0 + 16 ? s1 - s0 - 16 : 0;
+            start = s0 + __umulhi(hash_u32(i * 0x9e3779b9u + l * 0x85ebca6bu + 1u), room + 1);
+        }
+        const uint32_t p = start + (threadIdx.x & 15);
+        if (p < n) {
+            const uint32_t cell = key_of(__fsub_rn(gr[p], st[p])) >> 15;
+            atomicAdd(&h32[cell >> 1], 1u << (16 * (cell & 1)));
+            ++mine;
+        }
+    }
+    atomicAdd(&s_m, mine);
+    __syncthreads();
+    const uint32_t m = s_m;
+    auto cell_count = [&](uint32_t cell) { return (h32[cell >> 1] >> (16 * (cell & 1))) & 0xffffu; };
+    auto cell_sq = [&](uint32_t cell) { // square of the cell's middle value (planning only: float range is enough)
+        const float v = __uint_as_float((cell << 15) | 0x4000u);
+        return (double)(v * v);
+    };
+
+    // ---- per thread segment (cells 65535 - 64 t - (0..63)): sample count and squares; the reads of a warp are
+    // rotated so that its lanes hit different banks
+    {
+        uint32_t sum = 0;
+        double sq = 0.0;
+        const uint32_t top = 65535u - 64u * threadIdx.x;
+        for (uint32_t i0 = 0; i0 < 64; ++i0) {
+            const uint32_t i = (i0 + 2 * (threadIdx.x & 31)) & 63;
+            const uint32_t c = cell_count(top - i);
+            sum += c;
+            if (c) sq += (double)c * cell_sq(top - i);
+        }
+        uint32_t tot;
+        double totd;
+        const uint32_t ex = block_excl_scan<uint32_t, kBigThreads>(sum, s_w, &tot);
+        const double exd = block_excl_scan<double, kBigThreads>(sq, s_wd, &totd);
+        s_pre[threadIdx.x] = ex + sum;
+        s_sq[threadIdx.x] = totd - exd - sq; // squares in the segments below this one (higher thread index)
+    }
+    __syncthreads();
+    // cell holding sample rank rk (1-based, from the top)
+    auto cell_of_rank = [&](uint32_t rk) {
+        int lo = 0, hi = kBigThreads - 1;
+        while (lo < hi) { const int mid = (lo + hi) >> 1; if (s_pre[mid] >= rk) hi = mid; else lo = mid + 1; }
+        uint32_t before = lo ? s_pre[lo - 1] : 0u;
+        const uint32_t top = 65535u - 64u * lo;
+        for (uint32_t i = 0; i < 64; ++i) {
+            before += cell_count(top - i);
+            if (before >= rk) return top - i;
+        }
+        return top - 63u;
+    };
+
+    // ---- bands: the cells that can hold the k_j-th largest key, and how finely to cut them
+    if (threadIdx.x < K) {
+        const uint32_t j = threadIdx.x;
+        const uint64_t k = ktab[(size_t)l * K + j];
+        s_cb[j] = 1; s_ct[j] = 0; s_cs[j] = 15; // k == n keeps everything: no threshold, no band
+        if (k < n) {
+            uint32_t r_lo, r_hi;
+            if (whole) {
+                r_lo = r_hi = (uint32_t)k;
+            } else {
+                const double p = (double)k / (double)n;
+                const double rho = p * (double)m, sg = sqrt((double)m * p * (1.0 - p));
+                const double a = floor(rho - 6.0 * sg - 2.0), b = ceil(rho + 6.0 * sg + 2.0);
+                r_lo = a < 1.0 ? 0u : (uint32_t)a;
+                r_hi = b > (double)m ? 0u : (uint32_t)b;
+            }
+            // rank window clipped at the top: the threshold may lie above the largest sample, so the band goes one
+            // octave further up; clipped at the bottom: no bound from the sample, exact path
+            uint32_t c_top = cell_of_rank(max(r_lo, 1u));
+            if (r_lo == 0) c_top = min(c_top + 256u, 65279u);
+            if (r_hi == 0) s_flag = 1;
+            const uint32_t c_bot = cell_of_rank(max(r_hi, 1u));
+            const uint32_t ncell = c_top - c_bot + 1;
+            if (ncell > (uint32_t)kFineBins) {
+                s_flag = 2;
+            } else {
+                uint32_t inband = 0;
+                for (uint32_t c = c_bot; c <= c_top; ++c) inband += cell_count(c);
+                // estimate of this candidate's error: squares of everything below the band
+                const uint32_t seg = (65535u - c_bot) >> 6;
+                double below = s_sq[seg];
+                for (uint32_t c = 65535u - 64u * seg - 63u; c < c_bot; ++c) {
+                    const uint32_t cc = cell_count(c);
+                    if (cc) below += (double)cc * cell_sq(c);
+                }
+                const double scale = (double)n / (double)m;
+                const double per_cell = (double)inband / (double)ncell * scale; // entries per band cell
+                const double v2 = cell_sq(c_top);
+                // bins per cell: at most ~2048 entries per bin (what the select stage collects and sorts), and
+                // narrow enough that the uncertainty of the bin holding the threshold (its entries times its
+                // spread of squares, 2^-7 of v^2 for a whole cell) stays below ~5e-7 of the error
+                double bins = per_cell / 2048.0;
+                const double e_est = below * scale;
+                const double cert = e_est > 0.0 ? sqrt(per_cell * 0.0078125 * v2 / (1.5e-6 * e_est)) : 1024.0;
+                if (cert > bins) bins = cert;
+                uint32_t sh_j = 15;
+                while (sh_j > 5 && (double)(1u << (15 - sh_j)) < bins) --sh_j;
+                s_cb[j] = c_bot; s_ct[j] = c_top; s_cs[j] = sh_j;
+            }
+        }
+    }
+    __syncthreads();
+    // merge overlapping / adjacent bands (they descend in key with j) into groups; groups end up in s_c*[0..ng)
+    if (threadIdx.x == 0 && !s_flag) {
+        uint32_t ng = 0;
+        uint32_t gb = 1, gt = 0, gs = 15;
+        bool open = false;
+        for (uint32_t j = 0; j < K; ++j) {
+            const uint32_t cb = s_cb[j], ct = s_ct[j], cs = s_cs[j];
+            if (cb > ct) continue;
+            if (open && ct + 1 >= gb) {
+                gb = min(gb, cb); gt = max(gt, ct); gs = min(gs, cs);
+            } else {
+                if (open) { s_cb[ng] = gb; s_ct[ng] = gt; s_cs[ng] = gs; ++ng; } // ng <= j: slots already consumed
+                gb = cb; gt = ct; gs = cs; open = true;
+            }
+        }
+        if (open) { s_cb[ng] = gb; s_ct[ng] = gt; s_cs[ng] = gs; ++ng; }
+        // if the fine bins do not fit, scale every group's bins per cell down by the same factor (rounded
+        // down to a power of two, at least one bin per cell)
+        uint64_t fine = 0, cells = 0;
+        for (uint32_t g = 0; g < ng; ++g) {
+            fine += (uint64_t)(s_ct[g] - s_cb[g] + 1) << (15 - s_cs[g]);
+            cells += s_ct[g] - s_cb[g] + 1;
+        }
+        if (cells > (uint64_t)kFineBins) {
+            s_flag = 3;
+        } else if (fine > (uint64_t)kFineBins) {
+            uint32_t extra = 1;
+            while ((fine >> extra) > (uint64_t)kFineBins - cells) ++extra; // groups clamped at shift 15 keep 1 bin per cell
+            for (uint32_t g = 0; g < ng; ++g) s_cs[g] = min(15u, s_cs[g] + extra);
+        }
+        s_ng = ng;
+    }
+    __syncthreads();
+    const uint32_t ng = s_ng;
+    if (!s_flag)
+        for (uint32_t g = 0; g < ng; ++g)
+            for (uint32_t c = s_cb[g] + threadIdx.x; c <= s_ct[g]; c += kBigThreads) atomicOr(&bitmap[c >> 5], 1u << (c & 31));
+    __syncthreads();
+    auto shift_of = [&](uint32_t cell) {
+        for (uint32_t g = 0; g < ng; ++g)
+            if (cell >= s_cb[g] && cell <= s_ct[g]) return s_cs[g];
+        return 15u;
+    };
+
+    // ---- bin ids in ascending key order; thread t owns the 11-bit bins 2t and 2t+1
+    uint32_t word[2], nb[2];
+    uint32_t rows = 0, nbt = 0;
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        word[i] = bitmap[2 * threadIdx.x + i];
+        rows += word[i] != 0;
+        if (word[i]) {
+            const uint32_t z = ~word[i];
+            uint32_t cnt = __popc(z & ~(z << 1)); // gap runs
+            for (uint32_t wd = word[i]; wd; wd &= wd - 1)
+                cnt += 1u << (15 - shift_of(((2 * threadIdx.x + i) << 5) | (__ffs(wd) - 1)));
+            nb[i] = cnt;
+        } else {
+            nb[i] = 1;
+        }
+        nbt += nb[i];
+    }
+    uint32_t tot_rows, tot_bins;
+    const uint32_t ex_rows = block_excl_scan<uint32_t, kBigThreads>(rows, s_w, &tot_rows);
+    const uint32_t ex_bins = block_excl_scan<uint32_t, kBigThreads>(nbt, s_w, &tot_bins);
+    const bool bad = s_flag || tot_rows > (uint32_t)kMaxRows || tot_bins > (uint32_t)kMaxBins;
+    if (bad) {
+        if (threadIdx.x == 0) *mt = BandMeta{tot_bins, tot_rows, 2, s_flag};
+        return;
+    }
+    uint16_t* t1 = lut_t1 + wr * kL1Bins;
+    uint32_t* t2 = lut_t2 + wr * (kMaxRows * 32);
+    uint32_t* blo = bin_lo + wr * (kMaxBins + 1);
+    {
+        uint32_t base = ex_bins, row = ex_rows;
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const uint32_t b1 = 2 * threadIdx.x + i;
+            s_base[b1] = base;
+            if (word[i]) {
+                s_aux[b1] = row;
+                t1[b1] = (uint16_t)(0x8000u | row);
+                ++row;
+            } else {
+                t1[b1] = (uint16_t)base;
+                blo[base] = (b1 << 20) | kGapBit;
+            }
+            base += nb[i];
+        }
+    }
+    __syncthreads();
+    // split bins: one warp per bin, one lane per cell
+    for (uint32_t b1 = threadIdx.x >> 5; b1 < (uint32_t)kL1Bins; b1 += kBigThreads / 32) {
+        const uint32_t wd = bitmap[b1];
+        if (!wd) continue;
+        const uint32_t lane = threadIdx.x & 31;
+        const uint32_t cell = (b1 << 5) | lane;
+        const bool band = (wd >> lane) & 1u;
+        const bool gap_start = !band && (lane == 0 || ((wd >> (lane - 1)) & 1u));
+        const uint32_t shc = band ? shift_of(cell) : 15u;
+        const uint32_t contrib = band ? (1u << (15 - shc)) : (gap_start ? 1u : 0u);
+        uint32_t incl = contrib;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= (uint32_t)o) incl += y;
+        }
+        const uint32_t id = s_base[b1] + (band ? incl - contrib : incl - 1u);
+        t2[s_aux[b1] * 32 + lane] = id | (shc << 16);
+        if (band) {
+            for (uint32_t i = 0; i < contrib; ++i) blo[id + i] = (cell << 15) + (i << shc);
+        } else if (gap_start) {
+            blo[id] = (cell << 15) | kGapBit;
+        }
+    }
+    if (threadIdx.x == 0) {
+        blo[tot_bins] = 0x80000000u;
+        *mt = BandMeta{tot_bins, tot_rows, 0, 0};
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// k_pass_a: CTAs own runs of consecutive chunks; histogram words live in shared memory
+// ------------------------------------------------------------------------------------------------
+constexpr int kRunChunksA = 8;
+
+template <bool VEC>
+__global__ void __launch_bounds__(kBigThreads, 1)
+k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, float* __restrict__ dbuf,
+         const Chunk* __restrict__ chunks, uint32_t n_chunks, uint64_t stride, uint64_t dstride,
+         const uint32_t* __restrict__ reg_index /* [L], 0xffffffff: tiny layer */, uint32_t R,
+         const uint16_t* __restrict__ lut_t1, const uint32_t* __restrict__ lut_t2, const BandMeta* __restrict__ meta,
+         uint32_t* __restrict__ bh_cnt, unsigned long long* __restrict__ bh_sum) {
+    extern __shared__ __align__(16) uint32_t sh[];
+    uint32_t* h_cnt = sh;
+    uint32_t* h_hi = sh + kMaxBins;
+    uint32_t* h_lo = sh + 2 * kMaxBins;
+    uint32_t* t2 = sh + 3 * kMaxBins;                               // [kMaxRows * 32]
+    uint16_t* t1 = reinterpret_cast<uint16_t*>(t2 + kMaxRows * 32); // [2048]
+    static_assert((uint64_t)kRunChunksA * kChunkElems <= (1ull << 18), "u32 sums of 12-bit halves");
+    const uint32_t w = blockIdx.y;
+    const uint32_t c0 = blockIdx.x * kRunChunksA, c1 = min(n_chunks, c0 + kRunChunksA);
+    for (int i = threadIdx.x; i < 3 * kMaxBins; i += kBigThreads) sh[i] = 0;
+    const float* gr0 = grads + (size_t)w * stride;
+    const float* st0 = state + (size_t)w * stride;
+    float* dd0 = dbuf + (size_t)w * dstride;
+    int cur_layer = -1;
+    bool active = false, dirty = false;
+    uint32_t n_bins = 0;
+    uint32_t* gc = nullptr;
+    unsigned long long* gs = nullptr;
+
+    auto flush = [&]() {
+        __syncthreads();
+        for (uint32_t i = threadIdx.x; i < n_bins; i += kBigThreads) {
+            const uint32_t c = h_cnt[i];
+            if (c) {
+                atomicAdd(&gc[i], c);
+                atomicAdd(&gs[i], ((unsigned long long)h_hi[i] << 12) + h_lo[i]);
+                h_cnt[i] = 0; h_hi[i] = 0; h_lo[i] = 0;
+            }
+        }
+        __syncthreads();
+        dirty = false;
+    };
+    auto acc = [&](float dv) {
+        const uint32_t key = key_of(dv);
+        const uint32_t e1 = t1[key >> 20];
+        const bool split = e1 & 0x8000u;
+        const uint32_t e2 = t2[(split ? (e1 & 0x7fffu) : 0u) * 32 + ((key >> 15) & 31u)];
+        const uint32_t id = split ? (e2 & 0xffffu) + ((key & 0x7fffu) >> (e2 >> 16)) : e1;
+        // 24 significant bits of the square (truncation < 2^-22 relative), in two 12-bit halves: a run has at
+        // most 2^18 elements, so neither u32 sum can overflow before the flush at the end of the run
+        const uint32_t sq = (uint32_t)(sq_fixed(key) >> 8);
+        atomicAdd(&h_cnt[id], 1u);
+        atomicAdd(&h_hi[id], sq >> 12);
+        atomicAdd(&h_lo[id], sq & 0xfffu);
+    };
+
+    for (uint32_t c = c0; c < c1; ++c) {
+        const Chunk ch = chunks[c];
+        if ((int)ch.layer != cur_layer) {
+            if (dirty) flush();
+            cur_layer = (int)ch.layer;
+            const uint32_t r = reg_index[ch.layer];
+            active = false;
+            if (r != 0xffffffffu) {
+                const size_t wr = (size_t)w * R + r;
+                const BandMeta mt = meta[wr];
+                if (!mt.flagged) {
+                    active = true;
+                    n_bins = mt.n_bins;
+                    gc = bh_cnt + wr * kMaxBins;
+                    gs = bh_sum + wr * kMaxBins;
+                    __syncthreads();
+                    const uint32_t* g1 = reinterpret_cast<const uint32_t*>(lut_t1 + wr * kL1Bins);
+                    for (int i = threadIdx.x; i < kL1Bins / 2; i += kBigThreads) reinterpret_cast<uint32_t*>(t1)[i] = g1[i];
+                    const uint32_t* g2 = lut_t2 + wr * (kMaxRows * 32);
+                    for (uint32_t i = threadIdx.x; i < mt.n_rows * 32; i += kBigThreads) t2[i] = g2[i];
+                }
+            }
+            __syncthreads();
+        }
+        const ChunkView cv(ch);
+        const float* gr = gr0 + cv.a0;
+        const float* st = st0 + cv.a0;
+        float* dd = dd0 + cv.a0;
+        const uint32_t nq = cv.quads();
+        constexpr int U = 2;
+        for (uint32_t qb = 0; qb < nq; qb += kBigThreads * U) {
+            float4 a[U], b[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const uint32_t q = qb + u * kBigThreads + threadIdx.x;
+                if (VEC && q < nq && cv.quad_full(q)) {
+                    a[u] = __ldcs(reinterpret_cast<const float4*>(gr) + q);
+                    b[u] = __ldcs(reinterpret_cast<const float4*>(st) + q);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const uint32_t q = qb + u * kBigThreads + threadIdx.x;
+                if (q >= nq) continue;
+                if (VEC && cv.quad_full(q)) {
+                    float4 d;
+                    d.x = __fsub_rn(a[u].x, b[u].x); d.y = __fsub_rn(a[u].y, b[u].y);
+                    d.z = __fsub_rn(a[u].z, b[u].z); d.w = __fsub_rn(a[u].w, b[u].w);
+                    reinterpret_cast<float4*>(dd)[q] = d;
+                    if (active) { acc(d.x); acc(d.y); acc(d.z); acc(d.w); }
+                } else {
+                    for (uint32_t e = 4 * q; e < 4 * q + 4; ++e)
+                        if (e >= cv.first && e < cv.len) {
+                            const float d = __fsub_rn(gr[e], st[e]);
+                            dd[e] = d;
+                            if (active) acc(d);
+                        }
+                }
+            }
+        }
+        if (active) dirty = true;
+    }
+    if (dirty) flush();
+}
+
+// ------------------------------------------------------------------------------------------------
+// k_resolve_a: one CTA per (regular layer, worker)
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kBigThreads)
+k_resolve_a(const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ reg_layers, uint32_t R, uint32_t L,
+            const uint64_t* __restrict__ ktab, uint32_t K, const BandMeta* __restrict__ meta,
+            const uint32_t* __restrict__ bin_lo, uint32_t* __restrict__ bh_cnt, unsigned long long* __restrict__ bh_sum,
+            float* __restrict__ err_out, uint32_t* __restrict__ tau_out, uint32_t* __restrict__ rank_out,
+            uint32_t* __restrict__ shift_out, uint32_t* __restrict__ flags, FbList* __restrict__ fb,
+            uint2* __restrict__ fb_chunks, uint2* __restrict__ fb_layers) {
+    __shared__ uint32_t s_drop[KIMAD_MAX_RATIOS]; // entries not kept by candidate j: n - k_j
+    __shared__ uint32_t s_bin[KIMAD_MAX_RATIOS], s_before[KIMAD_MAX_RATIOS], s_cb[KIMAD_MAX_RATIOS];
+    __shared__ double s_below[KIMAD_MAX_RATIOS], s_sb[KIMAD_MAX_RATIOS];
+    __shared__ uint32_t s_w32[32];
+    __shared__ double s_w64[32];
+    __shared__ int s_bad;
+    const uint32_t r = blockIdx.x, w = blockIdx.y;
+    const uint32_t l = reg_layers[r];
+    const size_t wr = (size_t)w * R + r, wl = (size_t)w * L + l;
+    const BandMeta mt = meta[wr];
+    const LayerDesc ld = layers[l];
+    if (threadIdx.x == 0) s_bad = mt.flagged;
+    if (threadIdx.x < K) {
+        const uint64_t k = ktab[(size_t)l * K + threadIdx.x];
+        s_drop[threadIdx.x] = (uint32_t)(ld.n - k);
+        s_bin[threadIdx.x] = 0xffffffffu;
+    }
+    __syncthreads();
+    if (!mt.flagged) {
+        const uint32_t nb = mt.n_bins;
+        const uint32_t* blo = bin_lo + wr * (kMaxBins + 1);
+        uint32_t* gc = bh_cnt + wr * kMaxBins;
+        unsigned long long* gs = bh_sum + wr * kMaxBins;
+        uint32_t run_c = 0;   // entries in the bins swept so far (ascending keys)
+        double run_s = 0.0;   // their squares
+        bool nonfinite = false;
+        for (uint32_t base = 0; base < nb; base += kBigThreads) {
+            const uint32_t b = base + threadIdx.x;
+            uint32_t c = 0;
+            double sv = 0.0;
+            if (b < nb) {
+                c = gc[b];
+                const uint32_t klo = blo[b];
+                sv = (double)gs[b] * (256.0 * sq_scale(klo >> 23)); // the sweep summed squares in units of 2^8 sq_fixed
+                if (c) { gc[b] = 0; gs[b] = 0ull; }                    // clean for the next step
+                nonfinite |= c && klo >= 0x7f800000u;
+            }
+            uint32_t tc;
+            double ts;
+            const uint32_t before = run_c + block_excl_scan<uint32_t, kBigThreads>(c, s_w32, &tc);
+            const double below = run_s + block_excl_scan<double, kBigThreads>(sv, s_w64, &ts);
+            if (c)
+                for (uint32_t j = 0; j < K; ++j) { // the bin where the running count passes n - k_j holds the threshold
+                    const uint32_t dj = s_drop[j];
+                    if (dj >= before && dj - before < c) {
+                        s_bin[j] = b; s_before[j] = before; s_cb[j] = c; s_below[j] = below; s_sb[j] = sv;
+                    }
+                }
+            run_c += tc;
+            run_s += ts;
+        }
+        if (nonfinite) atomicOr(&flags[w], 1u);
+        __syncthreads();
+        for (uint32_t j = threadIdx.x; j < K; j += kBigThreads) {
+            const size_t o = wl * K + j;
+            if (s_drop[j] == 0) { // everything kept
+                err_out[o] = 0.f; tau_out[o] = 0; rank_out[o] = 0; shift_out[o] = 0;
+                continue;
+            }
+            const uint32_t bin = s_bin[j];
+            if (bin == 0xffffffffu || (blo[bin] & kGapBit)) { atomicMax(&s_bad, 3); continue; } // outside its band
+            const uint32_t klo = blo[bin], width = (blo[bin + 1] & ~kGapBit) - klo;
+            const uint32_t cb = s_cb[j];
+            const uint32_t drop = s_drop[j] - s_before[j]; // entries of the bin that are not kept, < cb
+            const double vlo = (double)__uint_as_float(klo);
+            // the dropped entries are the `drop` smallest of the bin: their squares sum to something in
+            // [drop * vlo^2, drop * mean]; take the midpoint and certify the half-width
+            const double upper = s_sb[j] * ((double)drop / (double)cb);
+            const double lower = (double)drop * vlo * vlo;
+            double part = 0.5 * (upper + lower), slack = 0.5 * (upper - lower);
+            if (drop == 0 || width == 1) { part = lower; slack = 0.0; }
+            const double e = s_below[j] + part;
+            if (slack > e * 5e-6) { atomicMax(&s_bad, 4); continue; } // acceptance bound on the curve is 1e-5
+            err_out[o] = (float)e;
+            tau_out[o] = klo;
+            rank_out[o] = cb - drop;
+            shift_out[o] = 31 - __clz(width);
+        }
+    }
+    __syncthreads();
+    const int bad = s_bad;
+    if (bad) { // hand the layer and its chunks to the exact path
+        __shared__ uint32_t s_at;
+        if (threadIdx.x == 0) {
+            s_at = atomicAdd(&fb->n_chunks, ld.n_chunks);
+            fb_layers[atomicAdd(&fb->n_layers, 1u)] = make_uint2(w, l);
+            atomicAdd(&fb->total_layers, 1u);
+            atomicAdd(&fb->why[bad - 1], 1u);
+        }
+        __syncthreads();
+        for (uint32_t i = threadIdx.x; i < ld.n_chunks; i += kBigThreads) fb_chunks[s_at + i] = make_uint2(w, ld.first_chunk + i);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// k_tiny_exact: layers of at most kTinyMax elements, sorted in shared memory (one CTA each)
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads)
+k_tiny_exact(const float* __restrict__ dbuf, uint64_t dstride, const LayerDesc* __restrict__ layers,
+             const uint32_t* __restrict__ tiny_layers, uint32_t L, const uint64_t* __restrict__ ktab, uint32_t K,
+             float* __restrict__ err_out, uint32_t* __restrict__ tau_out, uint32_t* __restrict__ rank_out,
+             uint32_t* __restrict__ shift_out, uint32_t* __restrict__ flags) {
+    extern __shared__ __align__(16) unsigned char tiny_smem[];
+    double* s_suf = reinterpret_cast<double*>(tiny_smem);                // [kTinyMax] squares of the entries ranked >= i
+    uint32_t* s_key = reinterpret_cast<uint32_t*>(s_suf + kTinyMax);     // [kTinyMax]
+    __shared__ double s_w64[8];
+    const uint32_t l = tiny_layers[blockIdx.x], w = blockIdx.y;
+    const LayerDesc ld = layers[l];
+    const uint32_t n = (uint32_t)ld.n;
+    const float* dd = dbuf + (size_t)w * dstride + ld.begin;
+    uint32_t np = 1;
+    while (np < n) np <<= 1;
+    bool nonfinite = false;
+    for (uint32_t i = threadIdx.x; i < np; i += kThreads) {
+        const uint32_t key = i < n ? key_of(dd[i]) : 0u;
+        nonfinite |= key >= 0x7f800000u;
+        s_key[i] = key;
+    }
+    if (nonfinite) atomicOr(&flags[w], 1u);
+    __syncthreads();
+    for (uint32_t size = 2; size <= np; size <<= 1)       // bitonic sort, descending
+        for (uint32_t str = size >> 1; str > 0; str >>= 1) {
+            for (uint32_t i = threadIdx.x; i < np / 2; i += kThreads) {
+                const uint32_t a = 2 * i - (i & (str - 1)), b = a + str;
+                const bool desc = (a & size) == 0;
+                const uint32_t ka = s_key[a], kb = s_key[b];
+                if ((ka < kb) == desc) { s_key[a] = kb; s_key[b] = ka; }
+            }
+            __syncthreads();
+        }
+    // suffix sums of squares, smallest magnitudes first: position q = n-1-i runs over ascending magnitude
+    constexpr int PER = kTinyMax / kThreads;
+    double loc[PER];
+    double sum = 0.0;
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+        const uint32_t q = threadIdx.x * PER + i; // q-th smallest
+        double v = 0.0;
+        if (q < n) v = (double)__uint_as_float(s_key[n - 1 - q]);
+        loc[i] = v * v;
+        sum += loc[i];
+    }
+    double run = block_excl_scan<double>(sum, s_w64, nullptr);
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+        const uint32_t q = threadIdx.x * PER + i;
+        run += loc[i];
+        if (q < n) s_suf[n - 1 - q] = run; // squares of the ranks >= n-1-q
+    }
+    __syncthreads();
+    const size_t wl = (size_t)w * L + l;
+    for (uint32_t j = threadIdx.x; j < K; j += kThreads) {
+        const uint32_t k = (uint32_t)ktab[(size_t)l * K + j];
+        const size_t o = wl * K + j;
+        const uint32_t t = s_key[k - 1];
+        int lo = 0, hi = (int)k - 1; // first rank whose key equals t
+        while (lo < hi) { const int mid = (lo + hi) >> 1; if (s_key[mid] == t) hi = mid; else lo = mid + 1; }
+        err_out[o] = k < n ? (float)s_suf[k] : 0.f;
+        tau_out[o] = t;
+        rank_out[o] = k - (uint32_t)lo;
+        shift_out[o] = 0;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// exact radix path over the handed-over chunks (global atomics: the list is short or empty)
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads)
+k_fb_hist1(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks, uint64_t dstride, uint32_t L,
+           const FbList* __restrict__ fb, const uint2* __restrict__ fb_chunks, uint32_t* __restrict__ g_cnt,
+           unsigned long long* __restrict__ g_ss, uint32_t* __restrict__ flags) {
+    __shared__ uint32_t s_cnt[kL1Bins], s_hi[kL1Bins], s_lo[kL1Bins];
+    const uint32_t n = fb->n_chunks;
+    for (uint32_t it = blockIdx.x; it < n; it += gridDim.x) {
+        const uint2 e = fb_chunks[it];
+        const Chunk ch = chunks[e.y];
+        const ChunkView cv(ch);
+        const float* dd = dbuf + (size_t)e.x * dstride + cv.a0;
+        for (int b = threadIdx.x; b < kL1Bins; b += kThreads) { s_cnt[b] = 0; s_hi[b] = 0; s_lo[b] = 0; }
+        __syncthreads();
+        for (uint32_t x = cv.first + threadIdx.x; x < cv.len; x += kThreads) {
+            const uint32_t key = key_of(dd[x]);
+            const uint32_t sq = (uint32_t)sq_fixed(key);
+            atomicAdd(&s_cnt[key >> 20], 1u);
+            atomicAdd(&s_hi[key >> 20], sq >> 16);
+            atomicAdd(&s_lo[key >> 20], sq & 0xffffu);
+            if (key >= 0x7f800000u) atomicOr(&flags[e.x], 1u);
+        }
+        __syncthreads();
+        uint32_t* gc = g_cnt + ((size_t)e.x * L + ch.layer) * kL1Bins;
+        unsigned long long* gs = g_ss + ((size_t)e.x * L + ch.layer) * kL1Bins;
+        for (int b = threadIdx.x; b < kL1Bins; b += kThreads)
+            if (s_cnt[b]) {
+                atomicAdd(&gc[b], s_cnt[b]);
+                atomicAdd(&gs[b], ((unsigned long long)s_hi[b] << 16) + s_lo[b]);
+            }
+        __syncthreads();
+    }
+}
+
+template <int LEVEL>
+__global__ void __launch_bounds__(kThreads)
+k_fb_hist23(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks, uint64_t dstride, uint32_t L, uint32_t K,
+            const FbList* __restrict__ fb, const uint2* __restrict__ fb_chunks, const SlotTab* __restrict__ slots,
+            uint32_t* __restrict__ g_cnt, unsigned long long* __restrict__ g_ss) {
+    __shared__ uint8_t s_first[kL1Bins]; // level-1 bin -> first slot whose prefix starts with it (0xff: none)
+    __shared__ uint8_t s_num[kL1Bins];   // ... and how many consecutive slots share that bin (level 3)
+    __shared__ uint32_t s_prefix[KIMAD_MAX_RATIOS];
+    const uint32_t n = fb->n_chunks;
+    for (uint32_t it = blockIdx.x; it < n; it += gridDim.x) {
+        const uint2 e = fb_chunks[it];
+        const Chunk ch = chunks[e.y];
+        const size_t wl = (size_t)e.x * L + ch.layer;
+        const SlotTab& stab = slots[wl];
+        const uint32_t ns = stab.n;
+        for (int b = threadIdx.x; b < kL1Bins; b += kThreads) { s_first[b] = 0xff; s_num[b] = 0; }
+        for (uint32_t s = threadIdx.x; s < ns; s += kThreads) s_prefix[s] = stab.prefix[s];
+        __syncthreads();
+        if (threadIdx.x == 0)
+            for (uint32_t s = 0; s < ns; ++s) {
+                const uint32_t b1 = LEVEL == 2 ? s_prefix[s] : (s_prefix[s] >> 10);
+                if (s_first[b1] == 0xff) s_first[b1] = (uint8_t)s;
+                s_num[b1]++;
+            }
+        __syncthreads();
+        const ChunkView cv(ch);
+        const float* dd = dbuf + (size_t)e.x * dstride + cv.a0;
+        uint32_t* gc = g_cnt + wl * K * kL23Bins;
+        unsigned long long* gs = g_ss + wl * K * kL23Bins;
+        for (uint32_t x = cv.first + threadIdx.x; x < cv.len; x += kThreads) {
+            const uint32_t key = key_of(dd[x]);
+            const uint32_t f = s_first[key >> 20];
+            if (f == 0xff) continue;
+            if (LEVEL == 2) {
+                const uint32_t bin = (key >> 10) & 1023u;
+                atomicAdd(&gc[(size_t)f * kL23Bins + bin], 1u);
+                atomicAdd(&gs[(size_t)f * kL23Bins + bin], (unsigned long long)sq_fixed(key));
+            } else {
+                const uint32_t nn = s_num[key >> 20], p21 = key >> 10;
+                for (uint32_t s = f; s < f + nn; ++s)
+                    if (s_prefix[s] == p21) { atomicAdd(&gc[(size_t)s * kL23Bins + (key & 1023u)], 1u); break; }
+            }
+        }
+        __syncthreads();
+    }
+}
+
+} // namespace kimad

@@ -26,11 +26,22 @@ constexpr int kL23Bins = 1024; // 10 bits each
 
 __device__ __forceinline__ uint32_t key_of(float d) { return __float_as_uint(d) & 0x7fffffffu; }
 
+// Aligned view of a chunk for 128-bit loads: quads start at a0 = begin & ~3; only the first and the
+// last quad can be partial.  All offsets are 32-bit and relative to a0.
+struct ChunkView {
+    uint64_t a0;
+    uint32_t first, len; // valid element offsets are [first, len)
+    __device__ __forceinline__ explicit ChunkView(const Chunk& ch)
+        : a0(ch.begin & ~3ull), first((uint32_t)(ch.begin - (ch.begin & ~3ull))), len((uint32_t)(ch.end - (ch.begin & ~3ull))) {}
+    __device__ __forceinline__ uint32_t quads() const { return (len + 3) >> 2; }
+    __device__ __forceinline__ bool quad_full(uint32_t q) const { return 4 * q >= first && 4 * q + 4 <= len; }
+};
+
 // ------------------------------------------------------------------------------------------------
 // block-wide exclusive scans (256 threads), result valid in every thread; `total` optional
 // ------------------------------------------------------------------------------------------------
-template <typename T>
-__device__ __forceinline__ T block_excl_scan(T v, T* s_warp /* [8] */, T* total) {
+template <typename T, int NT = kThreads>
+__device__ __forceinline__ T block_excl_scan(T v, T* s_warp /* [NT / 32] */, T* total) {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     T x = v;
 #pragma unroll
@@ -43,7 +54,7 @@ __device__ __forceinline__ T block_excl_scan(T v, T* s_warp /* [8] */, T* total)
     __syncthreads();
     T base = 0, tot = 0;
 #pragma unroll
-    for (int i = 0; i < kThreads / 32; ++i) {
+    for (int i = 0; i < NT / 32; ++i) {
         T t = s_warp[i];
         if (i < wid) base += t;
         tot += t;
@@ -65,91 +76,9 @@ __device__ __forceinline__ uint64_t sq_fixed(uint32_t key) {
     return ((uint64_t)M * (uint64_t)M) >> 16;
 }
 // scale that turns a bin's integer sum back into a sum of squared values; e = exponent field of the bin
-__device__ __forceinline__ double sq_scale(uint32_t e) { return ldexp(1.0, 2 * ((int)(e ? e : 1u) - 150) + 16); }
-
-// Shared-memory histogram words are u32 (native shared atomics): per bin a count, and the sum of
-// sq_fixed split into its high and low 16 bits.  A bin that received at most 2^16 entries since the
-// last flush cannot overflow either sum.
-struct L1Acc {
-    uint32_t* cnt;
-    uint32_t* hi;
-    uint32_t* lo;
-    uint32_t nonfinite;
-    __device__ __forceinline__ void add(float dv) {
-        const uint32_t key = key_of(dv);
-        const uint32_t sq = (uint32_t)sq_fixed(key);
-        const uint32_t b = key >> 20;
-        atomicAdd(&cnt[b], 1u);
-        atomicAdd(&hi[b], sq >> 16);
-        atomicAdd(&lo[b], sq & 0xffffu);
-        nonfinite |= ((key >> 23) == 255u);
-    }
-};
-
-template <bool VEC>
-__global__ void __launch_bounds__(kThreads)
-k_diff_hist1(const float* __restrict__ grads, const float* __restrict__ state, float* __restrict__ dbuf,
-             const Chunk* __restrict__ chunks, uint64_t stride, uint64_t dstride, uint32_t L,
-             uint32_t* __restrict__ g_cnt, unsigned long long* __restrict__ g_ss, uint32_t* __restrict__ flags) {
-    __shared__ uint32_t s_cnt[kL1Bins], s_hi[kL1Bins], s_lo[kL1Bins];
-    const Chunk ch = chunks[blockIdx.x];
-    const uint32_t w = blockIdx.y;
-    for (int b = threadIdx.x; b < kL1Bins; b += kThreads) { s_cnt[b] = 0; s_hi[b] = 0; s_lo[b] = 0; }
-    __syncthreads();
-    const float* gr = grads + (size_t)w * stride;
-    const float* st = state + (size_t)w * stride;
-    float* dd = dbuf + (size_t)w * dstride;
-    L1Acc acc{s_cnt, s_hi, s_lo, 0u};
-
-    const uint64_t q0 = ch.begin & ~3ull;
-    constexpr int U = 4;
-    for (uint64_t base = q0; base < ch.end; base += (uint64_t)4 * kThreads * U) {
-        float4 a[U], b[U];
-        bool full[U];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const uint64_t q = base + 4ull * (threadIdx.x + (uint64_t)u * kThreads);
-            full[u] = VEC && q >= ch.begin && q + 4 <= ch.end;
-            if (full[u]) {
-                a[u] = __ldcs(reinterpret_cast<const float4*>(gr + q));
-                b[u] = __ldcs(reinterpret_cast<const float4*>(st + q));
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const uint64_t q = base + 4ull * (threadIdx.x + (uint64_t)u * kThreads);
-            if (full[u]) {
-                float4 r;
-                r.x = __fsub_rn(a[u].x, b[u].x);
-                r.y = __fsub_rn(a[u].y, b[u].y);
-                r.z = __fsub_rn(a[u].z, b[u].z);
-                r.w = __fsub_rn(a[u].w, b[u].w);
-                *reinterpret_cast<float4*>(dd + q) = r;
-                acc.add(r.x); acc.add(r.y); acc.add(r.z); acc.add(r.w);
-            } else if (q < ch.end) {
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const uint64_t p = q + i;
-                    if (p >= ch.begin && p < ch.end) {
-                        const float r = __fsub_rn(gr[p], st[p]);
-                        dd[p] = r;
-                        acc.add(r);
-                    }
-                }
-            }
-        }
-    }
-    if (acc.nonfinite) atomicOr(&flags[w], 1u);
-    __syncthreads();
-    uint32_t* gc = g_cnt + ((size_t)w * L + ch.layer) * kL1Bins;
-    unsigned long long* gs = g_ss + ((size_t)w * L + ch.layer) * kL1Bins;
-    for (int b = threadIdx.x; b < kL1Bins; b += kThreads) {
-        const uint32_t c = s_cnt[b];
-        if (c) {
-            atomicAdd(&gc[b], c);
-            atomicAdd(&gs[b], ((unsigned long long)s_hi[b] << 16) + s_lo[b]);
-        }
-    }
+__device__ __forceinline__ double sq_scale(uint32_t e) { // 2^(2 (max(e,1) - 150) + 16), always a normal double
+    const int x = 2 * ((int)(e ? e : 1u) - 150) + 16;
+    return __longlong_as_double((long long)(x + 1023) << 52);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -205,22 +134,42 @@ __device__ __forceinline__ int find_pos(const uint32_t* s_incl, uint32_t rank) {
     return lo;
 }
 
+// The exact radix kernels below run over the list of layers handed over in this step (usually empty).
+struct FbList { // layers handed to the exact radix path in this step, and their chunks
+    uint32_t n_chunks;
+    uint32_t n_layers;
+    uint32_t total_layers; // never reset: how many layers were handed over since the workspace was attached
+    uint32_t why[5];       // never reset: ... because 0: forced, 1: bands too wide for the tables, 2: threshold
+                           // outside its band, 3: error bound too loose
+};
+
 __global__ void __launch_bounds__(kThreads)
-k_resolve1(uint32_t* __restrict__ g_cnt, unsigned long long* __restrict__ g_ss, const uint64_t* __restrict__ ktab,
-           uint32_t L, uint32_t K, Cand* __restrict__ cands, SlotTab* __restrict__ slots) {
+k_resolve1(const FbList* __restrict__ fb, const uint2* __restrict__ fb_layers, uint32_t* __restrict__ g_cnt,
+           unsigned long long* __restrict__ g_ss, const uint64_t* __restrict__ ktab, uint32_t L, uint32_t K,
+           Cand* __restrict__ cands, SlotTab* __restrict__ slots) {
     __shared__ __align__(16) uint32_t s_incl[kL1Bins];
     __shared__ __align__(16) double s_below[kL1Bins];
     __shared__ uint32_t s_w32[8];
     __shared__ double s_w64[8];
-    const uint32_t l = blockIdx.x, w = blockIdx.y;
+  for (uint32_t it = blockIdx.x; it < fb->n_layers; it += gridDim.x) {
+    const uint32_t l = fb_layers[it].y, w = fb_layers[it].x;
     const size_t wl = (size_t)w * L + l;
     uint32_t* gc = g_cnt + wl * kL1Bins;
     unsigned long long* gs = g_ss + wl * kL1Bins;
-    for (int b = threadIdx.x; b < kL1Bins; b += kThreads) {
-        s_incl[kL1Bins - 1 - b] = gc[b];
-        s_below[b] = (double)gs[b] * sq_scale((uint32_t)b >> 3);
-        gc[b] = 0; // leave the histogram clean for the next step
-        gs[b] = 0ull;
+    {
+        constexpr int PER = kL1Bins / kThreads;
+        uint32_t c[PER];
+        unsigned long long g[PER];
+#pragma unroll
+        for (int i = 0; i < PER; ++i) { c[i] = gc[threadIdx.x + i * kThreads]; g[i] = gs[threadIdx.x + i * kThreads]; }
+#pragma unroll
+        for (int i = 0; i < PER; ++i) {
+            const int b = threadIdx.x + i * kThreads;
+            s_incl[kL1Bins - 1 - b] = c[i];
+            s_below[b] = (double)g[i] * sq_scale((uint32_t)b >> 3);
+            gc[b] = 0; // leave the histogram clean for the next step
+            gs[b] = 0ull;
+        }
     }
     __syncthreads();
     scan_bins<kL1Bins>(s_incl, s_below, s_w32, s_w64);
@@ -247,37 +196,53 @@ k_resolve1(uint32_t* __restrict__ g_cnt, unsigned long long* __restrict__ g_ss, 
         }
         stab.n = ns;
     }
+    __syncthreads();
+  }
 }
 
 // LEVEL 2: refine inside a level-1 bin; LEVEL 3: inside a (level-1, level-2) bin.
 // One CTA per (layer, worker, slot).
 template <int LEVEL>
 __global__ void __launch_bounds__(kThreads)
-k_resolve23(uint32_t* __restrict__ g_cnt, unsigned long long* __restrict__ g_ss, uint32_t L, uint32_t K,
-            Cand* __restrict__ cands, const SlotTab* __restrict__ slots, float* __restrict__ err_out,
-            uint32_t* __restrict__ tau_out, uint32_t* __restrict__ keep_eq_out) {
+k_resolve23(const FbList* __restrict__ fb, const uint2* __restrict__ fb_layers, uint32_t* __restrict__ g_cnt,
+            unsigned long long* __restrict__ g_ss, uint32_t L, uint32_t K, Cand* __restrict__ cands,
+            const SlotTab* __restrict__ slots, float* __restrict__ err_out, uint32_t* __restrict__ tau_out,
+            uint32_t* __restrict__ keep_eq_out, uint32_t* __restrict__ shift_out) {
     __shared__ __align__(16) uint32_t s_incl[kL23Bins];
     __shared__ __align__(16) double s_below[kL23Bins];
     __shared__ uint32_t s_w32[8];
     __shared__ double s_w64[8];
-    const uint32_t l = blockIdx.x, w = blockIdx.y, s = blockIdx.z;
+  for (uint32_t it = blockIdx.x; it < fb->n_layers; it += gridDim.x) {
+    const uint32_t l = fb_layers[it].y, w = fb_layers[it].x, s = blockIdx.z;
     const size_t wl = (size_t)w * L + l;
     const SlotTab& stab = slots[wl];
-    if (s >= stab.n) return;
+    if (s >= stab.n) continue;
     Cand* cd = cands + wl * K;
     uint32_t* gc = g_cnt + (wl * K + s) * kL23Bins;
     unsigned long long* gs = g_ss + (wl * K + s) * kL23Bins;
     const uint32_t prefix = stab.prefix[s];
-    for (int b = threadIdx.x; b < kL23Bins; b += kThreads) {
-        const uint32_t c = gc[b];
-        s_incl[kL23Bins - 1 - b] = c;
-        gc[b] = 0;
-        if (LEVEL == 2) { // prefix = level-1 bin: 8 exponent bits + 3 mantissa bits
-            s_below[b] = (double)gs[b] * sq_scale(prefix >> 3);
-            gs[b] = 0ull;
-        } else { // all 31 bits known: the bin's sum of squares is count * value^2
-            const double v = (double)__uint_as_float((prefix << 10) | (uint32_t)b);
-            s_below[b] = (double)c * v * v;
+    {
+        constexpr int PER = kL23Bins / kThreads;
+        uint32_t cc[PER];
+        unsigned long long g[PER];
+#pragma unroll
+        for (int i = 0; i < PER; ++i) {
+            cc[i] = gc[threadIdx.x + i * kThreads];
+            g[i] = LEVEL == 2 ? gs[threadIdx.x + i * kThreads] : 0ull;
+        }
+        const double scale = sq_scale(prefix >> 3); // LEVEL 2: prefix = level-1 bin (8 exponent + 3 mantissa bits)
+#pragma unroll
+        for (int i = 0; i < PER; ++i) {
+            const int b = threadIdx.x + i * kThreads;
+            s_incl[kL23Bins - 1 - b] = cc[i];
+            gc[b] = 0;
+            if (LEVEL == 2) {
+                s_below[b] = (double)g[i] * scale;
+                gs[b] = 0ull;
+            } else { // all 31 bits known: the bin's sum of squares is count * value^2
+                const double v = (double)__uint_as_float((prefix << 10) | (uint32_t)b);
+                s_below[b] = (double)cc[i] * v * v;
+            }
         }
     }
     __syncthreads();
@@ -302,15 +267,20 @@ k_resolve23(uint32_t* __restrict__ g_cnt, unsigned long long* __restrict__ g_ss,
             err_out[wl * K + j] = (float)e;
             tau_out[wl * K + j] = c.prefix;
             keep_eq_out[wl * K + j] = keep;
+            shift_out[wl * K + j] = 0;
         }
     }
+    __syncthreads();
+  }
 }
 
 // After digit 2: new slots = distinct 21-bit prefixes (non-increasing in j).  One thread per (worker, layer).
 __global__ void __launch_bounds__(kThreads)
-k_rebuild_slots(uint32_t WL, uint32_t K, Cand* __restrict__ cands, SlotTab* __restrict__ slots) {
-    const uint32_t wl = blockIdx.x * kThreads + threadIdx.x;
-    if (wl >= WL) return;
+k_rebuild_slots(const FbList* __restrict__ fb, const uint2* __restrict__ fb_layers, uint32_t L, uint32_t K,
+                Cand* __restrict__ cands, SlotTab* __restrict__ slots) {
+    const uint32_t it = blockIdx.x * kThreads + threadIdx.x;
+    if (it >= fb->n_layers) return;
+    const size_t wl = (size_t)fb_layers[it].x * L + fb_layers[it].y;
     Cand* cd = cands + (size_t)wl * K;
     SlotTab& stab = slots[wl];
     uint32_t n2 = 0;
@@ -320,217 +290,6 @@ k_rebuild_slots(uint32_t WL, uint32_t K, Cand* __restrict__ cands, SlotTab* __re
         cd[j].slot = n2 - 1;
     }
     stab.n = n2;
-}
-
-// level-2 / level-3 histograms over the materialised difference
-template <int LEVEL, bool VEC>
-__global__ void __launch_bounds__(kThreads)
-k_hist23(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks, uint64_t dstride, uint32_t L,
-         uint32_t K, const SlotTab* __restrict__ slots, uint32_t* __restrict__ g_cnt,
-         unsigned long long* __restrict__ g_ss, uint32_t skip_up_to_slots) {
-    __shared__ uint8_t s_first[kL1Bins]; // level-1 bin -> first slot whose prefix starts with it (0xff: none)
-    __shared__ uint8_t s_num[kL1Bins];   // ... and how many consecutive slots share that bin (level 3)
-    __shared__ uint32_t s_prefix[KIMAD_MAX_RATIOS];
-    const Chunk ch = chunks[blockIdx.x];
-    const uint32_t w = blockIdx.y;
-    const size_t wl = (size_t)w * L + ch.layer;
-    const SlotTab& stab = slots[wl];
-    const uint32_t ns = stab.n;
-    if (ns <= skip_up_to_slots) return; // those layers belong to k_hist23_smem
-    for (int b = threadIdx.x; b < kL1Bins; b += kThreads) { s_first[b] = 0xff; s_num[b] = 0; }
-    for (uint32_t s = threadIdx.x; s < ns; s += kThreads) s_prefix[s] = stab.prefix[s];
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        for (uint32_t s = 0; s < ns; ++s) {
-            const uint32_t b1 = LEVEL == 2 ? s_prefix[s] : (s_prefix[s] >> 10);
-            if (s_first[b1] == 0xff) s_first[b1] = (uint8_t)s;
-            s_num[b1]++;
-        }
-    }
-    __syncthreads();
-    const float* dd = dbuf + (size_t)w * dstride;
-    uint32_t* gc = g_cnt + wl * K * kL23Bins;
-    unsigned long long* gs = g_ss + wl * K * kL23Bins;
-
-    auto visit = [&](float dv) {
-        const uint32_t key = key_of(dv);
-        const uint32_t f = s_first[key >> 20];
-        if (f == 0xff) return;
-        if (LEVEL == 2) {
-            const uint32_t bin = (key >> 10) & 1023u;
-            atomicAdd(&gc[(size_t)f * kL23Bins + bin], 1u);
-            atomicAdd(&gs[(size_t)f * kL23Bins + bin], (unsigned long long)sq_fixed(key));
-        } else {
-            const uint32_t n = s_num[key >> 20];
-            const uint32_t p21 = key >> 10;
-            for (uint32_t s = f; s < f + n; ++s)
-                if (s_prefix[s] == p21) { atomicAdd(&gc[(size_t)s * kL23Bins + (key & 1023u)], 1u); break; }
-        }
-    };
-
-    const uint64_t q0 = ch.begin & ~3ull;
-    constexpr int U = 4;
-    for (uint64_t base = q0; base < ch.end; base += (uint64_t)4 * kThreads * U) {
-        float4 a[U];
-        bool full[U];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const uint64_t q = base + 4ull * (threadIdx.x + (uint64_t)u * kThreads);
-            full[u] = VEC && q >= ch.begin && q + 4 <= ch.end;
-            if (full[u]) a[u] = __ldcs(reinterpret_cast<const float4*>(dd + q));
-        }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const uint64_t q = base + 4ull * (threadIdx.x + (uint64_t)u * kThreads);
-            if (full[u]) {
-                visit(a[u].x); visit(a[u].y); visit(a[u].z); visit(a[u].w);
-            } else if (q < ch.end) {
-                for (int i = 0; i < 4; ++i) {
-                    const uint64_t p = q + i;
-                    if (p >= ch.begin && p < ch.end) visit(dd[p]);
-                }
-            }
-        }
-    }
-}
-
-
-// Same histograms, accumulated in shared memory with u32 atomics by CTAs that own a run of
-// consecutive chunks; used for layers with at most kSmemSlots slots (the usual case, K <= 16).
-constexpr int kHThreads = 1024;
-constexpr int kSmemSlots = 16;
-constexpr int kRunChunks = 8;
-constexpr uint64_t kDirectElems = 2048; // chunks this small go straight to global atomics
-
-template <int LEVEL>
-__global__ void __launch_bounds__(kHThreads, 1)
-k_hist23_smem(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks, uint64_t dstride,
-              uint32_t L, uint32_t K, const SlotTab* __restrict__ slots, uint32_t* __restrict__ g_cnt,
-              unsigned long long* __restrict__ g_ss) {
-    extern __shared__ __align__(16) uint32_t sh[];
-    constexpr int NW = kSmemSlots * kL23Bins;
-    uint32_t* h_cnt = sh;
-    uint32_t* h_hi = sh + NW;     // LEVEL 2 only
-    uint32_t* h_lo = sh + 2 * NW; // LEVEL 2 only
-    uint8_t* s_first = reinterpret_cast<uint8_t*>(sh + (LEVEL == 2 ? 3 : 1) * NW);
-    uint8_t* s_num = s_first + kL1Bins;
-    uint32_t* s_prefix = reinterpret_cast<uint32_t*>(s_num + kL1Bins);
-    __shared__ int s_flag;
-    const uint32_t w = blockIdx.y;
-    const uint32_t c0 = blockIdx.x * kRunChunks, c1 = min(n_chunks, c0 + kRunChunks);
-    for (int i = threadIdx.x; i < (LEVEL == 2 ? 3 : 1) * NW; i += kHThreads) sh[i] = 0;
-    if (threadIdx.x == 0) s_flag = 0;
-    const float* dd = dbuf + (size_t)w * dstride;
-    int cur_layer = -1;
-    uint32_t ns = 0;
-    bool active = false, dirty = false;
-    uint32_t* gc = nullptr;
-    unsigned long long* gs = nullptr;
-
-    auto flush = [&]() {
-        __syncthreads();
-        for (uint32_t i = threadIdx.x; i < ns * kL23Bins; i += kHThreads) {
-            const uint32_t c = h_cnt[i];
-            if (c) {
-                atomicAdd(&gc[i], c);
-                h_cnt[i] = 0;
-                if (LEVEL == 2) {
-                    atomicAdd(&gs[i], ((unsigned long long)h_hi[i] << 16) + h_lo[i]);
-                    h_hi[i] = 0;
-                    h_lo[i] = 0;
-                }
-            }
-        }
-        if (threadIdx.x == 0) s_flag = 0;
-        __syncthreads();
-        dirty = false;
-    };
-
-    for (uint32_t c = c0; c < c1; ++c) {
-        const Chunk ch = chunks[c];
-        if ((int)ch.layer != cur_layer) {
-            if (dirty) flush();
-            cur_layer = (int)ch.layer;
-            const size_t wl = (size_t)w * L + ch.layer;
-            const SlotTab& stab = slots[wl];
-            ns = stab.n;
-            active = ns <= (uint32_t)kSmemSlots;
-            gc = g_cnt + wl * K * kL23Bins;
-            gs = g_ss + wl * K * kL23Bins;
-            if (active) {
-                __syncthreads();
-                for (int b = threadIdx.x; b < kL1Bins; b += kHThreads) { s_first[b] = 0xff; s_num[b] = 0; }
-                if (threadIdx.x < ns) s_prefix[threadIdx.x] = stab.prefix[threadIdx.x];
-                __syncthreads();
-                if (threadIdx.x == 0)
-                    for (uint32_t s = 0; s < ns; ++s) {
-                        const uint32_t b1 = LEVEL == 2 ? s_prefix[s] : (s_prefix[s] >> 10);
-                        if (s_first[b1] == 0xff) s_first[b1] = (uint8_t)s;
-                        s_num[b1]++;
-                    }
-                __syncthreads();
-            }
-        }
-        if (!active) continue;
-        const bool direct = ch.end - ch.begin <= kDirectElems;
-        auto visit = [&](float dv) {
-            const uint32_t key = key_of(dv);
-            const uint32_t f = s_first[key >> 20];
-            if (f == 0xff) return;
-            if (LEVEL == 2) {
-                const uint32_t i = f * kL23Bins + ((key >> 10) & 1023u);
-                const uint32_t sq = (uint32_t)sq_fixed(key);
-                if (direct) {
-                    atomicAdd(&gc[i], 1u);
-                    atomicAdd(&gs[i], (unsigned long long)sq);
-                } else {
-                    const uint32_t old = atomicAdd(&h_cnt[i], 1u);
-                    atomicAdd(&h_hi[i], sq >> 16);
-                    atomicAdd(&h_lo[i], sq & 0xffffu);
-                    if (old >= 32768u) s_flag = 1; // flush at the next chunk boundary, before any sum can overflow
-                }
-            } else {
-                const uint32_t n = s_num[key >> 20];
-                const uint32_t p21 = key >> 10;
-                for (uint32_t s = f; s < f + n; ++s)
-                    if (s_prefix[s] == p21) {
-                        const uint32_t i = s * kL23Bins + (key & 1023u);
-                        if (direct) atomicAdd(&gc[i], 1u); else atomicAdd(&h_cnt[i], 1u);
-                        break;
-                    }
-            }
-        };
-        const uint64_t q0 = ch.begin & ~3ull;
-        constexpr int U = 2;
-        for (uint64_t base = q0; base < ch.end; base += (uint64_t)4 * kHThreads * U) {
-            float4 a[U];
-            bool full[U];
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const uint64_t q = base + 4ull * (threadIdx.x + (uint64_t)u * kHThreads);
-                full[u] = q >= ch.begin && q + 4 <= ch.end;
-                if (full[u]) a[u] = __ldcs(reinterpret_cast<const float4*>(dd + q));
-            }
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const uint64_t q = base + 4ull * (threadIdx.x + (uint64_t)u * kHThreads);
-                if (full[u]) {
-                    visit(a[u].x); visit(a[u].y); visit(a[u].z); visit(a[u].w);
-                } else if (q < ch.end) {
-                    for (int i = 0; i < 4; ++i) {
-                        const uint64_t p = q + i;
-                        if (p >= ch.begin && p < ch.end) visit(dd[p]);
-                    }
-                }
-            }
-        }
-        if (!direct) {
-            dirty = true;
-            __syncthreads();
-            if (s_flag) flush();
-        }
-    }
-    if (dirty) flush();
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -610,32 +369,42 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
                 const uint32_t* un = s_units + (plan.tab_in_smem ? l * K : 0);
                 const float* er = s_err + (plan.tab_in_smem ? l * K : 0);
                 uint8_t* pdl = pd + (size_t)l * plan.pd_row_bytes;
-                // each thread owns the cell pair (2t, 2t+1): one PD byte holds both nibbles
+                // each thread owns the cell pair (2t, 2t+1): one PD byte holds both nibbles.  Candidates are
+                // taken eight at a time so that the eight prev[] reads of a batch are independent loads.
                 for (uint32_t b0 = 2 * threadIdx.x; b0 < row; b0 += 2 * blockDim.x) {
                     float best0 = kInf, best1 = kInf;
                     uint32_t bj0 = 0, bj1 = 0;
                     const uint32_t b1 = b0 + 1;
-#pragma unroll 4
-                    for (uint32_t j = 0; j < K; ++j) {
-                        const uint32_t u = un[j];
-                        if (u > b1) continue; // covers the "unusable" marker 0xffffffff too
-                        const float e = er[j];
-                        if (u <= b0) {
-                            const float t = __fadd_rn(prev[b0 - u], e);
-                            if (t < best0) { best0 = t; bj0 = j; }
+                    const bool has1 = b1 < row;
+                    for (uint32_t j0 = 0; j0 < K; j0 += 8) {
+                        uint32_t u[8];
+                        float e[8], p0[8], p1[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const bool ok = j0 + i < K;
+                            u[i] = ok ? un[j0 + i] : 0xffffffffu;
+                            e[i] = ok ? er[j0 + i] : 0.f;
                         }
-                        if (b1 < row) {
-                            const float t = __fadd_rn(prev[b1 - u], e);
-                            if (t < best1) { best1 = t; bj1 = j; }
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) { // an unusable candidate reads +inf: inf + e is never < best
+                            p0[i] = u[i] <= b0 ? prev[b0 - u[i]] : kInf;
+                            p1[i] = (has1 && u[i] <= b1) ? prev[b1 - u[i]] : kInf;
+                        }
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const float t0 = __fadd_rn(p0[i], e[i]);
+                            const float t1 = __fadd_rn(p1[i], e[i]);
+                            if (t0 < best0) { best0 = t0; bj0 = j0 + i; }
+                            if (t1 < best1) { best1 = t1; bj1 = j0 + i; }
                         }
                     }
                     cur[b0] = best0;
-                    if (b1 < row) cur[b1] = best1;
+                    if (has1) cur[b1] = best1;
                     if (plan.pd_nibble) {
                         pdl[b0 >> 1] = (uint8_t)(bj0 | (bj1 << 4));
                     } else {
                         pdl[b0] = (uint8_t)bj0;
-                        if (b1 < row) pdl[b1] = (uint8_t)bj1;
+                        if (has1) pdl[b1] = (uint8_t)bj1;
                     }
                 }
                 float* sw = prev; prev = cur; cur = sw;

@@ -8,13 +8,13 @@
 // output offset; k_sel_write compacts in index order and updates the estimator.  No kernel waits on
 // another: offsets come from stored per-chunk counts.
 #pragma once
-#include "kimad_kernels.cuh"
+#include "kimad_curve.cuh"
 
 namespace kimad {
 
 constexpr int kListCap = 32;                    // in-interval entries remembered per chunk
 constexpr uint32_t kListOverflow = 0xffffffffu; // more than that: the chunk is recounted exactly
-constexpr int kLowBins = 1024;                  // 2^shift never exceeds this
+constexpr int kLowBins = 1024;                  // bins of the in-interval histogram
 
 struct ChunkSel { // per (worker, chunk)
     uint32_t above;          // entries whose key lies above the interval
@@ -22,38 +22,35 @@ struct ChunkSel { // per (worker, chunk)
     uint16_t low[kListCap];  // key - lo of those entries (any order)
 };
 
-// Aligned view of a chunk for 128-bit loads: quads start at a0 = begin & ~3; only the first and the
-// last quad can be partial.  All offsets are 32-bit and relative to a0.
-struct ChunkView {
-    uint64_t a0;
-    uint32_t first, len; // valid element offsets are [first, len)
-    __device__ __forceinline__ explicit ChunkView(const Chunk& ch)
-        : a0(ch.begin & ~3ull), first((uint32_t)(ch.begin - (ch.begin & ~3ull))), len((uint32_t)(ch.end - (ch.begin & ~3ull))) {}
-    __device__ __forceinline__ uint32_t quads() const { return (len + 3) >> 2; }
-    __device__ __forceinline__ bool quad_full(uint32_t q) const { return 4 * q >= first && 4 * q + 4 <= len; }
+// Second round of the select stage: layers whose interval was wider than 2^10 keys and whose entries
+// inside it could not be collected (a chunk list overflowed, or more than kSortCap entries) get their
+// interval narrowed by the coarse histogram and are counted once more over their own chunks.
+struct Round2 {
+    uint32_t n_chunks;
+    uint32_t n_layers;
+    uint32_t _pad[2];
 };
+constexpr int kSortCap = 4096;
 
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kThreads)
-k_sel_count(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks, uint64_t dstride,
-            uint32_t L, const Sel* __restrict__ sel, const LayerDesc* __restrict__ layers, ChunkSel* __restrict__ csel,
-            uint32_t* __restrict__ low_hist, uint32_t* __restrict__ recount_n, uint2* __restrict__ recount_list) {
-    __shared__ uint32_t s_w[8];
-    __shared__ uint32_t s_hist[kLowBins];
-    __shared__ uint32_t s_n;
-    __shared__ uint16_t s_low[kListCap];
-    const Chunk ch = chunks[blockIdx.x];
-    const uint32_t w = blockIdx.y;
+// Counting sweep of one chunk (the whole CTA works on it).
+__device__ __forceinline__ void sel_count_chunk(const float* __restrict__ dbuf, const Chunk& ch, uint32_t w,
+                                                uint32_t chunk_id, uint32_t n_chunks, uint64_t dstride, uint32_t L,
+                                                const Sel* __restrict__ sel, const LayerDesc* __restrict__ layers,
+                                                ChunkSel* __restrict__ csel, uint32_t* __restrict__ low_hist,
+                                                uint32_t* __restrict__ recount_n, uint2* __restrict__ recount_list,
+                                                uint32_t* s_w, uint32_t* s_hist, uint32_t* s_n, uint16_t* s_low) {
     const size_t wl = (size_t)w * L + ch.layer;
     const Sel s = sel[wl];
-    ChunkSel* out = csel + (size_t)w * n_chunks + blockIdx.x;
+    ChunkSel* out = csel + (size_t)w * n_chunks + chunk_id;
     if (s.k == 0 || (uint64_t)s.k == layers[ch.layer].n) { // nothing / everything kept: no need to look at the data
         if (threadIdx.x == 0) { out->above = s.k ? (uint32_t)(ch.end - ch.begin) : 0u; out->n_in = 0; }
         return;
     }
     const uint32_t lo = s.tau, width = 1u << s.shift;
+    const uint32_t hshift = s.shift > 10 ? s.shift - 10 : 0; // the histogram has at most kLowBins bins
     for (int i = threadIdx.x; i < kLowBins; i += kThreads) s_hist[i] = 0;
-    if (threadIdx.x == 0) s_n = 0;
+    if (threadIdx.x == 0) *s_n = 0;
     __syncthreads();
     const ChunkView cv(ch);
     const float* dd = dbuf + (size_t)w * dstride + cv.a0;
@@ -61,8 +58,8 @@ k_sel_count(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks, ui
     auto visit = [&](float dv) {
         const uint32_t d1 = key_of(dv) - lo; // wraps to >= 2^31 for keys below the interval
         if (d1 < width) {
-            atomicAdd(&s_hist[d1], 1u);
-            const uint32_t p = atomicAdd(&s_n, 1u);
+            atomicAdd(&s_hist[d1 >> hshift], 1u);
+            const uint32_t p = atomicAdd(s_n, 1u);
             if (p < (uint32_t)kListCap) s_low[p] = (uint16_t)d1;
         } else {
             above += d1 < 0x80000000u;
@@ -92,10 +89,10 @@ k_sel_count(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks, ui
     uint32_t tot;
     block_excl_scan<uint32_t>(above, s_w, &tot);
     __syncthreads();
-    const uint32_t n_in = s_n;
+    const uint32_t n_in = *s_n;
     if (n_in) { // rare: publish this chunk's part of the layer's in-interval histogram
         uint32_t* gh = low_hist + wl * kLowBins;
-        for (uint32_t i = threadIdx.x; i < width; i += kThreads)
+        for (uint32_t i = threadIdx.x; i < (uint32_t)kLowBins; i += kThreads)
             if (s_hist[i]) atomicAdd(&gh[i], s_hist[i]);
     }
     if (threadIdx.x < min(n_in, (uint32_t)kListCap)) out->low[threadIdx.x] = s_low[threadIdx.x];
@@ -105,38 +102,157 @@ k_sel_count(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks, ui
             out->n_in = n_in;
         } else {
             out->n_in = kListOverflow;
-            recount_list[atomicAdd(recount_n, 1u)] = make_uint2(w, blockIdx.x);
+            recount_list[atomicAdd(recount_n, 1u)] = make_uint2(w, chunk_id);
         }
+    }
+    __syncthreads();
+}
+
+__global__ void __launch_bounds__(kThreads)
+k_sel_count(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks, uint64_t dstride,
+            uint32_t L, const Sel* __restrict__ sel, const LayerDesc* __restrict__ layers, ChunkSel* __restrict__ csel,
+            uint32_t* __restrict__ low_hist, uint32_t* __restrict__ recount_n, uint2* __restrict__ recount_list) {
+    __shared__ uint32_t s_w[8];
+    __shared__ uint32_t s_hist[kLowBins];
+    __shared__ uint32_t s_n;
+    __shared__ uint16_t s_low[kListCap];
+    sel_count_chunk(dbuf, chunks[blockIdx.x], blockIdx.y, blockIdx.x, n_chunks, dstride, L, sel, layers, csel, low_hist,
+                    recount_n, recount_list, s_w, s_hist, &s_n, s_low);
+}
+
+// second round: only the chunks of the layers listed in r2
+__global__ void __launch_bounds__(kThreads)
+k_sel_count_r2(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks, uint64_t dstride,
+               uint32_t L, const Sel* __restrict__ sel, const LayerDesc* __restrict__ layers,
+               ChunkSel* __restrict__ csel, uint32_t* __restrict__ low_hist, uint32_t* __restrict__ recount_n,
+               uint2* __restrict__ recount_list, const Round2* __restrict__ r2, const uint2* __restrict__ r2_chunks) {
+    __shared__ uint32_t s_w[8];
+    __shared__ uint32_t s_hist[kLowBins];
+    __shared__ uint32_t s_n;
+    __shared__ uint16_t s_low[kListCap];
+    const uint32_t n = r2->n_chunks;
+    for (uint32_t it = blockIdx.x; it < n; it += gridDim.x) {
+        const uint2 e = r2_chunks[it];
+        sel_count_chunk(dbuf, chunks[e.y], e.x, e.y, n_chunks, dstride, L, sel, layers, csel, low_hist, recount_n,
+                        recount_list, s_w, s_hist, &s_n, s_low);
     }
 }
 
-// Exact threshold of every (worker, layer) from the histogram of the entries inside its interval.
-__global__ void __launch_bounds__(kThreads)
-k_sel_resolve(uint32_t L, const LayerDesc* __restrict__ layers, uint32_t* __restrict__ low_hist, Sel* __restrict__ sel) {
-    __shared__ __align__(16) uint32_t s_incl[kLowBins];
-    __shared__ uint32_t s_w32[8];
-    const uint32_t l = blockIdx.x, w = blockIdx.y;
+// Exact threshold of one (worker, layer) from what the counting sweep left behind.  The whole CTA works on it.
+// round 1: may narrow the interval and list the layer for the second round; round 2: the interval is at
+// most 32 keys wide and the histogram is exact.
+__device__ __forceinline__ void sel_resolve_layer(uint32_t l, uint32_t w, uint32_t L, const LayerDesc* __restrict__ layers,
+                                                  uint32_t n_chunks, const ChunkSel* __restrict__ csel,
+                                                  uint32_t* __restrict__ low_hist, Sel* __restrict__ sel, bool round1,
+                                                  Round2* __restrict__ r2, uint2* __restrict__ r2_layers,
+                                                  uint2* __restrict__ r2_chunks, uint32_t* s_key /* [kSortCap] */,
+                                                  uint32_t* s_w32, uint32_t* s_n, uint32_t* s_over) {
     const size_t wl = (size_t)w * L + l;
+    const LayerDesc ld = layers[l];
     Sel s = sel[wl];
-    if (s.k == 0 || (uint64_t)s.k == layers[l].n) return;
-    const uint32_t width = 1u << s.shift;
+    if (s.k == 0 || (uint64_t)s.k == ld.n) return;
     uint32_t* gh = low_hist + wl * kLowBins;
-    for (int b = threadIdx.x; b < kLowBins; b += kThreads) {
-        uint32_t c = 0;
-        if ((uint32_t)b < width) { c = gh[b]; gh[b] = 0; }
-        s_incl[kLowBins - 1 - b] = c;
+    const uint32_t hshift = s.shift > 10 ? s.shift - 10 : 0;
+    if (s.shift == 0) { // already exact: bin 0 holds the number of entries equal to tau
+        if (threadIdx.x == 0) gh[0] = 0;
+        return;
+    }
+    bool sorted = false;
+    if (round1) { // collect the entries inside the interval from the chunk lists and sort them
+        if (threadIdx.x == 0) { *s_n = 0; *s_over = 0; }
+        __syncthreads();
+        const ChunkSel* cs = csel + (size_t)w * n_chunks + ld.first_chunk;
+        for (uint32_t i = threadIdx.x; i < ld.n_chunks; i += kThreads) {
+            const uint32_t n_in = cs[i].n_in;
+            if (n_in == kListOverflow) { *s_over = 1; continue; }
+            if (!n_in) continue;
+            const uint32_t at = atomicAdd(s_n, n_in);
+            if (at + n_in > (uint32_t)kSortCap) { *s_over = 1; continue; }
+            for (uint32_t e = 0; e < n_in; ++e) s_key[at + e] = cs[i].low[e];
+        }
+        __syncthreads();
+        sorted = !*s_over;
+        if (sorted) {
+            const uint32_t cnt = *s_n;
+            uint32_t np = 1;
+            while (np < cnt) np <<= 1;
+            for (uint32_t i = cnt + threadIdx.x; i < np; i += kThreads) s_key[i] = 0; // padding sorts last
+            __syncthreads();
+            for (uint32_t size = 2; size <= np; size <<= 1)
+                for (uint32_t str = size >> 1; str > 0; str >>= 1) {
+                    for (uint32_t i = threadIdx.x; i < np / 2; i += kThreads) {
+                        const uint32_t a = 2 * i - (i & (str - 1)), b = a + str;
+                        const bool desc = (a & size) == 0;
+                        const uint32_t ka = s_key[a], kb = s_key[b];
+                        if ((ka < kb) == desc) { s_key[a] = kb; s_key[b] = ka; }
+                    }
+                    __syncthreads();
+                }
+            if (threadIdx.x == 0) {
+                const uint32_t rank = s.keep_eq, t = s_key[rank - 1]; // rank <= cnt by construction
+                uint32_t first = rank - 1;
+                while (first > 0 && s_key[first - 1] == t) --first;
+                s.tau_low = t;
+                s.tau += t;
+                s.keep_eq = rank - first;
+                s.shift = 0;
+                sel[wl] = s;
+            }
+        }
     }
     __syncthreads();
-    scan_bins<kLowBins>(s_incl, nullptr, s_w32, nullptr);
-    if (threadIdx.x == 0) {
-        const int p = find_pos<kLowBins>(s_incl, s.keep_eq); // keep_eq holds the rank inside the interval
-        const uint32_t above = p ? s_incl[p - 1] : 0u;
-        const uint32_t bin = (uint32_t)(kLowBins - 1 - p);
-        s.tau_low = bin;
-        s.tau += bin;
-        s.keep_eq -= above;
-        sel[wl] = s;
+    if (!sorted) { // histogram of the interval: exact when it has at most kLowBins keys, else it narrows the interval
+        uint32_t* s_incl = s_key; // [kLowBins], reuse
+        for (int b = threadIdx.x; b < kLowBins; b += kThreads) s_incl[kLowBins - 1 - b] = gh[b];
+        __syncthreads();
+        scan_bins<kLowBins>(s_incl, nullptr, s_w32, nullptr);
+        if (threadIdx.x == 0) {
+            const int p = find_pos<kLowBins>(s_incl, s.keep_eq); // keep_eq holds the rank inside the interval
+            const uint32_t above = p ? s_incl[p - 1] : 0u;
+            const uint32_t bin = (uint32_t)(kLowBins - 1 - p);
+            s.keep_eq -= above;
+            s.tau += bin << hshift;
+            s.tau_low = hshift ? 0u : bin;
+            s.shift = hshift;
+            sel[wl] = s;
+        }
+        if (hshift) { // not exact yet: the layer and its chunks go to the second round
+            __shared__ uint32_t s_at;
+            if (threadIdx.x == 0) {
+                s_at = atomicAdd(&r2->n_chunks, ld.n_chunks);
+                r2_layers[atomicAdd(&r2->n_layers, 1u)] = make_uint2(w, l);
+            }
+            __syncthreads();
+            for (uint32_t i = threadIdx.x; i < ld.n_chunks; i += kThreads) r2_chunks[s_at + i] = make_uint2(w, ld.first_chunk + i);
+        }
     }
+    __syncthreads();
+    for (int b = threadIdx.x; b < kLowBins; b += kThreads) gh[b] = 0; // clean for the next use
+    __syncthreads();
+}
+
+__global__ void __launch_bounds__(kThreads)
+k_sel_resolve(uint32_t L, const LayerDesc* __restrict__ layers, uint32_t n_chunks, const ChunkSel* __restrict__ csel,
+              uint32_t* __restrict__ low_hist, Sel* __restrict__ sel, Round2* __restrict__ r2,
+              uint2* __restrict__ r2_layers, uint2* __restrict__ r2_chunks) {
+    __shared__ __align__(16) uint32_t s_key[kSortCap];
+    __shared__ uint32_t s_w32[8];
+    __shared__ uint32_t s_n, s_over;
+    sel_resolve_layer(blockIdx.x, blockIdx.y, L, layers, n_chunks, csel, low_hist, sel, true, r2, r2_layers, r2_chunks, s_key,
+                      s_w32, &s_n, &s_over);
+}
+
+__global__ void __launch_bounds__(kThreads)
+k_sel_resolve_r2(uint32_t L, const LayerDesc* __restrict__ layers, uint32_t n_chunks, const ChunkSel* __restrict__ csel,
+                 uint32_t* __restrict__ low_hist, Sel* __restrict__ sel, Round2* __restrict__ r2,
+                 uint2* __restrict__ r2_layers, uint2* __restrict__ r2_chunks) {
+    __shared__ __align__(16) uint32_t s_key[kSortCap];
+    __shared__ uint32_t s_w32[8];
+    __shared__ uint32_t s_n, s_over;
+    const uint32_t n = r2->n_layers;
+    for (uint32_t it = blockIdx.x; it < n; it += gridDim.x)
+        sel_resolve_layer(r2_layers[it].y, r2_layers[it].x, L, layers, n_chunks, csel, low_hist, sel, false, r2, r2_layers,
+                          r2_chunks, s_key, s_w32, &s_n, &s_over);
 }
 
 // Exact (gt, eq) of the chunks whose list overflowed.
@@ -171,7 +287,7 @@ k_sel_recount(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks, 
 __global__ void __launch_bounds__(kThreads)
 k_sel_scan(uint32_t L, const LayerDesc* __restrict__ layers, uint32_t n_chunks, const Sel* __restrict__ sel,
            const ChunkSel* __restrict__ csel, uint2* __restrict__ chunk_cnt, uint2* __restrict__ chunk_pre,
-           uint32_t* __restrict__ recount_n) {
+           uint32_t* __restrict__ recount_n, FbList* __restrict__ fb, Round2* __restrict__ r2) {
     __shared__ uint32_t s_w[8];
     const LayerDesc ld = layers[blockIdx.x];
     const uint32_t w = blockIdx.y;
@@ -179,7 +295,13 @@ k_sel_scan(uint32_t L, const LayerDesc* __restrict__ layers, uint32_t n_chunks, 
     const ChunkSel* cs = csel + (size_t)w * n_chunks + ld.first_chunk;
     uint2* cc = chunk_cnt + (size_t)w * n_chunks + ld.first_chunk;
     uint2* cp = chunk_pre + (size_t)w * n_chunks + ld.first_chunk;
-    if (blockIdx.x == 0 && w == 0 && threadIdx.x == 0) *recount_n = 0; // consumed by k_sel_recount already
+    if (blockIdx.x == 0 && w == 0 && threadIdx.x == 0) { // all work lists have been consumed by now
+        *recount_n = 0;
+        fb->n_chunks = 0;
+        fb->n_layers = 0;
+        r2->n_chunks = 0;
+        r2->n_layers = 0;
+    }
     uint32_t run_g = 0, run_e = 0;
     for (uint32_t base = 0; base < ld.n_chunks; base += kThreads) {
         const uint32_t i = base + threadIdx.x;
@@ -250,7 +372,6 @@ k_sel_write(const float* __restrict__ dbuf, float* __restrict__ state, const Chu
         uint32_t keepm = 0, eqm = 0;
         const bool interior = rb >= cv.first && rb + E * kThreads <= cv.len;
         if (interior) {
-#pragma unroll
             float v[E];
 #pragma unroll
             for (int u = 0; u < E / 4; ++u) {

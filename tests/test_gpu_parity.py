@@ -11,10 +11,10 @@ from tests._harness import Runner, u32
 pytestmark = pytest.mark.gpu
 
 
-def _run_workload(cfg, divisor, steps, grid=None, D=None):
+def _run_workload(cfg, divisor, steps, grid=None, D=None, curve_mode=0):
     wl = workloads.workload(cfg, divisor)
     grid = grid or wl.ratio_grid
-    r = Runner(wl.layer_sizes, wl.n_workers, grid, D or wl.D, wl.value_dtype)
+    r = Runner(wl.layer_sizes, wl.n_workers, grid, D or wl.D, wl.value_dtype, curve_mode=curve_mode)
     bw = workloads.bandwidth_trace(wl, max(steps, 60))
     pick = np.linspace(0, len(bw) - 1, steps).astype(int)  # spread over the trace: low and high budgets
     state = torch.zeros((wl.n_workers, wl.N), dtype=torch.float32, device="cuda")
@@ -25,6 +25,16 @@ def _run_workload(cfg, divisor, steps, grid=None, D=None):
         mismatched += not res["same_k"]
     # the free-running state after `steps` steps was compared bit for bit at every step
     assert mismatched == 0, f"{mismatched} steps chose another k than the oracle on its own curve"
+    n_reg = sum(1 for n in wl.layer_sizes if n > 4096) * wl.n_workers * steps * 2  # each step runs twice (inject check)
+    handed = kb.kimad_debug_exact_path_layers(r.ctx)
+    if curve_mode == 1:
+        assert handed == n_reg
+    else:  # the sampled bands must carry (nearly) all layers by themselves
+        why = kb.kimad_debug_exact_path_layers(r.ctx, detail=True)
+        # with 50 candidates the fine bins are shared by 50 bands and more error bounds come out too loose
+        limit = n_reg // 50 if len(grid) <= 16 else n_reg // 4
+        assert handed <= max(1, limit), f"{why} of {n_reg} layers fell back to the exact radix path"
+    return handed, n_reg
 
 
 def test_cfg1_mlp_full_size():
@@ -49,6 +59,16 @@ def test_cfg5_llama_shape_scaled_bf16():
 
 def test_paper_grid_50_candidates():
     _run_workload(2, 32, 2, grid=workloads.paper_grid_50())
+
+
+@pytest.mark.parametrize("cfg,divisor", [(2, 8), (4, 64), (5, 512)])
+def test_exact_radix_everywhere(cfg, divisor):
+    """curve_mode 1: every layer above the tiny size goes through the three-digit radix select."""
+    _run_workload(cfg, divisor, 2, curve_mode=1)
+
+
+def test_paper_grid_50_exact_radix():
+    _run_workload(2, 32, 2, grid=workloads.paper_grid_50(), curve_mode=1)
 
 
 def test_worked_example_on_gpu():
@@ -89,14 +109,15 @@ def _adversarial_layers(rng):
     return [np.ascontiguousarray(x, np.float32) for x in layers]
 
 
+@pytest.mark.parametrize("curve_mode", [0, 1])
 @pytest.mark.parametrize("value_dtype", [0, 1])
-def test_adversarial_inputs(value_dtype):
+def test_adversarial_inputs(value_dtype, curve_mode):
     rng = np.random.default_rng(77)
     layers = _adversarial_layers(rng)
     sizes = [x.size for x in layers]
     N = sum(sizes)
     grid = [0.001, 0.01, 0.1, 0.5, 0.9, 1.0]
-    r = Runner(sizes, 2, grid, value_dtype=value_dtype)
+    r = Runner(sizes, 2, grid, value_dtype=value_dtype, curve_mode=curve_mode)
     flat = np.concatenate(layers)
     grads = torch.from_numpy(np.stack([flat, flat[::-1].copy()])).cuda()   # worker 1: same values, other layout
     bpe = 8 if value_dtype == 0 else 6
