@@ -48,6 +48,7 @@ extern "C" {
 #define KIMAD_ERR_TIMEOUT (-5)   /* reserved: no kernel of this library waits on another             */
 #define KIMAD_ERR_CUDA (-6)      /* a CUDA runtime call failed                                       */
 #define KIMAD_ERR_NOMEM (-7)     /* host allocation failed                                           */
+#define KIMAD_ERR_TOO_LARGE (-8) /* kimad_step_builtin_scratch: scratch need above the built-in array */
 
 #define KIMAD_MAX_RATIOS 127 /* candidates per layer */
 #define KIMAD_MAX_D 16383    /* budget cells */
@@ -119,6 +120,32 @@ int kimad_set_workspace(kimad_ctx* ctx, void* dev_ptr, size_t bytes);
  * Returns 0 or a CUDA/argument error; per-worker outcomes land in out->stats[w].status. */
 int kimad_step(kimad_ctx* ctx, const float* grads_dev, float* state_dev, const double* bandwidth_bytes_per_s,
                double t_target_s, const kimad_packed* out, void* cuda_stream);
+
+/* kimad_step for callers that cannot allocate device memory.  (The paper has no counterpart: this is
+ * a deployment variant of the same pass.)  Some callers have no workspace to give to
+ * kimad_set_workspace and may not obtain one: a gradient hook that runs while other streams are busy
+ * (cudaMalloc synchronises the whole device and would stall them), or a plug-in inside a runtime that
+ * owns all device memory in a fixed arena and hands none out.  This call takes the same arguments as
+ * kimad_step and produces the same results, but keeps its scratch in an array of
+ * KIMAD_BUILTIN_SCRATCH_BYTES that is part of the library's device image: every GPU that loads the
+ * library holds those bytes until the process exits.  It calls no cudaMalloc / cudaFree and no
+ * allocating library routine; kimad_set_workspace is not needed (a workspace attached to ctx is left
+ * untouched).
+ *   - Limit: kimad_workspace_bytes(ctx) must not exceed KIMAD_BUILTIN_SCRATCH_BYTES, else the call
+ *     returns KIMAD_ERR_TOO_LARGE and does nothing (roughly: up to a million elements over all
+ *     workers with a dozen ratios).
+ *   - The first call on a device looks up the array's device address (that device must be current,
+ *     as for every call); make that first call before any stream capture.
+ *   - All contexts and all calls on a device share the one array, which keeps the previous call's
+ *     contents: every call re-uploads its tables and clears its histograms in stream order, so calls
+ *     that follow each other on one stream are safe, while calls that overlap on the GPU (different
+ *     streams, or different host threads) race on the scratch and must be serialised by the caller.
+ *   - The kimad_debug_* getters read the attached workspace, not the built-in array. */
+#define KIMAD_BUILTIN_SCRATCH_BYTES (32u << 20)
+#define KIMAD_BUILTIN_MAX_DEVICES 64
+int kimad_step_builtin_scratch(kimad_ctx* ctx, const float* grads_dev, float* state_dev,
+                               const double* bandwidth_bytes_per_s, double t_target_s, const kimad_packed* out,
+                               void* cuda_stream);
 
 /* Copies the last step's chosen k to host_k (host, u32 [W][L]; may be NULL) after synchronising
  * cuda_stream.  Returns the most severe per-worker status of that step: the lowest negative

@@ -23,6 +23,8 @@ KIMAD_ERR_NONFINITE = -4
 KIMAD_ERR_TIMEOUT = -5
 KIMAD_ERR_CUDA = -6
 KIMAD_ERR_NOMEM = -7
+KIMAD_ERR_TOO_LARGE = -8
+KIMAD_BUILTIN_SCRATCH_BYTES = 32 << 20
 
 
 class kimad_options(C.Structure):
@@ -80,6 +82,8 @@ def load():
     step_args = [vp, vp, vp, C.POINTER(dbl), dbl, C.POINTER(kimad_packed), vp]
     L.kimad_step.restype = C.c_int
     L.kimad_step.argtypes = step_args
+    L.kimad_step_builtin_scratch.restype = C.c_int
+    L.kimad_step_builtin_scratch.argtypes = step_args
     L.kimad_debug_step_with_err.restype = C.c_int
     L.kimad_debug_step_with_err.argtypes = step_args + [vp]
     L.kimad_debug_step_with_j.restype = C.c_int
@@ -203,6 +207,16 @@ def kimad_step(ctx: Ctx, grads, state, bandwidth_bytes_per_s, t_target_s, out: P
     bw = _bw(ctx, bandwidth_bytes_per_s)
     _check(load().kimad_step(ctx.handle, grads.data_ptr(), state.data_ptr(), bw.ctypes.data_as(C.POINTER(C.c_double)),
                              float(t_target_s), C.byref(out.c), _stream_ptr(stream)), "kimad_step")
+
+
+def kimad_step_builtin_scratch(ctx: Ctx, grads, state, bandwidth_bytes_per_s, t_target_s, out: Packed, stream=None) -> None:
+    """kimad_step with the scratch in the library's built-in device array: for callers that cannot allocate
+    device memory.  No workspace has to be attached to ``ctx``; raises KimadError(KIMAD_ERR_TOO_LARGE) when the
+    context needs more than KIMAD_BUILTIN_SCRATCH_BYTES."""
+    bw = _bw(ctx, bandwidth_bytes_per_s)
+    _check(load().kimad_step_builtin_scratch(ctx.handle, grads.data_ptr(), state.data_ptr(),
+                                             bw.ctypes.data_as(C.POINTER(C.c_double)), float(t_target_s),
+                                             C.byref(out.c), _stream_ptr(stream)), "kimad_step_builtin_scratch")
 
 
 def kimad_debug_step_with_err(ctx: Ctx, grads, state, bandwidth_bytes_per_s, t_target_s, out: Packed, err_dev,

@@ -491,6 +491,52 @@ int kimad_debug_exact_path_layers(kimad_ctx* c, uint64_t* host_count) {
 
 uint64_t kimad_launch_count(const kimad_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
+// ---------------------------------------------------------------------------------------------------
+// Allocation-free variant of kimad_step: the scratch is a fixed array inside the library's device image.
+// ---------------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_builtin_scratch[KIMAD_BUILTIN_SCRATCH_BYTES];
+// Host code may not pass the symbol itself to a kernel: its device address is looked up once per device.
+static unsigned char* g_builtin_ptr[KIMAD_BUILTIN_MAX_DEVICES] = {};
+
+int kimad_step_builtin_scratch(kimad_ctx* c, const float* grads_dev, float* state_dev, const double* bandwidth_bytes_per_s,
+                               double t_target_s, const kimad_packed* out, void* cuda_stream) {
+    if (!c) return KIMAD_ERR_INVALID_ARG;
+    if (c->lay.total > (size_t)KIMAD_BUILTIN_SCRATCH_BYTES) return KIMAD_ERR_TOO_LARGE;
+    int dev = -1;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= KIMAD_BUILTIN_MAX_DEVICES) return KIMAD_ERR_INVALID_ARG;
+    if (!g_builtin_ptr[dev]) { // first call on this device (it is the current one)
+        void* p = nullptr;
+        CUDA_TRY(cudaGetSymbolAddress(&p, g_builtin_scratch));
+        g_builtin_ptr[dev] = static_cast<unsigned char*>(p);
+    }
+    unsigned char* ws = g_builtin_ptr[dev];
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+    // The array keeps whatever the previous call (of any context) left: bring in this context's tables and
+    // clear everything that has to start at zero, in stream order before the kernels.
+    const Layout& y = c->lay;
+    CUDA_TRY(cudaMemcpyAsync(ws + y.chunks, c->chunks.data(), c->chunks.size() * sizeof(Chunk), cudaMemcpyHostToDevice, s));
+    CUDA_TRY(cudaMemcpyAsync(ws + y.layers, c->layers.data(), c->layers.size() * sizeof(LayerDesc), cudaMemcpyHostToDevice, s));
+    CUDA_TRY(cudaMemcpyAsync(ws + y.ktab, c->ktab.data(), c->ktab.size() * sizeof(uint64_t), cudaMemcpyHostToDevice, s));
+    if (!c->reg_layers.empty())
+        CUDA_TRY(cudaMemcpyAsync(ws + y.reg_layers, c->reg_layers.data(), c->reg_layers.size() * 4, cudaMemcpyHostToDevice, s));
+    if (!c->tiny_layers.empty())
+        CUDA_TRY(cudaMemcpyAsync(ws + y.tiny_layers, c->tiny_layers.data(), c->tiny_layers.size() * 4, cudaMemcpyHostToDevice, s));
+    CUDA_TRY(cudaMemcpyAsync(ws + y.reg_index, c->reg_index.data(), c->reg_index.size() * 4, cudaMemcpyHostToDevice, s));
+    CUDA_TRY(cudaMemsetAsync(ws + y.zero_from, 0, y.lut_t1 - y.zero_from, s));
+    CUDA_TRY(cudaFuncSetAttribute(k_dp, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->dp_smem));
+    CUDA_TRY(cudaFuncSetAttribute(k_sample, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->sample_smem));
+    CUDA_TRY(cudaFuncSetAttribute(k_pass_a<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->pass_a_smem));
+    CUDA_TRY(cudaFuncSetAttribute(k_pass_a<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->pass_a_smem));
+    CUDA_TRY(cudaFuncSetAttribute(k_tiny_exact, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->tiny_smem));
+    unsigned char* caller_ws = c->ws; // the context's own workspace (if any) is left untouched
+    c->ws = ws;
+    const int rc = run_step(c, grads_dev, state_dev, bandwidth_bytes_per_s, t_target_s, out, cuda_stream, kNormal, nullptr,
+                            nullptr);
+    c->ws = caller_ws;
+    return rc;
+}
+
 const char* kimad_strerror(int code) {
     switch (code) {
         case KIMAD_OK: return "ok";
@@ -503,6 +549,7 @@ const char* kimad_strerror(int code) {
         case KIMAD_ERR_TIMEOUT: return "device wait timed out";
         case KIMAD_ERR_CUDA: return "CUDA runtime error";
         case KIMAD_ERR_NOMEM: return "host allocation failed";
+        case KIMAD_ERR_TOO_LARGE: return "problem needs more scratch than the built-in array of kimad_step_builtin_scratch";
         default: return "unknown code";
     }
 }
