@@ -51,7 +51,7 @@ extern "C" {
 #define KIMAD_ERR_TOO_LARGE (-8) /* kimad_step_builtin_scratch: scratch need above the built-in array */
 
 #define KIMAD_MAX_RATIOS 127 /* candidates per layer */
-#define KIMAD_MAX_D 16383    /* budget cells */
+#define KIMAD_MAX_D 8191     /* budget cells */
 
 typedef struct kimad_ctx kimad_ctx;
 

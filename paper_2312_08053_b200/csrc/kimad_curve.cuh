@@ -81,23 +81,34 @@ k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint6
     const uint32_t n_units = (n + 15) / 16;
     const uint32_t m_units = min(n_units, (uint32_t)kSampleUnits);
     const bool whole = m_units == n_units;
-    const double stratum = (double)n / (double)m_units;
+    const uint32_t sq_ = n / (uint32_t)kSampleUnits, sr_ = n % (uint32_t)kSampleUnits; // used when sampled: m_units = kSampleUnits
     uint32_t mine = 0;
-    for (uint32_t i = threadIdx.x >> 4; i < m_units; i += kBigThreads / 16) { // a half-warp reads one unit
-        uint32_t start;
-        if (whole) {
-            start = 16 * i;
-        } else { // unit i somewhere inside stratum i
-            const uint32_t s0 = (uint32_t)((double)i * stratum), s1 = (uint32_t)((double)(i + 1) * stratum);
-            const uint32_t room = s1 > s0 + 16 ? s1 - s0 - 16 : 0;
-            start = s0 + __umulhi(hash_u32(i * 0x9e3779b9u + l * 0x85ebca6bu + 1u), room + 1);
+    // a half-warp reads one unit; eight units per thread are in flight before their keys are counted
+    for (uint32_t ib = threadIdx.x >> 4; ib < m_units; ib += 8 * (kBigThreads / 16)) {
+        float a[8], b[8];
+        bool ok[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const uint32_t i = ib + u * (kBigThreads / 16);
+            uint32_t start = 16 * i;
+            if (!whole && i < m_units) { // unit i somewhere inside stratum i = [i q + i r / m, (i+1) q + (i+1) r / m)
+                const uint32_t s0 = i * sq_ + (i * sr_) / (uint32_t)kSampleUnits;
+                const uint32_t s1 = (i + 1) * sq_ + ((i + 1) * sr_) / (uint32_t)kSampleUnits;
+                const uint32_t room = s1 > s0 + 16 ? s1 - s0 - 16 : 0;
+                start = s0 + __umulhi(hash_u32(i * 0x9e3779b9u + l * 0x85ebca6bu + 1u), room + 1);
+            }
+            const uint32_t p = start + (threadIdx.x & 15);
+            ok[u] = i < m_units && p < n;
+            a[u] = ok[u] ? gr[p] : 0.f;
+            b[u] = ok[u] ? st[p] : 0.f;
         }
-        const uint32_t p = start + (threadIdx.x & 15);
-        if (p < n) {
-            const uint32_t cell = key_of(__fsub_rn(gr[p], st[p])) >> 15;
-            atomicAdd(&h32[cell >> 1], 1u << (16 * (cell & 1)));
-            ++mine;
-        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            if (ok[u]) {
+                const uint32_t cell = key_of(__fsub_rn(a[u], b[u])) >> 15;
+                atomicAdd(&h32[cell >> 1], 1u << (16 * (cell & 1)));
+                ++mine;
+            }
     }
     atomicAdd(&s_m, mine);
     __syncthreads();
@@ -128,24 +139,33 @@ k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint6
         s_sq[threadIdx.x] = totd - exd - sq; // squares in the segments below this one (higher thread index)
     }
     __syncthreads();
-    // cell holding sample rank rk (1-based, from the top)
+    // cell holding sample rank rk (1-based, from the top); the whole warp takes part
+    const uint32_t lane = threadIdx.x & 31;
     auto cell_of_rank = [&](uint32_t rk) {
         int lo = 0, hi = kBigThreads - 1;
         while (lo < hi) { const int mid = (lo + hi) >> 1; if (s_pre[mid] >= rk) hi = mid; else lo = mid + 1; }
-        uint32_t before = lo ? s_pre[lo - 1] : 0u;
+        const uint32_t before = lo ? s_pre[lo - 1] : 0u;
         const uint32_t top = 65535u - 64u * lo;
-        for (uint32_t i = 0; i < 64; ++i) {
-            before += cell_count(top - i);
-            if (before >= rk) return top - i;
+        // lanes take cells top - 2 lane and top - 2 lane - 1; inclusive counts along the lanes
+        const uint32_t c0 = cell_count(top - 2 * lane), c1 = cell_count(top - 2 * lane - 1);
+        uint32_t incl = c0 + c1;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= (uint32_t)o) incl += y;
         }
-        return top - 63u;
+        const uint32_t upto0 = before + incl - c1; // entries in the cells top .. top - 2 lane
+        const uint32_t hit0 = __ballot_sync(0xffffffffu, upto0 >= rk);
+        const uint32_t hit1 = __ballot_sync(0xffffffffu, before + incl >= rk);
+        if (!hit1) return top - 63u;
+        const uint32_t l1 = __ffs(hit1) - 1;
+        return (hit0 >> l1) & 1u ? top - 2 * l1 : top - 2 * l1 - 1;
     };
 
-    // ---- bands: the cells that can hold the k_j-th largest key, and how finely to cut them
-    if (threadIdx.x < K) {
-        const uint32_t j = threadIdx.x;
+    // ---- bands: the cells that can hold the k_j-th largest key, and how finely to cut them (one warp per candidate)
+    for (uint32_t j = threadIdx.x >> 5; j < K; j += kBigThreads / 32) {
         const uint64_t k = ktab[(size_t)l * K + j];
-        s_cb[j] = 1; s_ct[j] = 0; s_cs[j] = 15; // k == n keeps everything: no threshold, no band
+        uint32_t o_cb = 1, o_ct = 0, o_cs = 15; // k == n keeps everything: no threshold, no band
         if (k < n) {
             uint32_t r_lo, r_hi;
             if (whole) {
@@ -161,36 +181,43 @@ k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint6
             // octave further up; clipped at the bottom: no bound from the sample, exact path
             uint32_t c_top = cell_of_rank(max(r_lo, 1u));
             if (r_lo == 0) c_top = min(c_top + 256u, 65279u);
-            if (r_hi == 0) s_flag = 1;
+            if (r_hi == 0 && lane == 0) s_flag = 1;
             const uint32_t c_bot = cell_of_rank(max(r_hi, 1u));
             const uint32_t ncell = c_top - c_bot + 1;
             if (ncell > (uint32_t)kFineBins) {
-                s_flag = 2;
+                if (lane == 0) s_flag = 2;
             } else {
                 uint32_t inband = 0;
-                for (uint32_t c = c_bot; c <= c_top; ++c) inband += cell_count(c);
+                for (uint32_t c = c_bot + lane; c <= c_top; c += 32) inband += cell_count(c);
                 // estimate of this candidate's error: squares of everything below the band
                 const uint32_t seg = (65535u - c_bot) >> 6;
-                double below = s_sq[seg];
-                for (uint32_t c = 65535u - 64u * seg - 63u; c < c_bot; ++c) {
+                double below = 0.0;
+                for (uint32_t c = 65535u - 64u * seg - 63u + lane; c < c_bot; c += 32) {
                     const uint32_t cc = cell_count(c);
                     if (cc) below += (double)cc * cell_sq(c);
                 }
+#pragma unroll
+                for (int o = 16; o; o >>= 1) {
+                    inband += __shfl_xor_sync(0xffffffffu, inband, o);
+                    below += __shfl_xor_sync(0xffffffffu, below, o);
+                }
+                below += s_sq[seg];
                 const double scale = (double)n / (double)m;
                 const double per_cell = (double)inband / (double)ncell * scale; // entries per band cell
                 const double v2 = cell_sq(c_top);
                 // bins per cell: at most ~2048 entries per bin (what the select stage collects and sorts), and
                 // narrow enough that the uncertainty of the bin holding the threshold (its entries times its
-                // spread of squares, 2^-7 of v^2 for a whole cell) stays below ~5e-7 of the error
+                // spread of squares, 2^-7 of v^2 for a whole cell) stays below ~1.5e-6 of the error
                 double bins = per_cell / 2048.0;
                 const double e_est = below * scale;
                 const double cert = e_est > 0.0 ? sqrt(per_cell * 0.0078125 * v2 / (1.5e-6 * e_est)) : 1024.0;
                 if (cert > bins) bins = cert;
                 uint32_t sh_j = 15;
                 while (sh_j > 5 && (double)(1u << (15 - sh_j)) < bins) --sh_j;
-                s_cb[j] = c_bot; s_ct[j] = c_top; s_cs[j] = sh_j;
+                o_cb = c_bot; o_ct = c_top; o_cs = sh_j;
             }
         }
+        if (lane == 0) { s_cb[j] = o_cb; s_ct[j] = o_ct; s_cs[j] = o_cs; }
     }
     __syncthreads();
     // merge overlapping / adjacent bands (they descend in key with j) into groups; groups end up in s_c*[0..ng)
@@ -470,24 +497,49 @@ k_resolve_a(const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ r
         const uint32_t* blo = bin_lo + wr * (kMaxBins + 1);
         uint32_t* gc = bh_cnt + wr * kMaxBins;
         unsigned long long* gs = bh_sum + wr * kMaxBins;
-        uint32_t run_c = 0;   // entries in the bins swept so far (ascending keys)
-        double run_s = 0.0;   // their squares
+        // Every warp owns a contiguous range of bins (ascending keys).  First sweep: the range's totals; then
+        // a scan over the 32 warps; second sweep: running count / running squares per bin, to find the bin
+        // where the running count passes n - k_j.  No block-wide barrier inside the sweeps.
+        const uint32_t lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+        const uint32_t per = ((nb + 31) / 32 + 31) & ~31u; // bins per warp, a multiple of 32
+        const uint32_t r0 = min(nb, wid * per), r1 = min(nb, r0 + per);
+        auto bin_sq = [&](uint32_t b) { // the sweep summed squares in units of 2^8 sq_fixed
+            return (double)gs[b] * (256.0 * sq_scale(blo[b] >> 23));
+        };
+        uint32_t c_tot = 0;
+        double s_tot = 0.0;
+        for (uint32_t b = r0 + lane; b < r1; b += 32) { c_tot += gc[b]; s_tot += bin_sq(b); }
+#pragma unroll
+        for (int o = 16; o; o >>= 1) {
+            c_tot += __shfl_xor_sync(0xffffffffu, c_tot, o);
+            s_tot += __shfl_xor_sync(0xffffffffu, s_tot, o);
+        }
+        if (lane == 0) { s_w32[wid] = c_tot; s_w64[wid] = s_tot; }
+        __syncthreads();
+        uint32_t run_c = 0;  // entries in the bins below this warp's range
+        double run_s = 0.0;  // their squares
+        for (uint32_t i = 0; i < wid; ++i) { run_c += s_w32[i]; run_s += s_w64[i]; }
         bool nonfinite = false;
-        for (uint32_t base = 0; base < nb; base += kBigThreads) {
-            const uint32_t b = base + threadIdx.x;
+        for (uint32_t base = r0; base < r1; base += 32) {
+            const uint32_t b = base + lane;
             uint32_t c = 0;
             double sv = 0.0;
-            if (b < nb) {
+            if (b < r1) {
                 c = gc[b];
-                const uint32_t klo = blo[b];
-                sv = (double)gs[b] * (256.0 * sq_scale(klo >> 23)); // the sweep summed squares in units of 2^8 sq_fixed
-                if (c) { gc[b] = 0; gs[b] = 0ull; }                    // clean for the next step
-                nonfinite |= c && klo >= 0x7f800000u;
+                sv = bin_sq(b);
+                if (c) { gc[b] = 0; gs[b] = 0ull; } // clean for the next step
+                nonfinite |= c && blo[b] >= 0x7f800000u;
             }
-            uint32_t tc;
-            double ts;
-            const uint32_t before = run_c + block_excl_scan<uint32_t, kBigThreads>(c, s_w32, &tc);
-            const double below = run_s + block_excl_scan<double, kBigThreads>(sv, s_w64, &ts);
+            uint32_t ic = c;
+            double is = sv;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t yc = __shfl_up_sync(0xffffffffu, ic, o);
+                const double ys = __shfl_up_sync(0xffffffffu, is, o);
+                if (lane >= (uint32_t)o) { ic += yc; is += ys; }
+            }
+            const uint32_t before = run_c + ic - c;
+            const double below = run_s + is - sv;
             if (c)
                 for (uint32_t j = 0; j < K; ++j) { // the bin where the running count passes n - k_j holds the threshold
                     const uint32_t dj = s_drop[j];
@@ -495,8 +547,8 @@ k_resolve_a(const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ r
                         s_bin[j] = b; s_before[j] = before; s_cb[j] = c; s_below[j] = below; s_sb[j] = sv;
                     }
                 }
-            run_c += tc;
-            run_s += ts;
+            run_c += __shfl_sync(0xffffffffu, ic, 31);
+            run_s += __shfl_sync(0xffffffffu, is, 31);
         }
         if (nonfinite) atomicOr(&flags[w], 1u);
         __syncthreads();

@@ -298,11 +298,14 @@ k_rebuild_slots(const FbList* __restrict__ fb, const uint2* __restrict__ fb_laye
 struct DpBudgets { uint64_t c[kDpWorkersPerLaunch]; };
 
 constexpr int kDpThreads = 512;
+constexpr int kDpCells = 2; // budget cells per thread
 
 // Shared-memory plan of k_dp (host computes the same sizes):
-//   prev[D+1], cur[D+1] f32 | j[L] u32 | units[L*K] u32, err[L*K] f32 (if tab_in_smem) | PD
-// PD holds the winning candidate of every (layer, cell): a nibble when K <= 16, else a byte; it lives
-// in shared memory when it fits, else in the caller's workspace.
+//   two rows of (D+2) +inf followed by D+1 values, f32 | j[L] u32 | usable[L or 1] u32 |
+//   units[(L or 1) * Kp] u32, err[(L or 1) * Kp] f32, Kp = K rounded up to 4 | PD
+// The +inf margin in front of each row lets prev[b - u] be read without a bounds test for every u <= D+1
+// (an unusable candidate has u = D+1).  PD holds the winning candidate of every (layer, cell): a nibble
+// when K <= 16, else a byte; it lives in shared memory when it fits, else in the caller's workspace.
 struct DpPlan {
     uint32_t tab_in_smem; // candidate tables preloaded for all layers (else one layer at a time)
     uint32_t pd_in_smem;
@@ -323,15 +326,17 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
     const uint32_t w = w_base + blockIdx.x;
     if (w >= W) return;
     const uint64_t c = budgets.c[blockIdx.x];
-    const uint32_t row = D + 1;
+    const uint32_t row = D + 1, pad = D + 2, rowp = row + pad, Kp = (K + 3) & ~3u;
     const float kInf = __int_as_float(0x7f800000);
-    float* prev = reinterpret_cast<float*>(smem_raw);
-    float* cur = prev + row;
-    uint32_t* s_j = reinterpret_cast<uint32_t*>(cur + row); // [L]
-    uint32_t* s_units = s_j + L;                             // [L*K] or [K]
-    const uint32_t ntab = plan.tab_in_smem ? L * K : K;
-    float* s_err = reinterpret_cast<float*>(s_units + ntab);
-    uint8_t* pd = plan.pd_in_smem ? reinterpret_cast<uint8_t*>(s_err + ntab)
+    float* rows = reinterpret_cast<float*>(smem_raw);
+    float* prev = rows + pad;          // prev[-pad .. -1] = +inf
+    float* cur = rows + rowp + pad;
+    uint32_t* s_j = reinterpret_cast<uint32_t*>(rows + 2 * rowp); // [L]
+    const uint32_t ltab = plan.tab_in_smem ? L : 1;
+    uint32_t* s_usable = s_j + L;                                 // [ltab] candidates that fit into D cells
+    uint32_t* s_units = s_usable + ltab;                          // [ltab * Kp]
+    float* s_err = reinterpret_cast<float*>(s_units + ltab * Kp); // [ltab * Kp]
+    uint8_t* pd = plan.pd_in_smem ? reinterpret_cast<uint8_t*>(s_err + ltab * Kp)
                                   : pd_global + (size_t)w * L * plan.pd_row_bytes;
     __shared__ float s_redv[32];
     __shared__ uint32_t s_redb[32];
@@ -352,59 +357,84 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
             status = KIMAD_STATUS_INFEASIBLE;
             for (uint32_t l = threadIdx.x; l < L; l += blockDim.x) s_j[l] = 0;
         } else {
-            auto load_tab = [&](uint32_t src, uint32_t dst) { // candidate src of the [L][K] tables -> smem slot dst
-                const uint64_t u = budget_cells(ktab[src] * bpe, D, c);
-                s_units[dst] = u > D ? 0xffffffffu : (uint32_t)u;
-                s_err[dst] = e_w[src];
+            // candidate (l, j) -> smem slot; units above D become D+1 (reads the +inf margin), padding likewise
+            auto load_tab = [&](uint32_t l, uint32_t j, uint32_t slot_l) {
+                uint32_t u = D + 1;
+                float e = 0.f;
+                if (j < K) {
+                    const uint64_t uu = budget_cells(ktab[(size_t)l * K + j] * bpe, D, c);
+                    u = uu > D ? D + 1 : (uint32_t)uu;
+                    e = e_w[(size_t)l * K + j];
+                }
+                s_units[slot_l * Kp + j] = u;
+                s_err[slot_l * Kp + j] = e;
             };
-            if (plan.tab_in_smem)
-                for (uint32_t i = threadIdx.x; i < L * K; i += blockDim.x) load_tab(i, i);
-            for (uint32_t b = threadIdx.x; b < row; b += blockDim.x) prev[b] = b ? kInf : 0.f;
+            auto count_usable = [&](uint32_t slot_l) { // sizes ascend with j, so the usable candidates come first
+                uint32_t nu = 0;
+                while (nu < K && s_units[slot_l * Kp + nu] <= D) ++nu;
+                s_usable[slot_l] = nu;
+            };
+            if (plan.tab_in_smem) {
+                for (uint32_t i = threadIdx.x; i < L * Kp; i += blockDim.x) load_tab(i / Kp, i % Kp, i / Kp);
+                __syncthreads();
+                for (uint32_t l = threadIdx.x; l < L; l += blockDim.x) count_usable(l);
+            }
+            for (uint32_t i = threadIdx.x; i < 2 * rowp; i += blockDim.x) rows[i] = kInf;
+            __syncthreads();
+            if (threadIdx.x == 0) prev[0] = 0.f;
             for (uint32_t l = 0; l < L; ++l) {
                 __syncthreads();
                 if (!plan.tab_in_smem) {
-                    if (threadIdx.x < K) load_tab(l * K + threadIdx.x, threadIdx.x);
+                    if (threadIdx.x < Kp) load_tab(l, threadIdx.x, 0);
+                    __syncthreads();
+                    if (threadIdx.x == 0) count_usable(0);
                     __syncthreads();
                 }
-                const uint32_t* un = s_units + (plan.tab_in_smem ? l * K : 0);
-                const float* er = s_err + (plan.tab_in_smem ? l * K : 0);
+                const uint32_t sl = plan.tab_in_smem ? l : 0;
+                const uint32_t* un = s_units + sl * Kp;
+                const float* er = s_err + sl * Kp;
+                const uint32_t nu = s_usable[sl];
                 uint8_t* pdl = pd + (size_t)l * plan.pd_row_bytes;
-                // each thread owns the cell pair (2t, 2t+1): one PD byte holds both nibbles.  Candidates are
-                // taken eight at a time so that the eight prev[] reads of a batch are independent loads.
-                for (uint32_t b0 = 2 * threadIdx.x; b0 < row; b0 += 2 * blockDim.x) {
-                    float best0 = kInf, best1 = kInf;
-                    uint32_t bj0 = 0, bj1 = 0;
-                    const uint32_t b1 = b0 + 1;
-                    const bool has1 = b1 < row;
-                    for (uint32_t j0 = 0; j0 < K; j0 += 8) {
-                        uint32_t u[8];
-                        float e[8], p0[8], p1[8];
+                // each thread owns the cells t, t + T, ... (consecutive threads read consecutive words of
+                // prev[]: no bank conflicts); candidates four at a time so that the prev[] reads of a batch are
+                // independent loads and a candidate's (cells, error) pair is fetched once for all cells of the thread
+                for (uint32_t bb = 0; bb < row; bb += kDpCells * blockDim.x) {
+                    const uint32_t b0 = bb + threadIdx.x;
+                    float best[kDpCells];
+                    uint32_t bj[kDpCells];
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            const bool ok = j0 + i < K;
-                            u[i] = ok ? un[j0 + i] : 0xffffffffu;
-                            e[i] = ok ? er[j0 + i] : 0.f;
-                        }
+                    for (int q = 0; q < kDpCells; ++q) { best[q] = kInf; bj[q] = 0; }
+                    for (uint32_t j0 = 0; j0 < nu; j0 += 4) {
+                        uint32_t u[4];
+                        float e[4], p[4][kDpCells];
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) { // an unusable candidate reads +inf: inf + e is never < best
-                            p0[i] = u[i] <= b0 ? prev[b0 - u[i]] : kInf;
-                            p1[i] = (has1 && u[i] <= b1) ? prev[b1 - u[i]] : kInf;
-                        }
+                        for (int i = 0; i < 4; ++i) { u[i] = un[j0 + i]; e[i] = er[j0 + i]; }
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            const float t0 = __fadd_rn(p0[i], e[i]);
-                            const float t1 = __fadd_rn(p1[i], e[i]);
-                            if (t0 < best0) { best0 = t0; bj0 = j0 + i; }
-                            if (t1 < best1) { best1 = t1; bj1 = j0 + i; }
-                        }
+                        for (int i = 0; i < 4; ++i)
+#pragma unroll
+                            for (int q = 0; q < kDpCells; ++q) {
+                                // cells beyond the row (last pass only) read the row itself: harmless, never stored
+                                const uint32_t b = min(b0 + q * blockDim.x, row - 1);
+                                p[i][q] = prev[(int)b - (int)u[i]];
+                            }
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+#pragma unroll
+                            for (int q = 0; q < kDpCells; ++q) {
+                                const float t = __fadd_rn(p[i][q], e[i]); // +inf when the candidate does not fit
+                                if (t < best[q]) { best[q] = t; bj[q] = j0 + i; }
+                            }
                     }
-                    cur[b0] = best0;
-                    if (has1) cur[b1] = best1;
-                    if (plan.pd_nibble) {
-                        pdl[b0 >> 1] = (uint8_t)(bj0 | (bj1 << 4));
-                    } else {
-                        pdl[b0] = (uint8_t)bj0;
-                        if (has1) pdl[b1] = (uint8_t)bj1;
+#pragma unroll
+                    for (int q = 0; q < kDpCells; ++q) {
+                        const uint32_t b = b0 + q * blockDim.x;
+                        if (b < row) cur[b] = best[q];
+                        if (plan.pd_nibble) { // even threads store their own nibble and their right neighbour's
+                            const uint32_t nb = __shfl_down_sync(0xffffffffu, bj[q], 1);
+                            if (!(threadIdx.x & 1) && b < row) pdl[b >> 1] = (uint8_t)(bj[q] | (nb << 4));
+                        } else if (b < row) {
+                            pdl[b] = (uint8_t)bj[q];
+                        }
                     }
                 }
                 float* sw = prev; prev = cur; cur = sw;
@@ -440,7 +470,7 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
                         const uint8_t* pdl = pd + (size_t)l * plan.pd_row_bytes;
                         const uint32_t j = plan.pd_nibble ? ((pdl[b >> 1] >> (4 * (b & 1))) & 15u) : pdl[b];
                         s_j[l] = j;
-                        b -= plan.tab_in_smem ? s_units[l * K + j]
+                        b -= plan.tab_in_smem ? s_units[l * Kp + j]
                                               : (uint32_t)budget_cells(ktab[(size_t)l * K + j] * bpe, D, c);
                     }
                 }
@@ -455,8 +485,8 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
 
     // totals, capacity check and outputs (prev/cur are free now: stage k_l and err_l there)
     uint32_t* s_k = reinterpret_cast<uint32_t*>(smem_raw);
-    float* s_e = reinterpret_cast<float*>(smem_raw) + row;
-    const bool staged = L <= row;
+    float* s_e = reinterpret_cast<float*>(smem_raw) + rowp;
+    const bool staged = L <= rowp;
     if (staged && status >= 0)
         for (uint32_t l = threadIdx.x; l < L; l += blockDim.x) {
             s_k[l] = (uint32_t)ktab[(size_t)l * K + s_j[l]];

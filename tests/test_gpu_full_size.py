@@ -1,0 +1,122 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py times.
+
+The oracle cannot sort a whole 0.5-2 G element step in test time, so: (1) for a sample of layers (always
+including the largest one) the oracle computes curve, threshold, packed entries and state one layer at a
+time and every value is compared; (2) the DP is re-run by the oracle on the GPU's complete curve; (3)
+properties that hold at any size are checked on ALL layers: counts, offsets, ascending indices, values
+equal to d at the indices, no dropped entry larger than a kept one, untouched entries of the state."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import kimad_oracle as ko
+from paper_2312_08053_b200 import binding as kb
+from paper_2312_08053_b200 import workloads
+
+pytestmark = pytest.mark.gpu
+
+
+def _full_size_step(cfg, step_of_trace, sample_layers, workers_checked):
+    wl = workloads.workload(cfg)
+    W, N, L, K = wl.n_workers, wl.N, wl.L, len(wl.ratio_grid)
+    bw_all = workloads.bandwidth_trace(wl)
+    bw = bw_all[step_of_trace]
+    bpe = 8 if wl.value_dtype == 0 else 6
+    cap = int(min(N, np.max(bw) * wl.t_target / bpe + L + 1))
+    ctx = kb.new_context(wl.layer_sizes, W, wl.ratio_grid, D=wl.D, value_dtype=wl.value_dtype, max_packed_elems=cap)
+    out = kb.Packed(ctx)
+    state = torch.zeros((W, N), dtype=torch.float32, device="cuda")
+    # one earlier step so that the EF state is not all zero
+    g0 = workloads.gradients(wl, 0, device="cuda")
+    kb.kimad_step(ctx, g0, state, bw_all[0], wl.t_target, out)
+    del g0
+    grads = workloads.gradients(wl, 1, device="cuda")
+    state_before = state.clone()
+    kb.kimad_step(ctx, grads, state, bw, wl.t_target, out)
+    status, k_gpu = kb.kimad_get_k(ctx)
+    assert status >= 0
+    err_g, tau_g, keq_g, shift_g = kb.kimad_debug_get_curve(ctx)
+    tau_s, keq_s = kb.kimad_debug_get_selection(ctx)
+    st = out.stats_host()
+    j_gpu = out.j.cpu().numpy().view(np.uint32)
+    offs = out.offs.cpu().numpy().astype(np.int64)
+    kt = ko.k_table(wl.layer_sizes, wl.ratio_grid)
+    loff = np.concatenate([[0], np.cumsum(wl.layer_sizes)]).astype(np.int64)
+
+    # (2) the DP on the GPU's own curve, and the bookkeeping
+    for w in range(W):
+        c = ko.budget_bytes(float(bw[w]), wl.t_target)
+        s_units, units = ko.units(kt, wl.value_dtype, c, wl.D)
+        assert s_units == 0
+        s_dp, j_ref, val, cell = ko.dp(err_g[w], units, wl.D)
+        assert s_dp == int(st["status"][w]) == 0
+        assert np.array_equal(j_ref, j_gpu[w])
+        k_ref = kt[np.arange(L), j_ref]
+        assert np.array_equal(k_ref.astype(np.uint32), k_gpu[w])
+        assert np.array_equal(offs[w], np.concatenate([[0], np.cumsum(k_ref)]).astype(np.int64))
+        assert int(st["used_bytes"][w]) == bpe * int(k_ref.sum()) <= c == int(st["budget_bytes"][w])
+        tot = np.float32(0)
+        for l in range(L):
+            tot = np.float32(tot + err_g[w, l, j_ref[l]])
+        assert tot == st["total_err"][w]
+
+    # (1) + (3) per layer, on the host copy of one worker at a time
+    for w in workers_checked:
+        d = (grads[w] - state_before[w]).cpu().numpy()
+        g_old = state_before[w].cpu().numpy()
+        g_new = state[w].cpu().numpy()
+        n_sel = int(offs[w, L])
+        idx_all = out.idx[w, :n_sel].cpu().numpy().view(np.uint32)
+        val_all = out.val[w, :n_sel].view(torch.int16 if wl.value_dtype else torch.int32).cpu().numpy()
+        for l in range(L):
+            lo, hi = int(loff[l]), int(loff[l + 1])
+            a, b = int(offs[w, l]), int(offs[w, l + 1])
+            k = b - a
+            idx = idx_all[a:b].astype(np.int64)
+            dl = d[lo:hi]
+            assert k == int(k_gpu[w, l]) and np.all(np.diff(idx) > 0) and (k == 0 or idx[-1] < hi - lo)
+            sent32 = dl[idx]
+            if wl.value_dtype == 0:
+                assert np.array_equal(val_all[a:b], sent32.view(np.int32))
+                sent = sent32
+            else:
+                ref16 = torch.from_numpy(sent32).to(torch.bfloat16)
+                assert np.array_equal(val_all[a:b], ref16.view(torch.int16).numpy())
+                sent = ref16.to(torch.float32).numpy()
+            expect = g_old[lo:hi].copy()
+            expect[idx] = expect[idx] + sent
+            assert np.array_equal(expect.view(np.uint32), g_new[lo:hi].view(np.uint32))
+            key = dl.view(np.uint32) & np.uint32(0x7FFFFFFF)
+            if 0 < k < hi - lo:
+                mask = np.zeros(hi - lo, bool)
+                mask[idx] = True
+                kmin = key[mask].min()
+                assert kmin >= key[~mask].max()
+                assert kmin == tau_s[w, l]
+                eq = np.nonzero(key == kmin)[0]
+                kept_eq = eq[mask[eq]]
+                assert len(kept_eq) == keq_s[w, l] and np.array_equal(kept_eq, eq[:len(kept_eq)])  # lowest indices first
+            if l in sample_layers:  # everything the oracle can say about this layer
+                cv = ko.layer_curve(dl, kt[l])
+                tol = 1e-5 * np.abs(cv.err.astype(np.float64))
+                assert np.all((err_g[w, l] == cv.err) | (np.abs(err_g[w, l].astype(np.float64) - cv.err) <= tol)), (l, err_g[w, l], cv.err)
+                ex = (shift_g[w, l] == 0) & (kt[l] < hi - lo)
+                assert np.array_equal(tau_g[w, l][ex], cv.tau[ex]) and np.array_equal(keq_g[w, l][ex], cv.keep_eq[ex])
+                if 0 < k:
+                    oi, ov = ko.select_pack(dl, k, wl.value_dtype)
+                    assert np.array_equal(oi.astype(np.int64), idx)
+                    assert np.array_equal(ov.view(np.int16 if wl.value_dtype else np.int32), val_all[a:b])
+        del d, g_old, g_new
+    return kb.kimad_debug_exact_path_layers(ctx, detail=True)
+
+
+def test_gpt2_small_shape_full_size():
+    # 4 workers x 124.4 M elements; layers: the 38.6 M embedding, position table, one of each block tensor, last norm
+    why = _full_size_step(4, step_of_trace=7, sample_layers={0, 1, 2, 4, 6, 10, 12, 147}, workers_checked=[0, 3])
+    assert why[0] <= 8, why
+
+
+def test_llama_1b_shape_full_size_bf16():
+    # 2 workers x 1.1 G elements, bf16 values; layers: 65.5 M embedding, q/k proj, one FFN matrix, a norm, lm_head slot
+    why = _full_size_step(5, step_of_trace=30, sample_layers={0, 2, 3, 7, 10}, workers_checked=[1])
+    assert why[0] <= 60, why
