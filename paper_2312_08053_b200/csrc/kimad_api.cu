@@ -81,7 +81,7 @@ void plan_layout(kimad_ctx* c) {
     y.r2 = take(sizeof(Round2));
     y.flags = take((size_t)c->W * sizeof(uint32_t));
     y.lut_t1 = take(WR * kL1Bins * sizeof(uint16_t));
-    y.lut_t2 = take(WR * kMaxRows * 32 * sizeof(uint32_t));
+    y.lut_t2 = take(WR * kLutWords * sizeof(uint32_t));
     y.bin_lo = take(WR * (kMaxBins + 1) * sizeof(uint32_t));
     y.meta = take(WR * sizeof(BandMeta));
     y.cands = take(WLK * sizeof(Cand));
@@ -328,7 +328,7 @@ int kimad_create(kimad_ctx** out, const uint64_t* layer_sizes, uint32_t n_layers
         c->dp_smem = used;
         c->curve_mode = o.curve_mode;
         c->sample_smem = (size_t)(2 * (1024 + 32) + 32768 + 2048 + 1024 + 2048 + 2048 + 32 + 3 * 128) * 4;
-        c->pass_a_smem = (size_t)(3 * kMaxBins + kMaxRows * 32) * 4 + kL1Bins * 2;
+        c->pass_a_smem = (size_t)(3 * kMaxBins + kLutWords) * 4 + kL1Bins * 2;
         c->tiny_smem = (size_t)kTinyMax * (8 + 4);
         plan_layout(c);
     } catch (const std::bad_alloc&) {

@@ -21,7 +21,8 @@ namespace kimad {
 
 constexpr int kTinyMax = 4096;
 constexpr int kFineBins = 12288;                    // fine bins per (worker, layer)
-constexpr int kMaxBins = kL1Bins + 256 + kFineBins; // + gap bins (one per 11-bit bin, plus pieces around bands)
+constexpr int kMaxGaps = KIMAD_MAX_RATIOS + 2;      // gap regions: below / between / above the band groups, + non-finite keys
+constexpr int kMaxBins = kFineBins + kL1Bins + 2 * kMaxGaps; // fine bins + gap regions cut at every 11-bit prefix
 constexpr int kMaxRows = 128;                       // 11-bit bins that contain band cells
 constexpr int kMaxShift = 15;                       // a fine bin is 2^shift keys wide, at most a whole cell
 constexpr int kSampleUnits = 4095;                  // sample = units of 16 consecutive elements (<= 65520 elements)
@@ -31,9 +32,11 @@ constexpr uint32_t kGapBit = 1u;                    // bin_lo entries carry this
 struct BandMeta { // per (worker, regular layer)
     uint32_t n_bins;
     uint32_t n_rows;
-    uint32_t flagged; // 1: this layer takes the exact radix path in this step
-    uint32_t _pad;
+    uint32_t flagged; // != 0: this layer takes the exact radix path in this step
+    uint32_t n_gaps;  // gap regions (when flagged: detail of the misfit)
 };
+// lookup entry of a cell: first bin id | shift << 16; the bin of a key is id + ((key & 0x7fff) >> shift)
+constexpr int kLutWords = kMaxRows * 32;
 
 __device__ __forceinline__ uint32_t hash_u32(uint32_t x) {
     x ^= x >> 16; x *= 0x7feb352du; x ^= x >> 15; x *= 0x846ca68bu; x ^= x >> 16;
@@ -258,56 +261,72 @@ k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint6
         for (uint32_t g = 0; g < ng; ++g)
             for (uint32_t c = s_cb[g] + threadIdx.x; c <= s_ct[g]; c += kBigThreads) atomicOr(&bitmap[c >> 5], 1u << (c & 31));
     __syncthreads();
-    auto shift_of = [&](uint32_t cell) {
-        for (uint32_t g = 0; g < ng; ++g)
-            if (cell >= s_cb[g] && cell <= s_ct[g]) return s_cs[g];
-        return 15u;
-    };
-
-    // ---- bin ids in ascending key order; thread t owns the 11-bit bins 2t and 2t+1
-    uint32_t word[2], nb[2];
-    uint32_t rows = 0, nbt = 0;
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-        word[i] = bitmap[2 * threadIdx.x + i];
-        rows += word[i] != 0;
-        if (word[i]) {
-            const uint32_t z = ~word[i];
-            uint32_t cnt = __popc(z & ~(z << 1)); // gap runs
-            for (uint32_t wd = word[i]; wd; wd &= wd - 1)
-                cnt += 1u << (15 - shift_of(((2 * threadIdx.x + i) << 5) | (__ffs(wd) - 1)));
-            nb[i] = cnt;
-        } else {
-            nb[i] = 1;
+    // ---- bin ids in ascending key order: gap_0, fine bins of the lowest group, gap_1, ..., gap_ng, non-finite gap.
+    // A gap region is cut at every 11-bit prefix (one bin per piece: keeps the shared-memory atomics of the sweep
+    // spread over many words).  Groups are stored with descending keys; a = ng - 1 - g is the ascending index.
+    // s_base[a] = first id of gap_a, s_aux[a] = lowest cell of gap_a; the non-finite gap is a = ng + 1.
+    uint32_t* s_glo = s_pre; // [kMaxGaps] reuse: the rank prefix is no longer needed
+    if (threadIdx.x == 0 && !s_flag) {
+        uint32_t id = 0;
+        for (uint32_t a = 0; a <= ng; ++a) {
+            const uint32_t lo = a == 0 ? 0u : s_ct[ng - a] + 1;              // lowest cell of the gap
+            const uint32_t hi = a == ng ? 65279u : s_cb[ng - 1 - a] - 1;      // highest cell (may be lo - 1: empty)
+            s_base[a] = id;
+            s_glo[a] = lo;
+            if (hi + 1 > lo) id += (hi >> 5) - (lo >> 5) + 1;
+            if (a < ng) {
+                const uint32_t g = ng - 1 - a;
+                s_base[kMaxGaps + a] = id; // first fine bin of group a
+                id += (s_ct[g] - s_cb[g] + 1) << (15 - s_cs[g]);
+            }
         }
-        nbt += nb[i];
+        s_base[ng + 1] = id; // keys with exponent 255: one bin
+        s_glo[ng + 1] = 65280u;
+        s_base[ng + 2] = id + 1; // number of bins
     }
-    uint32_t tot_rows, tot_bins;
-    const uint32_t ex_rows = block_excl_scan<uint32_t, kBigThreads>(rows, s_w, &tot_rows);
-    const uint32_t ex_bins = block_excl_scan<uint32_t, kBigThreads>(nbt, s_w, &tot_bins);
+    uint32_t rows = bitmap[2 * threadIdx.x] != 0;
+    rows += bitmap[2 * threadIdx.x + 1] != 0;
+    uint32_t tot_rows;
+    uint32_t row = block_excl_scan<uint32_t, kBigThreads>(rows, s_w, &tot_rows); // includes the barrier for s_base
+    const uint32_t tot_bins = s_flag ? 0u : s_base[ng + 2];
     const bool bad = s_flag || tot_rows > (uint32_t)kMaxRows || tot_bins > (uint32_t)kMaxBins;
     if (bad) {
         if (threadIdx.x == 0) *mt = BandMeta{tot_bins, tot_rows, 2, s_flag};
         return;
     }
-    uint16_t* t1 = lut_t1 + wr * kL1Bins;
-    uint32_t* t2 = lut_t2 + wr * (kMaxRows * 32);
-    uint32_t* blo = bin_lo + wr * (kMaxBins + 1);
-    {
-        uint32_t base = ex_bins, row = ex_rows;
-#pragma unroll
-        for (int i = 0; i < 2; ++i) {
-            const uint32_t b1 = 2 * threadIdx.x + i;
-            s_base[b1] = base;
-            if (word[i]) {
-                s_aux[b1] = row;
-                t1[b1] = (uint16_t)(0x8000u | row);
-                ++row;
-            } else {
-                t1[b1] = (uint16_t)base;
-                blo[base] = (b1 << 20) | kGapBit;
+    // cell -> (lookup entry, is this the first cell of a bin that is a gap piece?)
+    auto entry_of = [&](uint32_t cell, bool& gap_first) -> uint32_t {
+        gap_first = false;
+        uint32_t a = ng + 1; // gap ordinal if the cell is in no band
+        if (cell < 65280u) {
+            a = 0;
+            for (; a < ng; ++a) {
+                const uint32_t g = ng - 1 - a;
+                if (cell > s_ct[g]) continue;
+                if (cell >= s_cb[g]) return (s_base[kMaxGaps + a] + ((cell - s_cb[g]) << (15 - s_cs[g]))) | (s_cs[g] << 16);
+                break;
             }
-            base += nb[i];
+        }
+        const uint32_t lo = s_glo[a];
+        gap_first = cell == lo || (cell & 31u) == 0;
+        const uint32_t piece = a == ng + 1 ? 0u : (cell >> 5) - (lo >> 5);
+        return (s_base[a] + piece) | (15u << 16);
+    };
+    uint16_t* t1 = lut_t1 + wr * kL1Bins;
+    uint32_t* t2 = lut_t2 + wr * kLutWords;
+    uint32_t* blo = bin_lo + wr * (kMaxBins + 1);
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const uint32_t b1 = 2 * threadIdx.x + i;
+        if (bitmap[b1]) {
+            s_aux[b1] = row;
+            t1[b1] = (uint16_t)(0x8000u | row);
+            ++row;
+        } else { // no band cell inside: the whole 11-bit bin is one gap piece
+            bool first;
+            const uint32_t e = entry_of(b1 << 5, first);
+            t1[b1] = (uint16_t)(e & 0x7fffu);
+            if (first && (b1 <= 2040u)) blo[e & 0xffffu] = (b1 << 20) | kGapBit; // bins 2041.. share the non-finite bin
         }
     }
     __syncthreads();
@@ -315,29 +334,20 @@ k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint6
     for (uint32_t b1 = threadIdx.x >> 5; b1 < (uint32_t)kL1Bins; b1 += kBigThreads / 32) {
         const uint32_t wd = bitmap[b1];
         if (!wd) continue;
-        const uint32_t lane = threadIdx.x & 31;
         const uint32_t cell = (b1 << 5) | lane;
-        const bool band = (wd >> lane) & 1u;
-        const bool gap_start = !band && (lane == 0 || ((wd >> (lane - 1)) & 1u));
-        const uint32_t shc = band ? shift_of(cell) : 15u;
-        const uint32_t contrib = band ? (1u << (15 - shc)) : (gap_start ? 1u : 0u);
-        uint32_t incl = contrib;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= (uint32_t)o) incl += y;
-        }
-        const uint32_t id = s_base[b1] + (band ? incl - contrib : incl - 1u);
-        t2[s_aux[b1] * 32 + lane] = id | (shc << 16);
-        if (band) {
-            for (uint32_t i = 0; i < contrib; ++i) blo[id + i] = (cell << 15) + (i << shc);
-        } else if (gap_start) {
+        bool first;
+        const uint32_t e = entry_of(cell, first);
+        t2[s_aux[b1] * 32 + lane] = e;
+        const uint32_t id = e & 0xffffu, shc = e >> 16;
+        if ((wd >> lane) & 1u) {
+            for (uint32_t i = 0; i < (1u << (15 - shc)); ++i) blo[id + i] = (cell << 15) + (i << shc);
+        } else if (first) {
             blo[id] = (cell << 15) | kGapBit;
         }
     }
     if (threadIdx.x == 0) {
         blo[tot_bins] = 0x80000000u;
-        *mt = BandMeta{tot_bins, tot_rows, 0, 0};
+        *mt = BandMeta{tot_bins, tot_rows, 0, ng + 2};
     }
 }
 
@@ -357,8 +367,8 @@ k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, float
     uint32_t* h_cnt = sh;
     uint32_t* h_hi = sh + kMaxBins;
     uint32_t* h_lo = sh + 2 * kMaxBins;
-    uint32_t* t2 = sh + 3 * kMaxBins;                               // [kMaxRows * 32]
-    uint16_t* t1 = reinterpret_cast<uint16_t*>(t2 + kMaxRows * 32); // [2048]
+    uint32_t* t2 = sh + 3 * kMaxBins;                           // [kLutWords] cell rows, then gap ids
+    uint16_t* t1 = reinterpret_cast<uint16_t*>(t2 + kLutWords); // [2048]
     static_assert((uint64_t)kRunChunksA * kChunkElems <= (1ull << 18), "u32 sums of 12-bit halves");
     const uint32_t w = blockIdx.y;
     const uint32_t c0 = blockIdx.x * kRunChunksA, c1 = min(n_chunks, c0 + kRunChunksA);
@@ -417,7 +427,7 @@ k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, float
                     __syncthreads();
                     const uint32_t* g1 = reinterpret_cast<const uint32_t*>(lut_t1 + wr * kL1Bins);
                     for (int i = threadIdx.x; i < kL1Bins / 2; i += kBigThreads) reinterpret_cast<uint32_t*>(t1)[i] = g1[i];
-                    const uint32_t* g2 = lut_t2 + wr * (kMaxRows * 32);
+                    const uint32_t* g2 = lut_t2 + wr * kLutWords;
                     for (uint32_t i = threadIdx.x; i < mt.n_rows * 32; i += kBigThreads) t2[i] = g2[i];
                 }
             }
