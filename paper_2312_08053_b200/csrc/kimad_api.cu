@@ -165,7 +165,9 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
 
     const uint32_t R = (uint32_t)c->reg_layers.size(), T = (uint32_t)c->tiny_layers.size();
     const dim3 gch(nch, W), glw(L, W), blk(kThreads);
-    const dim3 grun((nch + kRunChunksA - 1) / kRunChunksA, W);
+    // long runs amortise the per-CTA table load and histogram flush; keep about eight waves of CTAs on 148 SMs
+    const uint32_t run_chunks = std::max<uint32_t>(4u, std::min<uint32_t>((uint32_t)kMaxRunChunksA, (uint32_t)(((uint64_t)nch * W) / (148 * 8))));
+    const dim3 grun((nch + run_chunks - 1) / run_chunks, W);
     int stage = 0;
     auto mark = [&]() { if (c->timing) cudaEventRecord(c->ev[stage++], s); };
     mark();
@@ -177,10 +179,10 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
     }
     mark();
     if (vec)
-        k_pass_a<true><<<grun, kBigThreads, c->pass_a_smem, s>>>(grads, state, dbuf, chunks, nch, c->stride, c->dstride,
+        k_pass_a<true><<<grun, kBigThreads, c->pass_a_smem, s>>>(grads, state, dbuf, chunks, nch, run_chunks, c->stride, c->dstride,
                                                                  reg_index, R, lut1, lut2, meta, bhc, bhs);
     else
-        k_pass_a<false><<<grun, kBigThreads, c->pass_a_smem, s>>>(grads, state, dbuf, chunks, nch, c->stride, c->dstride,
+        k_pass_a<false><<<grun, kBigThreads, c->pass_a_smem, s>>>(grads, state, dbuf, chunks, nch, run_chunks, c->stride, c->dstride,
                                                                   reg_index, R, lut1, lut2, meta, bhc, bhs);
     c->launches += 1;
     mark();
@@ -232,17 +234,18 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
                                           recount_list, r2, r2_chunks);
     k_sel_resolve_r2<<<std::min<uint32_t>(W * L, 128u), blk, 0, s>>>(L, layers, nch, csel, lowh, sel, r2, r2_layers,
                                                                    r2_chunks);
-    k_sel_recount<<<2 * 148, blk, 0, s>>>(dbuf, chunks, nch, c->dstride, L, sel, recount_n, recount_list, ccnt);
-    k_sel_scan<<<glw, blk, 0, s>>>(L, layers, nch, sel, csel, ccnt, cpre, recount_n, fb, r2);
+    k_sel_recount<<<2 * 148, blk, 0, s>>>(dbuf, chunks, nch, c->dstride, L, sel, recount_n, recount_list, csel);
+    k_sel_slices<<<(uint32_t)(((uint64_t)W * nch + 7) / 8), blk, 0, s>>>(chunks, nch, W, L, sel, csel, ccnt);
+    k_sel_scan<<<glw, blk, 0, s>>>(layers, nch, ccnt, cpre, recount_n, fb, r2);
     mark();
     if (c->value_dtype == 1)
-        k_sel_write<true><<<gch, blk, 0, s>>>(dbuf, state, chunks, nch, c->dstride, c->stride, L, sel, layers, ccnt, cpre,
-                                              c->cap, out->idx, out->val);
+        k_sel_write<true><<<gch, blk, 0, s>>>(dbuf, state, chunks, nch, c->dstride, c->stride, L, sel, layers, csel, ccnt,
+                                              cpre, c->cap, out->idx, out->val);
     else
-        k_sel_write<false><<<gch, blk, 0, s>>>(dbuf, state, chunks, nch, c->dstride, c->stride, L, sel, layers, ccnt, cpre,
-                                               c->cap, out->idx, out->val);
+        k_sel_write<false><<<gch, blk, 0, s>>>(dbuf, state, chunks, nch, c->dstride, c->stride, L, sel, layers, csel, ccnt,
+                                               cpre, c->cap, out->idx, out->val);
     mark();
-    c->launches += 7;
+    c->launches += 8;
     CUDA_TRY(cudaGetLastError());
     c->last_out = *out;
     c->have_last = true;

@@ -354,12 +354,12 @@ k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint6
 // ------------------------------------------------------------------------------------------------
 // k_pass_a: CTAs own runs of consecutive chunks; histogram words live in shared memory
 // ------------------------------------------------------------------------------------------------
-constexpr int kRunChunksA = 8;
+constexpr int kMaxRunChunksA = 32; // a run has at most 2^20 elements: the u32 sums of 12-bit halves cannot overflow
 
 template <bool VEC>
 __global__ void __launch_bounds__(kBigThreads, 1)
 k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, float* __restrict__ dbuf,
-         const Chunk* __restrict__ chunks, uint32_t n_chunks, uint64_t stride, uint64_t dstride,
+         const Chunk* __restrict__ chunks, uint32_t n_chunks, uint32_t run_chunks, uint64_t stride, uint64_t dstride,
          const uint32_t* __restrict__ reg_index /* [L], 0xffffffff: tiny layer */, uint32_t R,
          const uint16_t* __restrict__ lut_t1, const uint32_t* __restrict__ lut_t2, const BandMeta* __restrict__ meta,
          uint32_t* __restrict__ bh_cnt, unsigned long long* __restrict__ bh_sum) {
@@ -369,9 +369,9 @@ k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, float
     uint32_t* h_lo = sh + 2 * kMaxBins;
     uint32_t* t2 = sh + 3 * kMaxBins;                           // [kLutWords] cell rows, then gap ids
     uint16_t* t1 = reinterpret_cast<uint16_t*>(t2 + kLutWords); // [2048]
-    static_assert((uint64_t)kRunChunksA * kChunkElems <= (1ull << 18), "u32 sums of 12-bit halves");
+    static_assert((uint64_t)kMaxRunChunksA * kChunkElems <= (1ull << 20), "u32 sums of 12-bit halves");
     const uint32_t w = blockIdx.y;
-    const uint32_t c0 = blockIdx.x * kRunChunksA, c1 = min(n_chunks, c0 + kRunChunksA);
+    const uint32_t c0 = blockIdx.x * run_chunks, c1 = min(n_chunks, c0 + run_chunks);
     for (int i = threadIdx.x; i < 3 * kMaxBins; i += kBigThreads) sh[i] = 0;
     const float* gr0 = grads + (size_t)w * stride;
     const float* st0 = state + (size_t)w * stride;
@@ -402,7 +402,7 @@ k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, float
         const uint32_t e2 = t2[(split ? (e1 & 0x7fffu) : 0u) * 32 + ((key >> 15) & 31u)];
         const uint32_t id = split ? (e2 & 0xffffu) + ((key & 0x7fffu) >> (e2 >> 16)) : e1;
         // 24 significant bits of the square (truncation < 2^-22 relative), in two 12-bit halves: a run has at
-        // most 2^18 elements, so neither u32 sum can overflow before the flush at the end of the run
+        // most 2^20 elements, so neither u32 sum can overflow before the flush at the end of the run
         const uint32_t sq = (uint32_t)(sq_fixed(key) >> 8);
         atomicAdd(&h_cnt[id], 1u);
         atomicAdd(&h_hi[id], sq >> 12);

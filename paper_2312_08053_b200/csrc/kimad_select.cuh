@@ -16,10 +16,17 @@ constexpr int kListCap = 32;                    // in-interval entries remembere
 constexpr uint32_t kListOverflow = 0xffffffffu; // more than that: the chunk is recounted exactly
 constexpr int kLowBins = 1024;                  // bins of the in-interval histogram
 
+// A chunk (at most 32768 elements from its 16-byte aligned start) is cut into 16 slices of 2048 elements; in
+// the sweeps of this stage a warp works on a slice by itself, so no sweep needs a block-wide barrier.
+constexpr int kSliceElems = 2048;
+constexpr int kSlices = 16;
+
 struct ChunkSel { // per (worker, chunk)
-    uint32_t above;          // entries whose key lies above the interval
-    uint32_t n_in;           // entries inside the interval, or kListOverflow
-    uint16_t low[kListCap];  // key - lo of those entries (any order)
+    uint32_t n_in;             // entries inside the interval, or kListOverflow
+    uint16_t above[kSlices];   // per slice: entries whose key lies above the interval; after k_sel_scan: entries kept
+                               // before the slice inside the chunk
+    uint16_t eq[kSlices];      // after k_sel_recount / k_sel_scan: entries equal to tau per slice, then before the slice
+    uint32_t low[kListCap];    // the entries inside the interval: slice << 16 | (key - lo), any order
 };
 
 // Second round of the select stage: layers whose interval was wider than 2^10 keys and whose entries
@@ -33,18 +40,25 @@ struct Round2 {
 constexpr int kSortCap = 4096;
 
 // ------------------------------------------------------------------------------------------------
-// Counting sweep of one chunk (the whole CTA works on it).
+// Counting sweep of one chunk: warp w takes the slices w and w + 8.
 __device__ __forceinline__ void sel_count_chunk(const float* __restrict__ dbuf, const Chunk& ch, uint32_t w,
                                                 uint32_t chunk_id, uint32_t n_chunks, uint64_t dstride, uint32_t L,
                                                 const Sel* __restrict__ sel, const LayerDesc* __restrict__ layers,
                                                 ChunkSel* __restrict__ csel, uint32_t* __restrict__ low_hist,
                                                 uint32_t* __restrict__ recount_n, uint2* __restrict__ recount_list,
-                                                uint32_t* s_w, uint32_t* s_hist, uint32_t* s_n, uint16_t* s_low) {
+                                                uint32_t* s_hist, uint32_t* s_n, uint32_t* s_low) {
     const size_t wl = (size_t)w * L + ch.layer;
     const Sel s = sel[wl];
     ChunkSel* out = csel + (size_t)w * n_chunks + chunk_id;
+    const ChunkView cv(ch);
+    const uint32_t lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     if (s.k == 0 || (uint64_t)s.k == layers[ch.layer].n) { // nothing / everything kept: no need to look at the data
-        if (threadIdx.x == 0) { out->above = s.k ? (uint32_t)(ch.end - ch.begin) : 0u; out->n_in = 0; }
+        if (threadIdx.x < kSlices) {
+            const uint32_t lo = max(cv.first, threadIdx.x * kSliceElems), hi = min(cv.len, (threadIdx.x + 1) * kSliceElems);
+            out->above[threadIdx.x] = (uint16_t)((s.k && hi > lo) ? hi - lo : 0u);
+            out->eq[threadIdx.x] = 0;
+        }
+        if (threadIdx.x == 0) out->n_in = 0;
         return;
     }
     const uint32_t lo = s.tau, width = 1u << s.shift;
@@ -52,42 +66,42 @@ __device__ __forceinline__ void sel_count_chunk(const float* __restrict__ dbuf, 
     for (int i = threadIdx.x; i < kLowBins; i += kThreads) s_hist[i] = 0;
     if (threadIdx.x == 0) *s_n = 0;
     __syncthreads();
-    const ChunkView cv(ch);
     const float* dd = dbuf + (size_t)w * dstride + cv.a0;
-    uint32_t above = 0;
-    auto visit = [&](float dv) {
-        const uint32_t d1 = key_of(dv) - lo; // wraps to >= 2^31 for keys below the interval
-        if (d1 < width) {
-            atomicAdd(&s_hist[d1 >> hshift], 1u);
-            const uint32_t p = atomicAdd(s_n, 1u);
-            if (p < (uint32_t)kListCap) s_low[p] = (uint16_t)d1;
-        } else {
-            above += d1 < 0x80000000u;
-        }
-    };
-    const uint32_t nq = cv.quads();
-    constexpr int U = 4;
-    for (uint32_t qb = 0; qb < nq; qb += kThreads * U) {
-        float4 a[U];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const uint32_t q = qb + u * kThreads + threadIdx.x;
-            if (q < nq && cv.quad_full(q)) a[u] = __ldcs(reinterpret_cast<const float4*>(dd) + q);
-        }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const uint32_t q = qb + u * kThreads + threadIdx.x;
-            if (q >= nq) continue;
-            if (cv.quad_full(q)) {
-                visit(a[u].x); visit(a[u].y); visit(a[u].z); visit(a[u].w);
+    for (uint32_t sl = wid; sl < (uint32_t)kSlices; sl += kThreads / 32) {
+        uint32_t above = 0;
+        auto visit = [&](float dv) {
+            const uint32_t d1 = key_of(dv) - lo; // wraps to >= 2^31 for keys below the interval
+            if (d1 < width) {
+                atomicAdd(&s_hist[d1 >> hshift], 1u);
+                const uint32_t p = atomicAdd(s_n, 1u);
+                if (p < (uint32_t)kListCap) s_low[p] = (sl << 16) | d1;
             } else {
-                for (uint32_t e = 4 * q; e < 4 * q + 4; ++e)
-                    if (e >= cv.first && e < cv.len) visit(dd[e]);
+                above += d1 < 0x80000000u;
+            }
+        };
+        constexpr int H = kSliceElems / 256; // quads per lane and half slice
+        for (uint32_t q0 = sl * (kSliceElems / 4); q0 < (sl + 1) * (kSliceElems / 4) && 4 * q0 < cv.len; q0 += H * 32) {
+            float4 a[H];
+#pragma unroll
+            for (int i = 0; i < H; ++i) {
+                const uint32_t q = q0 + i * 32 + lane;
+                if (cv.quad_full(q)) a[i] = __ldcs(reinterpret_cast<const float4*>(dd) + q);
+            }
+#pragma unroll
+            for (int i = 0; i < H; ++i) {
+                const uint32_t q = q0 + i * 32 + lane;
+                if (cv.quad_full(q)) {
+                    visit(a[i].x); visit(a[i].y); visit(a[i].z); visit(a[i].w);
+                } else if (4 * q < cv.len) {
+                    for (uint32_t e = 4 * q; e < 4 * q + 4; ++e)
+                        if (e >= cv.first && e < cv.len) visit(dd[e]);
+                }
             }
         }
+#pragma unroll
+        for (int o = 16; o; o >>= 1) above += __shfl_xor_sync(0xffffffffu, above, o);
+        if (lane == 0) { out->above[sl] = (uint16_t)above; out->eq[sl] = 0; }
     }
-    uint32_t tot;
-    block_excl_scan<uint32_t>(above, s_w, &tot);
     __syncthreads();
     const uint32_t n_in = *s_n;
     if (n_in) { // rare: publish this chunk's part of the layer's in-interval histogram
@@ -97,7 +111,6 @@ __device__ __forceinline__ void sel_count_chunk(const float* __restrict__ dbuf, 
     }
     if (threadIdx.x < min(n_in, (uint32_t)kListCap)) out->low[threadIdx.x] = s_low[threadIdx.x];
     if (threadIdx.x == 0) {
-        out->above = tot;
         if (n_in <= (uint32_t)kListCap) {
             out->n_in = n_in;
         } else {
@@ -112,12 +125,11 @@ __global__ void __launch_bounds__(kThreads)
 k_sel_count(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks, uint64_t dstride,
             uint32_t L, const Sel* __restrict__ sel, const LayerDesc* __restrict__ layers, ChunkSel* __restrict__ csel,
             uint32_t* __restrict__ low_hist, uint32_t* __restrict__ recount_n, uint2* __restrict__ recount_list) {
-    __shared__ uint32_t s_w[8];
     __shared__ uint32_t s_hist[kLowBins];
     __shared__ uint32_t s_n;
-    __shared__ uint16_t s_low[kListCap];
+    __shared__ uint32_t s_low[kListCap];
     sel_count_chunk(dbuf, chunks[blockIdx.x], blockIdx.y, blockIdx.x, n_chunks, dstride, L, sel, layers, csel, low_hist,
-                    recount_n, recount_list, s_w, s_hist, &s_n, s_low);
+                    recount_n, recount_list, s_hist, &s_n, s_low);
 }
 
 // second round: only the chunks of the layers listed in r2
@@ -126,15 +138,14 @@ k_sel_count_r2(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks,
                uint32_t L, const Sel* __restrict__ sel, const LayerDesc* __restrict__ layers,
                ChunkSel* __restrict__ csel, uint32_t* __restrict__ low_hist, uint32_t* __restrict__ recount_n,
                uint2* __restrict__ recount_list, const Round2* __restrict__ r2, const uint2* __restrict__ r2_chunks) {
-    __shared__ uint32_t s_w[8];
     __shared__ uint32_t s_hist[kLowBins];
     __shared__ uint32_t s_n;
-    __shared__ uint16_t s_low[kListCap];
+    __shared__ uint32_t s_low[kListCap];
     const uint32_t n = r2->n_chunks;
     for (uint32_t it = blockIdx.x; it < n; it += gridDim.x) {
         const uint2 e = r2_chunks[it];
         sel_count_chunk(dbuf, chunks[e.y], e.x, e.y, n_chunks, dstride, L, sel, layers, csel, low_hist, recount_n,
-                        recount_list, s_w, s_hist, &s_n, s_low);
+                        recount_list, s_hist, &s_n, s_low);
     }
 }
 
@@ -168,7 +179,7 @@ __device__ __forceinline__ void sel_resolve_layer(uint32_t l, uint32_t w, uint32
             if (!n_in) continue;
             const uint32_t at = atomicAdd(s_n, n_in);
             if (at + n_in > (uint32_t)kSortCap) { *s_over = 1; continue; }
-            for (uint32_t e = 0; e < n_in; ++e) s_key[at + e] = cs[i].low[e];
+            for (uint32_t e = 0; e < n_in; ++e) s_key[at + e] = cs[i].low[e] & 0xffffu;
         }
         __syncthreads();
         sorted = !*s_over;
@@ -255,45 +266,79 @@ k_sel_resolve_r2(uint32_t L, const LayerDesc* __restrict__ layers, uint32_t n_ch
                           r2_chunks, s_key, s_w32, &s_n, &s_over);
 }
 
-// Exact (gt, eq) of the chunks whose list overflowed.
+// Exact per-slice (gt, eq) of the chunks whose list overflowed: warp w recounts the slices w and w + 8.
 __global__ void __launch_bounds__(kThreads)
 k_sel_recount(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks, uint64_t dstride,
               uint32_t L, const Sel* __restrict__ sel, const uint32_t* __restrict__ recount_n,
-              const uint2* __restrict__ recount_list, uint2* __restrict__ chunk_cnt) {
-    __shared__ uint32_t s_w[8];
+              const uint2* __restrict__ recount_list, ChunkSel* __restrict__ csel) {
     const uint32_t n = *recount_n;
+    const uint32_t lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     for (uint32_t it = blockIdx.x; it < n; it += gridDim.x) {
         const uint2 e = recount_list[it];
         const Chunk ch = chunks[e.y];
         const Sel s = sel[(size_t)e.x * L + ch.layer];
         const ChunkView cv(ch);
         const float* dd = dbuf + (size_t)e.x * dstride + cv.a0;
-        uint32_t gt = 0, eq = 0;
-        for (uint32_t x = cv.first + threadIdx.x; x < cv.len; x += kThreads) {
-            const uint32_t key = key_of(dd[x]);
-            gt += key > s.tau;
-            eq += key == s.tau;
+        ChunkSel* out = csel + (size_t)e.x * n_chunks + e.y;
+        for (uint32_t sl = wid; sl < (uint32_t)kSlices; sl += kThreads / 32) {
+            uint32_t gt = 0, eq = 0;
+            const uint32_t x0 = max(cv.first, sl * kSliceElems), x1 = min(cv.len, (sl + 1) * kSliceElems);
+            for (uint32_t x = x0 + lane; x < x1; x += 32) {
+                const uint32_t key = key_of(dd[x]);
+                gt += key > s.tau;
+                eq += key == s.tau;
+            }
+#pragma unroll
+            for (int o = 16; o; o >>= 1) {
+                gt += __shfl_xor_sync(0xffffffffu, gt, o);
+                eq += __shfl_xor_sync(0xffffffffu, eq, o);
+            }
+            if (lane == 0) { out->above[sl] = (uint16_t)gt; out->eq[sl] = (uint16_t)eq; }
         }
-        uint32_t tg, te;
-        block_excl_scan<uint32_t>(gt, s_w, &tg);
-        block_excl_scan<uint32_t>(eq, s_w, &te);
-        if (threadIdx.x == 0) chunk_cnt[(size_t)e.x * n_chunks + e.y] = make_uint2(tg, te);
-        __syncthreads();
     }
 }
 
-// chunk_cnt[(w, chunk)] = (entries above tau, entries equal to tau); chunk_pre = exclusive prefix of
-// both over the layer's earlier chunks.
+// Per chunk (one warp each, lane = slice): entries above tau and equal to tau in every slice (from the lists, or
+// already recounted), turned into prefixes inside the chunk; chunk_cnt = the chunk's totals.
 __global__ void __launch_bounds__(kThreads)
-k_sel_scan(uint32_t L, const LayerDesc* __restrict__ layers, uint32_t n_chunks, const Sel* __restrict__ sel,
-           const ChunkSel* __restrict__ csel, uint2* __restrict__ chunk_cnt, uint2* __restrict__ chunk_pre,
-           uint32_t* __restrict__ recount_n, FbList* __restrict__ fb, Round2* __restrict__ r2) {
+k_sel_slices(const Chunk* __restrict__ chunks, uint32_t n_chunks, uint32_t W, uint32_t L, const Sel* __restrict__ sel,
+             ChunkSel* __restrict__ csel, uint2* __restrict__ chunk_cnt) {
+    const uint32_t lane = threadIdx.x & 31;
+    const uint64_t it = (uint64_t)blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
+    if (it >= (uint64_t)W * n_chunks) return;
+    const uint32_t w = (uint32_t)(it / n_chunks), ci = (uint32_t)(it % n_chunks);
+    const Sel s = sel[(size_t)w * L + chunks[ci].layer];
+    ChunkSel& c = csel[it];
+    uint32_t g = 0, q = 0;
+    if (lane < (uint32_t)kSlices) { g = c.above[lane]; q = c.eq[lane]; }
+    const uint32_t n_in = c.n_in;
+    if (n_in != kListOverflow)
+        for (uint32_t e = 0; e < n_in; ++e) { // entries inside the interval join their slice's counts
+            const uint32_t en = c.low[e];
+            if ((en >> 16) == lane) {
+                g += (en & 0xffffu) > s.tau_low;
+                q += (en & 0xffffu) == s.tau_low;
+            }
+        }
+    uint32_t ig = g, iq = q;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t yg = __shfl_up_sync(0xffffffffu, ig, o), yq = __shfl_up_sync(0xffffffffu, iq, o);
+        if (lane >= (uint32_t)o) { ig += yg; iq += yq; }
+    }
+    if (lane < (uint32_t)kSlices) { c.above[lane] = (uint16_t)(ig - g); c.eq[lane] = (uint16_t)(iq - q); }
+    if (lane == 31) chunk_cnt[it] = make_uint2(ig, iq);
+}
+
+// chunk_pre = exclusive prefix of the chunk totals over the layer's earlier chunks.
+__global__ void __launch_bounds__(kThreads)
+k_sel_scan(const LayerDesc* __restrict__ layers, uint32_t n_chunks, const uint2* __restrict__ chunk_cnt,
+           uint2* __restrict__ chunk_pre, uint32_t* __restrict__ recount_n, FbList* __restrict__ fb,
+           Round2* __restrict__ r2) {
     __shared__ uint32_t s_w[8];
     const LayerDesc ld = layers[blockIdx.x];
     const uint32_t w = blockIdx.y;
-    const Sel s = sel[(size_t)w * L + blockIdx.x];
-    const ChunkSel* cs = csel + (size_t)w * n_chunks + ld.first_chunk;
-    uint2* cc = chunk_cnt + (size_t)w * n_chunks + ld.first_chunk;
+    const uint2* cc = chunk_cnt + (size_t)w * n_chunks + ld.first_chunk;
     uint2* cp = chunk_pre + (size_t)w * n_chunks + ld.first_chunk;
     if (blockIdx.x == 0 && w == 0 && threadIdx.x == 0) { // all work lists have been consumed by now
         *recount_n = 0;
@@ -305,21 +350,7 @@ k_sel_scan(uint32_t L, const LayerDesc* __restrict__ layers, uint32_t n_chunks, 
     uint32_t run_g = 0, run_e = 0;
     for (uint32_t base = 0; base < ld.n_chunks; base += kThreads) {
         const uint32_t i = base + threadIdx.x;
-        uint2 v = make_uint2(0, 0);
-        if (i < ld.n_chunks) {
-            const uint32_t n_in = cs[i].n_in;
-            if (n_in == kListOverflow) {
-                v = cc[i];
-            } else {
-                v.x = cs[i].above;
-                for (uint32_t e = 0; e < n_in; ++e) {
-                    const uint32_t low = cs[i].low[e];
-                    v.x += low > s.tau_low;
-                    v.y += low == s.tau_low;
-                }
-                cc[i] = v;
-            }
-        }
+        const uint2 v = i < ld.n_chunks ? cc[i] : make_uint2(0, 0);
         uint32_t tg, te;
         const uint32_t eg = block_excl_scan<uint32_t>(v.x, s_w, &tg);
         const uint32_t ee = block_excl_scan<uint32_t>(v.y, s_w, &te);
@@ -330,17 +361,16 @@ k_sel_scan(uint32_t L, const LayerDesc* __restrict__ layers, uint32_t n_chunks, 
 }
 
 // ------------------------------------------------------------------------------------------------
-// (e) + (f).  Every thread owns 16 consecutive elements of a 4096-element round, so that ranks inside
-// a round follow the index order.
+// (e) + (f).  A warp compacts a slice by itself: every lane owns 16 consecutive elements of a 512-element
+// round, so that ranks inside a round follow the index order; positions come from warp scans.
 // ------------------------------------------------------------------------------------------------
 template <bool BF16>
 __global__ void __launch_bounds__(kThreads)
 k_sel_write(const float* __restrict__ dbuf, float* __restrict__ state, const Chunk* __restrict__ chunks,
             uint32_t n_chunks, uint64_t dstride, uint64_t stride, uint32_t L, const Sel* __restrict__ sel,
-            const LayerDesc* __restrict__ layers, const uint2* __restrict__ chunk_cnt,
-            const uint2* __restrict__ chunk_pre, uint64_t cap, uint32_t* __restrict__ out_idx,
-            void* __restrict__ out_val) {
-    __shared__ uint32_t s_w[8];
+            const LayerDesc* __restrict__ layers, const ChunkSel* __restrict__ csel,
+            const uint2* __restrict__ chunk_cnt, const uint2* __restrict__ chunk_pre, uint64_t cap,
+            uint32_t* __restrict__ out_idx, void* __restrict__ out_val) {
     const Chunk ch = chunks[blockIdx.x];
     const uint32_t w = blockIdx.y;
     const Sel s = sel[(size_t)w * L + ch.layer];
@@ -350,82 +380,96 @@ k_sel_write(const float* __restrict__ dbuf, float* __restrict__ state, const Chu
     const uint2 cnt = chunk_cnt[(size_t)w * n_chunks + blockIdx.x];
     const uint2 pre = chunk_pre[(size_t)w * n_chunks + blockIdx.x];
     if (!all && cnt.x == 0 && (cnt.y == 0 || pre.y >= s.keep_eq)) return; // nothing kept in this chunk
-    // entries equal to tau are kept while their rank among equals (ascending index) is below keep_eq
-    // eq_mode 0: none of this chunk's equals is kept; 1: all are; 2: ranks must be counted
-    const int eq_mode = (all || cnt.y == 0 || pre.y >= s.keep_eq) ? 0 : (pre.y + cnt.y <= s.keep_eq ? 1 : 2);
-    // keep <=> key > thr, with thr = tau - 1 when this chunk's equals are all kept (tau >= 1 then, or all)
+    const ChunkSel& cs = csel[(size_t)w * n_chunks + blockIdx.x];
     const uint32_t tau = s.tau;
-    uint32_t eq_seen = pre.y;
-    uint32_t pos = 0; // kept so far in this chunk
     const ChunkView cv(ch);
     const float* dd = dbuf + (size_t)w * dstride + cv.a0;
     float* st = state + (size_t)w * stride + cv.a0;
-    const uint64_t obase = (size_t)w * cap + s.base + pre.x + min(pre.y, s.keep_eq);
-    uint32_t* oi = out_idx + obase;
-    float* ov32 = reinterpret_cast<float*>(out_val) + obase;
-    __nv_bfloat16* ov16 = reinterpret_cast<__nv_bfloat16*>(out_val) + obase;
+    uint32_t* oi = out_idx + (size_t)w * cap + s.base;
+    float* ov32 = reinterpret_cast<float*>(out_val) + (size_t)w * cap + s.base;
+    __nv_bfloat16* ov16 = reinterpret_cast<__nv_bfloat16*>(out_val) + (size_t)w * cap + s.base;
     const uint32_t idx0 = (uint32_t)(cv.a0 - ld.begin); // layer-local index of offset 0 (may wrap; added back below)
+    const uint32_t lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
 
-    constexpr int E = 16;
-    for (uint32_t rb = 0; rb < cv.len; rb += E * kThreads) {
-        const uint32_t t0 = rb + E * threadIdx.x;
-        uint32_t keepm = 0, eqm = 0;
-        const bool interior = rb >= cv.first && rb + E * kThreads <= cv.len;
-        if (interior) {
-            float v[E];
+    for (uint32_t sl = wid; sl < (uint32_t)kSlices; sl += kThreads / 32) {
+        const uint32_t x0 = sl * kSliceElems;
+        if (x0 >= cv.len) break;
+        // entries equal to tau are kept while their rank among equals (ascending index) is below keep_eq
+        const uint32_t gt_before = pre.x + cs.above[sl], eq_before = pre.y + cs.eq[sl];
+        const uint32_t gt_here = (sl + 1 < (uint32_t)kSlices ? cs.above[sl + 1] : cnt.x) - cs.above[sl];
+        const uint32_t eq_here = (sl + 1 < (uint32_t)kSlices ? cs.eq[sl + 1] : cnt.y) - cs.eq[sl];
+        // eq_mode 0: none of this slice's equals is kept; 1: all are; 2: ranks must be counted
+        const int eq_mode = (all || eq_here == 0 || eq_before >= s.keep_eq) ? 0 : (eq_before + eq_here <= s.keep_eq ? 1 : 2);
+        if (!all && gt_here == 0 && eq_mode == 0) continue; // nothing kept in this slice
+        uint32_t eq_seen = eq_before;
+        uint32_t pos = gt_before + min(eq_before, s.keep_eq); // position of the slice's first kept entry in the layer
+        constexpr int E = 16;
+        for (uint32_t rb = x0; rb < min(cv.len, x0 + kSliceElems); rb += E * 32) {
+            const uint32_t t0 = rb + E * lane;
+            uint32_t keepm = 0, eqm = 0;
+            if (rb >= cv.first && rb + E * 32 <= cv.len) { // round fully inside the chunk
+                float v[E];
 #pragma unroll
-            for (int u = 0; u < E / 4; ++u) {
-                const float4 a = __ldg(reinterpret_cast<const float4*>(dd + t0) + u);
-                v[4 * u] = a.x; v[4 * u + 1] = a.y; v[4 * u + 2] = a.z; v[4 * u + 3] = a.w;
+                for (int u = 0; u < E / 4; ++u) {
+                    const float4 a = __ldg(reinterpret_cast<const float4*>(dd + t0) + u);
+                    v[4 * u] = a.x; v[4 * u + 1] = a.y; v[4 * u + 2] = a.z; v[4 * u + 3] = a.w;
+                }
+#pragma unroll
+                for (int i = 0; i < E; ++i) {
+                    const uint32_t key = key_of(v[i]);
+                    if (all || key > tau || (eq_mode == 1 && key == tau)) keepm |= 1u << i;
+                    if (eq_mode == 2 && key == tau) eqm |= 1u << i;
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < E; ++i) {
+                    const uint32_t e = t0 + i;
+                    const bool in = e >= cv.first && e < cv.len;
+                    const uint32_t key = key_of(in ? __ldg(dd + e) : 0.f);
+                    if (in && (all || key > tau || (eq_mode == 1 && key == tau))) keepm |= 1u << i;
+                    if (in && eq_mode == 2 && key == tau) eqm |= 1u << i;
+                }
             }
+            if (eq_mode == 2) { // uniform over the warp
+                uint32_t incl = __popc(eqm);
 #pragma unroll
-            for (int i = 0; i < E; ++i) {
-                const uint32_t key = key_of(v[i]);
-                if (all || key > tau || (eq_mode == 1 && key == tau)) keepm |= 1u << i;
-                if (eq_mode == 2 && key == tau) eqm |= 1u << i;
-            }
-        } else {
-#pragma unroll
-            for (int i = 0; i < E; ++i) {
-                const uint32_t e = t0 + i;
-                const bool in = e >= cv.first && e < cv.len;
-                const uint32_t key = key_of(in ? __ldg(dd + e) : 0.f);
-                if (in && (all || key > tau || (eq_mode == 1 && key == tau))) keepm |= 1u << i;
-                if (in && eq_mode == 2 && key == tau) eqm |= 1u << i;
-            }
-        }
-        if (!__syncthreads_or((keepm | eqm) != 0)) continue;
-        if (eq_mode == 2) { // uniform over the CTA
-            uint32_t tot_eq;
-            uint32_t eq_rank = eq_seen + block_excl_scan<uint32_t>(__popc(eqm), s_w, &tot_eq);
-#pragma unroll
-            for (int i = 0; i < E; ++i)
-                if (eqm & (1u << i)) {
-                    if (eq_rank < s.keep_eq) keepm |= 1u << i;
+                for (int o = 1; o < 32; o <<= 1) {
+                    const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= (uint32_t)o) incl += y;
+                }
+                uint32_t eq_rank = eq_seen + incl - __popc(eqm);
+                for (uint32_t m = eqm; m; m &= m - 1) {
+                    if (eq_rank < s.keep_eq) keepm |= m & (0u - m);
                     ++eq_rank;
                 }
-            eq_seen += tot_eq;
-        }
-        uint32_t tot_keep;
-        uint32_t o = pos + block_excl_scan<uint32_t>(__popc(keepm), s_w, &tot_keep);
-        pos += tot_keep;
-        while (keepm) {
-            const int i = __ffs(keepm) - 1;
-            keepm &= keepm - 1;
-            const uint32_t e = t0 + i;
-            const float val = dd[e]; // loaded a moment ago: an L1 hit
-            oi[o] = idx0 + e;
-            float sent;
-            if (BF16) {
-                const __nv_bfloat16 h = __float2bfloat16_rn(val);
-                ov16[o] = h;
-                sent = __bfloat162float(h);
-            } else {
-                ov32[o] = val;
-                sent = val;
+                eq_seen += __shfl_sync(0xffffffffu, incl, 31);
             }
-            st[e] = __fadd_rn(st[e], sent);
-            ++o;
+            uint32_t incl = __popc(keepm);
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= (uint32_t)o) incl += y;
+            }
+            uint32_t o = pos + incl - __popc(keepm);
+            pos += __shfl_sync(0xffffffffu, incl, 31);
+            while (keepm) {
+                const int i = __ffs(keepm) - 1;
+                keepm &= keepm - 1;
+                const uint32_t e = t0 + i;
+                const float val = dd[e]; // loaded a moment ago: an L1 hit
+                oi[o] = idx0 + e;
+                float sent;
+                if (BF16) {
+                    const __nv_bfloat16 h = __float2bfloat16_rn(val);
+                    ov16[o] = h;
+                    sent = __bfloat162float(h);
+                } else {
+                    ov32[o] = val;
+                    sent = val;
+                }
+                st[e] = __fadd_rn(st[e], sent);
+                ++o;
+            }
         }
     }
 }
