@@ -490,6 +490,7 @@ int kimad_debug_exact_path_layers(kimad_ctx* c, uint64_t* host_count) {
     CUDA_TRY(cudaMemcpy(&f, c->ws + c->lay.fb, sizeof(FbList), cudaMemcpyDeviceToHost));
     host_count[0] = f.total_layers;
     for (int i = 0; i < 4; ++i) host_count[1 + i] = f.why[i];
+    for (uint32_t j = 0; j < c->K; ++j) host_count[5 + j] = f.loose_j[j];
     return KIMAD_OK;
 }
 

@@ -180,18 +180,24 @@ k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint6
                 r_lo = a < 1.0 ? 0u : (uint32_t)a;
                 r_hi = b > (double)m ? 0u : (uint32_t)b;
             }
-            // rank window clipped at the top: the threshold may lie above the largest sample, so the band goes one
-            // octave further up; clipped at the bottom: no bound from the sample, exact path
+            // rank window clipped at the top: the threshold may lie above the largest sample, so the band goes a
+            // quarter octave further up; clipped at the bottom: no bound from the sample, exact path
             uint32_t c_top = cell_of_rank(max(r_lo, 1u));
-            if (r_lo == 0) c_top = min(c_top + 256u, 65279u);
+            if (r_lo == 0) c_top = min(c_top + 64u, 65279u);
             if (r_hi == 0 && lane == 0) s_flag = 1;
             const uint32_t c_bot = cell_of_rank(max(r_hi, 1u));
             const uint32_t ncell = c_top - c_bot + 1;
             if (ncell > (uint32_t)kFineBins) {
                 if (lane == 0) s_flag = 2;
             } else {
-                uint32_t inband = 0;
-                for (uint32_t c = c_bot + lane; c <= c_top; c += 32) inband += cell_count(c);
+                // sample entries in each quarter of the band (a tail band is much denser at its bottom)
+                const uint32_t nq = (ncell + 3) / 4;
+                uint32_t inq[4] = {0, 0, 0, 0};
+                for (uint32_t c = c_bot + lane; c <= c_top; c += 32) {
+                    const uint32_t cc = cell_count(c), qi = (c - c_bot) / nq;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) inq[i] += qi == (uint32_t)i ? cc : 0u;
+                }
                 // estimate of this candidate's error: squares of everything below the band
                 const uint32_t seg = (65535u - c_bot) >> 6;
                 double below = 0.0;
@@ -201,19 +207,28 @@ k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint6
                 }
 #pragma unroll
                 for (int o = 16; o; o >>= 1) {
-                    inband += __shfl_xor_sync(0xffffffffu, inband, o);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) inq[i] += __shfl_xor_sync(0xffffffffu, inq[i], o);
                     below += __shfl_xor_sync(0xffffffffu, below, o);
                 }
                 below += s_sq[seg];
                 const double scale = (double)n / (double)m;
-                const double per_cell = (double)inband / (double)ncell * scale; // entries per band cell
-                const double v2 = cell_sq(c_top);
                 // bins per cell: at most ~2048 entries per bin (what the select stage collects and sorts), and
                 // narrow enough that the uncertainty of the bin holding the threshold (its entries times its
-                // spread of squares, 2^-7 of v^2 for a whole cell) stays below ~1.5e-6 of the error
-                double bins = per_cell / 2048.0;
+                // spread of squares, 2^-7 of v^2 for a whole cell) stays below ~3e-6 of the error; entries per
+                // cell and v^2 are taken quarter by quarter
+                double dens = 0.0, load = 0.0;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const uint32_t qtop = min(c_top, c_bot + (uint32_t)(i + 1) * nq - 1);
+                    const double per_cell = (double)(inq[i] + 1) / (double)nq * scale; // + 1: never plan on an empty sample
+                    dens = per_cell > dens ? per_cell : dens;
+                    const double ld = per_cell * cell_sq(qtop);
+                    load = ld > load ? ld : load;
+                }
+                double bins = dens / 2048.0;
                 const double e_est = below * scale;
-                const double cert = e_est > 0.0 ? sqrt(per_cell * 0.0078125 * v2 / (1.5e-6 * e_est)) : 1024.0;
+                const double cert = e_est > 0.0 ? sqrt(load * 0.0078125 / (3e-6 * e_est)) : 1024.0;
                 if (cert > bins) bins = cert;
                 uint32_t sh_j = 15;
                 while (sh_j > 5 && (double)(1u << (15 - sh_j)) < bins) --sh_j;
@@ -581,7 +596,7 @@ k_resolve_a(const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ r
             double part = 0.5 * (upper + lower), slack = 0.5 * (upper - lower);
             if (drop == 0 || width == 1) { part = lower; slack = 0.0; }
             const double e = s_below[j] + part;
-            if (slack > e * 5e-6) { atomicMax(&s_bad, 4); continue; } // acceptance bound on the curve is 1e-5
+            if (slack > e * 5e-6) { atomicMax(&s_bad, 4); atomicAdd(&fb->loose_j[j], 1u); continue; } // acceptance bound on the curve is 1e-5
             err_out[o] = (float)e;
             tau_out[o] = klo;
             rank_out[o] = cb - drop;

@@ -141,6 +141,7 @@ struct FbList { // layers handed to the exact radix path in this step, and their
     uint32_t total_layers; // never reset: how many layers were handed over since the workspace was attached
     uint32_t why[5];       // never reset: ... because 0: forced, 1: bands too wide for the tables, 2: threshold
                            // outside its band, 3: error bound too loose
+    uint32_t loose_j[KIMAD_MAX_RATIOS + 1]; // never reset: which candidate's bound was too loose
 };
 
 __global__ void __launch_bounds__(kThreads)
