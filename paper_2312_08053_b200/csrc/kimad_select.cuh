@@ -20,6 +20,7 @@ constexpr int kLowBins = 1024;                  // bins of the in-interval histo
 // the sweeps of this stage a warp works on a slice by itself, so no sweep needs a block-wide barrier.
 constexpr int kSliceElems = 2048;
 constexpr int kSlices = 16;
+constexpr int kSparseGroups = 32; // the write sweep reads a slice group by group when at most this many are marked
 
 struct ChunkSel { // per (worker, chunk)
     uint32_t n_in;             // entries inside the interval, or kListOverflow
@@ -27,6 +28,9 @@ struct ChunkSel { // per (worker, chunk)
                                // before the slice inside the chunk
     uint16_t eq[kSlices];      // after k_sel_recount / k_sel_scan: entries equal to tau per slice, then before the slice
     uint32_t low[kListCap];    // the entries inside the interval: slice << 16 | (key - lo), any order
+    uint32_t _pad;
+    uint64_t mask[kSlices];    // per slice: bit g set when the 32-element group g may hold a kept entry (key >= the
+                               // interval's lower end); a superset of the groups the write sweep has to read
 };
 
 // Second round of the select stage: layers whose interval was wider than 2^10 keys and whose entries
@@ -69,7 +73,8 @@ __device__ __forceinline__ void sel_count_chunk(const float* __restrict__ dbuf, 
     const float* dd = dbuf + (size_t)w * dstride + cv.a0;
     for (uint32_t sl = wid; sl < (uint32_t)kSlices; sl += kThreads / 32) {
         uint32_t above = 0;
-        auto visit = [&](float dv) {
+        uint64_t mask = 0;
+        auto visit = [&](float dv) -> bool { // true: the key is not below the interval
             const uint32_t d1 = key_of(dv) - lo; // wraps to >= 2^31 for keys below the interval
             if (d1 < width) {
                 atomicAdd(&s_hist[d1 >> hshift], 1u);
@@ -78,6 +83,7 @@ __device__ __forceinline__ void sel_count_chunk(const float* __restrict__ dbuf, 
             } else {
                 above += d1 < 0x80000000u;
             }
+            return d1 < 0x80000000u;
         };
         constexpr int H = kSliceElems / 256; // quads per lane and half slice
         for (uint32_t q0 = sl * (kSliceElems / 4); q0 < (sl + 1) * (kSliceElems / 4) && 4 * q0 < cv.len; q0 += H * 32) {
@@ -90,17 +96,24 @@ __device__ __forceinline__ void sel_count_chunk(const float* __restrict__ dbuf, 
 #pragma unroll
             for (int i = 0; i < H; ++i) {
                 const uint32_t q = q0 + i * 32 + lane;
+                bool f = false;
                 if (cv.quad_full(q)) {
-                    visit(a[i].x); visit(a[i].y); visit(a[i].z); visit(a[i].w);
+                    f = visit(a[i].x); f |= visit(a[i].y); f |= visit(a[i].z); f |= visit(a[i].w);
                 } else if (4 * q < cv.len) {
                     for (uint32_t e = 4 * q; e < 4 * q + 4; ++e)
-                        if (e >= cv.first && e < cv.len) visit(dd[e]);
+                        if (e >= cv.first && e < cv.len) f |= visit(dd[e]);
                 }
+                // a row of 128 elements = four groups of 8 lanes
+                const uint32_t b = __ballot_sync(0xffffffffu, f);
+                const uint32_t nib = ((b & 0xffu) != 0) | (((b & 0xff00u) != 0) << 1) | (((b & 0xff0000u) != 0) << 2) |
+                                     (((b & 0xff000000u) != 0) << 3);
+                const uint32_t row = (q0 - sl * (kSliceElems / 4)) / 32 + i;
+                mask |= (uint64_t)nib << (4 * row);
             }
         }
 #pragma unroll
         for (int o = 16; o; o >>= 1) above += __shfl_xor_sync(0xffffffffu, above, o);
-        if (lane == 0) { out->above[sl] = (uint16_t)above; out->eq[sl] = 0; }
+        if (lane == 0) { out->above[sl] = (uint16_t)above; out->eq[sl] = 0; out->mask[sl] = mask; }
     }
     __syncthreads();
     const uint32_t n_in = *s_n;
@@ -390,6 +403,7 @@ k_sel_write(const float* __restrict__ dbuf, float* __restrict__ state, const Chu
     __nv_bfloat16* ov16 = reinterpret_cast<__nv_bfloat16*>(out_val) + (size_t)w * cap + s.base;
     const uint32_t idx0 = (uint32_t)(cv.a0 - ld.begin); // layer-local index of offset 0 (may wrap; added back below)
     const uint32_t lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    __shared__ uint8_t s_pos[kThreads / 32][kSparseGroups]; // per warp: the marked groups of a slice, ascending
 
     for (uint32_t sl = wid; sl < (uint32_t)kSlices; sl += kThreads / 32) {
         const uint32_t x0 = sl * kSliceElems;
@@ -403,6 +417,79 @@ k_sel_write(const float* __restrict__ dbuf, float* __restrict__ state, const Chu
         if (!all && gt_here == 0 && eq_mode == 0) continue; // nothing kept in this slice
         uint32_t eq_seen = eq_before;
         uint32_t pos = gt_before + min(eq_before, s.keep_eq); // position of the slice's first kept entry in the layer
+        const uint64_t gm = cs.mask[sl];
+        const uint32_t n_groups = __popcll(gm);
+        if (!all && n_groups <= (uint32_t)kSparseGroups) {
+            // sparse slice: read only the 32-element groups the counting sweep marked; a quarter warp per group,
+            // four groups per pass, in ascending order, so that lane order is index order
+            uint8_t* sp = s_pos[wid];
+            const uint32_t lo32 = (uint32_t)gm, hi32 = (uint32_t)(gm >> 32), lt = (1u << lane) - 1u;
+            __syncwarp();
+            if ((lo32 >> lane) & 1u) sp[__popc(lo32 & lt)] = (uint8_t)lane;
+            if ((hi32 >> lane) & 1u) sp[__popc(lo32) + __popc(hi32 & lt)] = (uint8_t)(32u + lane);
+            __syncwarp();
+            for (uint32_t it = 0; it < n_groups; it += 4) {
+                const uint32_t r = it + (lane >> 3);
+                uint32_t keepm = 0, eqm = 0, e0 = 0;
+                auto classify = [&](float v, int i) {
+                    const uint32_t key = key_of(v);
+                    if (key > tau || (eq_mode == 1 && key == tau)) keepm |= 1u << i;
+                    if (eq_mode == 2 && key == tau) eqm |= 1u << i;
+                };
+                if (r < n_groups) {
+                    e0 = x0 + (uint32_t)sp[r] * 32u + (lane & 7u) * 4u;
+                    if (e0 >= cv.first && e0 + 4 <= cv.len) {
+                        const float4 a = __ldg(reinterpret_cast<const float4*>(dd + e0));
+                        classify(a.x, 0); classify(a.y, 1); classify(a.z, 2); classify(a.w, 3);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            if (e0 + i >= cv.first && e0 + i < cv.len) classify(__ldg(dd + e0 + i), i);
+                    }
+                }
+                if (eq_mode == 2) { // uniform over the warp
+                    uint32_t incl = __popc(eqm);
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
+                        if (lane >= (uint32_t)o) incl += y;
+                    }
+                    uint32_t eq_rank = eq_seen + incl - __popc(eqm);
+                    for (uint32_t m = eqm; m; m &= m - 1) {
+                        if (eq_rank < s.keep_eq) keepm |= m & (0u - m);
+                        ++eq_rank;
+                    }
+                    eq_seen += __shfl_sync(0xffffffffu, incl, 31);
+                }
+                uint32_t incl = __popc(keepm);
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= (uint32_t)o) incl += y;
+                }
+                uint32_t o = pos + incl - __popc(keepm);
+                pos += __shfl_sync(0xffffffffu, incl, 31);
+                while (keepm) {
+                    const int i = __ffs(keepm) - 1;
+                    keepm &= keepm - 1;
+                    const uint32_t e = e0 + i;
+                    const float val = dd[e]; // loaded a moment ago: an L1 hit
+                    oi[o] = idx0 + e;
+                    float sent;
+                    if (BF16) {
+                        const __nv_bfloat16 h = __float2bfloat16_rn(val);
+                        ov16[o] = h;
+                        sent = __bfloat162float(h);
+                    } else {
+                        ov32[o] = val;
+                        sent = val;
+                    }
+                    st[e] = __fadd_rn(st[e], sent);
+                    ++o;
+                }
+            }
+            continue;
+        }
         constexpr int E = 16;
         for (uint32_t rb = x0; rb < min(cv.len, x0 + kSliceElems); rb += E * 32) {
             const uint32_t t0 = rb + E * lane;
