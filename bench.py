@@ -305,6 +305,82 @@ def run_kimad(args, rank, world):
     print(json.dumps(res))
 
 
+def run_receive(args, rank, world):
+    """Secondary line: the receiving side of one round (Algorithm 1, server lines) on the same workload:
+    kimad_apply_packed of the W workers' messages, then kimad_aggregate over the W estimators.  The
+    dominant kernel is the dense model step, (W + 2) * 4 bytes per model element."""
+    import torch
+
+    from paper_2312_08053_b200 import binding as kb
+
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", 0)))
+    torch.cuda.set_device(dev)
+    wl = workloads.workload(args.config)
+    W, N, L = wl.n_workers, wl.N, wl.L
+    bw = workloads.bandwidth_trace(wl)
+    bpe = 8 if wl.value_dtype == 0 else 6
+    cap = int(min(N, np.max(bw) * wl.t_target / bpe + L + 1))
+    ctx = kb.new_context(wl.layer_sizes, W, wl.ratio_grid, device=dev, D=wl.D, value_dtype=wl.value_dtype,
+                         max_packed_elems=cap)
+    n_msgs = 4
+    msgs = []
+    state = torch.zeros((W, N), dtype=torch.float32, device=dev)
+    for s in range(n_msgs):  # messages of consecutive rounds, produced by the compression pass itself
+        out = kb.Packed(ctx, device=dev)
+        g = workloads.gradients(wl, 1000 * rank + s, device=dev)
+        kb.kimad_step(ctx, g, state, bw[s % len(bw)], wl.t_target, out)
+        torch.cuda.synchronize()
+        del g
+        msgs.append(out)
+    est = torch.zeros((W, N), dtype=torch.float32, device=dev)
+    x = torch.zeros(N, dtype=torch.float32, device=dev)
+    wts = np.full(W, 1.0 / W, np.float32)
+    stream = torch.cuda.current_stream()
+    ev_a = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    ev_b = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    ev_c = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+
+    def step(s, i=None):
+        if i is not None:
+            ev_a[i].record(stream)
+        kb.kimad_apply_packed(ctx, msgs[s % n_msgs], est, stream)
+        if i is not None:
+            ev_b[i].record(stream)
+        kb.kimad_aggregate(x, est, wts, 0.01, stream)
+        if i is not None:
+            ev_c[i].record(stream)
+
+    for s in range(args.warmup):
+        step(s)
+    barrier()
+    torch.cuda.synchronize()
+    for i in range(args.steps):
+        step(args.warmup + i, i)
+    torch.cuda.synchronize()
+    barrier()
+    total_ms = max_over_ranks(ev_a[0].elapsed_time(ev_c[-1]))
+    apply_ms = float(np.mean([a.elapsed_time(b) for a, b in zip(ev_a, ev_b)]))
+    agg_ms = float(np.mean([b.elapsed_time(c) for b, c in zip(ev_b, ev_c)]))
+    if rank != 0:
+        return
+    peak, peak_kind = peaks()
+    ms_per_step = total_ms / args.steps
+    algo_b = (W + 2) * 4.0 * N
+    achieved = algo_b / (agg_ms * 1e-3) / 1e9
+    n_entries = float(np.mean([int(m.stats_host()["n_selected"].sum()) for m in msgs]))
+    print(json.dumps({
+        "metric": "received_update_elements_per_second", "value": W * N * world / (ms_per_step * 1e-3), "unit": UNIT,
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": wl.name + " / receive", "cfg": wl.cfg, "senders": W, "elements_per_sender": N,
+                   "packed_entries_per_step": n_entries, "l2": "inputs_larger_than_l2"},
+        "gpu_launches": 2 * args.steps,
+        "roofline": {"bound": "hbm", "kernel": "k_aggregate", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                     "algorithmic_bytes_per_launch": algo_b, "kernel_ms": agg_ms},
+        "stage_ms": {"apply_packed": apply_ms, "aggregate": agg_ms}}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -313,6 +389,8 @@ def main():
     ap.add_argument("--config", type=int, default=4, help="workload 1..5 (default 4: GPT-2-small shape, 4 workers)")
     ap.add_argument("--impl", default="kimad", choices=["kimad", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--path", default="compress", choices=["compress", "receive"],
+                    help="compress: the worker-side pass (the headline); receive: apply + aggregate on the server")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "kimad" else args.warmup
     rank = int(os.environ.get("RANK", 0))
@@ -321,6 +399,9 @@ def main():
         run_reference(args, rank)
         return
     init_distributed("nccl")
+    if args.path == "receive":
+        run_receive(args, rank, world)
+        return
     run_kimad(args, rank, world)
 
 

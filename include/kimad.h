@@ -64,7 +64,11 @@ typedef struct {
     uint64_t worker_stride;     /* elements between consecutive workers in grads/state; 0 -> N       */
     uint32_t curve_mode;        /* 0: error curves from one sweep over sampled bands, exact radix select
                                    only where the certificate fails; 1: exact radix select everywhere   */
-    uint32_t reserved;
+    uint32_t policy;            /* 0: Kimad+, the knapsack search over the layers (Section 3.2, Algorithm 3);
+                                   1: Kimad, one ratio of the grid for every layer: the largest whose total
+                                      size fits c (Section 3.1; the fixed-ratio baseline of Section 4.3).
+                                      A context with a single layer of N elements and policy 1 is the
+                                      whole-model TopK baseline of Section 4.3 on the same grid.           */
 } kimad_options;
 
 /* Per-worker result record, written by the device. */
@@ -151,6 +155,30 @@ int kimad_step_builtin_scratch(kimad_ctx* ctx, const float* grads_dev, float* st
  * cuda_stream.  Returns the most severe per-worker status of that step: the lowest negative
  * error if any worker failed, else the largest soft status, else 0. */
 int kimad_get_k(kimad_ctx* ctx, uint32_t* host_k, void* cuda_stream);
+
+/* ---- Receiving side of a message and the model step (Algorithm 1, server lines) ---------------------
+ *
+ * kimad_apply_packed: the receiver of the messages keeps, per sender m, a copy of that sender's
+ * estimator and adds every message to it: u^_m <- u^_m + C_m(u_m - u^_m) ("Aggregate all update
+ * estimators" in Algorithm 1; the same line updates the model estimator x^ on the workers when the
+ * server's message is the one received).  msg: the buffers a kimad_step of a context with the SAME layer
+ * list, worker count and value_dtype filled (device pointers; offs decides how many entries are read,
+ * so a failed worker, whose offs are all zero, adds nothing).  est_dev: device, f32, worker w at
+ * est_dev + w * worker_stride of ctx, layers concatenated as in grads; updated in place, one binary32
+ * add per entry (after a step, the receiver's copy is bit-identical to the sender's state).  Entries
+ * whose index is not below their layer's size are skipped.  Asynchronous on cuda_stream; the workspace
+ * must be attached (it holds the layer table).  Errors: INVALID_ARG, WORKSPACE, CUDA. */
+int kimad_apply_packed(const kimad_ctx* ctx, const kimad_packed* msg, float* est_dev, void* cuda_stream);
+
+/* kimad_aggregate: the model step x <- x - gamma * sum_m w_m u^_m (last line of Algorithm 1).
+ * x_dev: device f32 [n], in place.  est_dev: device f32, estimator m at est_dev + m * stride (stride
+ * >= n, in elements).  weights: HOST f32 [n_workers], n_workers in [1, KIMAD_MAX_AGG_WORKERS].
+ * binary32 throughout, in this order: acc = 0; acc = acc + w_m * est_m for m = 0, 1, ... (product and
+ * sum rounded separately, no FMA); x = x - gamma * acc.  Asynchronous on cuda_stream; no context
+ * needed.  Errors: INVALID_ARG, CUDA. */
+#define KIMAD_MAX_AGG_WORKERS 64
+int kimad_aggregate(float* x_dev, const float* est_dev, uint64_t stride, uint32_t n_workers, uint64_t n,
+                    const float* weights, float gamma, void* cuda_stream);
 
 /* Static tables (host-only calls).  host_k_table: u64 [L][K] candidates k_{l,j}. */
 int kimad_get_k_table(const kimad_ctx* ctx, uint64_t* host_k_table);

@@ -21,6 +21,14 @@
  *   O7  TopK select + sparse pack            (Algorithm 1, upload line)
  *   O8  EF21 estimator update u^ += C(d)     (Algorithm 1 aggregate line, Eq. 6)
  *
+ * and, beyond the worker-side pass:
+ *
+ *   O9  Kimad without layer adaptivity: one ratio of the grid for every layer, the
+ *       largest whose total size fits c      (Section 3.1; the baseline of Section 4.3)
+ *   O10 receiver side of a message: u^_m += C_m(.) as a scatter-add of the packed
+ *       entries                              (Algorithm 1, "Aggregate all update estimators")
+ *   O11 model step x <- x - gamma sum_m w_m u^_m   (Algorithm 1, last line)
+ *
  * Floating point: the element-wise operations (O1, O8, the DP adds) are single
  * IEEE binary32 operations in a fixed order, because the compared results must be
  * bit-identical.  The error curve is accumulated in binary64 from the smallest
@@ -32,7 +40,9 @@
  * hand-computed three-layer example (tests/golden/), torch's bfloat16 cast for
  * the bf16 rounding.  The whole-step composition has no value printed in the
  * paper to compare with: it is pinned by the identities g_new - g = C(d),
- * ||d - C(d)||^2 = err and sum(bytes) <= c only.
+ * ||d - C(d)||^2 = err and sum(bytes) <= c only.  O9: brute force over the grid;
+ * O10: the receiver's estimator equals the sender's after every message; O11:
+ * numpy float32 re-computation and the closed form for equal estimators.
  *
  * Build: gcc -O2 -ffp-contract=off -fopenmp -shared -fPIC (see kimad_oracle.py).
  */
@@ -312,20 +322,76 @@ int ko_get_threads(void) {
 #endif
 }
 
+/* O9: Kimad with one ratio for all layers (Section 3.1): the candidate index j is shared by the
+ * layers and is the largest one whose total size sum_l k_{l,j} (4 + vb) fits the budget c.  Same
+ * shortcuts and soft statuses as the layer-adaptive search: c >= full size -> PLATEAU (j = K-1),
+ * nothing fits (or c == 0) -> INFEASIBLE (j = 0). */
+int ko_uniform(const uint64_t* k_table, uint32_t L, uint32_t K, uint32_t value_dtype, uint64_t c, uint32_t* j_out) {
+    if (!k_table || !j_out || L == 0 || K == 0 || value_dtype > 1) return KO_ERR_ARG;
+    const uint64_t bpe = value_dtype == 0 ? 8 : 6;
+    int found = 0;
+    uint32_t best = 0;
+    for (uint32_t j = 0; j < K; ++j) {
+        uint64_t bytes = 0;
+        for (uint32_t l = 0; l < L; ++l) bytes += k_table[(size_t)l * K + j] * bpe;
+        if (bytes <= c) { found = 1; best = j; }
+    }
+    *j_out = best;
+    if (!found || c == 0) return KO_STATUS_INFEASIBLE;
+    if (best == K - 1) return KO_STATUS_PLATEAU;
+    return KO_OK;
+}
+
+/* O10: the receiver of a packed message adds it to its copy of the sender's estimator
+ * (Algorithm 1: u^_m <- u^_m + C_m(u_m - u^_m)).  est: [N] binary32, layers concatenated;
+ * idx layer-local, offs [L+1].  One binary32 add per received entry. */
+int ko_apply_packed(const uint64_t* layer_sizes, uint32_t L, const uint32_t* idx, const void* val,
+                    const uint64_t* offs, uint32_t value_dtype, float* est) {
+    if (!layer_sizes || !idx || !val || !offs || !est || value_dtype > 1) return KO_ERR_ARG;
+    uint64_t begin = 0;
+    for (uint32_t l = 0; l < L; ++l) {
+        for (uint64_t p = offs[l]; p < offs[l + 1]; ++p) {
+            if (idx[p] >= layer_sizes[l]) return KO_ERR_ARG;
+            float v = value_dtype == 0 ? ((const float*)val)[p] : ko_bf16_to_f32(((const uint16_t*)val)[p]);
+            est[begin + idx[p]] = est[begin + idx[p]] + v;
+        }
+        begin += layer_sizes[l];
+    }
+    return KO_OK;
+}
+
+/* O11: x_i <- x_i - gamma * sum_m w_m u^_{m,i} (Algorithm 1, last line).  binary32 throughout:
+ * the sum runs over m = 0..W-1 in order, every product and every add rounded once (no FMA). */
+int ko_aggregate(float* x, const float* est, uint64_t stride, uint32_t W, uint64_t N, const float* weights,
+                 float gamma) {
+    if (!x || !est || !weights || stride < N) return KO_ERR_ARG;
+    for (uint64_t i = 0; i < N; ++i) {
+        float acc = 0.0f;
+        for (uint32_t m = 0; m < W; ++m) {
+            float prod = weights[m] * est[(size_t)m * stride + i];
+            acc = acc + prod;
+        }
+        float stepv = gamma * acc;
+        x[i] = x[i] - stepv;
+    }
+    return KO_OK;
+}
+
 /* The whole pass (O1..O8) for W workers.  Layout:
  *   grads, state : [W][stride] binary32, layers concatenated in list order (stride >= N)
  *   err/tau/keep_eq out : [W][L][K];  j_out/k_out : [W][L]
  *   idx_out : [W][cap] layer-local indices; val_out : [W][cap] float or uint16 (bf16)
  *   offs_out : [W][L+1] running sum of k_l
  * state is updated in place.  When inject_err != NULL the DP consumes that [W][L][K] table
- * instead of the curves computed here (the curves are still computed and returned). */
-int ko_step(const uint64_t* layer_sizes, uint32_t L, uint32_t W, const double* ratios, uint32_t K, uint32_t D,
+ * instead of the curves computed here (the curves are still computed and returned).
+ * policy 0: layer-adaptive search O6 (Kimad+); policy 1: one ratio for all layers O9 (Kimad). */
+int ko_step_policy(uint32_t policy, const uint64_t* layer_sizes, uint32_t L, uint32_t W, const double* ratios, uint32_t K, uint32_t D,
             uint32_t value_dtype, uint64_t stride, const float* grads, float* state,
             const double* bandwidth_bytes_per_s, double t_target_s, const float* inject_err, float* err_out,
             uint32_t* tau_out, uint32_t* keep_eq_out, uint32_t* j_out, uint32_t* k_out, uint32_t* idx_out,
             void* val_out, uint64_t cap, uint64_t* offs_out, ko_stats* stats_out) {
     if (!layer_sizes || !ratios || !grads || !state || !bandwidth_bytes_per_s || L == 0 || W == 0 || K == 0 ||
-        value_dtype > 1)
+        value_dtype > 1 || policy > 1)
         return KO_ERR_ARG;
     uint64_t N = 0;
     for (uint32_t l = 0; l < L; ++l) N += layer_sizes[l];
@@ -372,7 +438,11 @@ int ko_step(const uint64_t* layer_sizes, uint32_t L, uint32_t W, const double* r
         if (!units) { rc = KO_ERR_NOMEM; goto done; }
         int s = ko_units(ktab, L, K, value_dtype, c, D, units);
         uint32_t* js = jsel + (size_t)w * L;
-        if (s == KO_STATUS_PLATEAU) {
+        if (policy == 1) {
+            uint32_t ju = 0;
+            s = ko_uniform(ktab, L, K, value_dtype, c, &ju);
+            for (uint32_t l = 0; l < L; ++l) js[l] = ju;
+        } else if (s == KO_STATUS_PLATEAU) {
             for (uint32_t l = 0; l < L; ++l) js[l] = K - 1;
         } else if (s == KO_STATUS_INFEASIBLE) {
             for (uint32_t l = 0; l < L; ++l) js[l] = 0;
@@ -443,4 +513,14 @@ int ko_step(const uint64_t* layer_sizes, uint32_t L, uint32_t W, const double* r
 done:
     free(ktab); free(loff); free(err); free(jsel); free(st); free(d);
     return rc;
+}
+
+int ko_step(const uint64_t* layer_sizes, uint32_t L, uint32_t W, const double* ratios, uint32_t K, uint32_t D,
+            uint32_t value_dtype, uint64_t stride, const float* grads, float* state,
+            const double* bandwidth_bytes_per_s, double t_target_s, const float* inject_err, float* err_out,
+            uint32_t* tau_out, uint32_t* keep_eq_out, uint32_t* j_out, uint32_t* k_out, uint32_t* idx_out,
+            void* val_out, uint64_t cap, uint64_t* offs_out, ko_stats* stats_out) {
+    return ko_step_policy(0, layer_sizes, L, W, ratios, K, D, value_dtype, stride, grads, state, bandwidth_bytes_per_s,
+                          t_target_s, inject_err, err_out, tau_out, keep_eq_out, j_out, k_out, idx_out, val_out, cap,
+                          offs_out, stats_out);
 }

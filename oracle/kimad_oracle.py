@@ -185,9 +185,45 @@ class StepResult:
     state: np.ndarray     # float32 [W][stride], the updated estimator
 
 
+def uniform(ktab: np.ndarray, value_dtype: int, c: int):
+    """O9: (status, j) of Kimad with one grid ratio for all layers under a budget of c bytes."""
+    kt = np.ascontiguousarray(ktab, dtype=np.uint64)
+    L, K = kt.shape
+    j = C.c_uint32(0)
+    rc = lib().ko_uniform(_p(kt, C.c_uint64), C.c_uint32(L), C.c_uint32(K), C.c_uint32(value_dtype), C.c_uint64(int(c)),
+                          C.byref(j))
+    if rc < 0:
+        _chk(rc, "uniform")
+    return rc, int(j.value)
+
+
+def apply_packed(layer_sizes, idx, val, offs, value_dtype, est) -> np.ndarray:
+    """O10: returns a copy of ``est`` ([N] float32) with one worker's packed message added."""
+    ls = np.ascontiguousarray(layer_sizes, dtype=np.uint64)
+    ix = np.ascontiguousarray(idx, dtype=np.uint32)
+    vv = np.ascontiguousarray(val, dtype=_val_dtype(value_dtype))
+    of = np.ascontiguousarray(offs, dtype=np.uint64)
+    out = np.array(est, dtype=np.float32, copy=True)
+    _chk(lib().ko_apply_packed(_p(ls, C.c_uint64), C.c_uint32(ls.size), _p(ix, C.c_uint32), vv.ctypes.data_as(C.c_void_p),
+                               _p(of, C.c_uint64), C.c_uint32(value_dtype), _p(out, C.c_float)), "apply_packed")
+    return out
+
+
+def aggregate(x, est, weights, gamma) -> np.ndarray:
+    """O11: returns x - gamma * sum_m w_m est[m] in float32, est [W][N]."""
+    e = np.ascontiguousarray(est, dtype=np.float32)
+    W, N = e.shape
+    out = np.array(x, dtype=np.float32, copy=True).reshape(N)
+    w = np.ascontiguousarray(weights, dtype=np.float32).reshape(W)
+    _chk(lib().ko_aggregate(_p(out, C.c_float), _p(e, C.c_float), C.c_uint64(N), C.c_uint32(W), C.c_uint64(N),
+                            _p(w, C.c_float), C.c_float(gamma)), "aggregate")
+    return out
+
+
 def step(layer_sizes, W, ratios, D, value_dtype, grads, state, bandwidth, t_target, cap=None,
-         inject_err=None) -> StepResult:
-    """One full pass O1..O8 for W workers; ``state`` is copied, the copy is updated and returned."""
+         inject_err=None, policy=0) -> StepResult:
+    """One full pass O1..O8 for W workers; ``state`` is copied, the copy is updated and returned.
+    policy 0: layer-adaptive DP (Kimad+); 1: one grid ratio for all layers (Kimad, O9)."""
     ls = np.ascontiguousarray(layer_sizes, dtype=np.uint64)
     r = np.ascontiguousarray(ratios, dtype=np.float64)
     L, K = ls.size, r.size
@@ -210,7 +246,7 @@ def step(layer_sizes, W, ratios, D, value_dtype, grads, state, bandwidth, t_targ
     inj = None
     if inject_err is not None:
         inj = np.ascontiguousarray(inject_err, dtype=np.float32).reshape(W, L, K)
-    _chk(lib().ko_step(_p(ls, C.c_uint64), C.c_uint32(L), C.c_uint32(W), _p(r, C.c_double), C.c_uint32(K),
+    _chk(lib().ko_step_policy(C.c_uint32(policy), _p(ls, C.c_uint64), C.c_uint32(L), C.c_uint32(W), _p(r, C.c_double), C.c_uint32(K),
                        C.c_uint32(D), C.c_uint32(value_dtype), C.c_uint64(stride), _p(grads, C.c_float),
                        _p(st_new, C.c_float), _p(bw, C.c_double), C.c_double(t_target), _p(inj, C.c_float),
                        _p(err, C.c_float), _p(tau, C.c_uint32), _p(keq, C.c_uint32), _p(j, C.c_uint32),

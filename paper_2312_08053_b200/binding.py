@@ -30,7 +30,7 @@ KIMAD_BUILTIN_SCRATCH_BYTES = 32 << 20
 class kimad_options(C.Structure):
     _fields_ = [("D", C.c_uint32), ("value_dtype", C.c_uint32), ("check_finite", C.c_uint32),
                 ("infeasible_policy", C.c_uint32), ("max_packed_elems", C.c_uint64), ("worker_stride", C.c_uint64),
-                ("curve_mode", C.c_uint32), ("reserved", C.c_uint32)]
+                ("curve_mode", C.c_uint32), ("policy", C.c_uint32)]
 
 
 class kimad_stats(C.Structure):
@@ -88,6 +88,10 @@ def load():
     L.kimad_debug_step_with_err.argtypes = step_args + [vp]
     L.kimad_debug_step_with_j.restype = C.c_int
     L.kimad_debug_step_with_j.argtypes = step_args + [vp]
+    L.kimad_apply_packed.restype = C.c_int
+    L.kimad_apply_packed.argtypes = [vp, C.POINTER(kimad_packed), vp, vp]
+    L.kimad_aggregate.restype = C.c_int
+    L.kimad_aggregate.argtypes = [vp, vp, u64, u32, u64, C.POINTER(C.c_float), C.c_float, vp]
     L.kimad_get_k.restype = C.c_int
     L.kimad_get_k.argtypes = [vp, vp, vp]
     L.kimad_get_k_table.restype = C.c_int
@@ -142,10 +146,10 @@ class Ctx:
 
 
 def kimad_create(layer_sizes, n_workers, ratio_grid, D=0, value_dtype=0, check_finite=0, max_packed_elems=0,
-                 worker_stride=0, curve_mode=0) -> Ctx:
+                 worker_stride=0, curve_mode=0, policy=0) -> Ctx:
     ls = np.ascontiguousarray(layer_sizes, dtype=np.uint64)
     rg = np.ascontiguousarray(ratio_grid, dtype=np.float64)
-    opts = kimad_options(D, value_dtype, check_finite, 0, max_packed_elems, worker_stride, curve_mode, 0)
+    opts = kimad_options(D, value_dtype, check_finite, 0, max_packed_elems, worker_stride, curve_mode, policy)
     h = C.c_void_p()
     _check(load().kimad_create(C.byref(h), ls.ctypes.data_as(C.POINTER(C.c_uint64)), ls.size, n_workers,
                                rg.ctypes.data_as(C.POINTER(C.c_double)), rg.size, C.byref(opts)), "kimad_create")
@@ -195,6 +199,20 @@ def _stream_ptr(stream):
 
         return torch.cuda.current_stream().cuda_stream
     return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def kimad_apply_packed(ctx: Ctx, msg: "Packed", est, stream=None) -> int:
+    """est: CUDA float32 tensor [W][ctx.stride], the receiver's copies of the senders' estimators (in place)."""
+    return _check(load().kimad_apply_packed(ctx.handle, C.byref(msg.c), est.data_ptr(), _stream_ptr(stream)),
+                  "kimad_apply_packed")
+
+
+def kimad_aggregate(x, est, weights, gamma, stream=None) -> int:
+    """x: CUDA float32 [n] (in place); est: CUDA float32 [W][stride]; weights: W host floats."""
+    w = np.ascontiguousarray(weights, dtype=np.float32)
+    return _check(load().kimad_aggregate(x.data_ptr(), est.data_ptr(), est.stride(0), w.size, x.numel(),
+                                         w.ctypes.data_as(C.POINTER(C.c_float)), C.c_float(gamma),
+                                         _stream_ptr(stream)), "kimad_aggregate")
 
 
 def _bw(ctx, bandwidth):

@@ -11,6 +11,7 @@ LIB_PATH = os.path.join(_HERE, "libkimad.so")
 SOURCES = [os.path.join(_HERE, "csrc", "kimad_api.cu")]
 HEADERS = [os.path.join(_HERE, "csrc", "kimad_kernels.cuh"), os.path.join(_HERE, "csrc", "kimad_select.cuh"),
            os.path.join(_HERE, "csrc", "kimad_curve.cuh"), os.path.join(_HERE, "csrc", "kimad_common.h"),
+           os.path.join(_HERE, "csrc", "kimad_receiver.cuh"),
            os.path.join(_ROOT, "include", "kimad.h")]
 
 

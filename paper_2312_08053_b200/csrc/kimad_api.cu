@@ -8,6 +8,7 @@
 #include <vector>
 
 #include "kimad_select.cuh"
+#include "kimad_receiver.cuh"
 
 using namespace kimad;
 
@@ -39,6 +40,7 @@ struct kimad_ctx {
     std::vector<LayerDesc> layers;
     std::vector<uint32_t> reg_layers, tiny_layers, reg_index; // layers above / up to kTinyMax elements
     uint32_t curve_mode = 0;
+    uint32_t policy = 0;
     size_t sample_smem = 0, pass_a_smem = 0, tiny_smem = 0;
     Layout lay{};
     unsigned char* ws = nullptr;
@@ -220,7 +222,7 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
             b.c[i] = !(cb > 0.0) ? 0ull : (cb >= 18446744073709551615.0 ? ~0ull : (uint64_t)cb);
         }
         k_dp<<<nw, kDpThreads, c->dp_smem, s>>>(b, w0, W, L, K, c->D, c->bpe, c->full_bytes, c->cap, c->check_finite,
-                                                mode == kGivenJ ? 1 : 0, c->dp_plan, ktab,
+                                                mode == kGivenJ ? 1 : (c->policy == 1 ? 2 : 0), c->dp_plan, ktab,
                                                 mode == kInjectErr ? err_dev : err, tau, keq, shf, j_dev, flags, pd, sel,
                                                 out->k, out->j, out->offs, out->stats);
         c->launches += 1;
@@ -266,7 +268,8 @@ int kimad_create(kimad_ctx** out, const uint64_t* layer_sizes, uint32_t n_layers
     kimad_options o{};
     if (opt) o = *opt;
     if (o.D == 0) o.D = 1000;
-    if (o.D > KIMAD_MAX_D || o.D < n_layers || o.value_dtype > 1 || o.infeasible_policy != 0 || o.curve_mode > 1)
+    if (o.D > KIMAD_MAX_D || o.D < n_layers || o.value_dtype > 1 || o.infeasible_policy != 0 || o.curve_mode > 1 ||
+        o.policy > 1)
         return KIMAD_ERR_INVALID_ARG;
     for (uint32_t j = 0; j < n_ratios; ++j) {
         if (!(ratio_grid[j] > 0.0) || ratio_grid[j] > 1.0) return KIMAD_ERR_INVALID_ARG;
@@ -330,6 +333,7 @@ int kimad_create(kimad_ctx** out, const uint64_t* layer_sizes, uint32_t n_layers
         if (c->dp_plan.pd_in_smem) used += pd_bytes;
         c->dp_smem = used;
         c->curve_mode = o.curve_mode;
+        c->policy = o.policy;
         c->sample_smem = (size_t)(2 * (1024 + 32) + 32768 + 2048 + 1024 + 2048 + 2048 + 32 + 3 * 128) * 4;
         c->pass_a_smem = (size_t)(3 * kMaxBins + kLutWords) * 4 + kL1Bins * 2;
         c->tiny_smem = (size_t)kTinyMax * (8 + 4);
@@ -409,6 +413,40 @@ int kimad_debug_step_with_j(kimad_ctx* ctx, const float* grads_dev, float* state
                             void* cuda_stream, const uint32_t* j_dev) {
     return run_step(ctx, grads_dev, state_dev, bandwidth_bytes_per_s, t_target_s, out, cuda_stream, kGivenJ, nullptr,
                     j_dev);
+}
+
+int kimad_apply_packed(const kimad_ctx* c, const kimad_packed* msg, float* est_dev, void* cuda_stream) {
+    if (!c || !msg || !msg->idx || !msg->val || !msg->offs || !est_dev) return KIMAD_ERR_INVALID_ARG;
+    if (!c->ws) return KIMAD_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const LayerDesc* layers = reinterpret_cast<const LayerDesc*>(c->ws + c->lay.layers);
+    const dim3 grid(148 * 4, c->W);
+    if (c->value_dtype == 1)
+        k_apply_packed<true><<<grid, kThreads, 0, s>>>(msg->idx, msg->val, msg->offs, layers, c->L, c->cap, c->stride, est_dev);
+    else
+        k_apply_packed<false><<<grid, kThreads, 0, s>>>(msg->idx, msg->val, msg->offs, layers, c->L, c->cap, c->stride, est_dev);
+    CUDA_TRY(cudaGetLastError());
+    return KIMAD_OK;
+}
+
+int kimad_aggregate(float* x_dev, const float* est_dev, uint64_t stride, uint32_t n_workers, uint64_t n,
+                    const float* weights, float gamma, void* cuda_stream) {
+    if (!x_dev || !est_dev || !weights || n_workers == 0 || n_workers > KIMAD_MAX_AGG_WORKERS || stride < n)
+        return KIMAD_ERR_INVALID_ARG;
+    if (n == 0) return KIMAD_OK;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    AggWeights wt{};
+    for (uint32_t m = 0; m < n_workers; ++m) wt.w[m] = weights[m];
+    const bool vec = (reinterpret_cast<uintptr_t>(x_dev) % 16 == 0) && (reinterpret_cast<uintptr_t>(est_dev) % 16 == 0) &&
+                     (stride % 4 == 0);
+    const uint64_t units = vec ? (n + 3) / 4 : n;
+    const uint32_t grid = (uint32_t)std::min<uint64_t>((units + kThreads - 1) / kThreads, 148ull * 16);
+    if (vec)
+        k_aggregate<true><<<grid, kThreads, 0, s>>>(x_dev, est_dev, stride, n_workers, n, wt, gamma);
+    else
+        k_aggregate<false><<<grid, kThreads, 0, s>>>(x_dev, est_dev, stride, n_workers, n, wt, gamma);
+    CUDA_TRY(cudaGetLastError());
+    return KIMAD_OK;
 }
 
 int kimad_get_k(kimad_ctx* c, uint32_t* host_k, void* cuda_stream) {

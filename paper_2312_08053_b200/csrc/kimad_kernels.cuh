@@ -314,7 +314,8 @@ struct DpPlan {
     uint32_t pd_row_bytes;
 };
 
-// mode 0: DP; mode 1: candidates given (j_in)
+// mode 0: DP (Kimad+); mode 1: candidates given (j_in); mode 2: one candidate index for all layers, the
+// largest whose total size fits the budget (Kimad without layer adaptivity, Section 3.1)
 __global__ void __launch_bounds__(kDpThreads)
 k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uint32_t D, uint32_t bpe,
      uint64_t full_bytes, uint64_t cap, uint32_t check_finite, int mode, DpPlan plan,
@@ -357,6 +358,20 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
         } else if (c == 0) {
             status = KIMAD_STATUS_INFEASIBLE;
             for (uint32_t l = threadIdx.x; l < L; l += blockDim.x) s_j[l] = 0;
+        } else if (mode == 2) {
+            // total size of candidate j over the layers, one thread per j; sizes ascend with j
+            __shared__ uint32_t s_fit; // number of candidates that fit
+            if (threadIdx.x == 0) s_fit = 0;
+            __syncthreads();
+            for (uint32_t j = threadIdx.x; j < K; j += blockDim.x) {
+                uint64_t bytes = 0;
+                for (uint32_t l = 0; l < L; ++l) bytes += ktab[(size_t)l * K + j] * bpe;
+                if (bytes <= c) atomicMax(&s_fit, j + 1);
+            }
+            __syncthreads();
+            const uint32_t fit = s_fit;
+            if (fit == 0) status = KIMAD_STATUS_INFEASIBLE;
+            for (uint32_t l = threadIdx.x; l < L; l += blockDim.x) s_j[l] = fit ? fit - 1 : 0;
         } else {
             // candidate (l, j) -> smem slot; units above D become D+1 (reads the +inf margin), padding likewise
             auto load_tab = [&](uint32_t l, uint32_t j, uint32_t slot_l) {

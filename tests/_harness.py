@@ -17,13 +17,15 @@ def u32(t):
 
 class Runner:
     def __init__(self, layer_sizes, W, grid, D=1000, value_dtype=0, stride=None, cap=None, check_finite=0,
-                 curve_mode=0):
+                 curve_mode=0, policy=0):
         self.ls, self.W, self.grid, self.D, self.vd = list(layer_sizes), W, list(grid), D, value_dtype
+        self.policy = policy
         self.N = int(sum(self.ls))
         self.stride = stride or self.N
         self.cap = cap or self.N
         self.ctx = kb.new_context(self.ls, W, self.grid, D=D, value_dtype=value_dtype, worker_stride=self.stride,
-                                  max_packed_elems=self.cap, check_finite=check_finite, curve_mode=curve_mode)
+                                  max_packed_elems=self.cap, check_finite=check_finite, curve_mode=curve_mode,
+                                  policy=policy)
         self.out = kb.Packed(self.ctx)
         self.kt = ko.k_table(self.ls, self.grid)
 
@@ -42,7 +44,8 @@ class Runner:
         err_g, tau_g, keq_g, shift_g = kb.kimad_debug_get_curve(self.ctx)
         tau_s, keq_s = kb.kimad_debug_get_selection(self.ctx)
         # oracle on its own curves
-        ref = ko.step(self.ls, W, self.grid, self.D, self.vd, g_host, s_host, bw, t, cap=self.cap)
+        ref = ko.step(self.ls, W, self.grid, self.D, self.vd, g_host, s_host, bw, t, cap=self.cap,
+                      policy=self.policy)
         # (b) curve: thresholds exact, error within tolerance
         # where all 31 bits were resolved the threshold must be the oracle's; elsewhere the oracle's
         # threshold must lie in the reported key interval
@@ -61,7 +64,7 @@ class Runner:
         assert not bad.any(), f"err off at {np.argwhere(bad)[:5]}: {err_g[bad][:5]} vs {ref.err[bad][:5]}"
         # (c)-(f): oracle DP fed the GPU's curve must reproduce the GPU bit for bit
         forced = ko.step(self.ls, W, self.grid, self.D, self.vd, g_host, s_host, bw, t, cap=self.cap,
-                         inject_err=err_g)
+                         inject_err=err_g, policy=self.policy)
         st = self.out.stats_host()
         assert np.array_equal(st["status"], forced.status), (st["status"], forced.status)
         assert np.array_equal(u32(self.out.j), forced.j), "chosen candidates differ from oracle DP on the same curve"
