@@ -240,12 +240,18 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
     k_sel_slices<<<(uint32_t)(((uint64_t)W * nch + 7) / 8), blk, 0, s>>>(chunks, nch, W, L, sel, csel, ccnt);
     k_sel_scan<<<glw, blk, 0, s>>>(layers, nch, ccnt, cpre, recount_n, fb, r2);
     mark();
-    if (c->value_dtype == 1)
-        k_sel_write<true><<<gch, blk, 0, s>>>(dbuf, state, chunks, nch, c->dstride, c->stride, L, sel, layers, csel, ccnt,
-                                              cpre, c->cap, out->idx, out->val);
-    else
-        k_sel_write<false><<<gch, blk, 0, s>>>(dbuf, state, chunks, nch, c->dstride, c->stride, L, sel, layers, csel, ccnt,
-                                               cpre, c->cap, out->idx, out->val);
+    {
+        // budget share kept, from the host's view of the budgets: picks the tuning of the write sweep
+        double kept = 0.0;
+        for (uint32_t i = 0; i < W; ++i) kept = std::max(kept, std::floor(bw[i] * t) / ((double)c->bpe * (double)c->N));
+        const bool dense = kept >= 0.04;
+        auto launch = [&](auto kern) {
+            kern<<<gch, blk, 0, s>>>(dbuf, state, chunks, nch, c->dstride, c->stride, L, sel, layers, csel, ccnt, cpre, c->cap,
+                                     out->idx, out->val);
+        };
+        if (c->value_dtype == 1) { if (dense) launch(k_sel_write<true, true>); else launch(k_sel_write<true, false>); }
+        else { if (dense) launch(k_sel_write<false, true>); else launch(k_sel_write<false, false>); }
+    }
     mark();
     c->launches += 8;
     CUDA_TRY(cudaGetLastError());

@@ -377,7 +377,9 @@ k_sel_scan(const LayerDesc* __restrict__ layers, uint32_t n_chunks, const uint2*
 // (e) + (f).  A warp compacts a slice by itself: every lane owns 16 consecutive elements of a 512-element
 // round, so that ranks inside a round follow the index order; positions come from warp scans.
 // ------------------------------------------------------------------------------------------------
-template <bool BF16>
+// DENSE: tuned for steps whose budget keeps more than a few per cent of the entries (the host picks the
+// instantiation from the budgets; both are correct for any input).
+template <bool BF16, bool DENSE>
 __global__ void __launch_bounds__(kThreads)
 k_sel_write(const float* __restrict__ dbuf, float* __restrict__ state, const Chunk* __restrict__ chunks,
             uint32_t n_chunks, uint64_t dstride, uint64_t stride, uint32_t L, const Sel* __restrict__ sel,
@@ -403,6 +405,7 @@ k_sel_write(const float* __restrict__ dbuf, float* __restrict__ state, const Chu
     __nv_bfloat16* ov16 = reinterpret_cast<__nv_bfloat16*>(out_val) + (size_t)w * cap + s.base;
     const uint32_t idx0 = (uint32_t)(cv.a0 - ld.begin); // layer-local index of offset 0 (may wrap; added back below)
     const uint32_t lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    const bool st_vec = (reinterpret_cast<uintptr_t>(st) & 15u) == 0;
     __shared__ uint8_t s_pos[kThreads / 32][kSparseGroups]; // per warp: the marked groups of a slice, ascending
 
     for (uint32_t sl = wid; sl < (uint32_t)kSlices; sl += kThreads / 32) {
@@ -494,8 +497,9 @@ k_sel_write(const float* __restrict__ dbuf, float* __restrict__ state, const Chu
         for (uint32_t rb = x0; rb < min(cv.len, x0 + kSliceElems); rb += E * 32) {
             const uint32_t t0 = rb + E * lane;
             uint32_t keepm = 0, eqm = 0;
-            if (rb >= cv.first && rb + E * 32 <= cv.len) { // round fully inside the chunk
-                float v[E];
+            const bool full = rb >= cv.first && rb + E * 32 <= cv.len; // round fully inside the chunk
+            float v[E];
+            if (full) {
 #pragma unroll
                 for (int u = 0; u < E / 4; ++u) {
                     const float4 a = __ldg(reinterpret_cast<const float4*>(dd + t0) + u);
@@ -538,7 +542,52 @@ k_sel_write(const float* __restrict__ dbuf, float* __restrict__ state, const Chu
                 if (lane >= (uint32_t)o) incl += y;
             }
             uint32_t o = pos + incl - __popc(keepm);
-            pos += __shfl_sync(0xffffffffu, incl, 31);
+            const uint32_t round_total = __shfl_sync(0xffffffffu, incl, 31);
+            pos += round_total;
+            if (DENSE && full && round_total >= 48u) {
+                // many kept entries: values come from the registers and the state is read before it is needed,
+                // so that no store waits for a load of its own
+                float sv[E];
+                if (st_vec) {
+#pragma unroll
+                    for (int u = 0; u < E / 4; ++u) {
+                        const float4 b = *(reinterpret_cast<const float4*>(st + t0) + u);
+                        sv[4 * u] = b.x; sv[4 * u + 1] = b.y; sv[4 * u + 2] = b.z; sv[4 * u + 3] = b.w;
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < E; ++i) sv[i] = (keepm >> i) & 1u ? st[t0 + i] : 0.f;
+                }
+#pragma unroll
+                for (int i = 0; i < E; ++i)
+                    if ((keepm >> i) & 1u) {
+                        oi[o] = idx0 + t0 + i;
+                        float sent;
+                        if (BF16) {
+                            const __nv_bfloat16 h = __float2bfloat16_rn(v[i]);
+                            ov16[o] = h;
+                            sent = __bfloat162float(h);
+                        } else {
+                            ov32[o] = v[i];
+                            sent = v[i];
+                        }
+                        sv[i] = __fadd_rn(sv[i], sent);
+                        ++o;
+                    }
+                if (st_vec) {
+                    if (keepm) {
+#pragma unroll
+                        for (int u = 0; u < E / 4; ++u)
+                            if ((keepm >> (4 * u)) & 15u)
+                                *(reinterpret_cast<float4*>(st + t0) + u) = make_float4(sv[4 * u], sv[4 * u + 1], sv[4 * u + 2], sv[4 * u + 3]);
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < E; ++i)
+                        if ((keepm >> i) & 1u) st[t0 + i] = sv[i];
+                }
+                continue;
+            }
             while (keepm) {
                 const int i = __ffs(keepm) - 1;
                 keepm &= keepm - 1;
