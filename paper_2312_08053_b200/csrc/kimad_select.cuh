@@ -93,6 +93,7 @@ __device__ __forceinline__ void sel_count_chunk(const float* __restrict__ dbuf, 
                 const uint32_t q = q0 + i * 32 + lane;
                 if (cv.quad_full(q)) a[i] = __ldcs(reinterpret_cast<const float4*>(dd) + q);
             }
+            uint32_t fb = 0; // bit i: this lane's quad of row i holds a key that is not below the interval
 #pragma unroll
             for (int i = 0; i < H; ++i) {
                 const uint32_t q = q0 + i * 32 + lane;
@@ -103,13 +104,17 @@ __device__ __forceinline__ void sel_count_chunk(const float* __restrict__ dbuf, 
                     for (uint32_t e = 4 * q; e < 4 * q + 4; ++e)
                         if (e >= cv.first && e < cv.len) f |= visit(dd[e]);
                 }
-                // a row of 128 elements = four groups of 8 lanes
-                const uint32_t b = __ballot_sync(0xffffffffu, f);
-                const uint32_t nib = ((b & 0xffu) != 0) | (((b & 0xff00u) != 0) << 1) | (((b & 0xff0000u) != 0) << 2) |
-                                     (((b & 0xff000000u) != 0) << 3);
-                const uint32_t row = (q0 - sl * (kSliceElems / 4)) / 32 + i;
-                mask |= (uint64_t)nib << (4 * row);
+                fb |= (uint32_t)f << i;
             }
+            // a row of 128 elements = four groups of 8 lanes: OR the rows' flags inside each group, spread the
+            // 8 row bits to every fourth position, shift by the group, and OR the four groups
+            const uint32_t g = lane >> 3;
+            uint32_t r8 = __reduce_or_sync(0xffu << (8 * g), fb);
+            r8 = (r8 | (r8 << 12)) & 0x000f000fu;
+            r8 = (r8 | (r8 << 6)) & 0x03030303u;
+            r8 = (r8 | (r8 << 3)) & 0x11111111u;
+            const uint32_t half = __reduce_or_sync(0xffffffffu, r8 << g);
+            mask |= (uint64_t)half << (32 * ((q0 - sl * (kSliceElems / 4)) / (H * 32)));
         }
 #pragma unroll
         for (int o = 16; o; o >>= 1) above += __shfl_xor_sync(0xffffffffu, above, o);
