@@ -94,7 +94,7 @@ void plan_layout(kimad_ctx* c) {
     y.shift = take(WLK * sizeof(uint32_t));
     y.sel = take(WL * sizeof(Sel));
     y.chunk_cnt = take((size_t)c->W * nch * sizeof(uint2));
-    y.chunk_pre = take((size_t)c->W * nch * sizeof(uint2));
+    y.chunk_pre = take((size_t)c->W * nch * sizeof(ChunkJob));
     y.csel = take((size_t)c->W * nch * sizeof(ChunkSel));
     y.fb_chunks = take((size_t)c->W * nch * sizeof(uint2));
     y.fb_layers = take(WL * sizeof(uint2));
@@ -151,7 +151,7 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
     uint32_t* shf = c->at<uint32_t>(y.shift);
     Sel* sel = c->at<Sel>(y.sel);
     uint2* ccnt = c->at<uint2>(y.chunk_cnt);
-    uint2* cpre = c->at<uint2>(y.chunk_pre);
+    ChunkJob* jobs = c->at<ChunkJob>(y.chunk_pre);
     ChunkSel* csel = c->at<ChunkSel>(y.csel);
     uint32_t* lowh = c->at<uint32_t>(y.low_hist);
     uint32_t* recount_n = c->at<uint32_t>(y.recount);
@@ -238,7 +238,7 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
                                                                    r2_chunks);
     k_sel_recount<<<2 * 148, blk, 0, s>>>(dbuf, chunks, nch, c->dstride, L, sel, recount_n, recount_list, csel);
     k_sel_slices<<<(uint32_t)(((uint64_t)W * nch + 7) / 8), blk, 0, s>>>(chunks, nch, W, L, sel, csel, ccnt);
-    k_sel_scan<<<glw, blk, 0, s>>>(layers, nch, ccnt, cpre, recount_n, fb, r2);
+    k_sel_scan<<<glw, blk, 0, s>>>(layers, chunks, nch, L, sel, ccnt, jobs, recount_n, fb, r2);
     mark();
     {
         // budget share kept, from the host's view of the budgets: picks the tuning of the write sweep
@@ -246,8 +246,7 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
         for (uint32_t i = 0; i < W; ++i) kept = std::max(kept, std::floor(bw[i] * t) / ((double)c->bpe * (double)c->N));
         const bool dense = kept >= 0.04;
         auto launch = [&](auto kern) {
-            kern<<<gch, blk, 0, s>>>(dbuf, state, chunks, nch, c->dstride, c->stride, L, sel, layers, csel, ccnt, cpre, c->cap,
-                                     out->idx, out->val);
+            kern<<<gch, blk, 0, s>>>(dbuf, state, chunks, nch, c->dstride, c->stride, csel, jobs, c->cap, out->idx, out->val);
         };
         if (c->value_dtype == 1) { if (dense) launch(k_sel_write<true, true>); else launch(k_sel_write<true, false>); }
         else { if (dense) launch(k_sel_write<false, true>); else launch(k_sel_write<false, false>); }

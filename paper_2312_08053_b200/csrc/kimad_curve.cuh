@@ -414,7 +414,7 @@ k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, float
         const uint32_t key = key_of(dv);
         const uint32_t e1 = t1[key >> 20];
         const bool split = e1 & 0x8000u;
-        const uint32_t e2 = t2[(split ? (e1 & 0x7fffu) : 0u) * 32 + ((key >> 15) & 31u)];
+        const uint32_t e2 = split ? t2[(e1 & 0x7fffu) * 32 + ((key >> 15) & 31u)] : 0u; // lanes outside split bins issue no load
         const uint32_t id = split ? (e2 & 0xffffu) + ((key & 0x7fffu) >> (e2 >> 16)) : e1;
         // 24 significant bits of the square (truncation < 2^-22 relative), in two 12-bit halves: a run has at
         // most 2^20 elements, so neither u32 sum can overflow before the flush at the end of the run

@@ -33,6 +33,20 @@ struct ChunkSel { // per (worker, chunk)
                                // interval's lower end); a superset of the groups the write sweep has to read
 };
 
+// Everything the write sweep needs to know about a (worker, chunk) besides the data, gathered by k_sel_scan so
+// that the write sweep starts from loads whose addresses depend on the block index only.
+struct ChunkJob {
+    uint32_t mode;      // 0: nothing of this chunk is kept; 1: threshold tau; 2: the whole layer is kept
+    uint32_t tau;
+    uint32_t keep_eq;   // entries equal to tau that are kept, over the layer (lowest indices first)
+    uint32_t gt_before; // entries above tau in the layer's earlier chunks
+    uint32_t eq_before; // entries equal to tau in the layer's earlier chunks
+    uint32_t cnt_gt;    // entries above tau / equal to tau in this chunk
+    uint32_t cnt_eq;
+    uint32_t idx0;      // layer-local index of the chunk's aligned start (may wrap; added back by the sweep)
+    uint64_t base;      // first output position of the layer in the worker's packed buffers
+};
+
 // Second round of the select stage: layers whose interval was wider than 2^10 keys and whose entries
 // inside it could not be collected (a chunk list overflowed, or more than kSortCap entries) get their
 // interval narrowed by the coarse histogram and are counted once more over their own chunks.
@@ -348,16 +362,18 @@ k_sel_slices(const Chunk* __restrict__ chunks, uint32_t n_chunks, uint32_t W, ui
     if (lane == 31) chunk_cnt[it] = make_uint2(ig, iq);
 }
 
-// chunk_pre = exclusive prefix of the chunk totals over the layer's earlier chunks.
+// Exclusive prefix of the chunk totals over the layer's earlier chunks, stored with the layer's threshold as the
+// write sweep's job record of every chunk.
 __global__ void __launch_bounds__(kThreads)
-k_sel_scan(const LayerDesc* __restrict__ layers, uint32_t n_chunks, const uint2* __restrict__ chunk_cnt,
-           uint2* __restrict__ chunk_pre, uint32_t* __restrict__ recount_n, FbList* __restrict__ fb,
-           Round2* __restrict__ r2) {
+k_sel_scan(const LayerDesc* __restrict__ layers, const Chunk* __restrict__ chunks, uint32_t n_chunks, uint32_t L,
+           const Sel* __restrict__ sel, const uint2* __restrict__ chunk_cnt, ChunkJob* __restrict__ jobs,
+           uint32_t* __restrict__ recount_n, FbList* __restrict__ fb, Round2* __restrict__ r2) {
     __shared__ uint32_t s_w[8];
     const LayerDesc ld = layers[blockIdx.x];
     const uint32_t w = blockIdx.y;
+    const Sel s = sel[(size_t)w * L + blockIdx.x];
     const uint2* cc = chunk_cnt + (size_t)w * n_chunks + ld.first_chunk;
-    uint2* cp = chunk_pre + (size_t)w * n_chunks + ld.first_chunk;
+    ChunkJob* jb = jobs + (size_t)w * n_chunks + ld.first_chunk;
     if (blockIdx.x == 0 && w == 0 && threadIdx.x == 0) { // all work lists have been consumed by now
         *recount_n = 0;
         fb->n_chunks = 0;
@@ -365,6 +381,7 @@ k_sel_scan(const LayerDesc* __restrict__ layers, uint32_t n_chunks, const uint2*
         r2->n_chunks = 0;
         r2->n_layers = 0;
     }
+    const bool all = (uint64_t)s.k == ld.n;
     uint32_t run_g = 0, run_e = 0;
     for (uint32_t base = 0; base < ld.n_chunks; base += kThreads) {
         const uint32_t i = base + threadIdx.x;
@@ -372,7 +389,21 @@ k_sel_scan(const LayerDesc* __restrict__ layers, uint32_t n_chunks, const uint2*
         uint32_t tg, te;
         const uint32_t eg = block_excl_scan<uint32_t>(v.x, s_w, &tg);
         const uint32_t ee = block_excl_scan<uint32_t>(v.y, s_w, &te);
-        if (i < ld.n_chunks) cp[i] = make_uint2(run_g + eg, run_e + ee);
+        if (i < ld.n_chunks) {
+            const ChunkView cv(chunks[ld.first_chunk + i]);
+            ChunkJob j;
+            j.tau = s.tau;
+            j.keep_eq = s.keep_eq;
+            j.gt_before = run_g + eg;
+            j.eq_before = run_e + ee;
+            j.cnt_gt = v.x;
+            j.cnt_eq = v.y;
+            j.idx0 = (uint32_t)(cv.a0 - ld.begin);
+            j.base = s.base;
+            const bool none = s.k == 0 || (!all && v.x == 0 && (v.y == 0 || j.eq_before >= s.keep_eq));
+            j.mode = none ? 0u : (all ? 2u : 1u);
+            jb[i] = j;
+        }
         run_g += tg;
         run_e += te;
     }
@@ -387,28 +418,24 @@ k_sel_scan(const LayerDesc* __restrict__ layers, uint32_t n_chunks, const uint2*
 template <bool BF16, bool DENSE>
 __global__ void __launch_bounds__(kThreads)
 k_sel_write(const float* __restrict__ dbuf, float* __restrict__ state, const Chunk* __restrict__ chunks,
-            uint32_t n_chunks, uint64_t dstride, uint64_t stride, uint32_t L, const Sel* __restrict__ sel,
-            const LayerDesc* __restrict__ layers, const ChunkSel* __restrict__ csel,
-            const uint2* __restrict__ chunk_cnt, const uint2* __restrict__ chunk_pre, uint64_t cap,
-            uint32_t* __restrict__ out_idx, void* __restrict__ out_val) {
-    const Chunk ch = chunks[blockIdx.x];
+            uint32_t n_chunks, uint64_t dstride, uint64_t stride, const ChunkSel* __restrict__ csel,
+            const ChunkJob* __restrict__ jobs, uint64_t cap, uint32_t* __restrict__ out_idx, void* __restrict__ out_val) {
     const uint32_t w = blockIdx.y;
-    const Sel s = sel[(size_t)w * L + ch.layer];
-    if (s.k == 0) return;
-    const LayerDesc ld = layers[ch.layer];
-    const bool all = (uint64_t)s.k == ld.n;
-    const uint2 cnt = chunk_cnt[(size_t)w * n_chunks + blockIdx.x];
-    const uint2 pre = chunk_pre[(size_t)w * n_chunks + blockIdx.x];
-    if (!all && cnt.x == 0 && (cnt.y == 0 || pre.y >= s.keep_eq)) return; // nothing kept in this chunk
+    const ChunkJob jb = jobs[(size_t)w * n_chunks + blockIdx.x];
+    if (jb.mode == 0) return; // nothing kept in this chunk
+    const Chunk ch = chunks[blockIdx.x];
     const ChunkSel& cs = csel[(size_t)w * n_chunks + blockIdx.x];
-    const uint32_t tau = s.tau;
+    const bool all = jb.mode == 2;
+    const uint2 cnt = make_uint2(jb.cnt_gt, jb.cnt_eq), pre = make_uint2(jb.gt_before, jb.eq_before);
+    struct { uint32_t keep_eq; } s = {jb.keep_eq};
+    const uint32_t tau = jb.tau;
     const ChunkView cv(ch);
     const float* dd = dbuf + (size_t)w * dstride + cv.a0;
     float* st = state + (size_t)w * stride + cv.a0;
-    uint32_t* oi = out_idx + (size_t)w * cap + s.base;
-    float* ov32 = reinterpret_cast<float*>(out_val) + (size_t)w * cap + s.base;
-    __nv_bfloat16* ov16 = reinterpret_cast<__nv_bfloat16*>(out_val) + (size_t)w * cap + s.base;
-    const uint32_t idx0 = (uint32_t)(cv.a0 - ld.begin); // layer-local index of offset 0 (may wrap; added back below)
+    uint32_t* oi = out_idx + (size_t)w * cap + jb.base;
+    float* ov32 = reinterpret_cast<float*>(out_val) + (size_t)w * cap + jb.base;
+    __nv_bfloat16* ov16 = reinterpret_cast<__nv_bfloat16*>(out_val) + (size_t)w * cap + jb.base;
+    const uint32_t idx0 = jb.idx0;
     const uint32_t lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const bool st_vec = (reinterpret_cast<uintptr_t>(st) & 15u) == 0;
     __shared__ uint8_t s_pos[kThreads / 32][kSparseGroups]; // per warp: the marked groups of a slice, ascending
@@ -444,15 +471,31 @@ k_sel_write(const float* __restrict__ dbuf, float* __restrict__ state, const Chu
                     if (key > tau || (eq_mode == 1 && key == tau)) keepm |= 1u << i;
                     if (eq_mode == 2 && key == tau) eqm |= 1u << i;
                 };
+                float vq[4] = {0.f, 0.f, 0.f, 0.f}, sq[4] = {0.f, 0.f, 0.f, 0.f}; // d and the state of this lane's quad
                 if (r < n_groups) {
                     e0 = x0 + (uint32_t)sp[r] * 32u + (lane & 7u) * 4u;
                     if (e0 >= cv.first && e0 + 4 <= cv.len) {
+                        // the state is requested together with d: a kept entry's update then waits for one
+                        // memory round trip, not two
                         const float4 a = __ldg(reinterpret_cast<const float4*>(dd + e0));
-                        classify(a.x, 0); classify(a.y, 1); classify(a.z, 2); classify(a.w, 3);
+                        if (st_vec) {
+                            const float4 b = *reinterpret_cast<const float4*>(st + e0);
+                            sq[0] = b.x; sq[1] = b.y; sq[2] = b.z; sq[3] = b.w;
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) sq[i] = st[e0 + i];
+                        }
+                        vq[0] = a.x; vq[1] = a.y; vq[2] = a.z; vq[3] = a.w;
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) classify(vq[i], i);
                     } else {
 #pragma unroll
                         for (int i = 0; i < 4; ++i)
-                            if (e0 + i >= cv.first && e0 + i < cv.len) classify(__ldg(dd + e0 + i), i);
+                            if (e0 + i >= cv.first && e0 + i < cv.len) {
+                                vq[i] = __ldg(dd + e0 + i);
+                                sq[i] = st[e0 + i];
+                                classify(vq[i], i);
+                            }
                     }
                 }
                 if (eq_mode == 2) { // uniform over the warp
@@ -477,24 +520,22 @@ k_sel_write(const float* __restrict__ dbuf, float* __restrict__ state, const Chu
                 }
                 uint32_t o = pos + incl - __popc(keepm);
                 pos += __shfl_sync(0xffffffffu, incl, 31);
-                while (keepm) {
-                    const int i = __ffs(keepm) - 1;
-                    keepm &= keepm - 1;
-                    const uint32_t e = e0 + i;
-                    const float val = dd[e]; // loaded a moment ago: an L1 hit
-                    oi[o] = idx0 + e;
-                    float sent;
-                    if (BF16) {
-                        const __nv_bfloat16 h = __float2bfloat16_rn(val);
-                        ov16[o] = h;
-                        sent = __bfloat162float(h);
-                    } else {
-                        ov32[o] = val;
-                        sent = val;
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    if ((keepm >> i) & 1u) {
+                        oi[o] = idx0 + e0 + i;
+                        float sent;
+                        if (BF16) {
+                            const __nv_bfloat16 h = __float2bfloat16_rn(vq[i]);
+                            ov16[o] = h;
+                            sent = __bfloat162float(h);
+                        } else {
+                            ov32[o] = vq[i];
+                            sent = vq[i];
+                        }
+                        st[e0 + i] = __fadd_rn(sq[i], sent);
+                        ++o;
                     }
-                    st[e] = __fadd_rn(st[e], sent);
-                    ++o;
-                }
             }
             continue;
         }
