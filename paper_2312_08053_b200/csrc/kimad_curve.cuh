@@ -6,8 +6,9 @@
 //                (sample rank +- 6 sigma) form a band.  Band cells are cut into fine bins of 2^shift
 //                keys, everything else into coarse "gap" bins; the mapping key -> bin is a two-level
 //                table (11-bit bin -> row, row x 5 more bits -> bin base and shift).
-//   k_pass_a     the sweep: d = grad - g (written to scratch), bin = table(key(d)), three u32 shared-
-//                memory atomics per element (count, and the exact integer sum of squares in two halves).
+//   k_pass_a     the sweep: d = grad - g (written to scratch), bin = table(key(d)), two u32 shared-
+//                memory atomics per element: the count, and the exact integer sum of squares in a low u32 word
+//                whose (rare) carries go to a high word.
 //   k_resolve_a  per (worker, layer): walks the bins from the top, finds the bin that holds every
 //                candidate's threshold, sums the squares below it.  The candidate's error is certified
 //                to 2^-19 relative from the bin's width; if a threshold fell into a gap bin (the sample
@@ -369,7 +370,7 @@ k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint6
 // ------------------------------------------------------------------------------------------------
 // k_pass_a: CTAs own runs of consecutive chunks; histogram words live in shared memory
 // ------------------------------------------------------------------------------------------------
-constexpr int kMaxRunChunksA = 32; // a run has at most 2^20 elements: the u32 sums of 12-bit halves cannot overflow
+constexpr int kMaxRunChunksA = 32; // a run has at most 2^20 elements: its carry count stays far below 2^32
 
 template <bool VEC>
 __global__ void __launch_bounds__(kBigThreads, 1)
@@ -384,7 +385,7 @@ k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, float
     uint32_t* h_lo = sh + 2 * kMaxBins;
     uint32_t* t2 = sh + 3 * kMaxBins;                           // [kLutWords] cell rows, then gap ids
     uint16_t* t1 = reinterpret_cast<uint16_t*>(t2 + kLutWords); // [2048]
-    static_assert((uint64_t)kMaxRunChunksA * kChunkElems <= (1ull << 20), "u32 sums of 12-bit halves");
+    static_assert((uint64_t)kMaxRunChunksA * kChunkElems <= (1ull << 20), "run length");
     const uint32_t w = blockIdx.y;
     const uint32_t c0 = blockIdx.x * run_chunks, c1 = min(n_chunks, c0 + run_chunks);
     for (int i = threadIdx.x; i < 3 * kMaxBins; i += kBigThreads) sh[i] = 0;
@@ -403,7 +404,7 @@ k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, float
             const uint32_t c = h_cnt[i];
             if (c) {
                 atomicAdd(&gc[i], c);
-                atomicAdd(&gs[i], ((unsigned long long)h_hi[i] << 12) + h_lo[i]);
+                atomicAdd(&gs[i], ((unsigned long long)h_hi[i] << 32) + h_lo[i]);
                 h_cnt[i] = 0; h_hi[i] = 0; h_lo[i] = 0;
             }
         }
@@ -416,12 +417,12 @@ k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, float
         const bool split = e1 & 0x8000u;
         const uint32_t e2 = split ? t2[(e1 & 0x7fffu) * 32 + ((key >> 15) & 31u)] : 0u; // lanes outside split bins issue no load
         const uint32_t id = split ? (e2 & 0xffffu) + ((key & 0x7fffu) >> (e2 >> 16)) : e1;
-        // 24 significant bits of the square (truncation < 2^-22 relative), in two 12-bit halves: a run has at
-        // most 2^20 elements, so neither u32 sum can overflow before the flush at the end of the run
+        // 24 significant bits of the square (truncation < 2^-22 relative) summed exactly: the low word wraps, the
+        // returned old value tells when, and the wraps are counted in the high word
         const uint32_t sq = (uint32_t)(sq_fixed(key) >> 8);
         atomicAdd(&h_cnt[id], 1u);
-        atomicAdd(&h_hi[id], sq >> 12);
-        atomicAdd(&h_lo[id], sq & 0xfffu);
+        const uint32_t old = atomicAdd(&h_lo[id], sq);
+        if (old + sq < old) atomicAdd(&h_hi[id], 1u); // carry out of the low word (rare)
     };
 
     for (uint32_t c = c0; c < c1; ++c) {
