@@ -68,7 +68,14 @@ typedef struct {
                                    1: Kimad, one ratio of the grid for every layer: the largest whose total
                                       size fits c (Section 3.1; the fixed-ratio baseline of Section 4.3).
                                       A context with a single layer of N elements and policy 1 is the
-                                      whole-model TopK baseline of Section 4.3 on the same grid.           */
+                                      whole-model TopK baseline of Section 4.3 on the same grid.
+                                   2: Algorithm 3 read the other way round (its header speaks of an error
+                                      budget E_max and a step E_max / D): the knapsack axis is the error,
+                                      e_{l,j} = floor(err_{l,j} D / E_max) cells with E_max = sum_l err_{l,0}
+                                      (binary64), the value is the number of kept entries, and the answer is
+                                      the lowest error level whose smallest size fits c.  Needs L * K small
+                                      enough for the candidate tables to sit in shared memory (else
+                                      kimad_create returns INVALID_ARG).                                     */
 } kimad_options;
 
 /* Per-worker result record, written by the device. */

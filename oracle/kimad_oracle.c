@@ -28,6 +28,9 @@
  *   O10 receiver side of a message: u^_m += C_m(.) as a scatter-add of the packed
  *       entries                              (Algorithm 1, "Aggregate all update estimators")
  *   O11 model step x <- x - gamma sum_m w_m u^_m   (Algorithm 1, last line)
+ *   O12 the other reading of Algorithm 3: the knapsack axis is the discretised ERROR (its header:
+ *       "compression budget E_max", "discretization step E_max / D", "discretized L2"), the value the
+ *       size; the answer is the lowest error level whose smallest size fits c
  *
  * Floating point: the element-wise operations (O1, O8, the DP adds) are single
  * IEEE binary32 operations in a fixed order, because the compared results must be
@@ -42,7 +45,8 @@
  * paper to compare with: it is pinned by the identities g_new - g = C(d),
  * ||d - C(d)||^2 = err and sum(bytes) <= c only.  O9: brute force over the grid;
  * O10: the receiver's estimator equals the sender's after every message; O11:
- * numpy float32 re-computation and the closed form for equal estimators.
+ * numpy float32 re-computation and the closed form for equal estimators.  O12: exhaustive
+ * enumeration of the discretised objective.
  *
  * Build: gcc -O2 -ffp-contract=off -fopenmp -shared -fPIC (see kimad_oracle.py).
  */
@@ -377,6 +381,76 @@ int ko_aggregate(float* x, const float* est, uint64_t stride, uint32_t W, uint64
     return KO_OK;
 }
 
+/* O12: Algorithm 3 read with the ERROR as the knapsack axis (the reading its header suggests).
+ *   E_max  = sum_l err_{l,0} in binary64, layers in order: the error of the most aggressive candidate
+ *            everywhere, i.e. the largest total error any assignment can have;
+ *   cells  e_{l,j} = floor(err_{l,j} * D / E_max) (binary64 product, then quotient), 0 when E_max = 0;
+ *            rounding DOWN keeps every assignment on the axis: sum_l e_{l,j_l} <= D;
+ *   DP     value[l][e] = fewest kept entries sum k_{l,j} over assignments of layers 1..l whose cells add
+ *            up to exactly e; virtual row [0, inf, ...]; candidates ascending, strict '<';
+ *   answer the lowest e with value[L][e] * (4 + vb) <= c, then the walk back through PD.
+ * Same shortcuts and statuses as O6: c >= full size -> PLATEAU; nothing fits -> INFEASIBLE, all j = 0. */
+int ko_dp_error_axis(const float* err /* [L][K] */, const uint64_t* k_table /* [L][K] */, uint32_t L, uint32_t K,
+                     uint32_t D, uint32_t value_dtype, uint64_t c, uint32_t* j_out /* [L] */, uint32_t* best_cell) {
+    if (!err || !k_table || !j_out || L == 0 || K == 0 || D == 0 || value_dtype > 1) return KO_ERR_ARG;
+    const uint64_t bpe = value_dtype == 0 ? 8 : 6;
+    uint64_t full = 0;
+    for (uint32_t l = 0; l < L; ++l) full += k_table[(size_t)l * K + (K - 1)] * bpe;
+    if (c >= full) {
+        for (uint32_t l = 0; l < L; ++l) j_out[l] = K - 1;
+        return KO_STATUS_PLATEAU;
+    }
+    const uint64_t INF = UINT64_MAX;
+    const size_t row = (size_t)D + 1;
+    uint64_t* prev = (uint64_t*)malloc(row * sizeof(uint64_t));
+    uint64_t* cur = (uint64_t*)malloc(row * sizeof(uint64_t));
+    uint32_t* cells = (uint32_t*)malloc((size_t)L * K * sizeof(uint32_t));
+    uint8_t* pd = (uint8_t*)malloc((size_t)L * row);
+    if (!prev || !cur || !cells || !pd) { free(prev); free(cur); free(cells); free(pd); return KO_ERR_NOMEM; }
+    double emax = 0.0;
+    for (uint32_t l = 0; l < L; ++l) emax = emax + (double)err[(size_t)l * K];
+    for (size_t i = 0; i < (size_t)L * K; ++i) {
+        double q = 0.0;
+        if (emax > 0.0) {
+            double prod = (double)err[i] * (double)D;
+            q = floor(prod / emax);
+        }
+        cells[i] = q > (double)D ? D : (uint32_t)q;
+    }
+    for (size_t b = 0; b < row; ++b) prev[b] = INF;
+    prev[0] = 0;
+    for (uint32_t l = 0; l < L; ++l) {
+        for (size_t b = 0; b < row; ++b) cur[b] = INF;
+        for (uint32_t j = 0; j < K; ++j) {
+            const uint32_t u = cells[(size_t)l * K + j];
+            const uint64_t k = k_table[(size_t)l * K + j];
+            for (size_t b = u; b < row; ++b) {
+                if (prev[b - u] == INF) continue;
+                uint64_t t = prev[b - u] + k;
+                if (t < cur[b]) { cur[b] = t; pd[(size_t)l * row + b] = (uint8_t)j; }
+            }
+        }
+        uint64_t* sw = prev; prev = cur; cur = sw;
+    }
+    int status = KO_STATUS_INFEASIBLE;
+    size_t bstar = 0;
+    for (size_t b = 0; b < row; ++b)
+        if (prev[b] != INF && prev[b] * bpe <= c) { bstar = b; status = KO_OK; break; }
+    if (status == KO_OK) {
+        if (best_cell) *best_cell = (uint32_t)bstar;
+        size_t b = bstar;
+        for (uint32_t l = L; l-- > 0;) {
+            uint32_t j = pd[(size_t)l * row + b];
+            j_out[l] = j;
+            b -= cells[(size_t)l * K + j];
+        }
+    } else {
+        for (uint32_t l = 0; l < L; ++l) j_out[l] = 0;
+    }
+    free(prev); free(cur); free(cells); free(pd);
+    return status;
+}
+
 /* The whole pass (O1..O8) for W workers.  Layout:
  *   grads, state : [W][stride] binary32, layers concatenated in list order (stride >= N)
  *   err/tau/keep_eq out : [W][L][K];  j_out/k_out : [W][L]
@@ -384,14 +458,15 @@ int ko_aggregate(float* x, const float* est, uint64_t stride, uint32_t W, uint64
  *   offs_out : [W][L+1] running sum of k_l
  * state is updated in place.  When inject_err != NULL the DP consumes that [W][L][K] table
  * instead of the curves computed here (the curves are still computed and returned).
- * policy 0: layer-adaptive search O6 (Kimad+); policy 1: one ratio for all layers O9 (Kimad). */
+ * policy 0: layer-adaptive search O6 (Kimad+); policy 1: one ratio for all layers O9 (Kimad);
+ * policy 2: layer-adaptive search on the error axis O12. */
 int ko_step_policy(uint32_t policy, const uint64_t* layer_sizes, uint32_t L, uint32_t W, const double* ratios, uint32_t K, uint32_t D,
             uint32_t value_dtype, uint64_t stride, const float* grads, float* state,
             const double* bandwidth_bytes_per_s, double t_target_s, const float* inject_err, float* err_out,
             uint32_t* tau_out, uint32_t* keep_eq_out, uint32_t* j_out, uint32_t* k_out, uint32_t* idx_out,
             void* val_out, uint64_t cap, uint64_t* offs_out, ko_stats* stats_out) {
     if (!layer_sizes || !ratios || !grads || !state || !bandwidth_bytes_per_s || L == 0 || W == 0 || K == 0 ||
-        value_dtype > 1 || policy > 1)
+        value_dtype > 1 || policy > 2)
         return KO_ERR_ARG;
     uint64_t N = 0;
     for (uint32_t l = 0; l < L; ++l) N += layer_sizes[l];
@@ -442,6 +517,9 @@ int ko_step_policy(uint32_t policy, const uint64_t* layer_sizes, uint32_t L, uin
             uint32_t ju = 0;
             s = ko_uniform(ktab, L, K, value_dtype, c, &ju);
             for (uint32_t l = 0; l < L; ++l) js[l] = ju;
+        } else if (policy == 2) {
+            s = ko_dp_error_axis(e, ktab, L, K, D, value_dtype, c, js, NULL);
+            if (s < 0) { free(units); rc = s; goto done; }
         } else if (s == KO_STATUS_PLATEAU) {
             for (uint32_t l = 0; l < L; ++l) js[l] = K - 1;
         } else if (s == KO_STATUS_INFEASIBLE) {

@@ -197,6 +197,20 @@ def uniform(ktab: np.ndarray, value_dtype: int, c: int):
     return rc, int(j.value)
 
 
+def dp_error_axis(err: np.ndarray, ktab: np.ndarray, D: int, value_dtype: int, c: int):
+    """O12: (status, j [L], lowest feasible error cell) of the error-axis reading of Algorithm 3."""
+    e = np.ascontiguousarray(err, dtype=np.float32)
+    kt = np.ascontiguousarray(ktab, dtype=np.uint64)
+    L, K = e.shape
+    j = np.zeros(L, np.uint32)
+    cell = C.c_uint32(0)
+    rc = lib().ko_dp_error_axis(_p(e, C.c_float), _p(kt, C.c_uint64), C.c_uint32(L), C.c_uint32(K), C.c_uint32(D),
+                                C.c_uint32(value_dtype), C.c_uint64(int(c)), _p(j, C.c_uint32), C.byref(cell))
+    if rc < 0:
+        _chk(rc, "dp_error_axis")
+    return rc, j, int(cell.value)
+
+
 def apply_packed(layer_sizes, idx, val, offs, value_dtype, est) -> np.ndarray:
     """O10: returns a copy of ``est`` ([N] float32) with one worker's packed message added."""
     ls = np.ascontiguousarray(layer_sizes, dtype=np.uint64)
@@ -223,7 +237,8 @@ def aggregate(x, est, weights, gamma) -> np.ndarray:
 def step(layer_sizes, W, ratios, D, value_dtype, grads, state, bandwidth, t_target, cap=None,
          inject_err=None, policy=0) -> StepResult:
     """One full pass O1..O8 for W workers; ``state`` is copied, the copy is updated and returned.
-    policy 0: layer-adaptive DP (Kimad+); 1: one grid ratio for all layers (Kimad, O9)."""
+    policy 0: layer-adaptive DP (Kimad+); 1: one grid ratio for all layers (Kimad, O9); 2: the DP on the
+    error axis (O12)."""
     ls = np.ascontiguousarray(layer_sizes, dtype=np.uint64)
     r = np.ascontiguousarray(ratios, dtype=np.float64)
     L, K = ls.size, r.size

@@ -109,6 +109,8 @@ void plan_layout(kimad_ctx* c) {
         if ((x) != cudaSuccess) return KIMAD_ERR_CUDA; \
     } while (0)
 
+constexpr size_t kDpSmemMax = 225 * 1024; // dynamic shared memory the DP kernel may ask for
+
 enum StepMode { kNormal = 0, kInjectErr = 1, kGivenJ = 2 };
 
 int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, double t, const kimad_packed* out,
@@ -222,7 +224,7 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
             b.c[i] = !(cb > 0.0) ? 0ull : (cb >= 18446744073709551615.0 ? ~0ull : (uint64_t)cb);
         }
         k_dp<<<nw, kDpThreads, c->dp_smem, s>>>(b, w0, W, L, K, c->D, c->bpe, c->full_bytes, c->cap, c->check_finite,
-                                                mode == kGivenJ ? 1 : (c->policy == 1 ? 2 : 0), c->dp_plan, ktab,
+                                                mode == kGivenJ ? 1 : (c->policy == 1 ? 2 : (c->policy == 2 ? 3 : 0)), c->dp_plan, ktab,
                                                 mode == kInjectErr ? err_dev : err, tau, keq, shf, j_dev, flags, pd, sel,
                                                 out->k, out->j, out->offs, out->stats);
         c->launches += 1;
@@ -274,7 +276,7 @@ int kimad_create(kimad_ctx** out, const uint64_t* layer_sizes, uint32_t n_layers
     if (opt) o = *opt;
     if (o.D == 0) o.D = 1000;
     if (o.D > KIMAD_MAX_D || o.D < n_layers || o.value_dtype > 1 || o.infeasible_policy != 0 || o.curve_mode > 1 ||
-        o.policy > 1)
+        o.policy > 2)
         return KIMAD_ERR_INVALID_ARG;
     for (uint32_t j = 0; j < n_ratios; ++j) {
         if (!(ratio_grid[j] > 0.0) || ratio_grid[j] > 1.0) return KIMAD_ERR_INVALID_ARG;
@@ -324,7 +326,6 @@ int kimad_create(kimad_ctx** out, const uint64_t* layer_sizes, uint32_t n_layers
         if (c->stride < N || c->chunks.size() > 0x7fffffffull) { delete c; return KIMAD_ERR_INVALID_ARG; }
         c->dstride = (N + 3) / 4 * 4;
         // shared-memory plan of the DP kernel
-        const size_t kDpSmemMax = 225 * 1024;
         const size_t Kp = (c->K + 3) & ~(size_t)3;
         const size_t dp_base = ((size_t)2 * (2 * c->D + 3) + c->L) * 4;
         const size_t tab_all = (size_t)c->L * (Kp * 8 + 4), tab_one = Kp * 8 + 4;
@@ -339,6 +340,7 @@ int kimad_create(kimad_ctx** out, const uint64_t* layer_sizes, uint32_t n_layers
         c->dp_smem = used;
         c->curve_mode = o.curve_mode;
         c->policy = o.policy;
+        if (c->policy == 2 && !c->dp_plan.tab_in_smem) { delete c; return KIMAD_ERR_INVALID_ARG; }
         c->sample_smem = (size_t)(2 * (1024 + 32) + 32768 + 2048 + 1024 + 2048 + 2048 + 32 + 3 * 128) * 4;
         c->pass_a_smem = (size_t)(3 * kMaxBins + kLutWords) * 4 + kL1Bins * 2;
         c->tiny_smem = (size_t)kTinyMax * (8 + 4);
@@ -391,7 +393,8 @@ int kimad_set_workspace(kimad_ctx* c, void* dev_ptr, size_t bytes) {
     CUDA_TRY(cudaMemcpy(c->ws + y.reg_index, c->reg_index.data(), c->reg_index.size() * 4, cudaMemcpyHostToDevice));
     // histograms, work lists and flags start at zero and are kept clean by the kernels that consume them
     CUDA_TRY(cudaMemset(c->ws + y.zero_from, 0, y.lut_t1 - y.zero_from));
-    CUDA_TRY(cudaFuncSetAttribute(k_dp, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->dp_smem));
+    // the limit is a property of the function, shared by all contexts: raise it to the largest plan, not to this one's
+    CUDA_TRY(cudaFuncSetAttribute(k_dp, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDpSmemMax));
     CUDA_TRY(cudaFuncSetAttribute(k_sample, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->sample_smem));
     CUDA_TRY(cudaFuncSetAttribute(k_pass_a<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->pass_a_smem));
     CUDA_TRY(cudaFuncSetAttribute(k_pass_a<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->pass_a_smem));
@@ -572,7 +575,8 @@ int kimad_step_builtin_scratch(kimad_ctx* c, const float* grads_dev, float* stat
         CUDA_TRY(cudaMemcpyAsync(ws + y.tiny_layers, c->tiny_layers.data(), c->tiny_layers.size() * 4, cudaMemcpyHostToDevice, s));
     CUDA_TRY(cudaMemcpyAsync(ws + y.reg_index, c->reg_index.data(), c->reg_index.size() * 4, cudaMemcpyHostToDevice, s));
     CUDA_TRY(cudaMemsetAsync(ws + y.zero_from, 0, y.lut_t1 - y.zero_from, s));
-    CUDA_TRY(cudaFuncSetAttribute(k_dp, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->dp_smem));
+    // the limit is a property of the function, shared by all contexts: raise it to the largest plan, not to this one's
+    CUDA_TRY(cudaFuncSetAttribute(k_dp, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDpSmemMax));
     CUDA_TRY(cudaFuncSetAttribute(k_sample, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->sample_smem));
     CUDA_TRY(cudaFuncSetAttribute(k_pass_a<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->pass_a_smem));
     CUDA_TRY(cudaFuncSetAttribute(k_pass_a<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->pass_a_smem));

@@ -315,7 +315,8 @@ struct DpPlan {
 };
 
 // mode 0: DP (Kimad+); mode 1: candidates given (j_in); mode 2: one candidate index for all layers, the
-// largest whose total size fits the budget (Kimad without layer adaptivity, Section 3.1)
+// largest whose total size fits the budget (Kimad without layer adaptivity, Section 3.1); mode 3: Algorithm 3
+// read with the discretised error as the axis and the size as the value (needs plan.tab_in_smem)
 __global__ void __launch_bounds__(kDpThreads)
 k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uint32_t D, uint32_t bpe,
      uint64_t full_bytes, uint64_t cap, uint32_t check_finite, int mode, DpPlan plan,
@@ -372,6 +373,88 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
             const uint32_t fit = s_fit;
             if (fit == 0) status = KIMAD_STATUS_INFEASIBLE;
             for (uint32_t l = threadIdx.x; l < L; l += blockDim.x) s_j[l] = fit ? fit - 1 : 0;
+        } else if (mode == 3) {
+            // Error axis: E_max = sum_l err_{l,0} (binary64, layers in order), cells e_{l,j} = floor(err D / E_max),
+            // value = fewest kept entries for a total of exactly e cells; answer = lowest e whose value fits c.
+            __shared__ double s_emax;
+            __shared__ uint32_t s_best;
+            uint32_t* prow = reinterpret_cast<uint32_t*>(rows);
+            uint32_t* pv = prow + pad;
+            uint32_t* cu = prow + rowp + pad;
+            uint32_t* s_kk = reinterpret_cast<uint32_t*>(s_err);
+            const uint32_t kNone = 0xffffffffu;
+            if (threadIdx.x == 0) {
+                double e = 0.0;
+                for (uint32_t l = 0; l < L; ++l) e = __dadd_rn(e, (double)e_w[(size_t)l * K]);
+                s_emax = e;
+                s_best = kNone;
+            }
+            __syncthreads();
+            const double emax = s_emax;
+            for (uint32_t i = threadIdx.x; i < L * Kp; i += blockDim.x) {
+                const uint32_t l = i / Kp, j = i % Kp;
+                uint32_t u = D + 1, kk = 0; // padding reads the margin
+                if (j < K) {
+                    const double q = emax > 0.0 ? floor(__ddiv_rn(__dmul_rn((double)e_w[(size_t)l * K + j], (double)D), emax)) : 0.0;
+                    u = q > (double)D ? D : (uint32_t)q;
+                    kk = (uint32_t)ktab[(size_t)l * K + j];
+                }
+                s_units[i] = u;
+                s_kk[i] = kk;
+            }
+            for (uint32_t i = threadIdx.x; i < 2 * rowp; i += blockDim.x) prow[i] = kNone;
+            __syncthreads();
+            if (threadIdx.x == 0) pv[0] = 0;
+            for (uint32_t l = 0; l < L; ++l) {
+                __syncthreads();
+                const uint32_t* un = s_units + l * Kp;
+                const uint32_t* kk = s_kk + l * Kp;
+                uint8_t* pdl = pd + (size_t)l * plan.pd_row_bytes;
+                for (uint32_t bb = 0; bb < row; bb += kDpCells * blockDim.x) {
+#pragma unroll
+                    for (int q = 0; q < kDpCells; ++q) {
+                        const uint32_t b = bb + threadIdx.x + q * blockDim.x;
+                        const uint32_t bc = min(b, row - 1);
+                        uint32_t best = kNone, bj = 0;
+                        for (uint32_t j = 0; j < K; ++j) {
+                            const uint32_t p = pv[(int)bc - (int)un[j]];
+                            const uint32_t t = p > kNone - kk[j] ? kNone : p + kk[j];
+                            if (t < best) { best = t; bj = j; }
+                        }
+                        if (b < row) cu[b] = best;
+                        if (plan.pd_nibble) {
+                            const uint32_t nb = __shfl_down_sync(0xffffffffu, bj, 1);
+                            if (!(threadIdx.x & 1) && b < row) pdl[b >> 1] = (uint8_t)(bj | (nb << 4));
+                        } else if (b < row) {
+                            pdl[b] = (uint8_t)bj;
+                        }
+                    }
+                }
+                uint32_t* sw = pv; pv = cu; cu = sw;
+            }
+            __syncthreads();
+            const uint64_t cap_k = c / bpe;
+            for (uint32_t b = threadIdx.x; b < row; b += blockDim.x)
+                if (pv[b] != kNone && (uint64_t)pv[b] <= cap_k) atomicMin(&s_best, b);
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                if (s_best == kNone) {
+                    s_status = KIMAD_STATUS_INFEASIBLE;
+                } else {
+                    s_status = KIMAD_OK;
+                    uint32_t b = s_best;
+                    for (uint32_t l = L; l-- > 0;) {
+                        const uint8_t* pdl = pd + (size_t)l * plan.pd_row_bytes;
+                        const uint32_t j = plan.pd_nibble ? ((pdl[b >> 1] >> (4 * (b & 1))) & 15u) : pdl[b];
+                        s_j[l] = j;
+                        b -= s_units[l * Kp + j];
+                    }
+                }
+            }
+            __syncthreads();
+            status = s_status;
+            if (status == KIMAD_STATUS_INFEASIBLE)
+                for (uint32_t l = threadIdx.x; l < L; l += blockDim.x) s_j[l] = 0;
         } else {
             // candidate (l, j) -> smem slot; units above D become D+1 (reads the +inf margin), padding likewise
             auto load_tab = [&](uint32_t l, uint32_t j, uint32_t slot_l) {

@@ -68,6 +68,20 @@ def _llama_1b_layers(d=2048, ffn=5632, vocab=32000, blocks=22, kv=256):
 GRID_7 = [0.01, 0.02, 0.05, 0.10, 0.20, 0.50, 1.00]
 
 
+def block_layers(layer_sizes, block_elems: int):
+    """Block granularity (the paper's Section 5 names it as the next step after per-layer compression): every
+    tensor is cut into consecutive blocks of ``block_elems`` elements (the last one shorter) and each block is
+    handed to the compression pass as a segment of its own.  Returns the list of segment sizes; the flat
+    gradient vector is unchanged."""
+    out = []
+    for n in layer_sizes:
+        n = int(n)
+        out.extend([block_elems] * (n // block_elems))
+        if n % block_elems:
+            out.append(n % block_elems)
+    return out
+
+
 def _log_grid(lo_exp, n=16):
     g = [10.0 ** (lo_exp + (-lo_exp) * j / (n - 1)) for j in range(n)]
     g[-1] = 1.0

@@ -170,3 +170,45 @@ def test_bidirectional_ef21_loop_on_a_quadratic_matches_oracle_and_converges():
         torch.cuda.synchronize()
         assert torch.equal(xh_srv, xh_wrk) and torch.equal(uh_srv, uh_wrk)
         assert np.array_equal(x_d.cpu().numpy().view(np.uint32), xs_ref[k].view(np.uint32)), f"round {k}"
+
+
+def test_block_granularity_is_a_finer_layer_list():
+    """Blocks instead of whole tensors as the unit of allocation: same pass, finer segment list.  At a budget
+    where the cells' rounding-up costs little, the finer allocation reaches a lower error."""
+    wl = workloads.workload(2, 8)
+    blocks = workloads.block_layers(wl.layer_sizes, 16384)
+    assert sum(blocks) == wl.N and len(blocks) > len(wl.layer_sizes) and max(blocks) == 16384
+    fine = Runner(blocks, 1, wl.ratio_grid, 1000, 0)
+    coarse = Runner(wl.layer_sizes, 1, wl.ratio_grid, 1000, 0)
+    grads = workloads.gradients(wl, 0, device="cuda")[:1].contiguous()
+    budget = [0.2 * 8 * wl.N]
+    res_f = fine.compare_step(grads, torch.zeros_like(grads), budget, 1.0)
+    res_c = coarse.compare_step(grads, torch.zeros_like(grads), budget, 1.0)
+    assert res_f["same_k"] and res_c["same_k"]
+    assert float(res_f["ref"].total_err[0]) < float(res_c["ref"].total_err[0])
+
+
+@pytest.mark.parametrize("cfg,divisor", [(2, 8), (3, 16)])
+def test_error_axis_dp_matches_oracle(cfg, divisor):
+    """Algorithm 3 with the error as the knapsack axis (policy 2): decisions bit-identical to the oracle's, on its
+    own curves and on injected ones."""
+    wl = workloads.workload(cfg, divisor)
+    r = Runner(wl.layer_sizes, wl.n_workers, wl.ratio_grid, wl.D, wl.value_dtype, policy=2)
+    bw = workloads.bandwidth_trace(wl, 60)
+    state = torch.zeros((wl.n_workers, wl.N), dtype=torch.float32, device="cuda")
+    ks = set()
+    for s, b in enumerate((5, 25, 50)):
+        grads = workloads.gradients(wl, s, device="cuda")
+        res = r.compare_step(grads, state, bw[b], wl.t_target)
+        assert np.all(res["forced"].used_bytes <= res["forced"].budget_bytes)
+        ks.add(tuple(res["forced"].k[0]))
+    assert len(ks) > 1
+
+
+def test_error_axis_dp_worked_example_and_statuses():
+    sizes, grid = [10, 4, 6], [0.25, 0.5, 1.0]
+    r = Runner(sizes, 4, grid, 12, 0, policy=2)
+    d = torch.tensor([list(range(1, 11)) + [-8, .5, 8, -.5] + [3, -3, 3, 0, -0., 1]] * 4, dtype=torch.float32, device="cuda")
+    res = r.compare_step(d, torch.zeros_like(d), [96.0, 112.0, 47.0, 160.0], 1.0)
+    assert res["forced"].k.tolist() == [[5, 2, 2], [10, 2, 2], [3, 1, 2], [10, 4, 6]]
+    assert list(res["forced"].status) == [0, 0, ko.STATUS_INFEASIBLE, ko.STATUS_PLATEAU]

@@ -145,3 +145,60 @@ def test_aggregate_matches_float32_recomputation_and_closed_form():
     res = ko.step([x.size for x in layers], 1, grid, 12, 0, d, np.zeros_like(d), [96.0], 1.0)
     recv = ko.apply_packed([x.size for x in layers], res.idx[0], res.val[0], res.offs[0], 0, np.zeros(20, np.float32))
     assert np.array_equal(recv, est1)
+
+
+def test_error_axis_dp_hand_example():
+    layers, grid, _ = _golden_uniform()
+    cases = []
+    for line in open(GOLDEN):
+        if line.startswith("erroraxis"):
+            f = [s.split() for s in line[len("erroraxis"):].split(":")]
+            cases.append((int(f[0][0]), int(f[0][1]), [int(x) for x in f[1]], int(f[2][0]), int(f[3][0])))
+    assert len(cases) == 4
+    sizes = [x.size for x in layers]
+    kt = ko.k_table(sizes, grid)
+    d = np.concatenate(layers)[None]
+    for c, D, k, cell, status in cases:
+        res = ko.step(sizes, 1, grid, D, 0, d, np.zeros_like(d), [float(c)], 1.0, policy=2)
+        assert res.status[0] == status and list(res.k[0]) == k
+        st, j, got_cell = ko.dp_error_axis(res.err[0], kt, D, 0, c)
+        assert st == status and (status != ko.STATUS_OK or got_cell == cell)
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_error_axis_dp_brute_force(seed):
+    """Every assignment enumerated: the DP returns the lowest discretised error level that fits the budget and,
+    at that level, the fewest kept entries."""
+    import itertools
+    rng = np.random.default_rng(100 + seed)
+    for trial in range(40):
+        L, K = int(rng.integers(1, 6)), int(rng.integers(1, 5))
+        D = int(rng.integers(max(L, 2), 40))
+        sizes = rng.integers(1, 60, L)
+        grid = np.sort(rng.uniform(0.05, 1, K))
+        kt = ko.k_table(sizes, grid)
+        err = np.sort(rng.uniform(0, 10, (L, K)).astype(np.float32), axis=1)[:, ::-1].copy()
+        vd = trial % 2
+        bpe = 6 if vd else 8
+        c = int(rng.integers(0, int(kt[:, -1].sum()) * bpe + 20))
+        st, j, cell = ko.dp_error_axis(err, kt, D, vd, c)
+        emax = 0.0
+        for l in range(L):
+            emax = emax + float(err[l, 0])
+        cells = [[int(np.floor(float(err[l, q]) * float(D) / emax)) if emax > 0 else 0 for q in range(K)] for l in range(L)]
+        if c >= int(kt[:, -1].sum()) * bpe:
+            assert st == ko.STATUS_PLATEAU and all(j == K - 1)
+            continue
+        best = None
+        for a in itertools.product(range(K), repeat=L):
+            e = sum(cells[l][a[l]] for l in range(L))
+            b = sum(int(kt[l, a[l]]) for l in range(L)) * bpe
+            assert e <= D  # rounding down keeps every assignment on the axis
+            if b <= c and (best is None or (e, b) < best):
+                best = (e, b)
+        if best is None:
+            assert st == ko.STATUS_INFEASIBLE and all(j == 0)
+        else:
+            assert st == ko.STATUS_OK and cell == best[0]
+            assert sum(int(kt[l, j[l]]) for l in range(L)) * bpe == best[1]
+            assert sum(cells[l][j[l]] for l in range(L)) == best[0]
