@@ -51,6 +51,10 @@ struct kimad_ctx {
     bool have_last = false;
     bool timing = false;
     cudaEvent_t ev[KIMAD_N_STAGES + 1] = {};
+    // the tiny layers' exact curves depend on the step's inputs only: they run on a stream of their own, forked
+    // from and joined to the caller's stream with events
+    cudaStream_t side = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     bool have_ev = false;
     template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
 };
@@ -110,6 +114,14 @@ void plan_layout(kimad_ctx* c) {
     } while (0)
 
 constexpr size_t kDpSmemMax = 225 * 1024; // dynamic shared memory the DP kernel may ask for
+
+static int ensure_side_stream(kimad_ctx* c) {
+    if (c->side) return KIMAD_OK;
+    CUDA_TRY(cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking));
+    CUDA_TRY(cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming));
+    CUDA_TRY(cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming));
+    return KIMAD_OK;
+}
 
 enum StepMode { kNormal = 0, kInjectErr = 1, kGivenJ = 2 };
 
@@ -175,10 +187,19 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
     int stage = 0;
     auto mark = [&]() { if (c->timing) cudaEventRecord(c->ev[stage++], s); };
     mark();
+    if (T) CUDA_TRY(cudaEventRecord(c->ev_fork, s)); // fork point of the tiny layers' kernel: the step's start
     // (a) + (b): sample -> bands -> one sweep -> curves
     if (R) {
         k_sample<<<dim3(R, W), kBigThreads, c->sample_smem, s>>>(grads, state, c->stride, layers, reg_layers, R, ktab, K,
                                                                  c->curve_mode == 1 ? 1u : 0u, lut1, lut2, binlo, meta);
+        c->launches += 1;
+    }
+    if (T) { // tiny layers: sorted in shared memory on the side stream; issued after the sample kernel so that
+             // its CTAs fill the SMs the sample kernel leaves idle instead of delaying it
+        CUDA_TRY(cudaStreamWaitEvent(c->side, c->ev_fork, 0));
+        k_tiny_exact<<<dim3(T, W), blk, c->tiny_smem, c->side>>>(grads, state, c->stride, layers, tiny_layers, L, ktab, K, err,
+                                                                 tau, keq, shf, flags);
+        CUDA_TRY(cudaEventRecord(c->ev_join, c->side));
         c->launches += 1;
     }
     mark();
@@ -195,11 +216,7 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
                                                        keq, shf, flags, fb, fb_chunks, fb_layers);
         c->launches += 1;
     }
-    if (T) {
-        k_tiny_exact<<<dim3(T, W), blk, c->tiny_smem, s>>>(dbuf, c->dstride, layers, tiny_layers, L, ktab, K, err, tau, keq,
-                                                           shf, flags);
-        c->launches += 1;
-    }
+    if (T) CUDA_TRY(cudaStreamWaitEvent(s, c->ev_join, 0));
     mark();
     // exact radix select for the layers handed over by k_resolve_a (the lists are usually empty)
     if (R) {
@@ -356,6 +373,12 @@ int kimad_create(kimad_ctx** out, const uint64_t* layer_sizes, uint32_t n_layers
 void kimad_destroy(kimad_ctx* ctx) {
     if (ctx && ctx->have_ev)
         for (cudaEvent_t e : ctx->ev) cudaEventDestroy(e);
+    if (ctx && ctx->side) {
+        cudaStreamSynchronize(ctx->side);
+        cudaEventDestroy(ctx->ev_fork);
+        cudaEventDestroy(ctx->ev_join);
+        cudaStreamDestroy(ctx->side);
+    }
     delete ctx;
 }
 
@@ -399,6 +422,7 @@ int kimad_set_workspace(kimad_ctx* c, void* dev_ptr, size_t bytes) {
     CUDA_TRY(cudaFuncSetAttribute(k_pass_a<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->pass_a_smem));
     CUDA_TRY(cudaFuncSetAttribute(k_pass_a<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->pass_a_smem));
     CUDA_TRY(cudaFuncSetAttribute(k_tiny_exact, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->tiny_smem));
+    { const int rc_side = ensure_side_stream(c); if (rc_side != KIMAD_OK) return rc_side; }
     CUDA_TRY(cudaDeviceSynchronize());
     return KIMAD_OK;
 }
@@ -581,6 +605,7 @@ int kimad_step_builtin_scratch(kimad_ctx* c, const float* grads_dev, float* stat
     CUDA_TRY(cudaFuncSetAttribute(k_pass_a<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->pass_a_smem));
     CUDA_TRY(cudaFuncSetAttribute(k_pass_a<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->pass_a_smem));
     CUDA_TRY(cudaFuncSetAttribute(k_tiny_exact, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->tiny_smem));
+    { const int rc_side = ensure_side_stream(c); if (rc_side != KIMAD_OK) return rc_side; }
     unsigned char* caller_ws = c->ws; // the context's own workspace (if any) is left untouched
     c->ws = ws;
     const int rc = run_step(c, grads_dev, state_dev, bandwidth_bytes_per_s, t_target_s, out, cuda_stream, kNormal, nullptr,

@@ -623,7 +623,8 @@ k_resolve_a(const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ r
 // k_tiny_exact: layers of at most kTinyMax elements, sorted in shared memory (one CTA each)
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kThreads)
-k_tiny_exact(const float* __restrict__ dbuf, uint64_t dstride, const LayerDesc* __restrict__ layers,
+k_tiny_exact(const float* __restrict__ grads, const float* __restrict__ state, uint64_t stride,
+             const LayerDesc* __restrict__ layers,
              const uint32_t* __restrict__ tiny_layers, uint32_t L, const uint64_t* __restrict__ ktab, uint32_t K,
              float* __restrict__ err_out, uint32_t* __restrict__ tau_out, uint32_t* __restrict__ rank_out,
              uint32_t* __restrict__ shift_out, uint32_t* __restrict__ flags) {
@@ -634,12 +635,15 @@ k_tiny_exact(const float* __restrict__ dbuf, uint64_t dstride, const LayerDesc* 
     const uint32_t l = tiny_layers[blockIdx.x], w = blockIdx.y;
     const LayerDesc ld = layers[l];
     const uint32_t n = (uint32_t)ld.n;
-    const float* dd = dbuf + (size_t)w * dstride + ld.begin;
+    // d is recomputed here (the same single subtraction as in the sweep), so that this kernel depends on the
+    // step's inputs only and can run beside the sample and sweep kernels
+    const float* gr = grads + (size_t)w * stride + ld.begin;
+    const float* st = state + (size_t)w * stride + ld.begin;
     uint32_t np = 1;
     while (np < n) np <<= 1;
     bool nonfinite = false;
     for (uint32_t i = threadIdx.x; i < np; i += kThreads) {
-        const uint32_t key = i < n ? key_of(dd[i]) : 0u;
+        const uint32_t key = i < n ? key_of(__fsub_rn(gr[i], st[i])) : 0u;
         nonfinite |= key >= 0x7f800000u;
         s_key[i] = key;
     }
