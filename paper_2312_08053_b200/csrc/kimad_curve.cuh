@@ -82,7 +82,7 @@ k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint6
     // ---- stratified sample of |grad - g|
     const float* gr = grads + (size_t)w * stride + ld.begin;
     const float* st = state + (size_t)w * stride + ld.begin;
-    const uint32_t n_units = (n + 15) / 16;
+    const uint32_t n_units = n / 16 + ((n & 15u) != 0); // n may be as large as 2^32 - 1
     const uint32_t m_units = min(n_units, (uint32_t)kSampleUnits);
     const bool whole = m_units == n_units;
     const uint32_t sq_ = n / (uint32_t)kSampleUnits, sr_ = n % (uint32_t)kSampleUnits; // used when sampled: m_units = kSampleUnits
