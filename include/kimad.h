@@ -128,7 +128,9 @@ int kimad_set_workspace(kimad_ctx* ctx, void* dev_ptr, size_t bytes);
  *   t_target_s one-direction communication time; budget c_w = floor(B_w * t) bytes.  A caller
  *              following Eq. 2 passes (t - T_comp) / 2; a fixed byte budget is (B = bytes, t = 1)
  *   out        host struct of device pointers (see kimad_packed)
- * Returns 0 or a CUDA/argument error; per-worker outcomes land in out->stats[w].status. */
+ * Returns 0 or a CUDA/argument error; per-worker outcomes land in out->stats[w].status.
+ * The step's launches, including those on the context's own side stream, are ordered through events on
+ * cuda_stream, so a step can be captured into a CUDA graph; the budgets are then baked into the graph. */
 int kimad_step(kimad_ctx* ctx, const float* grads_dev, float* state_dev, const double* bandwidth_bytes_per_s,
                double t_target_s, const kimad_packed* out, void* cuda_stream);
 

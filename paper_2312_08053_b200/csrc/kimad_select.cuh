@@ -427,7 +427,7 @@ k_sel_write(const float* __restrict__ dbuf, float* __restrict__ state, const Chu
     const ChunkSel& cs = csel[(size_t)w * n_chunks + blockIdx.x];
     const bool all = jb.mode == 2;
     const uint2 cnt = make_uint2(jb.cnt_gt, jb.cnt_eq), pre = make_uint2(jb.gt_before, jb.eq_before);
-    struct { uint32_t keep_eq; } s = {jb.keep_eq};
+    const uint32_t keep_eq = jb.keep_eq;
     const uint32_t tau = jb.tau;
     const ChunkView cv(ch);
     const float* dd = dbuf + (size_t)w * dstride + cv.a0;
@@ -448,10 +448,10 @@ k_sel_write(const float* __restrict__ dbuf, float* __restrict__ state, const Chu
         const uint32_t gt_here = (sl + 1 < (uint32_t)kSlices ? cs.above[sl + 1] : cnt.x) - cs.above[sl];
         const uint32_t eq_here = (sl + 1 < (uint32_t)kSlices ? cs.eq[sl + 1] : cnt.y) - cs.eq[sl];
         // eq_mode 0: none of this slice's equals is kept; 1: all are; 2: ranks must be counted
-        const int eq_mode = (all || eq_here == 0 || eq_before >= s.keep_eq) ? 0 : (eq_before + eq_here <= s.keep_eq ? 1 : 2);
+        const int eq_mode = (all || eq_here == 0 || eq_before >= keep_eq) ? 0 : (eq_before + eq_here <= keep_eq ? 1 : 2);
         if (!all && gt_here == 0 && eq_mode == 0) continue; // nothing kept in this slice
         uint32_t eq_seen = eq_before;
-        uint32_t pos = gt_before + min(eq_before, s.keep_eq); // position of the slice's first kept entry in the layer
+        uint32_t pos = gt_before + min(eq_before, keep_eq); // position of the slice's first kept entry in the layer
         const uint64_t gm = cs.mask[sl];
         const uint32_t n_groups = __popcll(gm);
         if (!all && n_groups <= (uint32_t)kSparseGroups) {
@@ -507,7 +507,7 @@ k_sel_write(const float* __restrict__ dbuf, float* __restrict__ state, const Chu
                     }
                     uint32_t eq_rank = eq_seen + incl - __popc(eqm);
                     for (uint32_t m = eqm; m; m &= m - 1) {
-                        if (eq_rank < s.keep_eq) keepm |= m & (0u - m);
+                        if (eq_rank < keep_eq) keepm |= m & (0u - m);
                         ++eq_rank;
                     }
                     eq_seen += __shfl_sync(0xffffffffu, incl, 31);
@@ -576,7 +576,7 @@ k_sel_write(const float* __restrict__ dbuf, float* __restrict__ state, const Chu
                 }
                 uint32_t eq_rank = eq_seen + incl - __popc(eqm);
                 for (uint32_t m = eqm; m; m &= m - 1) {
-                    if (eq_rank < s.keep_eq) keepm |= m & (0u - m);
+                    if (eq_rank < keep_eq) keepm |= m & (0u - m);
                     ++eq_rank;
                 }
                 eq_seen += __shfl_sync(0xffffffffu, incl, 31);

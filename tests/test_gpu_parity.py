@@ -215,3 +215,34 @@ def test_run_to_run_determinism_of_decisions():
         outs.append((u32(r.out.k).copy(), u32(r.out.idx).copy(), u32(state).copy()))
     for o in outs[1:]:
         assert all(np.array_equal(a, b) for a, b in zip(outs[0], o))
+
+
+def test_step_is_capturable_in_a_cuda_graph():
+    """All work of a step, the forked side stream included, is ordered through the caller's stream: the step can
+    be captured once and replayed on new gradients (the budgets are baked into the captured launches)."""
+    wl = workloads.workload(1)
+    W, N = wl.n_workers, wl.N
+    bw = workloads.bandwidth_trace(wl)[0]
+    ctx = kb.new_context(wl.layer_sizes, W, wl.ratio_grid, D=wl.D, value_dtype=wl.value_dtype)
+    out = kb.Packed(ctx)
+    grads = workloads.gradients(wl, 0, device="cuda")
+    state = torch.zeros((W, N), device="cuda")
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        kb.kimad_step(ctx, grads, state, bw, wl.t_target, out, s)  # warm-up outside the capture
+    s.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=s):
+        kb.kimad_step(ctx, grads, state, bw, wl.t_target, out, torch.cuda.current_stream())
+    state.zero_()
+    ref_state = np.zeros((W, N), np.float32)
+    for step in range(3):
+        fresh = workloads.gradients(wl, 10 + step, device="cuda")
+        grads.copy_(fresh)
+        graph.replay()
+        torch.cuda.synchronize()
+        ref = ko.step(wl.layer_sizes, W, wl.ratio_grid, wl.D, wl.value_dtype, fresh.cpu().numpy(), ref_state, bw,
+                      wl.t_target)
+        ref_state = ref.state
+        assert np.array_equal(u32(out.k), ref.k)
+        assert np.array_equal(u32(state), ref_state.view(np.uint32))
