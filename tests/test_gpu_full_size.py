@@ -120,3 +120,70 @@ def test_llama_1b_shape_full_size_bf16():
     # 2 workers x 1.1 G elements, bf16 values; layers: 65.5 M embedding, q/k proj, one FFN matrix, a norm, lm_head slot
     why = _full_size_step(5, step_of_trace=30, sample_layers={0, 2, 3, 7, 10}, workers_checked=[1])
     assert why[0] <= 60, why
+
+
+@pytest.mark.parametrize("n", [(1 << 28) + 3, (1 << 31) + 5, (1 << 32) - 1])
+def test_one_very_large_layer(n):
+    """A single layer far larger than any in the workloads (8193 chunks and more, a ragged last one; the larger
+    sizes cross 2^31 layer-local indices and reach the largest layer the interface takes): the curve of every candidate against a full sort done by torch on the
+    device, and the selection properties on all entries.  The state starts at zero so that d = grad."""
+    grid = [0.0001, 0.003, 0.05, 0.4, 1.0]
+    ctx = kb.new_context([n], 1, grid, D=1000, value_dtype=0, max_packed_elems=n // 64)
+    out = kb.Packed(ctx)
+    gen = torch.Generator(device="cuda").manual_seed(28)
+    grads = torch.randn((1, n), device="cuda", generator=gen)
+    grads.mul_(torch.randn((1, n), device="cuda", generator=gen).abs_())  # heavier tails than a normal
+    state = torch.zeros((1, n), device="cuda")
+    d = grads[0]
+    kb.kimad_step(ctx, grads, state, [0.02 * 8 * n], 1.0, out)
+    status, k_gpu = kb.kimad_get_k(ctx)
+    assert status == 0
+    kt = ko.k_table([n], grid)[0]
+    err_g, tau_g, keq_g, shift_g = kb.kimad_debug_get_curve(ctx)
+    # curve: squares of the n - k smallest magnitudes, summed in float64.  torch sorts at most 2^31 - 1 elements,
+    # so the magnitudes are sorted in three parts; the k-th largest of the union is found by bisection over the
+    # 31-bit keys with searchsorted on the parts, and the dropped squares come from the parts' prefix sums.
+    third = n // 3
+    parts = []
+    for a, b in ((0, third), (third, 2 * third), (2 * third, n)):
+        srt, _ = torch.sort(d[a:b].abs())
+        parts.append((srt.view(torch.int32), torch.cumsum(srt.double().square_(), 0)))
+        del srt
+
+    def count_below(key, right):  # entries with magnitude key < `key` (right=False) or <= `key` (right=True)
+        probe = torch.tensor([key], dtype=torch.int32, device="cuda")
+        return [int(torch.searchsorted(p[0], probe, right=right)) for p in parts]
+
+    for j, k in enumerate(kt):
+        drop = n - int(k)
+        want = 0.0
+        if drop:
+            lo, hi = 0, 0x7F800000  # smallest key with at least `drop` entries <= key: the largest dropped magnitude
+            while lo < hi:
+                mid = (lo + hi) // 2
+                if sum(count_below(mid, True)) >= drop:
+                    hi = mid
+                else:
+                    lo = mid + 1
+            below = count_below(lo, False)
+            for p, c in zip(parts, below):
+                want += float(p[1][c - 1]) if c else 0.0
+            v = float(torch.tensor([lo], dtype=torch.int32).view(torch.float32))
+            want += (drop - sum(below)) * v * v  # dropped entries equal to that magnitude
+        assert abs(float(err_g[0, 0, j]) - want) <= 1e-5 * want, (j, err_g[0, 0, j], want)
+    del parts
+    j = int(out.j[0, 0])
+    assert j == 1 and int(k_gpu[0, 0]) == int(kt[1])  # 0.3 % fits 2 % of the dense bytes, 5 % does not
+    k = int(kt[j])
+    idx = out.idx[0, :k].long() & 0xFFFFFFFF  # u32 indices stored in an int32 tensor
+    val = out.val[0, :k]
+    assert bool(torch.all(idx[1:] > idx[:-1])) and int(idx[-1]) < n
+    assert torch.equal(val.view(torch.int32), d[idx].view(torch.int32))
+    kept = torch.zeros(n, dtype=torch.bool, device="cuda")
+    kept[idx] = True
+    key = d.view(torch.int32) & 0x7FFFFFFF
+    assert int(key[kept].min()) >= int(key[~kept].max())
+    del key
+    assert int(torch.count_nonzero(state[0])) == int(torch.count_nonzero(val))  # nothing but the kept entries changed
+    assert torch.equal(state[0][idx].view(torch.int32), val.view(torch.int32))
+    assert kb.kimad_debug_exact_path_layers(ctx) == 0
