@@ -439,6 +439,7 @@ k_sel_write(const float* __restrict__ dbuf, float* __restrict__ state, const Chu
     const uint32_t lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const bool st_vec = (reinterpret_cast<uintptr_t>(st) & 15u) == 0;
     __shared__ uint8_t s_pos[kThreads / 32][kSparseGroups]; // per warp: the marked groups of a slice, ascending
+    __shared__ uint32_t s_stage[DENSE ? kThreads / 32 : 1][DENSE ? 2 * 16 * 32 : 1]; // per warp: a round's indices, values
 
     for (uint32_t sl = wid; sl < (uint32_t)kSlices; sl += kThreads / 32) {
         const uint32_t x0 = sl * kSliceElems;
@@ -604,22 +605,35 @@ k_sel_write(const float* __restrict__ dbuf, float* __restrict__ state, const Chu
 #pragma unroll
                     for (int i = 0; i < E; ++i) sv[i] = (keepm >> i) & 1u ? st[t0 + i] : 0.f;
                 }
+                // the round's entries are laid out in shared memory first, so that the packed buffers are written
+                // with consecutive lanes on consecutive entries
+                uint32_t* sg_idx = s_stage[wid];
+                uint32_t* sg_val = sg_idx + E * 32;
+                uint32_t ol = incl - __popc(keepm); // position inside the round
 #pragma unroll
                 for (int i = 0; i < E; ++i)
                     if ((keepm >> i) & 1u) {
-                        oi[o] = idx0 + t0 + i;
+                        sg_idx[ol] = idx0 + t0 + i;
                         float sent;
                         if (BF16) {
                             const __nv_bfloat16 h = __float2bfloat16_rn(v[i]);
-                            ov16[o] = h;
+                            sg_val[ol] = (uint32_t)__bfloat16_as_ushort(h);
                             sent = __bfloat162float(h);
                         } else {
-                            ov32[o] = v[i];
+                            sg_val[ol] = __float_as_uint(v[i]);
                             sent = v[i];
                         }
                         sv[i] = __fadd_rn(sv[i], sent);
-                        ++o;
+                        ++ol;
                     }
+                __syncwarp();
+                const uint32_t round_pos = pos - round_total;
+                for (uint32_t q = lane; q < round_total; q += 32) {
+                    oi[round_pos + q] = sg_idx[q];
+                    if (BF16) ov16[round_pos + q] = __ushort_as_bfloat16((unsigned short)sg_val[q]);
+                    else ov32[round_pos + q] = __uint_as_float(sg_val[q]);
+                }
+                __syncwarp();
                 if (st_vec) {
                     if (keepm) {
 #pragma unroll
