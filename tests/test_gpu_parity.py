@@ -246,3 +246,19 @@ def test_step_is_capturable_in_a_cuda_graph():
         ref_state = ref.state
         assert np.array_equal(u32(out.k), ref.k)
         assert np.array_equal(u32(state), ref_state.view(np.uint32))
+
+
+@pytest.mark.parametrize("K,D", [(127, 1000), (1, 1000), (16, 8191), (7, 5)])
+def test_interface_limits(K, D):
+    """The largest ratio grid (127), a single ratio, the largest number of budget cells (8191) and the smallest one
+    the layer list allows (D = L)."""
+    rng = np.random.default_rng(K + D)
+    sizes = [70000, 33, 5000, 4097, 1]
+    grid = np.linspace(1.0 / K, 1.0, K) if K > 1 else [0.25]
+    r = Runner(sizes, 2, grid, D, 0)
+    N = sum(sizes)
+    grads = torch.from_numpy((rng.standard_normal((2, N)) * np.repeat([1.0, 30.0, 0.01, 3.0, 1.0], sizes)).astype(np.float32)).cuda()
+    state = torch.zeros_like(grads)
+    for budget in ([0.05 * 8 * N, 0.6 * 8 * N], [0.3 * 8 * N, 8.0 * N]):
+        res = r.compare_step(grads, state, budget, 1.0)
+        assert res["same_k"]
