@@ -262,3 +262,18 @@ def test_interface_limits(K, D):
     for budget in ([0.05 * 8 * N, 0.6 * 8 * N], [0.3 * 8 * N, 8.0 * N]):
         res = r.compare_step(grads, state, budget, 1.0)
         assert res["same_k"]
+
+
+def test_many_workers_with_different_budgets():
+    """40 workers on one GPU (the DP runs in several launches of workers), every worker with its own budget."""
+    sizes = [30000, 128, 9000, 10]
+    grid = [0.01, 0.02, 0.05, 0.1, 0.2, 0.5, 1.0]
+    W, N = 40, sum(sizes)
+    r = Runner(sizes, W, grid, 1000, 1)
+    gen = torch.Generator(device="cuda").manual_seed(40)
+    grads = torch.randn((W, N), device="cuda", generator=gen) * 0.01
+    state = torch.zeros_like(grads)
+    bw = np.linspace(0.0, 1.1, W) * 6 * N  # from nothing (infeasible) to more than everything (plateau)
+    res = r.compare_step(grads, state, bw, 1.0)
+    st = res["forced"].status
+    assert st[0] == ko.STATUS_INFEASIBLE and st[-1] == ko.STATUS_PLATEAU and np.count_nonzero(st == 0) > 30
