@@ -115,6 +115,24 @@ void plan_layout(kimad_ctx* c) {
 
 constexpr size_t kDpSmemMax = 225 * 1024; // dynamic shared memory the DP kernel may ask for
 
+// Kernels are loaded on their first launch; loading one takes about a millisecond.  Touching every kernel a
+// step can launch (the rarely taken ones included) when the workspace is attached keeps that out of the steps.
+static int preload_kernels() {
+    cudaFuncAttributes a;
+#define KIMAD_PRELOAD(f) CUDA_TRY(cudaFuncGetAttributes(&a, f))
+    KIMAD_PRELOAD(k_sample); KIMAD_PRELOAD(k_pass_a<true>); KIMAD_PRELOAD(k_pass_a<false>); KIMAD_PRELOAD(k_resolve_a);
+    KIMAD_PRELOAD(k_tiny_exact); KIMAD_PRELOAD(k_fb_hist1); KIMAD_PRELOAD(k_fb_hist23<2>); KIMAD_PRELOAD(k_fb_hist23<3>);
+    KIMAD_PRELOAD(k_resolve1); KIMAD_PRELOAD(k_resolve23<2>); KIMAD_PRELOAD(k_resolve23<3>); KIMAD_PRELOAD(k_rebuild_slots);
+    KIMAD_PRELOAD(k_dp); KIMAD_PRELOAD(k_sel_count); KIMAD_PRELOAD(k_sel_count_r2); KIMAD_PRELOAD(k_sel_resolve);
+    KIMAD_PRELOAD(k_sel_resolve_r2); KIMAD_PRELOAD(k_sel_recount); KIMAD_PRELOAD(k_sel_slices); KIMAD_PRELOAD(k_sel_scan);
+    KIMAD_PRELOAD((k_sel_write<false, false>)); KIMAD_PRELOAD((k_sel_write<false, true>));
+    KIMAD_PRELOAD((k_sel_write<true, false>)); KIMAD_PRELOAD((k_sel_write<true, true>));
+    KIMAD_PRELOAD(k_apply_packed<false>); KIMAD_PRELOAD(k_apply_packed<true>);
+    KIMAD_PRELOAD(k_aggregate<false>); KIMAD_PRELOAD(k_aggregate<true>);
+#undef KIMAD_PRELOAD
+    return KIMAD_OK;
+}
+
 static int ensure_side_stream(kimad_ctx* c) {
     if (c->side) return KIMAD_OK;
     CUDA_TRY(cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking));
@@ -423,6 +441,7 @@ int kimad_set_workspace(kimad_ctx* c, void* dev_ptr, size_t bytes) {
     CUDA_TRY(cudaFuncSetAttribute(k_pass_a<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->pass_a_smem));
     CUDA_TRY(cudaFuncSetAttribute(k_tiny_exact, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->tiny_smem));
     { const int rc_side = ensure_side_stream(c); if (rc_side != KIMAD_OK) return rc_side; }
+    { const int rc_pre = preload_kernels(); if (rc_pre != KIMAD_OK) return rc_pre; }
     CUDA_TRY(cudaDeviceSynchronize());
     return KIMAD_OK;
 }
@@ -606,6 +625,7 @@ int kimad_step_builtin_scratch(kimad_ctx* c, const float* grads_dev, float* stat
     CUDA_TRY(cudaFuncSetAttribute(k_pass_a<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->pass_a_smem));
     CUDA_TRY(cudaFuncSetAttribute(k_tiny_exact, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->tiny_smem));
     { const int rc_side = ensure_side_stream(c); if (rc_side != KIMAD_OK) return rc_side; }
+    { const int rc_pre = preload_kernels(); if (rc_pre != KIMAD_OK) return rc_pre; }
     unsigned char* caller_ws = c->ws; // the context's own workspace (if any) is left untouched
     c->ws = ws;
     const int rc = run_step(c, grads_dev, state_dev, bandwidth_bytes_per_s, t_target_s, out, cuda_stream, kNormal, nullptr,
