@@ -23,7 +23,7 @@ struct Layout {
     // zeroed at set_workspace and kept clean by the kernels
     size_t zero_from, h1_cnt, h1_ss, h23_cnt, h23_ss, bh_cnt, bh_sum, low_hist, recount, fb, r2, flags;
     // scratch without initial-state requirements
-    size_t lut_t1, lut_t2, bin_lo, meta, cands, slots, err, tau, keep_eq, shift, sel, chunk_cnt, chunk_pre, csel,
+    size_t lut_t1, lut_t2, bin_lo, meta, cands, slots, err, tau, keep_eq, shift, sel, chunk_cnt, jobs, csel,
         fb_chunks, fb_layers, r2_chunks, r2_layers, pd, total;
 };
 
@@ -98,7 +98,7 @@ void plan_layout(kimad_ctx* c) {
     y.shift = take(WLK * sizeof(uint32_t));
     y.sel = take(WL * sizeof(Sel));
     y.chunk_cnt = take((size_t)c->W * nch * sizeof(uint2));
-    y.chunk_pre = take((size_t)c->W * nch * sizeof(ChunkJob));
+    y.jobs = take((size_t)c->W * nch * sizeof(ChunkJob));
     y.csel = take((size_t)c->W * nch * sizeof(ChunkSel));
     y.fb_chunks = take((size_t)c->W * nch * sizeof(uint2));
     y.fb_layers = take(WL * sizeof(uint2));
@@ -183,7 +183,7 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
     uint32_t* shf = c->at<uint32_t>(y.shift);
     Sel* sel = c->at<Sel>(y.sel);
     uint2* ccnt = c->at<uint2>(y.chunk_cnt);
-    ChunkJob* jobs = c->at<ChunkJob>(y.chunk_pre);
+    ChunkJob* jobs = c->at<ChunkJob>(y.jobs);
     ChunkSel* csel = c->at<ChunkSel>(y.csel);
     uint32_t* lowh = c->at<uint32_t>(y.low_hist);
     uint32_t* recount_n = c->at<uint32_t>(y.recount);

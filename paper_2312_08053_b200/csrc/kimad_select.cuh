@@ -2,11 +2,12 @@
 //
 // After the DP every (worker, layer) knows a key interval [lo, lo + 2^shift) that contains its
 // threshold and the rank of the threshold inside that interval (shift = 0 when the curve stage already
-// resolved all 31 bits).  One sweep over the difference vector (k_sel_count) counts, per chunk, the
-// entries above the interval and remembers the few entries inside it; k_sel_resolve turns the
-// per-layer histogram of those entries into the exact threshold; k_sel_scan derives every chunk's
-// output offset; k_sel_write compacts in index order and updates the estimator.  No kernel waits on
-// another: offsets come from stored per-chunk counts.
+// resolved all 31 bits).  One sweep over the difference vector (k_sel_count) counts, per 2048-element slice,
+// the entries above the interval, remembers the few entries inside it and marks the 32-element groups that
+// can hold a kept entry; k_sel_resolve turns the remembered entries (or their per-layer histogram) into the
+// exact threshold; k_sel_slices and k_sel_scan derive every slice's and chunk's output offset and leave one
+// job record per chunk; k_sel_write compacts in index order and updates the estimator, reading only the
+// marked groups of sparse slices.  No kernel waits on another: offsets come from stored counts.
 #pragma once
 #include "kimad_curve.cuh"
 
