@@ -470,8 +470,12 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
             };
             auto count_usable = [&](uint32_t slot_l) { // sizes ascend with j, so the usable candidates come first
                 uint32_t nu = 0;
-                while (nu < K && s_units[slot_l * Kp + nu] <= D) ++nu;
-                s_usable[slot_l] = nu;
+                bool same = true; // all usable candidates take the same number of cells (small layers under a coarse cell)
+                while (nu < K && s_units[slot_l * Kp + nu] <= D) {
+                    same &= s_units[slot_l * Kp + nu] == s_units[slot_l * Kp];
+                    ++nu;
+                }
+                s_usable[slot_l] = nu | (same && nu > 1 ? 0x80000000u : 0u);
             };
             if (plan.tab_in_smem) {
                 for (uint32_t i = threadIdx.x; i < L * Kp; i += blockDim.x) load_tab(i / Kp, i % Kp, i / Kp);
@@ -492,7 +496,8 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
                 const uint32_t sl = plan.tab_in_smem ? l : 0;
                 const uint32_t* un = s_units + sl * Kp;
                 const float* er = s_err + sl * Kp;
-                const uint32_t nu = s_usable[sl];
+                const uint32_t nu = s_usable[sl] & 0xffffu;
+                const bool same_cells = s_usable[sl] >> 31;
                 uint8_t* pdl = pd + (size_t)l * plan.pd_row_bytes;
                 // each thread owns the cells t, t + T, ... (consecutive threads read consecutive words of
                 // prev[]: no bank conflicts); candidates four at a time so that the prev[] reads of a batch are
@@ -503,6 +508,20 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
                     uint32_t bj[kDpCells];
 #pragma unroll
                     for (int q = 0; q < kDpCells; ++q) { best[q] = kInf; bj[q] = 0; }
+                    if (same_cells) { // one read of prev[] serves all candidates; same adds, same order, same ties
+                        const int u0 = (int)un[0];
+                        float p0[kDpCells];
+#pragma unroll
+                        for (int q = 0; q < kDpCells; ++q) p0[q] = prev[(int)min(b0 + q * blockDim.x, row - 1) - u0];
+                        for (uint32_t j = 0; j < nu; ++j) {
+                            const float ej = er[j];
+#pragma unroll
+                            for (int q = 0; q < kDpCells; ++q) {
+                                const float t = __fadd_rn(p0[q], ej);
+                                if (t < best[q]) { best[q] = t; bj[q] = j; }
+                            }
+                        }
+                    } else
                     for (uint32_t j0 = 0; j0 < nu; j0 += 4) {
                         uint32_t u[4];
                         float e[4], p[4][kDpCells];
