@@ -417,7 +417,7 @@ k_sel_scan(const LayerDesc* __restrict__ layers, const Chunk* __restrict__ chunk
 // DENSE: tuned for steps whose budget keeps more than a few per cent of the entries (the host picks the
 // instantiation from the budgets; both are correct for any input).
 template <bool BF16, bool DENSE>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, DENSE ? 3 : 8)
 k_sel_write(const float* __restrict__ dbuf, float* __restrict__ state, const Chunk* __restrict__ chunks,
             uint32_t n_chunks, uint64_t dstride, uint64_t stride, const ChunkSel* __restrict__ csel,
             const ChunkJob* __restrict__ jobs, uint64_t cap, uint32_t* __restrict__ out_idx, void* __restrict__ out_val) {
