@@ -158,7 +158,8 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
     const bool vec = ((uintptr_t)grads % 16 == 0) && ((uintptr_t)state % 16 == 0) && (c->stride % 4 == 0);
 
     const Layout& y = c->lay;
-    float* dbuf = c->at<float>(y.dbuf);
+    // d as two 16-bit planes, each u16 [W][dstride], in the space of one f32 [W][dstride] array
+    const DPlanes dbuf{c->at<uint16_t>(y.dbuf), c->at<uint16_t>(y.dbuf) + (size_t)c->W * c->dstride};
     const Chunk* chunks = c->at<Chunk>(y.chunks);
     const LayerDesc* layers = c->at<LayerDesc>(y.layers);
     const uint64_t* ktab = c->at<uint64_t>(y.ktab);

@@ -374,7 +374,7 @@ constexpr int kMaxRunChunksA = 32; // a run has at most 2^20 elements: its carry
 
 template <bool VEC>
 __global__ void __launch_bounds__(kBigThreads, 1)
-k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, float* __restrict__ dbuf,
+k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, DPlanes dbuf,
          const Chunk* __restrict__ chunks, uint32_t n_chunks, uint32_t run_chunks, uint64_t stride, uint64_t dstride,
          const uint32_t* __restrict__ reg_index /* [L], 0xffffffff: tiny layer */, uint32_t R,
          const uint16_t* __restrict__ lut_t1, const uint32_t* __restrict__ lut_t2, const BandMeta* __restrict__ meta,
@@ -391,7 +391,8 @@ k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, float
     for (int i = threadIdx.x; i < 3 * kMaxBins; i += kBigThreads) sh[i] = 0;
     const float* gr0 = grads + (size_t)w * stride;
     const float* st0 = state + (size_t)w * stride;
-    float* dd0 = dbuf + (size_t)w * dstride;
+    uint16_t* dh0 = dbuf.hi + (size_t)w * dstride;
+    uint16_t* dl0 = dbuf.lo + (size_t)w * dstride;
     int cur_layer = -1;
     bool active = false, dirty = false;
     uint32_t n_bins = 0;
@@ -452,7 +453,8 @@ k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, float
         const ChunkView cv(ch);
         const float* gr = gr0 + cv.a0;
         const float* st = st0 + cv.a0;
-        float* dd = dd0 + cv.a0;
+        uint16_t* dh = dh0 + cv.a0;
+        uint16_t* dl = dl0 + cv.a0;
         const uint32_t nq = cv.quads();
         constexpr int U = 2;
         for (uint32_t qb = 0; qb < nq; qb += kBigThreads * U) {
@@ -473,13 +475,17 @@ k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, float
                     float4 d;
                     d.x = __fsub_rn(a[u].x, b[u].x); d.y = __fsub_rn(a[u].y, b[u].y);
                     d.z = __fsub_rn(a[u].z, b[u].z); d.w = __fsub_rn(a[u].w, b[u].w);
-                    reinterpret_cast<float4*>(dd)[q] = d;
+                    uint2 ph, pl;
+                    split_quad(d, ph, pl);
+                    reinterpret_cast<uint2*>(dh)[q] = ph;
+                    reinterpret_cast<uint2*>(dl)[q] = pl;
                     if (active) { acc(d.x); acc(d.y); acc(d.z); acc(d.w); }
                 } else {
                     for (uint32_t e = 4 * q; e < 4 * q + 4; ++e)
                         if (e >= cv.first && e < cv.len) {
                             const float d = __fsub_rn(gr[e], st[e]);
-                            dd[e] = d;
+                            dh[e] = (uint16_t)(__float_as_uint(d) >> 16);
+                            dl[e] = (uint16_t)__float_as_uint(d);
                             if (active) acc(d);
                         }
                 }
@@ -697,7 +703,7 @@ k_tiny_exact(const float* __restrict__ grads, const float* __restrict__ state, u
 // exact radix path over the handed-over chunks (global atomics: the list is short or empty)
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kThreads)
-k_fb_hist1(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks, uint64_t dstride, uint32_t L,
+k_fb_hist1(DPlanes dbuf, const Chunk* __restrict__ chunks, uint64_t dstride, uint32_t L,
            const FbList* __restrict__ fb, const uint2* __restrict__ fb_chunks, uint32_t* __restrict__ g_cnt,
            unsigned long long* __restrict__ g_ss, uint32_t* __restrict__ flags) {
     __shared__ uint32_t s_cnt[kL1Bins], s_hi[kL1Bins], s_lo[kL1Bins];
@@ -706,11 +712,11 @@ k_fb_hist1(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks, uin
         const uint2 e = fb_chunks[it];
         const Chunk ch = chunks[e.y];
         const ChunkView cv(ch);
-        const float* dd = dbuf + (size_t)e.x * dstride + cv.a0;
+        const DView dd(dbuf, (size_t)e.x * dstride + cv.a0);
         for (int b = threadIdx.x; b < kL1Bins; b += kThreads) { s_cnt[b] = 0; s_hi[b] = 0; s_lo[b] = 0; }
         __syncthreads();
         for (uint32_t x = cv.first + threadIdx.x; x < cv.len; x += kThreads) {
-            const uint32_t key = key_of(dd[x]);
+            const uint32_t key = key_of(dd.at(x));
             const uint32_t sq = (uint32_t)sq_fixed(key);
             atomicAdd(&s_cnt[key >> 20], 1u);
             atomicAdd(&s_hi[key >> 20], sq >> 16);
@@ -731,7 +737,7 @@ k_fb_hist1(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks, uin
 
 template <int LEVEL>
 __global__ void __launch_bounds__(kThreads)
-k_fb_hist23(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks, uint64_t dstride, uint32_t L, uint32_t K,
+k_fb_hist23(DPlanes dbuf, const Chunk* __restrict__ chunks, uint64_t dstride, uint32_t L, uint32_t K,
             const FbList* __restrict__ fb, const uint2* __restrict__ fb_chunks, const SlotTab* __restrict__ slots,
             uint32_t* __restrict__ g_cnt, unsigned long long* __restrict__ g_ss) {
     __shared__ uint8_t s_first[kL1Bins]; // level-1 bin -> first slot whose prefix starts with it (0xff: none)
@@ -755,11 +761,11 @@ k_fb_hist23(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks, ui
             }
         __syncthreads();
         const ChunkView cv(ch);
-        const float* dd = dbuf + (size_t)e.x * dstride + cv.a0;
+        const DView dd(dbuf, (size_t)e.x * dstride + cv.a0);
         uint32_t* gc = g_cnt + wl * K * kL23Bins;
         unsigned long long* gs = g_ss + wl * K * kL23Bins;
         for (uint32_t x = cv.first + threadIdx.x; x < cv.len; x += kThreads) {
-            const uint32_t key = key_of(dd[x]);
+            const uint32_t key = key_of(dd.at(x));
             const uint32_t f = s_first[key >> 20];
             if (f == 0xff) continue;
             if (LEVEL == 2) {

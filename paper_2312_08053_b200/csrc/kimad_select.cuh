@@ -60,7 +60,7 @@ constexpr int kSortCap = 4096;
 
 // ------------------------------------------------------------------------------------------------
 // Counting sweep of one chunk: warp w takes the slices w and w + 8.
-__device__ __forceinline__ void sel_count_chunk(const float* __restrict__ dbuf, const Chunk& ch, uint32_t w,
+__device__ __forceinline__ void sel_count_chunk(const DPlanes& dbuf, const Chunk& ch, uint32_t w,
                                                 uint32_t chunk_id, uint32_t n_chunks, uint64_t dstride, uint32_t L,
                                                 const Sel* __restrict__ sel, const LayerDesc* __restrict__ layers,
                                                 ChunkSel* __restrict__ csel, uint32_t* __restrict__ low_hist,
@@ -85,12 +85,18 @@ __device__ __forceinline__ void sel_count_chunk(const float* __restrict__ dbuf, 
     for (int i = threadIdx.x; i < kLowBins; i += kThreads) s_hist[i] = 0;
     if (threadIdx.x == 0) *s_n = 0;
     __syncthreads();
-    const float* dd = dbuf + (size_t)w * dstride + cv.a0;
+    const DView dd(dbuf, (size_t)w * dstride + cv.a0);
+    // Upper halves first: a key whose upper half lies above that of the interval's last key is above the interval,
+    // one below that of its first key is below; only keys sharing an upper half with the interval (a 2^16-key
+    // stretch of the axis or two) are completed from the lower plane.  The halves are 15-bit numbers after the
+    // sign is masked, so "x >= t" for both halves of a word is bit 15 / 31 of x + (0x8000 - t) * 0x10001.
+    const uint32_t hi_bot = lo >> 16, hi_top = (lo + width - 1) >> 16;
+    const uint32_t add_gt = (0x8000u - (hi_top + 1)) * 0x00010001u, add_ge = (0x8000u - hi_bot) * 0x00010001u;
     for (uint32_t sl = wid; sl < (uint32_t)kSlices; sl += kThreads / 32) {
         uint32_t above = 0;
         uint64_t mask = 0;
-        auto visit = [&](float dv) -> bool { // true: the key is not below the interval
-            const uint32_t d1 = key_of(dv) - lo; // wraps to >= 2^31 for keys below the interval
+        auto visit = [&](uint32_t key) -> bool { // true: the key is not below the interval
+            const uint32_t d1 = key - lo; // wraps to >= 2^31 for keys below the interval
             if (d1 < width) {
                 atomicAdd(&s_hist[d1 >> hshift], 1u);
                 const uint32_t p = atomicAdd(s_n, 1u);
@@ -102,22 +108,34 @@ __device__ __forceinline__ void sel_count_chunk(const float* __restrict__ dbuf, 
         };
         constexpr int H = kSliceElems / 256; // quads per lane and half slice
         for (uint32_t q0 = sl * (kSliceElems / 4); q0 < (sl + 1) * (kSliceElems / 4) && 4 * q0 < cv.len; q0 += H * 32) {
-            float4 a[H];
+            uint2 a[H];
 #pragma unroll
             for (int i = 0; i < H; ++i) {
                 const uint32_t q = q0 + i * 32 + lane;
-                if (cv.quad_full(q)) a[i] = __ldcs(reinterpret_cast<const float4*>(dd) + q);
+                if (cv.quad_full(q)) a[i] = __ldcs(reinterpret_cast<const uint2*>(dd.hi) + q);
             }
-            uint32_t fb = 0; // bit i: this lane's quad of row i holds a key that is not below the interval
+            uint32_t fb = 0; // bit i: this lane's quad of row i may hold a key that is not below the interval
 #pragma unroll
             for (int i = 0; i < H; ++i) {
                 const uint32_t q = q0 + i * 32 + lane;
                 bool f = false;
                 if (cv.quad_full(q)) {
-                    f = visit(a[i].x); f |= visit(a[i].y); f |= visit(a[i].z); f |= visit(a[i].w);
+                    const uint32_t x0_ = a[i].x & 0x7fff7fffu, x1_ = a[i].y & 0x7fff7fffu;
+                    const uint32_t gt0 = (x0_ + add_gt) & 0x80008000u, gt1 = (x1_ + add_gt) & 0x80008000u;
+                    const uint32_t ge0 = (x0_ + add_ge) & 0x80008000u, ge1 = (x1_ + add_ge) & 0x80008000u;
+                    above += __popc(gt0) + __popc(gt1);
+                    f = (ge0 | ge1) != 0;
+                    // rare: keys that share an upper half with the interval; bit 15 -> element 0 / 2, bit 31 -> 1 / 3
+                    uint32_t border = ((ge0 ^ gt0) >> 15 & 0x00010001u) | ((ge1 ^ gt1) >> 13 & 0x00040004u);
+                    while (border) {
+                        const uint32_t bit = __ffs(border) - 1; // 0, 16 (first word), 2, 18 (second word)
+                        border &= border - 1;
+                        const uint32_t k = (bit & 3u) + (bit >> 4);
+                        visit(key_of(dd.at(4 * q + k)));
+                    }
                 } else if (4 * q < cv.len) {
                     for (uint32_t e = 4 * q; e < 4 * q + 4; ++e)
-                        if (e >= cv.first && e < cv.len) f |= visit(dd[e]);
+                        if (e >= cv.first && e < cv.len) f |= visit(key_of(dd.at(e)));
                 }
                 fb |= (uint32_t)f << i;
             }
@@ -155,7 +173,7 @@ __device__ __forceinline__ void sel_count_chunk(const float* __restrict__ dbuf, 
 }
 
 __global__ void __launch_bounds__(kThreads)
-k_sel_count(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks, uint64_t dstride,
+k_sel_count(DPlanes dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks, uint64_t dstride,
             uint32_t L, const Sel* __restrict__ sel, const LayerDesc* __restrict__ layers, ChunkSel* __restrict__ csel,
             uint32_t* __restrict__ low_hist, uint32_t* __restrict__ recount_n, uint2* __restrict__ recount_list) {
     __shared__ uint32_t s_hist[kLowBins];
@@ -167,7 +185,7 @@ k_sel_count(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks, ui
 
 // second round: only the chunks of the layers listed in r2
 __global__ void __launch_bounds__(kThreads)
-k_sel_count_r2(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks, uint64_t dstride,
+k_sel_count_r2(DPlanes dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks, uint64_t dstride,
                uint32_t L, const Sel* __restrict__ sel, const LayerDesc* __restrict__ layers,
                ChunkSel* __restrict__ csel, uint32_t* __restrict__ low_hist, uint32_t* __restrict__ recount_n,
                uint2* __restrict__ recount_list, const Round2* __restrict__ r2, const uint2* __restrict__ r2_chunks) {
@@ -301,7 +319,7 @@ k_sel_resolve_r2(uint32_t L, const LayerDesc* __restrict__ layers, uint32_t n_ch
 
 // Exact per-slice (gt, eq) of the chunks whose list overflowed: warp w recounts the slices w and w + 8.
 __global__ void __launch_bounds__(kThreads)
-k_sel_recount(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks, uint64_t dstride,
+k_sel_recount(DPlanes dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks, uint64_t dstride,
               uint32_t L, const Sel* __restrict__ sel, const uint32_t* __restrict__ recount_n,
               const uint2* __restrict__ recount_list, ChunkSel* __restrict__ csel) {
     const uint32_t n = *recount_n;
@@ -311,13 +329,13 @@ k_sel_recount(const float* __restrict__ dbuf, const Chunk* __restrict__ chunks, 
         const Chunk ch = chunks[e.y];
         const Sel s = sel[(size_t)e.x * L + ch.layer];
         const ChunkView cv(ch);
-        const float* dd = dbuf + (size_t)e.x * dstride + cv.a0;
+        const DView dd(dbuf, (size_t)e.x * dstride + cv.a0);
         ChunkSel* out = csel + (size_t)e.x * n_chunks + e.y;
         for (uint32_t sl = wid; sl < (uint32_t)kSlices; sl += kThreads / 32) {
             uint32_t gt = 0, eq = 0;
             const uint32_t x0 = max(cv.first, sl * kSliceElems), x1 = min(cv.len, (sl + 1) * kSliceElems);
             for (uint32_t x = x0 + lane; x < x1; x += 32) {
-                const uint32_t key = key_of(dd[x]);
+                const uint32_t key = key_of(dd.at(x));
                 gt += key > s.tau;
                 eq += key == s.tau;
             }
@@ -418,7 +436,7 @@ k_sel_scan(const LayerDesc* __restrict__ layers, const Chunk* __restrict__ chunk
 // instantiation from the budgets; both are correct for any input).
 template <bool BF16, bool DENSE>
 __global__ void __launch_bounds__(kThreads, DENSE ? 3 : 8)
-k_sel_write(const float* __restrict__ dbuf, float* __restrict__ state, const Chunk* __restrict__ chunks,
+k_sel_write(DPlanes dbuf, float* __restrict__ state, const Chunk* __restrict__ chunks,
             uint32_t n_chunks, uint64_t dstride, uint64_t stride, const ChunkSel* __restrict__ csel,
             const ChunkJob* __restrict__ jobs, uint64_t cap, uint32_t* __restrict__ out_idx, void* __restrict__ out_val) {
     const uint32_t w = blockIdx.y;
@@ -431,7 +449,7 @@ k_sel_write(const float* __restrict__ dbuf, float* __restrict__ state, const Chu
     const uint32_t keep_eq = jb.keep_eq;
     const uint32_t tau = jb.tau;
     const ChunkView cv(ch);
-    const float* dd = dbuf + (size_t)w * dstride + cv.a0;
+    const DView dd(dbuf, (size_t)w * dstride + cv.a0);
     float* st = state + (size_t)w * stride + cv.a0;
     uint32_t* oi = out_idx + (size_t)w * cap + jb.base;
     float* ov32 = reinterpret_cast<float*>(out_val) + (size_t)w * cap + jb.base;
@@ -479,7 +497,7 @@ k_sel_write(const float* __restrict__ dbuf, float* __restrict__ state, const Chu
                     if (e0 >= cv.first && e0 + 4 <= cv.len) {
                         // the state is requested together with d: a kept entry's update then waits for one
                         // memory round trip, not two
-                        const float4 a = __ldg(reinterpret_cast<const float4*>(dd + e0));
+                        const float4 a = dd.quad(e0 >> 2);
                         if (st_vec) {
                             const float4 b = *reinterpret_cast<const float4*>(st + e0);
                             sq[0] = b.x; sq[1] = b.y; sq[2] = b.z; sq[3] = b.w;
@@ -494,7 +512,7 @@ k_sel_write(const float* __restrict__ dbuf, float* __restrict__ state, const Chu
 #pragma unroll
                         for (int i = 0; i < 4; ++i)
                             if (e0 + i >= cv.first && e0 + i < cv.len) {
-                                vq[i] = __ldg(dd + e0 + i);
+                                vq[i] = dd.at(e0 + i);
                                 sq[i] = st[e0 + i];
                                 classify(vq[i], i);
                             }
@@ -550,7 +568,7 @@ k_sel_write(const float* __restrict__ dbuf, float* __restrict__ state, const Chu
             if (full) {
 #pragma unroll
                 for (int u = 0; u < E / 4; ++u) {
-                    const float4 a = __ldg(reinterpret_cast<const float4*>(dd + t0) + u);
+                    const float4 a = dd.quad((t0 >> 2) + u);
                     v[4 * u] = a.x; v[4 * u + 1] = a.y; v[4 * u + 2] = a.z; v[4 * u + 3] = a.w;
                 }
 #pragma unroll
@@ -564,7 +582,7 @@ k_sel_write(const float* __restrict__ dbuf, float* __restrict__ state, const Chu
                 for (int i = 0; i < E; ++i) {
                     const uint32_t e = t0 + i;
                     const bool in = e >= cv.first && e < cv.len;
-                    const uint32_t key = key_of(in ? __ldg(dd + e) : 0.f);
+                    const uint32_t key = key_of(in ? dd.at(e) : 0.f);
                     if (in && (all || key > tau || (eq_mode == 1 && key == tau))) keepm |= 1u << i;
                     if (in && eq_mode == 2 && key == tau) eqm |= 1u << i;
                 }
@@ -653,7 +671,7 @@ k_sel_write(const float* __restrict__ dbuf, float* __restrict__ state, const Chu
                 const int i = __ffs(keepm) - 1;
                 keepm &= keepm - 1;
                 const uint32_t e = t0 + i;
-                const float val = dd[e]; // loaded a moment ago: an L1 hit
+                const float val = dd.at(e); // loaded a moment ago: an L1 hit
                 oi[o] = idx0 + e;
                 float sent;
                 if (BF16) {
