@@ -67,7 +67,7 @@ void plan_layout(kimad_ctx* c) {
     auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes); return at; };
     const size_t WL = (size_t)c->W * c->L, WLK = WL * c->K, WR = (size_t)c->W * c->reg_layers.size();
     const size_t nch = c->chunks.size();
-    y.dbuf = take((size_t)c->W * c->dstride * sizeof(float));
+    y.dbuf = take((size_t)c->W * c->dstride * sizeof(uint16_t));
     y.chunks = take(nch * sizeof(Chunk));
     y.layers = take(c->layers.size() * sizeof(LayerDesc));
     y.ktab = take(c->ktab.size() * sizeof(uint64_t));
@@ -158,8 +158,8 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
     const bool vec = ((uintptr_t)grads % 16 == 0) && ((uintptr_t)state % 16 == 0) && (c->stride % 4 == 0);
 
     const Layout& y = c->lay;
-    // d as two 16-bit planes, each u16 [W][dstride], in the space of one f32 [W][dstride] array
-    const DPlanes dbuf{c->at<uint16_t>(y.dbuf), c->at<uint16_t>(y.dbuf) + (size_t)c->W * c->dstride};
+    // the upper halves of d, u16 [W][dstride]; exact values are recomputed from grads and state
+    const DPlanes dbuf{c->at<uint16_t>(y.dbuf), grads, state, c->stride};
     const Chunk* chunks = c->at<Chunk>(y.chunks);
     const LayerDesc* layers = c->at<LayerDesc>(y.layers);
     const uint64_t* ktab = c->at<uint64_t>(y.ktab);
@@ -223,10 +223,10 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
     }
     mark();
     if (vec)
-        k_pass_a<true><<<grun, kBigThreads, c->pass_a_smem, s>>>(grads, state, dbuf, chunks, nch, run_chunks, c->stride, c->dstride,
+        k_pass_a<true><<<grun, kBigThreads, c->pass_a_smem, s>>>(grads, state, dbuf.hi, chunks, nch, run_chunks, c->stride, c->dstride,
                                                                  reg_index, R, lut1, lut2, meta, bhc, bhs);
     else
-        k_pass_a<false><<<grun, kBigThreads, c->pass_a_smem, s>>>(grads, state, dbuf, chunks, nch, run_chunks, c->stride, c->dstride,
+        k_pass_a<false><<<grun, kBigThreads, c->pass_a_smem, s>>>(grads, state, dbuf.hi, chunks, nch, run_chunks, c->stride, c->dstride,
                                                                   reg_index, R, lut1, lut2, meta, bhc, bhs);
     c->launches += 1;
     mark();
@@ -284,7 +284,7 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
         for (uint32_t i = 0; i < W; ++i) kept = std::max(kept, std::floor(bw[i] * t) / ((double)c->bpe * (double)c->N));
         const bool dense = kept >= 0.04;
         auto launch = [&](auto kern) {
-            kern<<<gch, blk, 0, s>>>(dbuf, state, chunks, nch, c->dstride, c->stride, csel, jobs, c->cap, out->idx, out->val);
+            kern<<<gch, blk, 0, s>>>(grads, state, chunks, nch, c->dstride, c->stride, csel, jobs, c->cap, out->idx, out->val);
         };
         if (c->value_dtype == 1) { if (dense) launch(k_sel_write<true, true>); else launch(k_sel_write<true, false>); }
         else { if (dense) launch(k_sel_write<false, true>); else launch(k_sel_write<false, false>); }

@@ -374,7 +374,7 @@ constexpr int kMaxRunChunksA = 32; // a run has at most 2^20 elements: its carry
 
 template <bool VEC>
 __global__ void __launch_bounds__(kBigThreads, 1)
-k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, DPlanes dbuf,
+k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, uint16_t* __restrict__ d_hi,
          const Chunk* __restrict__ chunks, uint32_t n_chunks, uint32_t run_chunks, uint64_t stride, uint64_t dstride,
          const uint32_t* __restrict__ reg_index /* [L], 0xffffffff: tiny layer */, uint32_t R,
          const uint16_t* __restrict__ lut_t1, const uint32_t* __restrict__ lut_t2, const BandMeta* __restrict__ meta,
@@ -391,8 +391,7 @@ k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, DPlan
     for (int i = threadIdx.x; i < 3 * kMaxBins; i += kBigThreads) sh[i] = 0;
     const float* gr0 = grads + (size_t)w * stride;
     const float* st0 = state + (size_t)w * stride;
-    uint16_t* dh0 = dbuf.hi + (size_t)w * dstride;
-    uint16_t* dl0 = dbuf.lo + (size_t)w * dstride;
+    uint16_t* dh0 = d_hi + (size_t)w * dstride;
     int cur_layer = -1;
     bool active = false, dirty = false;
     uint32_t n_bins = 0;
@@ -454,7 +453,6 @@ k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, DPlan
         const float* gr = gr0 + cv.a0;
         const float* st = st0 + cv.a0;
         uint16_t* dh = dh0 + cv.a0;
-        uint16_t* dl = dl0 + cv.a0;
         const uint32_t nq = cv.quads();
         constexpr int U = 2;
         for (uint32_t qb = 0; qb < nq; qb += kBigThreads * U) {
@@ -475,17 +473,13 @@ k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, DPlan
                     float4 d;
                     d.x = __fsub_rn(a[u].x, b[u].x); d.y = __fsub_rn(a[u].y, b[u].y);
                     d.z = __fsub_rn(a[u].z, b[u].z); d.w = __fsub_rn(a[u].w, b[u].w);
-                    uint2 ph, pl;
-                    split_quad(d, ph, pl);
-                    reinterpret_cast<uint2*>(dh)[q] = ph;
-                    reinterpret_cast<uint2*>(dl)[q] = pl;
+                    reinterpret_cast<uint2*>(dh)[q] = upper_halves(d);
                     if (active) { acc(d.x); acc(d.y); acc(d.z); acc(d.w); }
                 } else {
                     for (uint32_t e = 4 * q; e < 4 * q + 4; ++e)
                         if (e >= cv.first && e < cv.len) {
                             const float d = __fsub_rn(gr[e], st[e]);
                             dh[e] = (uint16_t)(__float_as_uint(d) >> 16);
-                            dl[e] = (uint16_t)__float_as_uint(d);
                             if (active) acc(d);
                         }
                 }
@@ -712,7 +706,7 @@ k_fb_hist1(DPlanes dbuf, const Chunk* __restrict__ chunks, uint64_t dstride, uin
         const uint2 e = fb_chunks[it];
         const Chunk ch = chunks[e.y];
         const ChunkView cv(ch);
-        const DView dd(dbuf, (size_t)e.x * dstride + cv.a0);
+        const DView dd(dbuf, e.x, dstride, cv.a0);
         for (int b = threadIdx.x; b < kL1Bins; b += kThreads) { s_cnt[b] = 0; s_hi[b] = 0; s_lo[b] = 0; }
         __syncthreads();
         for (uint32_t x = cv.first + threadIdx.x; x < cv.len; x += kThreads) {
@@ -761,7 +755,7 @@ k_fb_hist23(DPlanes dbuf, const Chunk* __restrict__ chunks, uint64_t dstride, ui
             }
         __syncthreads();
         const ChunkView cv(ch);
-        const DView dd(dbuf, (size_t)e.x * dstride + cv.a0);
+        const DView dd(dbuf, e.x, dstride, cv.a0);
         uint32_t* gc = g_cnt + wl * K * kL23Bins;
         unsigned long long* gs = g_ss + wl * K * kL23Bins;
         for (uint32_t x = cv.first + threadIdx.x; x < cv.len; x += kThreads) {

@@ -37,29 +37,29 @@ struct ChunkView {
     __device__ __forceinline__ bool quad_full(uint32_t q) const { return 4 * q >= first && 4 * q + 4 <= len; }
 };
 
-// The difference vector d = grad - g is kept as two 16-bit planes (upper and lower halves of the binary32 bit
-// patterns, each u16 [W][dstride]): the counting sweep of the select stage orders keys by their upper halves and
-// reads the lower plane only for the few keys that share the upper half of the threshold.
+// The difference vector d = grad - g is never stored whole.  The sweep leaves the UPPER halves of its binary32 bit
+// patterns (u16 [W][dstride]): the counting sweep of the select stage orders keys by them and needs the exact
+// value only for the few keys that share an upper half with the threshold; whoever needs an exact d recomputes
+// the one subtraction from the inputs (the estimator is not written before the write sweep, and there every
+// element is read before it is updated).
 struct DPlanes {
     uint16_t* hi;
-    uint16_t* lo;
+    const float* grads;
+    const float* state;
+    uint64_t stride; // elements between workers in grads / state
 };
-struct DView { // one worker's planes at a chunk's aligned start
+struct DView { // one worker's data at a chunk's aligned start
     const uint16_t* hi;
-    const uint16_t* lo;
-    __device__ __forceinline__ DView(const DPlanes& p, size_t offset) : hi(p.hi + offset), lo(p.lo + offset) {}
-    __device__ __forceinline__ float at(uint32_t e) const { return __uint_as_float(((uint32_t)hi[e] << 16) | lo[e]); }
-    __device__ __forceinline__ float4 quad(uint32_t q) const { // elements 4 q .. 4 q + 3 (8-byte aligned in both planes)
-        const uint2 h = __ldg(reinterpret_cast<const uint2*>(hi) + q), l = __ldg(reinterpret_cast<const uint2*>(lo) + q);
-        return make_float4(__uint_as_float(__byte_perm(l.x, h.x, 0x5410)), __uint_as_float(__byte_perm(l.x, h.x, 0x7632)),
-                           __uint_as_float(__byte_perm(l.y, h.y, 0x5410)), __uint_as_float(__byte_perm(l.y, h.y, 0x7632)));
-    }
+    const float* gr;
+    const float* st;
+    __device__ __forceinline__ DView(const DPlanes& p, uint32_t w, uint64_t dstride, uint64_t a0)
+        : hi(p.hi + (size_t)w * dstride + a0), gr(p.grads + (size_t)w * p.stride + a0), st(p.state + (size_t)w * p.stride + a0) {}
+    __device__ __forceinline__ float at(uint32_t e) const { return __fsub_rn(gr[e], st[e]); }
 };
-// the two plane words of a quad of values
-__device__ __forceinline__ void split_quad(const float4& d, uint2& h, uint2& l) {
-    const uint32_t x = __float_as_uint(d.x), y = __float_as_uint(d.y), z = __float_as_uint(d.z), w = __float_as_uint(d.w);
-    h = make_uint2(__byte_perm(x, y, 0x7632), __byte_perm(z, w, 0x7632));
-    l = make_uint2(__byte_perm(x, y, 0x5410), __byte_perm(z, w, 0x5410));
+// the upper halves of a quad of values as two words
+__device__ __forceinline__ uint2 upper_halves(const float4& d) {
+    return make_uint2(__byte_perm(__float_as_uint(d.x), __float_as_uint(d.y), 0x7632),
+                      __byte_perm(__float_as_uint(d.z), __float_as_uint(d.w), 0x7632));
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -85,7 +85,7 @@ __device__ __forceinline__ void sel_count_chunk(const DPlanes& dbuf, const Chunk
     for (int i = threadIdx.x; i < kLowBins; i += kThreads) s_hist[i] = 0;
     if (threadIdx.x == 0) *s_n = 0;
     __syncthreads();
-    const DView dd(dbuf, (size_t)w * dstride + cv.a0);
+    const DView dd(dbuf, w, dstride, cv.a0);
     // Upper halves first: a key whose upper half lies above that of the interval's last key is above the interval,
     // one below that of its first key is below; only keys sharing an upper half with the interval (a 2^16-key
     // stretch of the axis or two) are completed from the lower plane.  The halves are 15-bit numbers after the
@@ -329,7 +329,7 @@ k_sel_recount(DPlanes dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks,
         const Chunk ch = chunks[e.y];
         const Sel s = sel[(size_t)e.x * L + ch.layer];
         const ChunkView cv(ch);
-        const DView dd(dbuf, (size_t)e.x * dstride + cv.a0);
+        const DView dd(dbuf, e.x, dstride, cv.a0);
         ChunkSel* out = csel + (size_t)e.x * n_chunks + e.y;
         for (uint32_t sl = wid; sl < (uint32_t)kSlices; sl += kThreads / 32) {
             uint32_t gt = 0, eq = 0;
@@ -436,7 +436,7 @@ k_sel_scan(const LayerDesc* __restrict__ layers, const Chunk* __restrict__ chunk
 // instantiation from the budgets; both are correct for any input).
 template <bool BF16, bool DENSE>
 __global__ void __launch_bounds__(kThreads, DENSE ? 3 : 8)
-k_sel_write(DPlanes dbuf, float* __restrict__ state, const Chunk* __restrict__ chunks,
+k_sel_write(const float* __restrict__ grads, float* __restrict__ state, const Chunk* __restrict__ chunks,
             uint32_t n_chunks, uint64_t dstride, uint64_t stride, const ChunkSel* __restrict__ csel,
             const ChunkJob* __restrict__ jobs, uint64_t cap, uint32_t* __restrict__ out_idx, void* __restrict__ out_val) {
     const uint32_t w = blockIdx.y;
@@ -449,14 +449,15 @@ k_sel_write(DPlanes dbuf, float* __restrict__ state, const Chunk* __restrict__ c
     const uint32_t keep_eq = jb.keep_eq;
     const uint32_t tau = jb.tau;
     const ChunkView cv(ch);
-    const DView dd(dbuf, (size_t)w * dstride + cv.a0);
+    // d is recomputed from the inputs; every element of the estimator is read before this kernel updates it
+    const float* gr = grads + (size_t)w * stride + cv.a0;
     float* st = state + (size_t)w * stride + cv.a0;
     uint32_t* oi = out_idx + (size_t)w * cap + jb.base;
     float* ov32 = reinterpret_cast<float*>(out_val) + (size_t)w * cap + jb.base;
     __nv_bfloat16* ov16 = reinterpret_cast<__nv_bfloat16*>(out_val) + (size_t)w * cap + jb.base;
     const uint32_t idx0 = jb.idx0;
     const uint32_t lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    const bool st_vec = (reinterpret_cast<uintptr_t>(st) & 15u) == 0;
+    const bool st_vec = ((reinterpret_cast<uintptr_t>(st) | reinterpret_cast<uintptr_t>(gr)) & 15u) == 0; // 128-bit access to both
     __shared__ uint8_t s_pos[kThreads / 32][kSparseGroups]; // per warp: the marked groups of a slice, ascending
     __shared__ uint32_t s_stage[DENSE ? kThreads / 32 : 1][DENSE ? 2 * 16 * 32 : 1]; // per warp: a round's indices, values
 
@@ -497,23 +498,24 @@ k_sel_write(DPlanes dbuf, float* __restrict__ state, const Chunk* __restrict__ c
                     if (e0 >= cv.first && e0 + 4 <= cv.len) {
                         // the state is requested together with d: a kept entry's update then waits for one
                         // memory round trip, not two
-                        const float4 a = dd.quad(e0 >> 2);
+                        float gq[4];
                         if (st_vec) {
+                            const float4 a = __ldg(reinterpret_cast<const float4*>(gr + e0));
                             const float4 b = *reinterpret_cast<const float4*>(st + e0);
+                            gq[0] = a.x; gq[1] = a.y; gq[2] = a.z; gq[3] = a.w;
                             sq[0] = b.x; sq[1] = b.y; sq[2] = b.z; sq[3] = b.w;
                         } else {
 #pragma unroll
-                            for (int i = 0; i < 4; ++i) sq[i] = st[e0 + i];
+                            for (int i = 0; i < 4; ++i) { gq[i] = __ldg(gr + e0 + i); sq[i] = st[e0 + i]; }
                         }
-                        vq[0] = a.x; vq[1] = a.y; vq[2] = a.z; vq[3] = a.w;
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) classify(vq[i], i);
+                        for (int i = 0; i < 4; ++i) { vq[i] = __fsub_rn(gq[i], sq[i]); classify(vq[i], i); }
                     } else {
 #pragma unroll
                         for (int i = 0; i < 4; ++i)
                             if (e0 + i >= cv.first && e0 + i < cv.len) {
-                                vq[i] = dd.at(e0 + i);
                                 sq[i] = st[e0 + i];
+                                vq[i] = __fsub_rn(__ldg(gr + e0 + i), sq[i]);
                                 classify(vq[i], i);
                             }
                     }
@@ -565,11 +567,24 @@ k_sel_write(DPlanes dbuf, float* __restrict__ state, const Chunk* __restrict__ c
             uint32_t keepm = 0, eqm = 0;
             const bool full = rb >= cv.first && rb + E * 32 <= cv.len; // round fully inside the chunk
             float v[E];
+            float sv[DENSE ? E : 1]; // the dense instantiation keeps the estimator's values for its update
             if (full) {
+                if (st_vec) {
 #pragma unroll
-                for (int u = 0; u < E / 4; ++u) {
-                    const float4 a = dd.quad((t0 >> 2) + u);
-                    v[4 * u] = a.x; v[4 * u + 1] = a.y; v[4 * u + 2] = a.z; v[4 * u + 3] = a.w;
+                    for (int u = 0; u < E / 4; ++u) {
+                        const float4 a = __ldg(reinterpret_cast<const float4*>(gr + t0) + u);
+                        const float4 b = *(reinterpret_cast<const float4*>(st + t0) + u);
+                        v[4 * u] = __fsub_rn(a.x, b.x); v[4 * u + 1] = __fsub_rn(a.y, b.y);
+                        v[4 * u + 2] = __fsub_rn(a.z, b.z); v[4 * u + 3] = __fsub_rn(a.w, b.w);
+                        if (DENSE) { sv[4 * u] = b.x; sv[4 * u + 1] = b.y; sv[4 * u + 2] = b.z; sv[4 * u + 3] = b.w; }
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < E; ++i) {
+                        const float b = st[t0 + i];
+                        v[i] = __fsub_rn(__ldg(gr + t0 + i), b);
+                        if (DENSE) sv[i] = b;
+                    }
                 }
 #pragma unroll
                 for (int i = 0; i < E; ++i) {
@@ -582,7 +597,7 @@ k_sel_write(DPlanes dbuf, float* __restrict__ state, const Chunk* __restrict__ c
                 for (int i = 0; i < E; ++i) {
                     const uint32_t e = t0 + i;
                     const bool in = e >= cv.first && e < cv.len;
-                    const uint32_t key = key_of(in ? dd.at(e) : 0.f);
+                    const uint32_t key = key_of(in ? __fsub_rn(__ldg(gr + e), st[e]) : 0.f);
                     if (in && (all || key > tau || (eq_mode == 1 && key == tau))) keepm |= 1u << i;
                     if (in && eq_mode == 2 && key == tau) eqm |= 1u << i;
                 }
@@ -613,17 +628,6 @@ k_sel_write(DPlanes dbuf, float* __restrict__ state, const Chunk* __restrict__ c
             if (DENSE && full && round_total >= 48u) {
                 // many kept entries: values come from the registers and the state is read before it is needed,
                 // so that no store waits for a load of its own
-                float sv[E];
-                if (st_vec) {
-#pragma unroll
-                    for (int u = 0; u < E / 4; ++u) {
-                        const float4 b = *(reinterpret_cast<const float4*>(st + t0) + u);
-                        sv[4 * u] = b.x; sv[4 * u + 1] = b.y; sv[4 * u + 2] = b.z; sv[4 * u + 3] = b.w;
-                    }
-                } else {
-#pragma unroll
-                    for (int i = 0; i < E; ++i) sv[i] = (keepm >> i) & 1u ? st[t0 + i] : 0.f;
-                }
                 // the round's entries are laid out in shared memory first, so that the packed buffers are written
                 // with consecutive lanes on consecutive entries
                 uint32_t* sg_idx = s_stage[wid];
@@ -671,7 +675,8 @@ k_sel_write(DPlanes dbuf, float* __restrict__ state, const Chunk* __restrict__ c
                 const int i = __ffs(keepm) - 1;
                 keepm &= keepm - 1;
                 const uint32_t e = t0 + i;
-                const float val = dd.at(e); // loaded a moment ago: an L1 hit
+                const float was = st[e];
+                const float val = __fsub_rn(__ldg(gr + e), was); // both loaded a moment ago: L1 hits
                 oi[o] = idx0 + e;
                 float sent;
                 if (BF16) {
@@ -682,7 +687,7 @@ k_sel_write(DPlanes dbuf, float* __restrict__ state, const Chunk* __restrict__ c
                     ov32[o] = val;
                     sent = val;
                 }
-                st[e] = __fadd_rn(st[e], sent);
+                st[e] = __fadd_rn(was, sent);
                 ++o;
             }
         }
