@@ -113,7 +113,8 @@ int kimad_create(kimad_ctx** out, const uint64_t* layer_sizes, uint32_t n_layers
                  const double* ratio_grid, uint32_t n_ratios, const kimad_options* opt);
 void kimad_destroy(kimad_ctx* ctx);
 
-/* Scratch the kernels need (difference vector, histograms, DP back-pointers, tile counts). */
+/* Scratch the kernels need (upper halves of the difference vector, histograms, DP back-pointers, tile
+ * counts): about 2 bytes per element plus tables. */
 size_t kimad_workspace_bytes(const kimad_ctx* ctx);
 /* dev_ptr: device, 256-byte aligned, at least kimad_workspace_bytes(); stays owned by the
  * caller and must outlive the context's steps.  Uploads the static tables and zeroes the

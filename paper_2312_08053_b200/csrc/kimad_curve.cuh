@@ -6,7 +6,7 @@
 //                (sample rank +- 6 sigma) form a band.  Band cells are cut into fine bins of 2^shift
 //                keys, everything else into coarse "gap" bins; the mapping key -> bin is a two-level
 //                table (11-bit bin -> row, row x 5 more bits -> bin base and shift).
-//   k_pass_a     the sweep: d = grad - g (written to scratch), bin = table(key(d)), two u32 shared-
+//   k_pass_a     the sweep: d = grad - g (its upper 16 bits go to scratch), bin = table(key(d)), two u32 shared-
 //                memory atomics per element: the count, and the exact integer sum of squares in a low u32 word
 //                whose (rare) carries go to a high word.
 //   k_resolve_a  per (worker, layer): walks the bins from the top, finds the bin that holds every

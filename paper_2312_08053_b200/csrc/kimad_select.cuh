@@ -2,7 +2,7 @@
 //
 // After the DP every (worker, layer) knows a key interval [lo, lo + 2^shift) that contains its
 // threshold and the rank of the threshold inside that interval (shift = 0 when the curve stage already
-// resolved all 31 bits).  One sweep over the difference vector (k_sel_count) counts, per 2048-element slice,
+// resolved all 31 bits).  One sweep over the upper halves of the difference vector (k_sel_count) counts, per 2048-element slice,
 // the entries above the interval, remembers the few entries inside it and marks the 32-element groups that
 // can hold a kept entry; k_sel_resolve turns the remembered entries (or their per-layer histogram) into the
 // exact threshold; k_sel_slices and k_sel_scan derive every slice's and chunk's output offset and leave one
