@@ -133,6 +133,22 @@ static int preload_kernels() {
     return KIMAD_OK;
 }
 
+// Launch with programmatic stream serialisation (the kernel must start with pdl_wait()).
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+
 static int ensure_side_stream(kimad_ctx* c) {
     if (c->side) return KIMAD_OK;
     CUDA_TRY(cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking));
@@ -209,30 +225,30 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
     if (T) CUDA_TRY(cudaEventRecord(c->ev_fork, s)); // fork point of the tiny layers' kernel: the step's start
     // (a) + (b): sample -> bands -> one sweep -> curves
     if (R) {
-        k_sample<<<dim3(R, W), kBigThreads, c->sample_smem, s>>>(grads, state, c->stride, layers, reg_layers, R, ktab, K,
-                                                                 c->curve_mode == 1 ? 1u : 0u, lut1, lut2, binlo, meta);
+        CUDA_TRY(launch_pdl(k_sample, dim3(R, W), kBigThreads, c->sample_smem, s, grads, state, c->stride, layers, reg_layers, R,
+                            ktab, K, c->curve_mode == 1 ? 1u : 0u, lut1, lut2, binlo, meta));
         c->launches += 1;
     }
     if (T) { // tiny layers: sorted in shared memory on the side stream; issued after the sample kernel so that
              // its CTAs fill the SMs the sample kernel leaves idle instead of delaying it
         CUDA_TRY(cudaStreamWaitEvent(c->side, c->ev_fork, 0));
-        k_tiny_exact<<<dim3(T, W), blk, c->tiny_smem, c->side>>>(grads, state, c->stride, layers, tiny_layers, L, ktab, K, err,
-                                                                 tau, keq, shf, flags);
+        CUDA_TRY(launch_pdl(k_tiny_exact, dim3(T, W), blk, c->tiny_smem, c->side, grads, state, c->stride, layers, tiny_layers, L,
+                            ktab, K, err, tau, keq, shf, flags));
         CUDA_TRY(cudaEventRecord(c->ev_join, c->side));
         c->launches += 1;
     }
     mark();
     if (vec)
-        k_pass_a<true><<<grun, kBigThreads, c->pass_a_smem, s>>>(grads, state, dbuf.hi, chunks, nch, run_chunks, c->stride, c->dstride,
-                                                                 reg_index, R, lut1, lut2, meta, bhc, bhs);
+        CUDA_TRY(launch_pdl(k_pass_a<true>, grun, kBigThreads, c->pass_a_smem, s, grads, state, dbuf.hi, chunks, nch, run_chunks,
+                            c->stride, c->dstride, reg_index, R, lut1, lut2, meta, bhc, bhs));
     else
-        k_pass_a<false><<<grun, kBigThreads, c->pass_a_smem, s>>>(grads, state, dbuf.hi, chunks, nch, run_chunks, c->stride, c->dstride,
-                                                                  reg_index, R, lut1, lut2, meta, bhc, bhs);
+        CUDA_TRY(launch_pdl(k_pass_a<false>, grun, kBigThreads, c->pass_a_smem, s, grads, state, dbuf.hi, chunks, nch, run_chunks,
+                            c->stride, c->dstride, reg_index, R, lut1, lut2, meta, bhc, bhs));
     c->launches += 1;
     mark();
     if (R) {
-        k_resolve_a<<<dim3(R, W), kBigThreads, 0, s>>>(layers, reg_layers, R, L, ktab, K, meta, binlo, bhc, bhs, err, tau,
-                                                       keq, shf, flags, fb, fb_chunks, fb_layers);
+        CUDA_TRY(launch_pdl(k_resolve_a, dim3(R, W), kBigThreads, 0, s, layers, reg_layers, R, L, ktab, K, meta, binlo, bhc, bhs, err, tau,
+                                                       keq, shf, flags, fb, fb_chunks, fb_layers));
         c->launches += 1;
     }
     if (T) CUDA_TRY(cudaStreamWaitEvent(s, c->ev_join, 0));
@@ -241,13 +257,13 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
     if (R) {
         const uint32_t gfb = 2 * 148, glay = std::min<uint32_t>(W * R, 128u);
         const dim3 gslot(glay, 1, K);
-        k_fb_hist1<<<gfb, blk, 0, s>>>(dbuf, chunks, c->dstride, L, fb, fb_chunks, h1c, h1s, flags);
-        k_resolve1<<<glay, blk, 0, s>>>(fb, fb_layers, h1c, h1s, ktab, L, K, cands, slots);
-        k_fb_hist23<2><<<gfb, blk, 0, s>>>(dbuf, chunks, c->dstride, L, K, fb, fb_chunks, slots, h23c, h23s);
-        k_resolve23<2><<<gslot, blk, 0, s>>>(fb, fb_layers, h23c, h23s, L, K, cands, slots, err, tau, keq, shf);
-        k_rebuild_slots<<<(W * R + kThreads - 1) / kThreads, blk, 0, s>>>(fb, fb_layers, L, K, cands, slots);
-        k_fb_hist23<3><<<gfb, blk, 0, s>>>(dbuf, chunks, c->dstride, L, K, fb, fb_chunks, slots, h23c, h23s);
-        k_resolve23<3><<<gslot, blk, 0, s>>>(fb, fb_layers, h23c, h23s, L, K, cands, slots, err, tau, keq, shf);
+        CUDA_TRY(launch_pdl(k_fb_hist1, gfb, blk, 0, s, dbuf, chunks, c->dstride, L, fb, fb_chunks, h1c, h1s, flags));
+        CUDA_TRY(launch_pdl(k_resolve1, glay, blk, 0, s, fb, fb_layers, h1c, h1s, ktab, L, K, cands, slots));
+        CUDA_TRY(launch_pdl(k_fb_hist23<2>, gfb, blk, 0, s, dbuf, chunks, c->dstride, L, K, fb, fb_chunks, slots, h23c, h23s));
+        CUDA_TRY(launch_pdl(k_resolve23<2>, gslot, blk, 0, s, fb, fb_layers, h23c, h23s, L, K, cands, slots, err, tau, keq, shf));
+        CUDA_TRY(launch_pdl(k_rebuild_slots, (W * R + kThreads - 1) / kThreads, blk, 0, s, fb, fb_layers, L, K, cands, slots));
+        CUDA_TRY(launch_pdl(k_fb_hist23<3>, gfb, blk, 0, s, dbuf, chunks, c->dstride, L, K, fb, fb_chunks, slots, h23c, h23s));
+        CUDA_TRY(launch_pdl(k_resolve23<3>, gslot, blk, 0, s, fb, fb_layers, h23c, h23s, L, K, cands, slots, err, tau, keq, shf));
         c->launches += 7;
     }
     mark();
@@ -259,24 +275,24 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
             double cb = std::floor(bw[w0 + i] * t);
             b.c[i] = !(cb > 0.0) ? 0ull : (cb >= 18446744073709551615.0 ? ~0ull : (uint64_t)cb);
         }
-        k_dp<<<nw, kDpThreads, c->dp_smem, s>>>(b, w0, W, L, K, c->D, c->bpe, c->full_bytes, c->cap, c->check_finite,
-                                                mode == kGivenJ ? 1 : (c->policy == 1 ? 2 : (c->policy == 2 ? 3 : 0)), c->dp_plan, ktab,
-                                                mode == kInjectErr ? err_dev : err, tau, keq, shf, j_dev, flags, pd, sel,
-                                                out->k, out->j, out->offs, out->stats);
+        CUDA_TRY(launch_pdl(k_dp, nw, kDpThreads, c->dp_smem, s, b, w0, W, L, K, c->D, c->bpe, c->full_bytes, c->cap,
+                            c->check_finite, mode == kGivenJ ? 1 : (c->policy == 1 ? 2 : (c->policy == 2 ? 3 : 0)), c->dp_plan,
+                            ktab, mode == kInjectErr ? err_dev : err, tau, keq, shf, j_dev, flags, pd, sel, out->k, out->j,
+                            out->offs, out->stats));
         c->launches += 1;
     }
     mark();
     // (d), (e), (f)
-    k_sel_count<<<gch, blk, 0, s>>>(dbuf, chunks, nch, c->dstride, L, sel, layers, csel, lowh, recount_n, recount_list);
+    CUDA_TRY(launch_pdl(k_sel_count, gch, blk, 0, s, dbuf, chunks, nch, c->dstride, L, sel, layers, csel, lowh, recount_n, recount_list));
     mark();
-    k_sel_resolve<<<glw, blk, 0, s>>>(L, layers, nch, csel, lowh, sel, r2, r2_layers, r2_chunks);
-    k_sel_count_r2<<<2 * 148, blk, 0, s>>>(dbuf, chunks, nch, c->dstride, L, sel, layers, csel, lowh, recount_n,
-                                          recount_list, r2, r2_chunks);
-    k_sel_resolve_r2<<<std::min<uint32_t>(W * L, 128u), blk, 0, s>>>(L, layers, nch, csel, lowh, sel, r2, r2_layers,
-                                                                   r2_chunks);
-    k_sel_recount<<<2 * 148, blk, 0, s>>>(dbuf, chunks, nch, c->dstride, L, sel, recount_n, recount_list, csel);
-    k_sel_slices<<<(uint32_t)(((uint64_t)W * nch + 7) / 8), blk, 0, s>>>(chunks, nch, W, L, sel, csel, ccnt);
-    k_sel_scan<<<glw, blk, 0, s>>>(layers, chunks, nch, L, sel, ccnt, jobs, recount_n, fb, r2);
+    CUDA_TRY(launch_pdl(k_sel_resolve, glw, blk, 0, s, L, layers, nch, csel, lowh, sel, r2, r2_layers, r2_chunks));
+    CUDA_TRY(launch_pdl(k_sel_count_r2, 2 * 148, blk, 0, s, dbuf, chunks, nch, c->dstride, L, sel, layers, csel, lowh, recount_n,
+                                          recount_list, r2, r2_chunks));
+    CUDA_TRY(launch_pdl(k_sel_resolve_r2, std::min<uint32_t>(W * L, 128u), blk, 0, s, L, layers, nch, csel, lowh, sel, r2,
+                        r2_layers, r2_chunks));
+    CUDA_TRY(launch_pdl(k_sel_recount, 2 * 148, blk, 0, s, dbuf, chunks, nch, c->dstride, L, sel, recount_n, recount_list, csel));
+    CUDA_TRY(launch_pdl(k_sel_slices, (uint32_t)(((uint64_t)W * nch + 7) / 8), blk, 0, s, chunks, nch, W, L, sel, csel, ccnt));
+    CUDA_TRY(launch_pdl(k_sel_scan, glw, blk, 0, s, layers, chunks, nch, L, sel, ccnt, jobs, recount_n, fb, r2));
     mark();
     {
         // budget share kept, from the host's view of the budgets: picks the tuning of the write sweep
@@ -284,10 +300,11 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
         for (uint32_t i = 0; i < W; ++i) kept = std::max(kept, std::floor(bw[i] * t) / ((double)c->bpe * (double)c->N));
         const bool dense = kept >= 0.04;
         auto launch = [&](auto kern) {
-            kern<<<gch, blk, 0, s>>>(grads, state, chunks, nch, c->dstride, c->stride, csel, jobs, c->cap, out->idx, out->val);
+            return launch_pdl(kern, gch, blk, 0, s, grads, state, chunks, nch, c->dstride, c->stride, csel, jobs, c->cap,
+                              out->idx, out->val);
         };
-        if (c->value_dtype == 1) { if (dense) launch(k_sel_write<true, true>); else launch(k_sel_write<true, false>); }
-        else { if (dense) launch(k_sel_write<false, true>); else launch(k_sel_write<false, false>); }
+        if (c->value_dtype == 1) CUDA_TRY(dense ? launch(k_sel_write<true, true>) : launch(k_sel_write<true, false>));
+        else CUDA_TRY(dense ? launch(k_sel_write<false, true>) : launch(k_sel_write<false, false>));
     }
     mark();
     c->launches += 8;

@@ -52,6 +52,7 @@ k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint6
          const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ reg_layers, uint32_t R,
          const uint64_t* __restrict__ ktab, uint32_t K, uint32_t force_exact, uint16_t* __restrict__ lut_t1,
          uint32_t* __restrict__ lut_t2, uint32_t* __restrict__ bin_lo, BandMeta* __restrict__ meta) {
+    pdl_wait();
     extern __shared__ __align__(16) uint32_t sh[];
     double* s_sq = reinterpret_cast<double*>(sh); // [1024] squares (cell midpoints) below each thread segment
     double* s_wd = s_sq + 1024;                   // [32]
@@ -379,6 +380,7 @@ k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, uint1
          const uint32_t* __restrict__ reg_index /* [L], 0xffffffff: tiny layer */, uint32_t R,
          const uint16_t* __restrict__ lut_t1, const uint32_t* __restrict__ lut_t2, const BandMeta* __restrict__ meta,
          uint32_t* __restrict__ bh_cnt, unsigned long long* __restrict__ bh_sum) {
+    pdl_wait();
     extern __shared__ __align__(16) uint32_t sh[];
     uint32_t* h_cnt = sh;
     uint32_t* h_hi = sh + kMaxBins;
@@ -500,6 +502,7 @@ k_resolve_a(const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ r
             float* __restrict__ err_out, uint32_t* __restrict__ tau_out, uint32_t* __restrict__ rank_out,
             uint32_t* __restrict__ shift_out, uint32_t* __restrict__ flags, FbList* __restrict__ fb,
             uint2* __restrict__ fb_chunks, uint2* __restrict__ fb_layers) {
+    pdl_wait();
     __shared__ uint32_t s_drop[KIMAD_MAX_RATIOS]; // entries not kept by candidate j: n - k_j
     __shared__ uint32_t s_bin[KIMAD_MAX_RATIOS], s_before[KIMAD_MAX_RATIOS], s_cb[KIMAD_MAX_RATIOS];
     __shared__ double s_below[KIMAD_MAX_RATIOS], s_sb[KIMAD_MAX_RATIOS];
@@ -628,6 +631,7 @@ k_tiny_exact(const float* __restrict__ grads, const float* __restrict__ state, u
              const uint32_t* __restrict__ tiny_layers, uint32_t L, const uint64_t* __restrict__ ktab, uint32_t K,
              float* __restrict__ err_out, uint32_t* __restrict__ tau_out, uint32_t* __restrict__ rank_out,
              uint32_t* __restrict__ shift_out, uint32_t* __restrict__ flags) {
+    pdl_wait();
     extern __shared__ __align__(16) unsigned char tiny_smem[];
     double* s_suf = reinterpret_cast<double*>(tiny_smem);                // [kTinyMax] squares of the entries ranked >= i
     uint32_t* s_key = reinterpret_cast<uint32_t*>(s_suf + kTinyMax);     // [kTinyMax]
@@ -700,6 +704,7 @@ __global__ void __launch_bounds__(kThreads)
 k_fb_hist1(DPlanes dbuf, const Chunk* __restrict__ chunks, uint64_t dstride, uint32_t L,
            const FbList* __restrict__ fb, const uint2* __restrict__ fb_chunks, uint32_t* __restrict__ g_cnt,
            unsigned long long* __restrict__ g_ss, uint32_t* __restrict__ flags) {
+    pdl_wait();
     __shared__ uint32_t s_cnt[kL1Bins], s_hi[kL1Bins], s_lo[kL1Bins];
     const uint32_t n = fb->n_chunks;
     for (uint32_t it = blockIdx.x; it < n; it += gridDim.x) {
@@ -734,6 +739,7 @@ __global__ void __launch_bounds__(kThreads)
 k_fb_hist23(DPlanes dbuf, const Chunk* __restrict__ chunks, uint64_t dstride, uint32_t L, uint32_t K,
             const FbList* __restrict__ fb, const uint2* __restrict__ fb_chunks, const SlotTab* __restrict__ slots,
             uint32_t* __restrict__ g_cnt, unsigned long long* __restrict__ g_ss) {
+    pdl_wait();
     __shared__ uint8_t s_first[kL1Bins]; // level-1 bin -> first slot whose prefix starts with it (0xff: none)
     __shared__ uint8_t s_num[kL1Bins];   // ... and how many consecutive slots share that bin (level 3)
     __shared__ uint32_t s_prefix[KIMAD_MAX_RATIOS];

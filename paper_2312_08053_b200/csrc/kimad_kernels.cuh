@@ -28,6 +28,11 @@ __device__ __forceinline__ uint32_t key_of(float d) { return __float_as_uint(d) 
 
 // Aligned view of a chunk for 128-bit loads: quads start at a0 = begin & ~3; only the first and the
 // last quad can be partial.  All offsets are 32-bit and relative to a0.
+// Kernels launched with programmatic stream serialisation may be scheduled before their predecessor in the
+// stream has finished (which hides their launch latency); they wait here, before touching anything it wrote.
+// A no-op for an ordinary launch.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 struct ChunkView {
     uint64_t a0;
     uint32_t first, len; // valid element offsets are [first, len)
@@ -173,6 +178,7 @@ __global__ void __launch_bounds__(kThreads)
 k_resolve1(const FbList* __restrict__ fb, const uint2* __restrict__ fb_layers, uint32_t* __restrict__ g_cnt,
            unsigned long long* __restrict__ g_ss, const uint64_t* __restrict__ ktab, uint32_t L, uint32_t K,
            Cand* __restrict__ cands, SlotTab* __restrict__ slots) {
+    pdl_wait();
     __shared__ __align__(16) uint32_t s_incl[kL1Bins];
     __shared__ __align__(16) double s_below[kL1Bins];
     __shared__ uint32_t s_w32[8];
@@ -234,6 +240,7 @@ k_resolve23(const FbList* __restrict__ fb, const uint2* __restrict__ fb_layers, 
             unsigned long long* __restrict__ g_ss, uint32_t L, uint32_t K, Cand* __restrict__ cands,
             const SlotTab* __restrict__ slots, float* __restrict__ err_out, uint32_t* __restrict__ tau_out,
             uint32_t* __restrict__ keep_eq_out, uint32_t* __restrict__ shift_out) {
+    pdl_wait();
     __shared__ __align__(16) uint32_t s_incl[kL23Bins];
     __shared__ __align__(16) double s_below[kL23Bins];
     __shared__ uint32_t s_w32[8];
@@ -304,6 +311,7 @@ k_resolve23(const FbList* __restrict__ fb, const uint2* __restrict__ fb_layers, 
 __global__ void __launch_bounds__(kThreads)
 k_rebuild_slots(const FbList* __restrict__ fb, const uint2* __restrict__ fb_layers, uint32_t L, uint32_t K,
                 Cand* __restrict__ cands, SlotTab* __restrict__ slots) {
+    pdl_wait();
     const uint32_t it = blockIdx.x * kThreads + threadIdx.x;
     if (it >= fb->n_layers) return;
     const size_t wl = (size_t)fb_layers[it].x * L + fb_layers[it].y;
@@ -350,6 +358,7 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
      const uint32_t* __restrict__ j_in, uint32_t* __restrict__ flags,
      uint8_t* __restrict__ pd_global, Sel* __restrict__ sel, uint32_t* __restrict__ out_k,
      uint32_t* __restrict__ out_j, uint64_t* __restrict__ out_offs, kimad_stats* __restrict__ out_stats) {
+    pdl_wait();
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const uint32_t w = w_base + blockIdx.x;
     if (w >= W) return;

@@ -176,6 +176,7 @@ __global__ void __launch_bounds__(kThreads)
 k_sel_count(DPlanes dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks, uint64_t dstride,
             uint32_t L, const Sel* __restrict__ sel, const LayerDesc* __restrict__ layers, ChunkSel* __restrict__ csel,
             uint32_t* __restrict__ low_hist, uint32_t* __restrict__ recount_n, uint2* __restrict__ recount_list) {
+    pdl_wait();
     __shared__ uint32_t s_hist[kLowBins];
     __shared__ uint32_t s_n;
     __shared__ uint32_t s_low[kListCap];
@@ -189,6 +190,7 @@ k_sel_count_r2(DPlanes dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks
                uint32_t L, const Sel* __restrict__ sel, const LayerDesc* __restrict__ layers,
                ChunkSel* __restrict__ csel, uint32_t* __restrict__ low_hist, uint32_t* __restrict__ recount_n,
                uint2* __restrict__ recount_list, const Round2* __restrict__ r2, const uint2* __restrict__ r2_chunks) {
+    pdl_wait();
     __shared__ uint32_t s_hist[kLowBins];
     __shared__ uint32_t s_n;
     __shared__ uint32_t s_low[kListCap];
@@ -297,6 +299,7 @@ __global__ void __launch_bounds__(kThreads)
 k_sel_resolve(uint32_t L, const LayerDesc* __restrict__ layers, uint32_t n_chunks, const ChunkSel* __restrict__ csel,
               uint32_t* __restrict__ low_hist, Sel* __restrict__ sel, Round2* __restrict__ r2,
               uint2* __restrict__ r2_layers, uint2* __restrict__ r2_chunks) {
+    pdl_wait();
     __shared__ __align__(16) uint32_t s_key[kSortCap];
     __shared__ uint32_t s_w32[8];
     __shared__ uint32_t s_n, s_over;
@@ -308,6 +311,7 @@ __global__ void __launch_bounds__(kThreads)
 k_sel_resolve_r2(uint32_t L, const LayerDesc* __restrict__ layers, uint32_t n_chunks, const ChunkSel* __restrict__ csel,
                  uint32_t* __restrict__ low_hist, Sel* __restrict__ sel, Round2* __restrict__ r2,
                  uint2* __restrict__ r2_layers, uint2* __restrict__ r2_chunks) {
+    pdl_wait();
     __shared__ __align__(16) uint32_t s_key[kSortCap];
     __shared__ uint32_t s_w32[8];
     __shared__ uint32_t s_n, s_over;
@@ -322,6 +326,7 @@ __global__ void __launch_bounds__(kThreads)
 k_sel_recount(DPlanes dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks, uint64_t dstride,
               uint32_t L, const Sel* __restrict__ sel, const uint32_t* __restrict__ recount_n,
               const uint2* __restrict__ recount_list, ChunkSel* __restrict__ csel) {
+    pdl_wait();
     const uint32_t n = *recount_n;
     const uint32_t lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     for (uint32_t it = blockIdx.x; it < n; it += gridDim.x) {
@@ -354,6 +359,7 @@ k_sel_recount(DPlanes dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks,
 __global__ void __launch_bounds__(kThreads)
 k_sel_slices(const Chunk* __restrict__ chunks, uint32_t n_chunks, uint32_t W, uint32_t L, const Sel* __restrict__ sel,
              ChunkSel* __restrict__ csel, uint2* __restrict__ chunk_cnt) {
+    pdl_wait();
     const uint32_t lane = threadIdx.x & 31;
     const uint64_t it = (uint64_t)blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
     if (it >= (uint64_t)W * n_chunks) return;
@@ -387,6 +393,7 @@ __global__ void __launch_bounds__(kThreads)
 k_sel_scan(const LayerDesc* __restrict__ layers, const Chunk* __restrict__ chunks, uint32_t n_chunks, uint32_t L,
            const Sel* __restrict__ sel, const uint2* __restrict__ chunk_cnt, ChunkJob* __restrict__ jobs,
            uint32_t* __restrict__ recount_n, FbList* __restrict__ fb, Round2* __restrict__ r2) {
+    pdl_wait();
     __shared__ uint32_t s_w[8];
     const LayerDesc ld = layers[blockIdx.x];
     const uint32_t w = blockIdx.y;
@@ -439,6 +446,7 @@ __global__ void __launch_bounds__(kThreads, DENSE ? 3 : 8)
 k_sel_write(const float* __restrict__ grads, float* __restrict__ state, const Chunk* __restrict__ chunks,
             uint32_t n_chunks, uint64_t dstride, uint64_t stride, const ChunkSel* __restrict__ csel,
             const ChunkJob* __restrict__ jobs, uint64_t cap, uint32_t* __restrict__ out_idx, void* __restrict__ out_val) {
+    pdl_wait();
     const uint32_t w = blockIdx.y;
     const ChunkJob jb = jobs[(size_t)w * n_chunks + blockIdx.x];
     if (jb.mode == 0) return; // nothing kept in this chunk
