@@ -82,8 +82,10 @@ __device__ __forceinline__ void sel_count_chunk(const DPlanes& dbuf, const Chunk
     }
     const uint32_t lo = s.tau, width = 1u << s.shift;
     const uint32_t hshift = s.shift > 10 ? s.shift - 10 : 0; // the histogram has at most kLowBins bins
+    __shared__ uint32_t s_gm[kThreads / 32]; // per warp: group bits of the half slice in work (zero between uses)
     for (int i = threadIdx.x; i < kLowBins; i += kThreads) s_hist[i] = 0;
     if (threadIdx.x == 0) *s_n = 0;
+    if (threadIdx.x < kThreads / 32) s_gm[threadIdx.x] = 0;
     __syncthreads();
     const DView dd(dbuf, w, dstride, cv.a0);
     // Upper halves first: a key whose upper half lies above that of the interval's last key is above the interval,
@@ -139,14 +141,33 @@ __device__ __forceinline__ void sel_count_chunk(const DPlanes& dbuf, const Chunk
                 }
                 fb |= (uint32_t)f << i;
             }
-            // a row of 128 elements = four groups of 8 lanes: OR the rows' flags inside each group, spread the
-            // 8 row bits to every fourth position, shift by the group, and OR the four groups
+            // a row of 128 elements = four groups of 8 lanes: a lane's 8 row flags, spread to every fourth bit and
+            // shifted by its group, are its share of this half slice's 32 group bits.  Few marked lanes (sparse
+            // budgets): they OR their shares into a word of shared memory; many: two warp OR-reductions.
             const uint32_t g = lane >> 3;
-            uint32_t r8 = __reduce_or_sync(0xffu << (8 * g), fb);
-            r8 = (r8 | (r8 << 12)) & 0x000f000fu;
-            r8 = (r8 | (r8 << 6)) & 0x03030303u;
-            r8 = (r8 | (r8 << 3)) & 0x11111111u;
-            const uint32_t half = __reduce_or_sync(0xffffffffu, r8 << g);
+            const uint32_t marked = __ballot_sync(0xffffffffu, fb != 0);
+            uint32_t half = 0;
+            if (__popc(marked) <= 6) {
+                if (fb) {
+                    uint32_t r8 = fb;
+                    r8 = (r8 | (r8 << 12)) & 0x000f000fu;
+                    r8 = (r8 | (r8 << 6)) & 0x03030303u;
+                    r8 = (r8 | (r8 << 3)) & 0x11111111u;
+                    atomicOr(&s_gm[wid], r8 << g);
+                }
+                if (marked) {
+                    __syncwarp();
+                    half = s_gm[wid];
+                    __syncwarp();
+                    if (lane == 0) s_gm[wid] = 0;
+                }
+            } else {
+                uint32_t r8 = __reduce_or_sync(0xffu << (8 * g), fb);
+                r8 = (r8 | (r8 << 12)) & 0x000f000fu;
+                r8 = (r8 | (r8 << 6)) & 0x03030303u;
+                r8 = (r8 | (r8 << 3)) & 0x11111111u;
+                half = __reduce_or_sync(0xffffffffu, r8 << g);
+            }
             mask |= (uint64_t)half << (32 * ((q0 - sl * (kSliceElems / 4)) / (H * 32)));
         }
 #pragma unroll
