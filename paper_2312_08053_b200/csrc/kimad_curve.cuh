@@ -456,7 +456,7 @@ k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, uint1
         const float* st = st0 + cv.a0;
         uint16_t* dh = dh0 + cv.a0;
         const uint32_t nq = cv.quads();
-        constexpr int U = 2;
+        constexpr int U = 4; // quads in flight per thread: 16 KB per array and pass, two passes per full chunk
         for (uint32_t qb = 0; qb < nq; qb += kBigThreads * U) {
             float4 a[U], b[U];
 #pragma unroll
