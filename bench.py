@@ -32,7 +32,7 @@ UNIT = "elements/s"
 
 # DRAM traffic of the dominant kernel per input element, from the ncu capture summarised under
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum of one launch / elements of that launch).
-NCU_TRAFFIC_BYTES_PER_ELEM = {"sweep": 10.11}  # profiles/k_pass_a_resnet50_shape.md
+NCU_TRAFFIC_BYTES_PER_ELEM = {"sweep": 10.13}  # profiles/k_pass_a_resnet50_shape.md
 
 # algorithmic bytes per input element of each stage (what the stage must move at least once)
 STAGE_ALGO_BYTES = {"sweep": 10.0,  # read grad + g, write the upper halves of d
