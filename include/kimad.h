@@ -15,12 +15,19 @@
  *   (e) the sparse (index, value) message C(d)  (Algorithm 1, upload line)
  *   (f) g <- g + C(d)                  EF21 estimator update (Algorithm 1 aggregate line; Eq. 6)
  *
+ * Beside it: the receiving side of a message and the model step (kimad_apply_packed, kimad_aggregate:
+ * Algorithm 1, server lines), and, through kimad_options.policy, Kimad without layer adaptivity
+ * (Section 3.1) and the error-axis reading of Algorithm 3.
+ *
  * Conventions
  *   - L layers of sizes n_l, concatenated in list order into one flat vector of N elements.
  *     Worker w's vector starts at element w * worker_stride of `grads` and of `state`.
  *   - "device" pointers are CUDA device memory of the current device; "host" pointers are
  *     ordinary host memory.  The library never allocates or frees device memory: scratch is
- *     the caller's (kimad_set_workspace).  All kernels go to the caller's stream.
+ *     the caller's (kimad_set_workspace).  All kernels are ordered on the caller's stream (one of them
+ *     runs on a stream of the context's own, forked from and joined to the caller's with events).
+ *     grads and state of a step must not overlap and must not change while the step is in flight: the
+ *     kernels re-read them instead of keeping a copy of grad - g.
  *   - TopK order inside a layer: larger |d| first (compared on the 31 magnitude bits, so +0
  *     and -0 tie), then lower index.  Inputs must be finite.
  *   - Size of a layer compressed at k: k * (4 + vb) bytes (u32 index + value of vb = 4 or 2
