@@ -65,7 +65,7 @@ __device__ __forceinline__ void sel_count_chunk(const DPlanes& dbuf, const Chunk
                                                 const Sel* __restrict__ sel, const LayerDesc* __restrict__ layers,
                                                 ChunkSel* __restrict__ csel, uint32_t* __restrict__ low_hist,
                                                 uint32_t* __restrict__ recount_n, uint2* __restrict__ recount_list,
-                                                uint32_t* s_hist, uint32_t* s_n, uint32_t* s_low) {
+                                                uint32_t* s_n, uint32_t* s_low) {
     const size_t wl = (size_t)w * L + ch.layer;
     const Sel s = sel[wl];
     ChunkSel* out = csel + (size_t)w * n_chunks + chunk_id;
@@ -83,8 +83,8 @@ __device__ __forceinline__ void sel_count_chunk(const DPlanes& dbuf, const Chunk
     const uint32_t lo = s.tau, width = 1u << s.shift;
     const uint32_t hshift = s.shift > 10 ? s.shift - 10 : 0; // the histogram has at most kLowBins bins
     __shared__ uint32_t s_gm[kThreads / 32]; // per warp: group bits of the half slice in work (zero between uses)
-    for (int i = threadIdx.x; i < kLowBins; i += kThreads) s_hist[i] = 0;
     if (threadIdx.x == 0) *s_n = 0;
+    uint32_t* gh = low_hist + wl * kLowBins; // the layer's in-interval histogram: few entries, counted in place
     if (threadIdx.x < kThreads / 32) s_gm[threadIdx.x] = 0;
     __syncthreads();
     const DView dd(dbuf, w, dstride, cv.a0);
@@ -100,7 +100,7 @@ __device__ __forceinline__ void sel_count_chunk(const DPlanes& dbuf, const Chunk
         auto visit = [&](uint32_t key) -> bool { // true: the key is not below the interval
             const uint32_t d1 = key - lo; // wraps to >= 2^31 for keys below the interval
             if (d1 < width) {
-                atomicAdd(&s_hist[d1 >> hshift], 1u);
+                atomicAdd(&gh[d1 >> hshift], 1u);
                 const uint32_t p = atomicAdd(s_n, 1u);
                 if (p < (uint32_t)kListCap) s_low[p] = (sl << 16) | d1;
             } else {
@@ -176,11 +176,6 @@ __device__ __forceinline__ void sel_count_chunk(const DPlanes& dbuf, const Chunk
     }
     __syncthreads();
     const uint32_t n_in = *s_n;
-    if (n_in) { // rare: publish this chunk's part of the layer's in-interval histogram
-        uint32_t* gh = low_hist + wl * kLowBins;
-        for (uint32_t i = threadIdx.x; i < (uint32_t)kLowBins; i += kThreads)
-            if (s_hist[i]) atomicAdd(&gh[i], s_hist[i]);
-    }
     if (threadIdx.x < min(n_in, (uint32_t)kListCap)) out->low[threadIdx.x] = s_low[threadIdx.x];
     if (threadIdx.x == 0) {
         if (n_in <= (uint32_t)kListCap) {
@@ -198,11 +193,10 @@ k_sel_count(DPlanes dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks, u
             uint32_t L, const Sel* __restrict__ sel, const LayerDesc* __restrict__ layers, ChunkSel* __restrict__ csel,
             uint32_t* __restrict__ low_hist, uint32_t* __restrict__ recount_n, uint2* __restrict__ recount_list) {
     pdl_wait();
-    __shared__ uint32_t s_hist[kLowBins];
     __shared__ uint32_t s_n;
     __shared__ uint32_t s_low[kListCap];
     sel_count_chunk(dbuf, chunks[blockIdx.x], blockIdx.y, blockIdx.x, n_chunks, dstride, L, sel, layers, csel, low_hist,
-                    recount_n, recount_list, s_hist, &s_n, s_low);
+                    recount_n, recount_list, &s_n, s_low);
 }
 
 // second round: only the chunks of the layers listed in r2
@@ -212,14 +206,13 @@ k_sel_count_r2(DPlanes dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks
                ChunkSel* __restrict__ csel, uint32_t* __restrict__ low_hist, uint32_t* __restrict__ recount_n,
                uint2* __restrict__ recount_list, const Round2* __restrict__ r2, const uint2* __restrict__ r2_chunks) {
     pdl_wait();
-    __shared__ uint32_t s_hist[kLowBins];
     __shared__ uint32_t s_n;
     __shared__ uint32_t s_low[kListCap];
     const uint32_t n = r2->n_chunks;
     for (uint32_t it = blockIdx.x; it < n; it += gridDim.x) {
         const uint2 e = r2_chunks[it];
         sel_count_chunk(dbuf, chunks[e.y], e.x, e.y, n_chunks, dstride, L, sel, layers, csel, low_hist, recount_n,
-                        recount_list, s_hist, &s_n, s_low);
+                        recount_list, &s_n, s_low);
     }
 }
 
