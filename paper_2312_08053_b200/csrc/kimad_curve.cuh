@@ -568,7 +568,9 @@ k_resolve_a(const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ r
                 if (lane >= (uint32_t)o) { ic += yc; is += ys; }
             }
             const uint32_t before = run_c + ic - c;
-            const double below = run_s + is - sv;
+            double ex_s = __shfl_up_sync(0xffffffffu, is, 1); // exclusive value from the left neighbour: no cancellation
+            if (lane == 0) ex_s = 0.0;
+            const double below = run_s + ex_s;
             if (c)
                 for (uint32_t j = 0; j < K; ++j) { // the bin where the running count passes n - k_j holds the threshold
                     const uint32_t dj = s_drop[j];

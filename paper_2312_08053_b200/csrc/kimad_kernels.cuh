@@ -90,7 +90,11 @@ __device__ __forceinline__ T block_excl_scan(T v, T* s_warp /* [NT / 32] */, T* 
         tot += t;
     }
     if (total) *total = tot;
-    return base + x - v;
+    // the lane's exclusive value is taken from its left neighbour, not as inclusive - own: a subtraction would
+    // cancel the small terms of a floating-point scan whose values span many orders of magnitude
+    T ex = __shfl_up_sync(0xffffffffu, x, 1);
+    if (lane == 0) ex = 0;
+    return base + ex;
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -277,3 +277,53 @@ def test_many_workers_with_different_budgets():
     res = r.compare_step(grads, state, bw, 1.0)
     st = res["forced"].status
     assert st[0] == ko.STATUS_INFEASIBLE and st[-1] == ko.STATUS_PLATEAU and np.count_nonzero(st == 0) > 30
+
+
+def test_huge_dynamic_range_in_a_tiny_layer():
+    """Magnitudes spread over 26 orders: the curve's partial sums must not lose their small terms (an exclusive scan
+    taken as inclusive minus own would cancel them)."""
+    rng = np.random.default_rng(1095)
+    sizes = [48, 3000, 70000]
+    grid = [0.02, 0.1, 0.3, 0.6, 0.9, 1.0]
+    N = sum(sizes)
+    x = (rng.standard_normal((3, N)) * np.exp(rng.uniform(-30, 30, (3, N)))).astype(np.float32)
+    r = Runner(sizes, 3, grid, 1000, 0)
+    grads = torch.from_numpy(x).cuda()
+    state = torch.from_numpy((rng.standard_normal((3, N)) * 0.1).astype(np.float32)).cuda()
+    r.compare_step(grads, state, [0.1 * 8 * N, 0.5 * 8 * N, 2.0 * 8 * N], 1.0)
+
+
+@pytest.mark.parametrize("seed", [11, 12, 13])
+def test_randomized_configurations(seed):
+    """Random layer lists, grids, worker counts, strides, value types, cell counts and value patterns (ties, denormals,
+    mostly zeros, huge dynamic range, all-equal magnitudes), two steps each, all compared with the oracle."""
+    for it in range(25):
+        rng = np.random.default_rng(seed * 1000 + it)
+        L = int(rng.integers(1, 7))
+        sizes = [int(v) for v in np.exp(rng.uniform(np.log(1), np.log(400000), L)).astype(int) + 1]
+        grid = np.unique(np.round(np.sort(rng.uniform(0.0005, 1.0, int(rng.integers(1, 20)))), 6))
+        if rng.random() < 0.5:
+            grid[-1] = 1.0
+        W, vd = int(rng.integers(1, 4)), int(rng.integers(0, 2))
+        D = max(int(rng.choice([L, 50, 1000, 4000])), L)
+        N = sum(sizes)
+        stride = N + int(rng.integers(0, 9))
+        r = Runner(sizes, W, list(grid), D, vd, stride=stride)
+        kind = int(rng.integers(0, 6))
+        x = rng.standard_normal((W, stride)).astype(np.float32)
+        if kind == 1:
+            x = np.round(x * 4) / 4
+        elif kind == 2:
+            x *= np.float32(1e-40)
+        elif kind == 3:
+            x[rng.random(x.shape) < 0.9] = 0
+        elif kind == 4:
+            x = (x * np.exp(rng.uniform(-30, 30, x.shape))).astype(np.float32)
+        elif kind == 5:
+            x = np.sign(x) * np.float32(0.5)
+        grads = torch.from_numpy(x).cuda()
+        state = torch.from_numpy((rng.standard_normal((W, stride)) * (0.0 if kind in (2, 5) else 0.1)).astype(np.float32)).cuda()
+        for rep in range(2):
+            frac = float(np.exp(rng.uniform(np.log(0.002), np.log(1.5))))
+            bw = [frac * (8 if vd == 0 else 6) * N * float(rng.uniform(0.5, 1.5)) for _ in range(W)]
+            r.compare_step(grads, state, bw, 1.0, check_inject=bool(rng.integers(0, 2)))
