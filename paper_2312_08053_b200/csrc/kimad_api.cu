@@ -175,7 +175,7 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
 
     const Layout& y = c->lay;
     // the upper halves of d, u16 [W][dstride]; exact values are recomputed from grads and state
-    const DPlanes dbuf{c->at<uint16_t>(y.dbuf), grads, state, c->stride};
+    const DSource dbuf{c->at<uint16_t>(y.dbuf), grads, state, c->stride};
     const Chunk* chunks = c->at<Chunk>(y.chunks);
     const LayerDesc* layers = c->at<LayerDesc>(y.layers);
     const uint64_t* ktab = c->at<uint64_t>(y.ktab);

@@ -703,7 +703,7 @@ k_tiny_exact(const float* __restrict__ grads, const float* __restrict__ state, u
 // exact radix path over the handed-over chunks (global atomics: the list is short or empty)
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kThreads)
-k_fb_hist1(DPlanes dbuf, const Chunk* __restrict__ chunks, uint64_t dstride, uint32_t L,
+k_fb_hist1(DSource dbuf, const Chunk* __restrict__ chunks, uint64_t dstride, uint32_t L,
            const FbList* __restrict__ fb, const uint2* __restrict__ fb_chunks, uint32_t* __restrict__ g_cnt,
            unsigned long long* __restrict__ g_ss, uint32_t* __restrict__ flags) {
     pdl_wait();
@@ -738,7 +738,7 @@ k_fb_hist1(DPlanes dbuf, const Chunk* __restrict__ chunks, uint64_t dstride, uin
 
 template <int LEVEL>
 __global__ void __launch_bounds__(kThreads)
-k_fb_hist23(DPlanes dbuf, const Chunk* __restrict__ chunks, uint64_t dstride, uint32_t L, uint32_t K,
+k_fb_hist23(DSource dbuf, const Chunk* __restrict__ chunks, uint64_t dstride, uint32_t L, uint32_t K,
             const FbList* __restrict__ fb, const uint2* __restrict__ fb_chunks, const SlotTab* __restrict__ slots,
             uint32_t* __restrict__ g_cnt, unsigned long long* __restrict__ g_ss) {
     pdl_wait();

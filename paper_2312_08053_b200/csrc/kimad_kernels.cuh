@@ -47,7 +47,7 @@ struct ChunkView {
 // value only for the few keys that share an upper half with the threshold; whoever needs an exact d recomputes
 // the one subtraction from the inputs (the estimator is not written before the write sweep, and there every
 // element is read before it is updated).
-struct DPlanes {
+struct DSource {
     uint16_t* hi;
     const float* grads;
     const float* state;
@@ -57,7 +57,7 @@ struct DView { // one worker's data at a chunk's aligned start
     const uint16_t* hi;
     const float* gr;
     const float* st;
-    __device__ __forceinline__ DView(const DPlanes& p, uint32_t w, uint64_t dstride, uint64_t a0)
+    __device__ __forceinline__ DView(const DSource& p, uint32_t w, uint64_t dstride, uint64_t a0)
         : hi(p.hi + (size_t)w * dstride + a0), gr(p.grads + (size_t)w * p.stride + a0), st(p.state + (size_t)w * p.stride + a0) {}
     __device__ __forceinline__ float at(uint32_t e) const { return __fsub_rn(gr[e], st[e]); }
 };

@@ -60,7 +60,7 @@ constexpr int kSortCap = 4096;
 
 // ------------------------------------------------------------------------------------------------
 // Counting sweep of one chunk: warp w takes the slices w and w + 8.
-__device__ __forceinline__ void sel_count_chunk(const DPlanes& dbuf, const Chunk& ch, uint32_t w,
+__device__ __forceinline__ void sel_count_chunk(const DSource& dbuf, const Chunk& ch, uint32_t w,
                                                 uint32_t chunk_id, uint32_t n_chunks, uint64_t dstride, uint32_t L,
                                                 const Sel* __restrict__ sel, const LayerDesc* __restrict__ layers,
                                                 ChunkSel* __restrict__ csel, uint32_t* __restrict__ low_hist,
@@ -189,7 +189,7 @@ __device__ __forceinline__ void sel_count_chunk(const DPlanes& dbuf, const Chunk
 }
 
 __global__ void __launch_bounds__(kThreads)
-k_sel_count(DPlanes dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks, uint64_t dstride,
+k_sel_count(DSource dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks, uint64_t dstride,
             uint32_t L, const Sel* __restrict__ sel, const LayerDesc* __restrict__ layers, ChunkSel* __restrict__ csel,
             uint32_t* __restrict__ low_hist, uint32_t* __restrict__ recount_n, uint2* __restrict__ recount_list) {
     pdl_wait();
@@ -201,7 +201,7 @@ k_sel_count(DPlanes dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks, u
 
 // second round: only the chunks of the layers listed in r2
 __global__ void __launch_bounds__(kThreads)
-k_sel_count_r2(DPlanes dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks, uint64_t dstride,
+k_sel_count_r2(DSource dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks, uint64_t dstride,
                uint32_t L, const Sel* __restrict__ sel, const LayerDesc* __restrict__ layers,
                ChunkSel* __restrict__ csel, uint32_t* __restrict__ low_hist, uint32_t* __restrict__ recount_n,
                uint2* __restrict__ recount_list, const Round2* __restrict__ r2, const uint2* __restrict__ r2_chunks) {
@@ -337,7 +337,7 @@ k_sel_resolve_r2(uint32_t L, const LayerDesc* __restrict__ layers, uint32_t n_ch
 
 // Exact per-slice (gt, eq) of the chunks whose list overflowed: warp w recounts the slices w and w + 8.
 __global__ void __launch_bounds__(kThreads)
-k_sel_recount(DPlanes dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks, uint64_t dstride,
+k_sel_recount(DSource dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks, uint64_t dstride,
               uint32_t L, const Sel* __restrict__ sel, const uint32_t* __restrict__ recount_n,
               const uint2* __restrict__ recount_list, ChunkSel* __restrict__ csel) {
     pdl_wait();
