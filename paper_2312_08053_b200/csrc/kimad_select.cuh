@@ -365,6 +365,10 @@ k_sel_recount(DSource dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks,
             }
             if (lane == 0) { out->above[sl] = (uint16_t)gt; out->eq[sl] = (uint16_t)eq; }
         }
+        // The recount is authoritative.  A chunk listed in the first round may have been counted again in the
+        // second (narrowed interval) and then own a fresh in-interval list; k_sel_slices must not add that list
+        // on top of the exact counts written here.
+        if (threadIdx.x == 0) out->n_in = kListOverflow;
     }
 }
 

@@ -327,3 +327,29 @@ def test_randomized_configurations(seed):
             frac = float(np.exp(rng.uniform(np.log(0.002), np.log(1.5))))
             bw = [frac * (8 if vd == 0 else 6) * N * float(rng.uniform(0.5, 1.5)) for _ in range(W)]
             r.compare_step(grads, state, bw, 1.0, check_inject=bool(rng.integers(0, 2)))
+
+
+@pytest.mark.parametrize("seed", [3, 4])
+def test_concentrated_magnitudes_second_select_round(seed):
+    """Layers whose |d| sits within a third of an octave: the bin that holds a threshold is wide (many keys) and
+    full, so the select stage overflows its per-chunk lists, narrows the interval with the coarse histogram and
+    counts a second time.  Duplicates of the k-th value are planted in different chunks, so that kept ties span
+    chunks and any double count of an entry shifts the packed positions."""
+    rng = np.random.default_rng(seed)
+    sizes = [20000, 300007, 1000003, 32768, 150001, 2000000]
+    grid = [0.01, 0.1, 0.3, 0.5, 0.8, 1.0]
+    N = sum(sizes)
+    parts = []
+    for n in sizes:
+        a = np.float32(10.0 ** rng.uniform(-3, 0))
+        v = (a * rng.uniform(1.0, 1.3, n)).astype(np.float32)
+        for ratio in grid[:-1]:  # plant ties at every candidate's threshold value
+            kth = np.partition(v, n - int(np.ceil(ratio * n)))[n - int(np.ceil(ratio * n))]
+            v[rng.choice(n, 12, replace=False)] = kth
+        parts.append(v * np.where(rng.random(n) < 0.5, -1, 1).astype(np.float32))
+    x = np.concatenate(parts)[None, :]
+    r = Runner(sizes, 1, grid)
+    grads = torch.from_numpy(x).cuda()
+    state = torch.zeros_like(grads)
+    for frac in (0.05, 0.25, 0.45, 0.7):
+        r.compare_step(grads, state.clone(), [frac * 8 * N], 1.0)
