@@ -380,7 +380,7 @@ int kimad_create(kimad_ctx** out, const uint64_t* layer_sizes, uint32_t n_layers
         c->dstride = (N + 3) / 4 * 4;
         // shared-memory plan of the DP kernel
         const size_t Kp = (c->K + 3) & ~(size_t)3;
-        const size_t dp_base = ((size_t)2 * (2 * c->D + 3) + c->L) * 4;
+        const size_t dp_base = ((size_t)2 * (2 * c->D + 3) + c->L) * 4 + 16; // + alignment slack of the candidate tables
         const size_t tab_all = (size_t)c->L * (Kp * 8 + 4), tab_one = Kp * 8 + 4;
         c->dp_plan.pd_nibble = c->K <= 16 ? 1u : 0u;
         c->dp_plan.pd_row_bytes = c->dp_plan.pd_nibble ? (c->D + 2) / 2 : (c->D + 1);

@@ -337,6 +337,10 @@ struct DpBudgets { uint64_t c[kDpWorkersPerLaunch]; };
 
 constexpr int kDpThreads = 512;
 constexpr int kDpCells = 2; // budget cells per thread
+constexpr int kDpMaxChain = 16;                // layers carried through one barrier interval
+constexpr uint32_t kDpSameCells = 0x80000000u; // flags kept beside a layer's usable-candidate count
+constexpr uint32_t kDpChain = 0x40000000u;     // same cells, finite errors that do not increase with j
+constexpr uint32_t kDpInner = 0x20000000u;     // layer of a chained run that is not the run's last
 
 // Shared-memory plan of k_dp (host computes the same sizes):
 //   two rows of (D+2) +inf followed by D+1 values, f32 | j[L] u32 | usable[L or 1] u32 |
@@ -375,7 +379,8 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
     uint32_t* s_j = reinterpret_cast<uint32_t*>(rows + 2 * rowp); // [L]
     const uint32_t ltab = plan.tab_in_smem ? L : 1;
     uint32_t* s_usable = s_j + L;                                 // [ltab] candidates that fit into D cells
-    uint32_t* s_units = s_usable + ltab;                          // [ltab * Kp]
+    uint32_t* s_units = s_usable + ltab;                          // [ltab * Kp], 16-byte aligned (read four at a time)
+    s_units += (4u - ((2u * rowp + L + ltab) & 3u)) & 3u;
     float* s_err = reinterpret_cast<float*>(s_units + ltab * Kp); // [ltab * Kp]
     uint8_t* pd = plan.pd_in_smem ? reinterpret_cast<uint8_t*>(s_err + ltab * Kp)
                                   : pd_global + (size_t)w * L * plan.pd_row_bytes;
@@ -509,11 +514,14 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
             auto count_usable = [&](uint32_t slot_l) { // sizes ascend with j, so the usable candidates come first
                 uint32_t nu = 0;
                 bool same = true; // all usable candidates take the same number of cells (small layers under a coarse cell)
+                bool mono = true; // ... and their errors are finite and do not increase with j
                 while (nu < K && s_units[slot_l * Kp + nu] <= D) {
                     same &= s_units[slot_l * Kp + nu] == s_units[slot_l * Kp];
+                    const float e = s_err[slot_l * Kp + nu];
+                    mono &= e < kInf && e >= 0.f && (nu == 0 || e <= s_err[slot_l * Kp + nu - 1]);
                     ++nu;
                 }
-                s_usable[slot_l] = nu | (same && nu > 1 ? 0x80000000u : 0u);
+                s_usable[slot_l] = nu | (same && nu > 1 ? kDpSameCells : 0u) | (same && nu >= 1 && mono ? kDpChain : 0u);
             };
             if (plan.tab_in_smem) {
                 for (uint32_t i = threadIdx.x; i < L * Kp; i += blockDim.x) load_tab(i / Kp, i % Kp, i / Kp);
@@ -531,11 +539,77 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
                     if (threadIdx.x == 0) count_usable(0);
                     __syncthreads();
                 }
+                if (plan.tab_in_smem && (s_usable[l] & kDpChain)) {
+                    // A run of consecutive layers whose usable candidates all take the same number of cells (small
+                    // layers under a coarse cell).  Such a layer shifts the row by its cells and adds, per cell, the
+                    // smallest fl(p + e_j); with e non-increasing in j the candidates attaining it are the last ones,
+                    // and the first of them (the one a strict `<` over ascending j keeps) is found by bisection (when
+                    // the running sum dwarfs the layer's errors they all tie and candidate 0 is kept).  The shifts of
+                    // a run add up, so a thread carries its cells through the whole run by itself: one barrier per
+                    // run, and the back-pointers of the run's layers are stored at the cell the run ENDS in (the
+                    // backtracking below reads them there).
+                    uint32_t m = 1, U = s_units[l * Kp];
+                    while (l + m < L && m < (uint32_t)kDpMaxChain && (s_usable[l + m] & kDpChain)) { U += s_units[(l + m) * Kp]; ++m; }
+                    float v[kDpCells];
+                    for (uint32_t bb = 0; bb < row; bb += kDpCells * blockDim.x) {
+                        const uint32_t b0 = bb + threadIdx.x;
+#pragma unroll
+                        for (int q = 0; q < kDpCells; ++q) {
+                            const uint32_t b = b0 + q * blockDim.x;
+                            v[q] = (b < row && b >= U) ? prev[b - U] : kInf;
+                        }
+                        for (uint32_t i = 0; i < m; ++i) {
+                            const float* er = s_err + (l + i) * Kp;
+                            const uint32_t nu = s_usable[l + i] & 0xffffu;
+                            const float emin = er[nu - 1];
+                            uint8_t* pdl = pd + (size_t)(l + i) * plan.pd_row_bytes;
+                            // first j with fl(p + e_j) == fl(p + e_min): bisection in a fixed number of steps, the
+                            // thread's cells side by side (p = +inf compares equal everywhere and ends at j = 0, the
+                            // value an untouched cell holds)
+                            const int steps = nu > 1 ? 32 - __clz(nu - 1) : 0;
+                            float t[kDpCells];
+                            uint32_t lo[kDpCells], hi[kDpCells];
+#pragma unroll
+                            for (int q = 0; q < kDpCells; ++q) { t[q] = __fadd_rn(v[q], emin); lo[q] = 0; hi[q] = nu - 1; }
+                            for (int s = 0; s < steps; ++s) {
+#pragma unroll
+                                for (int q = 0; q < kDpCells; ++q) {
+                                    const uint32_t mid = (lo[q] + hi[q]) >> 1;
+                                    const bool eq = __fadd_rn(v[q], er[mid]) == t[q];
+                                    hi[q] = eq ? mid : hi[q];
+                                    lo[q] = eq ? lo[q] : min(mid + 1, hi[q]);
+                                }
+                            }
+#pragma unroll
+                            for (int q = 0; q < kDpCells; ++q) {
+                                const uint32_t b = b0 + q * blockDim.x;
+                                const uint32_t bj = lo[q];
+                                v[q] = t[q];
+                                if (plan.pd_nibble) {
+                                    const uint32_t nb = __shfl_down_sync(0xffffffffu, bj, 1);
+                                    if (!(threadIdx.x & 1) && b < row) pdl[b >> 1] = (uint8_t)(bj | (nb << 4));
+                                } else if (b < row) {
+                                    pdl[b] = (uint8_t)bj;
+                                }
+                            }
+                        }
+#pragma unroll
+                        for (int q = 0; q < kDpCells; ++q) {
+                            const uint32_t b = b0 + q * blockDim.x;
+                            if (b < row) cur[b] = v[q];
+                        }
+                    }
+                    if (threadIdx.x == 0)
+                        for (uint32_t i = 0; i + 1 < m; ++i) s_usable[l + i] |= kDpInner; // not the run's last layer
+                    float* sw = prev; prev = cur; cur = sw;
+                    l += m - 1;
+                    continue;
+                }
                 const uint32_t sl = plan.tab_in_smem ? l : 0;
                 const uint32_t* un = s_units + sl * Kp;
                 const float* er = s_err + sl * Kp;
                 const uint32_t nu = s_usable[sl] & 0xffffu;
-                const bool same_cells = s_usable[sl] >> 31;
+                const bool same_cells = (s_usable[sl] & kDpSameCells) != 0;
                 uint8_t* pdl = pd + (size_t)l * plan.pd_row_bytes;
                 // each thread owns the cells t, t + T, ... (consecutive threads read consecutive words of
                 // prev[]: no bank conflicts); candidates four at a time so that the prev[] reads of a batch are
@@ -561,10 +635,11 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
                         }
                     } else
                     for (uint32_t j0 = 0; j0 < nu; j0 += 4) {
-                        uint32_t u[4];
-                        float e[4], p[4][kDpCells];
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) { u[i] = un[j0 + i]; e[i] = er[j0 + i]; }
+                        float p[4][kDpCells];
+                        const uint4 u4 = *reinterpret_cast<const uint4*>(un + j0);
+                        const float4 e4 = *reinterpret_cast<const float4*>(er + j0);
+                        const uint32_t u[4] = {u4.x, u4.y, u4.z, u4.w};
+                        const float e[4] = {e4.x, e4.y, e4.z, e4.w};
 #pragma unroll
                         for (int i = 0; i < 4; ++i)
 #pragma unroll
@@ -621,10 +696,11 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
                     s_status = KIMAD_STATUS_INFEASIBLE;
                 } else {
                     s_status = KIMAD_OK;
-                    uint32_t b = bb;
+                    uint32_t b = bb, b_at = bb;
                     for (uint32_t l = L; l-- > 0;) { // walk the back-pointers
                         const uint8_t* pdl = pd + (size_t)l * plan.pd_row_bytes;
-                        const uint32_t j = plan.pd_nibble ? ((pdl[b >> 1] >> (4 * (b & 1))) & 15u) : pdl[b];
+                        if (!plan.tab_in_smem || !(s_usable[l] & kDpInner)) b_at = b; // inner layers of a run: the run's end cell
+                        const uint32_t j = plan.pd_nibble ? ((pdl[b_at >> 1] >> (4 * (b_at & 1))) & 15u) : pdl[b_at];
                         s_j[l] = j;
                         b -= plan.tab_in_smem ? s_units[l * Kp + j]
                                               : (uint32_t)budget_cells(ktab[(size_t)l * K + j] * bpe, D, c);
