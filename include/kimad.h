@@ -197,6 +197,21 @@ int kimad_apply_packed(const kimad_ctx* ctx, const kimad_packed* msg, float* est
 int kimad_aggregate(float* x_dev, const float* est_dev, uint64_t stride, uint32_t n_workers, uint64_t n,
                     const float* weights, float gamma, void* cuda_stream);
 
+/* ---- Bandwidth monitor (Section 2.4: every device estimates its bandwidth B_m^k from what it observed; the
+ * paper gives no formula, this is ours).  Host-only, no GPU.  The caller reports every finished transfer (the
+ * upload of a step's message: its bytes and how long it took); the estimate is the throughput over the last
+ * `window` transfers, sum of bytes / sum of seconds (long transfers weigh more), smoothed exponentially:
+ * est <- alpha * windowed + (1 - alpha) * est (alpha = 1: no smoothing; the first observation sets est).
+ * The estimate, in bytes per second, is what kimad_step takes as bandwidth_bytes_per_s.
+ *   kimad_monitor_create: window in [1, 65536], alpha in (0, 1]; errors INVALID_ARG, NOMEM.
+ *   kimad_monitor_observe: seconds > 0 and finite, else INVALID_ARG (nothing recorded).
+ *   kimad_monitor_estimate: 0.0 before the first observation. */
+typedef struct kimad_monitor kimad_monitor;
+int kimad_monitor_create(kimad_monitor** out, uint32_t window, double alpha);
+void kimad_monitor_destroy(kimad_monitor* m);
+int kimad_monitor_observe(kimad_monitor* m, uint64_t bytes, double seconds);
+double kimad_monitor_estimate(const kimad_monitor* m);
+
 /* Static tables (host-only calls).  host_k_table: u64 [L][K] candidates k_{l,j}. */
 int kimad_get_k_table(const kimad_ctx* ctx, uint64_t* host_k_table);
 /* Budget arithmetic of one worker exactly as the device applies it: c = floor(B * t); cells

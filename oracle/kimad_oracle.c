@@ -31,6 +31,12 @@
  *   O12 the other reading of Algorithm 3: the knapsack axis is the discretised ERROR (its header:
  *       "compression budget E_max", "discretization step E_max / D", "discretized L2"), the value the
  *       size; the answer is the lowest error level whose smallest size fits c
+ *   O9b Kimad as Section 3.1 states it: ONE ratio for all layers, SIZED TO THE BUDGET (not taken from
+ *       a grid): the largest ratio whose total size fits c.  With one layer spanning the model this is
+ *       the whole-model TopK of Section 4.3 at K = floor(c / (4 + vb))
+ *   O13 sizes with a dense fallback (Eq. 3 calls b_ij "the size of layer i compressed with c^j" and
+ *       fixes no encoding): a candidate whose sparse size reaches the layer's dense size is sent
+ *       densely -- all n values, no indices -- and then has no compression error
  *
  * Floating point: the element-wise operations (O1, O8, the DP adds) are single
  * IEEE binary32 operations in a fixed order, because the compared results must be
@@ -46,7 +52,9 @@
  * ||d - C(d)||^2 = err and sum(bytes) <= c only.  O9: brute force over the grid;
  * O10: the receiver's estimator equals the sender's after every message; O11:
  * numpy float32 re-computation and the closed form for equal estimators.  O12: exhaustive
- * enumeration of the discretised objective.
+ * enumeration of the discretised objective.  O9b: exact rational arithmetic over every breakpoint
+ * of the step function r -> sum_l floor(r n_l), hand values.  O13: hand-computed sizes on the
+ * three-layer example, exhaustive enumeration of the assignments with the modified tables.
  *
  * Build: gcc -O2 -ffp-contract=off -fopenmp -shared -fPIC (see kimad_oracle.py).
  */
@@ -451,6 +459,82 @@ int ko_dp_error_axis(const float* err /* [L][K] */, const uint64_t* k_table /* [
     return status;
 }
 
+/* O9b: Kimad as Section 3.1 states it: the same ratio on all layers, sized to the budget.  The ratio
+ * is a multiple of 2^-32: r = q / 2^32 with q in [0, 2^32], and layer l keeps
+ *     k_l(q) = min(n_l, max(1, floor(q * n_l / 2^32)))      (at least one entry: Omega = {TopK : K > 0})
+ * entries (exact integer arithmetic: n_l < 2^32, so the product fits 64 bits).  q is the LARGEST value with
+ * sum_l k_l(q) <= entries, where entries = floor(c / (4 + vb)) is what the budget pays for.  k_l(q) does not
+ * decrease with q, so q is found by bisection.
+ *   entries < L  : not even one entry per layer fits -> q = 0, every k_l = 1, KO_STATUS_INFEASIBLE
+ *   entries >= N : q = 2^32, every k_l = n_l, KO_STATUS_PLATEAU
+ * With L = 1 this gives k = min(N, max(1, entries)): TopK over the whole model at K = floor(c / (4 + vb))
+ * ("select K with the whole model information", Section 4.3), because floor(q N / 2^32) takes every value
+ * 0..N as q runs over 0..2^32. */
+static uint64_t ko_fit_sum(const uint64_t* layer_sizes, uint32_t L, uint64_t q, uint64_t* k_out) {
+    uint64_t sum = 0;
+    for (uint32_t l = 0; l < L; ++l) {
+        uint64_t n = layer_sizes[l];
+        uint64_t k = q >= 4294967296ull ? n : (q * n) >> 32;
+        if (k < 1) k = 1;
+        if (k > n) k = n;
+        if (k_out) k_out[l] = k;
+        sum += k;
+    }
+    return sum;
+}
+
+int ko_fit_ratio(const uint64_t* layer_sizes, uint32_t L, uint64_t entries, uint64_t* q_out, uint64_t* k_out /* [L] */) {
+    if (!layer_sizes || L == 0) return KO_ERR_ARG;
+    uint64_t N = 0;
+    for (uint32_t l = 0; l < L; ++l) {
+        if (layer_sizes[l] == 0 || layer_sizes[l] > 0xffffffffull) return KO_ERR_ARG;
+        N += layer_sizes[l];
+    }
+    uint64_t q;
+    int status = KO_OK;
+    if (entries < (uint64_t)L) {
+        q = 0;
+        status = KO_STATUS_INFEASIBLE;
+    } else if (entries >= N) {
+        q = 4294967296ull;
+        status = KO_STATUS_PLATEAU;
+    } else {
+        uint64_t lo = 0, hi = 4294967296ull; /* sum(lo) <= entries < sum(hi) */
+        while (hi - lo > 1) {
+            uint64_t mid = lo + (hi - lo) / 2;
+            if (ko_fit_sum(layer_sizes, L, mid, NULL) <= entries) lo = mid; else hi = mid;
+        }
+        q = lo;
+    }
+    ko_fit_sum(layer_sizes, L, q, k_out);
+    if (q_out) *q_out = q;
+    return status;
+}
+
+/* O13: size and effect of candidate k of a layer of n elements under the two cost models.
+ *   cost_model 0: bytes = k (4 + vb): u32 index + value for every kept entry (also at k = n).
+ *   cost_model 1: if k (4 + vb) >= vb n the layer is sent DENSELY: all n values in order, no indices,
+ *                 bytes = vb n; the candidate then keeps every entry (k_eff = n) and its error is 0.
+ *                 Otherwise as cost model 0. */
+void ko_candidate(uint64_t n, uint64_t k, uint32_t value_dtype, uint32_t cost_model, uint64_t* bytes, uint64_t* k_eff,
+                  int* dense) {
+    const uint64_t vb = value_dtype == 0 ? 4 : 2, bpe = 4 + vb;
+    const int d = cost_model == 1 && k * bpe >= vb * n;
+    if (bytes) *bytes = d ? vb * n : k * bpe;
+    if (k_eff) *k_eff = d ? n : k;
+    if (dense) *dense = d;
+}
+
+/* O5 on a table of sizes: cells_{l,j} = ceil(bytes_{l,j} * D / c); same return values as ko_units. */
+int ko_units_from_bytes(const uint64_t* bytes_tab, uint32_t L, uint32_t K, uint64_t c, uint32_t D, uint64_t* units_out) {
+    uint64_t full = 0;
+    for (uint32_t l = 0; l < L; ++l) full += bytes_tab[(size_t)l * K + (K - 1)];
+    if (c >= full) return KO_STATUS_PLATEAU;
+    if (c == 0) return KO_STATUS_INFEASIBLE;
+    for (size_t i = 0; i < (size_t)L * K; ++i) units_out[i] = (bytes_tab[i] * (uint64_t)D + c - 1) / c;
+    return KO_OK;
+}
+
 /* The whole pass (O1..O8) for W workers.  Layout:
  *   grads, state : [W][stride] binary32, layers concatenated in list order (stride >= N)
  *   err/tau/keep_eq out : [W][L][K];  j_out/k_out : [W][L]
@@ -458,32 +542,50 @@ int ko_dp_error_axis(const float* err /* [L][K] */, const uint64_t* k_table /* [
  *   offs_out : [W][L+1] running sum of k_l
  * state is updated in place.  When inject_err != NULL the DP consumes that [W][L][K] table
  * instead of the curves computed here (the curves are still computed and returned).
- * policy 0: layer-adaptive search O6 (Kimad+); policy 1: one ratio for all layers O9 (Kimad);
- * policy 2: layer-adaptive search on the error axis O12. */
-int ko_step_policy(uint32_t policy, const uint64_t* layer_sizes, uint32_t L, uint32_t W, const double* ratios, uint32_t K, uint32_t D,
+ * policy 0: layer-adaptive search O6 (Kimad+); policy 1: one ratio of the grid for all layers O9;
+ * policy 2: layer-adaptive search on the error axis O12; policy 3: one ratio sized to the budget O9b
+ * (K must be 1: err/tau/keep_eq then describe the fitted k of every layer).  cost_model: O13 (0 or 1;
+ * 1 only with policies 0 and 1); dense_out [W][L]: 1 where the chosen candidate is sent densely. */
+int ko_step_ex(uint32_t policy, uint32_t cost_model, const uint64_t* layer_sizes, uint32_t L, uint32_t W, const double* ratios, uint32_t K, uint32_t D,
             uint32_t value_dtype, uint64_t stride, const float* grads, float* state,
             const double* bandwidth_bytes_per_s, double t_target_s, const float* inject_err, float* err_out,
             uint32_t* tau_out, uint32_t* keep_eq_out, uint32_t* j_out, uint32_t* k_out, uint32_t* idx_out,
-            void* val_out, uint64_t cap, uint64_t* offs_out, ko_stats* stats_out) {
+            void* val_out, uint64_t cap, uint64_t* offs_out, ko_stats* stats_out, uint32_t* dense_out /* [W][L] or NULL */) {
     if (!layer_sizes || !ratios || !grads || !state || !bandwidth_bytes_per_s || L == 0 || W == 0 || K == 0 ||
-        value_dtype > 1 || policy > 2)
+        value_dtype > 1 || policy > 3 || cost_model > 1)
         return KO_ERR_ARG;
+    if (policy == 3 && (K != 1 || cost_model != 0)) return KO_ERR_ARG; /* the fitted ratio is the only candidate */
+    if (policy == 2 && cost_model != 0) return KO_ERR_ARG;
     uint64_t N = 0;
     for (uint32_t l = 0; l < L; ++l) N += layer_sizes[l];
     if (stride < N) return KO_ERR_ARG;
-    uint64_t* ktab = (uint64_t*)malloc((size_t)L * K * sizeof(uint64_t));
+    /* the candidate table is per worker: policies 0..2 fill every worker's copy from the ratio grid, policy 3
+     * from the ratio fitted to that worker's budget */
+    uint64_t* ktab = (uint64_t*)malloc((size_t)W * L * K * sizeof(uint64_t));
+    uint64_t* keff = (uint64_t*)malloc((size_t)W * L * sizeof(uint64_t)); /* entries actually kept per layer */
     uint64_t* loff = (uint64_t*)malloc(((size_t)L + 1) * sizeof(uint64_t));
     float* err = (float*)malloc((size_t)W * L * K * sizeof(float));
     uint32_t* jsel = (uint32_t*)malloc((size_t)W * L * sizeof(uint32_t));
     ko_stats* st = (ko_stats*)malloc((size_t)W * sizeof(ko_stats));
     float* d = (float*)malloc((size_t)W * (N ? N : 1) * sizeof(float));
+    int* fit_status = (int*)calloc(W, sizeof(int));
     int rc = KO_OK;
     int fail = 0;
     const uint64_t bpe = value_dtype == 0 ? 8 : 6; /* bytes per kept entry: u32 index + value */
     const size_t vsz = value_dtype == 0 ? 4 : 2;
-    if (!ktab || !loff || !err || !jsel || !st || !d) { rc = KO_ERR_NOMEM; goto done; }
-    rc = ko_k_table(layer_sizes, L, ratios, K, ktab);
-    if (rc != KO_OK) goto done;
+    if (!ktab || !keff || !loff || !err || !jsel || !st || !d || !fit_status) { rc = KO_ERR_NOMEM; goto done; }
+    for (uint32_t w = 0; w < W; ++w) {
+        if (policy == 3) {
+            uint64_t c = ko_budget_bytes(bandwidth_bytes_per_s[w], t_target_s);
+            rc = ko_fit_ratio(layer_sizes, L, c / bpe, NULL, ktab + (size_t)w * L);
+            if (rc < 0) goto done;
+            fit_status[w] = rc;
+            rc = KO_OK;
+        } else {
+            rc = ko_k_table(layer_sizes, L, ratios, K, ktab + (size_t)w * L * K);
+            if (rc != KO_OK) goto done;
+        }
+    }
     loff[0] = 0;
     for (uint32_t l = 0; l < L; ++l) loff[l + 1] = loff[l] + layer_sizes[l];
 
@@ -495,7 +597,7 @@ int ko_step_policy(uint32_t policy, const uint64_t* layer_sizes, uint32_t L, uin
             float* dl = d + (size_t)w * N + loff[l];
             ko_diff(grads + (size_t)w * stride + loff[l], state + (size_t)w * stride + loff[l], dl, n);
             size_t o = ((size_t)w * L + l) * K;
-            int r = ko_layer_curve(dl, n, ktab + (size_t)l * K, K, err + o, tau_out ? tau_out + o : NULL,
+            int r = ko_layer_curve(dl, n, ktab + ((size_t)w * L + l) * K, K, err + o, tau_out ? tau_out + o : NULL,
                                    keep_eq_out ? keep_eq_out + o : NULL, NULL, NULL);
             if (r != KO_OK) {
 #pragma omp atomic write
@@ -507,40 +609,66 @@ int ko_step_policy(uint32_t policy, const uint64_t* layer_sizes, uint32_t L, uin
 
     /* O5 + O6 per worker */
     for (uint32_t w = 0; w < W; ++w) {
-        const float* e = (inject_err ? inject_err : err) + (size_t)w * L * K;
+        const float* e_in = (inject_err ? inject_err : err) + (size_t)w * L * K;
+        const uint64_t* kt = ktab + (size_t)w * L * K;
         uint64_t c = ko_budget_bytes(bandwidth_bytes_per_s[w], t_target_s);
         uint64_t* units = (uint64_t*)malloc((size_t)L * K * sizeof(uint64_t));
-        if (!units) { rc = KO_ERR_NOMEM; goto done; }
-        int s = ko_units(ktab, L, K, value_dtype, c, D, units);
+        uint64_t* bytes = (uint64_t*)malloc((size_t)L * K * sizeof(uint64_t));
+        uint64_t* kk = (uint64_t*)malloc((size_t)L * K * sizeof(uint64_t));
+        float* e = (float*)malloc((size_t)L * K * sizeof(float));
+        int* dense = (int*)malloc((size_t)L * K * sizeof(int));
+        if (!units || !bytes || !kk || !e || !dense) { free(units); free(bytes); free(kk); free(e); free(dense); rc = KO_ERR_NOMEM; goto done; }
+        /* O13: what every candidate costs, keeps and loses under the cost model */
+        for (uint32_t l = 0; l < L; ++l)
+            for (uint32_t j = 0; j < K; ++j) {
+                size_t i = (size_t)l * K + j;
+                ko_candidate(layer_sizes[l], kt[i], value_dtype, cost_model, &bytes[i], &kk[i], &dense[i]);
+                e[i] = dense[i] ? 0.0f : e_in[i];
+            }
         uint32_t* js = jsel + (size_t)w * L;
-        if (policy == 1) {
-            uint32_t ju = 0;
-            s = ko_uniform(ktab, L, K, value_dtype, c, &ju);
-            for (uint32_t l = 0; l < L; ++l) js[l] = ju;
-        } else if (policy == 2) {
-            s = ko_dp_error_axis(e, ktab, L, K, D, value_dtype, c, js, NULL);
-            if (s < 0) { free(units); rc = s; goto done; }
-        } else if (s == KO_STATUS_PLATEAU) {
-            for (uint32_t l = 0; l < L; ++l) js[l] = K - 1;
-        } else if (s == KO_STATUS_INFEASIBLE) {
+        int s;
+        if (policy == 3) {
+            s = fit_status[w];
             for (uint32_t l = 0; l < L; ++l) js[l] = 0;
+        } else if (policy == 1) {
+            /* O9 on the sizes of the cost model: the largest j whose total size fits */
+            int found = 0;
+            uint32_t best = 0;
+            for (uint32_t j = 0; j < K; ++j) {
+                uint64_t tot_b = 0;
+                for (uint32_t l = 0; l < L; ++l) tot_b += bytes[(size_t)l * K + j];
+                if (tot_b <= c) { found = 1; best = j; }
+            }
+            s = (!found || c == 0) ? KO_STATUS_INFEASIBLE : (best == K - 1 ? KO_STATUS_PLATEAU : KO_OK);
+            for (uint32_t l = 0; l < L; ++l) js[l] = best;
+        } else if (policy == 2) {
+            s = ko_dp_error_axis(e, kt, L, K, D, value_dtype, c, js, NULL);
         } else {
-            s = ko_dp(e, units, L, K, D, js, NULL, NULL);
-            if (s < 0) { free(units); rc = s; goto done; }
+            s = ko_units_from_bytes(bytes, L, K, c, D, units);
+            if (s == KO_STATUS_PLATEAU) {
+                for (uint32_t l = 0; l < L; ++l) js[l] = K - 1;
+            } else if (s == KO_STATUS_INFEASIBLE) {
+                for (uint32_t l = 0; l < L; ++l) js[l] = 0;
+            } else {
+                s = ko_dp(e, units, L, K, D, js, NULL, NULL);
+            }
         }
-        free(units);
+        if (s < 0) { free(units); free(bytes); free(kk); free(e); free(dense); rc = s; goto done; }
         st[w].budget_bytes = c;
         st[w].status = s;
         st[w].used_bytes = 0;
         st[w].n_selected = 0;
         float tot = 0.0f;
         for (uint32_t l = 0; l < L; ++l) {
-            uint64_t k = ktab[(size_t)l * K + js[l]];
-            st[w].used_bytes += k * bpe;
-            st[w].n_selected += k;
-            tot = tot + e[(size_t)l * K + js[l]];
+            size_t i = (size_t)l * K + js[l];
+            keff[(size_t)w * L + l] = kk[i];
+            if (dense_out) dense_out[(size_t)w * L + l] = (uint32_t)dense[i];
+            st[w].used_bytes += bytes[i];
+            st[w].n_selected += kk[i];
+            tot = tot + e[i];
         }
         st[w].total_err = tot;
+        free(units); free(bytes); free(kk); free(e); free(dense);
         if (st[w].n_selected > cap && idx_out) { rc = KO_ERR_CAPACITY; goto done; }
     }
 
@@ -549,7 +677,7 @@ int ko_step_policy(uint32_t policy, const uint64_t* layer_sizes, uint32_t L, uin
         uint64_t run = 0;
         for (uint32_t l = 0; l < L; ++l) {
             if (offs_out) offs_out[(size_t)w * (L + 1) + l] = run;
-            run += ktab[(size_t)l * K + jsel[(size_t)w * L + l]];
+            run += keff[(size_t)w * L + l];
         }
         if (offs_out) offs_out[(size_t)w * (L + 1) + L] = run;
     }
@@ -558,11 +686,11 @@ int ko_step_policy(uint32_t policy, const uint64_t* layer_sizes, uint32_t L, uin
         for (uint32_t l = 0; l < L; ++l) {
             uint64_t n = layer_sizes[l];
             uint32_t j = jsel[(size_t)w * L + l];
-            uint64_t k = ktab[(size_t)l * K + j];
+            uint64_t k = keff[(size_t)w * L + l];
             if (j_out) j_out[(size_t)w * L + l] = j;
             if (k_out) k_out[(size_t)w * L + l] = (uint32_t)k;
             uint64_t off = 0;
-            for (uint32_t q = 0; q < l; ++q) off += ktab[(size_t)q * K + jsel[(size_t)w * L + q]];
+            for (uint32_t q = 0; q < l; ++q) off += keff[(size_t)w * L + q];
             const float* dl = d + (size_t)w * N + loff[l];
             uint32_t* ib;
             void* vb;
@@ -589,8 +717,18 @@ int ko_step_policy(uint32_t policy, const uint64_t* layer_sizes, uint32_t L, uin
     if (fail) { rc = fail; goto done; }
     if (stats_out) memcpy(stats_out, st, (size_t)W * sizeof(ko_stats));
 done:
-    free(ktab); free(loff); free(err); free(jsel); free(st); free(d);
+    free(ktab); free(keff); free(loff); free(err); free(jsel); free(st); free(d); free(fit_status);
     return rc;
+}
+
+int ko_step_policy(uint32_t policy, const uint64_t* layer_sizes, uint32_t L, uint32_t W, const double* ratios, uint32_t K, uint32_t D,
+            uint32_t value_dtype, uint64_t stride, const float* grads, float* state,
+            const double* bandwidth_bytes_per_s, double t_target_s, const float* inject_err, float* err_out,
+            uint32_t* tau_out, uint32_t* keep_eq_out, uint32_t* j_out, uint32_t* k_out, uint32_t* idx_out,
+            void* val_out, uint64_t cap, uint64_t* offs_out, ko_stats* stats_out) {
+    return ko_step_ex(policy, 0, layer_sizes, L, W, ratios, K, D, value_dtype, stride, grads, state, bandwidth_bytes_per_s,
+                      t_target_s, inject_err, err_out, tau_out, keep_eq_out, j_out, k_out, idx_out, val_out, cap,
+                      offs_out, stats_out, NULL);
 }
 
 int ko_step(const uint64_t* layer_sizes, uint32_t L, uint32_t W, const double* ratios, uint32_t K, uint32_t D,

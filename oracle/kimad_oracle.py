@@ -183,6 +183,7 @@ class StepResult:
     total_err: np.ndarray
     status: np.ndarray
     state: np.ndarray     # float32 [W][stride], the updated estimator
+    dense: np.ndarray = None  # uint32 [W][L]: 1 where the chosen candidate is sent densely (cost model 1)
 
 
 def uniform(ktab: np.ndarray, value_dtype: int, c: int):
@@ -195,6 +196,34 @@ def uniform(ktab: np.ndarray, value_dtype: int, c: int):
     if rc < 0:
         _chk(rc, "uniform")
     return rc, int(j.value)
+
+
+def fit_ratio(layer_sizes, entries: int):
+    """O9b: (status, q, k [L]) of the one ratio q / 2^32 sized to a budget of ``entries`` kept entries."""
+    ls = np.ascontiguousarray(layer_sizes, dtype=np.uint64)
+    k = np.zeros(ls.size, np.uint64)
+    q = C.c_uint64(0)
+    rc = lib().ko_fit_ratio(_p(ls, C.c_uint64), C.c_uint32(ls.size), C.c_uint64(int(entries)), C.byref(q), _p(k, C.c_uint64))
+    if rc < 0:
+        _chk(rc, "fit_ratio")
+    return rc, int(q.value), k
+
+
+def candidate(n: int, k: int, value_dtype: int, cost_model: int):
+    """O13: (bytes, entries kept, dense flag) of candidate k of a layer of n elements."""
+    b, ke, dn = C.c_uint64(0), C.c_uint64(0), C.c_int(0)
+    lib().ko_candidate(C.c_uint64(int(n)), C.c_uint64(int(k)), C.c_uint32(value_dtype), C.c_uint32(cost_model),
+                       C.byref(b), C.byref(ke), C.byref(dn))
+    return int(b.value), int(ke.value), int(dn.value)
+
+
+def units_from_bytes(bytes_tab: np.ndarray, c: int, D: int):
+    bt = np.ascontiguousarray(bytes_tab, dtype=np.uint64)
+    L, K = bt.shape
+    out = np.zeros((L, K), np.uint64)
+    st = _chk(lib().ko_units_from_bytes(_p(bt, C.c_uint64), C.c_uint32(L), C.c_uint32(K), C.c_uint64(int(c)), C.c_uint32(D),
+                                        _p(out, C.c_uint64)), "units_from_bytes")
+    return st, out
 
 
 def dp_error_axis(err: np.ndarray, ktab: np.ndarray, D: int, value_dtype: int, c: int):
@@ -235,10 +264,11 @@ def aggregate(x, est, weights, gamma) -> np.ndarray:
 
 
 def step(layer_sizes, W, ratios, D, value_dtype, grads, state, bandwidth, t_target, cap=None,
-         inject_err=None, policy=0) -> StepResult:
+         inject_err=None, policy=0, cost_model=0) -> StepResult:
     """One full pass O1..O8 for W workers; ``state`` is copied, the copy is updated and returned.
     policy 0: layer-adaptive DP (Kimad+); 1: one grid ratio for all layers (Kimad, O9); 2: the DP on the
-    error axis (O12)."""
+    error axis (O12); 3: one ratio sized to the budget (O9b; ``ratios`` must have one entry, which plays no
+    role).  cost_model 1: sizes with the dense fallback (O13)."""
     ls = np.ascontiguousarray(layer_sizes, dtype=np.uint64)
     r = np.ascontiguousarray(ratios, dtype=np.float64)
     L, K = ls.size, r.size
@@ -261,15 +291,16 @@ def step(layer_sizes, W, ratios, D, value_dtype, grads, state, bandwidth, t_targ
     inj = None
     if inject_err is not None:
         inj = np.ascontiguousarray(inject_err, dtype=np.float32).reshape(W, L, K)
-    _chk(lib().ko_step_policy(C.c_uint32(policy), _p(ls, C.c_uint64), C.c_uint32(L), C.c_uint32(W), _p(r, C.c_double), C.c_uint32(K),
+    dense = np.zeros((W, L), np.uint32)
+    _chk(lib().ko_step_ex(C.c_uint32(policy), C.c_uint32(cost_model), _p(ls, C.c_uint64), C.c_uint32(L), C.c_uint32(W), _p(r, C.c_double), C.c_uint32(K),
                        C.c_uint32(D), C.c_uint32(value_dtype), C.c_uint64(stride), _p(grads, C.c_float),
                        _p(st_new, C.c_float), _p(bw, C.c_double), C.c_double(t_target), _p(inj, C.c_float),
                        _p(err, C.c_float), _p(tau, C.c_uint32), _p(keq, C.c_uint32), _p(j, C.c_uint32),
                        _p(k, C.c_uint32), _p(idx, C.c_uint32), val.ctypes.data_as(C.c_void_p), C.c_uint64(cap),
-                       _p(offs, C.c_uint64), stats), "step")
+                       _p(offs, C.c_uint64), stats, _p(dense, C.c_uint32)), "step")
     return StepResult(err, tau, keq, j, k, idx, val, offs,
                       np.array([s.budget_bytes for s in stats], np.uint64),
                       np.array([s.used_bytes for s in stats], np.uint64),
                       np.array([s.n_selected for s in stats], np.uint64),
                       np.array([s.total_err for s in stats], np.float32),
-                      np.array([s.status for s in stats], np.int32), st_new)
+                      np.array([s.status for s in stats], np.int32), st_new, dense)

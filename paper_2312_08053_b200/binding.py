@@ -112,6 +112,14 @@ def load():
     L.kimad_debug_exact_path_layers.argtypes = [vp, C.POINTER(u64)]
     L.kimad_launch_count.restype = u64
     L.kimad_launch_count.argtypes = [vp]
+    L.kimad_monitor_create.restype = C.c_int
+    L.kimad_monitor_create.argtypes = [C.POINTER(vp), u32, dbl]
+    L.kimad_monitor_destroy.restype = None
+    L.kimad_monitor_destroy.argtypes = [vp]
+    L.kimad_monitor_observe.restype = C.c_int
+    L.kimad_monitor_observe.argtypes = [vp, u64, dbl]
+    L.kimad_monitor_estimate.restype = dbl
+    L.kimad_monitor_estimate.argtypes = [vp]
     L.kimad_strerror.restype = C.c_char_p
     L.kimad_strerror.argtypes = [C.c_int]
     _lib = L
@@ -341,3 +349,35 @@ def new_context(layer_sizes, n_workers, ratio_grid, device="cuda", **opts):
     kimad_set_workspace(ctx, ws[off:])
     ctx._keep.append(ws)
     return ctx
+
+
+class Monitor:
+    """Owning handle of a ``kimad_monitor*`` (bandwidth estimate from the history of finished transfers)."""
+
+    def __init__(self, window: int = 8, alpha: float = 1.0):
+        h = C.c_void_p()
+        _check(load().kimad_monitor_create(C.byref(h), int(window), float(alpha)), "kimad_monitor_create")
+        self.handle = h
+
+    def __del__(self):
+        h, self.handle = getattr(self, "handle", None), None
+        if h and _lib is not None:
+            _lib.kimad_monitor_destroy(h)
+
+
+def kimad_monitor_create(window: int = 8, alpha: float = 1.0) -> Monitor:
+    return Monitor(window, alpha)
+
+
+def kimad_monitor_observe(m: Monitor, n_bytes: int, seconds: float) -> None:
+    _check(load().kimad_monitor_observe(m.handle, int(n_bytes), float(seconds)), "kimad_monitor_observe")
+
+
+def kimad_monitor_estimate(m: Monitor) -> float:
+    return float(load().kimad_monitor_estimate(m.handle))
+
+
+def kimad_monitor_destroy(m: Monitor) -> None:
+    h, m.handle = m.handle, None
+    if h:
+        load().kimad_monitor_destroy(h)

@@ -604,6 +604,62 @@ int kimad_debug_exact_path_layers(kimad_ctx* c, uint64_t* host_count) {
 uint64_t kimad_launch_count(const kimad_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
 // ---------------------------------------------------------------------------------------------------
+// Bandwidth monitor: windowed throughput of the reported transfers with exponential smoothing (host only)
+// ---------------------------------------------------------------------------------------------------
+} // extern "C"
+struct kimad_monitor {
+    std::vector<uint64_t> bytes;
+    std::vector<double> secs;
+    uint32_t window = 1, head = 0, filled = 0;
+    double alpha = 1.0, est = 0.0;
+    bool any = false;
+};
+extern "C" {
+
+int kimad_monitor_create(kimad_monitor** out, uint32_t window, double alpha) {
+    if (!out) return KIMAD_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (window == 0 || window > 65536 || !(alpha > 0.0) || !(alpha <= 1.0)) return KIMAD_ERR_INVALID_ARG;
+    kimad_monitor* m = new (std::nothrow) kimad_monitor();
+    if (!m) return KIMAD_ERR_NOMEM;
+    try {
+        m->bytes.assign(window, 0);
+        m->secs.assign(window, 0.0);
+    } catch (const std::bad_alloc&) {
+        delete m;
+        return KIMAD_ERR_NOMEM;
+    }
+    m->window = window;
+    m->alpha = alpha;
+    *out = m;
+    return KIMAD_OK;
+}
+
+void kimad_monitor_destroy(kimad_monitor* m) { delete m; }
+
+int kimad_monitor_observe(kimad_monitor* m, uint64_t bytes, double seconds) {
+    if (!m || !(seconds > 0.0) || !std::isfinite(seconds)) return KIMAD_ERR_INVALID_ARG;
+    m->bytes[m->head] = bytes;
+    m->secs[m->head] = seconds;
+    m->head = (m->head + 1) % m->window;
+    if (m->filled < m->window) ++m->filled;
+    // sums are taken afresh over the window, oldest entry first: no drift from adding and removing terms
+    double sb = 0.0, ss = 0.0;
+    const uint32_t first = (m->head + m->window - m->filled) % m->window;
+    for (uint32_t i = 0; i < m->filled; ++i) {
+        const uint32_t at = (first + i) % m->window;
+        sb += (double)m->bytes[at];
+        ss += m->secs[at];
+    }
+    const double windowed = sb / ss;
+    m->est = m->any ? m->alpha * windowed + (1.0 - m->alpha) * m->est : windowed;
+    m->any = true;
+    return KIMAD_OK;
+}
+
+double kimad_monitor_estimate(const kimad_monitor* m) { return m && m->any ? m->est : 0.0; }
+
+// ---------------------------------------------------------------------------------------------------
 // Allocation-free variant of kimad_step: the scratch is a fixed array inside the library's device image.
 // ---------------------------------------------------------------------------------------------------
 static __device__ __align__(256) unsigned char g_builtin_scratch[KIMAD_BUILTIN_SCRATCH_BYTES];

@@ -1,16 +1,27 @@
-// Device code of the Kimad+ compression pass for sm_100a.
+// Device code of the Kimad+ compression pass for sm_100a: helpers shared by all stages, the exact radix
+// resolve kernels and the knapsack DP.
 //
-// Stage map (letters as in include/kimad.h):
-//   k_diff_hist1          (a) d = grad - g, written to scratch, fused with the first digit
-//                             (11 bits) of a 3-digit radix histogram of the magnitude key
-//   k_resolve1/2/3        (b) locate, for every candidate k_j of every layer, the bin that holds
-//   k_hist2, k_hist3          the k_j-th largest key, digit by digit (11 + 10 + 10 bits), while
-//                             summing the squares of everything below it -> err, tau, keep_eq
-//   k_dp                  (c) Algorithm 3 on the budget axis, one CTA per worker
-//   k_select_count/scan   (d) per-chunk counts of entries above / equal to the chosen threshold
-//   k_select_write        (e)+(f) ordered compaction into (idx, val) and g += C(d)
+// Stage map of one step (letters as in include/kimad.h; file in brackets):
+//   k_sample        (a)+(b) per (worker, layer): stratified sample of |grad - g| -> for every candidate k_j the
+//                   band of 16-bit key prefixes that can hold its threshold -> bin tables        [kimad_curve.cuh]
+//   k_pass_a        (a)+(b) the sweep: d = grad - g (Section 3 footnote, Eq. 6), bin = table(key(d)), count and
+//                   exact integer sum of squares per bin in shared memory; the upper halves of the bit patterns
+//                   of d go to scratch (d itself is never stored)                                [kimad_curve.cuh]
+//   k_resolve_a     (b) Eq. 4 / the "Errors" matrix of Algorithm 3: err_l(k_j) from the bins, certified to the
+//                   curve tolerance; layers that fail the certificate are handed to the exact path [kimad_curve.cuh]
+//   k_tiny_exact    (b) layers of at most 4096 elements, sorted in shared memory                 [kimad_curve.cuh]
+//   k_fb_hist1, k_fb_hist23<2|3>, k_resolve1, k_resolve23<2|3>, k_rebuild_slots
+//                   (b) exact 11+10+10-bit radix select over the handed-over layers (usually none)
+//                                                                          [kimad_curve.cuh, this file]
+//   k_dp            (c) Algorithm 3 on the budget axis (Eq. 2, Eq. 3, Section 3.2), one CTA per worker; also the
+//                   uniform-ratio policies and the error-axis reading                            [this file]
+//   k_sel_count, k_sel_resolve(_r2), k_sel_count_r2, k_sel_recount, k_sel_slices, k_sel_scan
+//                   (d) exact threshold and per-slice output offsets at the chosen k             [kimad_select.cuh]
+//   k_sel_write     (e)+(f) ordered (index, value) pack and g += C(d) (Algorithm 1, Eq. 6)       [kimad_select.cuh]
+//   k_apply_packed, k_aggregate   receiving side and model step (Algorithm 1, server lines)      [kimad_receiver.cuh]
 //
-// Everything is HBM- or latency-bound; there is no dense contraction, so no tensor-core path.
+// Nothing here is a dense contraction, so there is no tensor-core path.  The sweep is bound by instruction issue and
+// shared-memory latency (it keeps 0.9 of its time when its loads are served from cache); the other sweeps by HBM.
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
