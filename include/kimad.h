@@ -82,13 +82,33 @@ typedef struct {
                                       (binary64), the value is the number of kept entries, and the answer is
                                       the lowest error level whose smallest size fits c.  Needs L * K small
                                       enough for the candidate tables to sit in shared memory (else
-                                      kimad_create returns INVALID_ARG).                                     */
+                                      kimad_create returns INVALID_ARG).
+                                   3: Kimad as Section 3.1 states it: ONE ratio for all layers, SIZED TO THE
+                                      BUDGET instead of taken from a grid: r = q / 2^32 with the largest q in
+                                      [0, 2^32] such that sum_l k_l fits floor(c / (4 + vb)) entries, where
+                                      k_l = min(n_l, max(1, floor(q n_l / 2^32))).  The ratio grid plays no
+                                      role and must be {1.0} (n_ratios = 1); every layer has the one candidate
+                                      j = 0, whose k is the fitted one (err/tau of kimad_debug_get_curve
+                                      describe it; kimad_get_k_table still returns the static table, k = n_l).
+                                      Fewer than one entry per layer affordable -> every k_l = 1, INFEASIBLE;
+                                      everything affordable -> PLATEAU.  A context with a single layer of N
+                                      elements is TopK over the whole model at K = floor(c / (4 + vb))
+                                      (Section 4.3: "select K with the whole model information").            */
+    uint32_t cost_model;        /* how a compressed layer is sized (Eq. 3's b_ij; the paper fixes no encoding):
+                                   0: k (4 + vb) bytes, also at k = n_l;
+                                   1: dense fallback: a candidate whose sparse size reaches the layer's dense size,
+                                      k (4 + vb) >= vb n_l, is sent DENSELY: all n_l values in index order, no
+                                      indices, vb n_l bytes; it keeps every entry and has no compression error.
+                                      kimad_packed.dense flags such layers; idx is still filled (0 .. n_l - 1)
+                                      so that the receiving side reads the message the same way, but a transport
+                                      would not send it (used_bytes counts vb n_l).  Policies 0 and 1 only.  */
 } kimad_options;
 
 /* Per-worker result record, written by the device. */
 typedef struct {
     uint64_t budget_bytes; /* c                                                          */
-    uint64_t used_bytes;   /* sum_l k_l * (4 + vb); <= c unless status is INFEASIBLE     */
+    uint64_t used_bytes;   /* sum of the chosen candidates' sizes (k_l (4 + vb), or vb n_l for a layer
+                              sent densely under cost model 1); <= c unless status is INFEASIBLE */
     uint64_t n_selected;   /* sum_l k_l                                                  */
     float total_err;       /* err_1(k_1) + ... + err_L(k_L), added left to right in f32  */
     int32_t status;        /* 0, a KIMAD_STATUS_* or a KIMAD_ERR_* of this worker        */
@@ -101,7 +121,8 @@ typedef struct {
  *   offs  u64 [W][L+1]               running sum of k_l
  *   k     u32 [W][L]                 chosen k per layer
  *   j     u32 [W][L]                 chosen candidate (index into the ratio grid) per layer
- *   stats [W]                                                                                  */
+ *   stats [W]
+ *   dense u32 [W][L]                 1 where the layer is sent densely (cost model 1), else 0; may be NULL */
 typedef struct {
     uint32_t* idx;
     void* val;
@@ -109,6 +130,7 @@ typedef struct {
     uint32_t* k;
     uint32_t* j;
     kimad_stats* stats;
+    uint32_t* dense;
 } kimad_packed;
 
 /* Problem statement of Section 3.2: the layers, the workers and the discrete ratio set

@@ -30,7 +30,7 @@ KIMAD_BUILTIN_SCRATCH_BYTES = 32 << 20
 class kimad_options(C.Structure):
     _fields_ = [("D", C.c_uint32), ("value_dtype", C.c_uint32), ("check_finite", C.c_uint32),
                 ("infeasible_policy", C.c_uint32), ("max_packed_elems", C.c_uint64), ("worker_stride", C.c_uint64),
-                ("curve_mode", C.c_uint32), ("policy", C.c_uint32)]
+                ("curve_mode", C.c_uint32), ("policy", C.c_uint32), ("cost_model", C.c_uint32)]
 
 
 class kimad_stats(C.Structure):
@@ -40,7 +40,7 @@ class kimad_stats(C.Structure):
 
 class kimad_packed(C.Structure):
     _fields_ = [("idx", C.c_void_p), ("val", C.c_void_p), ("offs", C.c_void_p), ("k", C.c_void_p),
-                ("j", C.c_void_p), ("stats", C.c_void_p)]
+                ("j", C.c_void_p), ("stats", C.c_void_p), ("dense", C.c_void_p)]
 
 
 STATS_DTYPE = np.dtype([("budget_bytes", "<u8"), ("used_bytes", "<u8"), ("n_selected", "<u8"),
@@ -154,10 +154,10 @@ class Ctx:
 
 
 def kimad_create(layer_sizes, n_workers, ratio_grid, D=0, value_dtype=0, check_finite=0, max_packed_elems=0,
-                 worker_stride=0, curve_mode=0, policy=0) -> Ctx:
+                 worker_stride=0, curve_mode=0, policy=0, cost_model=0) -> Ctx:
     ls = np.ascontiguousarray(layer_sizes, dtype=np.uint64)
     rg = np.ascontiguousarray(ratio_grid, dtype=np.float64)
-    opts = kimad_options(D, value_dtype, check_finite, 0, max_packed_elems, worker_stride, curve_mode, policy)
+    opts = kimad_options(D, value_dtype, check_finite, 0, max_packed_elems, worker_stride, curve_mode, policy, cost_model)
     h = C.c_void_p()
     _check(load().kimad_create(C.byref(h), ls.ctypes.data_as(C.POINTER(C.c_uint64)), ls.size, n_workers,
                                rg.ctypes.data_as(C.POINTER(C.c_double)), rg.size, C.byref(opts)), "kimad_create")
@@ -194,8 +194,9 @@ class Packed:
         self.k = torch.zeros((W, L), dtype=torch.int32, device=device)
         self.j = torch.zeros((W, L), dtype=torch.int32, device=device)
         self.stats = torch.zeros((W, STATS_DTYPE.itemsize), dtype=torch.uint8, device=device)
+        self.dense = torch.zeros((W, L), dtype=torch.int32, device=device)
         self.c = kimad_packed(self.idx.data_ptr(), self.val.data_ptr(), self.offs.data_ptr(), self.k.data_ptr(),
-                              self.j.data_ptr(), self.stats.data_ptr())
+                              self.j.data_ptr(), self.stats.data_ptr(), self.dense.data_ptr())
 
     def stats_host(self) -> np.ndarray:
         return self.stats.cpu().numpy().view(STATS_DTYPE).reshape(-1)

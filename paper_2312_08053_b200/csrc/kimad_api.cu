@@ -19,7 +19,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
     // static tables
-    size_t dbuf, chunks, layers, ktab, reg_layers, tiny_layers, reg_index;
+    size_t dbuf, chunks, layers, ktab, ktab_dyn, reg_layers, tiny_layers, reg_index;
     // zeroed at set_workspace and kept clean by the kernels
     size_t zero_from, h1_cnt, h1_ss, h23_cnt, h23_ss, bh_cnt, bh_sum, low_hist, recount, fb, r2, flags;
     // scratch without initial-state requirements
@@ -40,7 +40,7 @@ struct kimad_ctx {
     std::vector<LayerDesc> layers;
     std::vector<uint32_t> reg_layers, tiny_layers, reg_index; // layers above / up to kTinyMax elements
     uint32_t curve_mode = 0;
-    uint32_t policy = 0;
+    uint32_t policy = 0, cost_model = 0;
     size_t sample_smem = 0, pass_a_smem = 0, tiny_smem = 0;
     Layout lay{};
     unsigned char* ws = nullptr;
@@ -71,6 +71,7 @@ void plan_layout(kimad_ctx* c) {
     y.chunks = take(nch * sizeof(Chunk));
     y.layers = take(c->layers.size() * sizeof(LayerDesc));
     y.ktab = take(c->ktab.size() * sizeof(uint64_t));
+    y.ktab_dyn = take(c->policy == 3 ? (size_t)c->W * c->L * sizeof(uint64_t) : 0); // per-worker rows of the fitted ratio
     y.reg_layers = take(c->reg_layers.size() * sizeof(uint32_t));
     y.tiny_layers = take(c->tiny_layers.size() * sizeof(uint32_t));
     y.reg_index = take(c->reg_index.size() * sizeof(uint32_t));
@@ -123,7 +124,7 @@ static int preload_kernels() {
     KIMAD_PRELOAD(k_sample); KIMAD_PRELOAD(k_pass_a<true>); KIMAD_PRELOAD(k_pass_a<false>); KIMAD_PRELOAD(k_resolve_a);
     KIMAD_PRELOAD(k_tiny_exact); KIMAD_PRELOAD(k_fb_hist1); KIMAD_PRELOAD(k_fb_hist23<2>); KIMAD_PRELOAD(k_fb_hist23<3>);
     KIMAD_PRELOAD(k_resolve1); KIMAD_PRELOAD(k_resolve23<2>); KIMAD_PRELOAD(k_resolve23<3>); KIMAD_PRELOAD(k_rebuild_slots);
-    KIMAD_PRELOAD(k_dp); KIMAD_PRELOAD(k_sel_count); KIMAD_PRELOAD(k_sel_count_r2); KIMAD_PRELOAD(k_sel_resolve);
+    KIMAD_PRELOAD(k_dp); KIMAD_PRELOAD(k_fit_ratio); KIMAD_PRELOAD(k_sel_count); KIMAD_PRELOAD(k_sel_count_r2); KIMAD_PRELOAD(k_sel_resolve);
     KIMAD_PRELOAD(k_sel_resolve_r2); KIMAD_PRELOAD(k_sel_recount); KIMAD_PRELOAD(k_sel_slices); KIMAD_PRELOAD(k_sel_scan);
     KIMAD_PRELOAD((k_sel_write<false, false>)); KIMAD_PRELOAD((k_sel_write<false, true>));
     KIMAD_PRELOAD((k_sel_write<true, false>)); KIMAD_PRELOAD((k_sel_write<true, true>));
@@ -178,7 +179,9 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
     const DSource dbuf{c->at<uint16_t>(y.dbuf), grads, state, c->stride};
     const Chunk* chunks = c->at<Chunk>(y.chunks);
     const LayerDesc* layers = c->at<LayerDesc>(y.layers);
-    const uint64_t* ktab = c->at<uint64_t>(y.ktab);
+    // candidates: the grid's table for every worker, or (policy 3) each worker's row of the ratio fitted to its budget
+    const KTab ktab = c->policy == 3 && mode != kGivenJ ? KTab{c->at<uint64_t>(y.ktab_dyn), (uint64_t)c->L * c->K}
+                                                        : KTab{c->at<uint64_t>(y.ktab), 0};
     const uint32_t* reg_layers = c->at<uint32_t>(y.reg_layers);
     const uint32_t* tiny_layers = c->at<uint32_t>(y.tiny_layers);
     const uint32_t* reg_index = c->at<uint32_t>(y.reg_index);
@@ -221,7 +224,23 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
     const dim3 grun((nch + run_chunks - 1) / run_chunks, W);
     int stage = 0;
     auto mark = [&]() { if (c->timing) cudaEventRecord(c->ev[stage++], s); };
+    auto budgets_of = [&](uint32_t w0, uint32_t nw) {
+        DpBudgets b{};
+        for (uint32_t i = 0; i < nw; ++i) {
+            double cb = std::floor(bw[w0 + i] * t);
+            b.c[i] = !(cb > 0.0) ? 0ull : (cb >= 18446744073709551615.0 ? ~0ull : (uint64_t)cb);
+        }
+        return b;
+    };
     mark();
+    if (c->policy == 3 && mode != kGivenJ) { // Section 3.1: the one ratio sized to each worker's budget
+        for (uint32_t w0 = 0; w0 < W; w0 += kDpWorkersPerLaunch) {
+            const uint32_t nw = std::min<uint32_t>(kDpWorkersPerLaunch, W - w0);
+            CUDA_TRY(launch_pdl(k_fit_ratio, nw, blk, 0, s, budgets_of(w0, nw), w0, W, L, c->bpe, c->N, layers,
+                                c->at<uint64_t>(y.ktab_dyn)));
+            c->launches += 1;
+        }
+    }
     if (T) CUDA_TRY(cudaEventRecord(c->ev_fork, s)); // fork point of the tiny layers' kernel: the step's start
     // (a) + (b): sample -> bands -> one sweep -> curves
     if (R) {
@@ -269,16 +288,12 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
     mark();
     // (c)
     for (uint32_t w0 = 0; w0 < W; w0 += kDpWorkersPerLaunch) {
-        DpBudgets b{};
         const uint32_t nw = std::min<uint32_t>(kDpWorkersPerLaunch, W - w0);
-        for (uint32_t i = 0; i < nw; ++i) {
-            double cb = std::floor(bw[w0 + i] * t);
-            b.c[i] = !(cb > 0.0) ? 0ull : (cb >= 18446744073709551615.0 ? ~0ull : (uint64_t)cb);
-        }
-        CUDA_TRY(launch_pdl(k_dp, nw, kDpThreads, c->dp_smem, s, b, w0, W, L, K, c->D, c->bpe, c->full_bytes, c->cap,
-                            c->check_finite, mode == kGivenJ ? 1 : (c->policy == 1 ? 2 : (c->policy == 2 ? 3 : 0)), c->dp_plan,
+        const int dp_mode = mode == kGivenJ ? 1 : (c->policy == 1 ? 2 : (c->policy == 2 ? 3 : (c->policy == 3 ? 4 : 0)));
+        CUDA_TRY(launch_pdl(k_dp, nw, kDpThreads, c->dp_smem, s, budgets_of(w0, nw), w0, W, L, K, c->D, c->bpe, c->full_bytes, c->cap,
+                            c->check_finite, dp_mode, c->cost_model, c->dp_plan, layers,
                             ktab, mode == kInjectErr ? err_dev : err, tau, keq, shf, j_dev, flags, pd, sel, out->k, out->j,
-                            out->offs, out->stats));
+                            out->offs, out->stats, out->dense));
         c->launches += 1;
     }
     mark();
@@ -329,8 +344,10 @@ int kimad_create(kimad_ctx** out, const uint64_t* layer_sizes, uint32_t n_layers
     if (opt) o = *opt;
     if (o.D == 0) o.D = 1000;
     if (o.D > KIMAD_MAX_D || o.D < n_layers || o.value_dtype > 1 || o.infeasible_policy != 0 || o.curve_mode > 1 ||
-        o.policy > 2)
+        o.policy > 3 || o.cost_model > 1)
         return KIMAD_ERR_INVALID_ARG;
+    if (o.cost_model == 1 && o.policy >= 2) return KIMAD_ERR_INVALID_ARG;               // dense fallback: policies 0 and 1
+    if (o.policy == 3 && (n_ratios != 1 || ratio_grid[0] != 1.0)) return KIMAD_ERR_INVALID_ARG; // the ratio is fitted, not listed
     for (uint32_t j = 0; j < n_ratios; ++j) {
         if (!(ratio_grid[j] > 0.0) || ratio_grid[j] > 1.0) return KIMAD_ERR_INVALID_ARG;
         if (j && !(ratio_grid[j] > ratio_grid[j - 1])) return KIMAD_ERR_INVALID_ARG;
@@ -354,7 +371,7 @@ int kimad_create(kimad_ctx** out, const uint64_t* layer_sizes, uint32_t n_layers
                 if (k > n) k = n;
                 c->ktab[(size_t)l * n_ratios + j] = k;
             }
-            c->full_bytes += c->ktab[(size_t)l * n_ratios + n_ratios - 1] * c->bpe;
+            c->full_bytes += candidate_bytes(n, c->ktab[(size_t)l * n_ratios + n_ratios - 1], c->bpe, o.cost_model, nullptr);
             // chunk table: aligned windows of the flat vector intersected with this layer
             LayerDesc ld{N, n, (uint32_t)c->chunks.size(), 0};
             for (uint64_t p = N; p < N + n;) {
@@ -393,6 +410,7 @@ int kimad_create(kimad_ctx** out, const uint64_t* layer_sizes, uint32_t n_layers
         c->dp_smem = used;
         c->curve_mode = o.curve_mode;
         c->policy = o.policy;
+        c->cost_model = o.cost_model;
         if (c->policy == 2 && !c->dp_plan.tab_in_smem) { delete c; return KIMAD_ERR_INVALID_ARG; }
         c->sample_smem = (size_t)(2 * (1024 + 32) + 32768 + 2048 + 1024 + 2048 + 2048 + 32 + 3 * 128) * 4;
         c->pass_a_smem = (size_t)(3 * kMaxBins + kLutWords) * 4 + kL1Bins * 2;
@@ -549,7 +567,8 @@ int kimad_plan_budget(const kimad_ctx* c, double bandwidth_bytes_per_s, double t
     if (cc >= c->full_bytes) return KIMAD_STATUS_PLATEAU;
     if (cc == 0) return KIMAD_STATUS_INFEASIBLE;
     if (cells)
-        for (size_t i = 0; i < c->ktab.size(); ++i) cells[i] = budget_cells(c->ktab[i] * c->bpe, c->D, cc);
+        for (size_t i = 0; i < c->ktab.size(); ++i)
+            cells[i] = budget_cells(candidate_bytes(c->layer_sizes[i / c->K], c->ktab[i], c->bpe, c->cost_model, nullptr), c->D, cc);
     return KIMAD_OK;
 }
 

@@ -58,6 +58,24 @@ struct Sel {
     uint64_t base;    // first output position of the layer in the worker's packed buffers
 };
 
+// The candidate table k_{l,j}: one table for all workers (wstride = 0: the ratio grid applied to the layer sizes), or
+// one per worker (the ratio fitted to each worker's budget).
+struct KTab {
+    const uint64_t* p;
+    uint64_t wstride;
+    KIMAD_HD uint64_t at(uint32_t w, size_t i) const { return p[(size_t)w * wstride + i]; }
+};
+
+// Size in bytes of candidate k of a layer of n elements and the entries it keeps (Eq. 3's b_ij; the paper fixes no
+// encoding).  cost model 0: k (4 + vb).  cost model 1: once the sparse size reaches the dense size vb n the layer is
+// sent densely: every value, no indices; it then keeps all n entries and loses nothing.
+KIMAD_HD uint64_t candidate_bytes(uint64_t n, uint64_t k, uint32_t bpe, uint32_t cost_model, bool* dense) {
+    const uint64_t vb = bpe - 4;
+    const bool d = cost_model == 1 && k * bpe >= vb * n;
+    if (dense) *dense = d;
+    return d ? vb * n : k * bpe;
+}
+
 // Budget cells a candidate of `bytes` occupies when c bytes are split into D cells (rounded up, so
 // the byte constraint of Eq. 3 can never be exceeded).  c > 0.
 KIMAD_HD uint64_t budget_cells(uint64_t bytes, uint32_t D, uint64_t c) { return (bytes * (uint64_t)D + c - 1) / c; }

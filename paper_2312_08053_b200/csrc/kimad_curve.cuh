@@ -50,7 +50,7 @@ __device__ __forceinline__ uint32_t hash_u32(uint32_t x) {
 __global__ void __launch_bounds__(kBigThreads, 1)
 k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint64_t stride,
          const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ reg_layers, uint32_t R,
-         const uint64_t* __restrict__ ktab, uint32_t K, uint32_t force_exact, uint16_t* __restrict__ lut_t1,
+         const KTab ktab, uint32_t K, uint32_t force_exact, uint16_t* __restrict__ lut_t1,
          uint32_t* __restrict__ lut_t2, uint32_t* __restrict__ bin_lo, BandMeta* __restrict__ meta) {
     pdl_wait();
     extern __shared__ __align__(16) uint32_t sh[];
@@ -169,7 +169,7 @@ k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint6
 
     // ---- bands: the cells that can hold the k_j-th largest key, and how finely to cut them (one warp per candidate)
     for (uint32_t j = threadIdx.x >> 5; j < K; j += kBigThreads / 32) {
-        const uint64_t k = ktab[(size_t)l * K + j];
+        const uint64_t k = ktab.at(w, (size_t)l * K + j);
         uint32_t o_cb = 1, o_ct = 0, o_cs = 15; // k == n keeps everything: no threshold, no band
         if (k < n) {
             uint32_t r_lo, r_hi;
@@ -517,7 +517,7 @@ k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, uint1
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kBigThreads)
 k_resolve_a(const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ reg_layers, uint32_t R, uint32_t L,
-            const uint64_t* __restrict__ ktab, uint32_t K, const BandMeta* __restrict__ meta,
+            const KTab ktab, uint32_t K, const BandMeta* __restrict__ meta,
             const uint32_t* __restrict__ bin_lo, uint32_t* __restrict__ bh_cnt, unsigned long long* __restrict__ bh_sum,
             float* __restrict__ err_out, uint32_t* __restrict__ tau_out, uint32_t* __restrict__ rank_out,
             uint32_t* __restrict__ shift_out, uint32_t* __restrict__ flags, FbList* __restrict__ fb,
@@ -536,7 +536,7 @@ k_resolve_a(const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ r
     const LayerDesc ld = layers[l];
     if (threadIdx.x == 0) s_bad = mt.flagged;
     if (threadIdx.x < K) {
-        const uint64_t k = ktab[(size_t)l * K + threadIdx.x];
+        const uint64_t k = ktab.at(w, (size_t)l * K + threadIdx.x);
         s_drop[threadIdx.x] = (uint32_t)(ld.n - k);
         s_bin[threadIdx.x] = 0xffffffffu;
     }
@@ -650,7 +650,7 @@ k_resolve_a(const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ r
 __global__ void __launch_bounds__(kThreads)
 k_tiny_exact(const float* __restrict__ grads, const float* __restrict__ state, uint64_t stride,
              const LayerDesc* __restrict__ layers,
-             const uint32_t* __restrict__ tiny_layers, uint32_t L, const uint64_t* __restrict__ ktab, uint32_t K,
+             const uint32_t* __restrict__ tiny_layers, uint32_t L, const KTab ktab, uint32_t K,
              float* __restrict__ err_out, uint32_t* __restrict__ tau_out, uint32_t* __restrict__ rank_out,
              uint32_t* __restrict__ shift_out, uint32_t* __restrict__ flags) {
     pdl_wait();
@@ -707,7 +707,7 @@ k_tiny_exact(const float* __restrict__ grads, const float* __restrict__ state, u
     __syncthreads();
     const size_t wl = (size_t)w * L + l;
     for (uint32_t j = threadIdx.x; j < K; j += kThreads) {
-        const uint32_t k = (uint32_t)ktab[(size_t)l * K + j];
+        const uint32_t k = (uint32_t)ktab.at(w, (size_t)l * K + j);
         const size_t o = wl * K + j;
         const uint32_t t = s_key[k - 1];
         int lo = 0, hi = (int)k - 1; // first rank whose key equals t

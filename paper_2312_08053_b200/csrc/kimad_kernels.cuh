@@ -191,7 +191,7 @@ struct FbList { // layers handed to the exact radix path in this step, and their
 
 __global__ void __launch_bounds__(kThreads)
 k_resolve1(const FbList* __restrict__ fb, const uint2* __restrict__ fb_layers, uint32_t* __restrict__ g_cnt,
-           unsigned long long* __restrict__ g_ss, const uint64_t* __restrict__ ktab, uint32_t L, uint32_t K,
+           unsigned long long* __restrict__ g_ss, const KTab ktab, uint32_t L, uint32_t K,
            Cand* __restrict__ cands, SlotTab* __restrict__ slots) {
     pdl_wait();
     __shared__ __align__(16) uint32_t s_incl[kL1Bins];
@@ -222,7 +222,7 @@ k_resolve1(const FbList* __restrict__ fb, const uint2* __restrict__ fb_layers, u
     scan_bins<kL1Bins>(s_incl, s_below, s_w32, s_w64);
     Cand* cd = cands + wl * K;
     for (uint32_t j = threadIdx.x; j < K; j += kThreads) {
-        const uint32_t k = (uint32_t)ktab[(size_t)l * K + j];
+        const uint32_t k = (uint32_t)ktab.at(w, (size_t)l * K + j);
         const int p = find_pos<kL1Bins>(s_incl, k);
         const uint32_t above = p ? s_incl[p - 1] : 0u;
         Cand c;
@@ -367,16 +367,19 @@ struct DpPlan {
 };
 
 // mode 0: DP (Kimad+); mode 1: candidates given (j_in); mode 2: one candidate index for all layers, the
-// largest whose total size fits the budget (Kimad without layer adaptivity, Section 3.1); mode 3: Algorithm 3
-// read with the discretised error as the axis and the size as the value (needs plan.tab_in_smem)
+// largest whose total size fits the budget (Kimad on the grid, Section 3.1); mode 3: Algorithm 3 read with the
+// discretised error as the axis and the size as the value (needs plan.tab_in_smem); mode 4: the table holds, per
+// worker, the single candidate of the ratio fitted to the budget (k_fit_ratio): nothing to search.
+// cost_model 1: a candidate whose sparse size reaches the layer's dense size is sent densely (candidate_bytes).
 __global__ void __launch_bounds__(kDpThreads)
 k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uint32_t D, uint32_t bpe,
-     uint64_t full_bytes, uint64_t cap, uint32_t check_finite, int mode, DpPlan plan,
-     const uint64_t* __restrict__ ktab, const float* __restrict__ err, const uint32_t* __restrict__ tau,
+     uint64_t full_bytes, uint64_t cap, uint32_t check_finite, int mode, uint32_t cost_model, DpPlan plan,
+     const LayerDesc* __restrict__ layers, const KTab ktab, const float* __restrict__ err, const uint32_t* __restrict__ tau,
      const uint32_t* __restrict__ keep_eq, const uint32_t* __restrict__ shift /* may be null: all exact */,
      const uint32_t* __restrict__ j_in, uint32_t* __restrict__ flags,
      uint8_t* __restrict__ pd_global, Sel* __restrict__ sel, uint32_t* __restrict__ out_k,
-     uint32_t* __restrict__ out_j, uint64_t* __restrict__ out_offs, kimad_stats* __restrict__ out_stats) {
+     uint32_t* __restrict__ out_j, uint64_t* __restrict__ out_offs, kimad_stats* __restrict__ out_stats,
+     uint32_t* __restrict__ out_dense /* may be null */) {
     pdl_wait();
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const uint32_t w = w_base + blockIdx.x;
@@ -420,13 +423,15 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
             __syncthreads();
             for (uint32_t j = threadIdx.x; j < K; j += blockDim.x) {
                 uint64_t bytes = 0;
-                for (uint32_t l = 0; l < L; ++l) bytes += ktab[(size_t)l * K + j] * bpe;
+                for (uint32_t l = 0; l < L; ++l) bytes += candidate_bytes(layers[l].n, ktab.at(w, (size_t)l * K + j), bpe, cost_model, nullptr);
                 if (bytes <= c) atomicMax(&s_fit, j + 1);
             }
             __syncthreads();
             const uint32_t fit = s_fit;
             if (fit == 0) status = KIMAD_STATUS_INFEASIBLE;
             for (uint32_t l = threadIdx.x; l < L; l += blockDim.x) s_j[l] = fit ? fit - 1 : 0;
+        } else if (mode == 4) {
+            for (uint32_t l = threadIdx.x; l < L; l += blockDim.x) s_j[l] = 0; // feasibility is judged on the totals below
         } else if (mode == 3) {
             // Error axis: E_max = sum_l err_{l,0} (binary64, layers in order), cells e_{l,j} = floor(err D / E_max),
             // value = fewest kept entries for a total of exactly e cells; answer = lowest e whose value fits c.
@@ -451,7 +456,7 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
                 if (j < K) {
                     const double q = emax > 0.0 ? floor(__ddiv_rn(__dmul_rn((double)e_w[(size_t)l * K + j], (double)D), emax)) : 0.0;
                     u = q > (double)D ? D : (uint32_t)q;
-                    kk = (uint32_t)ktab[(size_t)l * K + j];
+                    kk = (uint32_t)ktab.at(w, (size_t)l * K + j);
                 }
                 s_units[i] = u;
                 s_kk[i] = kk;
@@ -515,9 +520,10 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
                 uint32_t u = D + 1;
                 float e = 0.f;
                 if (j < K) {
-                    const uint64_t uu = budget_cells(ktab[(size_t)l * K + j] * bpe, D, c);
+                    bool dense;
+                    const uint64_t uu = budget_cells(candidate_bytes(layers[l].n, ktab.at(w, (size_t)l * K + j), bpe, cost_model, &dense), D, c);
                     u = uu > D ? D + 1 : (uint32_t)uu;
-                    e = e_w[(size_t)l * K + j];
+                    e = dense ? 0.f : e_w[(size_t)l * K + j]; // a layer sent densely loses nothing
                 }
                 s_units[slot_l * Kp + j] = u;
                 s_err[slot_l * Kp + j] = e;
@@ -714,7 +720,7 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
                         const uint32_t j = plan.pd_nibble ? ((pdl[b_at >> 1] >> (4 * (b_at & 1))) & 15u) : pdl[b_at];
                         s_j[l] = j;
                         b -= plan.tab_in_smem ? s_units[l * Kp + j]
-                                              : (uint32_t)budget_cells(ktab[(size_t)l * K + j] * bpe, D, c);
+                                              : (uint32_t)budget_cells(candidate_bytes(layers[l].n, ktab.at(w, (size_t)l * K + j), bpe, cost_model, nullptr), D, c);
                     }
                 }
             }
@@ -726,36 +732,50 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
     }
     __syncthreads();
 
-    // totals, capacity check and outputs (prev/cur are free now: stage k_l and err_l there)
+    // totals, capacity check and outputs (prev/cur are free now: k_l and err_l of the chosen candidates are staged
+    // there; L <= D < the rows' size).  Entries kept and bytes are order-free integer sums; the error is added left
+    // to right in binary32.
     uint32_t* s_k = reinterpret_cast<uint32_t*>(smem_raw);
     float* s_e = reinterpret_cast<float*>(smem_raw) + rowp;
-    const bool staged = L <= rowp;
-    if (staged && status >= 0)
+    __shared__ unsigned long long s_nsel, s_used;
+    if (threadIdx.x == 0) { s_nsel = 0; s_used = 0; }
+    __syncthreads();
+    if (status >= 0) {
+        unsigned long long my_n = 0, my_b = 0;
         for (uint32_t l = threadIdx.x; l < L; l += blockDim.x) {
-            s_k[l] = (uint32_t)ktab[(size_t)l * K + s_j[l]];
-            s_e[l] = e_w[(size_t)l * K + s_j[l]];
+            const uint64_t n = layers[l].n, k = ktab.at(w, (size_t)l * K + s_j[l]);
+            bool dense;
+            my_b += candidate_bytes(n, k, bpe, cost_model, &dense);
+            const uint32_t k_eff = (uint32_t)(dense ? n : k);
+            my_n += k_eff;
+            s_k[l] = k_eff;
+            s_e[l] = dense ? 0.f : e_w[(size_t)l * K + s_j[l]];
+            if (out_dense) out_dense[(size_t)w * L + l] = dense ? 1u : 0u;
         }
+        atomicAdd(&s_nsel, my_n);
+        atomicAdd(&s_used, my_b);
+    } else if (out_dense) {
+        for (uint32_t l = threadIdx.x; l < L; l += blockDim.x) out_dense[(size_t)w * L + l] = 0u;
+    }
     __syncthreads();
     if (threadIdx.x == 0) {
-        uint64_t nsel = 0;
+        const uint64_t nsel = s_nsel;
         float tot = 0.f;
         if (status >= 0)
-            for (uint32_t l = 0; l < L; ++l) {
-                nsel += staged ? s_k[l] : ktab[(size_t)l * K + s_j[l]];
-                tot = __fadd_rn(tot, staged ? s_e[l] : e_w[(size_t)l * K + s_j[l]]);
-            }
+            for (uint32_t l = 0; l < L; ++l) tot = __fadd_rn(tot, s_e[l]);
+        if (status == KIMAD_OK && mode == 4 && s_used > c) status = KIMAD_STATUS_INFEASIBLE; // not even one entry per layer fits
         if (status >= 0 && nsel > cap) status = KIMAD_ERR_CAPACITY;
         kimad_stats s;
         s.budget_bytes = c;
         s.n_selected = status >= 0 ? nsel : 0;
-        s.used_bytes = s.n_selected * bpe;
+        s.used_bytes = status >= 0 ? s_used : 0;
         s.total_err = status >= 0 ? tot : 0.f;
         s.status = status;
         out_stats[w] = s;
         uint64_t run = 0;
         for (uint32_t l = 0; l < L; ++l) {
             out_offs[(size_t)w * (L + 1) + l] = run;
-            if (status >= 0) run += staged ? s_k[l] : ktab[(size_t)l * K + s_j[l]];
+            if (status >= 0) run += s_k[l];
         }
         out_offs[(size_t)w * (L + 1) + L] = run;
         s_status = status;
@@ -768,13 +788,12 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
         Sel s;
         if (status >= 0) {
             const uint32_t j = s_j[l];
-            const uint64_t k = ktab[(size_t)l * K + j];
             s.tau = tau[wl * K + j];
             s.keep_eq = keep_eq[wl * K + j];
-            s.k = (uint32_t)k;
+            s.k = s_k[l];
             s.shift = shift ? shift[wl * K + j] : 0u;
             s.base = out_offs[(size_t)w * (L + 1) + l];
-            out_k[wl] = (uint32_t)k;
+            out_k[wl] = s_k[l];
             out_j[wl] = j;
         } else {
             s.tau = 0; s.keep_eq = 0; s.k = 0; s.shift = 0; s.base = 0;
@@ -785,6 +804,45 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
         s._pad = 0;
         sel[wl] = s;
     }
+}
+
+// The ratio of Section 3.1 sized to the budget: r = q / 2^32 with the largest q whose entries
+// sum_l min(n_l, max(1, floor(q n_l / 2^32))) fit floor(c / (4 + vb)); the worker's table row gets those k_l.
+// One CTA per worker; the sum is an order-free integer reduction, q is found by bisection (33 steps).
+__global__ void __launch_bounds__(kThreads)
+k_fit_ratio(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t bpe, uint64_t N,
+            const LayerDesc* __restrict__ layers, uint64_t* __restrict__ ktab_w /* [W][L] */) {
+    pdl_wait();
+    const uint32_t w = w_base + blockIdx.x;
+    if (w >= W) return;
+    __shared__ unsigned long long s_sum;
+    const uint64_t entries = budgets.c[blockIdx.x] / bpe;
+    auto k_of = [&](uint64_t q, uint64_t n) {
+        uint64_t k = q >= 4294967296ull ? n : (q * n) >> 32;
+        k = k < 1 ? 1 : k;
+        return k > n ? n : k;
+    };
+    uint64_t q;
+    if (entries < (uint64_t)L) q = 0;
+    else if (entries >= N) q = 4294967296ull;
+    else {
+        uint64_t lo = 0, hi = 4294967296ull; // sum(lo) <= entries < sum(hi)
+        while (hi - lo > 1) {
+            const uint64_t mid = lo + (hi - lo) / 2;
+            if (threadIdx.x == 0) s_sum = 0;
+            __syncthreads();
+            unsigned long long mine = 0;
+            for (uint32_t l = threadIdx.x; l < L; l += kThreads) mine += k_of(mid, layers[l].n);
+#pragma unroll
+            for (int o = 16; o; o >>= 1) mine += __shfl_xor_sync(0xffffffffu, mine, o);
+            if ((threadIdx.x & 31) == 0) atomicAdd(&s_sum, mine);
+            __syncthreads();
+            if (s_sum <= entries) lo = mid; else hi = mid;
+            __syncthreads();
+        }
+        q = lo;
+    }
+    for (uint32_t l = threadIdx.x; l < L; l += kThreads) ktab_w[(size_t)w * L + l] = k_of(q, layers[l].n);
 }
 
 } // namespace kimad

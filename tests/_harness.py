@@ -17,15 +17,15 @@ def u32(t):
 
 class Runner:
     def __init__(self, layer_sizes, W, grid, D=1000, value_dtype=0, stride=None, cap=None, check_finite=0,
-                 curve_mode=0, policy=0):
+                 curve_mode=0, policy=0, cost_model=0):
         self.ls, self.W, self.grid, self.D, self.vd = list(layer_sizes), W, list(grid), D, value_dtype
-        self.policy = policy
+        self.policy, self.cost_model = policy, cost_model
         self.N = int(sum(self.ls))
         self.stride = stride or self.N
         self.cap = cap or self.N
         self.ctx = kb.new_context(self.ls, W, self.grid, D=D, value_dtype=value_dtype, worker_stride=self.stride,
                                   max_packed_elems=self.cap, check_finite=check_finite, curve_mode=curve_mode,
-                                  policy=policy)
+                                  policy=policy, cost_model=cost_model)
         self.out = kb.Packed(self.ctx)
         self.kt = ko.k_table(self.ls, self.grid)
 
@@ -45,12 +45,15 @@ class Runner:
         tau_s, keq_s = kb.kimad_debug_get_selection(self.ctx)
         # oracle on its own curves
         ref = ko.step(self.ls, W, self.grid, self.D, self.vd, g_host, s_host, bw, t, cap=self.cap,
-                      policy=self.policy)
+                      policy=self.policy, cost_model=self.cost_model)
         # (b) curve: thresholds exact, error within tolerance
         # where all 31 bits were resolved the threshold must be the oracle's; elsewhere the oracle's
         # threshold must lie in the reported key interval
         exact = shift_g == 0
-        full = np.broadcast_to((self.kt == np.array(self.ls, np.uint64)[:, None])[None], exact.shape)  # k = n: no threshold
+        if self.policy == 3:  # the one candidate of every (worker, layer) is the ratio fitted to the worker's budget
+            full = (ref.k == np.array(self.ls, np.uint32)[None, :])[:, :, None]
+        else:
+            full = np.broadcast_to((self.kt == np.array(self.ls, np.uint64)[:, None])[None], exact.shape)  # k = n: no threshold
         chk = exact & ~full
         assert np.array_equal(tau_g[chk], ref.tau[chk]), "tau differs"
         assert np.array_equal(keq_g[chk], ref.keep_eq[chk]), "keep_eq differs"
@@ -64,11 +67,12 @@ class Runner:
         assert not bad.any(), f"err off at {np.argwhere(bad)[:5]}: {err_g[bad][:5]} vs {ref.err[bad][:5]}"
         # (c)-(f): oracle DP fed the GPU's curve must reproduce the GPU bit for bit
         forced = ko.step(self.ls, W, self.grid, self.D, self.vd, g_host, s_host, bw, t, cap=self.cap,
-                         inject_err=err_g, policy=self.policy)
+                         inject_err=err_g, policy=self.policy, cost_model=self.cost_model)
         st = self.out.stats_host()
         assert np.array_equal(st["status"], forced.status), (st["status"], forced.status)
         assert np.array_equal(u32(self.out.j), forced.j), "chosen candidates differ from oracle DP on the same curve"
         assert np.array_equal(k_gpu, forced.k)
+        assert np.array_equal(u32(self.out.dense), forced.dense), "dense flags differ"
         # the exact threshold found for the chosen candidate of every layer
         jj = forced.j.astype(np.int64)
         t_ref = np.take_along_axis(ref.tau, jj[:, :, None], axis=2)[:, :, 0]
