@@ -1,6 +1,7 @@
 """Parity at the benchmark's full sizes, in the launch configuration bench.py times.
 
-The oracle cannot sort a whole 0.5-2 G element step in test time, so: (1) for a sample of layers (always
+Every element: workload 4 (all layers of all workers) and one whole worker of workload 5 go through the oracle's
+complete pass and everything is compared.  The quicker sampled variant below stays as well: (1) for a sample of layers (always
 including the largest one) the oracle computes curve, threshold, packed entries and state one layer at a
 time and every value is compared; (2) the DP is re-run by the oracle on the GPU's complete curve; (3)
 properties that hold at any size are checked on ALL layers: counts, offsets, ascending indices, values
@@ -108,6 +109,88 @@ def _full_size_step(cfg, step_of_trace, sample_layers, workers_checked):
                     assert np.array_equal(ov.view(np.int16 if wl.value_dtype else np.int32), val_all[a:b])
         del d, g_old, g_new
     return kb.kimad_debug_exact_path_layers(ctx, detail=True)
+
+
+def _every_element(cfg, step_of_trace, workers):
+    """One full-size step in the benchmark's launch configuration, EVERY element of the listed workers compared
+    with the oracle's whole pass (curves of all layers and candidates to the curve tolerance; decisions, packed
+    indices and values, offsets, statistics and the EF21 state bit for bit)."""
+    wl = workloads.workload(cfg)
+    W, N, L = wl.n_workers, wl.N, wl.L
+    bw_all = workloads.bandwidth_trace(wl)
+    bw = bw_all[step_of_trace]
+    bpe = 8 if wl.value_dtype == 0 else 6
+    cap = int(min(N, np.max(bw_all) * wl.t_target / bpe + L + 1))  # as bench.py sizes the packed buffers
+    ctx = kb.new_context(wl.layer_sizes, W, wl.ratio_grid, D=wl.D, value_dtype=wl.value_dtype, max_packed_elems=cap)
+    out = kb.Packed(ctx)
+    state = torch.zeros((W, N), dtype=torch.float32, device="cuda")
+    g0 = workloads.gradients(wl, 0, device="cuda")
+    kb.kimad_step(ctx, g0, state, bw_all[0], wl.t_target, out)  # an earlier step: the EF state is not all zero
+    del g0
+    grads = workloads.gradients(wl, 1, device="cuda")
+    state_before = state.clone()
+    kb.kimad_step(ctx, grads, state, bw, wl.t_target, out)
+    status, k_gpu = kb.kimad_get_k(ctx)
+    assert status == 0
+    err_g, tau_g, keq_g, shift_g = kb.kimad_debug_get_curve(ctx)
+    tau_s, keq_s = kb.kimad_debug_get_selection(ctx)
+    st = out.stats_host()
+    j_gpu = out.j.cpu().numpy().view(np.uint32)
+    offs_g = out.offs.cpu().numpy().astype(np.uint64)
+    sizes = np.array(wl.layer_sizes, np.uint32)
+    kt = ko.k_table(wl.layer_sizes, wl.ratio_grid)
+    for w in workers:
+        g_host = grads[w:w + 1].cpu().numpy()
+        s_host = state_before[w:w + 1].cpu().numpy()
+        ref = ko.step(wl.layer_sizes, 1, wl.ratio_grid, wl.D, wl.value_dtype, g_host, s_host, [bw[w]], wl.t_target,
+                      cap=cap)
+        # (b) the curve of every layer and candidate
+        tol = 1e-5 * np.abs(ref.err[0].astype(np.float64))
+        bad = (err_g[w] != ref.err[0]) & ~(np.abs(err_g[w].astype(np.float64) - ref.err[0].astype(np.float64)) <= tol)
+        assert not bad.any(), np.argwhere(bad)[:5]
+        full = kt == sizes[:, None].astype(np.uint64)
+        ex = (shift_g[w] == 0) & ~full
+        assert np.array_equal(tau_g[w][ex], ref.tau[0][ex]) and np.array_equal(keq_g[w][ex], ref.keep_eq[0][ex])
+        lazy = (shift_g[w] != 0) & ~full
+        assert np.all((ref.tau[0][lazy] >= tau_g[w][lazy]) &
+                      (ref.tau[0][lazy] - tau_g[w][lazy] < (1 << shift_g[w][lazy].astype(np.uint64))))
+        # (c) decisions: the oracle's own curve must lead to the same k here; if the two curves (equal within the
+        # tolerance) ever led to different decisions, the oracle's DP is run on the GPU's curve instead
+        if not np.array_equal(ref.k[0], k_gpu[w]):
+            ref = ko.step(wl.layer_sizes, 1, wl.ratio_grid, wl.D, wl.value_dtype, g_host, s_host, [bw[w]],
+                          wl.t_target, cap=cap, inject_err=err_g[w:w + 1])
+        assert np.array_equal(ref.j[0], j_gpu[w]) and np.array_equal(ref.k[0], k_gpu[w])
+        assert np.array_equal(ref.offs[0], offs_g[w])
+        assert int(st["status"][w]) == int(ref.status[0]) and int(st["used_bytes"][w]) == int(ref.used_bytes[0])
+        assert int(st["n_selected"][w]) == int(ref.n_selected[0]) and int(st["budget_bytes"][w]) == int(ref.budget_bytes[0])
+        # (d) exact thresholds of the chosen candidates
+        jj = ref.j[0].astype(np.int64)
+        part = (ref.k[0] > 0) & (ref.k[0] < sizes)
+        assert np.array_equal(tau_s[w][part], ref.tau[0][np.arange(L), jj][part])
+        assert np.array_equal(keq_s[w][part], ref.keep_eq[0][np.arange(L), jj][part])
+        # (e) + (f) every packed entry and every element of the state
+        n = int(ref.offs[0, L])
+        assert np.array_equal(out.idx[w, :n].cpu().numpy().view(np.uint32), ref.idx[0, :n])
+        val_g = out.val[w, :n].view(torch.int16 if wl.value_dtype else torch.int32).cpu().numpy()
+        assert np.array_equal(val_g, ref.val[0, :n].view(np.int16 if wl.value_dtype else np.int32))
+        assert np.array_equal(state[w].cpu().numpy().view(np.uint32), ref.state[0].view(np.uint32))
+        del g_host, s_host, ref
+
+
+def test_gpt2_small_shape_full_size_every_element():
+    # all 148 layers of all 4 workers (4 x 124.4 M elements), a low-budget step of the trace
+    _every_element(4, step_of_trace=7, workers=[0, 1, 2, 3])
+
+
+def test_gpt2_small_shape_full_size_every_element_burst():
+    # a burst of the trace (25 Gbit/s: about 16 % of the entries kept), one worker
+    bw = workloads.bandwidth_trace(workloads.workload(4))
+    _every_element(4, step_of_trace=int(np.argmax(bw[:, 0])), workers=[2])
+
+
+def test_llama_1b_shape_full_size_every_element_of_one_worker():
+    # all 201 layers of one worker (1.1 G elements, bf16 values)
+    _every_element(5, step_of_trace=30, workers=[1])
 
 
 def test_gpt2_small_shape_full_size():
