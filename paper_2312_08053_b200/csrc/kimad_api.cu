@@ -39,6 +39,7 @@ struct kimad_ctx {
     std::vector<Chunk> chunks;
     std::vector<LayerDesc> layers;
     std::vector<uint32_t> reg_layers, tiny_layers, reg_index; // layers above / up to kTinyMax elements
+    std::vector<unsigned char> static_image;                  // the static tables as they lie in the workspace, one block
     uint32_t curve_mode = 0;
     uint32_t policy = 0, cost_model = 0;
     size_t sample_smem = 0, pass_a_smem = 0, tiny_smem = 0;
@@ -156,6 +157,25 @@ static int ensure_side_stream(kimad_ctx* c) {
     CUDA_TRY(cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming));
     CUDA_TRY(cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming));
     return KIMAD_OK;
+}
+
+// Once per device and process: shared-memory limits of the kernels (a property of the function, shared by all
+// contexts: the limits do not depend on the context) and the kernel preload.  Per context: its side stream.
+static int prepare_device(kimad_ctx* c) {
+    static bool ready[KIMAD_BUILTIN_MAX_DEVICES] = {};
+    int dev = -1;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= KIMAD_BUILTIN_MAX_DEVICES) return KIMAD_ERR_INVALID_ARG;
+    if (!ready[dev]) {
+        CUDA_TRY(cudaFuncSetAttribute(k_dp, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDpSmemMax));
+        CUDA_TRY(cudaFuncSetAttribute(k_sample, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->sample_smem));
+        CUDA_TRY(cudaFuncSetAttribute(k_pass_a<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->pass_a_smem));
+        CUDA_TRY(cudaFuncSetAttribute(k_pass_a<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->pass_a_smem));
+        CUDA_TRY(cudaFuncSetAttribute(k_tiny_exact, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->tiny_smem));
+        { const int rc_pre = preload_kernels(); if (rc_pre != KIMAD_OK) return rc_pre; }
+        ready[dev] = true;
+    }
+    return ensure_side_stream(c);
 }
 
 enum StepMode { kNormal = 0, kInjectErr = 1, kGivenJ = 2 };
@@ -416,6 +436,17 @@ int kimad_create(kimad_ctx** out, const uint64_t* layer_sizes, uint32_t n_layers
         c->pass_a_smem = (size_t)(3 * kMaxBins + kLutWords) * 4 + kL1Bins * 2;
         c->tiny_smem = (size_t)kTinyMax * (8 + 4);
         plan_layout(c);
+        { // host image of the static tables [chunks, zero_from): attached workspaces get it in one copy
+            const Layout& y = c->lay;
+            c->static_image.assign(y.zero_from - y.chunks, 0);
+            unsigned char* im = c->static_image.data() - y.chunks;
+            std::memcpy(im + y.chunks, c->chunks.data(), c->chunks.size() * sizeof(Chunk));
+            std::memcpy(im + y.layers, c->layers.data(), c->layers.size() * sizeof(LayerDesc));
+            std::memcpy(im + y.ktab, c->ktab.data(), c->ktab.size() * sizeof(uint64_t));
+            if (!c->reg_layers.empty()) std::memcpy(im + y.reg_layers, c->reg_layers.data(), c->reg_layers.size() * 4);
+            if (!c->tiny_layers.empty()) std::memcpy(im + y.tiny_layers, c->tiny_layers.data(), c->tiny_layers.size() * 4);
+            std::memcpy(im + y.reg_index, c->reg_index.data(), c->reg_index.size() * 4);
+        }
     } catch (const std::bad_alloc&) {
         delete c;
         return KIMAD_ERR_NOMEM;
@@ -460,24 +491,10 @@ int kimad_set_workspace(kimad_ctx* c, void* dev_ptr, size_t bytes) {
     if (!dev_ptr || bytes < c->lay.total || (uintptr_t)dev_ptr % kAlign) return KIMAD_ERR_WORKSPACE;
     c->ws = static_cast<unsigned char*>(dev_ptr);
     const Layout& y = c->lay;
-    CUDA_TRY(cudaMemcpy(c->ws + y.chunks, c->chunks.data(), c->chunks.size() * sizeof(Chunk), cudaMemcpyHostToDevice));
-    CUDA_TRY(cudaMemcpy(c->ws + y.layers, c->layers.data(), c->layers.size() * sizeof(LayerDesc), cudaMemcpyHostToDevice));
-    CUDA_TRY(cudaMemcpy(c->ws + y.ktab, c->ktab.data(), c->ktab.size() * sizeof(uint64_t), cudaMemcpyHostToDevice));
-    if (!c->reg_layers.empty())
-        CUDA_TRY(cudaMemcpy(c->ws + y.reg_layers, c->reg_layers.data(), c->reg_layers.size() * 4, cudaMemcpyHostToDevice));
-    if (!c->tiny_layers.empty())
-        CUDA_TRY(cudaMemcpy(c->ws + y.tiny_layers, c->tiny_layers.data(), c->tiny_layers.size() * 4, cudaMemcpyHostToDevice));
-    CUDA_TRY(cudaMemcpy(c->ws + y.reg_index, c->reg_index.data(), c->reg_index.size() * 4, cudaMemcpyHostToDevice));
+    CUDA_TRY(cudaMemcpy(c->ws + y.chunks, c->static_image.data(), c->static_image.size(), cudaMemcpyHostToDevice));
     // histograms, work lists and flags start at zero and are kept clean by the kernels that consume them
     CUDA_TRY(cudaMemset(c->ws + y.zero_from, 0, y.lut_t1 - y.zero_from));
-    // the limit is a property of the function, shared by all contexts: raise it to the largest plan, not to this one's
-    CUDA_TRY(cudaFuncSetAttribute(k_dp, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDpSmemMax));
-    CUDA_TRY(cudaFuncSetAttribute(k_sample, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->sample_smem));
-    CUDA_TRY(cudaFuncSetAttribute(k_pass_a<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->pass_a_smem));
-    CUDA_TRY(cudaFuncSetAttribute(k_pass_a<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->pass_a_smem));
-    CUDA_TRY(cudaFuncSetAttribute(k_tiny_exact, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->tiny_smem));
-    { const int rc_side = ensure_side_stream(c); if (rc_side != KIMAD_OK) return rc_side; }
-    { const int rc_pre = preload_kernels(); if (rc_pre != KIMAD_OK) return rc_pre; }
+    { const int rc_dev = prepare_device(c); if (rc_dev != KIMAD_OK) return rc_dev; }
     CUDA_TRY(cudaDeviceSynchronize());
     return KIMAD_OK;
 }
@@ -687,7 +704,10 @@ static unsigned char* g_builtin_ptr[KIMAD_BUILTIN_MAX_DEVICES] = {};
 
 int kimad_step_builtin_scratch(kimad_ctx* c, const float* grads_dev, float* state_dev, const double* bandwidth_bytes_per_s,
                                double t_target_s, const kimad_packed* out, void* cuda_stream) {
-    if (!c) return KIMAD_ERR_INVALID_ARG;
+    // arguments first: nothing of the shared array is touched by a call that is going to be refused
+    if (!c || !grads_dev || !state_dev || !bandwidth_bytes_per_s || !out || !out->idx || !out->val || !out->offs || !out->k ||
+        !out->j || !out->stats || !(t_target_s >= 0.0))
+        return KIMAD_ERR_INVALID_ARG;
     if (c->lay.total > (size_t)KIMAD_BUILTIN_SCRATCH_BYTES) return KIMAD_ERR_TOO_LARGE;
     int dev = -1;
     CUDA_TRY(cudaGetDevice(&dev));
@@ -697,28 +717,14 @@ int kimad_step_builtin_scratch(kimad_ctx* c, const float* grads_dev, float* stat
         CUDA_TRY(cudaGetSymbolAddress(&p, g_builtin_scratch));
         g_builtin_ptr[dev] = static_cast<unsigned char*>(p);
     }
+    { const int rc_dev = prepare_device(c); if (rc_dev != KIMAD_OK) return rc_dev; } // once per device / per context
     unsigned char* ws = g_builtin_ptr[dev];
     cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
-    // The array keeps whatever the previous call (of any context) left: bring in this context's tables and
-    // clear everything that has to start at zero, in stream order before the kernels.
+    // The array keeps whatever the previous call (of any context) left: bring in this context's tables (one block)
+    // and clear everything that has to start at zero, in stream order before the kernels.
     const Layout& y = c->lay;
-    CUDA_TRY(cudaMemcpyAsync(ws + y.chunks, c->chunks.data(), c->chunks.size() * sizeof(Chunk), cudaMemcpyHostToDevice, s));
-    CUDA_TRY(cudaMemcpyAsync(ws + y.layers, c->layers.data(), c->layers.size() * sizeof(LayerDesc), cudaMemcpyHostToDevice, s));
-    CUDA_TRY(cudaMemcpyAsync(ws + y.ktab, c->ktab.data(), c->ktab.size() * sizeof(uint64_t), cudaMemcpyHostToDevice, s));
-    if (!c->reg_layers.empty())
-        CUDA_TRY(cudaMemcpyAsync(ws + y.reg_layers, c->reg_layers.data(), c->reg_layers.size() * 4, cudaMemcpyHostToDevice, s));
-    if (!c->tiny_layers.empty())
-        CUDA_TRY(cudaMemcpyAsync(ws + y.tiny_layers, c->tiny_layers.data(), c->tiny_layers.size() * 4, cudaMemcpyHostToDevice, s));
-    CUDA_TRY(cudaMemcpyAsync(ws + y.reg_index, c->reg_index.data(), c->reg_index.size() * 4, cudaMemcpyHostToDevice, s));
+    CUDA_TRY(cudaMemcpyAsync(ws + y.chunks, c->static_image.data(), c->static_image.size(), cudaMemcpyHostToDevice, s));
     CUDA_TRY(cudaMemsetAsync(ws + y.zero_from, 0, y.lut_t1 - y.zero_from, s));
-    // the limit is a property of the function, shared by all contexts: raise it to the largest plan, not to this one's
-    CUDA_TRY(cudaFuncSetAttribute(k_dp, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDpSmemMax));
-    CUDA_TRY(cudaFuncSetAttribute(k_sample, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->sample_smem));
-    CUDA_TRY(cudaFuncSetAttribute(k_pass_a<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->pass_a_smem));
-    CUDA_TRY(cudaFuncSetAttribute(k_pass_a<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->pass_a_smem));
-    CUDA_TRY(cudaFuncSetAttribute(k_tiny_exact, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->tiny_smem));
-    { const int rc_side = ensure_side_stream(c); if (rc_side != KIMAD_OK) return rc_side; }
-    { const int rc_pre = preload_kernels(); if (rc_pre != KIMAD_OK) return rc_pre; }
     unsigned char* caller_ws = c->ws; // the context's own workspace (if any) is left untouched
     c->ws = ws;
     const int rc = run_step(c, grads_dev, state_dev, bandwidth_bytes_per_s, t_target_s, out, cuda_stream, kNormal, nullptr,

@@ -1,9 +1,9 @@
 """Parity at the benchmark's full sizes, in the launch configuration bench.py times.
 
 Every element: workload 4 (all layers of all workers) and one whole worker of workload 5 go through the oracle's
-complete pass and everything is compared.  The quicker sampled variant below stays as well: (1) for a sample of layers (always
-including the largest one) the oracle computes curve, threshold, packed entries and state one layer at a
-time and every value is compared; (2) the DP is re-run by the oracle on the GPU's complete curve; (3)
+complete pass and everything is compared.  The quicker sampled variant below stays as well: (1) for a sample of
+layers (always including the largest one) the oracle computes curve, threshold, packed entries and state one
+layer at a time and every value is compared; (2) the DP is re-run by the oracle on the GPU's complete curve; (3)
 properties that hold at any size are checked on ALL layers: counts, offsets, ascending indices, values
 equal to d at the indices, no dropped entry larger than a kept one, untouched entries of the state."""
 import numpy as np
@@ -191,6 +191,26 @@ def test_gpt2_small_shape_full_size_every_element_burst():
 def test_llama_1b_shape_full_size_every_element_of_one_worker():
     # all 201 layers of one worker (1.1 G elements, bf16 values)
     _every_element(5, step_of_trace=30, workers=[1])
+
+
+@pytest.mark.parametrize("block,D", [(65536, 4096), (16384, 8191)])
+def test_gpt2_small_shape_full_size_in_blocks(block, D):
+    """Block granularity (the paper's Section 5: from layers to blocks) on a full-size workload: the GPT-2-small
+    shaped gradient of one worker (124.4 M elements) cut into blocks of 64 K and of 16 K elements (1995 and 7686
+    segments; every segment takes at least one budget cell, so D >= segments), every element compared."""
+    from tests._harness import Runner
+
+    wl = workloads.workload(4)
+    blocks = workloads.block_layers(wl.layer_sizes, block)
+    assert sum(blocks) == wl.N and max(blocks) == block and len(blocks) <= D
+    r = Runner(blocks, 1, wl.ratio_grid, D, 0)
+    grads = workloads.gradients(wl, 3, device="cuda", workers=[1])
+    state = (workloads.gradients(wl, 2, device="cuda", workers=[1]) * 0.5).contiguous()  # a non-trivial estimator
+    bw = workloads.bandwidth_trace(wl)
+    res = r.compare_step(grads, state, [float(bw[int(np.argmax(bw[:, 0])), 0]) * 0.3], wl.t_target, check_inject=False)
+    assert res["status"] == 0
+    k = res["forced"].k[0]
+    assert len(set(k.tolist())) > 3  # the blocks of one tensor do not all get the same k
 
 
 def test_gpt2_small_shape_full_size():
