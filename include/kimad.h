@@ -284,6 +284,14 @@ int kimad_debug_get_band_meta(kimad_ctx* ctx, uint32_t* host_meta);
 int kimad_debug_enable_stage_timing(kimad_ctx* ctx, int enable);
 int kimad_debug_stage_times(kimad_ctx* ctx, float* host_ms);
 
+/* Checked build of the library (compiled with -DKIMAD_CHECKED; the stand-in for a memory checker): the kernels
+ * test their indices into the workspace and the output buffers before use -- a failed test sets its bit in a
+ * status word and the access is skipped, nothing traps -- and the workspace regions are separated by canary words.
+ * kimad_debug_check synchronises the device and reports the status word (0: no test failed since the library was
+ * loaded) and the number of canaries of ctx's attached workspace that no longer hold their pattern.  Returns 1 in
+ * a checked build, 0 in an ordinary build (both outputs are then 0), < 0 on error.  Either pointer may be NULL. */
+int kimad_debug_check(kimad_ctx* ctx, uint32_t* failed_checks, uint32_t* damaged_canaries);
+
 /* Kernels launched by this context so far (for launch accounting in benchmarks). */
 uint64_t kimad_launch_count(const kimad_ctx* ctx);
 /* Static description of a code returned by this library. */

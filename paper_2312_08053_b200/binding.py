@@ -56,7 +56,8 @@ class KimadError(RuntimeError):
 
 
 def lib_path() -> str:
-    return _build.LIB_PATH
+    """The ordinary build, or the checked build when the environment has KIMAD_CHECKED=1."""
+    return _build.CHECKED_LIB_PATH if os.environ.get("KIMAD_CHECKED") == "1" else _build.LIB_PATH
 
 
 def load():
@@ -110,6 +111,8 @@ def load():
     L.kimad_debug_get_band_meta.argtypes = [vp, vp]
     L.kimad_debug_exact_path_layers.restype = C.c_int
     L.kimad_debug_exact_path_layers.argtypes = [vp, C.POINTER(u64)]
+    L.kimad_debug_check.restype = C.c_int
+    L.kimad_debug_check.argtypes = [vp, C.POINTER(u32), C.POINTER(u32)]
     L.kimad_launch_count.restype = u64
     L.kimad_launch_count.argtypes = [vp]
     L.kimad_monitor_create.restype = C.c_int
@@ -334,6 +337,13 @@ def kimad_debug_exact_path_layers(ctx: Ctx, detail: bool = False):
     n = (C.c_uint64 * (5 + ctx.K))()
     _check(load().kimad_debug_exact_path_layers(ctx.handle, n), "kimad_debug_exact_path_layers")
     return [int(x) for x in n] if detail else int(n[0])
+
+
+def kimad_debug_check(ctx: Ctx):
+    """Returns (checked build?, failed-check bits, damaged canaries) -- see kimad.h."""
+    w, b = C.c_uint32(0), C.c_uint32(0)
+    rc = _check(load().kimad_debug_check(ctx.handle, C.byref(w), C.byref(b)), "kimad_debug_check")
+    return bool(rc), int(w.value), int(b.value)
 
 
 def kimad_launch_count(ctx: Ctx) -> int:

@@ -15,6 +15,7 @@ using namespace kimad;
 namespace {
 
 constexpr size_t kAlign = 256;
+constexpr int kCanaryByte = 0xA5; // checked build: fill of the guard words between workspace regions
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
@@ -40,6 +41,7 @@ struct kimad_ctx {
     std::vector<LayerDesc> layers;
     std::vector<uint32_t> reg_layers, tiny_layers, reg_index; // layers above / up to kTinyMax elements
     std::vector<unsigned char> static_image;                  // the static tables as they lie in the workspace, one block
+    std::vector<size_t> guards;                               // checked build: offsets of the canary words between regions
     uint32_t curve_mode = 0;
     uint32_t policy = 0, cost_model = 0;
     size_t sample_smem = 0, pass_a_smem = 0, tiny_smem = 0;
@@ -65,7 +67,16 @@ namespace {
 void plan_layout(kimad_ctx* c) {
     Layout& y = c->lay;
     size_t o = 0;
-    auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes); return at; };
+    c->guards.clear();
+    auto take = [&](size_t bytes) {
+        size_t at = o;
+        o = align_up(o + bytes);
+#ifdef KIMAD_CHECKED
+        c->guards.push_back(o); // a canary of kAlign bytes behind every region
+        o += kAlign;
+#endif
+        return at;
+    };
     const size_t WL = (size_t)c->W * c->L, WLK = WL * c->K, WR = (size_t)c->W * c->reg_layers.size();
     const size_t nch = c->chunks.size();
     y.dbuf = take((size_t)c->W * c->dstride * sizeof(uint16_t));
@@ -178,6 +189,12 @@ static int prepare_device(kimad_ctx* c) {
     return ensure_side_stream(c);
 }
 
+// Checked build: (re)writes the canaries of a workspace, in stream order.  A no-op otherwise (no guards are planned).
+static int fill_guards(const kimad_ctx* c, unsigned char* ws, cudaStream_t s) {
+    for (size_t g : c->guards) CUDA_TRY(cudaMemsetAsync(ws + g, kCanaryByte, kAlign, s));
+    return KIMAD_OK;
+}
+
 enum StepMode { kNormal = 0, kInjectErr = 1, kGivenJ = 2 };
 
 int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, double t, const kimad_packed* out,
@@ -287,7 +304,7 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
     mark();
     if (R) {
         CUDA_TRY(launch_pdl(k_resolve_a, dim3(R, W), kBigThreads, 0, s, layers, reg_layers, R, L, ktab, K, meta, binlo, bhc, bhs, err, tau,
-                                                       keq, shf, flags, fb, fb_chunks, fb_layers));
+                                                       keq, shf, flags, fb, fb_chunks, fb_layers, nch));
         c->launches += 1;
     }
     if (T) CUDA_TRY(cudaStreamWaitEvent(s, c->ev_join, 0));
@@ -446,6 +463,8 @@ int kimad_create(kimad_ctx** out, const uint64_t* layer_sizes, uint32_t n_layers
             if (!c->reg_layers.empty()) std::memcpy(im + y.reg_layers, c->reg_layers.data(), c->reg_layers.size() * 4);
             if (!c->tiny_layers.empty()) std::memcpy(im + y.tiny_layers, c->tiny_layers.data(), c->tiny_layers.size() * 4);
             std::memcpy(im + y.reg_index, c->reg_index.data(), c->reg_index.size() * 4);
+            for (size_t g : c->guards)
+                if (g >= y.chunks && g + kAlign <= y.zero_from) std::memset(im + g, kCanaryByte, kAlign);
         }
     } catch (const std::bad_alloc&) {
         delete c;
@@ -494,6 +513,7 @@ int kimad_set_workspace(kimad_ctx* c, void* dev_ptr, size_t bytes) {
     CUDA_TRY(cudaMemcpy(c->ws + y.chunks, c->static_image.data(), c->static_image.size(), cudaMemcpyHostToDevice));
     // histograms, work lists and flags start at zero and are kept clean by the kernels that consume them
     CUDA_TRY(cudaMemset(c->ws + y.zero_from, 0, y.lut_t1 - y.zero_from));
+    { const int rc_g = fill_guards(c, c->ws, nullptr); if (rc_g != KIMAD_OK) return rc_g; }
     { const int rc_dev = prepare_device(c); if (rc_dev != KIMAD_OK) return rc_dev; }
     CUDA_TRY(cudaDeviceSynchronize());
     return KIMAD_OK;
@@ -637,6 +657,30 @@ int kimad_debug_exact_path_layers(kimad_ctx* c, uint64_t* host_count) {
     return KIMAD_OK;
 }
 
+int kimad_debug_check(kimad_ctx* c, uint32_t* failed_checks, uint32_t* damaged_canaries) {
+    if (!c) return KIMAD_ERR_INVALID_ARG;
+    if (failed_checks) *failed_checks = 0;
+    if (damaged_canaries) *damaged_canaries = 0;
+#ifdef KIMAD_CHECKED
+    if (!c->ws) return KIMAD_ERR_WORKSPACE;
+    CUDA_TRY(cudaDeviceSynchronize());
+    unsigned int word = 0;
+    CUDA_TRY(cudaMemcpyFromSymbol(&word, g_kimad_check_word, sizeof(word)));
+    if (failed_checks) *failed_checks = word;
+    uint32_t bad = 0;
+    unsigned char buf[kAlign];
+    for (size_t g : c->guards) {
+        CUDA_TRY(cudaMemcpy(buf, c->ws + g, kAlign, cudaMemcpyDeviceToHost));
+        for (size_t i = 0; i < kAlign; ++i)
+            if (buf[i] != (unsigned char)kCanaryByte) { ++bad; break; }
+    }
+    if (damaged_canaries) *damaged_canaries = bad;
+    return 1;
+#else
+    return 0;
+#endif
+}
+
 uint64_t kimad_launch_count(const kimad_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
 // ---------------------------------------------------------------------------------------------------
@@ -725,6 +769,7 @@ int kimad_step_builtin_scratch(kimad_ctx* c, const float* grads_dev, float* stat
     const Layout& y = c->lay;
     CUDA_TRY(cudaMemcpyAsync(ws + y.chunks, c->static_image.data(), c->static_image.size(), cudaMemcpyHostToDevice, s));
     CUDA_TRY(cudaMemsetAsync(ws + y.zero_from, 0, y.lut_t1 - y.zero_from, s));
+    { const int rc_g = fill_guards(c, ws, s); if (rc_g != KIMAD_OK) return rc_g; }
     unsigned char* caller_ws = c->ws; // the context's own workspace (if any) is left untouched
     c->ws = ws;
     const int rc = run_step(c, grads_dev, state_dev, bandwidth_bytes_per_s, t_target_s, out, cuda_stream, kNormal, nullptr,

@@ -10,6 +10,19 @@
 #define KIMAD_HD inline
 #endif
 
+// Checked build (-DKIMAD_CHECKED): indices into the workspace and the output buffers are tested before use; a failed
+// test sets its bit in a status word that the host reads (kimad_debug_check) and the access is skipped -- nothing
+// traps.  Bits: 0 sweep: bin outside the layer's histogram; 1 counting sweep: bin outside the in-interval histogram;
+// 2 a work list (exact path, second select round, recount) appended beyond its capacity; 3 write sweep: packed
+// position beyond the capacity; 4 write sweep: element index outside its layer; 5 DP: cell or back-pointer outside
+// its row; 6 curve: bin outside the layer's histogram.  In the ordinary build KIMAD_CHECK(cond, bit) is `true`.
+#if defined(KIMAD_CHECKED) && defined(__CUDACC__)
+__device__ unsigned int g_kimad_check_word;
+#define KIMAD_CHECK(cond, bit) ((cond) ? true : (atomicOr(&g_kimad_check_word, 1u << (bit)), false))
+#else
+#define KIMAD_CHECK(cond, bit) (true)
+#endif
+
 namespace kimad {
 
 // A chunk is the part of one layer that falls inside one aligned window of kChunkElems elements of

@@ -424,6 +424,7 @@ k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, uint1
         // 24 significant bits of the square (truncation < 2^-22 relative) summed exactly: the low word wraps, the
         // returned old value tells when, and the wraps are counted in the high word
         const uint32_t sq = (uint32_t)(sq_fixed(key) >> 8);
+        if (!KIMAD_CHECK(id < n_bins, 0)) return;
         atomicAdd(&h_cnt[id], 1u);
         const uint32_t old = atomicAdd(&h_lo[id], sq);
         if (old + sq < old) atomicAdd(&h_hi[id], 1u); // carry out of the low word (rare)
@@ -521,7 +522,7 @@ k_resolve_a(const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ r
             const uint32_t* __restrict__ bin_lo, uint32_t* __restrict__ bh_cnt, unsigned long long* __restrict__ bh_sum,
             float* __restrict__ err_out, uint32_t* __restrict__ tau_out, uint32_t* __restrict__ rank_out,
             uint32_t* __restrict__ shift_out, uint32_t* __restrict__ flags, FbList* __restrict__ fb,
-            uint2* __restrict__ fb_chunks, uint2* __restrict__ fb_layers) {
+            uint2* __restrict__ fb_chunks, uint2* __restrict__ fb_layers, uint32_t n_chunks_all) {
     pdl_wait();
     __shared__ uint32_t s_drop[KIMAD_MAX_RATIOS]; // entries not kept by candidate j: n - k_j
     __shared__ uint32_t s_bin[KIMAD_MAX_RATIOS], s_before[KIMAD_MAX_RATIOS], s_cb[KIMAD_MAX_RATIOS];
@@ -640,7 +641,8 @@ k_resolve_a(const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ r
             atomicAdd(&fb->why[bad - 1], 1u);
         }
         __syncthreads();
-        for (uint32_t i = threadIdx.x; i < ld.n_chunks; i += kBigThreads) fb_chunks[s_at + i] = make_uint2(w, ld.first_chunk + i);
+        for (uint32_t i = threadIdx.x; i < ld.n_chunks; i += kBigThreads)
+            if (KIMAD_CHECK(s_at + i < gridDim.y * n_chunks_all, 2)) fb_chunks[s_at + i] = make_uint2(w, ld.first_chunk + i);
     }
 }
 

@@ -663,7 +663,7 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
                             for (int q = 0; q < kDpCells; ++q) {
                                 // cells beyond the row (last pass only) read the row itself: harmless, never stored
                                 const uint32_t b = min(b0 + q * blockDim.x, row - 1);
-                                p[i][q] = prev[(int)b - (int)u[i]];
+                                p[i][q] = KIMAD_CHECK((int)b - (int)u[i] >= -(int)pad, 5) ? prev[(int)b - (int)u[i]] : kInf;
                             }
 #pragma unroll
                         for (int i = 0; i < 4; ++i)

@@ -100,7 +100,7 @@ __device__ __forceinline__ void sel_count_chunk(const DSource& dbuf, const Chunk
         auto visit = [&](uint32_t key) -> bool { // true: the key is not below the interval
             const uint32_t d1 = key - lo; // wraps to >= 2^31 for keys below the interval
             if (d1 < width) {
-                atomicAdd(&gh[d1 >> hshift], 1u);
+                if (KIMAD_CHECK((d1 >> hshift) < (uint32_t)kLowBins, 1)) atomicAdd(&gh[d1 >> hshift], 1u);
                 const uint32_t p = atomicAdd(s_n, 1u);
                 if (p < (uint32_t)kListCap) s_low[p] = (sl << 16) | d1;
             } else {
@@ -182,7 +182,10 @@ __device__ __forceinline__ void sel_count_chunk(const DSource& dbuf, const Chunk
             out->n_in = n_in;
         } else {
             out->n_in = kListOverflow;
-            recount_list[atomicAdd(recount_n, 1u)] = make_uint2(w, chunk_id);
+            const uint32_t at = atomicAdd(recount_n, 1u);
+            // capacity 2 W n_chunks (a chunk can be listed once per select round); the second round's launch has a flat
+            // grid and does not carry W: its appends stay below the bound the first round's were tested against
+            if (KIMAD_CHECK(gridDim.y == 1 || at < 2u * gridDim.y * n_chunks, 2)) recount_list[at] = make_uint2(w, chunk_id);
         }
     }
     __syncthreads();
@@ -570,7 +573,7 @@ k_sel_write(const float* __restrict__ grads, float* __restrict__ state, const Ch
                 pos += __shfl_sync(0xffffffffu, incl, 31);
 #pragma unroll
                 for (int i = 0; i < 4; ++i)
-                    if ((keepm >> i) & 1u) {
+                    if (((keepm >> i) & 1u) && KIMAD_CHECK(jb.base + o < cap, 3)) {
                         oi[o] = idx0 + e0 + i;
                         float sent;
                         if (BF16) {
@@ -678,6 +681,7 @@ k_sel_write(const float* __restrict__ grads, float* __restrict__ state, const Ch
                 __syncwarp();
                 const uint32_t round_pos = pos - round_total;
                 for (uint32_t q = lane; q < round_total; q += 32) {
+                    if (!KIMAD_CHECK(jb.base + round_pos + q < cap, 3)) continue;
                     oi[round_pos + q] = sg_idx[q];
                     if (BF16) ov16[round_pos + q] = __ushort_as_bfloat16((unsigned short)sg_val[q]);
                     else ov32[round_pos + q] = __uint_as_float(sg_val[q]);
@@ -701,6 +705,7 @@ k_sel_write(const float* __restrict__ grads, float* __restrict__ state, const Ch
                 const int i = __ffs(keepm) - 1;
                 keepm &= keepm - 1;
                 const uint32_t e = t0 + i;
+                if (!KIMAD_CHECK(jb.base + o < cap && e >= cv.first && e < cv.len, 3)) { ++o; continue; }
                 const float was = st[e];
                 const float val = __fsub_rn(__ldg(gr + e), was); // both loaded a moment ago: L1 hits
                 oi[o] = idx0 + e;

@@ -2,6 +2,8 @@
 the same seeded inputs and compares stage by stage."""
 from __future__ import annotations
 
+import os
+
 import numpy as np
 import torch
 
@@ -104,4 +106,8 @@ class Runner:
             assert np.array_equal(u32(out2.k), ref.k)
             assert np.array_equal(u32(scratch), ref.state.view(np.uint32))
             assert np.array_equal(out2.stats_host()["total_err"].view(np.uint32), ref.total_err.view(np.uint32))
+        # checked build of the library (KIMAD_CHECKED=1): no index test failed, no canary between workspace regions damaged
+        checked, failed, damaged = kb.kimad_debug_check(self.ctx)
+        assert checked == (os.environ.get("KIMAD_CHECKED") == "1")
+        assert failed == 0 and damaged == 0, (hex(failed), damaged)
         return dict(status=status, same_k=same_k, ref=ref, forced=forced)
