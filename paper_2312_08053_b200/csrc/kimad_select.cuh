@@ -123,17 +123,19 @@ __device__ __forceinline__ void sel_count_chunk(const DSource& dbuf, const Chunk
                 bool f = false;
                 if (cv.quad_full(q)) {
                     const uint32_t x0_ = a[i].x & 0x7fff7fffu, x1_ = a[i].y & 0x7fff7fffu;
-                    const uint32_t gt0 = (x0_ + add_gt) & 0x80008000u, gt1 = (x1_ + add_gt) & 0x80008000u;
                     const uint32_t ge0 = (x0_ + add_ge) & 0x80008000u, ge1 = (x1_ + add_ge) & 0x80008000u;
-                    above += __popc(gt0) + __popc(gt1);
-                    f = (gt0 | gt1) != 0; // keys sharing an upper half with the interval mark the group only if not below it
-                    // rare: keys that share an upper half with the interval; bit 15 -> element 0 / 2, bit 31 -> 1 / 3
-                    uint32_t border = ((ge0 ^ gt0) >> 15 & 0x00010001u) | ((ge1 ^ gt1) >> 13 & 0x00040004u);
-                    while (border) {
-                        const uint32_t bit = __ffs(border) - 1; // 0, 16 (first word), 2, 18 (second word)
-                        border &= border - 1;
-                        const uint32_t k = (bit & 3u) + (bit >> 4);
-                        f |= visit(key_of(dd.at(4 * q + k)));
+                    if (ge0 | ge1) { // with a sparse budget few quads hold a key that is not below the interval's upper half
+                        const uint32_t gt0 = (x0_ + add_gt) & 0x80008000u, gt1 = (x1_ + add_gt) & 0x80008000u;
+                        above += __popc(gt0) + __popc(gt1);
+                        f = (gt0 | gt1) != 0; // keys sharing an upper half with the interval mark the group only if not below it
+                        // rare: keys that share an upper half with the interval; bit 15 -> element 0 / 2, bit 31 -> 1 / 3
+                        uint32_t border = ((ge0 ^ gt0) >> 15 & 0x00010001u) | ((ge1 ^ gt1) >> 13 & 0x00040004u);
+                        while (border) {
+                            const uint32_t bit = __ffs(border) - 1; // 0, 16 (first word), 2, 18 (second word)
+                            border &= border - 1;
+                            const uint32_t k = (bit & 3u) + (bit >> 4);
+                            f |= visit(key_of(dd.at(4 * q + k)));
+                        }
                     }
                 } else if (4 * q < cv.len) {
                     for (uint32_t e = 4 * q; e < 4 * q + 4; ++e)
