@@ -212,3 +212,34 @@ def test_error_axis_dp_worked_example_and_statuses():
     res = r.compare_step(d, torch.zeros_like(d), [96.0, 112.0, 47.0, 160.0], 1.0)
     assert res["forced"].k.tolist() == [[5, 2, 2], [10, 2, 2], [3, 1, 2], [10, 4, 6]]
     assert list(res["forced"].status) == [0, 0, ko.STATUS_INFEASIBLE, ko.STATUS_PLATEAU]
+
+
+def test_overlapped_host_driver_gives_the_serial_results_and_feeds_the_monitor():
+    """The double-buffered driver (next step copied in and compressed while this step's message is copied out)
+    against the plain one-after-the-other driver: same messages, same estimator; the message copies' sizes and
+    durations reach the bandwidth monitor."""
+    from paper_2312_08053_b200 import pipeline
+
+    wl = workloads.workload(2, 8)
+    W, N = wl.n_workers, wl.N
+    bw = workloads.bandwidth_trace(wl, 12)
+    host = [workloads.gradients(wl, s).pin_memory() for s in range(3)]
+    results = {}
+    for mode in ("serial", "overlapped"):
+        ctx = kb.new_context(wl.layer_sizes, W, wl.ratio_grid, D=wl.D, max_packed_elems=N)
+        mon = kb.kimad_monitor_create(window=4, alpha=1.0)
+        drv = pipeline.HostDriver(ctx, wl, N, monitor=mon)
+        state = torch.zeros((W, N), dtype=torch.float32, device="cuda")
+        moved = drv.run(mode, host, state, bw, 7)
+        torch.cuda.synchronize()
+        last = 6 % 2 if mode == "overlapped" else 0
+        st = drv.h_stats[last].numpy().view(kb.STATS_DTYPE).reshape(-1).copy()
+        n = int(st["n_selected"][0])
+        results[mode] = (moved, state.cpu().numpy().copy(), st, drv.h_idx[last][0, :n].numpy().copy(),
+                         drv.h_val[last][0, :n].numpy().copy())
+        assert kb.kimad_monitor_estimate(mon) > 0.0  # bytes per second of the message copies
+    a, b = results["serial"], results["overlapped"]
+    assert a[0] == b[0] and a[0] > 0
+    assert np.array_equal(a[1].view(np.uint32), b[1].view(np.uint32))
+    assert a[2].tobytes() == b[2].tobytes()
+    assert np.array_equal(a[3], b[3]) and np.array_equal(a[4].view(np.uint32), b[4].view(np.uint32))
