@@ -34,7 +34,7 @@ UNIT = "elements/s"
 # launch of the sweep kernel in an ncu capture on workload 3 (inputs larger than L2), divided by the elements of
 # that launch.  Every element is read once from each input and its upper half written once, so the figure
 # carries over to the other workloads; it has to be re-captured when the sweep's data movement changes.
-NCU_TRAFFIC_BYTES_PER_ELEM = {"sweep": 10.13}
+NCU_TRAFFIC_BYTES_PER_ELEM = {"sweep": 10.14}
 
 # algorithmic bytes per input element of each stage (what the stage must move at least once)
 STAGE_ALGO_BYTES = {"sweep": 10.0,  # read grad + g, write the upper halves of d
@@ -335,6 +335,13 @@ def run_kimad(args, rank, world):
                 "step_roofline": sr2, "roofline": rf2, "stage_ms": stage2}
         del ctx2, out2, grads2, state2, step2
         torch.cuda.empty_cache()
+    # ---- the receiving side of a round on the same workload (apply the messages, model step), device-timed
+    receive = None
+    if not args.no_also:
+        torch.cuda.empty_cache()
+        rcv = _measure_receive(args, rank, world, max(3, min(args.steps, 10)), 3)
+        receive = {k: rcv[k] for k in ("metric", "value", "unit", "ms_per_step", "steps", "warmup", "roofline", "stage_ms")}
+        torch.cuda.empty_cache()
     if rank != 0:
         return
     res = {
@@ -354,15 +361,17 @@ def run_kimad(args, rank, world):
     }
     if also is not None:
         res["also"] = also
+    if receive is not None:
+        res["receive"] = receive
     if world == 1 and not args.no_cpu_baseline:
         res["cpu_baseline"] = cpu_baseline(args.config)
     print(json.dumps(res))
 
 
-def run_receive(args, rank, world):
-    """Secondary line: the receiving side of one round (Algorithm 1, server lines) on the same workload:
+def _measure_receive(args, rank, world, steps, warmup):
+    """The receiving side of one round (Algorithm 1, server lines) on the configured workload:
     kimad_apply_packed of the W workers' messages, then kimad_aggregate over the W estimators.  The
-    dominant kernel is the dense model step, (W + 2) * 4 bytes per model element."""
+    dominant kernel is the dense model step, (W + 2) * 4 bytes per model element.  Returns the result dict."""
     import torch
 
     from paper_2312_08053_b200 import binding as kb
@@ -390,9 +399,9 @@ def run_receive(args, rank, world):
     x = torch.zeros(N, dtype=torch.float32, device=dev)
     wts = np.full(W, 1.0 / W, np.float32)
     stream = torch.cuda.current_stream()
-    ev_a = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
-    ev_b = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
-    ev_c = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    ev_a = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    ev_b = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    ev_c = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
 
     def step(s, i=None):
         if i is not None:
@@ -404,35 +413,40 @@ def run_receive(args, rank, world):
         if i is not None:
             ev_c[i].record(stream)
 
-    for s in range(args.warmup):
+    for s in range(warmup):
         step(s)
     barrier()
     torch.cuda.synchronize()
-    for i in range(args.steps):
-        step(args.warmup + i, i)
+    for i in range(steps):
+        step(warmup + i, i)
     torch.cuda.synchronize()
     barrier()
     total_ms = max_over_ranks(ev_a[0].elapsed_time(ev_c[-1]))
     apply_ms = float(np.mean([a.elapsed_time(b) for a, b in zip(ev_a, ev_b)]))
     agg_ms = float(np.mean([b.elapsed_time(c) for b, c in zip(ev_b, ev_c)]))
-    if rank != 0:
-        return
     peak, peak_kind = peaks()
-    ms_per_step = total_ms / args.steps
+    ms_per_step = total_ms / steps
     algo_b = (W + 2) * 4.0 * N
     achieved = algo_b / (agg_ms * 1e-3) / 1e9
     n_entries = float(np.mean([int(m.stats_host()["n_selected"].sum()) for m in msgs]))
-    print(json.dumps({
+    return {
         "metric": "received_update_elements_per_second", "value": W * N * world / (ms_per_step * 1e-3), "unit": UNIT,
-        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+        "n_gpus": world, "steps": steps, "warmup": warmup, "ms_per_step": ms_per_step,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": wl.name + " / receive", "cfg": wl.cfg, "senders": W, "elements_per_sender": N,
                    "packed_entries_per_step": n_entries, "l2": "inputs_larger_than_l2"},
-        "gpu_launches": 2 * args.steps,
+        "gpu_launches": 2 * steps,
         "roofline": {"bound": "hbm", "kernel": "k_aggregate", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
                      "algorithmic_bytes_per_launch": algo_b, "kernel_ms": agg_ms},
-        "stage_ms": {"apply_packed": apply_ms, "aggregate": agg_ms}}))
+        "stage_ms": {"apply_packed": apply_ms, "aggregate": agg_ms}}
+
+
+def run_receive(args, rank, world):
+    """Secondary line (``--path receive``): the receiving side alone."""
+    res = _measure_receive(args, rank, world, args.steps, args.warmup)
+    if rank == 0:
+        print(json.dumps(res))
 
 
 def main():
