@@ -431,7 +431,7 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
             if (fit == 0) status = KIMAD_STATUS_INFEASIBLE;
             for (uint32_t l = threadIdx.x; l < L; l += blockDim.x) s_j[l] = fit ? fit - 1 : 0;
         } else if (mode == 4) {
-            for (uint32_t l = threadIdx.x; l < L; l += blockDim.x) s_j[l] = 0; // feasibility is judged on the totals below
+            for (uint32_t l = threadIdx.x; l < L; l += blockDim.x) s_j[l] = 0; // feasibility is decided on the totals below
         } else if (mode == 3) {
             // Error axis: E_max = sum_l err_{l,0} (binary64, layers in order), cells e_{l,j} = floor(err D / E_max),
             // value = fewest kept entries for a total of exactly e cells; answer = lowest e whose value fits c.

@@ -222,7 +222,7 @@ k_sel_count_r2(DSource dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks
 }
 
 // Exact threshold of one (worker, layer) from what the counting sweep left behind.  The whole CTA works on it.
-// round 1: may narrow the interval and list the layer for the second round; round 2: the interval is at
+// first round: may narrow the interval and list the layer for the second round; second round: the interval is at
 // most 32 keys wide and the histogram is exact.
 __device__ __forceinline__ void sel_resolve_layer(uint32_t l, uint32_t w, uint32_t L, const LayerDesc* __restrict__ layers,
                                                   uint32_t n_chunks, const ChunkSel* __restrict__ csel,
