@@ -123,3 +123,36 @@ def test_create_validates_policy_and_cost_model():
                dict(ratio_grid=[0.5, 1.0], cost_model=2)):
         with pytest.raises(kb.KimadError):
             kb.kimad_create([100, 20], 1, **kw)
+
+
+@pytest.mark.parametrize("seed", [21, 22])
+def test_randomized_policies_and_cost_models(seed):
+    """Random layer lists, grids, worker counts, strides, value types and budgets under every policy (layer-adaptive,
+    grid ratio, error axis, fitted ratio) and both cost models where they apply; two steps each, everything compared
+    with the oracle."""
+    for it in range(16):
+        rng = np.random.default_rng(seed * 1000 + it)
+        policy = int(rng.integers(0, 4))
+        cost_model = int(rng.integers(0, 2)) if policy < 2 else 0
+        L = int(rng.integers(1, 7))
+        sizes = [int(v) for v in np.exp(rng.uniform(np.log(1), np.log(200000), L)).astype(int) + 1]
+        if policy == 3:
+            grid = [1.0]
+        else:
+            grid = np.unique(np.round(np.sort(rng.uniform(0.0005, 1.0, int(rng.integers(1, 12)))), 6))
+            if rng.random() < 0.5:
+                grid[-1] = 1.0
+        W, vd = int(rng.integers(1, 4)), int(rng.integers(0, 2))
+        D = max(int(rng.choice([L, 50, 1000])), L)
+        N = sum(sizes)
+        stride = N + int(rng.integers(0, 9))
+        r = Runner(sizes, W, list(grid), D, vd, stride=stride, policy=policy, cost_model=cost_model)
+        x = (rng.standard_normal((W, stride)) * np.exp(rng.uniform(-4, 4, (W, stride)))).astype(np.float32)
+        if it % 5 == 4:
+            x = np.round(x * 2) / 2  # heavy ties, many zeros
+        grads = torch.from_numpy(x).cuda()
+        state = torch.from_numpy((rng.standard_normal((W, stride)) * 0.1).astype(np.float32)).cuda()
+        for rep in range(2):
+            frac = float(np.exp(rng.uniform(np.log(0.002), np.log(1.5))))
+            bw = [frac * (8 if vd == 0 else 6) * N * float(rng.uniform(0.5, 1.5)) for _ in range(W)]
+            r.compare_step(grads, state, bw, 1.0, check_inject=bool(rng.integers(0, 2)))
