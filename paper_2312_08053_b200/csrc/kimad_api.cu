@@ -20,11 +20,11 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
     // static tables
-    size_t dbuf, chunks, layers, ktab, ktab_dyn, reg_layers, tiny_layers, reg_index;
+    size_t dbuf, chunks, layers, ktab, ktab_dyn, reg_layers, tiny_layers, reg_index, runs;
     // zeroed at set_workspace and kept clean by the kernels
     size_t zero_from, h1_cnt, h1_ss, h23_cnt, h23_ss, bh_cnt, bh_sum, low_hist, recount, fb, r2, flags;
     // scratch without initial-state requirements
-    size_t lut_t1, lut_t2, bin_lo, meta, cands, slots, err, tau, keep_eq, shift, sel, chunk_cnt, jobs, csel,
+    size_t cell_tab, cell_win, bin_lo, meta, cands, slots, err, tau, keep_eq, shift, sel, chunk_cnt, jobs, csel,
         fb_chunks, fb_layers, r2_chunks, r2_layers, pd, total;
 };
 
@@ -40,6 +40,7 @@ struct kimad_ctx {
     std::vector<Chunk> chunks;
     std::vector<LayerDesc> layers;
     std::vector<uint32_t> reg_layers, tiny_layers, reg_index; // layers above / up to kTinyMax elements
+    std::vector<SweepRun> runs;                               // the sweep's CTAs: static runs of chunks, balanced by elements
     std::vector<unsigned char> static_image;                  // the static tables as they lie in the workspace, one block
     std::vector<size_t> guards;                               // checked build: offsets of the canary words between regions
     uint32_t curve_mode = 0;
@@ -87,6 +88,7 @@ void plan_layout(kimad_ctx* c) {
     y.reg_layers = take(c->reg_layers.size() * sizeof(uint32_t));
     y.tiny_layers = take(c->tiny_layers.size() * sizeof(uint32_t));
     y.reg_index = take(c->reg_index.size() * sizeof(uint32_t));
+    y.runs = take(c->runs.size() * sizeof(SweepRun));
     y.zero_from = o;
     y.h1_cnt = take(WL * kL1Bins * sizeof(uint32_t));
     y.h1_ss = take(WL * kL1Bins * sizeof(uint64_t));
@@ -99,8 +101,8 @@ void plan_layout(kimad_ctx* c) {
     y.fb = take(sizeof(FbList));
     y.r2 = take(sizeof(Round2));
     y.flags = take((size_t)c->W * sizeof(uint32_t));
-    y.lut_t1 = take(WR * kL1Bins * sizeof(uint16_t));
-    y.lut_t2 = take(WR * kLutWords * sizeof(uint32_t));
+    y.cell_tab = take(WR * kCellTab * sizeof(uint32_t));
+    y.cell_win = take(WR * sizeof(int4));
     y.bin_lo = take(WR * (kMaxBins + 1) * sizeof(uint32_t));
     y.meta = take(WR * sizeof(BandMeta));
     y.cands = take(WLK * sizeof(Cand));
@@ -127,6 +129,7 @@ void plan_layout(kimad_ctx* c) {
     } while (0)
 
 constexpr size_t kDpSmemMax = 225 * 1024; // dynamic shared memory the DP kernel may ask for
+constexpr uint32_t kSweepWaves = 2;       // CTAs of the sweep per SM (148 SMs), one resident at a time
 
 // Kernels are loaded on their first launch; loading one takes about a millisecond.  Touching every kernel a
 // step can launch (the rarely taken ones included) when the workspace is attached keeps that out of the steps.
@@ -228,8 +231,8 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
     unsigned long long* h23s = c->at<unsigned long long>(y.h23_ss);
     uint32_t* bhc = c->at<uint32_t>(y.bh_cnt);
     unsigned long long* bhs = c->at<unsigned long long>(y.bh_sum);
-    uint16_t* lut1 = c->at<uint16_t>(y.lut_t1);
-    uint32_t* lut2 = c->at<uint32_t>(y.lut_t2);
+    uint32_t* cell_tab = c->at<uint32_t>(y.cell_tab);
+    int4* cell_win = c->at<int4>(y.cell_win);
     uint32_t* binlo = c->at<uint32_t>(y.bin_lo);
     BandMeta* meta = c->at<BandMeta>(y.meta);
     Cand* cands = c->at<Cand>(y.cands);
@@ -256,9 +259,8 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
 
     const uint32_t R = (uint32_t)c->reg_layers.size(), T = (uint32_t)c->tiny_layers.size();
     const dim3 gch(nch, W), glw(L, W), blk(kThreads);
-    // long runs amortise the per-CTA table load and histogram flush; keep about eight waves of CTAs on 148 SMs
-    const uint32_t run_chunks = std::max<uint32_t>(4u, std::min<uint32_t>((uint32_t)kMaxRunChunksA, (uint32_t)(((uint64_t)nch * W) / (148 * 8))));
-    const dim3 grun((nch + run_chunks - 1) / run_chunks, W);
+    const SweepRun* runs = c->at<SweepRun>(y.runs);
+    const uint32_t n_runs = (uint32_t)c->runs.size();
     int stage = 0;
     auto mark = [&]() { if (c->timing) cudaEventRecord(c->ev[stage++], s); };
     auto budgets_of = [&](uint32_t w0, uint32_t nw) {
@@ -278,30 +280,31 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
             c->launches += 1;
         }
     }
-    if (T) CUDA_TRY(cudaEventRecord(c->ev_fork, s)); // fork point of the tiny layers' kernel: the step's start
     // (a) + (b): sample -> bands -> one sweep -> curves
     if (R) {
         CUDA_TRY(launch_pdl(k_sample, dim3(R, W), kBigThreads, c->sample_smem, s, grads, state, c->stride, layers, reg_layers, R,
-                            ktab, K, c->curve_mode == 1 ? 1u : 0u, lut1, lut2, binlo, meta));
+                            ktab, K, c->curve_mode == 1 ? 1u : 0u, cell_tab, cell_win, binlo, meta));
         c->launches += 1;
     }
-    if (T) { // tiny layers: sorted in shared memory on the side stream; issued after the sample kernel so that
-             // its CTAs fill the SMs the sample kernel leaves idle instead of delaying it
+    mark();
+    if (vec)
+        CUDA_TRY(launch_pdl(k_pass_a<true>, n_runs, kBigThreads, c->pass_a_smem, s, grads, state, dbuf.hi, chunks, runs,
+                            c->stride, c->dstride, reg_index, R, cell_tab, cell_win, meta, bhc, bhs));
+    else
+        CUDA_TRY(launch_pdl(k_pass_a<false>, n_runs, kBigThreads, c->pass_a_smem, s, grads, state, dbuf.hi, chunks, runs,
+                            c->stride, c->dstride, reg_index, R, cell_tab, cell_win, meta, bhc, bhs));
+    c->launches += 1;
+    mark();
+    if (T) { // tiny layers: sorted in shared memory on the side stream, beside the kernels that turn the sweep's
+             // histograms into curves (all of them latency-bound).  Not beside the sweep: CTAs of another kernel on
+             // an SM keep the sweep's CTA, which takes most of the SM's shared memory, from starting there.
+        CUDA_TRY(cudaEventRecord(c->ev_fork, s));
         CUDA_TRY(cudaStreamWaitEvent(c->side, c->ev_fork, 0));
         CUDA_TRY(launch_pdl(k_tiny_exact, dim3(T, W), blk, c->tiny_smem, c->side, grads, state, c->stride, layers, tiny_layers, L,
                             ktab, K, err, tau, keq, shf, flags));
         CUDA_TRY(cudaEventRecord(c->ev_join, c->side));
         c->launches += 1;
     }
-    mark();
-    if (vec)
-        CUDA_TRY(launch_pdl(k_pass_a<true>, grun, kBigThreads, c->pass_a_smem, s, grads, state, dbuf.hi, chunks, nch, run_chunks,
-                            c->stride, c->dstride, reg_index, R, lut1, lut2, meta, bhc, bhs));
-    else
-        CUDA_TRY(launch_pdl(k_pass_a<false>, grun, kBigThreads, c->pass_a_smem, s, grads, state, dbuf.hi, chunks, nch, run_chunks,
-                            c->stride, c->dstride, reg_index, R, lut1, lut2, meta, bhc, bhs));
-    c->launches += 1;
-    mark();
     if (R) {
         CUDA_TRY(launch_pdl(k_resolve_a, dim3(R, W), kBigThreads, 0, s, layers, reg_layers, R, L, ktab, K, meta, binlo, bhc, bhs, err, tau,
                                                        keq, shf, flags, fb, fb_chunks, fb_layers, nch));
@@ -449,8 +452,22 @@ int kimad_create(kimad_ctx** out, const uint64_t* layer_sizes, uint32_t n_layers
         c->policy = o.policy;
         c->cost_model = o.cost_model;
         if (c->policy == 2 && !c->dp_plan.tab_in_smem) { delete c; return KIMAD_ERR_INVALID_ARG; }
-        c->sample_smem = (size_t)(2 * (1024 + 32) + 32768 + 2048 + 1024 + 2048 + 2048 + 32 + 3 * 128) * 4;
-        c->pass_a_smem = (size_t)(3 * kMaxBins + kLutWords) * 4 + kL1Bins * 2;
+        c->sample_smem = (size_t)(2 * (1024 + 32) + 32768 + 1024 + 2 * kMaxGaps + 32 + 3 * 128) * 4;
+        c->pass_a_smem = (size_t)(2 * kMaxBins + kCellTab) * 4;
+        { // the sweep's runs: every worker's chunk list is cut into pieces of about equal element counts, about
+          // kSweepWaves CTAs per SM in all (one CTA is resident per SM)
+            const uint32_t nch = (uint32_t)c->chunks.size();
+            const uint32_t per_w = std::max<uint32_t>(1u, std::min<uint32_t>(nch, (kSweepWaves * 148u + c->W - 1) / c->W));
+            for (uint32_t w = 0; w < c->W; ++w) {
+                uint64_t acc = 0;
+                uint32_t g = 0, start = 0;
+                for (uint32_t f = 0; f < nch; ++f) {
+                    if (g + 1 < per_w && f > start && acc >= (N * (uint64_t)(g + 1)) / per_w) { c->runs.push_back(SweepRun{w, start, f}); start = f; ++g; }
+                    acc += c->chunks[f].end - c->chunks[f].begin;
+                }
+                c->runs.push_back(SweepRun{w, start, nch});
+            }
+        }
         c->tiny_smem = (size_t)kTinyMax * (8 + 4);
         plan_layout(c);
         { // host image of the static tables [chunks, zero_from): attached workspaces get it in one copy
@@ -463,6 +480,7 @@ int kimad_create(kimad_ctx** out, const uint64_t* layer_sizes, uint32_t n_layers
             if (!c->reg_layers.empty()) std::memcpy(im + y.reg_layers, c->reg_layers.data(), c->reg_layers.size() * 4);
             if (!c->tiny_layers.empty()) std::memcpy(im + y.tiny_layers, c->tiny_layers.data(), c->tiny_layers.size() * 4);
             std::memcpy(im + y.reg_index, c->reg_index.data(), c->reg_index.size() * 4);
+            std::memcpy(im + y.runs, c->runs.data(), c->runs.size() * sizeof(SweepRun));
             for (size_t g : c->guards)
                 if (g >= y.chunks && g + kAlign <= y.zero_from) std::memset(im + g, kCanaryByte, kAlign);
         }
@@ -512,7 +530,7 @@ int kimad_set_workspace(kimad_ctx* c, void* dev_ptr, size_t bytes) {
     const Layout& y = c->lay;
     CUDA_TRY(cudaMemcpy(c->ws + y.chunks, c->static_image.data(), c->static_image.size(), cudaMemcpyHostToDevice));
     // histograms, work lists and flags start at zero and are kept clean by the kernels that consume them
-    CUDA_TRY(cudaMemset(c->ws + y.zero_from, 0, y.lut_t1 - y.zero_from));
+    CUDA_TRY(cudaMemset(c->ws + y.zero_from, 0, y.cell_tab - y.zero_from));
     { const int rc_g = fill_guards(c, c->ws, nullptr); if (rc_g != KIMAD_OK) return rc_g; }
     { const int rc_dev = prepare_device(c); if (rc_dev != KIMAD_OK) return rc_dev; }
     CUDA_TRY(cudaDeviceSynchronize());
@@ -768,7 +786,7 @@ int kimad_step_builtin_scratch(kimad_ctx* c, const float* grads_dev, float* stat
     // and clear everything that has to start at zero, in stream order before the kernels.
     const Layout& y = c->lay;
     CUDA_TRY(cudaMemcpyAsync(ws + y.chunks, c->static_image.data(), c->static_image.size(), cudaMemcpyHostToDevice, s));
-    CUDA_TRY(cudaMemsetAsync(ws + y.zero_from, 0, y.lut_t1 - y.zero_from, s));
+    CUDA_TRY(cudaMemsetAsync(ws + y.zero_from, 0, y.cell_tab - y.zero_from, s));
     { const int rc_g = fill_guards(c, ws, s); if (rc_g != KIMAD_OK) return rc_g; }
     unsigned char* caller_ws = c->ws; // the context's own workspace (if any) is left untouched
     c->ws = ws;

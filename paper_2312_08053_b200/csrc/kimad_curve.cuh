@@ -4,11 +4,13 @@
 //   k_sample     per (worker, layer): histogram of a stratified sample of |d| over 16-bit key prefixes
 //                ("cells"); for every candidate k_j the cells that can contain the k_j-th largest key
 //                (sample rank +- 6 sigma) form a band.  Band cells are cut into fine bins of 2^shift
-//                keys, everything else into coarse "gap" bins; the mapping key -> bin is a two-level
-//                table (11-bit bin -> row, row x 5 more bits -> bin base and shift).
-//   k_pass_a     the sweep: d = grad - g (its upper 16 bits go to scratch), bin = table(key(d)), two u32 shared-
-//                memory atomics per element: the count, and the exact integer sum of squares in a low u32 word
-//                whose (rare) carries go to a high word.
+//                keys, everything else into coarse "gap" bins.  Every region (a gap, or a group of bands with
+//                one bin width) maps a key to its bin as base + (key >> shift); which region a key lies in is
+//                read from a table over the window of cells between the lowest and the highest band.
+//   k_pass_a     the sweep: d = grad - g (its upper 16 bits go to scratch), bin = base + (key >> shift) with
+//                (base, shift) = table(cell(key)), two u32 shared-memory atomics per element: the count, and the
+//                exact integer sum of squares in a u32 word whose (rare) carries go straight to the 64-bit sum in
+//                global memory.  CTAs own static runs of chunks balanced by elements.
 //   k_resolve_a  per (worker, layer): walks the bins from the top, finds the bin that holds every
 //                candidate's threshold, sums the squares below it.  The candidate's error is certified
 //                to 2^-19 relative from the bin's width; if a threshold fell into a gap bin (the sample
@@ -21,10 +23,14 @@
 namespace kimad {
 
 constexpr int kTinyMax = 4096;
-constexpr int kFineBins = 12288;                    // fine bins per (worker, layer)
+#ifndef KIMAD_FINE_BINS
+#define KIMAD_FINE_BINS 12288
+#endif
+constexpr int kFineBins = KIMAD_FINE_BINS;          // fine bins per (worker, layer)
 constexpr int kMaxGaps = KIMAD_MAX_RATIOS + 2;      // gap regions: below / between / above the band groups, + non-finite keys
 constexpr int kMaxBins = kFineBins + kL1Bins + 2 * kMaxGaps; // fine bins + gap regions cut at every 11-bit prefix
-constexpr int kMaxRows = 128;                       // 11-bit bins that contain band cells
+constexpr int kCellTab = 4096;                      // entries of the cell table: the window of cells from the lowest to the
+                                                    // highest band (32 octaves) and one entry on either side
 constexpr int kMaxShift = 15;                       // a fine bin is 2^shift keys wide, at most a whole cell
 constexpr int kSampleUnits = 4095;                  // sample = units of 16 consecutive elements (<= 65520 elements)
 constexpr int kBigThreads = 1024;
@@ -32,12 +38,11 @@ constexpr uint32_t kGapBit = 1u;                    // bin_lo entries carry this
 
 struct BandMeta { // per (worker, regular layer)
     uint32_t n_bins;
-    uint32_t n_rows;
+    uint32_t n_cells; // entries of the cell table in use
     uint32_t flagged; // != 0: this layer takes the exact radix path in this step
     uint32_t n_gaps;  // gap regions (when flagged: detail of the misfit)
 };
-// lookup entry of a cell: first bin id | shift << 16; the bin of a key is id + ((key & 0x7fff) >> shift)
-constexpr int kLutWords = kMaxRows * 32;
+// entry of the cell table: base << 5 | shift (base signed); the bin of a key is base + (key >> shift)
 
 __device__ __forceinline__ uint32_t hash_u32(uint32_t x) {
     x ^= x >> 16; x *= 0x7feb352du; x ^= x >> 15; x *= 0x846ca68bu; x ^= x >> 16;
@@ -50,22 +55,20 @@ __device__ __forceinline__ uint32_t hash_u32(uint32_t x) {
 __global__ void __launch_bounds__(kBigThreads, 1)
 k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint64_t stride,
          const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ reg_layers, uint32_t R,
-         const KTab ktab, uint32_t K, uint32_t force_exact, uint16_t* __restrict__ lut_t1,
-         uint32_t* __restrict__ lut_t2, uint32_t* __restrict__ bin_lo, BandMeta* __restrict__ meta) {
+         const KTab ktab, uint32_t K, uint32_t force_exact, uint32_t* __restrict__ cell_tab,
+         int4* __restrict__ cell_win, uint32_t* __restrict__ bin_lo, BandMeta* __restrict__ meta) {
     pdl_wait();
     extern __shared__ __align__(16) uint32_t sh[];
     double* s_sq = reinterpret_cast<double*>(sh); // [1024] squares (cell midpoints) below each thread segment
     double* s_wd = s_sq + 1024;                   // [32]
     uint32_t* h32 = sh + 2 * (1024 + 32);         // [32768] two u16 cell counters per word
-    uint32_t* bitmap = h32 + 32768;               // [2048] bit c of word b: cell (b << 5 | c) belongs to a band
-    uint32_t* s_pre = bitmap + 2048;              // [1024] inclusive sample count of the thread segments, from the top
-    uint32_t* s_base = s_pre + 1024;              // [2048] first bin id of every 11-bit bin
-    uint32_t* s_aux = s_base + 2048;              // [2048] row index of split 11-bit bins
-    uint32_t* s_w = s_aux + 2048;                 // [32]
+    uint32_t* s_pre = h32 + 32768;                // [1024] inclusive sample count of the thread segments, from the top
+    uint32_t* s_base = s_pre + 1024;              // [2 kMaxGaps] first bin id of every gap region, of every group
+    uint32_t* s_w = s_base + 2 * kMaxGaps;        // [32]
     uint32_t* s_cb = s_w + 32;                    // [128] per candidate, then per merged group: lowest cell,
     uint32_t* s_ct = s_cb + 128;                  // [128] highest cell,
     uint32_t* s_cs = s_ct + 128;                  // [128] shift
-    __shared__ uint32_t s_m, s_flag, s_ng;
+    __shared__ uint32_t s_m, s_flag, s_ng, s_cg;
     const uint32_t r = blockIdx.x, w = blockIdx.y;
     const uint32_t l = reg_layers[r];
     const size_t wr = (size_t)w * R + r;
@@ -76,8 +79,8 @@ k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint6
     }
     const LayerDesc ld = layers[l];
     const uint32_t n = (uint32_t)ld.n;
-    for (int i = threadIdx.x; i < 32768 + 2048; i += kBigThreads) h32[i] = 0;
-    if (threadIdx.x == 0) { s_m = 0; s_flag = 0; s_ng = 0; }
+    for (int i = threadIdx.x; i < 32768; i += kBigThreads) h32[i] = 0;
+    if (threadIdx.x == 0) { s_m = 0; s_flag = 0; s_ng = 0; s_cg = 0; }
     __syncthreads();
 
     // ---- stratified sample of |grad - g|
@@ -184,10 +187,11 @@ k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint6
             }
             // rank window clipped at the top: the threshold may lie above the largest sample, so the band goes a
             // quarter octave further up; clipped at the bottom: no bound from the sample, exact path
-            uint32_t c_top = cell_of_rank(max(r_lo, 1u));
+            // bands stay among the finite keys (a sample with non-finite values is reported by the curve stage)
+            uint32_t c_top = min(cell_of_rank(max(r_lo, 1u)), 65279u);
             if (r_lo == 0) c_top = min(c_top + 64u, 65279u);
             if (r_hi == 0 && lane == 0) s_flag = 1;
-            const uint32_t c_bot = cell_of_rank(max(r_hi, 1u));
+            const uint32_t c_bot = min(cell_of_rank(max(r_hi, 1u)), c_top);
             const uint32_t ncell = c_top - c_bot + 1;
             if (ncell > (uint32_t)kFineBins) {
                 if (lane == 0) s_flag = 2;
@@ -242,12 +246,24 @@ k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint6
     __syncthreads();
     // merge overlapping / adjacent bands (they descend in key with j) into groups; groups end up in s_c*[0..ng)
     if (threadIdx.x == 0 && !s_flag) {
+        // The sweep reads a key's region from a table over the cells between the lowest and the highest band.  If
+        // that window has more cells than the table has entries, an entry stands for 2^cg cells and the bands
+        // are widened to whole entries (more fine bins; the common case is cg = 0).
+        uint32_t lo_all = 0xffffffffu, hi_all = 0, cg = 0;
+        for (uint32_t j = 0; j < K; ++j)
+            if (s_cb[j] <= s_ct[j]) { lo_all = min(lo_all, s_cb[j]); hi_all = max(hi_all, s_ct[j]); }
+        if (lo_all <= hi_all)
+            while ((hi_all >> cg) - (lo_all >> cg) + 3 > (uint32_t)kCellTab) ++cg;
+        s_cg = cg;
+        const uint32_t cmask = (1u << cg) - 1u;
         uint32_t ng = 0;
         uint32_t gb = 1, gt = 0, gs = 15;
         bool open = false;
         for (uint32_t j = 0; j < K; ++j) {
-            const uint32_t cb = s_cb[j], ct = s_ct[j], cs = s_cs[j];
+            uint32_t cb = s_cb[j], ct = s_ct[j];
+            const uint32_t cs = s_cs[j];
             if (cb > ct) continue;
+            cb &= ~cmask; ct |= cmask; // stays below the non-finite cells: 65279 ends a block of 32
             if (open && ct + 1 >= gb) {
                 gb = min(gb, cb); gt = max(gt, ct); gs = min(gs, cs);
             } else {
@@ -273,15 +289,14 @@ k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint6
         s_ng = ng;
     }
     __syncthreads();
-    const uint32_t ng = s_ng;
-    if (!s_flag)
-        for (uint32_t g = 0; g < ng; ++g)
-            for (uint32_t c = s_cb[g] + threadIdx.x; c <= s_ct[g]; c += kBigThreads) atomicOr(&bitmap[c >> 5], 1u << (c & 31));
-    __syncthreads();
-    // ---- bin ids in ascending key order: gap_0, fine bins of the lowest group, gap_1, ..., gap_ng, non-finite gap.
+    const uint32_t ng = s_ng, cg = s_cg;
+    // ---- bin ids in ascending key order: gap_0, fine bins of the lowest group, gap_1, ..., gap_ng, non-finite keys.
     // A gap region is cut at every 11-bit prefix (one bin per piece: keeps the shared-memory atomics of the sweep
-    // spread over many words).  Groups are stored with descending keys; a = ng - 1 - g is the ascending index.
-    // s_base[a] = first id of gap_a, s_aux[a] = lowest cell of gap_a; the non-finite gap is a = ng + 1.
+    // spread over many words); keys with exponent 255 take the eight pieces that follow gap_ng's, so that one
+    // formula serves everything above the highest band.  Groups are stored with descending keys; a = ng - 1 - g
+    // is the ascending index.  s_base[a] = first id of gap_a, s_glo[a] = lowest cell of gap_a.
+    // Every region -- a gap or a group of fine bins -- maps a key to its bin as base + (key >> shift) with one
+    // (base, shift) pair: shift 20 for the gap pieces, the group's bin width for the fine bins.
     uint32_t* s_glo = s_pre; // [kMaxGaps] reuse: the rank prefix is no longer needed
     if (threadIdx.x == 0 && !s_flag) {
         uint32_t id = 0;
@@ -297,215 +312,212 @@ k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint6
                 id += (s_ct[g] - s_cb[g] + 1) << (15 - s_cs[g]);
             }
         }
-        s_base[ng + 1] = id; // keys with exponent 255: one bin
-        s_glo[ng + 1] = 65280u;
-        s_base[ng + 2] = id + 1; // number of bins
-    }
-    uint32_t rows = bitmap[2 * threadIdx.x] != 0;
-    rows += bitmap[2 * threadIdx.x + 1] != 0;
-    uint32_t tot_rows;
-    uint32_t row = block_excl_scan<uint32_t, kBigThreads>(rows, s_w, &tot_rows); // includes the barrier for s_base
-    const uint32_t tot_bins = s_flag ? 0u : s_base[ng + 2];
-    const bool bad = s_flag || tot_rows > (uint32_t)kMaxRows || tot_bins > (uint32_t)kMaxBins;
-    if (bad) {
-        if (threadIdx.x == 0) *mt = BandMeta{tot_bins, tot_rows, 2, s_flag};
-        return;
-    }
-    // cell -> (lookup entry, is this the first cell of a bin that is a gap piece?)
-    auto entry_of = [&](uint32_t cell, bool& gap_first) -> uint32_t {
-        gap_first = false;
-        uint32_t a = ng + 1; // gap ordinal if the cell is in no band
-        if (cell < 65280u) {
-            a = 0;
-            for (; a < ng; ++a) {
-                const uint32_t g = ng - 1 - a;
-                if (cell > s_ct[g]) continue;
-                if (cell >= s_cb[g]) return (s_base[kMaxGaps + a] + ((cell - s_cb[g]) << (15 - s_cs[g]))) | (s_cs[g] << 16);
-                break;
-            }
-        }
-        const uint32_t lo = s_glo[a];
-        gap_first = cell == lo || (cell & 31u) == 0;
-        const uint32_t piece = a == ng + 1 ? 0u : (cell >> 5) - (lo >> 5);
-        return (s_base[a] + piece) | (15u << 16);
-    };
-    uint16_t* t1 = lut_t1 + wr * kL1Bins;
-    uint32_t* t2 = lut_t2 + wr * kLutWords;
-    uint32_t* blo = bin_lo + wr * (kMaxBins + 1);
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-        const uint32_t b1 = 2 * threadIdx.x + i;
-        if (bitmap[b1]) {
-            s_aux[b1] = row;
-            t1[b1] = (uint16_t)(0x8000u | row);
-            ++row;
-        } else { // no band cell inside: the whole 11-bit bin is one gap piece
-            bool first;
-            const uint32_t e = entry_of(b1 << 5, first);
-            t1[b1] = (uint16_t)(e & 0x7fffu);
-            if (first && (b1 <= 2040u)) blo[e & 0xffffu] = (b1 << 20) | kGapBit; // bins 2041.. share the non-finite bin
-        }
+        s_base[ng + 1] = id;     // keys with exponent 255: the pieces 2040..2047
+        s_base[ng + 2] = id + 8; // number of bins
     }
     __syncthreads();
-    // split bins: one warp per bin, one lane per cell
-    for (uint32_t b1 = threadIdx.x >> 5; b1 < (uint32_t)kL1Bins; b1 += kBigThreads / 32) {
-        const uint32_t wd = bitmap[b1];
-        if (!wd) continue;
-        const uint32_t cell = (b1 << 5) | lane;
-        bool first;
-        const uint32_t e = entry_of(cell, first);
-        t2[s_aux[b1] * 32 + lane] = e;
-        const uint32_t id = e & 0xffffu, shc = e >> 16;
-        if ((wd >> lane) & 1u) {
-            for (uint32_t i = 0; i < (1u << (15 - shc)); ++i) blo[id + i] = (cell << 15) + (i << shc);
-        } else if (first) {
-            blo[id] = (cell << 15) | kGapBit;
+    const uint32_t tot_bins = s_flag ? 0u : s_base[ng + 2];
+    // window of the cell table: the cells from the lowest to the highest band cell and one entry on either side
+    // (everything below lies in gap_0, everything above in gap_ng or among the non-finite keys)
+    // (in table entries of 2^cg cells each)
+    const uint32_t wlo = (ng ? s_cb[ng - 1] : 1u) >> cg, whi = (ng ? s_ct[0] : 1u) >> cg;
+    const uint32_t used = whi - wlo + 3;
+    const bool bad = s_flag || tot_bins > (uint32_t)kMaxBins || used > (uint32_t)kCellTab;
+    if (bad) {
+        if (threadIdx.x == 0) *mt = BandMeta{tot_bins, used, 2, s_flag};
+        return;
+    }
+    // (base, shift) of the region that holds a cell, as base << 5 | shift (base may be negative)
+    auto entry_of = [&](uint32_t cell) -> uint32_t {
+        uint32_t a = 0;
+        for (; a < ng; ++a) {
+            const uint32_t g = ng - 1 - a;
+            if (cell > s_ct[g]) continue;
+            if (cell >= s_cb[g]) {
+                const uint32_t cs = s_cs[g];
+                return (uint32_t)(((int)s_base[kMaxGaps + a] - (int)(s_cb[g] << (15 - cs))) * 32) | cs;
+            }
+            break;
         }
+        return (uint32_t)(((int)s_base[a] - (int)(s_glo[a] >> 5)) * 32) | 20u;
+    };
+    uint32_t* tab = cell_tab + wr * kCellTab;
+    uint32_t* blo = bin_lo + wr * (kMaxBins + 1);
+    // entry i serves the cells (wlo - 1 + i) << cg ...; the first one everything below the window, the last one
+    // everything above it
+    for (uint32_t i = threadIdx.x; i < used; i += kBigThreads) tab[i] = entry_of(i + 1 == used ? 65535u : (wlo + i - 1u) << cg);
+    // lower key of every bin: the pieces of the gaps ...
+    for (uint32_t b1 = threadIdx.x; b1 < (uint32_t)kL1Bins; b1 += kBigThreads) {
+        const uint32_t c0 = b1 << 5, c1 = c0 + 31;
+        if (b1 >= 2040u) { blo[s_base[ng + 1] + (b1 - 2040u)] = (b1 << 20) | kGapBit; continue; }
+        for (uint32_t a = 0; a <= ng; ++a) {
+            const uint32_t lo = s_glo[a];
+            const uint32_t hi = a == ng ? 65279u : s_cb[ng - 1 - a] - 1;
+            if (hi + 1 <= lo || hi < c0 || lo > c1) continue;
+            blo[s_base[a] + b1 - (lo >> 5)] = (max(lo, c0) << 15) | kGapBit;
+        }
+    }
+    // ... and the fine bins of the groups
+    for (uint32_t a = 0; a < ng; ++a) {
+        const uint32_t g = ng - 1 - a, cs = s_cs[g], first = s_base[kMaxGaps + a];
+        const uint32_t nf = (s_ct[g] - s_cb[g] + 1) << (15 - cs);
+        for (uint32_t x = threadIdx.x; x < nf; x += kBigThreads) blo[first + x] = (s_cb[g] << 15) + (x << cs);
     }
     if (threadIdx.x == 0) {
         blo[tot_bins] = 0x80000000u;
-        *mt = BandMeta{tot_bins, tot_rows, 0, ng + 2};
+        cell_win[wr] = make_int4((int)wlo - 1, (int)whi + 1, (int)(15 + cg), 0);
+        *mt = BandMeta{tot_bins, used, 0, ng + 2};
     }
 }
 
 // ------------------------------------------------------------------------------------------------
-// k_pass_a: CTAs own runs of consecutive chunks; histogram words live in shared memory
+// k_pass_a: every CTA owns one static run of consecutive chunks of one worker (runs balanced by elements, a few
+// per SM); histogram words and the cell table of the current layer live in shared memory
 // ------------------------------------------------------------------------------------------------
-constexpr int kMaxRunChunksA = 32; // a run has at most 2^20 elements: its carry count stays far below 2^32
+struct SweepRun { uint32_t w, c0, c1; }; // chunks [c0, c1) of worker w
+constexpr int kRunDesc = 64;             // chunk descriptors staged in shared memory at a time
 
 template <bool VEC>
 __global__ void __launch_bounds__(kBigThreads, 1)
 k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, uint16_t* __restrict__ d_hi,
-         const Chunk* __restrict__ chunks, uint32_t n_chunks, uint32_t run_chunks, uint64_t stride, uint64_t dstride,
+         const Chunk* __restrict__ chunks, const SweepRun* __restrict__ runs, uint64_t stride, uint64_t dstride,
          const uint32_t* __restrict__ reg_index /* [L], 0xffffffff: tiny layer */, uint32_t R,
-         const uint16_t* __restrict__ lut_t1, const uint32_t* __restrict__ lut_t2, const BandMeta* __restrict__ meta,
+         const uint32_t* __restrict__ cell_tab, const int4* __restrict__ cell_win, const BandMeta* __restrict__ meta,
          uint32_t* __restrict__ bh_cnt, unsigned long long* __restrict__ bh_sum) {
-    pdl_wait();
     extern __shared__ __align__(16) uint32_t sh[];
+    __shared__ Chunk s_desc[kRunDesc];
     uint32_t* h_cnt = sh;
-    uint32_t* h_hi = sh + kMaxBins;
-    uint32_t* h_lo = sh + 2 * kMaxBins;
-    uint32_t* t2 = sh + 3 * kMaxBins;                           // [kLutWords] cell rows, then gap ids
-    uint16_t* t1 = reinterpret_cast<uint16_t*>(t2 + kLutWords); // [2048]
-    static_assert((uint64_t)kMaxRunChunksA * kChunkElems <= (1ull << 20), "run length");
-    const uint32_t w = blockIdx.y;
-    const uint32_t c0 = blockIdx.x * run_chunks, c1 = min(n_chunks, c0 + run_chunks);
-    for (int i = threadIdx.x; i < 3 * kMaxBins; i += kBigThreads) sh[i] = 0;
-    const float* gr0 = grads + (size_t)w * stride;
-    const float* st0 = state + (size_t)w * stride;
-    uint16_t* dh0 = d_hi + (size_t)w * dstride;
+    uint32_t* h_lo = sh + kMaxBins;
+    uint32_t* tab = sh + 2 * kMaxBins; // [kCellTab]
+    // the run, its first chunk descriptors and the clean histogram do not depend on the kernels before this one
+    const SweepRun run = runs[blockIdx.x];
+    for (int i = threadIdx.x; i < 2 * kMaxBins; i += kBigThreads) sh[i] = 0;
+    for (uint32_t i = threadIdx.x; i < min(run.c1 - run.c0, (uint32_t)kRunDesc); i += kBigThreads) s_desc[i] = chunks[run.c0 + i];
+    pdl_wait();
+    __syncthreads();
+    const float* gr0 = grads + (size_t)run.w * stride;
+    const float* st0 = state + (size_t)run.w * stride;
+    uint16_t* dh0 = d_hi + (size_t)run.w * dstride;
     int cur_layer = -1;
-    bool active = false, dirty = false;
-    uint32_t n_bins = 0;
-    uint32_t* gc = nullptr;
-    unsigned long long* gs = nullptr;
+    uint32_t wr = 0xffffffffu; // slot of the current layer's histogram; 0xffffffff: none (tiny or handed-over layer)
+    bool dirty = false;
+    int wlo_m1 = 0, whi_p1 = 0;  // cells of the table's first and last entry, in units of 2^(cshift - 15) cells
+    uint32_t cshift = 15;
 
     auto flush = [&]() {
         __syncthreads();
+        const uint32_t n_bins = meta[wr].n_bins;
+        uint32_t* gc = bh_cnt + (size_t)wr * kMaxBins;
+        unsigned long long* gs = bh_sum + (size_t)wr * kMaxBins;
         for (uint32_t i = threadIdx.x; i < n_bins; i += kBigThreads) {
             const uint32_t c = h_cnt[i];
             if (c) {
                 atomicAdd(&gc[i], c);
-                atomicAdd(&gs[i], ((unsigned long long)h_hi[i] << 32) + h_lo[i]);
-                h_cnt[i] = 0; h_hi[i] = 0; h_lo[i] = 0;
+                atomicAdd(&gs[i], (unsigned long long)h_lo[i]);
+                h_cnt[i] = 0; h_lo[i] = 0;
             }
         }
         __syncthreads();
         dirty = false;
     };
-    // bin of a key: first-level entry (11-bit prefix), then, inside split prefixes, the cell's entry
-    auto entry1 = [&](uint32_t key) -> uint32_t { return t1[key >> 20]; };
-    auto bin_of = [&](uint32_t key, uint32_t e1) -> uint32_t {
-        const bool split = e1 & 0x8000u;
-        const uint32_t e2 = split ? t2[(e1 & 0x7fffu) * 32 + ((key >> 15) & 31u)] : 0u; // lanes outside split bins issue no load
-        return split ? (e2 & 0xffffu) + ((key & 0x7fffu) >> (e2 >> 16)) : e1;
-    };
+    // (base, shift) of the region a key lies in: one table read; the clamp sends everything outside the window to
+    // the table's first or last entry
+    auto look = [&](uint32_t key) -> uint32_t { return tab[min(max((int)(key >> cshift), wlo_m1), whi_p1) - wlo_m1]; };
+    auto bin_of = [&](uint32_t key, uint32_t e) -> uint32_t { return (uint32_t)(((int)e >> 5) + (int)(key >> (e & 31u))); };
     auto add = [&](uint32_t id, uint32_t key) {
-        // 24 significant bits of the square (truncation < 2^-22 relative) summed exactly: the low word wraps, the
-        // returned old value tells when, and the wraps are counted in the high word
+        // 24 significant bits of the square (truncation < 2^-22 relative) summed exactly: the word wraps, the
+        // returned old value tells when, and a wrap adds 2^32 to the layer's 64-bit sum in global memory
         const uint32_t sq = (uint32_t)(sq_fixed(key) >> 8);
-        if (!KIMAD_CHECK(id < n_bins, 0)) return;
+#ifdef KIMAD_CHECKED
+        if (!KIMAD_CHECK(id < meta[wr].n_bins, 0)) return;
+#endif
         atomicAdd(&h_cnt[id], 1u);
         const uint32_t old = atomicAdd(&h_lo[id], sq);
-        if (old + sq < old) atomicAdd(&h_hi[id], 1u); // carry out of the low word (rare)
+        if (old + sq < old) atomicAdd(bh_sum + (size_t)wr * kMaxBins + id, 1ull << 32); // rare
     };
     auto acc = [&](float dv) {
         const uint32_t key = key_of(dv);
-        add(bin_of(key, entry1(key)), key);
+        add(bin_of(key, look(key)), key);
     };
-    // The four elements of a quad go through the stages together (all first-level reads, then all second-level
-    // reads, then the atomics): four independent chains of dependent shared-memory accesses instead of one after
-    // the other (3 % on the sweep; the kernel is bound by instruction issue and shared-memory latency, not by DRAM:
-    // with its loads served from cache it still takes 0.9 of its time)
+    // The four elements of a quad go through the stages together (all table reads, then the bin ids, then the
+    // atomics): four independent chains of dependent shared-memory accesses instead of one after the other
     auto acc4 = [&](const float4& d) {
         const uint32_t k[4] = {key_of(d.x), key_of(d.y), key_of(d.z), key_of(d.w)};
         uint32_t e[4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) e[i] = entry1(k[i]);
+        for (int i = 0; i < 4; ++i) e[i] = look(k[i]);
 #pragma unroll
         for (int i = 0; i < 4; ++i) e[i] = bin_of(k[i], e[i]);
 #pragma unroll
         for (int i = 0; i < 4; ++i) add(e[i], k[i]);
     };
 
-    for (uint32_t c = c0; c < c1; ++c) {
-        const Chunk ch = chunks[c];
+    for (uint32_t c = run.c0; c < run.c1; ++c) {
+        const uint32_t di = (c - run.c0) % (uint32_t)kRunDesc;
+        if (di == 0 && c != run.c0) { // next window of descriptors
+            __syncthreads();
+            for (uint32_t i = threadIdx.x; i < min(run.c1 - c, (uint32_t)kRunDesc); i += kBigThreads) s_desc[i] = chunks[c + i];
+            __syncthreads();
+        }
+        const Chunk ch = s_desc[di];
         if ((int)ch.layer != cur_layer) {
             if (dirty) flush();
             cur_layer = (int)ch.layer;
             const uint32_t r = reg_index[ch.layer];
-            active = false;
-            if (r != 0xffffffffu) {
-                const size_t wr = (size_t)w * R + r;
-                const BandMeta mt = meta[wr];
-                if (!mt.flagged) {
-                    active = true;
-                    n_bins = mt.n_bins;
-                    gc = bh_cnt + wr * kMaxBins;
-                    gs = bh_sum + wr * kMaxBins;
-                    __syncthreads();
-                    const uint32_t* g1 = reinterpret_cast<const uint32_t*>(lut_t1 + wr * kL1Bins);
-                    for (int i = threadIdx.x; i < kL1Bins / 2; i += kBigThreads) reinterpret_cast<uint32_t*>(t1)[i] = g1[i];
-                    const uint32_t* g2 = lut_t2 + wr * kLutWords;
-                    for (uint32_t i = threadIdx.x; i < mt.n_rows * 32; i += kBigThreads) t2[i] = g2[i];
-                }
+            wr = 0xffffffffu;
+            __syncthreads(); // the table is no longer read
+            if (r != 0xffffffffu && !meta[run.w * R + r].flagged) {
+                wr = run.w * R + r;
+                const int4 win = cell_win[wr];
+                wlo_m1 = win.x; whi_p1 = win.y; cshift = (uint32_t)win.z;
+                const uint32_t* g2 = cell_tab + (size_t)wr * kCellTab;
+                const uint32_t used = meta[wr].n_cells;
+                for (uint32_t i = threadIdx.x; i < used; i += kBigThreads) tab[i] = g2[i];
             }
             __syncthreads();
         }
+        const bool active = wr != 0xffffffffu;
         const ChunkView cv(ch);
-        const float* gr = gr0 + cv.a0;
-        const float* st = st0 + cv.a0;
         uint16_t* dh = dh0 + cv.a0;
-        const uint32_t nq = cv.quads();
-        constexpr int U = 4; // quads in flight per thread: 16 KB per array and pass, two passes per full chunk
-        for (uint32_t qb = 0; qb < nq; qb += kBigThreads * U) {
-            float4 a[U], b[U];
+        if (VEC) {
+            const float4* gr4 = reinterpret_cast<const float4*>(gr0 + cv.a0);
+            const float4* st4 = reinterpret_cast<const float4*>(st0 + cv.a0);
+            const uint32_t q_lo = (cv.first + 3) >> 2, q_hi = cv.len >> 2; // whole quads [q_lo, q_hi)
+            constexpr int U = 4; // quads in flight per thread: 16 KB per array and pass, two passes per full chunk
+            for (uint32_t qb = q_lo + threadIdx.x; qb < q_hi; qb += kBigThreads * U) {
+                float4 a[U], b[U];
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const uint32_t q = qb + u * kBigThreads + threadIdx.x;
-                if (VEC && q < nq && cv.quad_full(q)) {
-                    a[u] = __ldcs(reinterpret_cast<const float4*>(gr) + q);
-                    b[u] = __ldcs(reinterpret_cast<const float4*>(st) + q);
+                for (int u = 0; u < U; ++u) {
+                    const uint32_t q = qb + u * kBigThreads;
+                    if (q < q_hi) { a[u] = __ldcg(gr4 + q); b[u] = __ldcg(st4 + q); }
+                }
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const uint32_t q = qb + u * kBigThreads;
+                    if (q < q_hi) {
+                        float4 d;
+                        d.x = __fsub_rn(a[u].x, b[u].x); d.y = __fsub_rn(a[u].y, b[u].y);
+                        d.z = __fsub_rn(a[u].z, b[u].z); d.w = __fsub_rn(a[u].w, b[u].w);
+                        reinterpret_cast<uint2*>(dh)[q] = upper_halves(d);
+                        if (active) acc4(d);
+                    }
                 }
             }
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const uint32_t q = qb + u * kBigThreads + threadIdx.x;
-                if (q >= nq) continue;
-                if (VEC && cv.quad_full(q)) {
-                    float4 d;
-                    d.x = __fsub_rn(a[u].x, b[u].x); d.y = __fsub_rn(a[u].y, b[u].y);
-                    d.z = __fsub_rn(a[u].z, b[u].z); d.w = __fsub_rn(a[u].w, b[u].w);
-                    reinterpret_cast<uint2*>(dh)[q] = upper_halves(d);
-                    if (active) acc4(d);
-                } else {
-                    for (uint32_t e = 4 * q; e < 4 * q + 4; ++e)
-                        if (e >= cv.first && e < cv.len) {
-                            const float d = __fsub_rn(gr[e], st[e]);
-                            dh[e] = (uint16_t)(__float_as_uint(d) >> 16);
-                            if (active) acc(d);
-                        }
+            if (threadIdx.x < 8) { // ragged edges: [first, min(4 q_lo, len)) and [max(4 q_hi, 4 q_lo), len)
+                uint32_t e;
+                if (threadIdx.x < 4) { e = cv.first + threadIdx.x; if (e >= min(4 * q_lo, cv.len)) e = 0xffffffffu; }
+                else { e = max(4 * q_hi, 4 * q_lo) + (threadIdx.x - 4); if (e >= cv.len) e = 0xffffffffu; }
+                if (e != 0xffffffffu) {
+                    const float d = __fsub_rn(gr0[cv.a0 + e], st0[cv.a0 + e]);
+                    dh[e] = (uint16_t)(__float_as_uint(d) >> 16);
+                    if (active) acc(d);
                 }
+            }
+        } else {
+            for (uint32_t e = cv.first + threadIdx.x; e < cv.len; e += kBigThreads) {
+                const float d = __fsub_rn(gr0[cv.a0 + e], st0[cv.a0 + e]);
+                dh[e] = (uint16_t)(__float_as_uint(d) >> 16);
+                if (active) acc(d);
             }
         }
         if (active) dirty = true;
