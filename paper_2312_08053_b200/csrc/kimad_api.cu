@@ -80,7 +80,7 @@ void plan_layout(kimad_ctx* c) {
     };
     const size_t WL = (size_t)c->W * c->L, WLK = WL * c->K, WR = (size_t)c->W * c->reg_layers.size();
     const size_t nch = c->chunks.size();
-    y.dbuf = take((size_t)c->W * c->dstride * sizeof(uint16_t));
+    y.dbuf = take((size_t)c->W * c->dstride * sizeof(uint8_t));
     y.chunks = take(nch * sizeof(Chunk));
     y.layers = take(c->layers.size() * sizeof(LayerDesc));
     y.ktab = take(c->ktab.size() * sizeof(uint64_t));
@@ -215,8 +215,8 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
     const bool vec = ((uintptr_t)grads % 16 == 0) && ((uintptr_t)state % 16 == 0) && (c->stride % 4 == 0);
 
     const Layout& y = c->lay;
-    // the upper halves of d, u16 [W][dstride]; exact values are recomputed from grads and state
-    const DSource dbuf{c->at<uint16_t>(y.dbuf), grads, state, c->stride};
+    // one code byte per element, u8 [W][dstride]; exact values are recomputed from grads and state
+    const DSource dbuf{c->at<uint8_t>(y.dbuf), grads, state, c->stride};
     const Chunk* chunks = c->at<Chunk>(y.chunks);
     const LayerDesc* layers = c->at<LayerDesc>(y.layers);
     // candidates: the grid's table for every worker, or (policy 3) each worker's row of the ratio fitted to its budget
@@ -288,10 +288,10 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
     }
     mark();
     if (vec)
-        CUDA_TRY(launch_pdl(k_pass_a<true>, n_runs, kBigThreads, c->pass_a_smem, s, grads, state, dbuf.hi, chunks, runs,
+        CUDA_TRY(launch_pdl(k_pass_a<true>, n_runs, kBigThreads, c->pass_a_smem, s, grads, state, dbuf.code, chunks, runs,
                             c->stride, c->dstride, reg_index, R, cell_tab, cell_win, meta, bhc, bhs));
     else
-        CUDA_TRY(launch_pdl(k_pass_a<false>, n_runs, kBigThreads, c->pass_a_smem, s, grads, state, dbuf.hi, chunks, runs,
+        CUDA_TRY(launch_pdl(k_pass_a<false>, n_runs, kBigThreads, c->pass_a_smem, s, grads, state, dbuf.code, chunks, runs,
                             c->stride, c->dstride, reg_index, R, cell_tab, cell_win, meta, bhc, bhs));
     c->launches += 1;
     mark();
@@ -333,7 +333,7 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
         CUDA_TRY(launch_pdl(k_dp, nw, kDpThreads, c->dp_smem, s, budgets_of(w0, nw), w0, W, L, K, c->D, c->bpe, c->full_bytes, c->cap,
                             c->check_finite, dp_mode, c->cost_model, c->dp_plan, layers,
                             ktab, mode == kInjectErr ? err_dev : err, tau, keq, shf, j_dev, flags, pd, sel, out->k, out->j,
-                            out->offs, out->stats, out->dense));
+                            out->offs, out->stats, out->dense, CodeSpace{reg_index, meta, cell_tab, cell_win, R}));
         c->launches += 1;
     }
     mark();
@@ -434,7 +434,7 @@ int kimad_create(kimad_ctx** out, const uint64_t* layer_sizes, uint32_t n_layers
         c->stride = o.worker_stride ? o.worker_stride : N;
         c->cap = o.max_packed_elems ? o.max_packed_elems : N;
         if (c->stride < N || c->chunks.size() > 0x7fffffffull) { delete c; return KIMAD_ERR_INVALID_ARG; }
-        c->dstride = (N + 3) / 4 * 4;
+        c->dstride = (N + 15) / 16 * 16; // every worker's code plane starts on a 16-byte boundary
         // shared-memory plan of the DP kernel
         const size_t Kp = (c->K + 3) & ~(size_t)3;
         const size_t dp_base = ((size_t)2 * (2 * c->D + 3) + c->L) * 4 + 16; // + alignment slack of the candidate tables

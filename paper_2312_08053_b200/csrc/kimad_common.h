@@ -67,7 +67,8 @@ struct Sel {
     uint32_t k;       // 0: nothing to pack for this layer (the worker failed)
     uint32_t shift;   // log2 of the interval width (<= 10)
     uint32_t tau_low; // exact threshold minus the interval's lower key
-    uint32_t _pad;
+    uint32_t code;    // the code (byte plane of the sweep) of the keys of the interval: entries with a larger code lie
+                      // above the interval, entries with a smaller one below
     uint64_t base;    // first output position of the layer in the worker's packed buffers
 };
 

@@ -29,20 +29,11 @@ constexpr int kTinyMax = 4096;
 constexpr int kFineBins = KIMAD_FINE_BINS;          // fine bins per (worker, layer)
 constexpr int kMaxGaps = KIMAD_MAX_RATIOS + 2;      // gap regions: below / between / above the band groups, + non-finite keys
 constexpr int kMaxBins = kFineBins + kL1Bins + 2 * kMaxGaps; // fine bins + gap regions cut at every 11-bit prefix
-constexpr int kCellTab = 4096;                      // entries of the cell table: the window of cells from the lowest to the
-                                                    // highest band (32 octaves) and one entry on either side
 constexpr int kMaxShift = 15;                       // a fine bin is 2^shift keys wide, at most a whole cell
 constexpr int kSampleUnits = 4095;                  // sample = units of 16 consecutive elements (<= 65520 elements)
 constexpr int kBigThreads = 1024;
 constexpr uint32_t kGapBit = 1u;                    // bin_lo entries carry this bit when the bin is a gap bin
 
-struct BandMeta { // per (worker, regular layer)
-    uint32_t n_bins;
-    uint32_t n_cells; // entries of the cell table in use
-    uint32_t flagged; // != 0: this layer takes the exact radix path in this step
-    uint32_t n_gaps;  // gap regions (when flagged: detail of the misfit)
-};
-// entry of the cell table: base << 5 | shift (base signed); the bin of a key is base + (key >> shift)
 
 __device__ __forceinline__ uint32_t hash_u32(uint32_t x) {
     x ^= x >> 16; x *= 0x7feb352du; x ^= x >> 15; x *= 0x846ca68bu; x ^= x >> 16;
@@ -365,7 +356,9 @@ k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint6
     }
     if (threadIdx.x == 0) {
         blo[tot_bins] = 0x80000000u;
-        cell_win[wr] = make_int4((int)wlo - 1, (int)whi + 1, (int)(15 + cg), 0);
+        uint32_t ls = 0; // bins per code of the byte plane: the codes stay below 128
+        while (((tot_bins - 1) >> ls) > 127u) ++ls;
+        cell_win[wr] = make_int4((int)wlo - 1, (int)whi + 1, (int)(15 + cg), (int)ls);
         *mt = BandMeta{tot_bins, used, 0, ng + 2};
     }
 }
@@ -379,7 +372,7 @@ constexpr int kRunDesc = 64;             // chunk descriptors staged in shared m
 
 template <bool VEC>
 __global__ void __launch_bounds__(kBigThreads, 1)
-k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, uint16_t* __restrict__ d_hi,
+k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, uint8_t* __restrict__ d_code,
          const Chunk* __restrict__ chunks, const SweepRun* __restrict__ runs, uint64_t stride, uint64_t dstride,
          const uint32_t* __restrict__ reg_index /* [L], 0xffffffff: tiny layer */, uint32_t R,
          const uint32_t* __restrict__ cell_tab, const int4* __restrict__ cell_win, const BandMeta* __restrict__ meta,
@@ -397,12 +390,12 @@ k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, uint1
     __syncthreads();
     const float* gr0 = grads + (size_t)run.w * stride;
     const float* st0 = state + (size_t)run.w * stride;
-    uint16_t* dh0 = d_hi + (size_t)run.w * dstride;
+    uint8_t* dc0 = d_code + (size_t)run.w * dstride;
     int cur_layer = -1;
     uint32_t wr = 0xffffffffu; // slot of the current layer's histogram; 0xffffffff: none (tiny or handed-over layer)
     bool dirty = false;
     int wlo_m1 = 0, whi_p1 = 0;  // cells of the table's first and last entry, in units of 2^(cshift - 15) cells
-    uint32_t cshift = 15;
+    uint32_t cshift = 15, lshift = 0; // keys per table entry, bins per code (log2)
 
     auto flush = [&]() {
         __syncthreads();
@@ -435,14 +428,16 @@ k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, uint1
         const uint32_t old = atomicAdd(&h_lo[id], sq);
         if (old + sq < old) atomicAdd(bh_sum + (size_t)wr * kMaxBins + id, 1ull << 32); // rare
     };
-    auto acc = [&](float dv) {
-        const uint32_t key = key_of(dv);
-        add(bin_of(key, look(key)), key);
+    // one element: its bin's count and sum; returns its code
+    auto acc = [&](uint32_t key) -> uint32_t {
+        const uint32_t id = bin_of(key, look(key));
+        add(id, key);
+        return id >> lshift;
     };
     // The four elements of a quad go through the stages together (all table reads, then the bin ids, then the
-    // atomics): four independent chains of dependent shared-memory accesses instead of one after the other
-    auto acc4 = [&](const float4& d) {
-        const uint32_t k[4] = {key_of(d.x), key_of(d.y), key_of(d.z), key_of(d.w)};
+    // atomics): four independent chains of dependent shared-memory accesses instead of one after the other.
+    // Returns the quad's four codes.
+    auto acc4 = [&](const uint32_t (&k)[4]) -> uint32_t {
         uint32_t e[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) e[i] = look(k[i]);
@@ -450,6 +445,7 @@ k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, uint1
         for (int i = 0; i < 4; ++i) e[i] = bin_of(k[i], e[i]);
 #pragma unroll
         for (int i = 0; i < 4; ++i) add(e[i], k[i]);
+        return pack_low_bytes(e[0] >> lshift, e[1] >> lshift, e[2] >> lshift, e[3] >> lshift);
     };
 
     for (uint32_t c = run.c0; c < run.c1; ++c) {
@@ -469,7 +465,7 @@ k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, uint1
             if (r != 0xffffffffu && !meta[run.w * R + r].flagged) {
                 wr = run.w * R + r;
                 const int4 win = cell_win[wr];
-                wlo_m1 = win.x; whi_p1 = win.y; cshift = (uint32_t)win.z;
+                wlo_m1 = win.x; whi_p1 = win.y; cshift = (uint32_t)win.z; lshift = (uint32_t)win.w;
                 const uint32_t* g2 = cell_tab + (size_t)wr * kCellTab;
                 const uint32_t used = meta[wr].n_cells;
                 for (uint32_t i = threadIdx.x; i < used; i += kBigThreads) tab[i] = g2[i];
@@ -478,7 +474,7 @@ k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, uint1
         }
         const bool active = wr != 0xffffffffu;
         const ChunkView cv(ch);
-        uint16_t* dh = dh0 + cv.a0;
+        uint8_t* dc = dc0 + cv.a0;
         if (VEC) {
             const float4* gr4 = reinterpret_cast<const float4*>(gr0 + cv.a0);
             const float4* st4 = reinterpret_cast<const float4*>(st0 + cv.a0);
@@ -495,11 +491,9 @@ k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, uint1
                 for (int u = 0; u < U; ++u) {
                     const uint32_t q = qb + u * kBigThreads;
                     if (q < q_hi) {
-                        float4 d;
-                        d.x = __fsub_rn(a[u].x, b[u].x); d.y = __fsub_rn(a[u].y, b[u].y);
-                        d.z = __fsub_rn(a[u].z, b[u].z); d.w = __fsub_rn(a[u].w, b[u].w);
-                        reinterpret_cast<uint2*>(dh)[q] = upper_halves(d);
-                        if (active) acc4(d);
+                        const uint32_t k[4] = {key_of(__fsub_rn(a[u].x, b[u].x)), key_of(__fsub_rn(a[u].y, b[u].y)),
+                                               key_of(__fsub_rn(a[u].z, b[u].z)), key_of(__fsub_rn(a[u].w, b[u].w))};
+                        reinterpret_cast<uint32_t*>(dc)[q] = active ? acc4(k) : pack_key_codes(k[0], k[1], k[2], k[3]);
                     }
                 }
             }
@@ -508,16 +502,14 @@ k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, uint1
                 if (threadIdx.x < 4) { e = cv.first + threadIdx.x; if (e >= min(4 * q_lo, cv.len)) e = 0xffffffffu; }
                 else { e = max(4 * q_hi, 4 * q_lo) + (threadIdx.x - 4); if (e >= cv.len) e = 0xffffffffu; }
                 if (e != 0xffffffffu) {
-                    const float d = __fsub_rn(gr0[cv.a0 + e], st0[cv.a0 + e]);
-                    dh[e] = (uint16_t)(__float_as_uint(d) >> 16);
-                    if (active) acc(d);
+                    const uint32_t key = key_of(__fsub_rn(gr0[cv.a0 + e], st0[cv.a0 + e]));
+                    dc[e] = (uint8_t)(active ? acc(key) : code_of_key(key));
                 }
             }
         } else {
             for (uint32_t e = cv.first + threadIdx.x; e < cv.len; e += kBigThreads) {
-                const float d = __fsub_rn(gr0[cv.a0 + e], st0[cv.a0 + e]);
-                dh[e] = (uint16_t)(__float_as_uint(d) >> 16);
-                if (active) acc(d);
+                const uint32_t key = key_of(__fsub_rn(gr0[cv.a0 + e], st0[cv.a0 + e]));
+                dc[e] = (uint8_t)(active ? acc(key) : code_of_key(key));
             }
         }
         if (active) dirty = true;

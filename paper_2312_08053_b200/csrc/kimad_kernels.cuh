@@ -5,8 +5,8 @@
 //   k_sample        (a)+(b) per (worker, layer): stratified sample of |grad - g| -> for every candidate k_j the
 //                   band of 16-bit key prefixes that can hold its threshold -> bin tables        [kimad_curve.cuh]
 //   k_pass_a        (a)+(b) the sweep: d = grad - g (Section 3 footnote, Eq. 6), bin = table(key(d)), count and
-//                   exact integer sum of squares per bin in shared memory; the upper halves of the bit patterns
-//                   of d go to scratch (d itself is never stored)                                [kimad_curve.cuh]
+//                   exact integer sum of squares per bin in shared memory; one byte per element (a monotone code
+//                   of its bin) goes to scratch, d itself is never stored                         [kimad_curve.cuh]
 //   k_resolve_a     (b) Eq. 4 / the "Errors" matrix of Algorithm 3: err_l(k_j) from the bins, certified to the
 //                   curve tolerance; layers that fail the certificate are handed to the exact path [kimad_curve.cuh]
 //   k_tiny_exact    (b) layers of at most 4096 elements, sorted in shared memory                 [kimad_curve.cuh]
@@ -37,45 +37,53 @@ constexpr int kL23Bins = 1024; // 10 bits each
 
 __device__ __forceinline__ uint32_t key_of(float d) { return __float_as_uint(d) & 0x7fffffffu; }
 
-// Aligned view of a chunk for 128-bit loads: quads start at a0 = begin & ~3; only the first and the
-// last quad can be partial.  All offsets are 32-bit and relative to a0.
 // Kernels launched with programmatic stream serialisation may be scheduled before their predecessor in the
 // stream has finished (which hides their launch latency); they wait here, before touching anything it wrote.
 // A no-op for an ordinary launch.
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
+// Aligned view of a chunk for 128-bit loads of the inputs (quads of elements) and of the code plane (sixteen
+// codes): units start at a0 = begin & ~15; only the first and the last ones can be partial.  All offsets are
+// 32-bit and relative to a0.
 struct ChunkView {
     uint64_t a0;
     uint32_t first, len; // valid element offsets are [first, len)
     __device__ __forceinline__ explicit ChunkView(const Chunk& ch)
-        : a0(ch.begin & ~3ull), first((uint32_t)(ch.begin - (ch.begin & ~3ull))), len((uint32_t)(ch.end - (ch.begin & ~3ull))) {}
+        : a0(ch.begin & ~15ull), first((uint32_t)(ch.begin - (ch.begin & ~15ull))), len((uint32_t)(ch.end - (ch.begin & ~15ull))) {}
     __device__ __forceinline__ uint32_t quads() const { return (len + 3) >> 2; }
     __device__ __forceinline__ bool quad_full(uint32_t q) const { return 4 * q >= first && 4 * q + 4 <= len; }
 };
 
-// The difference vector d = grad - g is never stored whole.  The sweep leaves the UPPER halves of its binary32 bit
-// patterns (u16 [W][dstride]): the counting sweep of the select stage orders keys by them and needs the exact
-// value only for the few keys that share an upper half with the threshold; whoever needs an exact d recomputes
-// the one subtraction from the inputs (the estimator is not written before the write sweep, and there every
-// element is read before it is updated).
+// The difference vector d = grad - g is never stored.  The sweep leaves one BYTE per element (u8 [W][dstride]): a
+// 7-bit code that never decreases with the magnitude key inside a layer -- the element's histogram bin divided by
+// a power of two for layers swept with a histogram, the upper seven bits of the key otherwise (code_of_key).  The
+// counting sweep of the select stage classifies an entry as above or below the threshold by its code and needs the
+// exact value only for the entries whose code equals the threshold's; whoever needs an exact d recomputes the one
+// subtraction from the inputs (the estimator is not written before the write sweep, and there every element is
+// read before it is updated).
 struct DSource {
-    uint16_t* hi;
+    uint8_t* code;
     const float* grads;
     const float* state;
     uint64_t stride; // elements between workers in grads / state
 };
 struct DView { // one worker's data at a chunk's aligned start
-    const uint16_t* hi;
+    const uint8_t* code;
     const float* gr;
     const float* st;
     __device__ __forceinline__ DView(const DSource& p, uint32_t w, uint64_t dstride, uint64_t a0)
-        : hi(p.hi + (size_t)w * dstride + a0), gr(p.grads + (size_t)w * p.stride + a0), st(p.state + (size_t)w * p.stride + a0) {}
+        : code(p.code + (size_t)w * dstride + a0), gr(p.grads + (size_t)w * p.stride + a0), st(p.state + (size_t)w * p.stride + a0) {}
     __device__ __forceinline__ float at(uint32_t e) const { return __fsub_rn(gr[e], st[e]); }
 };
-// the upper halves of a quad of values as two words
-__device__ __forceinline__ uint2 upper_halves(const float4& d) {
-    return make_uint2(__byte_perm(__float_as_uint(d.x), __float_as_uint(d.y), 0x7632),
-                      __byte_perm(__float_as_uint(d.z), __float_as_uint(d.w), 0x7632));
+// code of layers without a histogram: the upper seven bits of the 31-bit key
+__device__ __forceinline__ uint32_t code_of_key(uint32_t key) { return key >> 24; }
+// the lowest bytes of four words as one word (element 0 in the lowest byte)
+__device__ __forceinline__ uint32_t pack_low_bytes(uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    return __byte_perm(__byte_perm(a, b, 0x0040), __byte_perm(c, d, 0x0040), 0x5410);
+}
+// the codes of a quad of keys of a layer without a histogram (the highest byte of every key)
+__device__ __forceinline__ uint32_t pack_key_codes(uint32_t k0, uint32_t k1, uint32_t k2, uint32_t k3) {
+    return __byte_perm(__byte_perm(k0, k1, 0x0073), __byte_perm(k2, k3, 0x0073), 0x5410);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -342,6 +350,38 @@ k_rebuild_slots(const FbList* __restrict__ fb, const uint2* __restrict__ fb_laye
 }
 
 // ------------------------------------------------------------------------------------------------
+// What the sample kernel leaves per (worker, regular layer) for the sweep (details in kimad_curve.cuh)
+// ------------------------------------------------------------------------------------------------
+constexpr int kCellTab = 4096; // entries of the cell table: the window of cells from the lowest to the highest band
+                               // and one entry on either side
+struct BandMeta {
+    uint32_t n_bins;
+    uint32_t n_cells; // entries of the cell table in use
+    uint32_t flagged; // != 0: this layer takes the exact radix path in this step (and is swept without a histogram)
+    uint32_t n_gaps;  // gap regions (when flagged: detail of the misfit)
+};
+// entry of the cell table: base << 5 | shift (base signed): the bin of a key is base + (key >> shift).
+// window of a layer: {cell of the first entry, cell of the last entry, log2 of the keys per entry, log2 of the bins
+// per code of the byte plane}
+struct CodeSpace { // how the sweep coded the elements of one (worker, layer)
+    const uint32_t* reg_index; // [L], 0xffffffff: tiny layer
+    const BandMeta* meta;      // [W][R]
+    const uint32_t* cell_tab;  // [W][R][kCellTab]
+    const int4* cell_win;      // [W][R]
+    uint32_t R;
+    // code of a key of layer l of worker w, as the sweep wrote it for every element of that layer
+    __device__ __forceinline__ uint32_t code(uint32_t w, uint32_t l, uint32_t key) const {
+        const uint32_t r = reg_index[l];
+        if (r == 0xffffffffu) return key >> 24;
+        const size_t wr = (size_t)w * R + r;
+        if (meta[wr].flagged) return key >> 24;
+        const int4 win = cell_win[wr];
+        const uint32_t e = cell_tab[wr * kCellTab + (size_t)(min(max((int)(key >> win.z), win.x), win.y) - win.x)];
+        return (uint32_t)(((int)e >> 5) + (int)(key >> (e & 31u))) >> win.w;
+    }
+};
+
+// ------------------------------------------------------------------------------------------------
 // (c) knapsack DP over the budget axis, one CTA per worker
 // ------------------------------------------------------------------------------------------------
 struct DpBudgets { uint64_t c[kDpWorkersPerLaunch]; };
@@ -379,7 +419,7 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
      const uint32_t* __restrict__ j_in, uint32_t* __restrict__ flags,
      uint8_t* __restrict__ pd_global, Sel* __restrict__ sel, uint32_t* __restrict__ out_k,
      uint32_t* __restrict__ out_j, uint64_t* __restrict__ out_offs, kimad_stats* __restrict__ out_stats,
-     uint32_t* __restrict__ out_dense /* may be null */) {
+     uint32_t* __restrict__ out_dense /* may be null */, const CodeSpace codes) {
     pdl_wait();
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const uint32_t w = w_base + blockIdx.x;
@@ -793,15 +833,15 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
             s.k = s_k[l];
             s.shift = shift ? shift[wl * K + j] : 0u;
             s.base = out_offs[(size_t)w * (L + 1) + l];
+            s.code = codes.code(w, l, s.tau); // the whole interval lies in one bin, hence has one code
             out_k[wl] = s_k[l];
             out_j[wl] = j;
         } else {
-            s.tau = 0; s.keep_eq = 0; s.k = 0; s.shift = 0; s.base = 0;
+            s.tau = 0; s.keep_eq = 0; s.k = 0; s.shift = 0; s.base = 0; s.code = 0;
             out_k[wl] = 0;
             out_j[wl] = 0;
         }
         s.tau_low = 0;
-        s._pad = 0;
         sel[wl] = s;
     }
 }

@@ -2,7 +2,7 @@
 //
 // After the DP every (worker, layer) knows a key interval [lo, lo + 2^shift) that contains its
 // threshold and the rank of the threshold inside that interval (shift = 0 when the curve stage already
-// resolved all 31 bits).  One sweep over the upper halves of the difference vector (k_sel_count) counts, per 2048-element slice,
+// resolved all 31 bits).  One sweep over the byte codes the curve stage left (k_sel_count) counts, per 2048-element slice,
 // the entries above the interval, remembers the few entries inside it and marks the 32-element groups that
 // can hold a kept entry; k_sel_resolve turns the remembered entries (or their per-layer histogram) into the
 // exact threshold; k_sel_slices and k_sel_scan derive every slice's and chunk's output offset and leave one
@@ -82,18 +82,15 @@ __device__ __forceinline__ void sel_count_chunk(const DSource& dbuf, const Chunk
     }
     const uint32_t lo = s.tau, width = 1u << s.shift;
     const uint32_t hshift = s.shift > 10 ? s.shift - 10 : 0; // the histogram has at most kLowBins bins
-    __shared__ uint32_t s_gm[kThreads / 32]; // per warp: group bits of the half slice in work (zero between uses)
     if (threadIdx.x == 0) *s_n = 0;
     uint32_t* gh = low_hist + wl * kLowBins; // the layer's in-interval histogram: few entries, counted in place
-    if (threadIdx.x < kThreads / 32) s_gm[threadIdx.x] = 0;
     __syncthreads();
     const DView dd(dbuf, w, dstride, cv.a0);
-    // Upper halves first: a key whose upper half lies above that of the interval's last key is above the interval,
-    // one below that of its first key is below; only keys sharing an upper half with the interval (a 2^16-key
-    // stretch of the axis or two) are completed from the lower plane.  The halves are 15-bit numbers after the
-    // sign is masked, so "x >= t" for both halves of a word is bit 15 / 31 of x + (0x8000 - t) * 0x10001.
-    const uint32_t hi_bot = lo >> 16, hi_top = (lo + width - 1) >> 16;
-    const uint32_t add_gt = (0x8000u - (hi_top + 1)) * 0x00010001u, add_ge = (0x8000u - hi_bot) * 0x00010001u;
+    // Codes first: an entry whose code (the byte the sweep left for it) is larger than the code of the interval's
+    // keys lies above the interval, one with a smaller code below; only entries with the interval's own code are
+    // completed from the inputs.  Codes are 7-bit numbers, so "x >= t" for the four bytes of a word is bit 7 of
+    // every byte of x + (0x80 - t) * 0x01010101.
+    const uint32_t add_gt = (0x80u - (s.code + 1u)) * 0x01010101u, add_ge = (0x80u - s.code) * 0x01010101u;
     for (uint32_t sl = wid; sl < (uint32_t)kSlices; sl += kThreads / 32) {
         uint32_t above = 0;
         uint64_t mask = 0;
@@ -108,69 +105,52 @@ __device__ __forceinline__ void sel_count_chunk(const DSource& dbuf, const Chunk
             }
             return d1 < 0x80000000u;
         };
-        constexpr int H = kSliceElems / 256; // quads per lane and half slice
-        for (uint32_t q0 = sl * (kSliceElems / 4); q0 < (sl + 1) * (kSliceElems / 4) && 4 * q0 < cv.len; q0 += H * 32) {
-            uint2 a[H];
+        // a lane takes sixteen consecutive codes (one 128-bit load) of each of the slice's four rows of 512 elements;
+        // a 32-element group is a pair of lanes
+        constexpr int ROWS = kSliceElems / 512;
+        const uint32_t u0 = sl * (kSliceElems / 16) + lane; // this lane's 16-element unit in row 0
+        uint4 a[ROWS];
 #pragma unroll
-            for (int i = 0; i < H; ++i) {
-                const uint32_t q = q0 + i * 32 + lane;
-                if (cv.quad_full(q)) a[i] = __ldcs(reinterpret_cast<const uint2*>(dd.hi) + q);
-            }
-            uint32_t fb = 0; // bit i: this lane's quad of row i may hold a key that is not below the interval
+        for (int r = 0; r < ROWS; ++r) {
+            const uint32_t e0 = 16 * (u0 + r * 32);
+            if (e0 >= cv.first && e0 + 16 <= cv.len) a[r] = __ldcs(reinterpret_cast<const uint4*>(dd.code) + u0 + r * 32);
+        }
 #pragma unroll
-            for (int i = 0; i < H; ++i) {
-                const uint32_t q = q0 + i * 32 + lane;
-                bool f = false;
-                if (cv.quad_full(q)) {
-                    const uint32_t x0_ = a[i].x & 0x7fff7fffu, x1_ = a[i].y & 0x7fff7fffu;
-                    const uint32_t ge0 = (x0_ + add_ge) & 0x80008000u, ge1 = (x1_ + add_ge) & 0x80008000u;
-                    if (ge0 | ge1) { // with a sparse budget few quads hold a key that is not below the interval's upper half
-                        const uint32_t gt0 = (x0_ + add_gt) & 0x80008000u, gt1 = (x1_ + add_gt) & 0x80008000u;
-                        above += __popc(gt0) + __popc(gt1);
-                        f = (gt0 | gt1) != 0; // keys sharing an upper half with the interval mark the group only if not below it
-                        // rare: keys that share an upper half with the interval; bit 15 -> element 0 / 2, bit 31 -> 1 / 3
-                        uint32_t border = ((ge0 ^ gt0) >> 15 & 0x00010001u) | ((ge1 ^ gt1) >> 13 & 0x00040004u);
+        for (int r = 0; r < ROWS; ++r) {
+            const uint32_t e0 = 16 * (u0 + r * 32);
+            bool f = false; // this lane holds an entry that is not below the interval
+            if (e0 >= cv.first && e0 + 16 <= cv.len) {
+                const uint32_t x[4] = {a[r].x, a[r].y, a[r].z, a[r].w};
+                uint32_t ge[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) ge[j] = (x[j] + add_ge) & 0x80808080u;
+                if (ge[0] | ge[1] | ge[2] | ge[3]) { // with a sparse budget few lanes hold a code that is not below the interval's
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const uint32_t gt = (x[j] + add_gt) & 0x80808080u;
+                        above += __popc(gt);
+                        f |= gt != 0; // entries with the interval's code mark the group only if they are not below it
+                        uint32_t border = ge[j] ^ gt; // rare: entries with the interval's code; bit 8 k + 7 -> element k
                         while (border) {
-                            const uint32_t bit = __ffs(border) - 1; // 0, 16 (first word), 2, 18 (second word)
+                            const uint32_t bit = __ffs(border) - 1;
                             border &= border - 1;
-                            const uint32_t k = (bit & 3u) + (bit >> 4);
-                            f |= visit(key_of(dd.at(4 * q + k)));
+                            f |= visit(key_of(dd.at(e0 + 4 * j + (bit >> 3))));
                         }
                     }
-                } else if (4 * q < cv.len) {
-                    for (uint32_t e = 4 * q; e < 4 * q + 4; ++e)
-                        if (e >= cv.first && e < cv.len) f |= visit(key_of(dd.at(e)));
                 }
-                fb |= (uint32_t)f << i;
+            } else if (e0 < cv.len) { // ragged first or last unit of the chunk
+                for (uint32_t e = e0; e < e0 + 16; ++e)
+                    if (e >= cv.first && e < cv.len) f |= visit(key_of(dd.at(e)));
             }
-            // a row of 128 elements = four groups of 8 lanes: a lane's 8 row flags, spread to every fourth bit and
-            // shifted by its group, are its share of this half slice's 32 group bits.  Few marked lanes (sparse
-            // budgets): they OR their shares into a word of shared memory; many: two warp OR-reductions.
-            const uint32_t g = lane >> 3;
-            const uint32_t marked = __ballot_sync(0xffffffffu, fb != 0);
-            uint32_t half = 0;
-            if (__popc(marked) <= 6) {
-                if (fb) {
-                    uint32_t r8 = fb;
-                    r8 = (r8 | (r8 << 12)) & 0x000f000fu;
-                    r8 = (r8 | (r8 << 6)) & 0x03030303u;
-                    r8 = (r8 | (r8 << 3)) & 0x11111111u;
-                    atomicOr(&s_gm[wid], r8 << g);
-                }
-                if (marked) {
-                    __syncwarp();
-                    half = s_gm[wid];
-                    __syncwarp();
-                    if (lane == 0) s_gm[wid] = 0;
-                }
-            } else {
-                uint32_t r8 = __reduce_or_sync(0xffu << (8 * g), fb);
-                r8 = (r8 | (r8 << 12)) & 0x000f000fu;
-                r8 = (r8 | (r8 << 6)) & 0x03030303u;
-                r8 = (r8 | (r8 << 3)) & 0x11111111u;
-                half = __reduce_or_sync(0xffffffffu, r8 << g);
+            uint32_t m = __ballot_sync(0xffffffffu, f);
+            if (m) { // pairs of lanes -> 16 group bits of this row
+                m = (m | (m >> 1)) & 0x55555555u;
+                m = (m | (m >> 1)) & 0x33333333u;
+                m = (m | (m >> 2)) & 0x0f0f0f0fu;
+                m = (m | (m >> 4)) & 0x00ff00ffu;
+                m = (m | (m >> 8)) & 0x0000ffffu;
+                mask |= (uint64_t)m << (16 * r);
             }
-            mask |= (uint64_t)half << (32 * ((q0 - sl * (kSliceElems / 4)) / (H * 32)));
         }
 #pragma unroll
         for (int o = 16; o; o >>= 1) above += __shfl_xor_sync(0xffffffffu, above, o);
