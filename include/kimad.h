@@ -271,7 +271,7 @@ int kimad_debug_step_with_j(kimad_ctx* ctx, const float* grads_dev, float* state
 int kimad_debug_exact_path_layers(kimad_ctx* ctx, uint64_t* host_count);
 
 /* Band tables of the last step, one record of four u32 per (worker, layer above the tiny size), in
- * worker-major order: bins used, 11-bit bins split into cells, flag (0: sampled bands in use, 1: exact
+ * worker-major order: bins used, entries of the cell table in use, flag (0: sampled bands in use, 1: exact
  * path forced, 2: bands did not fit the tables), detail of the misfit.  host_meta: host, u32 [W][R][4]. */
 int kimad_debug_get_band_meta(kimad_ctx* ctx, uint32_t* host_meta);
 
@@ -283,6 +283,15 @@ int kimad_debug_get_band_meta(kimad_ctx* ctx, uint32_t* host_meta);
 #define KIMAD_N_STAGES 8
 int kimad_debug_enable_stage_timing(kimad_ctx* ctx, int enable);
 int kimad_debug_stage_times(kimad_ctx* ctx, float* host_ms);
+
+/* How a step schedules its workers (Section 3: every worker decides on its own, so workers are independent
+ * problems).  After the sample kernel the workers are taken through the remaining stages as two groups on two
+ * internal streams, forked from and joined to the step's stream, the first group with the higher priority: while
+ * one group is in its latency-bound stages (curves, DP, offsets) the other one streams.  Results do not depend on
+ * the schedule.  mode 0 (default): two groups when W >= 2 and W * N >= 2^25 elements; 1: two groups whenever
+ * W >= 2; 2: one group (every kernel covers all workers, on the step's stream).  Steps with stage timing enabled
+ * always run as one group. */
+int kimad_debug_set_schedule(kimad_ctx* ctx, int mode);
 
 /* Checked build of the library (compiled with -DKIMAD_CHECKED; the stand-in for a memory checker): the kernels
  * test their indices into the workspace and the output buffers before use -- a failed test sets its bit in a

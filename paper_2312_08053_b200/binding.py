@@ -107,6 +107,8 @@ def load():
     L.kimad_debug_enable_stage_timing.argtypes = [vp, C.c_int]
     L.kimad_debug_stage_times.restype = C.c_int
     L.kimad_debug_stage_times.argtypes = [vp, vp]
+    L.kimad_debug_set_schedule.restype = C.c_int
+    L.kimad_debug_set_schedule.argtypes = [vp, C.c_int]
     L.kimad_debug_get_band_meta.restype = C.c_int
     L.kimad_debug_get_band_meta.argtypes = [vp, vp]
     L.kimad_debug_exact_path_layers.restype = C.c_int
@@ -315,6 +317,11 @@ STAGE_NAMES = ["sample", "sweep", "curve", "exact_fallback", "dp", "select_count
 
 def kimad_debug_enable_stage_timing(ctx: Ctx, enable: bool) -> None:
     _check(load().kimad_debug_enable_stage_timing(ctx.handle, int(bool(enable))), "kimad_debug_enable_stage_timing")
+
+
+def kimad_debug_set_schedule(ctx: Ctx, mode: int) -> None:
+    """0: two worker groups for large steps, 1: whenever W >= 2, 2: one group."""
+    _check(load().kimad_debug_set_schedule(ctx.handle, int(mode)), "kimad_debug_set_schedule")
 
 
 def kimad_debug_stage_times(ctx: Ctx) -> np.ndarray:

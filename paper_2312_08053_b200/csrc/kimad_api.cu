@@ -14,6 +14,7 @@ using namespace kimad;
 
 namespace {
 
+constexpr int kGroups = 2; // groups of workers in flight at a time (see kimad_ctx::gstream)
 constexpr size_t kAlign = 256;
 constexpr int kCanaryByte = 0xA5; // checked build: fill of the guard words between workspace regions
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
@@ -22,7 +23,7 @@ struct Layout {
     // static tables
     size_t dbuf, chunks, layers, ktab, ktab_dyn, reg_layers, tiny_layers, reg_index, runs;
     // zeroed at set_workspace and kept clean by the kernels
-    size_t zero_from, h1_cnt, h1_ss, h23_cnt, h23_ss, bh_cnt, bh_sum, low_hist, recount, fb, r2, flags;
+    size_t zero_from, h1_cnt, h1_ss, h23_cnt, h23_ss, bh_cnt, bh_sum, low_hist, recount, recount_bytes, fb, r2, flags;
     // scratch without initial-state requirements
     size_t cell_tab, cell_win, bin_lo, meta, cands, slots, err, tau, keep_eq, shift, sel, chunk_cnt, jobs, csel,
         fb_chunks, fb_layers, r2_chunks, r2_layers, pd, total;
@@ -59,6 +60,11 @@ struct kimad_ctx {
     // from and joined to the caller's stream with events
     cudaStream_t side = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    // two groups of workers are taken through the stages after the sample on streams of their own, the first with
+    // the higher priority: while one group is in its latency-bound stages (curves, DP, offsets) the other one streams
+    cudaStream_t gstream[kGroups] = {};
+    cudaEvent_t ev_go = nullptr, ev_done[kGroups] = {};
+    int pipeline_mode = 0; // 0: two groups when the step is large enough, 1: whenever W >= 2, 2: never
     bool have_ev = false;
     template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
 };
@@ -97,9 +103,11 @@ void plan_layout(kimad_ctx* c) {
     y.bh_cnt = take(WR * kMaxBins * sizeof(uint32_t));
     y.bh_sum = take(WR * kMaxBins * sizeof(uint64_t));
     y.low_hist = take(WL * kLowBins * sizeof(uint32_t));
-    y.recount = take(256 + (size_t)2 * c->W * nch * sizeof(uint2));
-    y.fb = take(sizeof(FbList));
-    y.r2 = take(sizeof(Round2));
+    // work lists, one set per group of workers
+    y.recount_bytes = align_up(256 + (size_t)2 * c->W * nch * sizeof(uint2));
+    y.recount = take(kGroups * y.recount_bytes);
+    y.fb = take(kGroups * align_up(sizeof(FbList)));
+    y.r2 = take(kGroups * align_up(sizeof(Round2)));
     y.flags = take((size_t)c->W * sizeof(uint32_t));
     y.cell_tab = take(WR * kCellTab * sizeof(uint32_t));
     y.cell_win = take(WR * sizeof(int4));
@@ -115,10 +123,10 @@ void plan_layout(kimad_ctx* c) {
     y.chunk_cnt = take((size_t)c->W * nch * sizeof(uint2));
     y.jobs = take((size_t)c->W * nch * sizeof(ChunkJob));
     y.csel = take((size_t)c->W * nch * sizeof(ChunkSel));
-    y.fb_chunks = take((size_t)c->W * nch * sizeof(uint2));
-    y.fb_layers = take(WL * sizeof(uint2));
-    y.r2_chunks = take((size_t)c->W * nch * sizeof(uint2));
-    y.r2_layers = take(WL * sizeof(uint2));
+    y.fb_chunks = take(kGroups * align_up((size_t)c->W * nch * sizeof(uint2)));
+    y.fb_layers = take(kGroups * align_up(WL * sizeof(uint2)));
+    y.r2_chunks = take(kGroups * align_up((size_t)c->W * nch * sizeof(uint2)));
+    y.r2_layers = take(kGroups * align_up(WL * sizeof(uint2)));
     y.pd = take(c->dp_plan.pd_in_smem ? 0 : (size_t)c->W * c->L * c->dp_plan.pd_row_bytes);
     y.total = o;
 }
@@ -130,6 +138,7 @@ void plan_layout(kimad_ctx* c) {
 
 constexpr size_t kDpSmemMax = 225 * 1024; // dynamic shared memory the DP kernel may ask for
 constexpr uint32_t kSweepWaves = 2;       // CTAs of the sweep per SM (148 SMs), one resident at a time
+constexpr uint64_t kPipelineMinElems = 1ull << 25; // W N from which a step is run as two groups of workers
 
 // Kernels are loaded on their first launch; loading one takes about a millisecond.  Touching every kernel a
 // step can launch (the rarely taken ones included) when the workspace is attached keeps that out of the steps.
@@ -170,6 +179,13 @@ static int ensure_side_stream(kimad_ctx* c) {
     CUDA_TRY(cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking));
     CUDA_TRY(cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming));
     CUDA_TRY(cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming));
+    int prio_least = 0, prio_greatest = 0;
+    CUDA_TRY(cudaDeviceGetStreamPriorityRange(&prio_least, &prio_greatest));
+    for (int g = 0; g < kGroups; ++g) {
+        CUDA_TRY(cudaStreamCreateWithPriority(&c->gstream[g], cudaStreamNonBlocking, g == 0 ? prio_greatest : prio_least));
+        CUDA_TRY(cudaEventCreateWithFlags(&c->ev_done[g], cudaEventDisableTiming));
+    }
+    CUDA_TRY(cudaEventCreateWithFlags(&c->ev_go, cudaEventDisableTiming));
     return KIMAD_OK;
 }
 
@@ -246,23 +262,15 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
     ChunkJob* jobs = c->at<ChunkJob>(y.jobs);
     ChunkSel* csel = c->at<ChunkSel>(y.csel);
     uint32_t* lowh = c->at<uint32_t>(y.low_hist);
-    uint32_t* recount_n = c->at<uint32_t>(y.recount);
-    uint2* recount_list = c->at<uint2>(y.recount + 256);
-    FbList* fb = c->at<FbList>(y.fb);
-    uint2* fb_chunks = c->at<uint2>(y.fb_chunks);
-    uint2* fb_layers = c->at<uint2>(y.fb_layers);
-    Round2* r2 = c->at<Round2>(y.r2);
-    uint2* r2_chunks = c->at<uint2>(y.r2_chunks);
-    uint2* r2_layers = c->at<uint2>(y.r2_layers);
     uint32_t* flags = c->at<uint32_t>(y.flags);
     uint8_t* pd = c->at<uint8_t>(y.pd);
+    const SweepRun* runs = c->at<SweepRun>(y.runs);
 
     const uint32_t R = (uint32_t)c->reg_layers.size(), T = (uint32_t)c->tiny_layers.size();
-    const dim3 gch(nch, W), glw(L, W), blk(kThreads);
-    const SweepRun* runs = c->at<SweepRun>(y.runs);
-    const uint32_t n_runs = (uint32_t)c->runs.size();
+    const dim3 blk(kThreads);
+    const uint32_t list_cap = W * nch; // entries of every chunk list (twice that for the recount list)
     int stage = 0;
-    auto mark = [&]() { if (c->timing) cudaEventRecord(c->ev[stage++], s); };
+    auto mark = [&](cudaStream_t st) { if (c->timing) cudaEventRecord(c->ev[stage++], st); };
     auto budgets_of = [&](uint32_t w0, uint32_t nw) {
         DpBudgets b{};
         for (uint32_t i = 0; i < nw; ++i) {
@@ -271,7 +279,12 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
         }
         return b;
     };
-    mark();
+    // Two groups of workers (none when the stages are being timed, or for small steps, where it gains nothing)
+    const bool two = !c->timing && W >= 2 && c->pipeline_mode != 2 &&
+                     (c->pipeline_mode == 1 || (uint64_t)W * c->N >= kPipelineMinElems);
+    const uint32_t n_groups = two ? 2u : 1u;
+
+    mark(s);
     if (c->policy == 3 && mode != kGivenJ) { // Section 3.1: the one ratio sized to each worker's budget
         for (uint32_t w0 = 0; w0 < W; w0 += kDpWorkersPerLaunch) {
             const uint32_t nw = std::min<uint32_t>(kDpWorkersPerLaunch, W - w0);
@@ -280,89 +293,116 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
             c->launches += 1;
         }
     }
-    // (a) + (b): sample -> bands -> one sweep -> curves
+    if (T) CUDA_TRY(cudaEventRecord(c->ev_fork, s)); // fork point of the tiny layers' kernel: the step's start
+    // (a) + (b): sample -> bands, all workers
     if (R) {
         CUDA_TRY(launch_pdl(k_sample, dim3(R, W), kBigThreads, c->sample_smem, s, grads, state, c->stride, layers, reg_layers, R,
                             ktab, K, c->curve_mode == 1 ? 1u : 0u, cell_tab, cell_win, binlo, meta));
         c->launches += 1;
     }
-    mark();
-    if (vec)
-        CUDA_TRY(launch_pdl(k_pass_a<true>, n_runs, kBigThreads, c->pass_a_smem, s, grads, state, dbuf.code, chunks, runs,
-                            c->stride, c->dstride, reg_index, R, cell_tab, cell_win, meta, bhc, bhs));
-    else
-        CUDA_TRY(launch_pdl(k_pass_a<false>, n_runs, kBigThreads, c->pass_a_smem, s, grads, state, dbuf.code, chunks, runs,
-                            c->stride, c->dstride, reg_index, R, cell_tab, cell_win, meta, bhc, bhs));
-    c->launches += 1;
-    mark();
-    if (T) { // tiny layers: sorted in shared memory on the side stream, beside the kernels that turn the sweep's
-             // histograms into curves (all of them latency-bound).  Not beside the sweep: CTAs of another kernel on
-             // an SM keep the sweep's CTA, which takes most of the SM's shared memory, from starting there.
-        CUDA_TRY(cudaEventRecord(c->ev_fork, s));
+    if (T) { // tiny layers: sorted in shared memory on the side stream, beside the sample kernel (its CTAs fill what
+             // that kernel leaves idle); joined before the sweep, whose CTAs take most of an SM's shared memory and
+             // could not start on an SM that still holds CTAs of another kernel
         CUDA_TRY(cudaStreamWaitEvent(c->side, c->ev_fork, 0));
         CUDA_TRY(launch_pdl(k_tiny_exact, dim3(T, W), blk, c->tiny_smem, c->side, grads, state, c->stride, layers, tiny_layers, L,
                             ktab, K, err, tau, keq, shf, flags));
         CUDA_TRY(cudaEventRecord(c->ev_join, c->side));
+        CUDA_TRY(cudaStreamWaitEvent(s, c->ev_join, 0));
         c->launches += 1;
     }
-    if (R) {
-        CUDA_TRY(launch_pdl(k_resolve_a, dim3(R, W), kBigThreads, 0, s, layers, reg_layers, R, L, ktab, K, meta, binlo, bhc, bhs, err, tau,
-                                                       keq, shf, flags, fb, fb_chunks, fb_layers, nch));
+    mark(s);
+    if (two) CUDA_TRY(cudaEventRecord(c->ev_go, s));
+    // budget share kept, from the host's view of the budgets: picks the tuning of the write sweep
+    double kept = 0.0;
+    for (uint32_t i = 0; i < W; ++i) kept = std::max(kept, std::floor(bw[i] * t) / ((double)c->bpe * (double)c->N));
+    const bool dense_write = kept >= 0.04;
+
+    for (uint32_t g = 0; g < n_groups; ++g) {
+        // workers [w0, w0 + nw) on stream gs; every group has work lists of its own
+        const uint32_t w0 = two ? (g == 0 ? 0u : W / 2) : 0u, nw = two ? (g == 0 ? W / 2 : W - W / 2) : W;
+        cudaStream_t gs = two ? c->gstream[g] : s;
+        if (two) CUDA_TRY(cudaStreamWaitEvent(gs, c->ev_go, 0));
+        uint32_t* recount_n = c->at<uint32_t>(y.recount + g * y.recount_bytes);
+        uint2* recount_list = c->at<uint2>(y.recount + g * y.recount_bytes + 256);
+        FbList* fb = c->at<FbList>(y.fb + g * align_up(sizeof(FbList)));
+        Round2* r2 = c->at<Round2>(y.r2 + g * align_up(sizeof(Round2)));
+        uint2* fb_chunks = c->at<uint2>(y.fb_chunks + g * align_up((size_t)W * nch * sizeof(uint2)));
+        uint2* r2_chunks = c->at<uint2>(y.r2_chunks + g * align_up((size_t)W * nch * sizeof(uint2)));
+        uint2* fb_layers = c->at<uint2>(y.fb_layers + g * align_up((size_t)W * L * sizeof(uint2)));
+        uint2* r2_layers = c->at<uint2>(y.r2_layers + g * align_up((size_t)W * L * sizeof(uint2)));
+        const dim3 gch(nch, nw), glw(L, nw);
+        // the group's runs of the sweep: the run table is sorted by worker
+        uint32_t run0 = 0, run1 = 0;
+        for (uint32_t i = 0; i < (uint32_t)c->runs.size(); ++i) {
+            if (c->runs[i].w < w0) run0 = i + 1;
+            if (c->runs[i].w < w0 + nw) run1 = i + 1;
+        }
+        if (vec)
+            CUDA_TRY(launch_pdl(k_pass_a<true>, run1 - run0, kBigThreads, c->pass_a_smem, gs, grads, state, dbuf.code, chunks, runs + run0,
+                                c->stride, c->dstride, reg_index, R, cell_tab, cell_win, meta, bhc, bhs));
+        else
+            CUDA_TRY(launch_pdl(k_pass_a<false>, run1 - run0, kBigThreads, c->pass_a_smem, gs, grads, state, dbuf.code, chunks, runs + run0,
+                                c->stride, c->dstride, reg_index, R, cell_tab, cell_win, meta, bhc, bhs));
         c->launches += 1;
+        mark(gs);
+        if (R) {
+            CUDA_TRY(launch_pdl(k_resolve_a, dim3(R, nw), kBigThreads, 0, gs, layers, reg_layers, R, L, ktab, K, meta, binlo, bhc, bhs,
+                                err, tau, keq, shf, flags, fb, fb_chunks, fb_layers, list_cap, w0));
+            c->launches += 1;
+        }
+        mark(gs);
+        // exact radix select for the layers handed over by k_resolve_a (the lists are usually empty)
+        if (R) {
+            const uint32_t gfb = 2 * 148, glay = std::min<uint32_t>(nw * R, 128u);
+            const dim3 gslot(glay, 1, K);
+            CUDA_TRY(launch_pdl(k_fb_hist1, gfb, blk, 0, gs, dbuf, chunks, c->dstride, L, fb, fb_chunks, h1c, h1s, flags));
+            CUDA_TRY(launch_pdl(k_resolve1, glay, blk, 0, gs, fb, fb_layers, h1c, h1s, ktab, L, K, cands, slots));
+            CUDA_TRY(launch_pdl(k_fb_hist23<2>, gfb, blk, 0, gs, dbuf, chunks, c->dstride, L, K, fb, fb_chunks, slots, h23c, h23s));
+            CUDA_TRY(launch_pdl(k_resolve23<2>, gslot, blk, 0, gs, fb, fb_layers, h23c, h23s, L, K, cands, slots, err, tau, keq, shf));
+            CUDA_TRY(launch_pdl(k_rebuild_slots, (nw * R + kThreads - 1) / kThreads, blk, 0, gs, fb, fb_layers, L, K, cands, slots));
+            CUDA_TRY(launch_pdl(k_fb_hist23<3>, gfb, blk, 0, gs, dbuf, chunks, c->dstride, L, K, fb, fb_chunks, slots, h23c, h23s));
+            CUDA_TRY(launch_pdl(k_resolve23<3>, gslot, blk, 0, gs, fb, fb_layers, h23c, h23s, L, K, cands, slots, err, tau, keq, shf));
+            c->launches += 7;
+        }
+        mark(gs);
+        // (c)
+        for (uint32_t wa = w0; wa < w0 + nw; wa += kDpWorkersPerLaunch) {
+            const uint32_t nwa = std::min<uint32_t>(kDpWorkersPerLaunch, w0 + nw - wa);
+            const int dp_mode = mode == kGivenJ ? 1 : (c->policy == 1 ? 2 : (c->policy == 2 ? 3 : (c->policy == 3 ? 4 : 0)));
+            CUDA_TRY(launch_pdl(k_dp, nwa, kDpThreads, c->dp_smem, gs, budgets_of(wa, nwa), wa, W, L, K, c->D, c->bpe, c->full_bytes, c->cap,
+                                c->check_finite, dp_mode, c->cost_model, c->dp_plan, layers,
+                                ktab, mode == kInjectErr ? err_dev : err, tau, keq, shf, j_dev, flags, pd, sel, out->k, out->j,
+                                out->offs, out->stats, out->dense, CodeSpace{reg_index, meta, cell_tab, cell_win, R}));
+            c->launches += 1;
+        }
+        mark(gs);
+        // (d), (e), (f)
+        CUDA_TRY(launch_pdl(k_sel_count, gch, blk, 0, gs, dbuf, chunks, nch, c->dstride, L, sel, layers, csel, lowh, recount_n,
+                            recount_list, 2 * list_cap, w0));
+        mark(gs);
+        CUDA_TRY(launch_pdl(k_sel_resolve, glw, blk, 0, gs, L, layers, nch, csel, lowh, sel, r2, r2_layers, r2_chunks, w0));
+        CUDA_TRY(launch_pdl(k_sel_count_r2, 2 * 148, blk, 0, gs, dbuf, chunks, nch, c->dstride, L, sel, layers, csel, lowh, recount_n,
+                            recount_list, 2 * list_cap, r2, r2_chunks));
+        CUDA_TRY(launch_pdl(k_sel_resolve_r2, std::min<uint32_t>(nw * L, 128u), blk, 0, gs, L, layers, nch, csel, lowh, sel, r2,
+                            r2_layers, r2_chunks));
+        CUDA_TRY(launch_pdl(k_sel_recount, 2 * 148, blk, 0, gs, dbuf, chunks, nch, c->dstride, L, sel, recount_n, recount_list, csel));
+        CUDA_TRY(launch_pdl(k_sel_slices, (uint32_t)(((uint64_t)nw * nch + 7) / 8), blk, 0, gs, chunks, nch, w0, nw, L, sel, csel, ccnt));
+        CUDA_TRY(launch_pdl(k_sel_scan, glw, blk, 0, gs, layers, chunks, nch, L, sel, ccnt, jobs, recount_n, fb, r2, w0));
+        mark(gs);
+        {
+            auto launch = [&](auto kern) {
+                return launch_pdl(kern, gch, blk, 0, gs, grads, state, chunks, nch, c->dstride, c->stride, csel, jobs, c->cap,
+                                  out->idx, out->val, w0);
+            };
+            if (c->value_dtype == 1) CUDA_TRY(dense_write ? launch(k_sel_write<true, true>) : launch(k_sel_write<true, false>));
+            else CUDA_TRY(dense_write ? launch(k_sel_write<false, true>) : launch(k_sel_write<false, false>));
+        }
+        mark(gs);
+        c->launches += 8;
+        if (two) CUDA_TRY(cudaEventRecord(c->ev_done[g], gs));
     }
-    if (T) CUDA_TRY(cudaStreamWaitEvent(s, c->ev_join, 0));
-    mark();
-    // exact radix select for the layers handed over by k_resolve_a (the lists are usually empty)
-    if (R) {
-        const uint32_t gfb = 2 * 148, glay = std::min<uint32_t>(W * R, 128u);
-        const dim3 gslot(glay, 1, K);
-        CUDA_TRY(launch_pdl(k_fb_hist1, gfb, blk, 0, s, dbuf, chunks, c->dstride, L, fb, fb_chunks, h1c, h1s, flags));
-        CUDA_TRY(launch_pdl(k_resolve1, glay, blk, 0, s, fb, fb_layers, h1c, h1s, ktab, L, K, cands, slots));
-        CUDA_TRY(launch_pdl(k_fb_hist23<2>, gfb, blk, 0, s, dbuf, chunks, c->dstride, L, K, fb, fb_chunks, slots, h23c, h23s));
-        CUDA_TRY(launch_pdl(k_resolve23<2>, gslot, blk, 0, s, fb, fb_layers, h23c, h23s, L, K, cands, slots, err, tau, keq, shf));
-        CUDA_TRY(launch_pdl(k_rebuild_slots, (W * R + kThreads - 1) / kThreads, blk, 0, s, fb, fb_layers, L, K, cands, slots));
-        CUDA_TRY(launch_pdl(k_fb_hist23<3>, gfb, blk, 0, s, dbuf, chunks, c->dstride, L, K, fb, fb_chunks, slots, h23c, h23s));
-        CUDA_TRY(launch_pdl(k_resolve23<3>, gslot, blk, 0, s, fb, fb_layers, h23c, h23s, L, K, cands, slots, err, tau, keq, shf));
-        c->launches += 7;
-    }
-    mark();
-    // (c)
-    for (uint32_t w0 = 0; w0 < W; w0 += kDpWorkersPerLaunch) {
-        const uint32_t nw = std::min<uint32_t>(kDpWorkersPerLaunch, W - w0);
-        const int dp_mode = mode == kGivenJ ? 1 : (c->policy == 1 ? 2 : (c->policy == 2 ? 3 : (c->policy == 3 ? 4 : 0)));
-        CUDA_TRY(launch_pdl(k_dp, nw, kDpThreads, c->dp_smem, s, budgets_of(w0, nw), w0, W, L, K, c->D, c->bpe, c->full_bytes, c->cap,
-                            c->check_finite, dp_mode, c->cost_model, c->dp_plan, layers,
-                            ktab, mode == kInjectErr ? err_dev : err, tau, keq, shf, j_dev, flags, pd, sel, out->k, out->j,
-                            out->offs, out->stats, out->dense, CodeSpace{reg_index, meta, cell_tab, cell_win, R}));
-        c->launches += 1;
-    }
-    mark();
-    // (d), (e), (f)
-    CUDA_TRY(launch_pdl(k_sel_count, gch, blk, 0, s, dbuf, chunks, nch, c->dstride, L, sel, layers, csel, lowh, recount_n, recount_list));
-    mark();
-    CUDA_TRY(launch_pdl(k_sel_resolve, glw, blk, 0, s, L, layers, nch, csel, lowh, sel, r2, r2_layers, r2_chunks));
-    CUDA_TRY(launch_pdl(k_sel_count_r2, 2 * 148, blk, 0, s, dbuf, chunks, nch, c->dstride, L, sel, layers, csel, lowh, recount_n,
-                                          recount_list, r2, r2_chunks));
-    CUDA_TRY(launch_pdl(k_sel_resolve_r2, std::min<uint32_t>(W * L, 128u), blk, 0, s, L, layers, nch, csel, lowh, sel, r2,
-                        r2_layers, r2_chunks));
-    CUDA_TRY(launch_pdl(k_sel_recount, 2 * 148, blk, 0, s, dbuf, chunks, nch, c->dstride, L, sel, recount_n, recount_list, csel));
-    CUDA_TRY(launch_pdl(k_sel_slices, (uint32_t)(((uint64_t)W * nch + 7) / 8), blk, 0, s, chunks, nch, W, L, sel, csel, ccnt));
-    CUDA_TRY(launch_pdl(k_sel_scan, glw, blk, 0, s, layers, chunks, nch, L, sel, ccnt, jobs, recount_n, fb, r2));
-    mark();
-    {
-        // budget share kept, from the host's view of the budgets: picks the tuning of the write sweep
-        double kept = 0.0;
-        for (uint32_t i = 0; i < W; ++i) kept = std::max(kept, std::floor(bw[i] * t) / ((double)c->bpe * (double)c->N));
-        const bool dense = kept >= 0.04;
-        auto launch = [&](auto kern) {
-            return launch_pdl(kern, gch, blk, 0, s, grads, state, chunks, nch, c->dstride, c->stride, csel, jobs, c->cap,
-                              out->idx, out->val);
-        };
-        if (c->value_dtype == 1) CUDA_TRY(dense ? launch(k_sel_write<true, true>) : launch(k_sel_write<true, false>));
-        else CUDA_TRY(dense ? launch(k_sel_write<false, true>) : launch(k_sel_write<false, false>));
-    }
-    mark();
-    c->launches += 8;
+    if (two)
+        for (uint32_t g = 0; g < n_groups; ++g) CUDA_TRY(cudaStreamWaitEvent(s, c->ev_done[g], 0));
     CUDA_TRY(cudaGetLastError());
     c->last_out = *out;
     c->have_last = true;
@@ -500,6 +540,11 @@ void kimad_destroy(kimad_ctx* ctx) {
         cudaEventDestroy(ctx->ev_fork);
         cudaEventDestroy(ctx->ev_join);
         cudaStreamDestroy(ctx->side);
+        for (int g = 0; g < kGroups; ++g) {
+            if (ctx->gstream[g]) { cudaStreamSynchronize(ctx->gstream[g]); cudaStreamDestroy(ctx->gstream[g]); }
+            if (ctx->ev_done[g]) cudaEventDestroy(ctx->ev_done[g]);
+        }
+        if (ctx->ev_go) cudaEventDestroy(ctx->ev_go);
     }
     delete ctx;
 }
@@ -511,6 +556,12 @@ int kimad_debug_enable_stage_timing(kimad_ctx* c, int enable) {
         c->have_ev = true;
     }
     c->timing = enable != 0;
+    return KIMAD_OK;
+}
+
+int kimad_debug_set_schedule(kimad_ctx* c, int mode) {
+    if (!c || mode < 0 || mode > 2) return KIMAD_ERR_INVALID_ARG;
+    c->pipeline_mode = mode;
     return KIMAD_OK;
 }
 
@@ -666,12 +717,15 @@ int kimad_debug_get_band_meta(kimad_ctx* c, uint32_t* host_meta) {
 int kimad_debug_exact_path_layers(kimad_ctx* c, uint64_t* host_count) {
     if (!c || !host_count) return KIMAD_ERR_INVALID_ARG;
     if (!c->ws) return KIMAD_ERR_WORKSPACE;
-    FbList f{};
     CUDA_TRY(cudaDeviceSynchronize());
-    CUDA_TRY(cudaMemcpy(&f, c->ws + c->lay.fb, sizeof(FbList), cudaMemcpyDeviceToHost));
-    host_count[0] = f.total_layers;
-    for (int i = 0; i < 4; ++i) host_count[1 + i] = f.why[i];
-    for (uint32_t j = 0; j < c->K; ++j) host_count[5 + j] = f.loose_j[j];
+    for (uint32_t i = 0; i < 5 + c->K; ++i) host_count[i] = 0;
+    for (int g = 0; g < kGroups; ++g) { // every group of workers keeps counters of its own
+        FbList f{};
+        CUDA_TRY(cudaMemcpy(&f, c->ws + c->lay.fb + g * align_up(sizeof(FbList)), sizeof(FbList), cudaMemcpyDeviceToHost));
+        host_count[0] += f.total_layers;
+        for (int i = 0; i < 4; ++i) host_count[1 + i] += f.why[i];
+        for (uint32_t j = 0; j < c->K; ++j) host_count[5 + j] += f.loose_j[j];
+    }
     return KIMAD_OK;
 }
 

@@ -526,7 +526,7 @@ k_resolve_a(const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ r
             const uint32_t* __restrict__ bin_lo, uint32_t* __restrict__ bh_cnt, unsigned long long* __restrict__ bh_sum,
             float* __restrict__ err_out, uint32_t* __restrict__ tau_out, uint32_t* __restrict__ rank_out,
             uint32_t* __restrict__ shift_out, uint32_t* __restrict__ flags, FbList* __restrict__ fb,
-            uint2* __restrict__ fb_chunks, uint2* __restrict__ fb_layers, uint32_t n_chunks_all) {
+            uint2* __restrict__ fb_chunks, uint2* __restrict__ fb_layers, uint32_t list_cap, uint32_t w_base) {
     pdl_wait();
     __shared__ uint32_t s_drop[KIMAD_MAX_RATIOS]; // entries not kept by candidate j: n - k_j
     __shared__ uint32_t s_bin[KIMAD_MAX_RATIOS], s_before[KIMAD_MAX_RATIOS], s_cb[KIMAD_MAX_RATIOS];
@@ -534,7 +534,7 @@ k_resolve_a(const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ r
     __shared__ uint32_t s_w32[32];
     __shared__ double s_w64[32];
     __shared__ int s_bad;
-    const uint32_t r = blockIdx.x, w = blockIdx.y;
+    const uint32_t r = blockIdx.x, w = w_base + blockIdx.y;
     const uint32_t l = reg_layers[r];
     const size_t wr = (size_t)w * R + r, wl = (size_t)w * L + l;
     const BandMeta mt = meta[wr];
@@ -646,7 +646,7 @@ k_resolve_a(const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ r
         }
         __syncthreads();
         for (uint32_t i = threadIdx.x; i < ld.n_chunks; i += kBigThreads)
-            if (KIMAD_CHECK(s_at + i < gridDim.y * n_chunks_all, 2)) fb_chunks[s_at + i] = make_uint2(w, ld.first_chunk + i);
+            if (KIMAD_CHECK(s_at + i < list_cap, 2)) fb_chunks[s_at + i] = make_uint2(w, ld.first_chunk + i);
     }
 }
 

@@ -65,7 +65,7 @@ __device__ __forceinline__ void sel_count_chunk(const DSource& dbuf, const Chunk
                                                 const Sel* __restrict__ sel, const LayerDesc* __restrict__ layers,
                                                 ChunkSel* __restrict__ csel, uint32_t* __restrict__ low_hist,
                                                 uint32_t* __restrict__ recount_n, uint2* __restrict__ recount_list,
-                                                uint32_t* s_n, uint32_t* s_low) {
+                                                uint32_t list_cap, uint32_t* s_n, uint32_t* s_low) {
     const size_t wl = (size_t)w * L + ch.layer;
     const Sel s = sel[wl];
     ChunkSel* out = csel + (size_t)w * n_chunks + chunk_id;
@@ -165,9 +165,8 @@ __device__ __forceinline__ void sel_count_chunk(const DSource& dbuf, const Chunk
         } else {
             out->n_in = kListOverflow;
             const uint32_t at = atomicAdd(recount_n, 1u);
-            // capacity 2 W n_chunks (a chunk can be listed once per select round); the second round's launch has a flat
-            // grid and does not carry W: its appends stay below the bound the first round's were tested against
-            if (KIMAD_CHECK(gridDim.y == 1 || at < 2u * gridDim.y * n_chunks, 2)) recount_list[at] = make_uint2(w, chunk_id);
+            // capacity: a chunk can be listed once per select round
+            if (KIMAD_CHECK(at < list_cap, 2)) recount_list[at] = make_uint2(w, chunk_id);
         }
     }
     __syncthreads();
@@ -176,12 +175,13 @@ __device__ __forceinline__ void sel_count_chunk(const DSource& dbuf, const Chunk
 __global__ void __launch_bounds__(kThreads)
 k_sel_count(DSource dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks, uint64_t dstride,
             uint32_t L, const Sel* __restrict__ sel, const LayerDesc* __restrict__ layers, ChunkSel* __restrict__ csel,
-            uint32_t* __restrict__ low_hist, uint32_t* __restrict__ recount_n, uint2* __restrict__ recount_list) {
+            uint32_t* __restrict__ low_hist, uint32_t* __restrict__ recount_n, uint2* __restrict__ recount_list,
+            uint32_t list_cap, uint32_t w_base) {
     pdl_wait();
     __shared__ uint32_t s_n;
     __shared__ uint32_t s_low[kListCap];
-    sel_count_chunk(dbuf, chunks[blockIdx.x], blockIdx.y, blockIdx.x, n_chunks, dstride, L, sel, layers, csel, low_hist,
-                    recount_n, recount_list, &s_n, s_low);
+    sel_count_chunk(dbuf, chunks[blockIdx.x], w_base + blockIdx.y, blockIdx.x, n_chunks, dstride, L, sel, layers, csel, low_hist,
+                    recount_n, recount_list, list_cap, &s_n, s_low);
 }
 
 // second round: only the chunks of the layers listed in r2
@@ -189,7 +189,8 @@ __global__ void __launch_bounds__(kThreads)
 k_sel_count_r2(DSource dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks, uint64_t dstride,
                uint32_t L, const Sel* __restrict__ sel, const LayerDesc* __restrict__ layers,
                ChunkSel* __restrict__ csel, uint32_t* __restrict__ low_hist, uint32_t* __restrict__ recount_n,
-               uint2* __restrict__ recount_list, const Round2* __restrict__ r2, const uint2* __restrict__ r2_chunks) {
+               uint2* __restrict__ recount_list, uint32_t list_cap, const Round2* __restrict__ r2,
+               const uint2* __restrict__ r2_chunks) {
     pdl_wait();
     __shared__ uint32_t s_n;
     __shared__ uint32_t s_low[kListCap];
@@ -197,7 +198,7 @@ k_sel_count_r2(DSource dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks
     for (uint32_t it = blockIdx.x; it < n; it += gridDim.x) {
         const uint2 e = r2_chunks[it];
         sel_count_chunk(dbuf, chunks[e.y], e.x, e.y, n_chunks, dstride, L, sel, layers, csel, low_hist, recount_n,
-                        recount_list, &s_n, s_low);
+                        recount_list, list_cap, &s_n, s_low);
     }
 }
 
@@ -297,12 +298,12 @@ __device__ __forceinline__ void sel_resolve_layer(uint32_t l, uint32_t w, uint32
 __global__ void __launch_bounds__(kThreads)
 k_sel_resolve(uint32_t L, const LayerDesc* __restrict__ layers, uint32_t n_chunks, const ChunkSel* __restrict__ csel,
               uint32_t* __restrict__ low_hist, Sel* __restrict__ sel, Round2* __restrict__ r2,
-              uint2* __restrict__ r2_layers, uint2* __restrict__ r2_chunks) {
+              uint2* __restrict__ r2_layers, uint2* __restrict__ r2_chunks, uint32_t w_base) {
     pdl_wait();
     __shared__ __align__(16) uint32_t s_key[kSortCap];
     __shared__ uint32_t s_w32[8];
     __shared__ uint32_t s_n, s_over;
-    sel_resolve_layer(blockIdx.x, blockIdx.y, L, layers, n_chunks, csel, low_hist, sel, true, r2, r2_layers, r2_chunks, s_key,
+    sel_resolve_layer(blockIdx.x, w_base + blockIdx.y, L, layers, n_chunks, csel, low_hist, sel, true, r2, r2_layers, r2_chunks, s_key,
                       s_w32, &s_n, &s_over);
 }
 
@@ -360,12 +361,13 @@ k_sel_recount(DSource dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks,
 // Per chunk (one warp each, lane = slice): entries above tau and equal to tau in every slice (from the lists, or
 // already recounted), turned into prefixes inside the chunk; chunk_cnt = the chunk's totals.
 __global__ void __launch_bounds__(kThreads)
-k_sel_slices(const Chunk* __restrict__ chunks, uint32_t n_chunks, uint32_t W, uint32_t L, const Sel* __restrict__ sel,
-             ChunkSel* __restrict__ csel, uint2* __restrict__ chunk_cnt) {
+k_sel_slices(const Chunk* __restrict__ chunks, uint32_t n_chunks, uint32_t w_base, uint32_t n_workers, uint32_t L,
+             const Sel* __restrict__ sel, ChunkSel* __restrict__ csel, uint2* __restrict__ chunk_cnt) {
     pdl_wait();
     const uint32_t lane = threadIdx.x & 31;
-    const uint64_t it = (uint64_t)blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
-    if (it >= (uint64_t)W * n_chunks) return;
+    uint64_t it = (uint64_t)blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
+    if (it >= (uint64_t)n_workers * n_chunks) return;
+    it += (uint64_t)w_base * n_chunks; // workers w_base .. w_base + n_workers - 1
     const uint32_t w = (uint32_t)(it / n_chunks), ci = (uint32_t)(it % n_chunks);
     const Sel s = sel[(size_t)w * L + chunks[ci].layer];
     ChunkSel& c = csel[it];
@@ -395,15 +397,15 @@ k_sel_slices(const Chunk* __restrict__ chunks, uint32_t n_chunks, uint32_t W, ui
 __global__ void __launch_bounds__(kThreads)
 k_sel_scan(const LayerDesc* __restrict__ layers, const Chunk* __restrict__ chunks, uint32_t n_chunks, uint32_t L,
            const Sel* __restrict__ sel, const uint2* __restrict__ chunk_cnt, ChunkJob* __restrict__ jobs,
-           uint32_t* __restrict__ recount_n, FbList* __restrict__ fb, Round2* __restrict__ r2) {
+           uint32_t* __restrict__ recount_n, FbList* __restrict__ fb, Round2* __restrict__ r2, uint32_t w_base) {
     pdl_wait();
     __shared__ uint32_t s_w[8];
     const LayerDesc ld = layers[blockIdx.x];
-    const uint32_t w = blockIdx.y;
+    const uint32_t w = w_base + blockIdx.y;
     const Sel s = sel[(size_t)w * L + blockIdx.x];
     const uint2* cc = chunk_cnt + (size_t)w * n_chunks + ld.first_chunk;
     ChunkJob* jb = jobs + (size_t)w * n_chunks + ld.first_chunk;
-    if (blockIdx.x == 0 && w == 0 && threadIdx.x == 0) { // all work lists have been consumed by now
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) { // all work lists (of these workers) have been consumed by now
         *recount_n = 0;
         fb->n_chunks = 0;
         fb->n_layers = 0;
@@ -448,9 +450,10 @@ template <bool BF16, bool DENSE>
 __global__ void __launch_bounds__(kThreads, DENSE ? 3 : 8)
 k_sel_write(const float* __restrict__ grads, float* __restrict__ state, const Chunk* __restrict__ chunks,
             uint32_t n_chunks, uint64_t dstride, uint64_t stride, const ChunkSel* __restrict__ csel,
-            const ChunkJob* __restrict__ jobs, uint64_t cap, uint32_t* __restrict__ out_idx, void* __restrict__ out_val) {
+            const ChunkJob* __restrict__ jobs, uint64_t cap, uint32_t* __restrict__ out_idx, void* __restrict__ out_val,
+            uint32_t w_base) {
     pdl_wait();
-    const uint32_t w = blockIdx.y;
+    const uint32_t w = w_base + blockIdx.y;
     const ChunkJob jb = jobs[(size_t)w * n_chunks + blockIdx.x];
     if (jb.mode == 0) return; // nothing kept in this chunk
     const Chunk ch = chunks[blockIdx.x];

@@ -19,7 +19,7 @@ def u32(t):
 
 class Runner:
     def __init__(self, layer_sizes, W, grid, D=1000, value_dtype=0, stride=None, cap=None, check_finite=0,
-                 curve_mode=0, policy=0, cost_model=0):
+                 curve_mode=0, policy=0, cost_model=0, schedule=0):
         self.ls, self.W, self.grid, self.D, self.vd = list(layer_sizes), W, list(grid), D, value_dtype
         self.policy, self.cost_model = policy, cost_model
         self.N = int(sum(self.ls))
@@ -28,6 +28,7 @@ class Runner:
         self.ctx = kb.new_context(self.ls, W, self.grid, D=D, value_dtype=value_dtype, worker_stride=self.stride,
                                   max_packed_elems=self.cap, check_finite=check_finite, curve_mode=curve_mode,
                                   policy=policy, cost_model=cost_model)
+        kb.kimad_debug_set_schedule(self.ctx, schedule)  # 1: two groups of workers on two streams whenever W >= 2
         self.out = kb.Packed(self.ctx)
         self.kt = ko.k_table(self.ls, self.grid)
 

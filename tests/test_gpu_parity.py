@@ -11,10 +11,10 @@ from tests._harness import Runner, u32
 pytestmark = pytest.mark.gpu
 
 
-def _run_workload(cfg, divisor, steps, grid=None, D=None, curve_mode=0):
+def _run_workload(cfg, divisor, steps, grid=None, D=None, curve_mode=0, schedule=0):
     wl = workloads.workload(cfg, divisor)
     grid = grid or wl.ratio_grid
-    r = Runner(wl.layer_sizes, wl.n_workers, grid, D or wl.D, wl.value_dtype, curve_mode=curve_mode)
+    r = Runner(wl.layer_sizes, wl.n_workers, grid, D or wl.D, wl.value_dtype, curve_mode=curve_mode, schedule=schedule)
     bw = workloads.bandwidth_trace(wl, max(steps, 60))
     pick = np.linspace(0, len(bw) - 1, steps).astype(int)  # spread over the trace: low and high budgets
     state = torch.zeros((wl.n_workers, wl.N), dtype=torch.float32, device="cuda")
@@ -55,6 +55,13 @@ def test_cfg4_gpt2_shape_scaled():
 
 def test_cfg5_llama_shape_scaled_bf16():
     _run_workload(5, 512, 4)
+
+
+@pytest.mark.parametrize("cfg,divisor,curve_mode", [(2, 8, 0), (3, 16, 0), (4, 64, 0), (5, 512, 0), (3, 32, 1)])
+def test_two_worker_groups(cfg, divisor, curve_mode):
+    """The schedule large steps use (two groups of workers on two streams, each with work lists of its own),
+    forced on the scaled workloads: every result as with one group."""
+    _run_workload(cfg, divisor, 3, curve_mode=curve_mode, schedule=1)
 
 
 def test_paper_grid_50_candidates():
