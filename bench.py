@@ -171,6 +171,9 @@ def _dtype_label(wl):
     return "f32" if wl.value_dtype == 0 else "f32 (bf16 packed values)"
 
 
+SCHEDULE = 0  # kimad_debug_set_schedule of every context the bench creates (--schedule)
+
+
 def _time_steps(kb, torch, wl, dev, rank, steps, warmup, max_buf_bytes=70e9):
     """Device-timed steps of one workload: returns (ctx, out, grads, state, bw, cap, per-step ms list, launches)."""
     W, N, L = wl.n_workers, wl.N, wl.L
@@ -179,6 +182,7 @@ def _time_steps(kb, torch, wl, dev, rank, steps, warmup, max_buf_bytes=70e9):
     cap = int(min(N, np.max(bw) * wl.t_target / bpe + L + 1))
     ctx = kb.new_context(wl.layer_sizes, W, wl.ratio_grid, device=dev, D=wl.D, value_dtype=wl.value_dtype,
                          max_packed_elems=cap)
+    kb.kimad_debug_set_schedule(ctx, SCHEDULE)
     out = kb.Packed(ctx, device=dev)
     # fresh gradients for every step (as in training), as far as the device memory allowed for them goes; beyond
     # that the buffers are cycled.  Every rank draws its own streams (seed offset by rank).
@@ -457,10 +461,14 @@ def main():
     ap.add_argument("--config", type=int, default=4, help="workload 1..5 (default 4: GPT-2-small shape, 4 workers)")
     ap.add_argument("--impl", default="kimad", choices=["kimad", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--schedule", type=int, default=0, choices=[0, 1, 2],
+                    help="0: the library's choice (two worker groups for large steps), 1: always two groups, 2: one group")
     ap.add_argument("--no-also", action="store_true", help="skip the second large workload's device-timed block")
     ap.add_argument("--path", default="compress", choices=["compress", "receive"],
                     help="compress: the worker-side pass (the headline); receive: apply + aggregate on the server")
     args = ap.parse_args()
+    global SCHEDULE
+    SCHEDULE = args.schedule
     args.warmup = max(args.warmup, 3) if args.impl == "kimad" else args.warmup
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))

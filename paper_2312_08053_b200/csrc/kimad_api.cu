@@ -62,8 +62,11 @@ struct kimad_ctx {
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     // two groups of workers are taken through the stages after the sample on streams of their own, the first with
     // the higher priority: while one group is in its latency-bound stages (curves, DP, offsets) the other one streams
-    cudaStream_t gstream[kGroups] = {};
-    cudaEvent_t ev_go = nullptr, ev_done[kGroups] = {};
+    // (every group has a stream for its sweeps, of low priority, and one for its short kernels, of high priority, so
+    // that a DP or an offset scan is not queued behind another group's sweep; events hand the group over between
+    // the two)
+    cudaStream_t gstream[kGroups] = {}, gshort[kGroups] = {};
+    cudaEvent_t ev_go = nullptr, ev_done[kGroups] = {}, ev_hand[kGroups][4] = {};
     int pipeline_mode = 0; // 0: two groups when the step is large enough, 1: whenever W >= 2, 2: never
     bool have_ev = false;
     template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
@@ -182,8 +185,10 @@ static int ensure_side_stream(kimad_ctx* c) {
     int prio_least = 0, prio_greatest = 0;
     CUDA_TRY(cudaDeviceGetStreamPriorityRange(&prio_least, &prio_greatest));
     for (int g = 0; g < kGroups; ++g) {
-        CUDA_TRY(cudaStreamCreateWithPriority(&c->gstream[g], cudaStreamNonBlocking, g == 0 ? prio_greatest : prio_least));
+        CUDA_TRY(cudaStreamCreateWithPriority(&c->gstream[g], cudaStreamNonBlocking, prio_least));
+        CUDA_TRY(cudaStreamCreateWithPriority(&c->gshort[g], cudaStreamNonBlocking, prio_greatest));
         CUDA_TRY(cudaEventCreateWithFlags(&c->ev_done[g], cudaEventDisableTiming));
+        for (cudaEvent_t& e : c->ev_hand[g]) CUDA_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
     }
     CUDA_TRY(cudaEventCreateWithFlags(&c->ev_go, cudaEventDisableTiming));
     return KIMAD_OK;
@@ -320,8 +325,16 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
     for (uint32_t g = 0; g < n_groups; ++g) {
         // workers [w0, w0 + nw) on stream gs; every group has work lists of its own
         const uint32_t w0 = two ? (g == 0 ? 0u : W / 2) : 0u, nw = two ? (g == 0 ? W / 2 : W - W / 2) : W;
-        cudaStream_t gs = two ? c->gstream[g] : s;
-        if (two) CUDA_TRY(cudaStreamWaitEvent(gs, c->ev_go, 0));
+        cudaStream_t big = two ? c->gstream[g] : s, small = two ? c->gshort[g] : s; // sweeps / short kernels
+        if (two) CUDA_TRY(cudaStreamWaitEvent(big, c->ev_go, 0));
+        int hand = 0;
+        auto hand_over = [&](cudaStream_t from, cudaStream_t to) -> cudaError_t { // `to` continues where `from` stands
+            if (!two) return cudaSuccess;
+            cudaError_t e = cudaEventRecord(c->ev_hand[g][hand], from);
+            if (e == cudaSuccess) e = cudaStreamWaitEvent(to, c->ev_hand[g][hand], 0);
+            ++hand;
+            return e;
+        };
         uint32_t* recount_n = c->at<uint32_t>(y.recount + g * y.recount_bytes);
         uint2* recount_list = c->at<uint2>(y.recount + g * y.recount_bytes + 256);
         FbList* fb = c->at<FbList>(y.fb + g * align_up(sizeof(FbList)));
@@ -338,68 +351,72 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
             if (c->runs[i].w < w0 + nw) run1 = i + 1;
         }
         if (vec)
-            CUDA_TRY(launch_pdl(k_pass_a<true>, run1 - run0, kBigThreads, c->pass_a_smem, gs, grads, state, dbuf.code, chunks, runs + run0,
+            CUDA_TRY(launch_pdl(k_pass_a<true>, run1 - run0, kBigThreads, c->pass_a_smem, big, grads, state, dbuf.code, chunks, runs + run0,
                                 c->stride, c->dstride, reg_index, R, cell_tab, cell_win, meta, bhc, bhs));
         else
-            CUDA_TRY(launch_pdl(k_pass_a<false>, run1 - run0, kBigThreads, c->pass_a_smem, gs, grads, state, dbuf.code, chunks, runs + run0,
+            CUDA_TRY(launch_pdl(k_pass_a<false>, run1 - run0, kBigThreads, c->pass_a_smem, big, grads, state, dbuf.code, chunks, runs + run0,
                                 c->stride, c->dstride, reg_index, R, cell_tab, cell_win, meta, bhc, bhs));
         c->launches += 1;
-        mark(gs);
+        mark(big);
+        CUDA_TRY(hand_over(big, small));
         if (R) {
-            CUDA_TRY(launch_pdl(k_resolve_a, dim3(R, nw), kBigThreads, 0, gs, layers, reg_layers, R, L, ktab, K, meta, binlo, bhc, bhs,
+            CUDA_TRY(launch_pdl(k_resolve_a, dim3(R, nw), kBigThreads, 0, small, layers, reg_layers, R, L, ktab, K, meta, binlo, bhc, bhs,
                                 err, tau, keq, shf, flags, fb, fb_chunks, fb_layers, list_cap, w0));
             c->launches += 1;
         }
-        mark(gs);
+        mark(small);
         // exact radix select for the layers handed over by k_resolve_a (the lists are usually empty)
         if (R) {
             const uint32_t gfb = 2 * 148, glay = std::min<uint32_t>(nw * R, 128u);
             const dim3 gslot(glay, 1, K);
-            CUDA_TRY(launch_pdl(k_fb_hist1, gfb, blk, 0, gs, dbuf, chunks, c->dstride, L, fb, fb_chunks, h1c, h1s, flags));
-            CUDA_TRY(launch_pdl(k_resolve1, glay, blk, 0, gs, fb, fb_layers, h1c, h1s, ktab, L, K, cands, slots));
-            CUDA_TRY(launch_pdl(k_fb_hist23<2>, gfb, blk, 0, gs, dbuf, chunks, c->dstride, L, K, fb, fb_chunks, slots, h23c, h23s));
-            CUDA_TRY(launch_pdl(k_resolve23<2>, gslot, blk, 0, gs, fb, fb_layers, h23c, h23s, L, K, cands, slots, err, tau, keq, shf));
-            CUDA_TRY(launch_pdl(k_rebuild_slots, (nw * R + kThreads - 1) / kThreads, blk, 0, gs, fb, fb_layers, L, K, cands, slots));
-            CUDA_TRY(launch_pdl(k_fb_hist23<3>, gfb, blk, 0, gs, dbuf, chunks, c->dstride, L, K, fb, fb_chunks, slots, h23c, h23s));
-            CUDA_TRY(launch_pdl(k_resolve23<3>, gslot, blk, 0, gs, fb, fb_layers, h23c, h23s, L, K, cands, slots, err, tau, keq, shf));
+            CUDA_TRY(launch_pdl(k_fb_hist1, gfb, blk, 0, small, dbuf, chunks, c->dstride, L, fb, fb_chunks, h1c, h1s, flags));
+            CUDA_TRY(launch_pdl(k_resolve1, glay, blk, 0, small, fb, fb_layers, h1c, h1s, ktab, L, K, cands, slots));
+            CUDA_TRY(launch_pdl(k_fb_hist23<2>, gfb, blk, 0, small, dbuf, chunks, c->dstride, L, K, fb, fb_chunks, slots, h23c, h23s));
+            CUDA_TRY(launch_pdl(k_resolve23<2>, gslot, blk, 0, small, fb, fb_layers, h23c, h23s, L, K, cands, slots, err, tau, keq, shf));
+            CUDA_TRY(launch_pdl(k_rebuild_slots, (nw * R + kThreads - 1) / kThreads, blk, 0, small, fb, fb_layers, L, K, cands, slots));
+            CUDA_TRY(launch_pdl(k_fb_hist23<3>, gfb, blk, 0, small, dbuf, chunks, c->dstride, L, K, fb, fb_chunks, slots, h23c, h23s));
+            CUDA_TRY(launch_pdl(k_resolve23<3>, gslot, blk, 0, small, fb, fb_layers, h23c, h23s, L, K, cands, slots, err, tau, keq, shf));
             c->launches += 7;
         }
-        mark(gs);
+        mark(small);
         // (c)
         for (uint32_t wa = w0; wa < w0 + nw; wa += kDpWorkersPerLaunch) {
             const uint32_t nwa = std::min<uint32_t>(kDpWorkersPerLaunch, w0 + nw - wa);
             const int dp_mode = mode == kGivenJ ? 1 : (c->policy == 1 ? 2 : (c->policy == 2 ? 3 : (c->policy == 3 ? 4 : 0)));
-            CUDA_TRY(launch_pdl(k_dp, nwa, kDpThreads, c->dp_smem, gs, budgets_of(wa, nwa), wa, W, L, K, c->D, c->bpe, c->full_bytes, c->cap,
+            CUDA_TRY(launch_pdl(k_dp, nwa, kDpThreads, c->dp_smem, small, budgets_of(wa, nwa), wa, W, L, K, c->D, c->bpe, c->full_bytes, c->cap,
                                 c->check_finite, dp_mode, c->cost_model, c->dp_plan, layers,
                                 ktab, mode == kInjectErr ? err_dev : err, tau, keq, shf, j_dev, flags, pd, sel, out->k, out->j,
                                 out->offs, out->stats, out->dense, CodeSpace{reg_index, meta, cell_tab, cell_win, R}));
             c->launches += 1;
         }
-        mark(gs);
+        mark(small);
+        CUDA_TRY(hand_over(small, big));
         // (d), (e), (f)
-        CUDA_TRY(launch_pdl(k_sel_count, gch, blk, 0, gs, dbuf, chunks, nch, c->dstride, L, sel, layers, csel, lowh, recount_n,
+        CUDA_TRY(launch_pdl(k_sel_count, gch, blk, 0, big, dbuf, chunks, nch, c->dstride, L, sel, layers, csel, lowh, recount_n,
                             recount_list, 2 * list_cap, w0));
-        mark(gs);
-        CUDA_TRY(launch_pdl(k_sel_resolve, glw, blk, 0, gs, L, layers, nch, csel, lowh, sel, r2, r2_layers, r2_chunks, w0));
-        CUDA_TRY(launch_pdl(k_sel_count_r2, 2 * 148, blk, 0, gs, dbuf, chunks, nch, c->dstride, L, sel, layers, csel, lowh, recount_n,
+        mark(big);
+        CUDA_TRY(hand_over(big, small));
+        CUDA_TRY(launch_pdl(k_sel_resolve, glw, blk, 0, small, L, layers, nch, csel, lowh, sel, r2, r2_layers, r2_chunks, w0));
+        CUDA_TRY(launch_pdl(k_sel_count_r2, 2 * 148, blk, 0, small, dbuf, chunks, nch, c->dstride, L, sel, layers, csel, lowh, recount_n,
                             recount_list, 2 * list_cap, r2, r2_chunks));
-        CUDA_TRY(launch_pdl(k_sel_resolve_r2, std::min<uint32_t>(nw * L, 128u), blk, 0, gs, L, layers, nch, csel, lowh, sel, r2,
+        CUDA_TRY(launch_pdl(k_sel_resolve_r2, std::min<uint32_t>(nw * L, 128u), blk, 0, small, L, layers, nch, csel, lowh, sel, r2,
                             r2_layers, r2_chunks));
-        CUDA_TRY(launch_pdl(k_sel_recount, 2 * 148, blk, 0, gs, dbuf, chunks, nch, c->dstride, L, sel, recount_n, recount_list, csel));
-        CUDA_TRY(launch_pdl(k_sel_slices, (uint32_t)(((uint64_t)nw * nch + 7) / 8), blk, 0, gs, chunks, nch, w0, nw, L, sel, csel, ccnt));
-        CUDA_TRY(launch_pdl(k_sel_scan, glw, blk, 0, gs, layers, chunks, nch, L, sel, ccnt, jobs, recount_n, fb, r2, w0));
-        mark(gs);
+        CUDA_TRY(launch_pdl(k_sel_recount, 2 * 148, blk, 0, small, dbuf, chunks, nch, c->dstride, L, sel, recount_n, recount_list, csel));
+        CUDA_TRY(launch_pdl(k_sel_slices, (uint32_t)(((uint64_t)nw * nch + 7) / 8), blk, 0, small, chunks, nch, w0, nw, L, sel, csel, ccnt));
+        CUDA_TRY(launch_pdl(k_sel_scan, glw, blk, 0, small, layers, chunks, nch, L, sel, ccnt, jobs, recount_n, fb, r2, w0));
+        mark(small);
+        CUDA_TRY(hand_over(small, big));
         {
             auto launch = [&](auto kern) {
-                return launch_pdl(kern, gch, blk, 0, gs, grads, state, chunks, nch, c->dstride, c->stride, csel, jobs, c->cap,
+                return launch_pdl(kern, gch, blk, 0, big, grads, state, chunks, nch, c->dstride, c->stride, csel, jobs, c->cap,
                                   out->idx, out->val, w0);
             };
             if (c->value_dtype == 1) CUDA_TRY(dense_write ? launch(k_sel_write<true, true>) : launch(k_sel_write<true, false>));
             else CUDA_TRY(dense_write ? launch(k_sel_write<false, true>) : launch(k_sel_write<false, false>));
         }
-        mark(gs);
+        mark(big);
         c->launches += 8;
-        if (two) CUDA_TRY(cudaEventRecord(c->ev_done[g], gs));
+        if (two) CUDA_TRY(cudaEventRecord(c->ev_done[g], big));
     }
     if (two)
         for (uint32_t g = 0; g < n_groups; ++g) CUDA_TRY(cudaStreamWaitEvent(s, c->ev_done[g], 0));
@@ -542,7 +559,9 @@ void kimad_destroy(kimad_ctx* ctx) {
         cudaStreamDestroy(ctx->side);
         for (int g = 0; g < kGroups; ++g) {
             if (ctx->gstream[g]) { cudaStreamSynchronize(ctx->gstream[g]); cudaStreamDestroy(ctx->gstream[g]); }
+            if (ctx->gshort[g]) { cudaStreamSynchronize(ctx->gshort[g]); cudaStreamDestroy(ctx->gshort[g]); }
             if (ctx->ev_done[g]) cudaEventDestroy(ctx->ev_done[g]);
+            for (cudaEvent_t e : ctx->ev_hand[g]) if (e) cudaEventDestroy(e);
         }
         if (ctx->ev_go) cudaEventDestroy(ctx->ev_go);
     }
