@@ -32,13 +32,13 @@ UNIT = "elements/s"
 
 # DRAM traffic of the dominant kernel per input element: dram__bytes_read.sum + dram__bytes_write.sum of one
 # launch of the sweep kernel in an ncu capture on workload 3 (inputs larger than L2), divided by the elements of
-# that launch.  Every element is read once from each input and its upper half written once, so the figure
+# that launch.  Every element is read once from each input and one code byte written for it, so the figure
 # carries over to the other workloads; it has to be re-captured when the sweep's data movement changes.
-NCU_TRAFFIC_BYTES_PER_ELEM = {"sweep": 10.14}
+NCU_TRAFFIC_BYTES_PER_ELEM = {"sweep": 9.13}
 
 # algorithmic bytes per input element of each stage (what the stage must move at least once)
-STAGE_ALGO_BYTES = {"sweep": 10.0,  # read grad + g, write the upper halves of d
-                    "select_count": 2.0, "select_write": 8.0}
+STAGE_ALGO_BYTES = {"sweep": 9.0,  # read grad + g, write one code byte per element
+                    "select_count": 1.0, "select_write": 8.0}
 
 
 def peaks():

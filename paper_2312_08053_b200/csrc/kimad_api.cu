@@ -367,7 +367,8 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
         mark(small);
         // exact radix select for the layers handed over by k_resolve_a (the lists are usually empty)
         if (R) {
-            const uint32_t gfb = 2 * 148, glay = std::min<uint32_t>(nw * R, 128u);
+            // small grids: the lists are usually empty, and every kernel of the chain then costs only its launch
+            const uint32_t gfb = 148, glay = std::min<uint32_t>(nw * R, 32u);
             const dim3 gslot(glay, 1, K);
             CUDA_TRY(launch_pdl(k_fb_hist1, gfb, blk, 0, small, dbuf, chunks, c->dstride, L, fb, fb_chunks, h1c, h1s, flags));
             CUDA_TRY(launch_pdl(k_resolve1, glay, blk, 0, small, fb, fb_layers, h1c, h1s, ktab, L, K, cands, slots));
@@ -397,11 +398,11 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
         mark(big);
         CUDA_TRY(hand_over(big, small));
         CUDA_TRY(launch_pdl(k_sel_resolve, glw, blk, 0, small, L, layers, nch, csel, lowh, sel, r2, r2_layers, r2_chunks, w0));
-        CUDA_TRY(launch_pdl(k_sel_count_r2, 2 * 148, blk, 0, small, dbuf, chunks, nch, c->dstride, L, sel, layers, csel, lowh, recount_n,
+        CUDA_TRY(launch_pdl(k_sel_count_r2, 148, blk, 0, small, dbuf, chunks, nch, c->dstride, L, sel, layers, csel, lowh, recount_n,
                             recount_list, 2 * list_cap, r2, r2_chunks));
-        CUDA_TRY(launch_pdl(k_sel_resolve_r2, std::min<uint32_t>(nw * L, 128u), blk, 0, small, L, layers, nch, csel, lowh, sel, r2,
+        CUDA_TRY(launch_pdl(k_sel_resolve_r2, std::min<uint32_t>(nw * L, 32u), blk, 0, small, L, layers, nch, csel, lowh, sel, r2,
                             r2_layers, r2_chunks));
-        CUDA_TRY(launch_pdl(k_sel_recount, 2 * 148, blk, 0, small, dbuf, chunks, nch, c->dstride, L, sel, recount_n, recount_list, csel));
+        CUDA_TRY(launch_pdl(k_sel_recount, 148, blk, 0, small, dbuf, chunks, nch, c->dstride, L, sel, recount_n, recount_list, csel));
         CUDA_TRY(launch_pdl(k_sel_slices, (uint32_t)(((uint64_t)nw * nch + 7) / 8), blk, 0, small, chunks, nch, w0, nw, L, sel, csel, ccnt));
         CUDA_TRY(launch_pdl(k_sel_scan, glw, blk, 0, small, layers, chunks, nch, L, sel, ccnt, jobs, recount_n, fb, r2, w0));
         mark(small);
