@@ -24,8 +24,8 @@
  *     Worker w's vector starts at element w * worker_stride of `grads` and of `state`.
  *   - "device" pointers are CUDA device memory of the current device; "host" pointers are
  *     ordinary host memory.  The library never allocates or frees device memory: scratch is
- *     the caller's (kimad_set_workspace).  All kernels are ordered on the caller's stream (one of them
- *     runs on a stream of the context's own, forked from and joined to the caller's with events).
+ *     the caller's (kimad_set_workspace).  All kernels are ordered on the caller's stream (some of them
+ *     run on streams of the context's own, forked from and joined to the caller's with events).
  *     grads and state of a step must not overlap and must not change while the step is in flight: the
  *     kernels re-read them instead of keeping a copy of grad - g.
  *   - TopK order inside a layer: larger |d| first (compared on the 31 magnitude bits, so +0
@@ -142,8 +142,9 @@ int kimad_create(kimad_ctx** out, const uint64_t* layer_sizes, uint32_t n_layers
                  const double* ratio_grid, uint32_t n_ratios, const kimad_options* opt);
 void kimad_destroy(kimad_ctx* ctx);
 
-/* Scratch the kernels need (upper halves of the difference vector, histograms, DP back-pointers, tile
- * counts): about 2 bytes per element plus tables. */
+/* Scratch the kernels need (one code byte per element of the difference vector, histograms, tables, DP
+ * back-pointers, per-chunk counts): about 1 byte per element plus about 0.4 MB per (worker, layer above 4096
+ * elements). */
 size_t kimad_workspace_bytes(const kimad_ctx* ctx);
 /* dev_ptr: device, 256-byte aligned, at least kimad_workspace_bytes(); stays owned by the
  * caller and must outlive the context's steps.  Uploads the static tables and zeroes the
@@ -159,7 +160,7 @@ int kimad_set_workspace(kimad_ctx* ctx, void* dev_ptr, size_t bytes);
  *              following Eq. 2 passes (t - T_comp) / 2; a fixed byte budget is (B = bytes, t = 1)
  *   out        host struct of device pointers (see kimad_packed)
  * Returns 0 or a CUDA/argument error; per-worker outcomes land in out->stats[w].status.
- * The step's launches, including those on the context's own side stream, are ordered through events on
+ * The step's launches, including those on the context's own streams, are ordered through events on
  * cuda_stream, so a step can be captured into a CUDA graph; the budgets are then baked into the graph. */
 int kimad_step(kimad_ctx* ctx, const float* grads_dev, float* state_dev, const double* bandwidth_bytes_per_s,
                double t_target_s, const kimad_packed* out, void* cuda_stream);
@@ -285,10 +286,10 @@ int kimad_debug_enable_stage_timing(kimad_ctx* ctx, int enable);
 int kimad_debug_stage_times(kimad_ctx* ctx, float* host_ms);
 
 /* How a step schedules its workers (Section 3: every worker decides on its own, so workers are independent
- * problems).  After the sample kernel the workers are taken through the remaining stages as two groups on two
- * internal streams, forked from and joined to the step's stream, the first group with the higher priority: while
- * one group is in its latency-bound stages (curves, DP, offsets) the other one streams.  Results do not depend on
- * the schedule.  mode 0 (default): two groups when W >= 2 and W * N >= 2^25 elements; 1: two groups whenever
+ * problems).  After the sample kernel the workers are taken through the remaining stages as two groups, each on a
+ * low-priority internal stream for its sweeps and a high-priority one for its short kernels (curves, DP, offsets),
+ * forked from and joined to the step's stream: the short kernels of one group run beside the sweeps of the other.
+ * Results do not depend on the schedule.  mode 0 (default): two groups when W >= 2 and W * N >= 2^25 elements; 1: two groups whenever
  * W >= 2; 2: one group (every kernel covers all workers, on the step's stream).  Steps with stage timing enabled
  * always run as one group. */
 int kimad_debug_set_schedule(kimad_ctx* ctx, int mode);

@@ -332,7 +332,7 @@ def kimad_debug_stage_times(ctx: Ctx) -> np.ndarray:
 
 
 def kimad_debug_get_band_meta(ctx: Ctx, n_regular: int) -> np.ndarray:
-    """u32 [W][n_regular][4]: bins, split 11-bit bins, flag, detail (see kimad.h)."""
+    """u32 [W][n_regular][4]: bins, entries of the cell table in use, flag, detail (see kimad.h)."""
     out = np.zeros((ctx.W, n_regular, 4), np.uint32)
     _check(load().kimad_debug_get_band_meta(ctx.handle, out.ctypes.data), "kimad_debug_get_band_meta")
     return out
