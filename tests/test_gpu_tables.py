@@ -1,0 +1,81 @@
+"""GPU parity on inputs that stress the sweep's tables: a window of cells wider than the cell table (table entries
+then stand for several cells), sparse gradients whose thresholds fall among exact zeros, and the byte codes the
+sweep leaves for the counting sweep (layers with and without a histogram, both worker groups)."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2312_08053_b200 import binding as kb
+from tests._harness import Runner
+
+pytestmark = pytest.mark.gpu
+
+
+def _meta(r):
+    n_reg = sum(1 for n in r.ls if n > 4096)
+    return kb.kimad_debug_get_band_meta(r.ctx, n_reg)
+
+
+@pytest.mark.parametrize("schedule", [0, 1])
+def test_window_wider_than_the_cell_table(schedule):
+    """Two populations 83 octaves apart, thresholds in both: the window between the lowest and the highest band
+    has about 10,000 cells, more than the table's 4096 entries.  The sweep must run with its histograms (tables with
+    several cells per entry) and everything must match the oracle bit for bit; layers whose error bound comes out
+    too loose (the fine bins are shared by bands in both populations) may still be handed to the exact path afterwards."""
+    rng = np.random.default_rng(7)
+    sizes = [300000, 5000, 120000]
+    grid = [0.01, 0.05, 0.2, 0.45, 0.7, 0.9, 1.0]  # 0.45 .. 0.9 fall into the small population
+    W, N = 2, sum(sizes)
+    x = rng.standard_normal((W, N)).astype(np.float32)
+    small = rng.random((W, N)) < 0.6
+    x[small] *= np.float32(1e-25)
+    r = Runner(sizes, W, grid, 1000, 0, schedule=schedule)
+    grads = torch.from_numpy(x).cuda()
+    state = torch.zeros_like(grads)
+    res = r.compare_step(grads, state, [0.05 * 8 * N, 0.3 * 8 * N], 1.0)
+    assert res["same_k"]
+    m = _meta(r)
+    assert np.all(m[:, :, 2] == 0), "a layer was swept without its histogram"
+    assert np.all(m[:, :, 1] <= 4096) and np.all(m[:, [0, 2], 1] > 1500)  # table entries in use: several cells per entry
+    why = kb.kimad_debug_exact_path_layers(r.ctx, detail=True)
+    assert why[1] == 0 and why[2] == 0 and why[3] == 0  # none forced, none without tables, no threshold outside its band
+    # with the state of that step the kept entries difference to exactly zero: a third population at key 0 (the
+    # window then starts at cell 0; layers whose widened bands no longer fit are handed to the exact path)
+    res = r.compare_step(grads, state, [0.6 * 8 * N, 0.02 * 8 * N], 1.0)
+    assert res["same_k"]
+
+
+@pytest.mark.parametrize("value_dtype", [0, 1])
+def test_sparse_gradients_thresholds_among_zeros(value_dtype):
+    """90 % exact zeros (of both signs): candidates beyond the non-zero count have their threshold at key 0, where
+    only the index order decides; the state of the step before makes some differences non-zero again."""
+    rng = np.random.default_rng(21)
+    sizes = [200000, 70000, 4097, 900]
+    grid = [0.02, 0.08, 0.15, 0.5, 1.0]
+    W, N = 2, sum(sizes)
+    r = Runner(sizes, W, grid, 1000, value_dtype, schedule=1)
+    state = torch.zeros((W, N), dtype=torch.float32, device="cuda")
+    for step in range(3):
+        x = rng.standard_normal((W, N)).astype(np.float32)
+        x[rng.random((W, N)) < 0.9] = 0.0
+        x[rng.random((W, N)) < 0.05] *= -0.0  # some negative zeros
+        grads = torch.from_numpy(x).cuda()
+        bpe = 8 if value_dtype == 0 else 6
+        res = r.compare_step(grads, state, [0.3 * bpe * N, 0.12 * bpe * N], 1.0)
+        assert res["same_k"]
+
+
+def test_codes_of_layers_without_a_histogram():
+    """curve_mode 1 sweeps every layer without a histogram (codes = upper bits of the key) and resolves through the
+    exact path; mixed with tiny layers and a layer of one repeated magnitude, on two worker groups."""
+    rng = np.random.default_rng(5)
+    sizes = [150000, 12, 40000, 3000, 65536]
+    grid = [0.001, 0.01, 0.1, 0.5, 1.0]
+    W, N = 3, sum(sizes)
+    x = rng.standard_normal((W, N)).astype(np.float32)
+    x[:, -65536:] = np.sign(x[:, -65536:]) * np.float32(0.75)
+    r = Runner(sizes, W, grid, 1000, 0, curve_mode=1, schedule=1)
+    grads = torch.from_numpy(x).cuda()
+    state = torch.from_numpy((rng.standard_normal((W, N)) * 0.01).astype(np.float32)).cuda()
+    for budget in ([0.05 * 8 * N] * 3, [0.4 * 8 * N, 0.01 * 8 * N, 0.9 * 8 * N]):
+        r.compare_step(grads, state, budget, 1.0)
