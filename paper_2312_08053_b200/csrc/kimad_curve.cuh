@@ -30,7 +30,8 @@ constexpr int kFineBins = KIMAD_FINE_BINS;          // fine bins per (worker, la
 constexpr int kMaxGaps = KIMAD_MAX_RATIOS + 2;      // gap regions: below / between / above the band groups, + non-finite keys
 constexpr int kMaxBins = kFineBins + kL1Bins + 2 * kMaxGaps; // fine bins + gap regions cut at every 11-bit prefix
 constexpr int kMaxShift = 15;                       // a fine bin is 2^shift keys wide, at most a whole cell
-constexpr int kSampleUnits = 4095;                  // sample = units of 16 consecutive elements (<= 65520 elements)
+constexpr int kSampleUnit = 32;                     // consecutive elements read together (128 bytes, one warp)
+constexpr int kSampleUnits = 2047;                  // units of a sample (<= 65504 elements: the u16 cell counters cannot overflow)
 constexpr int kBigThreads = 1024;
 constexpr uint32_t kGapBit = 1u;                    // bin_lo entries carry this bit when the bin is a gap bin
 
@@ -43,7 +44,8 @@ __device__ __forceinline__ uint32_t hash_u32(uint32_t x) {
 // ------------------------------------------------------------------------------------------------
 // k_sample: one CTA per (regular layer, worker)
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kBigThreads, 1)
+// (48 registers: a CTA of the tiny layers' kernel, which runs beside this one, then fits on the same SM)
+__global__ void __maxnreg__(48)
 k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint64_t stride,
          const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ reg_layers, uint32_t R,
          const KTab ktab, uint32_t K, uint32_t force_exact, uint32_t* __restrict__ cell_tab,
@@ -77,26 +79,26 @@ k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint6
     // ---- stratified sample of |grad - g|
     const float* gr = grads + (size_t)w * stride + ld.begin;
     const float* st = state + (size_t)w * stride + ld.begin;
-    const uint32_t n_units = n / 16 + ((n & 15u) != 0); // n may be as large as 2^32 - 1
+    const uint32_t n_units = n / kSampleUnit + ((n % kSampleUnit) != 0); // n may be as large as 2^32 - 1
     const uint32_t m_units = min(n_units, (uint32_t)kSampleUnits);
     const bool whole = m_units == n_units;
     const uint32_t sq_ = n / (uint32_t)kSampleUnits, sr_ = n % (uint32_t)kSampleUnits; // used when sampled: m_units = kSampleUnits
     uint32_t mine = 0;
-    // a half-warp reads one unit; eight units per thread are in flight before their keys are counted
-    for (uint32_t ib = threadIdx.x >> 4; ib < m_units; ib += 8 * (kBigThreads / 16)) {
+    // a warp reads one unit (128 bytes); eight units per thread are in flight before their keys are counted
+    for (uint32_t ib = threadIdx.x / kSampleUnit; ib < m_units; ib += 8 * (kBigThreads / kSampleUnit)) {
         float a[8], b[8];
         bool ok[8];
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
-            const uint32_t i = ib + u * (kBigThreads / 16);
-            uint32_t start = 16 * i;
+            const uint32_t i = ib + u * (kBigThreads / kSampleUnit);
+            uint32_t start = kSampleUnit * i;
             if (!whole && i < m_units) { // unit i somewhere inside stratum i = [i q + i r / m, (i+1) q + (i+1) r / m)
                 const uint32_t s0 = i * sq_ + (i * sr_) / (uint32_t)kSampleUnits;
                 const uint32_t s1 = (i + 1) * sq_ + ((i + 1) * sr_) / (uint32_t)kSampleUnits;
-                const uint32_t room = s1 > s0 + 16 ? s1 - s0 - 16 : 0;
+                const uint32_t room = s1 > s0 + kSampleUnit ? s1 - s0 - kSampleUnit : 0;
                 start = s0 + __umulhi(hash_u32(i * 0x9e3779b9u + l * 0x85ebca6bu + 1u), room + 1);
             }
-            const uint32_t p = start + (threadIdx.x & 15);
+            const uint32_t p = start + (threadIdx.x % kSampleUnit);
             ok[u] = i < m_units && p < n;
             a[u] = ok[u] ? gr[p] : 0.f;
             b[u] = ok[u] ? st[p] : 0.f;
