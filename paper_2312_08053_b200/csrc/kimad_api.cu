@@ -140,7 +140,7 @@ void plan_layout(kimad_ctx* c) {
     } while (0)
 
 constexpr size_t kDpSmemMax = 225 * 1024; // dynamic shared memory the DP kernel may ask for
-constexpr uint32_t kSweepWaves = 2;       // CTAs of the sweep per SM (148 SMs), one resident at a time
+constexpr uint64_t kSweepRunElems = 4ull << 20; // elements a CTA of the sweep takes at most (as long as four waves suffice)
 constexpr uint64_t kPipelineMinElems = 1ull << 25; // W N from which a step is run as two groups of workers
 
 // Kernels are loaded on their first launch; loading one takes about a millisecond.  Touching every kernel a
@@ -512,10 +512,14 @@ int kimad_create(kimad_ctx** out, const uint64_t* layer_sizes, uint32_t n_layers
         if (c->policy == 2 && !c->dp_plan.tab_in_smem) { delete c; return KIMAD_ERR_INVALID_ARG; }
         c->sample_smem = (size_t)(2 * (1024 + 32) + 32768 + 1024 + 2 * kMaxGaps + 32 + 3 * 128) * 4;
         c->pass_a_smem = (size_t)(2 * kMaxBins + kCellTab) * 4;
-        { // the sweep's runs: every worker's chunk list is cut into pieces of about equal element counts, about
-          // kSweepWaves CTAs per SM in all (one CTA is resident per SM)
+        { // the sweep's runs, one CTA each: every worker's chunk list is cut into pieces of about equal element counts.
+          // The sweep of a group of workers ((W + 1) / 2 of them) is one wave of CTAs (148 SMs, one CTA resident per
+          // SM), or up to four waves when a run would otherwise exceed kSweepRunElems: long static runs end
+          // unevenly, and later waves even that out.
             const uint32_t nch = (uint32_t)c->chunks.size();
-            const uint32_t per_w = std::max<uint32_t>(1u, std::min<uint32_t>(nch, (kSweepWaves * 148u + c->W - 1) / c->W));
+            const uint32_t gw = (c->W + 1) / 2; // workers in the larger group (1 for a single worker)
+            const uint64_t waves = std::min<uint64_t>(4, std::max<uint64_t>(1, (N * gw + 148ull * kSweepRunElems - 1) / (148ull * kSweepRunElems)));
+            const uint32_t per_w = std::max<uint32_t>(1u, std::min<uint32_t>(nch, (uint32_t)((waves * 148u + gw - 1) / gw)));
             for (uint32_t w = 0; w < c->W; ++w) {
                 uint64_t acc = 0;
                 uint32_t g = 0, start = 0;
