@@ -3,7 +3,7 @@
 //
 // Stage map of one step (letters as in include/kimad.h; file in brackets):
 //   k_sample        (a)+(b) per (worker, layer): stratified sample of |grad - g| -> for every candidate k_j the
-//                   band of 16-bit key prefixes that can hold its threshold -> bin tables        [kimad_curve.cuh]
+//                   band of 16-bit key prefixes that can hold its threshold -> bins and the cell table [kimad_curve.cuh]
 //   k_pass_a        (a)+(b) the sweep: d = grad - g (Section 3 footnote, Eq. 6), bin = table(key(d)), count and
 //                   exact integer sum of squares per bin in shared memory; one byte per element (a monotone code
 //                   of its bin) goes to scratch, d itself is never stored                         [kimad_curve.cuh]
@@ -20,8 +20,10 @@
 //   k_sel_write     (e)+(f) ordered (index, value) pack and g += C(d) (Algorithm 1, Eq. 6)       [kimad_select.cuh]
 //   k_apply_packed, k_aggregate   receiving side and model step (Algorithm 1, server lines)      [kimad_receiver.cuh]
 //
-// Nothing here is a dense contraction, so there is no tensor-core path.  The sweep is bound by instruction issue and
-// shared-memory latency (it keeps 0.9 of its time when its loads are served from cache); the other sweeps by HBM.
+// Nothing here is a dense contraction, so there is no tensor-core path.  The sweep runs at 83-90 % of the measured HBM
+// copy rate on its 9 bytes per element (one shared-memory table read and two shared-memory atomics per element keep it
+// from the rest); the counting and write sweeps are bound by HBM on large layers and by load latency on small ones.
+// After the sample kernel the workers go through the stages as two groups on streams of their own (kimad_api.cu).
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
