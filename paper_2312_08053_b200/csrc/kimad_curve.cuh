@@ -457,7 +457,15 @@ k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, uint8
             for (uint32_t i = threadIdx.x; i < min(run.c1 - c, (uint32_t)kRunDesc); i += kBigThreads) s_desc[i] = chunks[c + i];
             __syncthreads();
         }
-        const Chunk ch = s_desc[di];
+        Chunk ch = s_desc[di];
+        // the chunks of one layer follow each other without a gap: those among the staged descriptors are swept as
+        // one span, so that the load pipeline below is filled once per span and not once per chunk
+        while (c + 1 < run.c1 && (c + 1 - run.c0) % (uint32_t)kRunDesc != 0) {
+            const Chunk& nx = s_desc[(c + 1 - run.c0) % (uint32_t)kRunDesc];
+            if (nx.layer != ch.layer || nx.begin != ch.end) break;
+            ch.end = nx.end;
+            ++c;
+        }
         if ((int)ch.layer != cur_layer) {
             if (dirty) flush();
             cur_layer = (int)ch.layer;
@@ -481,23 +489,26 @@ k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, uint8
             const float4* gr4 = reinterpret_cast<const float4*>(gr0 + cv.a0);
             const float4* st4 = reinterpret_cast<const float4*>(st0 + cv.a0);
             const uint32_t q_lo = (cv.first + 3) >> 2, q_hi = cv.len >> 2; // whole quads [q_lo, q_hi)
-            constexpr int U = 4; // quads in flight per thread: 16 KB per array and pass, two passes per full chunk
-            for (uint32_t qb = q_lo + threadIdx.x; qb < q_hi; qb += kBigThreads * U) {
-                float4 a[U], b[U];
-#pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    const uint32_t q = qb + u * kBigThreads;
-                    if (q < q_hi) { a[u] = __ldcg(gr4 + q); b[u] = __ldcg(st4 + q); }
-                }
-#pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    const uint32_t q = qb + u * kBigThreads;
-                    if (q < q_hi) {
-                        const uint32_t k[4] = {key_of(__fsub_rn(a[u].x, b[u].x)), key_of(__fsub_rn(a[u].y, b[u].y)),
-                                               key_of(__fsub_rn(a[u].z, b[u].z)), key_of(__fsub_rn(a[u].w, b[u].w))};
-                        reinterpret_cast<uint32_t*>(dc)[q] = active ? acc4(k) : pack_key_codes(k[0], k[1], k[2], k[3]);
-                    }
-                }
+            // One quad per thread and round; the loads of the round three rounds ahead are issued before the current
+            // round is processed (four register sets, taken in turn), so that a round's memory latency lies behind
+            // the work of the rounds before it
+            auto fetch = [&](float4& a, float4& b, uint32_t q) {
+                if (q < q_hi) { a = __ldcg(gr4 + q); b = __ldcg(st4 + q); }
+            };
+            auto work = [&](const float4& a, const float4& b, uint32_t q) {
+                const uint32_t k[4] = {key_of(__fsub_rn(a.x, b.x)), key_of(__fsub_rn(a.y, b.y)),
+                                       key_of(__fsub_rn(a.z, b.z)), key_of(__fsub_rn(a.w, b.w))};
+                reinterpret_cast<uint32_t*>(dc)[q] = active ? acc4(k) : pack_key_codes(k[0], k[1], k[2], k[3]);
+            };
+            float4 a0, b0, a1, b1, a2, b2, a3, b3;
+            uint32_t qb = q_lo + threadIdx.x;
+            constexpr uint32_t S = kBigThreads;
+            fetch(a0, b0, qb); fetch(a1, b1, qb + S); fetch(a2, b2, qb + 2 * S);
+            while (qb < q_hi) {
+                fetch(a3, b3, qb + 3 * S); work(a0, b0, qb); qb += S; if (qb >= q_hi) break;
+                fetch(a0, b0, qb + 3 * S); work(a1, b1, qb); qb += S; if (qb >= q_hi) break;
+                fetch(a1, b1, qb + 3 * S); work(a2, b2, qb); qb += S; if (qb >= q_hi) break;
+                fetch(a2, b2, qb + 3 * S); work(a3, b3, qb); qb += S;
             }
             if (threadIdx.x < 8) { // ragged edges: [first, min(4 q_lo, len)) and [max(4 q_hi, 4 q_lo), len)
                 uint32_t e;
