@@ -224,13 +224,16 @@ def test_run_to_run_determinism_of_decisions():
         assert all(np.array_equal(a, b) for a, b in zip(outs[0], o))
 
 
-def test_step_is_capturable_in_a_cuda_graph():
-    """All work of a step, the forked side stream included, is ordered through the caller's stream: the step can
-    be captured once and replayed on new gradients (the budgets are baked into the captured launches)."""
-    wl = workloads.workload(1)
+@pytest.mark.parametrize("cfg,divisor,schedule", [(1, 1, 0), (2, 16, 1)])
+def test_step_is_capturable_in_a_cuda_graph(cfg, divisor, schedule):
+    """All work of a step, the forked streams included (the tiny layers' side stream; with schedule 1 the two worker
+    groups' sweep and short-kernel streams), is ordered through the caller's stream: the step can be captured once
+    and replayed on new gradients (the budgets are baked into the captured launches)."""
+    wl = workloads.workload(cfg, divisor)
     W, N = wl.n_workers, wl.N
     bw = workloads.bandwidth_trace(wl)[0]
     ctx = kb.new_context(wl.layer_sizes, W, wl.ratio_grid, D=wl.D, value_dtype=wl.value_dtype)
+    kb.kimad_debug_set_schedule(ctx, schedule)
     out = kb.Packed(ctx)
     grads = workloads.gradients(wl, 0, device="cuda")
     state = torch.zeros((W, N), device="cuda")
