@@ -237,28 +237,50 @@ __device__ __forceinline__ void sel_resolve_layer(uint32_t l, uint32_t w, uint32
         __syncthreads();
         sorted = !*s_over;
         if (sorted) {
+            // the rank-th largest of the collected entries (16-bit numbers) by two 8-bit digits: a histogram of the
+            // upper digit, then one of the lower digit among the entries that share the upper digit found
             const uint32_t cnt = *s_n;
-            uint32_t np = 1;
-            while (np < cnt) np <<= 1;
-            for (uint32_t i = cnt + threadIdx.x; i < np; i += kThreads) s_key[i] = 0; // padding sorts last
-            __syncthreads();
-            for (uint32_t size = 2; size <= np; size <<= 1)
-                for (uint32_t str = size >> 1; str > 0; str >>= 1) {
-                    for (uint32_t i = threadIdx.x; i < np / 2; i += kThreads) {
-                        const uint32_t a = 2 * i - (i & (str - 1)), b = a + str;
-                        const bool desc = (a & size) == 0;
-                        const uint32_t ka = s_key[a], kb = s_key[b];
-                        if ((ka < kb) == desc) { s_key[a] = kb; s_key[b] = ka; }
-                    }
-                    __syncthreads();
+            static_assert(kThreads == 256, "one thread per digit");
+            __shared__ uint32_t s_h[256];
+            __shared__ uint32_t s_digit, s_gt;
+            uint32_t rank = s.keep_eq, hi_digit = 0, greater = 0; // rank <= cnt by construction
+            for (int pass = 0; pass < 2; ++pass) {
+                s_h[threadIdx.x] = 0; // kThreads == 256
+                __syncthreads();
+                for (uint32_t i = threadIdx.x; i < cnt; i += kThreads) {
+                    const uint32_t k = s_key[i];
+                    if (pass == 0) atomicAdd(&s_h[k >> 8], 1u);
+                    else if ((k >> 8) == hi_digit) atomicAdd(&s_h[k & 255u], 1u);
                 }
+                __syncthreads();
+                if (threadIdx.x < 32) { // warp 0: lane L takes the digits 255 - 8 L down to 248 - 8 L
+                    const uint32_t lane = threadIdx.x, top = 255u - 8u * lane;
+                    uint32_t mine = 0;
+#pragma unroll
+                    for (uint32_t j = 0; j < 8; ++j) mine += s_h[top - j];
+                    uint32_t incl = mine;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
+                        if (lane >= (uint32_t)o) incl += y;
+                    }
+                    const uint32_t hit = __ballot_sync(0xffffffffu, incl >= rank);
+                    if (hit && lane == (uint32_t)(__ffs(hit) - 1)) {
+                        uint32_t acc = incl - mine, d = top;
+                        while (acc + s_h[d] < rank) { acc += s_h[d]; --d; }
+                        s_digit = d;
+                        s_gt = acc; // entries of this pass's candidates with a larger digit
+                    }
+                }
+                __syncthreads();
+                if (pass == 0) { hi_digit = s_digit; greater = s_gt; rank -= s_gt; }
+                else { greater += s_gt; }
+            }
             if (threadIdx.x == 0) {
-                const uint32_t rank = s.keep_eq, t = s_key[rank - 1]; // rank <= cnt by construction
-                uint32_t first = rank - 1;
-                while (first > 0 && s_key[first - 1] == t) --first;
+                const uint32_t t = (hi_digit << 8) | s_digit;
                 s.tau_low = t;
                 s.tau += t;
-                s.keep_eq = rank - first;
+                s.keep_eq = s.keep_eq - greater; // rank among the entries equal to t: those above t come first
                 s.shift = 0;
                 sel[wl] = s;
             }
