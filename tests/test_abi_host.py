@@ -83,3 +83,14 @@ def test_step_without_workspace_is_refused():
     assert rc == kb.KIMAD_ERR_WORKSPACE
     assert "workspace" in kb.kimad_strerror(rc)
     assert kb.load().kimad_set_workspace(ctx.handle, None, 0) == kb.KIMAD_ERR_WORKSPACE
+
+
+def test_schedule_modes_are_validated():
+    ctx = kb.kimad_create([8, 9000], 3, [0.5, 1.0])
+    for mode in (0, 1, 2):
+        kb.kimad_debug_set_schedule(ctx, mode)
+    for mode in (-1, 3):
+        with pytest.raises(kb.KimadError) as e:
+            kb.kimad_debug_set_schedule(ctx, mode)
+        assert e.value.code == kb.KIMAD_ERR_INVALID_ARG
+    kb.kimad_destroy(ctx)
