@@ -276,6 +276,15 @@ def run_kimad(args, rank, world):
     status, _ = kb.kimad_get_k(ctx)
     if status < 0:
         raise RuntimeError(f"kimad step failed on rank {rank}: {kb.kimad_strerror(status)}")
+    if args.timeline and rank == 0:
+        # one more step with events around every launch: which kernels ran beside each other, on which stream
+        s = args.warmup + args.steps
+        text = kb.kimad_debug_trace_step(ctx, grads[s % n_bufs], state, bw[s % len(bw)], wl.t_target, out, stream)
+        dense = W * N * bpe
+        with open(args.timeline, "w") as f:
+            f.write(f"# workload {args.config}, schedule {SCHEDULE}, step {s}: budget = "
+                    f"{100.0 * float(np.sum(bw[s % len(bw)])) * wl.t_target / dense:.2f} % of the dense bytes\n")
+            f.write(text)
 
     # ---- end to end: host buffers in, packed message out, copies inside the timed region.  Two drivers of the
     # same public calls: one after the other (copy in, step, copy out), and the double-buffered driver that
@@ -463,6 +472,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--schedule", type=int, default=0, choices=[0, 1, 2],
                     help="0: the library's choice (two worker groups for large steps), 1: always two groups, 2: one group")
+    ap.add_argument("--timeline", default=None, metavar="FILE",
+                    help="after the timed steps, run one step with events around every launch and write its timeline")
     ap.add_argument("--no-also", action="store_true", help="skip the second large workload's device-timed block")
     ap.add_argument("--path", default="compress", choices=["compress", "receive"],
                     help="compress: the worker-side pass (the headline); receive: apply + aggregate on the server")

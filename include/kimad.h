@@ -294,6 +294,15 @@ int kimad_debug_stage_times(kimad_ctx* ctx, float* host_ms);
  * always run as one group. */
 int kimad_debug_set_schedule(kimad_ctx* ctx, int mode);
 
+/* kimad_step with a pair of CUDA events around every kernel launch; synchronises the device before and after and
+ * writes one line per launch to text (host, text_len bytes, NUL-terminated, truncated if too short): kernel, ordinal
+ * of its stream (in order of first use: 0 is the step's stream), start and end in milliseconds after the step was
+ * issued.  Shows which kernels of the two worker groups run beside each other.  The events keep a kernel from being
+ * scheduled ahead of its predecessor, so a traced step takes a few per cent longer than an untraced one.  A
+ * development aid: one traced step at a time per process.  Arguments and errors as kimad_step. */
+int kimad_debug_trace_step(kimad_ctx* ctx, const float* grads_dev, float* state_dev, const double* bandwidth_bytes_per_s,
+                           double t_target_s, const kimad_packed* out, void* cuda_stream, char* text, size_t text_len);
+
 /* Checked build of the library (compiled with -DKIMAD_CHECKED; the stand-in for a memory checker): the kernels
  * test their indices into the workspace and the output buffers before use -- a failed test sets its bit in a
  * status word and the access is skipped, nothing traps -- and the workspace regions are separated by canary words.

@@ -109,6 +109,8 @@ def load():
     L.kimad_debug_stage_times.argtypes = [vp, vp]
     L.kimad_debug_set_schedule.restype = C.c_int
     L.kimad_debug_set_schedule.argtypes = [vp, C.c_int]
+    L.kimad_debug_trace_step.restype = C.c_int
+    L.kimad_debug_trace_step.argtypes = [vp, vp, vp, C.POINTER(dbl), dbl, vp, vp, C.c_char_p, C.c_size_t]
     L.kimad_debug_get_band_meta.restype = C.c_int
     L.kimad_debug_get_band_meta.argtypes = [vp, vp]
     L.kimad_debug_exact_path_layers.restype = C.c_int
@@ -322,6 +324,16 @@ def kimad_debug_enable_stage_timing(ctx: Ctx, enable: bool) -> None:
 def kimad_debug_set_schedule(ctx: Ctx, mode: int) -> None:
     """0: two worker groups for large steps, 1: whenever W >= 2, 2: one group."""
     _check(load().kimad_debug_set_schedule(ctx.handle, int(mode)), "kimad_debug_set_schedule")
+
+
+def kimad_debug_trace_step(ctx: Ctx, grads, state, bandwidth_bytes_per_s, t_target_s, out: "Packed", stream=None) -> str:
+    """One step with CUDA events around every launch; returns the timeline, one line per launch."""
+    bw = _bw(ctx, bandwidth_bytes_per_s)
+    buf = C.create_string_buffer(1 << 16)
+    _check(load().kimad_debug_trace_step(ctx.handle, grads.data_ptr(), state.data_ptr(),
+                                         bw.ctypes.data_as(C.POINTER(C.c_double)), float(t_target_s), C.byref(out.c),
+                                         _stream_ptr(stream), buf, len(buf)), "kimad_debug_trace_step")
+    return buf.value.decode()
 
 
 def kimad_debug_stage_times(ctx: Ctx) -> np.ndarray:

@@ -3,6 +3,7 @@
 // here; the caller's workspace is carved into the regions listed in `Layout`.
 #include <cmath>
 #include <cstdlib>
+#include <cstdio>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -161,9 +162,20 @@ static int preload_kernels() {
     return KIMAD_OK;
 }
 
+// Launch trace (kimad_debug_trace_step): while a traced step is being issued every launch is bracketed by a pair of
+// CUDA events on its stream.  One traced step at a time per process (a development aid, not thread-safe).
+struct LaunchRec { const char* name; cudaStream_t s; cudaEvent_t a, b; };
+static std::vector<LaunchRec>* g_launch_trace = nullptr;
+
 // Launch with programmatic stream serialisation (the kernel must start with pdl_wait()).
 template <typename... KArgs, typename... Args>
-static cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
+static cudaError_t launch_named(const char* name, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                                Args... args) {
+    LaunchRec rec{name, s, nullptr, nullptr};
+    if (g_launch_trace) {
+        if (cudaEventCreate(&rec.a) != cudaSuccess || cudaEventCreate(&rec.b) != cudaSuccess) return cudaErrorUnknown;
+        cudaEventRecord(rec.a, s);
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = block;
@@ -174,8 +186,14 @@ static cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, siz
     at[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+    if (g_launch_trace) {
+        cudaEventRecord(rec.b, s);
+        g_launch_trace->push_back(rec);
+    }
+    return e;
 }
+#define launch_pdl(kern, ...) launch_named(#kern, kern, __VA_ARGS__)
 
 static int ensure_side_stream(kimad_ctx* c) {
     if (c->side) return KIMAD_OK;
@@ -367,8 +385,9 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
         mark(small);
         // exact radix select for the layers handed over by k_resolve_a (the lists are usually empty)
         if (R) {
-            // small grids: the lists are usually empty, and every kernel of the chain then costs only its launch
-            const uint32_t gfb = 148, glay = std::min<uint32_t>(nw * R, 32u);
+            // small grids: the lists are usually empty, and every kernel of the chain then costs only its launch; the
+            // histogram kernels get four CTAs per SM, enough to stream a large handed-over layer
+            const uint32_t gfb = 4 * 148, glay = std::min<uint32_t>(nw * R, 32u);
             const dim3 gslot(glay, 1, K);
             CUDA_TRY(launch_pdl(k_fb_hist1, gfb, blk, 0, small, dbuf, chunks, c->dstride, L, fb, fb_chunks, h1c, h1s, flags));
             CUDA_TRY(launch_pdl(k_resolve1, glay, blk, 0, small, fb, fb_layers, h1c, h1s, ktab, L, K, cands, slots));
@@ -409,8 +428,8 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
         CUDA_TRY(hand_over(small, big));
         {
             auto launch = [&](auto kern) {
-                return launch_pdl(kern, gch, blk, 0, big, grads, state, chunks, nch, c->dstride, c->stride, csel, jobs, c->cap,
-                                  out->idx, out->val, w0);
+                return launch_named("k_sel_write", kern, gch, blk, 0, big, grads, state, chunks, nch, c->dstride, c->stride, csel,
+                                    jobs, c->cap, out->idx, out->val, w0);
             };
             if (c->value_dtype == 1) CUDA_TRY(dense_write ? launch(k_sel_write<true, true>) : launch(k_sel_write<true, false>));
             else CUDA_TRY(dense_write ? launch(k_sel_write<false, true>) : launch(k_sel_write<false, false>));
@@ -581,6 +600,45 @@ int kimad_debug_enable_stage_timing(kimad_ctx* c, int enable) {
     }
     c->timing = enable != 0;
     return KIMAD_OK;
+}
+
+int kimad_debug_trace_step(kimad_ctx* c, const float* grads_dev, float* state_dev, const double* bandwidth_bytes_per_s,
+                           double t_target_s, const kimad_packed* out, void* cuda_stream, char* text, size_t text_len) {
+    if (!text || text_len == 0) return KIMAD_ERR_INVALID_ARG;
+    text[0] = 0;
+    if (g_launch_trace) return KIMAD_ERR_INVALID_ARG; // another traced step is being issued
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+    std::vector<LaunchRec> recs;
+    cudaEvent_t start = nullptr;
+    CUDA_TRY(cudaEventCreate(&start));
+    CUDA_TRY(cudaDeviceSynchronize());
+    CUDA_TRY(cudaEventRecord(start, s));
+    g_launch_trace = &recs;
+    const int rc = run_step(c, grads_dev, state_dev, bandwidth_bytes_per_s, t_target_s, out, cuda_stream, kNormal, nullptr, nullptr);
+    g_launch_trace = nullptr;
+    const cudaError_t sync = cudaDeviceSynchronize();
+    std::vector<cudaStream_t> streams; // ordinal of a stream = order of its first launch
+    size_t at = 0;
+    for (const LaunchRec& r : recs) {
+        float t0 = 0.f, t1 = 0.f;
+        if (sync == cudaSuccess && rc == KIMAD_OK) {
+            cudaEventElapsedTime(&t0, start, r.a);
+            cudaEventElapsedTime(&t1, start, r.b);
+            size_t si = 0;
+            while (si < streams.size() && streams[si] != r.s) ++si;
+            if (si == streams.size()) streams.push_back(r.s);
+            if (at < text_len) {
+                const int n = snprintf(text + at, text_len - at, "%-28s stream %zu  %8.3f -> %8.3f ms\n", r.name, si, t0, t1);
+                if (n > 0) at += (size_t)n;
+            }
+        }
+        cudaEventDestroy(r.a);
+        cudaEventDestroy(r.b);
+    }
+    cudaEventDestroy(start);
+    text[text_len - 1] = 0;
+    if (sync != cudaSuccess) return KIMAD_ERR_CUDA;
+    return rc;
 }
 
 int kimad_debug_set_schedule(kimad_ctx* c, int mode) {

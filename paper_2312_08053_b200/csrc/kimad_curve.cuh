@@ -739,8 +739,13 @@ k_tiny_exact(const float* __restrict__ grads, const float* __restrict__ state, u
 }
 
 // ------------------------------------------------------------------------------------------------
-// exact radix path over the handed-over chunks (global atomics: the list is short or empty)
+// exact radix path over the handed-over chunks.  The list is usually empty, but a handed-over layer may be large and
+// may hold one key millions of times (the exact zeros of a sparse gradient): every thread therefore adds up the run
+// of consecutive elements of its own that fall into one bin and issues its atomics when the bin changes, and keeps
+// four elements' loads in flight.
 // ------------------------------------------------------------------------------------------------
+constexpr int kFbAhead = 4; // elements per thread whose loads are issued together
+
 __global__ void __launch_bounds__(kThreads)
 k_fb_hist1(DSource dbuf, const Chunk* __restrict__ chunks, uint64_t dstride, uint32_t L,
            const FbList* __restrict__ fb, const uint2* __restrict__ fb_chunks, uint32_t* __restrict__ g_cnt,
@@ -755,14 +760,28 @@ k_fb_hist1(DSource dbuf, const Chunk* __restrict__ chunks, uint64_t dstride, uin
         const DView dd(dbuf, e.x, dstride, cv.a0);
         for (int b = threadIdx.x; b < kL1Bins; b += kThreads) { s_cnt[b] = 0; s_hi[b] = 0; s_lo[b] = 0; }
         __syncthreads();
-        for (uint32_t x = cv.first + threadIdx.x; x < cv.len; x += kThreads) {
-            const uint32_t key = key_of(dd.at(x));
-            const uint32_t sq = (uint32_t)sq_fixed(key);
-            atomicAdd(&s_cnt[key >> 20], 1u);
-            atomicAdd(&s_hi[key >> 20], sq >> 16);
-            atomicAdd(&s_lo[key >> 20], sq & 0xffffu);
-            if (key >= 0x7f800000u) atomicOr(&flags[e.x], 1u);
+        // a thread sees at most kChunkElems / kThreads elements of a chunk: its two partial sums stay below 2^32
+        uint32_t cur = 0, cn = 0, chi = 0, clo = 0;
+        bool nonfinite = false;
+        auto flush = [&]() {
+            if (cn) { atomicAdd(&s_cnt[cur], cn); atomicAdd(&s_hi[cur], chi); atomicAdd(&s_lo[cur], clo); }
+        };
+        for (uint32_t x0 = cv.first + threadIdx.x; x0 < cv.len; x0 += kFbAhead * kThreads) {
+            float v[kFbAhead];
+#pragma unroll
+            for (int u = 0; u < kFbAhead; ++u) v[u] = x0 + u * kThreads < cv.len ? dd.at(x0 + u * kThreads) : 0.f;
+#pragma unroll
+            for (int u = 0; u < kFbAhead; ++u) {
+                if (x0 + u * kThreads >= cv.len) break;
+                const uint32_t key = key_of(v[u]);
+                const uint32_t sq = (uint32_t)sq_fixed(key);
+                if ((key >> 20) != cur) { flush(); cur = key >> 20; cn = 0; chi = 0; clo = 0; }
+                ++cn; chi += sq >> 16; clo += sq & 0xffffu;
+                nonfinite |= key >= 0x7f800000u;
+            }
         }
+        flush();
+        if (nonfinite) atomicOr(&flags[e.x], 1u);
         __syncthreads();
         uint32_t* gc = g_cnt + ((size_t)e.x * L + ch.layer) * kL1Bins;
         unsigned long long* gs = g_ss + ((size_t)e.x * L + ch.layer) * kL1Bins;
@@ -805,20 +824,39 @@ k_fb_hist23(DSource dbuf, const Chunk* __restrict__ chunks, uint64_t dstride, ui
         const DView dd(dbuf, e.x, dstride, cv.a0);
         uint32_t* gc = g_cnt + wl * K * kL23Bins;
         unsigned long long* gs = g_ss + wl * K * kL23Bins;
-        for (uint32_t x = cv.first + threadIdx.x; x < cv.len; x += kThreads) {
-            const uint32_t key = key_of(dd.at(x));
-            const uint32_t f = s_first[key >> 20];
-            if (f == 0xff) continue;
-            if (LEVEL == 2) {
-                const uint32_t bin = (key >> 10) & 1023u;
-                atomicAdd(&gc[(size_t)f * kL23Bins + bin], 1u);
-                atomicAdd(&gs[(size_t)f * kL23Bins + bin], (unsigned long long)sq_fixed(key));
-            } else {
-                const uint32_t nn = s_num[key >> 20], p21 = key >> 10;
-                for (uint32_t s = f; s < f + nn; ++s)
-                    if (s_prefix[s] == p21) { atomicAdd(&gc[(size_t)s * kL23Bins + (key & 1023u)], 1u); break; }
+        uint32_t cur = 0xffffffffu, cn = 0; // (slot, bin) of the thread's current run, its entries and squares
+        unsigned long long csq = 0;
+        auto flush = [&]() {
+            if (cn) {
+                atomicAdd(&gc[cur], cn);
+                if (LEVEL == 2) atomicAdd(&gs[cur], csq);
+            }
+        };
+        for (uint32_t x0 = cv.first + threadIdx.x; x0 < cv.len; x0 += kFbAhead * kThreads) {
+            float v[kFbAhead];
+#pragma unroll
+            for (int u = 0; u < kFbAhead; ++u) v[u] = x0 + u * kThreads < cv.len ? dd.at(x0 + u * kThreads) : 0.f;
+#pragma unroll
+            for (int u = 0; u < kFbAhead; ++u) {
+                if (x0 + u * kThreads >= cv.len) break;
+                const uint32_t key = key_of(v[u]);
+                const uint32_t f = s_first[key >> 20];
+                if (f == 0xff) continue;
+                uint32_t at = 0xffffffffu;
+                if (LEVEL == 2) {
+                    at = f * (uint32_t)kL23Bins + ((key >> 10) & 1023u);
+                } else {
+                    const uint32_t nn = s_num[key >> 20], p21 = key >> 10;
+                    for (uint32_t s = f; s < f + nn; ++s)
+                        if (s_prefix[s] == p21) { at = s * (uint32_t)kL23Bins + (key & 1023u); break; }
+                    if (at == 0xffffffffu) continue;
+                }
+                if (at != cur) { flush(); cur = at; cn = 0; csq = 0; }
+                ++cn;
+                if (LEVEL == 2) csq += (unsigned long long)sq_fixed(key);
             }
         }
+        flush();
         __syncthreads();
     }
 }

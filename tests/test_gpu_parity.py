@@ -363,3 +363,22 @@ def test_concentrated_magnitudes_second_select_round(seed):
     state = torch.zeros_like(grads)
     for frac in (0.05, 0.25, 0.45, 0.7):
         r.compare_step(grads, state.clone(), [frac * 8 * N], 1.0)
+
+
+def test_traced_step_equals_a_plain_step():
+    """The launch trace only adds events: results equal the oracle's, and the timeline names both groups' sweeps."""
+    rng = np.random.default_rng(3)
+    sizes = [90000, 700, 40000, 5000]
+    W, N = 4, sum(sizes)
+    r = Runner(sizes, W, [0.01, 0.1, 0.5, 1.0], 1000, 0, schedule=1)
+    grads = torch.from_numpy(rng.standard_normal((W, N)).astype(np.float32)).cuda()
+    state = torch.zeros_like(grads)
+    r.compare_step(grads, state, [0.2 * 8 * N] * W, 1.0)
+    ref_state = state.clone()
+    state.zero_()
+    text = kb.kimad_debug_trace_step(r.ctx, grads, state, [0.2 * 8 * N] * W, 1.0, r.out)
+    assert torch.equal(state, ref_state)
+    lines = [ln.split() for ln in text.strip().splitlines()]
+    sweeps = [ln for ln in lines if ln[0].startswith("k_pass_a")]
+    assert len(sweeps) == 2 and sweeps[0][2] != sweeps[1][2]  # one sweep per group, on different streams
+    assert all(float(ln[3]) <= float(ln[5]) for ln in lines)
