@@ -266,9 +266,10 @@ int kimad_debug_step_with_j(kimad_ctx* ctx, const float* grads_dev, float* state
                             void* cuda_stream, const uint32_t* j_dev);
 
 /* How many (worker, layer) pairs took the exact radix path since the workspace was attached.
- * host_count: host, u64 [5 + K]: total, then by reason: forced by curve_mode 1; bands too wide for
- * the tables; a threshold outside its sampled band; error bound too loose; then, per candidate, how often
- * its bound was the loose one.  Synchronises the device. */
+ * host_count: host, u64 [6 + K]: total, then by reason: forced by curve_mode 1; bands too wide for
+ * the tables; a threshold outside its sampled band; error bound too loose even after refinement; then the
+ * number of pairs whose loose candidates were refined (one more pass over the layer's code bytes, not the
+ * exact path); then, per candidate, how often its first bound was the loose one.  Synchronises the device. */
 int kimad_debug_exact_path_layers(kimad_ctx* ctx, uint64_t* host_count);
 
 /* Band tables of the last step, one record of four u32 per (worker, layer above the tiny size), in

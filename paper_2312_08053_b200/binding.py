@@ -352,8 +352,9 @@ def kimad_debug_get_band_meta(ctx: Ctx, n_regular: int) -> np.ndarray:
 
 def kimad_debug_exact_path_layers(ctx: Ctx, detail: bool = False):
     """Layers handed to the exact radix path so far; with detail also the count per reason
-    (forced, bands too wide, threshold outside band, bound too loose)."""
-    n = (C.c_uint64 * (5 + ctx.K))()
+    (forced, bands too wide, threshold outside band, bound too loose even after refinement), the number of
+    layers refined, and per candidate how often its first bound was loose."""
+    n = (C.c_uint64 * (6 + ctx.K))()
     _check(load().kimad_debug_exact_path_layers(ctx.handle, n), "kimad_debug_exact_path_layers")
     return [int(x) for x in n] if detail else int(n[0])
 

@@ -27,7 +27,7 @@ struct Layout {
     size_t zero_from, h1_cnt, h1_ss, h23_cnt, h23_ss, bh_cnt, bh_sum, low_hist, recount, recount_bytes, fb, r2, flags;
     // scratch without initial-state requirements
     size_t cell_tab, cell_win, bin_lo, meta, cands, slots, err, tau, keep_eq, shift, sel, chunk_cnt, jobs, csel,
-        fb_chunks, fb_layers, r2_chunks, r2_layers, pd, total;
+        fb_chunks, fb_layers, r2_chunks, r2_layers, rf, rf_chunks, rf_layers, pd, total;
 };
 
 } // namespace
@@ -131,6 +131,9 @@ void plan_layout(kimad_ctx* c) {
     y.fb_layers = take(kGroups * align_up(WL * sizeof(uint2)));
     y.r2_chunks = take(kGroups * align_up((size_t)c->W * nch * sizeof(uint2)));
     y.r2_layers = take(kGroups * align_up(WL * sizeof(uint2)));
+    y.rf = take(WLK * sizeof(RefineCand));
+    y.rf_chunks = take(kGroups * align_up((size_t)c->W * nch * sizeof(uint2)));
+    y.rf_layers = take(kGroups * align_up(WL * sizeof(uint2)));
     y.pd = take(c->dp_plan.pd_in_smem ? 0 : (size_t)c->W * c->L * c->dp_plan.pd_row_bytes);
     y.total = o;
 }
@@ -360,6 +363,9 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
         uint2* fb_chunks = c->at<uint2>(y.fb_chunks + g * align_up((size_t)W * nch * sizeof(uint2)));
         uint2* r2_chunks = c->at<uint2>(y.r2_chunks + g * align_up((size_t)W * nch * sizeof(uint2)));
         uint2* fb_layers = c->at<uint2>(y.fb_layers + g * align_up((size_t)W * L * sizeof(uint2)));
+        RefineCand* rf = c->at<RefineCand>(y.rf);
+        uint2* rf_chunks = c->at<uint2>(y.rf_chunks + g * align_up((size_t)W * nch * sizeof(uint2)));
+        uint2* rf_layers = c->at<uint2>(y.rf_layers + g * align_up((size_t)W * L * sizeof(uint2)));
         uint2* r2_layers = c->at<uint2>(y.r2_layers + g * align_up((size_t)W * L * sizeof(uint2)));
         const dim3 gch(nch, nw), glw(L, nw);
         // the group's runs of the sweep: the run table is sorted by worker
@@ -379,7 +385,7 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
         CUDA_TRY(hand_over(big, small));
         if (R) {
             CUDA_TRY(launch_pdl(k_resolve_a, dim3(R, nw), kBigThreads, 0, small, layers, reg_layers, R, L, ktab, K, meta, binlo, bhc, bhs,
-                                err, tau, keq, shf, flags, fb, fb_chunks, fb_layers, list_cap, w0));
+                                err, tau, keq, shf, flags, fb, fb_chunks, fb_layers, rf, rf_chunks, rf_layers, list_cap, w0));
             c->launches += 1;
         }
         mark(small);
@@ -389,6 +395,11 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
             // histogram kernels get four CTAs per SM, enough to stream a large handed-over layer
             const uint32_t gfb = 4 * 148, glay = std::min<uint32_t>(nw * R, 32u);
             const dim3 gslot(glay, 1, K);
+            // candidates with a loose bound first (they may still end on the exact path's lists)
+            CUDA_TRY(launch_pdl(k_refine_hist, gfb, blk, 0, small, dbuf, chunks, c->dstride, L, K, fb, rf_chunks, rf,
+                                CodeSpace{reg_index, meta, cell_tab, cell_win, R}, h23c, h23s));
+            CUDA_TRY(launch_pdl(k_refine_resolve, glay, blk, 0, small, layers, L, K, fb, rf_layers, rf, h23c, h23s, err, tau, keq, shf,
+                                fb_chunks, fb_layers, list_cap));
             CUDA_TRY(launch_pdl(k_fb_hist1, gfb, blk, 0, small, dbuf, chunks, c->dstride, L, fb, fb_chunks, h1c, h1s, flags));
             CUDA_TRY(launch_pdl(k_resolve1, glay, blk, 0, small, fb, fb_layers, h1c, h1s, ktab, L, K, cands, slots));
             CUDA_TRY(launch_pdl(k_fb_hist23<2>, gfb, blk, 0, small, dbuf, chunks, c->dstride, L, K, fb, fb_chunks, slots, h23c, h23s));
@@ -396,7 +407,7 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
             CUDA_TRY(launch_pdl(k_rebuild_slots, (nw * R + kThreads - 1) / kThreads, blk, 0, small, fb, fb_layers, L, K, cands, slots));
             CUDA_TRY(launch_pdl(k_fb_hist23<3>, gfb, blk, 0, small, dbuf, chunks, c->dstride, L, K, fb, fb_chunks, slots, h23c, h23s));
             CUDA_TRY(launch_pdl(k_resolve23<3>, gslot, blk, 0, small, fb, fb_layers, h23c, h23s, L, K, cands, slots, err, tau, keq, shf));
-            c->launches += 7;
+            c->launches += 9;
         }
         mark(small);
         // (c)
@@ -800,13 +811,14 @@ int kimad_debug_exact_path_layers(kimad_ctx* c, uint64_t* host_count) {
     if (!c || !host_count) return KIMAD_ERR_INVALID_ARG;
     if (!c->ws) return KIMAD_ERR_WORKSPACE;
     CUDA_TRY(cudaDeviceSynchronize());
-    for (uint32_t i = 0; i < 5 + c->K; ++i) host_count[i] = 0;
+    for (uint32_t i = 0; i < 6 + c->K; ++i) host_count[i] = 0;
     for (int g = 0; g < kGroups; ++g) { // every group of workers keeps counters of its own
         FbList f{};
         CUDA_TRY(cudaMemcpy(&f, c->ws + c->lay.fb + g * align_up(sizeof(FbList)), sizeof(FbList), cudaMemcpyDeviceToHost));
         host_count[0] += f.total_layers;
         for (int i = 0; i < 4; ++i) host_count[1 + i] += f.why[i];
-        for (uint32_t j = 0; j < c->K; ++j) host_count[5 + j] += f.loose_j[j];
+        host_count[5] += f.refined;
+        for (uint32_t j = 0; j < c->K; ++j) host_count[6 + j] += f.loose_j[j];
     }
     return KIMAD_OK;
 }

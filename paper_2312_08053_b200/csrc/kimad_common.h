@@ -15,7 +15,8 @@
 // traps.  Bits: 0 sweep: bin outside the layer's histogram; 1 counting sweep: bin outside the in-interval histogram;
 // 2 a work list (exact path, second select round, recount) appended beyond its capacity; 3 write sweep: packed
 // position beyond the capacity; 4 write sweep: element index outside its layer; 5 DP: cell or back-pointer outside
-// its row; 6 curve: bin outside the layer's histogram.  In the ordinary build KIMAD_CHECK(cond, bit) is `true`.
+// its row; 6 curve: bin outside the layer's histogram; 7 curve: the pieces of a refined bin do not add up to the bin.
+// In the ordinary build KIMAD_CHECK(cond, bit) is `true`.
 #if defined(KIMAD_CHECKED) && defined(__CUDACC__)
 __device__ unsigned int g_kimad_check_word;
 #define KIMAD_CHECK(cond, bit) ((cond) ? true : (atomicOr(&g_kimad_check_word, 1u << (bit)), false))

@@ -19,6 +19,7 @@
 //   k_fb_*       exact three-digit radix select over the chunks of the layers handed over (rare).
 #pragma once
 #include "kimad_kernels.cuh"
+#include <type_traits>
 
 namespace kimad {
 
@@ -61,7 +62,8 @@ k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint6
     uint32_t* s_cb = s_w + 32;                    // [128] per candidate, then per merged group: lowest cell,
     uint32_t* s_ct = s_cb + 128;                  // [128] highest cell,
     uint32_t* s_cs = s_ct + 128;                  // [128] shift
-    __shared__ uint32_t s_m, s_flag, s_ng, s_cg;
+    __shared__ uint32_t s_m, s_flag, s_ng, s_cg, s_z;
+    __shared__ unsigned long long s_zz;
     const uint32_t r = blockIdx.x, w = blockIdx.y;
     const uint32_t l = reg_layers[r];
     const size_t wr = (size_t)w * R + r;
@@ -73,10 +75,11 @@ k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint6
     const LayerDesc ld = layers[l];
     const uint32_t n = (uint32_t)ld.n;
     for (int i = threadIdx.x; i < 32768; i += kBigThreads) h32[i] = 0;
-    if (threadIdx.x == 0) { s_m = 0; s_flag = 0; s_ng = 0; s_cg = 0; }
+    if (threadIdx.x == 0) { s_m = 0; s_flag = 0; s_ng = 0; s_cg = 0; s_z = 0; s_zz = 0ull; }
     __syncthreads();
 
-    // ---- stratified sample of |grad - g|
+    // ---- stratified sample of |grad - g|.  Exact zeros (the untouched rows of a sparse gradient) are counted apart:
+    // they sit below every other key, add nothing to any error, and the sweep leaves them out of its histogram.
     const float* gr = grads + (size_t)w * stride + ld.begin;
     const float* st = state + (size_t)w * stride + ld.begin;
     const uint32_t n_units = n / kSampleUnit + ((n % kSampleUnit) != 0); // n may be as large as 2^32 - 1
@@ -104,16 +107,27 @@ k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint6
             b[u] = ok[u] ? st[p] : 0.f;
         }
 #pragma unroll
-        for (int u = 0; u < 8; ++u)
+        for (int u = 0; u < 8; ++u) {
+            const uint32_t key = ok[u] ? key_of(__fsub_rn(a[u], b[u])) : 1u;
+            const uint32_t zu = __popc(__ballot_sync(0xffffffffu, key == 0u)); // the unit's exact zeros
+            if (zu && (threadIdx.x & 31) == 0) { atomicAdd(&s_z, zu); atomicAdd(&s_zz, (unsigned long long)(zu * zu)); }
             if (ok[u]) {
-                const uint32_t cell = key_of(__fsub_rn(a[u], b[u])) >> 15;
-                atomicAdd(&h32[cell >> 1], 1u << (16 * (cell & 1)));
+                if (key) atomicAdd(&h32[key >> 16], 1u << (16 * ((key >> 15) & 1)));
                 ++mine;
             }
+        }
     }
     atomicAdd(&s_m, mine);
     __syncthreads();
+    // fewer zeros than 1/64 of the sample are treated like any other key (cell 0)
     const uint32_t m = s_m;
+    const uint32_t z = s_z * 64u >= m ? s_z : 0u, mz = m - z; // sample size, its zero mass, the rest
+    if (threadIdx.x == 0 && z == 0 && s_z) h32[0] += s_z;
+    __syncthreads();
+    // variance of the sample's zero count from the spread of the units' zero counts: zeros that come in runs (whole
+    // rows) make the sample's share of zeros, and with it the sample rank of every threshold among the other keys,
+    // far less certain than independent draws would
+    const double var_z = z ? fmax(0.0, (double)s_zz - (double)z * (double)z / (double)m_units) : 0.0;
     auto cell_count = [&](uint32_t cell) { return (h32[cell >> 1] >> (16 * (cell & 1))) & 0xffffu; };
     auto cell_sq = [&](uint32_t cell) { // square of the cell's middle value (planning only: float range is enough)
         const float v = __uint_as_float((cell << 15) | 0x4000u);
@@ -173,18 +187,30 @@ k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint6
                 r_lo = r_hi = (uint32_t)k;
             } else {
                 const double p = (double)k / (double)n;
-                const double rho = p * (double)m, sg = sqrt((double)m * p * (1.0 - p));
+                const double rho = p * (double)m, rel = mz ? rho / (double)mz : 0.0;
+                const double sg = sqrt((double)m * p * (1.0 - p) + rel * rel * var_z);
                 const double a = floor(rho - 6.0 * sg - 2.0), b = ceil(rho + 6.0 * sg + 2.0);
                 r_lo = a < 1.0 ? 0u : (uint32_t)a;
                 r_hi = b > (double)m ? 0u : (uint32_t)b;
+            }
+            // a rank window wholly among the zeros: the threshold is 0 unless the sample misleads, no band (the curve
+            // stage knows the exact number of zeros); a window that reaches into the zeros ends at the lowest cell
+            // the sample saw, a quarter octave further down
+            const bool zero_cand = z && (mz == 0 || r_lo > mz);
+            const bool clip_bot = z && !zero_cand && (r_hi == 0 || r_hi > mz);
+            if (zero_cand) {
+                if (lane == 0) { s_cb[j] = o_cb; s_ct[j] = o_ct; s_cs[j] = o_cs; }
+                continue;
             }
             // rank window clipped at the top: the threshold may lie above the largest sample, so the band goes a
             // quarter octave further up; clipped at the bottom: no bound from the sample, exact path
             // bands stay among the finite keys (a sample with non-finite values is reported by the curve stage)
             uint32_t c_top = min(cell_of_rank(max(r_lo, 1u)), 65279u);
             if (r_lo == 0) c_top = min(c_top + 64u, 65279u);
-            if (r_hi == 0 && lane == 0) s_flag = 1;
-            const uint32_t c_bot = min(cell_of_rank(max(r_hi, 1u)), c_top);
+            if (r_hi == 0 && !z && lane == 0) s_flag = 1;
+            uint32_t c_bot = cell_of_rank(clip_bot ? mz : max(r_hi, 1u));
+            if (clip_bot) c_bot = c_bot > 64u ? c_bot - 64u : 0u;
+            c_bot = min(c_bot, c_top);
             const uint32_t ncell = c_top - c_bot + 1;
             if (ncell > (uint32_t)kFineBins) {
                 if (lane == 0) s_flag = 2;
@@ -360,7 +386,7 @@ k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint6
         blo[tot_bins] = 0x80000000u;
         uint32_t ls = 0; // bins per code of the byte plane: the codes stay below 128
         while (((tot_bins - 1) >> ls) > 127u) ++ls;
-        cell_win[wr] = make_int4((int)wlo - 1, (int)whi + 1, (int)(15 + cg), (int)ls);
+        cell_win[wr] = make_int4((int)wlo - 1, (int)whi + 1, (int)(15 + cg), (int)(ls | (z ? 256u : 0u))); // bit 8: zeros are left out
         *mt = BandMeta{tot_bins, used, 0, ng + 2};
     }
 }
@@ -394,16 +420,20 @@ k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, uint8
     const float* st0 = state + (size_t)run.w * stride;
     uint8_t* dc0 = d_code + (size_t)run.w * dstride;
     int cur_layer = -1;
-    uint32_t wr = 0xffffffffu; // slot of the current layer's histogram; 0xffffffff: none (tiny or handed-over layer)
+    // slot of the current layer's histogram; 0xffffffff: none (tiny or handed-over layer); bit 30 (kSkipZeros): the
+    // layer's exact zeros are left out of the histogram
+    constexpr uint32_t kSkipZeros = 0x40000000u;
+    uint32_t wr = 0xffffffffu;
     bool dirty = false;
     int wlo_m1 = 0, whi_p1 = 0;  // cells of the table's first and last entry, in units of 2^(cshift - 15) cells
     uint32_t cshift = 15, lshift = 0; // keys per table entry, bins per code (log2)
 
     auto flush = [&]() {
         __syncthreads();
-        const uint32_t n_bins = meta[wr].n_bins;
-        uint32_t* gc = bh_cnt + (size_t)wr * kMaxBins;
-        unsigned long long* gs = bh_sum + (size_t)wr * kMaxBins;
+        const uint32_t slot = wr & ~kSkipZeros;
+        const uint32_t n_bins = meta[slot].n_bins;
+        uint32_t* gc = bh_cnt + (size_t)slot * kMaxBins;
+        unsigned long long* gs = bh_sum + (size_t)slot * kMaxBins;
         for (uint32_t i = threadIdx.x; i < n_bins; i += kBigThreads) {
             const uint32_t c = h_cnt[i];
             if (c) {
@@ -424,29 +454,37 @@ k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, uint8
         // returned old value tells when, and a wrap adds 2^32 to the layer's 64-bit sum in global memory
         const uint32_t sq = (uint32_t)(sq_fixed(key) >> 8);
 #ifdef KIMAD_CHECKED
-        if (!KIMAD_CHECK(id < meta[wr].n_bins, 0)) return;
+        if (!KIMAD_CHECK(id < meta[wr & ~kSkipZeros].n_bins, 0)) return;
 #endif
         atomicAdd(&h_cnt[id], 1u);
         const uint32_t old = atomicAdd(&h_lo[id], sq);
-        if (old + sq < old) atomicAdd(bh_sum + (size_t)wr * kMaxBins + id, 1ull << 32); // rare
+        if (old + sq < old) atomicAdd(bh_sum + (size_t)(wr & ~kSkipZeros) * kMaxBins + id, 1ull << 32); // rare
     };
     // one element: its bin's count and sum; returns its code
     auto acc = [&](uint32_t key) -> uint32_t {
         const uint32_t id = bin_of(key, look(key));
-        add(id, key);
+        if (key || !(wr & kSkipZeros)) add(id, key);
         return id >> lshift;
     };
     // The four elements of a quad go through the stages together (all table reads, then the bin ids, then the
     // atomics): four independent chains of dependent shared-memory accesses instead of one after the other.
     // Returns the quad's four codes.
-    auto acc4 = [&](const uint32_t (&k)[4]) -> uint32_t {
+    // Where the sample found a mass of exact zeros (the untouched rows of a sparse gradient), zeros are left out:
+    // they add nothing to any sum, they would all hit one word, and the curve stage takes their number from the
+    // layer's size.
+    auto acc4 = [&](const uint32_t (&k)[4], auto skip) -> uint32_t {
         uint32_t e[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) e[i] = look(k[i]);
 #pragma unroll
         for (int i = 0; i < 4; ++i) e[i] = bin_of(k[i], e[i]);
+        if (decltype(skip)::value) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) add(e[i], k[i]);
+            for (int i = 0; i < 4; ++i) if (k[i]) add(e[i], k[i]);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) add(e[i], k[i]);
+        }
         return pack_low_bytes(e[0] >> lshift, e[1] >> lshift, e[2] >> lshift, e[3] >> lshift);
     };
 
@@ -475,10 +513,11 @@ k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, uint8
             if (r != 0xffffffffu && !meta[run.w * R + r].flagged) {
                 wr = run.w * R + r;
                 const int4 win = cell_win[wr];
-                wlo_m1 = win.x; whi_p1 = win.y; cshift = (uint32_t)win.z; lshift = (uint32_t)win.w;
+                wlo_m1 = win.x; whi_p1 = win.y; cshift = (uint32_t)win.z; lshift = (uint32_t)win.w & 31u;
                 const uint32_t* g2 = cell_tab + (size_t)wr * kCellTab;
                 const uint32_t used = meta[wr].n_cells;
                 for (uint32_t i = threadIdx.x; i < used; i += kBigThreads) tab[i] = g2[i];
+                if ((uint32_t)win.w & 256u) wr |= kSkipZeros;
             }
             __syncthreads();
         }
@@ -495,21 +534,27 @@ k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, uint8
             auto fetch = [&](float4& a, float4& b, uint32_t q) {
                 if (q < q_hi) { a = __ldcg(gr4 + q); b = __ldcg(st4 + q); }
             };
-            auto work = [&](const float4& a, const float4& b, uint32_t q) {
+            auto work = [&](const float4& a, const float4& b, uint32_t q, auto skip) {
                 const uint32_t k[4] = {key_of(__fsub_rn(a.x, b.x)), key_of(__fsub_rn(a.y, b.y)),
                                        key_of(__fsub_rn(a.z, b.z)), key_of(__fsub_rn(a.w, b.w))};
-                reinterpret_cast<uint32_t*>(dc)[q] = active ? acc4(k) : pack_key_codes(k[0], k[1], k[2], k[3]);
+                reinterpret_cast<uint32_t*>(dc)[q] = active ? acc4(k, skip) : pack_key_codes(k[0], k[1], k[2], k[3]);
             };
             float4 a0, b0, a1, b1, a2, b2, a3, b3;
             uint32_t qb = q_lo + threadIdx.x;
             constexpr uint32_t S = kBigThreads;
             fetch(a0, b0, qb); fetch(a1, b1, qb + S); fetch(a2, b2, qb + 2 * S);
-            while (qb < q_hi) {
-                fetch(a3, b3, qb + 3 * S); work(a0, b0, qb); qb += S; if (qb >= q_hi) break;
-                fetch(a0, b0, qb + 3 * S); work(a1, b1, qb); qb += S; if (qb >= q_hi) break;
-                fetch(a1, b1, qb + 3 * S); work(a2, b2, qb); qb += S; if (qb >= q_hi) break;
-                fetch(a2, b2, qb + 3 * S); work(a3, b3, qb); qb += S;
-            }
+            // four rounds; false when the span ends inside them.  Two forms (with and without the exact zeros), chosen
+            // once per four rounds
+            auto rounds = [&](auto skip) -> bool {
+                fetch(a3, b3, qb + 3 * S); work(a0, b0, qb, skip); qb += S; if (qb >= q_hi) return false;
+                fetch(a0, b0, qb + 3 * S); work(a1, b1, qb, skip); qb += S; if (qb >= q_hi) return false;
+                fetch(a1, b1, qb + 3 * S); work(a2, b2, qb, skip); qb += S; if (qb >= q_hi) return false;
+                fetch(a2, b2, qb + 3 * S); work(a3, b3, qb, skip); qb += S;
+                return true;
+            };
+            const bool zs = active && (wr & kSkipZeros);
+            while (qb < q_hi)
+                if (!(zs ? rounds(std::true_type{}) : rounds(std::false_type{}))) break;
             if (threadIdx.x < 8) { // ragged edges: [first, min(4 q_lo, len)) and [max(4 q_hi, 4 q_lo), len)
                 uint32_t e;
                 if (threadIdx.x < 4) { e = cv.first + threadIdx.x; if (e >= min(4 * q_lo, cv.len)) e = 0xffffffffu; }
@@ -539,9 +584,11 @@ k_resolve_a(const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ r
             const uint32_t* __restrict__ bin_lo, uint32_t* __restrict__ bh_cnt, unsigned long long* __restrict__ bh_sum,
             float* __restrict__ err_out, uint32_t* __restrict__ tau_out, uint32_t* __restrict__ rank_out,
             uint32_t* __restrict__ shift_out, uint32_t* __restrict__ flags, FbList* __restrict__ fb,
-            uint2* __restrict__ fb_chunks, uint2* __restrict__ fb_layers, uint32_t list_cap, uint32_t w_base) {
+            uint2* __restrict__ fb_chunks, uint2* __restrict__ fb_layers, RefineCand* __restrict__ rf,
+            uint2* __restrict__ rf_chunks, uint2* __restrict__ rf_layers, uint32_t list_cap, uint32_t w_base) {
     pdl_wait();
     __shared__ uint32_t s_drop[KIMAD_MAX_RATIOS]; // entries not kept by candidate j: n - k_j
+    __shared__ int s_loose;
     __shared__ uint32_t s_bin[KIMAD_MAX_RATIOS], s_before[KIMAD_MAX_RATIOS], s_cb[KIMAD_MAX_RATIOS];
     __shared__ double s_below[KIMAD_MAX_RATIOS], s_sb[KIMAD_MAX_RATIOS];
     __shared__ uint32_t s_w32[32];
@@ -552,7 +599,7 @@ k_resolve_a(const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ r
     const size_t wr = (size_t)w * R + r, wl = (size_t)w * L + l;
     const BandMeta mt = meta[wr];
     const LayerDesc ld = layers[l];
-    if (threadIdx.x == 0) s_bad = mt.flagged;
+    if (threadIdx.x == 0) { s_bad = mt.flagged; s_loose = 0; }
     if (threadIdx.x < K) {
         const uint64_t k = ktab.at(w, (size_t)l * K + threadIdx.x);
         s_drop[threadIdx.x] = (uint32_t)(ld.n - k);
@@ -583,9 +630,16 @@ k_resolve_a(const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ r
         }
         if (lane == 0) { s_w32[wid] = c_tot; s_w64[wid] = s_tot; }
         __syncthreads();
-        uint32_t run_c = 0;  // entries in the bins below this warp's range
-        double run_s = 0.0;  // their squares
+        uint32_t counted = 0;
+        for (uint32_t i = 0; i < kBigThreads / 32; ++i) counted += s_w32[i];
+        const uint32_t zeros = (uint32_t)ld.n - counted; // the sweep leaves exact zeros out of its histogram
+        uint32_t run_c = zeros; // entries below this warp's range: the zeros and the bins of the warps before
+        double run_s = 0.0;     // their squares
         for (uint32_t i = 0; i < wid; ++i) { run_c += s_w32[i]; run_s += s_w64[i]; }
+        if (threadIdx.x < K && s_drop[threadIdx.x] < zeros) { // the threshold is 0: every other key is kept
+            s_bin[threadIdx.x] = 0xfffffffeu;
+            s_cb[threadIdx.x] = zeros - s_drop[threadIdx.x]; // zeros kept
+        }
         bool nonfinite = false;
         for (uint32_t base = r0; base < r1; base += 32) {
             const uint32_t b = base + lane;
@@ -623,11 +677,16 @@ k_resolve_a(const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ r
         __syncthreads();
         for (uint32_t j = threadIdx.x; j < K; j += kBigThreads) {
             const size_t o = wl * K + j;
+            rf[o].shift = kNoRefine;
             if (s_drop[j] == 0) { // everything kept
                 err_out[o] = 0.f; tau_out[o] = 0; rank_out[o] = 0; shift_out[o] = 0;
                 continue;
             }
             const uint32_t bin = s_bin[j];
+            if (bin == 0xfffffffeu) { // exactly: nothing but zeros is dropped
+                err_out[o] = 0.f; tau_out[o] = 0; rank_out[o] = s_cb[j]; shift_out[o] = 0;
+                continue;
+            }
             if (bin == 0xffffffffu || (blo[bin] & kGapBit)) { atomicMax(&s_bad, 3); continue; } // outside its band
             const uint32_t klo = blo[bin], width = (blo[bin + 1] & ~kGapBit) - klo;
             const uint32_t cb = s_cb[j];
@@ -640,7 +699,13 @@ k_resolve_a(const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ r
             double part = 0.5 * (upper + lower), slack = 0.5 * (upper - lower);
             if (drop == 0 || width == 1) { part = lower; slack = 0.0; }
             const double e = s_below[j] + part;
-            if (slack > e * 5e-6) { atomicMax(&s_bad, 4); atomicAdd(&fb->loose_j[j], 1u); continue; } // acceptance bound on the curve is 1e-5
+            if (slack > e * 5e-6) { // acceptance bound on the curve is 1e-5: this candidate's bin is looked at once more
+                if (klo == 0u && zeros) { atomicMax(&s_bad, 4); continue; } // (not a bin whose zeros were left out)
+                s_loose = 1;
+                atomicAdd(&fb->loose_j[j], 1u);
+                rf[o] = RefineCand{klo, (uint32_t)(31 - __clz(width)), cb, drop, s_below[j]};
+                continue;
+            }
             err_out[o] = (float)e;
             tau_out[o] = klo;
             rank_out[o] = cb - drop;
@@ -649,8 +714,8 @@ k_resolve_a(const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ r
     }
     __syncthreads();
     const int bad = s_bad;
+    __shared__ uint32_t s_at;
     if (bad) { // hand the layer and its chunks to the exact path
-        __shared__ uint32_t s_at;
         if (threadIdx.x == 0) {
             s_at = atomicAdd(&fb->n_chunks, ld.n_chunks);
             fb_layers[atomicAdd(&fb->n_layers, 1u)] = make_uint2(w, l);
@@ -660,6 +725,183 @@ k_resolve_a(const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ r
         __syncthreads();
         for (uint32_t i = threadIdx.x; i < ld.n_chunks; i += kBigThreads)
             if (KIMAD_CHECK(s_at + i < list_cap, 2)) fb_chunks[s_at + i] = make_uint2(w, ld.first_chunk + i);
+    } else if (s_loose) { // only loose bounds: refine those candidates
+        if (threadIdx.x == 0) {
+            s_at = atomicAdd(&fb->rf_chunks, ld.n_chunks);
+            rf_layers[atomicAdd(&fb->rf_layers, 1u)] = make_uint2(w, l);
+            atomicAdd(&fb->refined, 1u);
+        }
+        __syncthreads();
+        for (uint32_t i = threadIdx.x; i < ld.n_chunks; i += kBigThreads)
+            if (KIMAD_CHECK(s_at + i < list_cap, 2)) rf_chunks[s_at + i] = make_uint2(w, ld.first_chunk + i);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Refinement of loose candidates: the bin that holds such a candidate's threshold is cut into up to 1024 pieces, and
+// the entries of the bin -- found by their code byte, completed from the inputs -- are counted and their squares
+// summed per piece (the level-2/3 arrays of the exact path serve as storage: a layer is never on both paths at once).
+// Costs one pass over the layer's code bytes instead of the exact path's three passes over its inputs.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads)
+k_refine_hist(DSource dbuf, const Chunk* __restrict__ chunks, uint64_t dstride, uint32_t L, uint32_t K,
+              const FbList* __restrict__ fb, const uint2* __restrict__ rf_chunks, const RefineCand* __restrict__ rf,
+              const CodeSpace codes, uint32_t* __restrict__ g_cnt, unsigned long long* __restrict__ g_ss) {
+    pdl_wait();
+    __shared__ uint32_t s_klo[KIMAD_MAX_RATIOS], s_shift[KIMAD_MAX_RATIOS], s_j[KIMAD_MAX_RATIOS];
+    __shared__ uint32_t s_mask[4]; // the 7-bit codes of the loose candidates' bins
+    __shared__ uint32_t s_n;
+    const uint32_t n = fb->rf_chunks;
+    for (uint32_t it = blockIdx.x; it < n; it += gridDim.x) {
+        const uint2 e = rf_chunks[it];
+        const Chunk ch = chunks[e.y];
+        const size_t wl = (size_t)e.x * L + ch.layer;
+        __syncthreads();
+        if (threadIdx.x < 4) s_mask[threadIdx.x] = 0;
+        if (threadIdx.x == 0) s_n = 0;
+        __syncthreads();
+        if (threadIdx.x == 0) { // the layer's loose candidates in order of j, every bin once (under its lowest j)
+            uint32_t p = 0;
+            for (uint32_t j = 0; j < K; ++j) {
+                const RefineCand rc = rf[wl * K + j];
+                if (rc.shift == kNoRefine || (p && s_klo[p - 1] == rc.klo)) continue; // thresholds descend with j
+                s_klo[p] = rc.klo; s_shift[p] = rc.shift; s_j[p] = j;
+                ++p;
+                const uint32_t code = codes.code(e.x, ch.layer, rc.klo) & 127u;
+                s_mask[code >> 5] |= 1u << (code & 31u);
+            }
+            s_n = p;
+        }
+        __syncthreads();
+        const uint32_t nc = s_n;
+        const uint32_t m0 = s_mask[0], m1 = s_mask[1], m2 = s_mask[2], m3 = s_mask[3];
+        const ChunkView cv(ch);
+        const DView dd(dbuf, e.x, dstride, cv.a0);
+        auto wanted = [&](uint32_t code) -> bool {
+            const uint32_t word = code < 64u ? (code < 32u ? m0 : m1) : (code < 96u ? m2 : m3);
+            return (word >> (code & 31u)) & 1u;
+        };
+        auto visit = [&](uint32_t x) {
+            const uint32_t key = key_of(dd.at(x));
+            for (uint32_t p = 0; p < nc; ++p) {
+                const uint32_t d1 = key - s_klo[p], sh = s_shift[p];
+                if (d1 < (1u << sh)) {
+                    const size_t at = (wl * K + s_j[p]) * kL23Bins + (d1 >> (sh > 10u ? sh - 10u : 0u));
+                    atomicAdd(&g_cnt[at], 1u);
+                    atomicAdd(&g_ss[at], (unsigned long long)sq_fixed(key));
+                    break; // bins are disjoint; candidates that share a bin share a piece histogram (see k_refine_resolve)
+                }
+            }
+        };
+        const uint32_t units = (cv.len + 15u) >> 4;
+        for (uint32_t u = threadIdx.x; u < units; u += kThreads) {
+            const uint32_t e0 = 16u * u;
+            if (e0 >= cv.first && e0 + 16u <= cv.len) {
+                const uint4 a = __ldcs(reinterpret_cast<const uint4*>(dd.code) + u);
+                const uint32_t x[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                    for (int b = 0; b < 4; ++b)
+                        if (wanted((x[i] >> (8 * b)) & 127u)) visit(e0 + 4 * i + b);
+            } else {
+                for (uint32_t x = max(e0, cv.first); x < min(e0 + 16u, cv.len); ++x)
+                    if (wanted(dd.code[x] & 127u)) visit(x);
+            }
+        }
+    }
+}
+
+// One CTA per refined layer and pass of the loop; its loose candidates one after the other.  Candidates that share a
+// bin were counted into the histogram of the first of them (the lowest j): the later ones read it there.
+__global__ void __launch_bounds__(kThreads)
+k_refine_resolve(const LayerDesc* __restrict__ layers, uint32_t L, uint32_t K, FbList* __restrict__ fb,
+                 const uint2* __restrict__ rf_layers, RefineCand* __restrict__ rf, uint32_t* __restrict__ g_cnt,
+                 unsigned long long* __restrict__ g_ss, float* __restrict__ err_out, uint32_t* __restrict__ tau_out,
+                 uint32_t* __restrict__ rank_out, uint32_t* __restrict__ shift_out, uint2* __restrict__ fb_chunks,
+                 uint2* __restrict__ fb_layers, uint32_t list_cap) {
+    pdl_wait();
+    __shared__ uint32_t s_w32[8];
+    __shared__ double s_w64[8];
+    __shared__ int s_bad;
+    __shared__ uint32_t s_at;
+    const uint32_t n = fb->rf_layers;
+    for (uint32_t it = blockIdx.x; it < n; it += gridDim.x) {
+        const uint32_t w = rf_layers[it].x, l = rf_layers[it].y;
+        const size_t wl = (size_t)w * L + l;
+        __syncthreads();
+        if (threadIdx.x == 0) s_bad = 0;
+        __syncthreads();
+        for (uint32_t j = 0; j < K; ++j) {
+            const RefineCand rc = rf[wl * K + j];
+            if (rc.shift == kNoRefine) continue;
+            uint32_t owner = j; // the first loose candidate with this bin holds the pieces
+            for (uint32_t i = 0; i < j; ++i) {
+                const RefineCand o = rf[wl * K + i];
+                if (o.shift != kNoRefine && o.klo == rc.klo) { owner = i; break; }
+            }
+            const uint32_t sub = rc.shift > 10u ? rc.shift - 10u : 0u, nsub = 1u << (rc.shift - sub);
+            const uint32_t* gc = g_cnt + (wl * K + owner) * kL23Bins;
+            const unsigned long long* gs = g_ss + (wl * K + owner) * kL23Bins;
+            const double scale = sq_scale(rc.klo >> 23);
+            // four consecutive pieces per thread, ascending keys
+            uint32_t c[4], csum = 0;
+            double q[4], qsum = 0.0;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint32_t b = 4 * threadIdx.x + i;
+                c[i] = b < nsub ? gc[b] : 0u;
+                q[i] = b < nsub ? (double)gs[b] * scale : 0.0;
+                csum += c[i];
+                qsum += q[i];
+            }
+            uint32_t tot;
+            uint32_t before = block_excl_scan<uint32_t>(csum, s_w32, &tot);
+            double below = block_excl_scan<double>(qsum, s_w64, nullptr);
+            if (!KIMAD_CHECK(tot == rc.cb, 7)) s_bad = 1;
+            const size_t o = wl * K + j;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                if (c[i] && rc.drop >= before && rc.drop - before < c[i]) { // the piece that holds the threshold
+                    const uint32_t b = 4 * threadIdx.x + i, klo = rc.klo + (b << sub), d2 = rc.drop - before;
+                    const double vlo = (double)__uint_as_float(klo);
+                    const double upper = q[i] * ((double)d2 / (double)c[i]), lower = (double)d2 * vlo * vlo;
+                    double part = 0.5 * (upper + lower), slack = 0.5 * (upper - lower);
+                    if (d2 == 0 || sub == 0) { part = lower; slack = 0.0; }
+                    const double e = rc.below + below + part;
+                    if (slack > e * 5e-6) {
+                        s_bad = 1;
+                    } else {
+                        err_out[o] = (float)e; tau_out[o] = klo; rank_out[o] = c[i] - d2; shift_out[o] = sub;
+                    }
+                }
+                before += c[i];
+                below += q[i];
+            }
+            __syncthreads();
+        }
+        // clean the pieces, close the candidates
+        for (uint32_t j = 0; j < K; ++j) {
+            if (rf[wl * K + j].shift == kNoRefine) continue;
+            for (uint32_t b = threadIdx.x; b < (uint32_t)kL23Bins; b += kThreads) {
+                g_cnt[(wl * K + j) * kL23Bins + b] = 0;
+                g_ss[(wl * K + j) * kL23Bins + b] = 0ull;
+            }
+        }
+        __syncthreads();
+        for (uint32_t j = threadIdx.x; j < K; j += kThreads) rf[wl * K + j].shift = kNoRefine;
+        if (s_bad) { // still too loose (a bin with very many entries): the exact path after all
+            const LayerDesc ld = layers[l];
+            if (threadIdx.x == 0) {
+                s_at = atomicAdd(&fb->n_chunks, ld.n_chunks);
+                fb_layers[atomicAdd(&fb->n_layers, 1u)] = make_uint2(w, l);
+                atomicAdd(&fb->total_layers, 1u);
+                atomicAdd(&fb->why[3], 1u);
+            }
+            __syncthreads();
+            for (uint32_t i = threadIdx.x; i < ld.n_chunks; i += kThreads)
+                if (KIMAD_CHECK(s_at + i < list_cap, 2)) fb_chunks[s_at + i] = make_uint2(w, ld.first_chunk + i);
+        }
     }
 }
 

@@ -197,7 +197,20 @@ struct FbList { // layers handed to the exact radix path in this step, and their
     uint32_t why[5];       // never reset: ... because 0: forced, 1: bands too wide for the tables, 2: threshold
                            // outside its band, 3: error bound too loose
     uint32_t loose_j[KIMAD_MAX_RATIOS + 1]; // never reset: which candidate's bound was too loose
+    // layers whose only defect is a loose bound are refined instead: one more look at the entries of the bins that
+    // hold the loose candidates' thresholds (k_refine_hist, k_refine_resolve)
+    uint32_t rf_chunks;
+    uint32_t rf_layers;
+    uint32_t refined; // never reset: layers that took the refinement
 };
+// A candidate of a refined layer: its threshold lies in the bin [klo, klo + 2^shift), which holds cb entries of which
+// the `drop` smallest are not kept; `below` = the squares of everything below the bin.  shift = kNoRefine: this
+// candidate's curve entry is final.
+struct RefineCand {
+    uint32_t klo, shift, cb, drop;
+    double below;
+};
+constexpr uint32_t kNoRefine = 0xffffffffu;
 
 __global__ void __launch_bounds__(kThreads)
 k_resolve1(const FbList* __restrict__ fb, const uint2* __restrict__ fb_layers, uint32_t* __restrict__ g_cnt,
@@ -364,7 +377,7 @@ struct BandMeta {
 };
 // entry of the cell table: base << 5 | shift (base signed): the bin of a key is base + (key >> shift).
 // window of a layer: {cell of the first entry, cell of the last entry, log2 of the keys per entry, log2 of the bins
-// per code of the byte plane}
+// per code of the byte plane (bits 0..4) | 256 when the sweep leaves the layer's exact zeros out of its histogram}
 struct CodeSpace { // how the sweep coded the elements of one (worker, layer)
     const uint32_t* reg_index; // [L], 0xffffffff: tiny layer
     const BandMeta* meta;      // [W][R]
@@ -379,7 +392,7 @@ struct CodeSpace { // how the sweep coded the elements of one (worker, layer)
         if (meta[wr].flagged) return key >> 24;
         const int4 win = cell_win[wr];
         const uint32_t e = cell_tab[wr * kCellTab + (size_t)(min(max((int)(key >> win.z), win.x), win.y) - win.x)];
-        return (uint32_t)(((int)e >> 5) + (int)(key >> (e & 31u))) >> win.w;
+        return (uint32_t)(((int)e >> 5) + (int)(key >> (e & 31u))) >> (win.w & 31);
     }
 };
 

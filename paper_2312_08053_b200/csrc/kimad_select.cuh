@@ -82,6 +82,7 @@ __device__ __forceinline__ void sel_count_chunk(const DSource& dbuf, const Chunk
     }
     const uint32_t lo = s.tau, width = 1u << s.shift;
     const uint32_t hshift = s.shift > 10 ? s.shift - 10 : 0; // the histogram has at most kLowBins bins
+    const bool exact = s.shift == 0;
     if (threadIdx.x == 0) *s_n = 0;
     uint32_t* gh = low_hist + wl * kLowBins; // the layer's in-interval histogram: few entries, counted in place
     __syncthreads();
@@ -92,14 +93,20 @@ __device__ __forceinline__ void sel_count_chunk(const DSource& dbuf, const Chunk
     // every byte of x + (0x80 - t) * 0x01010101.
     const uint32_t add_gt = (0x80u - (s.code + 1u)) * 0x01010101u, add_ge = (0x80u - s.code) * 0x01010101u;
     for (uint32_t sl = wid; sl < (uint32_t)kSlices; sl += kThreads / 32) {
-        uint32_t above = 0;
+        uint32_t above = 0; // low half: entries above the interval; high half: entries equal to an exact threshold
         uint64_t mask = 0;
         auto visit = [&](uint32_t key) -> bool { // true: the key is not below the interval
             const uint32_t d1 = key - lo; // wraps to >= 2^31 for keys below the interval
             if (d1 < width) {
-                if (KIMAD_CHECK((d1 >> hshift) < (uint32_t)kLowBins, 1)) atomicAdd(&gh[d1 >> hshift], 1u);
-                const uint32_t p = atomicAdd(s_n, 1u);
-                if (p < (uint32_t)kListCap) s_low[p] = (sl << 16) | d1;
+                // an exact threshold needs no list and no histogram, only the slice's number of equal entries (there
+                // may be millions of them: the exact zeros of a sparse gradient)
+                if (exact) {
+                    above += 0x10000u;
+                } else {
+                    if (KIMAD_CHECK((d1 >> hshift) < (uint32_t)kLowBins, 1)) atomicAdd(&gh[d1 >> hshift], 1u);
+                    const uint32_t p = atomicAdd(s_n, 1u);
+                    if (p < (uint32_t)kListCap) s_low[p] = (sl << 16) | d1;
+                }
             } else {
                 above += d1 < 0x80000000u;
             }
@@ -154,7 +161,7 @@ __device__ __forceinline__ void sel_count_chunk(const DSource& dbuf, const Chunk
         }
 #pragma unroll
         for (int o = 16; o; o >>= 1) above += __shfl_xor_sync(0xffffffffu, above, o);
-        if (lane == 0) { out->above[sl] = (uint16_t)above; out->eq[sl] = 0; out->mask[sl] = mask; }
+        if (lane == 0) { out->above[sl] = (uint16_t)above; out->eq[sl] = (uint16_t)(above >> 16); out->mask[sl] = mask; }
     }
     __syncthreads();
     const uint32_t n_in = *s_n;
@@ -431,6 +438,8 @@ k_sel_scan(const LayerDesc* __restrict__ layers, const Chunk* __restrict__ chunk
         *recount_n = 0;
         fb->n_chunks = 0;
         fb->n_layers = 0;
+        fb->rf_chunks = 0;
+        fb->rf_layers = 0;
         r2->n_chunks = 0;
         r2->n_layers = 0;
     }
