@@ -172,6 +172,7 @@ def _dtype_label(wl):
 
 
 SCHEDULE = 0  # kimad_debug_set_schedule of every context the bench creates (--schedule)
+ZERO_ROWS = 0.0  # fraction of exactly-zero rows in the token embedding's gradient (--zero-rows; workloads 4 and 5)
 
 
 def _time_steps(kb, torch, wl, dev, rank, steps, warmup, max_buf_bytes=70e9):
@@ -187,7 +188,7 @@ def _time_steps(kb, torch, wl, dev, rank, steps, warmup, max_buf_bytes=70e9):
     # fresh gradients for every step (as in training), as far as the device memory allowed for them goes; beyond
     # that the buffers are cycled.  Every rank draws its own streams (seed offset by rank).
     n_bufs = int(max(2, min(warmup + steps, max_buf_bytes // (W * N * 4))))
-    grads = [workloads.gradients(wl, 1000 * rank + s, device=dev) for s in range(n_bufs)]
+    grads = [workloads.gradients(wl, 1000 * rank + s, device=dev, zero_rows=ZERO_ROWS) for s in range(n_bufs)]
     state = torch.zeros((W, N), dtype=torch.float32, device=dev)
     stream = torch.cuda.current_stream()
 
@@ -364,7 +365,8 @@ def run_kimad(args, rank, world):
         "config": {"workload": wl.name, "cfg": wl.cfg, "workers_per_gpu": W, "layers": L, "elements_per_worker": N,
                    "ratios": len(wl.ratio_grid), "D": wl.D, "value_dtype": "bf16" if wl.value_dtype else "f32",
                    "l2": "inputs_larger_than_l2" if W * N * 4 > 200e6 else "inputs_fit_l2",
-                   "budget_trace": "cycled", "gradient_buffers": n_bufs, "parallelism": f"worker-sharded x{world}"},
+                   "budget_trace": "cycled", "gradient_buffers": n_bufs, "parallelism": f"worker-sharded x{world}",
+                   "zero_rows": ZERO_ROWS},
         "step_roofline": step_roofline,
         "e2e": e2e_out, "gpu_launches": int(launches),
         "roofline": roofline,
@@ -472,14 +474,20 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--schedule", type=int, default=0, choices=[0, 1, 2],
                     help="0: the library's choice (two worker groups for large steps), 1: always two groups, 2: one group")
+    ap.add_argument("--zero-rows", type=float, default=0.0,
+                    help="workloads 4 and 5: this fraction of the token embedding's gradient rows is exactly zero (a sparse "
+                         "gradient; not the headline workload: the line says so in config.zero_rows)")
     ap.add_argument("--timeline", default=None, metavar="FILE",
                     help="after the timed steps, run one step with events around every launch and write its timeline")
     ap.add_argument("--no-also", action="store_true", help="skip the second large workload's device-timed block")
     ap.add_argument("--path", default="compress", choices=["compress", "receive"],
                     help="compress: the worker-side pass (the headline); receive: apply + aggregate on the server")
     args = ap.parse_args()
-    global SCHEDULE
+    global SCHEDULE, ZERO_ROWS
     SCHEDULE = args.schedule
+    ZERO_ROWS = args.zero_rows
+    if ZERO_ROWS and args.config not in (4, 5):
+        ap.error("--zero-rows needs --config 4 or 5")
     args.warmup = max(args.warmup, 3) if args.impl == "kimad" else args.warmup
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))

@@ -7,14 +7,21 @@
 //                keys, everything else into coarse "gap" bins.  Every region (a gap, or a group of bands with
 //                one bin width) maps a key to its bin as base + (key >> shift); which region a key lies in is
 //                read from a table over the window of cells between the lowest and the highest band.
-//   k_pass_a     the sweep: d = grad - g (its upper 16 bits go to scratch), bin = base + (key >> shift) with
-//                (base, shift) = table(cell(key)), two u32 shared-memory atomics per element: the count, and the
-//                exact integer sum of squares in a u32 word whose (rare) carries go straight to the 64-bit sum in
-//                global memory.  CTAs own static runs of chunks balanced by elements.
-//   k_resolve_a  per (worker, layer): walks the bins from the top, finds the bin that holds every
-//                candidate's threshold, sums the squares below it.  The candidate's error is certified
-//                to 2^-19 relative from the bin's width; if a threshold fell into a gap bin (the sample
-//                mispredicted) or the bound is too loose, the layer is handed to the exact radix path.
+//                A mass of exact zeros in the sample (a sparse gradient) is counted apart: such a layer's zeros
+//                stay out of the sweep's histogram, candidates whose rank lies among them need no band, and
+//                sigma grows by what the spread of the zeros over the sampled units says about their clustering.
+//   k_pass_a     the sweep: d = grad - g (one code byte per element goes to scratch), bin = base + (key >> shift)
+//                with (base, shift) = table(cell(key)), two u32 shared-memory atomics per element: the count, and
+//                the exact integer sum of squares in a u32 word whose (rare) carries go straight to the 64-bit sum
+//                in global memory.  CTAs own static runs of chunks balanced by elements.
+//   k_resolve_a  per (worker, layer): walks the bins from the bottom (zeros left out by the sweep = the layer's
+//                size minus the counted entries), finds the bin that holds every candidate's threshold, sums the
+//                squares below it.  The candidate's error is certified to 5e-6 relative from the bin's width.  A
+//                threshold in a gap bin (the sample mispredicted) sends the layer to the exact radix path; a bound
+//                that is too loose sends the candidate to the refinement.
+//   k_refine_hist, k_refine_resolve
+//                loose candidates: the entries of the threshold's bin, found by their code byte, are counted in
+//                1024 pieces of the bin; error and interval from the pieces (still loose: exact path).
 //   k_tiny_exact layers of at most kTinyMax elements are sorted in shared memory instead.
 //   k_fb_*       exact three-digit radix select over the chunks of the layers handed over (rare).
 #pragma once

@@ -10,6 +10,8 @@
 //   k_resolve_a     (b) Eq. 4 / the "Errors" matrix of Algorithm 3: err_l(k_j) from the bins, certified to the
 //                   curve tolerance; layers that fail the certificate are handed to the exact path [kimad_curve.cuh]
 //   k_tiny_exact    (b) layers of at most 4096 elements, sorted in shared memory                 [kimad_curve.cuh]
+//   k_refine_hist, k_refine_resolve
+//                   (b) candidates whose certified bound is too loose: one more look at their bin (usually none)
 //   k_fb_hist1, k_fb_hist23<2|3>, k_resolve1, k_resolve23<2|3>, k_rebuild_slots
 //                   (b) exact 11+10+10-bit radix select over the handed-over layers (usually none)
 //                                                                          [kimad_curve.cuh, this file]

@@ -139,9 +139,14 @@ def workload(cfg: int, divisor: int = 1, n_workers: int | None = None) -> Worklo
 
 
 # ----------------------------------------------------------------------------- gradients
-def gradients(wl: Workload, step: int, device="cpu", workers=None, stride: int | None = None):
+EMBED_COLS = {4: 768, 5: 2048}  # row length of layer 0 (the token embedding) of the two language-model shapes
+
+
+def gradients(wl: Workload, step: int, device="cpu", workers=None, stride: int | None = None, zero_rows: float = 0.0):
     """float32 tensor [W][stride] of fresh gradients for ``step`` (seeded per (cfg, step, worker)).
-    Padding beyond N (when stride > N) is zero."""
+    Padding beyond N (when stride > N) is zero.  ``zero_rows`` > 0 (workloads 4 and 5, undivided): that fraction of the
+    rows of the token embedding's gradient, drawn per worker and step, is exactly zero -- the rows of the tokens
+    a batch does not contain."""
     import torch
 
     W = wl.n_workers
@@ -177,6 +182,10 @@ def gradients(wl: Workload, step: int, device="cpu", workers=None, stride: int |
             raise ValueError(wl.dist)
         out[row, :N] = x * scale_vec
         del x, z
+        if zero_rows > 0.0:
+            cols = EMBED_COLS[wl.cfg]
+            emb = out[row, :wl.layer_sizes[0]].view(-1, cols)
+            emb[torch.rand(emb.shape[0], generator=gen, device=dev) < zero_rows] = 0.0
     return out
 
 

@@ -79,3 +79,50 @@ def test_codes_of_layers_without_a_histogram():
     state = torch.from_numpy((rng.standard_normal((W, N)) * 0.01).astype(np.float32)).cuda()
     for budget in ([0.05 * 8 * N] * 3, [0.4 * 8 * N, 0.01 * 8 * N, 0.9 * 8 * N]):
         r.compare_step(grads, state, budget, 1.0)
+
+
+def _row_sparse(rng, W, rows, cols, zero_frac, tail):
+    """[W][rows * cols + tail]: a matrix whose untouched rows are exactly zero (an embedding gradient), then a dense tail."""
+    x = rng.standard_normal((W, rows * cols + tail)).astype(np.float32)
+    m = x[:, :rows * cols].reshape(W, rows, cols)
+    m[rng.random((W, rows)) < zero_frac] = 0.0
+    return x
+
+
+@pytest.mark.parametrize("zero_frac,schedule", [(0.5, 0), (0.9, 1), (0.995, 1)])
+def test_row_sparse_layer(zero_frac, schedule):
+    """A 1.2 M-element layer with whole rows of exact zeros: candidates below the number of non-zeros have ordinary
+    thresholds, the others have threshold 0 and keep zeros in index order.  Nothing of it may need the exact path:
+    zeros are counted apart, loose candidates are refined from the code bytes."""
+    rng = np.random.default_rng(int(zero_frac * 1000))
+    rows, cols, tail = 600, 2048, 70000
+    sizes = [rows * cols, tail]
+    grid = [0.001, 0.004, 0.02, 0.05, 0.1, 0.2, 0.4, 0.6, 0.9, 1.0]
+    W, N = 2, sum(sizes)
+    r = Runner(sizes, W, grid, 1000, 0, schedule=schedule)
+    state = torch.zeros((W, N), dtype=torch.float32, device="cuda")
+    for step, frac in enumerate([0.02, 0.3, 0.7]):  # the last budget reaches candidates whose threshold is 0
+        grads = torch.from_numpy(_row_sparse(rng, W, rows, cols, zero_frac, tail)).cuda()
+        res = r.compare_step(grads, state, [frac * 8 * N, 0.5 * frac * 8 * N], 1.0)
+        assert res["same_k"]
+    why = kb.kimad_debug_exact_path_layers(r.ctx, detail=True)
+    assert why[0] == 0, f"exact path taken: {why[:6]}"
+
+
+def test_loose_candidates_are_refined():
+    """Few, very wide bands (two populations 40 octaves apart under a coarse grid) leave bins whose error bound is too
+    loose; those candidates are refined, and the refined curve, thresholds and selection equal the oracle's."""
+    rng = np.random.default_rng(77)
+    sizes = [900000, 50000]
+    grid = [0.02, 0.3, 0.55, 0.8, 1.0]
+    W, N = 2, sum(sizes)
+    x = rng.standard_normal((W, N)).astype(np.float32)
+    x[rng.random((W, N)) < 0.5] *= np.float32(1e-12)
+    r = Runner(sizes, W, grid, 1000, 0, schedule=1)
+    grads = torch.from_numpy(x).cuda()
+    state = torch.zeros_like(grads)
+    for budget in ([0.1 * 8 * N] * 2, [0.6 * 8 * N, 0.35 * 8 * N]):
+        res = r.compare_step(grads, state, budget, 1.0)
+        assert res["same_k"]
+    why = kb.kimad_debug_exact_path_layers(r.ctx, detail=True)
+    assert why[1] == 0 and why[2] == 0
