@@ -66,8 +66,8 @@ struct kimad_ctx {
     // (every group has a stream for its sweeps, of low priority, and one for its short kernels, of high priority, so
     // that a DP or an offset scan is not queued behind another group's sweep; events hand the group over between
     // the two)
-    cudaStream_t gstream[kGroups] = {}, gshort[kGroups] = {};
-    cudaEvent_t ev_go = nullptr, ev_done[kGroups] = {}, ev_hand[kGroups][4] = {};
+    cudaStream_t gstream[kGroups] = {}, gshort[kGroups] = {}, glist[kGroups] = {};
+    cudaEvent_t ev_go = nullptr, ev_done[kGroups] = {}, ev_hand[kGroups][4] = {}, ev_list[kGroups][2] = {};
     int pipeline_mode = 0; // 0: two groups when the step is large enough, 1: whenever W >= 2, 2: never
     bool have_ev = false;
     template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
@@ -153,6 +153,7 @@ static int preload_kernels() {
     cudaFuncAttributes a;
 #define KIMAD_PRELOAD(f) CUDA_TRY(cudaFuncGetAttributes(&a, f))
     KIMAD_PRELOAD(k_sample); KIMAD_PRELOAD(k_pass_a<true>); KIMAD_PRELOAD(k_pass_a<false>); KIMAD_PRELOAD(k_resolve_a);
+    KIMAD_PRELOAD(k_refine_hist); KIMAD_PRELOAD(k_refine_resolve);
     KIMAD_PRELOAD(k_tiny_exact); KIMAD_PRELOAD(k_fb_hist1); KIMAD_PRELOAD(k_fb_hist23<2>); KIMAD_PRELOAD(k_fb_hist23<3>);
     KIMAD_PRELOAD(k_resolve1); KIMAD_PRELOAD(k_resolve23<2>); KIMAD_PRELOAD(k_resolve23<3>); KIMAD_PRELOAD(k_rebuild_slots);
     KIMAD_PRELOAD(k_dp); KIMAD_PRELOAD(k_fit_ratio); KIMAD_PRELOAD(k_sel_count); KIMAD_PRELOAD(k_sel_count_r2); KIMAD_PRELOAD(k_sel_resolve);
@@ -208,6 +209,8 @@ static int ensure_side_stream(kimad_ctx* c) {
     for (int g = 0; g < kGroups; ++g) {
         CUDA_TRY(cudaStreamCreateWithPriority(&c->gstream[g], cudaStreamNonBlocking, prio_least));
         CUDA_TRY(cudaStreamCreateWithPriority(&c->gshort[g], cudaStreamNonBlocking, prio_greatest));
+        CUDA_TRY(cudaStreamCreateWithPriority(&c->glist[g], cudaStreamNonBlocking, prio_greatest));
+        for (cudaEvent_t& e : c->ev_list[g]) CUDA_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
         CUDA_TRY(cudaEventCreateWithFlags(&c->ev_done[g], cudaEventDisableTiming));
         for (cudaEvent_t& e : c->ev_hand[g]) CUDA_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
     }
@@ -389,36 +392,57 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
             c->launches += 1;
         }
         mark(small);
-        // exact radix select for the layers handed over by k_resolve_a (the lists are usually empty)
-        if (R) {
+        // (c) as a launch sequence on stream st; `when`: 0 always, 1 only if no layer is listed for the refinement or
+        // the exact path, 2 only if one is
+        auto launch_dp = [&](cudaStream_t st, uint32_t when) -> int {
+            for (uint32_t wa = w0; wa < w0 + nw; wa += kDpWorkersPerLaunch) {
+                const uint32_t nwa = std::min<uint32_t>(kDpWorkersPerLaunch, w0 + nw - wa);
+                const int dp_mode = mode == kGivenJ ? 1 : (c->policy == 1 ? 2 : (c->policy == 2 ? 3 : (c->policy == 3 ? 4 : 0)));
+                CUDA_TRY(launch_pdl(k_dp, nwa, kDpThreads, c->dp_smem, st, budgets_of(wa, nwa), wa, W, L, K, c->D, c->bpe, c->full_bytes,
+                                    c->cap, c->check_finite, dp_mode, c->cost_model, c->dp_plan, layers,
+                                    ktab, mode == kInjectErr ? err_dev : err, tau, keq, shf, j_dev, flags, pd, sel, out->k, out->j,
+                                    out->offs, out->stats, out->dense, CodeSpace{reg_index, meta, cell_tab, cell_win, R}, when, fb));
+                c->launches += 1;
+            }
+            return KIMAD_OK;
+        };
+        // refinement and exact radix select for the layers listed by k_resolve_a (the lists are usually empty)
+        auto launch_lists = [&](cudaStream_t st) -> int {
             // small grids: the lists are usually empty, and every kernel of the chain then costs only its launch; the
             // histogram kernels get four CTAs per SM, enough to stream a large handed-over layer
             const uint32_t gfb = 4 * 148, glay = std::min<uint32_t>(nw * R, 32u);
             const dim3 gslot(glay, 1, K);
             // candidates with a loose bound first (they may still end on the exact path's lists)
-            CUDA_TRY(launch_pdl(k_refine_hist, gfb, blk, 0, small, dbuf, chunks, c->dstride, L, K, fb, rf_chunks, rf,
+            CUDA_TRY(launch_pdl(k_refine_hist, gfb, blk, 0, st, dbuf, chunks, c->dstride, L, K, fb, rf_chunks, rf,
                                 CodeSpace{reg_index, meta, cell_tab, cell_win, R}, h23c, h23s));
-            CUDA_TRY(launch_pdl(k_refine_resolve, glay, blk, 0, small, layers, L, K, fb, rf_layers, rf, h23c, h23s, err, tau, keq, shf,
+            CUDA_TRY(launch_pdl(k_refine_resolve, glay, blk, 0, st, layers, L, K, fb, rf_layers, rf, h23c, h23s, err, tau, keq, shf,
                                 fb_chunks, fb_layers, list_cap));
-            CUDA_TRY(launch_pdl(k_fb_hist1, gfb, blk, 0, small, dbuf, chunks, c->dstride, L, fb, fb_chunks, h1c, h1s, flags));
-            CUDA_TRY(launch_pdl(k_resolve1, glay, blk, 0, small, fb, fb_layers, h1c, h1s, ktab, L, K, cands, slots));
-            CUDA_TRY(launch_pdl(k_fb_hist23<2>, gfb, blk, 0, small, dbuf, chunks, c->dstride, L, K, fb, fb_chunks, slots, h23c, h23s));
-            CUDA_TRY(launch_pdl(k_resolve23<2>, gslot, blk, 0, small, fb, fb_layers, h23c, h23s, L, K, cands, slots, err, tau, keq, shf));
-            CUDA_TRY(launch_pdl(k_rebuild_slots, (nw * R + kThreads - 1) / kThreads, blk, 0, small, fb, fb_layers, L, K, cands, slots));
-            CUDA_TRY(launch_pdl(k_fb_hist23<3>, gfb, blk, 0, small, dbuf, chunks, c->dstride, L, K, fb, fb_chunks, slots, h23c, h23s));
-            CUDA_TRY(launch_pdl(k_resolve23<3>, gslot, blk, 0, small, fb, fb_layers, h23c, h23s, L, K, cands, slots, err, tau, keq, shf));
+            CUDA_TRY(launch_pdl(k_fb_hist1, gfb, blk, 0, st, dbuf, chunks, c->dstride, L, fb, fb_chunks, h1c, h1s, flags));
+            CUDA_TRY(launch_pdl(k_resolve1, glay, blk, 0, st, fb, fb_layers, h1c, h1s, ktab, L, K, cands, slots));
+            CUDA_TRY(launch_pdl(k_fb_hist23<2>, gfb, blk, 0, st, dbuf, chunks, c->dstride, L, K, fb, fb_chunks, slots, h23c, h23s));
+            CUDA_TRY(launch_pdl(k_resolve23<2>, gslot, blk, 0, st, fb, fb_layers, h23c, h23s, L, K, cands, slots, err, tau, keq, shf));
+            CUDA_TRY(launch_pdl(k_rebuild_slots, (nw * R + kThreads - 1) / kThreads, blk, 0, st, fb, fb_layers, L, K, cands, slots));
+            CUDA_TRY(launch_pdl(k_fb_hist23<3>, gfb, blk, 0, st, dbuf, chunks, c->dstride, L, K, fb, fb_chunks, slots, h23c, h23s));
+            CUDA_TRY(launch_pdl(k_resolve23<3>, gslot, blk, 0, st, fb, fb_layers, h23c, h23s, L, K, cands, slots, err, tau, keq, shf));
             c->launches += 9;
-        }
-        mark(small);
-        // (c)
-        for (uint32_t wa = w0; wa < w0 + nw; wa += kDpWorkersPerLaunch) {
-            const uint32_t nwa = std::min<uint32_t>(kDpWorkersPerLaunch, w0 + nw - wa);
-            const int dp_mode = mode == kGivenJ ? 1 : (c->policy == 1 ? 2 : (c->policy == 2 ? 3 : (c->policy == 3 ? 4 : 0)));
-            CUDA_TRY(launch_pdl(k_dp, nwa, kDpThreads, c->dp_smem, small, budgets_of(wa, nwa), wa, W, L, K, c->D, c->bpe, c->full_bytes, c->cap,
-                                c->check_finite, dp_mode, c->cost_model, c->dp_plan, layers,
-                                ktab, mode == kInjectErr ? err_dev : err, tau, keq, shf, j_dev, flags, pd, sel, out->k, out->j,
-                                out->offs, out->stats, out->dense, CodeSpace{reg_index, meta, cell_tab, cell_win, R}));
-            c->launches += 1;
+            return KIMAD_OK;
+        };
+        if (R && !c->timing) {
+            // The lists are usually empty, so the DP is launched at once and goes ahead only if they are; the nine
+            // list-driven kernels run beside it on a stream of their own, followed by a second launch of the DP that
+            // goes ahead only if something was listed.  Their launch latencies leave the step's critical path.
+            cudaStream_t lst = c->glist[g];
+            CUDA_TRY(cudaEventRecord(c->ev_list[g][0], small));
+            CUDA_TRY(cudaStreamWaitEvent(lst, c->ev_list[g][0], 0));
+            { const int rc = launch_dp(small, 1); if (rc != KIMAD_OK) return rc; }
+            { const int rc = launch_lists(lst); if (rc != KIMAD_OK) return rc; }
+            { const int rc = launch_dp(lst, 2); if (rc != KIMAD_OK) return rc; }
+            CUDA_TRY(cudaEventRecord(c->ev_list[g][1], lst));
+            CUDA_TRY(cudaStreamWaitEvent(small, c->ev_list[g][1], 0));
+        } else {
+            if (R) { const int rc = launch_lists(small); if (rc != KIMAD_OK) return rc; }
+            mark(small);
+            { const int rc = launch_dp(small, 0); if (rc != KIMAD_OK) return rc; }
         }
         mark(small);
         CUDA_TRY(hand_over(small, big));
@@ -595,6 +619,8 @@ void kimad_destroy(kimad_ctx* ctx) {
         for (int g = 0; g < kGroups; ++g) {
             if (ctx->gstream[g]) { cudaStreamSynchronize(ctx->gstream[g]); cudaStreamDestroy(ctx->gstream[g]); }
             if (ctx->gshort[g]) { cudaStreamSynchronize(ctx->gshort[g]); cudaStreamDestroy(ctx->gshort[g]); }
+            if (ctx->glist[g]) { cudaStreamSynchronize(ctx->glist[g]); cudaStreamDestroy(ctx->glist[g]); }
+            for (cudaEvent_t e : ctx->ev_list[g]) if (e) cudaEventDestroy(e);
             if (ctx->ev_done[g]) cudaEventDestroy(ctx->ev_done[g]);
             for (cudaEvent_t e : ctx->ev_hand[g]) if (e) cudaEventDestroy(e);
         }

@@ -436,11 +436,19 @@ k_dp(DpBudgets budgets, uint32_t w_base, uint32_t W, uint32_t L, uint32_t K, uin
      const uint32_t* __restrict__ j_in, uint32_t* __restrict__ flags,
      uint8_t* __restrict__ pd_global, Sel* __restrict__ sel, uint32_t* __restrict__ out_k,
      uint32_t* __restrict__ out_j, uint64_t* __restrict__ out_offs, kimad_stats* __restrict__ out_stats,
-     uint32_t* __restrict__ out_dense /* may be null */, const CodeSpace codes) {
+     uint32_t* __restrict__ out_dense /* may be null */, const CodeSpace codes,
+     uint32_t when /* 0: always; 1: only if no layer is listed for refinement or the exact path; 2: only if one is */,
+     const FbList* __restrict__ lists) {
     pdl_wait();
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const uint32_t w = w_base + blockIdx.x;
     if (w >= W) return;
+    if (when) {
+        // a layer listed for refinement may move on to the exact path's list while this kernel runs, but then the
+        // refinement's list alone decides
+        const bool listed = lists->rf_layers != 0u || lists->n_layers != 0u;
+        if (listed != (when == 2u)) return;
+    }
     const uint64_t c = budgets.c[blockIdx.x];
     const uint32_t row = D + 1, pad = D + 2, rowp = row + pad, Kp = (K + 3) & ~3u;
     const float kInf = __int_as_float(0x7f800000);
