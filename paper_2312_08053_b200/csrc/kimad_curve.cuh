@@ -116,8 +116,10 @@ k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint6
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
             const uint32_t key = ok[u] ? key_of(__fsub_rn(a[u], b[u])) : 1u;
-            const uint32_t zu = __popc(__ballot_sync(0xffffffffu, key == 0u)); // the unit's exact zeros
-            if (zu && (threadIdx.x & 31) == 0) { atomicAdd(&s_z, zu); atomicAdd(&s_zz, (unsigned long long)(zu * zu)); }
+            if ((u & 3) == 0) { // every fourth unit: its exact zeros, for the spread of the zeros over the units
+                const uint32_t zu = __popc(__ballot_sync(0xffffffffu, key == 0u));
+                if (zu && (threadIdx.x & 31) == 0) { atomicAdd(&s_z, zu); atomicAdd(&s_zz, (unsigned long long)(zu * zu)); }
+            }
             if (ok[u]) {
                 if (key) atomicAdd(&h32[key >> 16], 1u << (16 * ((key >> 15) & 1)));
                 ++mine;
@@ -126,15 +128,7 @@ k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint6
     }
     atomicAdd(&s_m, mine);
     __syncthreads();
-    // fewer zeros than 1/64 of the sample are treated like any other key (cell 0)
-    const uint32_t m = s_m;
-    const uint32_t z = s_z * 64u >= m ? s_z : 0u, mz = m - z; // sample size, its zero mass, the rest
-    if (threadIdx.x == 0 && z == 0 && s_z) h32[0] += s_z;
-    __syncthreads();
-    // variance of the sample's zero count from the spread of the units' zero counts: zeros that come in runs (whole
-    // rows) make the sample's share of zeros, and with it the sample rank of every threshold among the other keys,
-    // far less certain than independent draws would
-    const double var_z = z ? fmax(0.0, (double)s_zz - (double)z * (double)z / (double)m_units) : 0.0;
+    const uint32_t m = s_m; // sample size, exact zeros included
     auto cell_count = [&](uint32_t cell) { return (h32[cell >> 1] >> (16 * (cell & 1))) & 0xffffu; };
     auto cell_sq = [&](uint32_t cell) { // square of the cell's middle value (planning only: float range is enough)
         const float v = __uint_as_float((cell << 15) | 0x4000u);
@@ -143,6 +137,7 @@ k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint6
 
     // ---- per thread segment (cells 65535 - 64 t - (0..63)): sample count and squares; the reads of a warp are
     // rotated so that its lanes hit different banks
+    uint32_t mz; // sample entries in the histogram: all but the exact zeros
     {
         uint32_t sum = 0;
         double sq = 0.0;
@@ -153,14 +148,22 @@ k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint6
             sum += c;
             if (c) sq += (double)c * cell_sq(top - i);
         }
-        uint32_t tot;
         double totd;
-        const uint32_t ex = block_excl_scan<uint32_t, kBigThreads>(sum, s_w, &tot);
+        const uint32_t ex = block_excl_scan<uint32_t, kBigThreads>(sum, s_w, &mz);
         const double exd = block_excl_scan<double, kBigThreads>(sq, s_wd, &totd);
         s_pre[threadIdx.x] = ex + sum;
         s_sq[threadIdx.x] = totd - exd - sq; // squares in the segments below this one (higher thread index)
     }
     __syncthreads();
+    const uint32_t z = m - mz; // the sample's exact zeros
+    // Variance of the sample's zero count, from the spread of the zero counts of the units looked at (the units i with
+    // i mod 128 < 32): zeros that come in runs (whole rows) make the sample's share of zeros, and with it the sample
+    // rank of every threshold among the other keys, far less certain than independent draws would.
+    double var_z = 0.0;
+    if (z && !whole) {
+        const double ns = (double)((m_units / 128u) * 32u + min(m_units % 128u, 32u)), zs = (double)s_z;
+        var_z = fmax(0.0, ((double)s_zz - zs * zs / ns) / ns) * (double)m_units;
+    }
     // cell holding sample rank rk (1-based, from the top); the whole warp takes part
     const uint32_t lane = threadIdx.x & 31;
     auto cell_of_rank = [&](uint32_t rk) {
