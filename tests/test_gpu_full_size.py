@@ -111,7 +111,7 @@ def _full_size_step(cfg, step_of_trace, sample_layers, workers_checked):
     return kb.kimad_debug_exact_path_layers(ctx, detail=True)
 
 
-def _every_element(cfg, step_of_trace, workers):
+def _every_element(cfg, step_of_trace, workers, zero_rows=0.0):
     """One full-size step in the benchmark's launch configuration, EVERY element of the listed workers compared
     with the oracle's whole pass (curves of all layers and candidates to the curve tolerance; decisions, packed
     indices and values, offsets, statistics and the EF21 state bit for bit)."""
@@ -124,10 +124,10 @@ def _every_element(cfg, step_of_trace, workers):
     ctx = kb.new_context(wl.layer_sizes, W, wl.ratio_grid, D=wl.D, value_dtype=wl.value_dtype, max_packed_elems=cap)
     out = kb.Packed(ctx)
     state = torch.zeros((W, N), dtype=torch.float32, device="cuda")
-    g0 = workloads.gradients(wl, 0, device="cuda")
+    g0 = workloads.gradients(wl, 0, device="cuda", zero_rows=zero_rows)
     kb.kimad_step(ctx, g0, state, bw_all[0], wl.t_target, out)  # an earlier step: the EF state is not all zero
     del g0
-    grads = workloads.gradients(wl, 1, device="cuda")
+    grads = workloads.gradients(wl, 1, device="cuda", zero_rows=zero_rows)
     state_before = state.clone()
     kb.kimad_step(ctx, grads, state, bw, wl.t_target, out)
     status, k_gpu = kb.kimad_get_k(ctx)
@@ -186,6 +186,18 @@ def test_gpt2_small_shape_full_size_every_element_burst():
     # a burst of the trace (25 Gbit/s: about 16 % of the entries kept), one worker
     bw = workloads.bandwidth_trace(workloads.workload(4))
     _every_element(4, step_of_trace=int(np.argmax(bw[:, 0])), workers=[2])
+
+
+def test_llama_1b_shape_full_size_sparse_embedding_rows():
+    # 90 % of the token embedding's gradient rows exactly zero (drawn per worker and step): the 65.5 M-element layer
+    # is swept without its zeros, its loose candidates are refined; a high-budget step, so that candidates whose
+    # threshold lies among the zeros are in play; every element of one worker
+    bw = workloads.bandwidth_trace(workloads.workload(5))
+    _every_element(5, step_of_trace=int(np.argmax(bw[:, 0])), workers=[0], zero_rows=0.9)
+
+
+def test_gpt2_small_shape_full_size_sparse_embedding_rows():
+    _every_element(4, step_of_trace=7, workers=[1, 3], zero_rows=0.6)
 
 
 def test_llama_1b_shape_full_size_every_element_of_one_worker():
