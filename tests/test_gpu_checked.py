@@ -26,8 +26,10 @@ def _run_checked(code_or_args, is_code):
 def test_parity_selection_under_the_checked_build():
     sel = ("cfg1 or cfg2 or cfg3 or cfg4 or adversarial or unaligned or concentrated or interface_limits or "
            "randomized_configurations or huge_dynamic or fitted_ratio_matches or dense_fallback_matches or "
-           "exact_radix_everywhere or paper_grid")
-    res = _run_checked(["tests/test_gpu_parity.py", "tests/test_gpu_policies.py", "-k", sel], is_code=False)
+           "exact_radix_everywhere or paper_grid or row_sparse or loose_candidates or thresholds_among_zeros or "
+           "window_wider")
+    res = _run_checked(["tests/test_gpu_parity.py", "tests/test_gpu_policies.py", "tests/test_gpu_tables.py", "-k", sel],
+                       is_code=False)
     assert res.returncode == 0, res.stdout[-3000:] + res.stderr[-2000:]
     assert " passed" in res.stdout and "failed" not in res.stdout
 
