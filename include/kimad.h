@@ -69,8 +69,9 @@ typedef struct {
     uint32_t infeasible_policy; /* 0: take candidate 0 everywhere and report KIMAD_STATUS_INFEASIBLE */
     uint64_t max_packed_elems;  /* capacity (entries) of each worker's idx/val buffer; 0 -> N        */
     uint64_t worker_stride;     /* elements between consecutive workers in grads/state; 0 -> N       */
-    uint32_t curve_mode;        /* 0: error curves from one sweep over sampled bands, exact radix select
-                                   only where the certificate fails; 1: exact radix select everywhere   */
+    uint32_t curve_mode;        /* 0: error curves from one sweep over sampled bands; a candidate whose certified
+                                   bound is too loose is refined, a layer whose threshold fell outside its band
+                                   takes the exact radix select; 1: exact radix select everywhere          */
     uint32_t policy;            /* 0: Kimad+, the knapsack search over the layers (Section 3.2, Algorithm 3);
                                    1: Kimad, one ratio of the grid for every layer: the largest whose total
                                       size fits c (Section 3.1; the fixed-ratio baseline of Section 4.3).
@@ -281,7 +282,7 @@ int kimad_debug_get_band_meta(kimad_ctx* ctx, uint32_t* host_meta);
  * around its stages on the step's stream (first use creates the events).  kimad_debug_stage_times
  * synchronises the device and writes the last step's stage durations in milliseconds to host_ms
  * (host, f32 [KIMAD_N_STAGES]), stage order: sample, sweep (difference + banded histogram), curve
- * (resolve + tiny layers), exact radix fallback, dp, select_count, select_scan, select_write. */
+ * (resolve + tiny layers), refinement and exact radix fallback, dp, select_count, select_scan, select_write. */
 #define KIMAD_N_STAGES 8
 int kimad_debug_enable_stage_timing(kimad_ctx* ctx, int enable);
 int kimad_debug_stage_times(kimad_ctx* ctx, float* host_ms);
