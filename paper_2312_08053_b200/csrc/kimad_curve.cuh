@@ -98,17 +98,23 @@ k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint6
     for (uint32_t ib = threadIdx.x / kSampleUnit; ib < m_units; ib += 8 * (kBigThreads / kSampleUnit)) {
         float a[8], b[8];
         bool ok[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const uint32_t i = ib + u * (kBigThreads / kSampleUnit);
-            uint32_t start = kSampleUnit * i;
+        // where the round's eight units start is the same for all lanes: lane u (mod 8) works out unit u's start
+        // and the others fetch it with a shuffle
+        uint32_t my_start;
+        {
+            const uint32_t i = ib + (threadIdx.x & 7u) * (kBigThreads / kSampleUnit);
+            my_start = kSampleUnit * i;
             if (!whole && i < m_units) { // unit i somewhere inside stratum i = [i q + i r / m, (i+1) q + (i+1) r / m)
                 const uint32_t s0 = i * sq_ + (i * sr_) / (uint32_t)kSampleUnits;
                 const uint32_t s1 = (i + 1) * sq_ + ((i + 1) * sr_) / (uint32_t)kSampleUnits;
                 const uint32_t room = s1 > s0 + kSampleUnit ? s1 - s0 - kSampleUnit : 0;
-                start = s0 + __umulhi(hash_u32(i * 0x9e3779b9u + l * 0x85ebca6bu + 1u), room + 1);
+                my_start = s0 + __umulhi(hash_u32(i * 0x9e3779b9u + l * 0x85ebca6bu + 1u), room + 1);
             }
-            const uint32_t p = start + (threadIdx.x % kSampleUnit);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const uint32_t i = ib + u * (kBigThreads / kSampleUnit);
+            const uint32_t p = __shfl_sync(0xffffffffu, my_start, u) + (threadIdx.x % kSampleUnit);
             ok[u] = i < m_units && p < n;
             a[u] = ok[u] ? gr[p] : 0.f;
             b[u] = ok[u] ? st[p] : 0.f;
@@ -916,6 +922,90 @@ k_refine_resolve(const LayerDesc* __restrict__ layers, uint32_t L, uint32_t K, F
 }
 
 // ------------------------------------------------------------------------------------------------
+// Bitonic sort (descending) of np = 512 .. kTinyMax keys in shared memory with sixteen consecutive keys per thread
+// held in registers: compare-exchanges at distances below 16 stay inside a thread, distances 16 .. 256 are a
+// shuffle with the thread 1 .. 16 lanes away, and only distances of 512 and more (six of the 78 stages at 4096
+// keys) go through shared memory.  The first np / 16 threads hold keys (whole warps: np >= 512); all threads of
+// the CTA take part in the barriers.
+// ------------------------------------------------------------------------------------------------
+template <int STRIDE>
+__device__ __forceinline__ void tiny_ce_inside(uint32_t (&v)[16], bool desc) {
+#pragma unroll
+    for (int e = 0; e < 16; ++e)
+        if (!(e & STRIDE)) {
+            const uint32_t hi = max(v[e], v[e | STRIDE]), lo = min(v[e], v[e | STRIDE]);
+            v[e] = desc ? hi : lo;
+            v[e | STRIDE] = desc ? lo : hi;
+        }
+}
+// the stages of the sizes 2 .. 8: direction by the key's position inside the thread
+template <int SIZE>
+__device__ __forceinline__ void tiny_sort_inside(uint32_t (&v)[16]) {
+#pragma unroll
+    for (int str = SIZE / 2; str > 0; str >>= 1)
+#pragma unroll
+        for (int e = 0; e < 16; ++e)
+            if (!(e & str)) {
+                const uint32_t hi = max(v[e], v[e | str]), lo = min(v[e], v[e | str]);
+                const bool desc = (e & SIZE) == 0;
+                v[e] = desc ? hi : lo;
+                v[e | str] = desc ? lo : hi;
+            }
+}
+__device__ __forceinline__ void tiny_sort_blocked(uint32_t* s_key, uint32_t np) {
+    const uint32_t t = threadIdx.x, nthr = np >> 4;
+    const bool holds = t < nthr;
+    uint32_t v[16];
+    if (holds) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const uint4 x = reinterpret_cast<const uint4*>(s_key)[4 * t + q];
+            v[4 * q] = x.x; v[4 * q + 1] = x.y; v[4 * q + 2] = x.z; v[4 * q + 3] = x.w;
+        }
+        tiny_sort_inside<2>(v); tiny_sort_inside<4>(v); tiny_sort_inside<8>(v);
+    }
+    for (uint32_t size = 16; size <= np; size <<= 1) { // from here on the direction depends on the thread
+        const bool desc = ((16u * t) & size) == 0;
+        for (uint32_t str = size >> 1; str >= 16u; str >>= 1) {
+            const uint32_t dt = str >> 4;                  // the partner thread is t ^ dt
+            const bool keep_max = ((t & dt) == 0) == desc; // the lower position keeps the larger key when descending
+            if (dt >= 32u) { // another warp: through shared memory
+                __syncthreads(); // s_key is no longer read
+                if (holds) {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        reinterpret_cast<uint4*>(s_key)[4 * t + q] = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+                }
+                __syncthreads();
+                if (holds) {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const uint4 x = reinterpret_cast<const uint4*>(s_key)[4 * (t ^ dt) + q];
+                        const uint32_t pv[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) v[4 * q + i] = keep_max ? max(v[4 * q + i], pv[i]) : min(v[4 * q + i], pv[i]);
+                    }
+                }
+            } else if (holds) { // a lane of the same warp (the warps that hold keys are whole)
+#pragma unroll
+                for (int e = 0; e < 16; ++e) {
+                    const uint32_t pv = __shfl_xor_sync(0xffffffffu, v[e], dt);
+                    v[e] = keep_max ? max(v[e], pv) : min(v[e], pv);
+                }
+            }
+        }
+        if (holds) { tiny_ce_inside<8>(v, desc); tiny_ce_inside<4>(v, desc); tiny_ce_inside<2>(v, desc); tiny_ce_inside<1>(v, desc); }
+    }
+    __syncthreads();
+    if (holds) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            reinterpret_cast<uint4*>(s_key)[4 * t + q] = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+    }
+    __syncthreads();
+}
+
+// ------------------------------------------------------------------------------------------------
 // k_tiny_exact: layers of at most kTinyMax elements, sorted in shared memory (one CTA each)
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kThreads)
@@ -946,6 +1036,8 @@ k_tiny_exact(const float* __restrict__ grads, const float* __restrict__ state, u
     }
     if (nonfinite) atomicOr(&flags[w], 1u);
     __syncthreads();
+    if (np >= 512u) tiny_sort_blocked(s_key, np);
+    else
     for (uint32_t size = 2; size <= np; size <<= 1)       // bitonic sort, descending
         for (uint32_t str = size >> 1; str > 0; str >>= 1) {
             for (uint32_t i = threadIdx.x; i < np / 2; i += kThreads) {
