@@ -81,7 +81,7 @@ k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint6
     }
     const LayerDesc ld = layers[l];
     const uint32_t n = (uint32_t)ld.n;
-    for (int i = threadIdx.x; i < 32768; i += kBigThreads) h32[i] = 0;
+    for (int i = threadIdx.x; i < 32768 / 4; i += kBigThreads) reinterpret_cast<uint4*>(h32)[i] = make_uint4(0u, 0u, 0u, 0u);
     if (threadIdx.x == 0) { s_m = 0; s_flag = 0; s_ng = 0; s_cg = 0; s_z = 0; s_zz = 0ull; }
     __syncthreads();
 
@@ -142,17 +142,25 @@ k_sample(const float* __restrict__ grads, const float* __restrict__ state, uint6
     };
 
     // ---- per thread segment (cells 65535 - 64 t - (0..63)): sample count and squares; the reads of a warp are
-    // rotated so that its lanes hit different banks
+    // rotated so that the lanes of a quarter warp hit different banks
     uint32_t mz; // sample entries in the histogram: all but the exact zeros
     {
         uint32_t sum = 0;
         double sq = 0.0;
-        const uint32_t top = 65535u - 64u * threadIdx.x;
-        for (uint32_t i0 = 0; i0 < 64; ++i0) {
-            const uint32_t i = (i0 + 2 * (threadIdx.x & 31)) & 63;
-            const uint32_t c = cell_count(top - i);
-            sum += c;
-            if (c) sq += (double)c * cell_sq(top - i);
+        // the segment is 32 words (two cells each), read four at a time; most words are empty
+        const uint32_t w0 = 32736u - 32u * threadIdx.x; // first word of the segment: cells 2 w0 .. 2 w0 + 63
+        for (uint32_t q0 = 0; q0 < 8; ++q0) {
+            const uint32_t q = (q0 + threadIdx.x) & 7u;
+            const uint4 x4 = reinterpret_cast<const uint4*>(h32)[(w0 >> 2) + q];
+            const uint32_t x[4] = {x4.x, x4.y, x4.z, x4.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                if (x[i]) {
+                    const uint32_t cell = 2u * (w0 + 4u * q + (uint32_t)i), c0 = x[i] & 0xffffu, c1 = x[i] >> 16;
+                    sum += c0 + c1;
+                    if (c0) sq += (double)c0 * cell_sq(cell);
+                    if (c1) sq += (double)c1 * cell_sq(cell + 1u);
+                }
         }
         double totd;
         const uint32_t ex = block_excl_scan<uint32_t, kBigThreads>(sum, s_w, &mz);
