@@ -14,9 +14,9 @@
 //                with (base, shift) = table(cell(key)), two u32 shared-memory atomics per element: the count, and
 //                the exact integer sum of squares in a u32 word whose (rare) carries go straight to the 64-bit sum
 //                in global memory.  CTAs own static runs of chunks balanced by elements.
-//   k_resolve_a  per (worker, layer): walks the bins from the bottom (zeros left out by the sweep = the layer's
-//                size minus the counted entries), finds the bin that holds every candidate's threshold, sums the
-//                squares below it.  The candidate's error is certified to 5e-6 relative from the bin's width.  A
+//   k_resolve_a  per (worker, layer): totals of every group of 32 bins, a scan over the groups, then a warp per
+//                candidate finds the group and the bin that hold its threshold (zeros left out by the sweep = the
+//                layer's size minus the counted entries) and the squares below it.  The candidate's error is certified to 5e-6 relative from the bin's width.  A
 //                threshold in a gap bin (the sample mispredicted) sends the layer to the exact radix path; a bound
 //                that is too loose sends the candidate to the refinement.
 //   k_refine_hist, k_refine_resolve
@@ -613,8 +613,9 @@ k_resolve_a(const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ r
     pdl_wait();
     __shared__ uint32_t s_drop[KIMAD_MAX_RATIOS]; // entries not kept by candidate j: n - k_j
     __shared__ int s_loose;
-    __shared__ uint32_t s_bin[KIMAD_MAX_RATIOS], s_before[KIMAD_MAX_RATIOS], s_cb[KIMAD_MAX_RATIOS];
-    __shared__ double s_below[KIMAD_MAX_RATIOS], s_sb[KIMAD_MAX_RATIOS];
+    constexpr int kGroups32 = (kMaxBins + 31) / 32;
+    __shared__ uint32_t s_gc[kGroups32]; // per group of 32 bins: entries, then the entries of the groups below it
+    __shared__ double s_gs[kGroups32];   // ... and their squares
     __shared__ uint32_t s_w32[32];
     __shared__ double s_w64[32];
     __shared__ int s_bad;
@@ -627,107 +628,94 @@ k_resolve_a(const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ r
     if (threadIdx.x < K) {
         const uint64_t k = ktab.at(w, (size_t)l * K + threadIdx.x);
         s_drop[threadIdx.x] = (uint32_t)(ld.n - k);
-        s_bin[threadIdx.x] = 0xffffffffu;
     }
     __syncthreads();
     if (!mt.flagged) {
-        const uint32_t nb = mt.n_bins;
+        const uint32_t nb = mt.n_bins, ngrp = (nb + 31u) >> 5; // groups of 32 consecutive bins (ascending keys)
         const uint32_t* blo = bin_lo + wr * (kMaxBins + 1);
         uint32_t* gc = bh_cnt + wr * kMaxBins;
         unsigned long long* gs = bh_sum + wr * kMaxBins;
-        // Every warp owns a contiguous range of bins (ascending keys).  First sweep: the range's totals; then
-        // a scan over the 32 warps; second sweep: running count / running squares per bin, to find the bin
-        // where the running count passes n - k_j.  No block-wide barrier inside the sweeps.
         const uint32_t lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-        const uint32_t per = ((nb + 31) / 32 + 31) & ~31u; // bins per warp, a multiple of 32
-        const uint32_t r0 = min(nb, wid * per), r1 = min(nb, r0 + per);
         auto bin_sq = [&](uint32_t b) { // the sweep summed squares in units of 2^8 sq_fixed
             return (double)gs[b] * (256.0 * sq_scale(blo[b] >> 23));
         };
-        uint32_t c_tot = 0;
-        double s_tot = 0.0;
-        for (uint32_t b = r0 + lane; b < r1; b += 32) { c_tot += gc[b]; s_tot += bin_sq(b); }
-#pragma unroll
-        for (int o = 16; o; o >>= 1) {
-            c_tot += __shfl_xor_sync(0xffffffffu, c_tot, o);
-            s_tot += __shfl_xor_sync(0xffffffffu, s_tot, o);
-        }
-        if (lane == 0) { s_w32[wid] = c_tot; s_w64[wid] = s_tot; }
-        __syncthreads();
-        uint32_t counted = 0;
-        for (uint32_t i = 0; i < kBigThreads / 32; ++i) counted += s_w32[i];
-        const uint32_t zeros = (uint32_t)ld.n - counted; // the sweep leaves exact zeros out of its histogram
-        uint32_t run_c = zeros; // entries below this warp's range: the zeros and the bins of the warps before
-        double run_s = 0.0;     // their squares
-        for (uint32_t i = 0; i < wid; ++i) { run_c += s_w32[i]; run_s += s_w64[i]; }
-        if (threadIdx.x < K && s_drop[threadIdx.x] < zeros) { // the threshold is 0: every other key is kept
-            s_bin[threadIdx.x] = 0xfffffffeu;
-            s_cb[threadIdx.x] = zeros - s_drop[threadIdx.x]; // zeros kept
-        }
+        // (1) entries and squares of every group; (2) exclusive prefixes over the groups; (3) a warp per candidate:
+        // the group where the running count passes n - k_j by bisection over the prefixes, then the bin inside it
         bool nonfinite = false;
-        for (uint32_t base = r0; base < r1; base += 32) {
-            const uint32_t b = base + lane;
+        for (uint32_t g = wid; g < ngrp; g += kBigThreads / 32) {
+            const uint32_t bb = 32u * g + lane;
             uint32_t c = 0;
             double sv = 0.0;
-            if (b < r1) {
-                c = gc[b];
-                sv = bin_sq(b);
-                if (c) { gc[b] = 0; gs[b] = 0ull; } // clean for the next step
-                nonfinite |= c && blo[b] >= 0x7f800000u;
+            if (bb < nb) {
+                c = gc[bb];
+                if (c) { sv = bin_sq(bb); nonfinite |= blo[bb] >= 0x7f800000u; }
             }
-            uint32_t ic = c;
-            double is = sv;
 #pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const uint32_t yc = __shfl_up_sync(0xffffffffu, ic, o);
-                const double ys = __shfl_up_sync(0xffffffffu, is, o);
-                if (lane >= (uint32_t)o) { ic += yc; is += ys; }
+            for (int o = 16; o; o >>= 1) {
+                c += __shfl_xor_sync(0xffffffffu, c, o);
+                sv += __shfl_xor_sync(0xffffffffu, sv, o);
             }
-            const uint32_t before = run_c + ic - c;
-            double ex_s = __shfl_up_sync(0xffffffffu, is, 1); // exclusive value from the left neighbour: no cancellation
-            if (lane == 0) ex_s = 0.0;
-            const double below = run_s + ex_s;
-            if (c)
-                for (uint32_t j = 0; j < K; ++j) { // the bin where the running count passes n - k_j holds the threshold
-                    const uint32_t dj = s_drop[j];
-                    if (dj >= before && dj - before < c) {
-                        s_bin[j] = b; s_before[j] = before; s_cb[j] = c; s_below[j] = below; s_sb[j] = sv;
-                    }
-                }
-            run_c += __shfl_sync(0xffffffffu, ic, 31);
-            run_s += __shfl_sync(0xffffffffu, is, 31);
+            if (lane == 0) { s_gc[g] = c; s_gs[g] = sv; }
         }
         if (nonfinite) atomicOr(&flags[w], 1u);
         __syncthreads();
-        for (uint32_t j = threadIdx.x; j < K; j += kBigThreads) {
+        uint32_t counted;
+        {
+            const uint32_t c = threadIdx.x < ngrp ? s_gc[threadIdx.x] : 0u;
+            const double sv = threadIdx.x < ngrp ? s_gs[threadIdx.x] : 0.0;
+            const uint32_t ec = block_excl_scan<uint32_t, kBigThreads>(c, s_w32, &counted);
+            const double es = block_excl_scan<double, kBigThreads>(sv, s_w64, nullptr);
+            __syncthreads();
+            if (threadIdx.x < ngrp) { s_gc[threadIdx.x] = ec; s_gs[threadIdx.x] = es; }
+        }
+        __syncthreads();
+        const uint32_t zeros = (uint32_t)ld.n - counted; // the sweep leaves exact zeros out of its histogram
+        for (uint32_t j = wid; j < K; j += kBigThreads / 32) {
             const size_t o = wl * K + j;
-            rf[o].shift = kNoRefine;
-            if (s_drop[j] == 0) { // everything kept
-                err_out[o] = 0.f; tau_out[o] = 0; rank_out[o] = 0; shift_out[o] = 0;
+            const uint32_t dj = s_drop[j];
+            if (lane == 0) rf[o].shift = kNoRefine;
+            if (dj == 0 || dj < zeros) { // everything kept; or the threshold is 0 and nothing but zeros is dropped
+                if (lane == 0) { err_out[o] = 0.f; tau_out[o] = 0; rank_out[o] = dj ? zeros - dj : 0u; shift_out[o] = 0; }
                 continue;
             }
-            const uint32_t bin = s_bin[j];
-            if (bin == 0xfffffffeu) { // exactly: nothing but zeros is dropped
-                err_out[o] = 0.f; tau_out[o] = 0; rank_out[o] = s_cb[j]; shift_out[o] = 0;
-                continue;
+            const uint32_t target = dj - zeros; // entries of the histogram that are dropped, counted from the bottom
+            uint32_t lo = 0, hi = ngrp - 1;     // the last group whose prefix does not exceed the target
+            while (lo < hi) { const uint32_t mid = (lo + hi + 1) >> 1; if (s_gc[mid] <= target) lo = mid; else hi = mid - 1; }
+            const uint32_t bin = 32u * lo + lane;
+            uint32_t c = 0;
+            double sv = 0.0;
+            if (bin < nb) { c = gc[bin]; if (c) sv = bin_sq(bin); }
+            uint32_t ic = c;
+            double is = sv;
+#pragma unroll
+            for (int q = 1; q < 32; q <<= 1) {
+                const uint32_t yc = __shfl_up_sync(0xffffffffu, ic, q);
+                const double ys = __shfl_up_sync(0xffffffffu, is, q);
+                if (lane >= (uint32_t)q) { ic += yc; is += ys; }
             }
-            if (bin == 0xffffffffu || (blo[bin] & kGapBit)) { atomicMax(&s_bad, 3); continue; } // outside its band
+            const uint32_t before = s_gc[lo] + ic - c;
+            double ex_s = __shfl_up_sync(0xffffffffu, is, 1); // exclusive value from the left neighbour: no cancellation
+            if (lane == 0) ex_s = 0.0;
+            const double below = s_gs[lo] + ex_s;
+            const bool mine = c && target >= before && target - before < c; // this bin holds the threshold
+            if (!__ballot_sync(0xffffffffu, mine)) { if (lane == 0) atomicMax(&s_bad, 3); continue; }
+            if (!mine) continue;
+            if (blo[bin] & kGapBit) { atomicMax(&s_bad, 3); continue; } // outside its band
             const uint32_t klo = blo[bin], width = (blo[bin + 1] & ~kGapBit) - klo;
-            const uint32_t cb = s_cb[j];
-            const uint32_t drop = s_drop[j] - s_before[j]; // entries of the bin that are not kept, < cb
+            const uint32_t cb = c, drop = target - before; // entries of the bin that are not kept, < cb
             const double vlo = (double)__uint_as_float(klo);
             // the dropped entries are the `drop` smallest of the bin: their squares sum to something in
             // [drop * vlo^2, drop * mean]; take the midpoint and certify the half-width
-            const double upper = s_sb[j] * ((double)drop / (double)cb);
+            const double upper = sv * ((double)drop / (double)cb);
             const double lower = (double)drop * vlo * vlo;
             double part = 0.5 * (upper + lower), slack = 0.5 * (upper - lower);
             if (drop == 0 || width == 1) { part = lower; slack = 0.0; }
-            const double e = s_below[j] + part;
+            const double e = below + part;
             if (slack > e * 5e-6) { // acceptance bound on the curve is 1e-5: this candidate's bin is looked at once more
                 if (klo == 0u && zeros) { atomicMax(&s_bad, 4); continue; } // (not a bin whose zeros were left out)
                 s_loose = 1;
                 atomicAdd(&fb->loose_j[j], 1u);
-                rf[o] = RefineCand{klo, (uint32_t)(31 - __clz(width)), cb, drop, s_below[j]};
+                rf[o] = RefineCand{klo, (uint32_t)(31 - __clz(width)), cb, drop, below};
                 continue;
             }
             err_out[o] = (float)e;
@@ -735,6 +723,9 @@ k_resolve_a(const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ r
             rank_out[o] = cb - drop;
             shift_out[o] = 31 - __clz(width);
         }
+        __syncthreads();
+        for (uint32_t bb = threadIdx.x; bb < nb; bb += kBigThreads) // clean for the next step
+            if (gc[bb]) { gc[bb] = 0; gs[bb] = 0ull; }
     }
     __syncthreads();
     const int bad = s_bad;
