@@ -126,3 +126,45 @@ def test_loose_candidates_are_refined():
         assert res["same_k"]
     why = kb.kimad_debug_exact_path_layers(r.ctx, detail=True)
     assert why[1] == 0 and why[2] == 0
+
+
+@pytest.mark.parametrize("schedule", [0, 1])
+def test_steps_issued_back_to_back(schedule):
+    """Seven steps issued without a host synchronisation in between -- sparse, quantised and dense gradients in turn,
+    so that the lists of the refinement and of the second select round fill and empty from step to step -- leave
+    the same messages and states as the same steps run one by one, each of which is compared with the oracle."""
+    rng = np.random.default_rng(11)
+    cols, sizes = 1024, [400 * 1024, 3000, 150000, 768]
+    grid = [0.001, 0.005, 0.02, 0.05, 0.1, 0.2, 0.4, 0.7, 1.0]
+    W, N, S = 4, sum(sizes), 7
+    grads = []
+    for kind in [1, 0, 2, 1, 3, 0, 1]:
+        x = rng.standard_normal((W, N)).astype(np.float32)
+        if kind == 1:
+            m = x[:, :sizes[0]].reshape(W, -1, cols)
+            m[rng.random((W, m.shape[1])) < 0.9] = 0
+        elif kind == 2:
+            x = np.round(x * 3) / 3
+        elif kind == 3:
+            x[rng.random(x.shape) < 0.5] *= np.float32(1e-15)
+        grads.append(torch.from_numpy(x).cuda())
+    bws = [rng.uniform(0.005, 0.9, W) * 8 * N for _ in range(S)]
+    one = Runner(sizes, W, grid, 1000, 0, schedule=schedule)
+    state = torch.zeros((W, N), dtype=torch.float32, device="cuda")
+    ref = []
+    for s in range(S):
+        one.compare_step(grads[s], state, bws[s], 1.0, check_inject=False)
+        ref.append((one.out.idx.clone(), one.out.val.clone(), one.out.offs.clone(), state.clone()))
+    run = Runner(sizes, W, grid, 1000, 0, schedule=schedule)
+    state2 = torch.zeros((W, N), dtype=torch.float32, device="cuda")
+    got = []
+    for s in range(S):
+        kb.kimad_step(run.ctx, grads[s], state2, bws[s], 1.0, run.out)
+        got.append((run.out.idx.clone(), run.out.val.clone(), run.out.offs.clone(), state2.clone()))
+    torch.cuda.synchronize()
+    for s in range(S):
+        offs = ref[s][2].cpu().numpy()
+        assert torch.equal(ref[s][2], got[s][2]) and torch.equal(ref[s][3], got[s][3]), f"step {s}"
+        for w in range(W):
+            n = int(offs[w, len(sizes)])
+            assert torch.equal(ref[s][0][w, :n], got[s][0][w, :n]) and torch.equal(ref[s][1][w, :n], got[s][1][w, :n]), f"step {s}"
