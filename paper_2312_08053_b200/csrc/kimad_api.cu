@@ -413,7 +413,7 @@ int run_step(kimad_ctx* c, const float* grads, float* state, const double* bw, d
             const uint32_t gfb = 4 * 148, glay = std::min<uint32_t>(nw * R, 32u);
             const dim3 gslot(glay, 1, K);
             // candidates with a loose bound first (they may still end on the exact path's lists)
-            CUDA_TRY(launch_pdl(k_refine_hist, gfb, blk, 0, st, dbuf, chunks, c->dstride, L, K, fb, rf_chunks, rf,
+            CUDA_TRY(launch_pdl(k_refine_hist, 6 * 148, blk, 0, st, dbuf, chunks, c->dstride, L, K, fb, rf_chunks, rf,
                                 CodeSpace{reg_index, meta, cell_tab, cell_win, R}, h23c, h23s));
             CUDA_TRY(launch_pdl(k_refine_resolve, glay, blk, 0, st, layers, L, K, fb, rf_layers, rf, h23c, h23s, err, tau, keq, shf,
                                 fb_chunks, fb_layers, list_cap));

@@ -758,7 +758,7 @@ k_resolve_a(const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ r
 // summed per piece (the level-2/3 arrays of the exact path serve as storage: a layer is never on both paths at once).
 // Costs one pass over the layer's code bytes instead of the exact path's three passes over its inputs.
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 6)
 k_refine_hist(DSource dbuf, const Chunk* __restrict__ chunks, uint64_t dstride, uint32_t L, uint32_t K,
               const FbList* __restrict__ fb, const uint2* __restrict__ rf_chunks, const RefineCand* __restrict__ rf,
               const CodeSpace codes, uint32_t* __restrict__ g_cnt, unsigned long long* __restrict__ g_ss) {
@@ -796,8 +796,7 @@ k_refine_hist(DSource dbuf, const Chunk* __restrict__ chunks, uint64_t dstride, 
             const uint32_t word = code < 64u ? (code < 32u ? m0 : m1) : (code < 96u ? m2 : m3);
             return (word >> (code & 31u)) & 1u;
         };
-        auto visit = [&](uint32_t x) {
-            const uint32_t key = key_of(dd.at(x));
+        auto place = [&](uint32_t key) { // the entry's piece, if it lies in one of the loose bins
             for (uint32_t p = 0; p < nc; ++p) {
                 const uint32_t d1 = key - s_klo[p], sh = s_shift[p];
                 if (d1 < (1u << sh)) {
@@ -811,6 +810,7 @@ k_refine_hist(DSource dbuf, const Chunk* __restrict__ chunks, uint64_t dstride, 
         const uint32_t units = (cv.len + 15u) >> 4;
         for (uint32_t u = threadIdx.x; u < units; u += kThreads) {
             const uint32_t e0 = 16u * u;
+            uint32_t hit = 0; // the unit's elements whose code is one of the loose bins' codes
             if (e0 >= cv.first && e0 + 16u <= cv.len) {
                 const uint4 a = __ldcs(reinterpret_cast<const uint4*>(dd.code) + u);
                 const uint32_t x[4] = {a.x, a.y, a.z, a.w};
@@ -818,10 +818,24 @@ k_refine_hist(DSource dbuf, const Chunk* __restrict__ chunks, uint64_t dstride, 
                 for (int i = 0; i < 4; ++i)
 #pragma unroll
                     for (int b = 0; b < 4; ++b)
-                        if (wanted((x[i] >> (8 * b)) & 127u)) visit(e0 + 4 * i + b);
+                        if (wanted((x[i] >> (8 * b)) & 127u)) hit |= 1u << (4 * i + b);
             } else {
                 for (uint32_t x = max(e0, cv.first); x < min(e0 + 16u, cv.len); ++x)
-                    if (wanted(dd.code[x] & 127u)) visit(x);
+                    if (wanted(dd.code[x] & 127u)) hit |= 1u << (x - e0);
+            }
+            while (hit) { // completed from the inputs four at a time: their loads are independent
+                uint32_t pos[4];
+                float v[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    pos[i] = hit ? (uint32_t)__ffs(hit) - 1u : 0xffffffffu;
+                    if (hit) hit &= hit - 1u;
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i) v[i] = pos[i] != 0xffffffffu ? dd.at(e0 + pos[i]) : 0.f;
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    if (pos[i] != 0xffffffffu) place(key_of(v[i]));
             }
         }
     }
