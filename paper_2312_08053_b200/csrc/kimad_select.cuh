@@ -132,17 +132,23 @@ __device__ __forceinline__ void sel_count_chunk(const DSource& dbuf, const Chunk
 #pragma unroll
                 for (int j = 0; j < 4; ++j) ge[j] = (x[j] + add_ge) & 0x80808080u;
                 if (ge[0] | ge[1] | ge[2] | ge[3]) { // with a sparse budget few lanes hold a code that is not below the interval's
+                    uint32_t hit = 0; // rare: the unit's entries with the interval's own code, bit k -> element k
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         const uint32_t gt = (x[j] + add_gt) & 0x80808080u;
                         above += __popc(gt);
                         f |= gt != 0; // entries with the interval's code mark the group only if they are not below it
-                        uint32_t border = ge[j] ^ gt; // rare: entries with the interval's code; bit 8 k + 7 -> element k
-                        while (border) {
-                            const uint32_t bit = __ffs(border) - 1;
-                            border &= border - 1;
-                            f |= visit(key_of(dd.at(e0 + 4 * j + (bit >> 3))));
-                        }
+                        const uint32_t border = ge[j] ^ gt; // bit 8 k + 7 -> element k of this word
+                        hit |= (((border >> 7) & 1u) | ((border >> 14) & 2u) | ((border >> 21) & 4u) | ((border >> 28) & 8u)) << (4 * j);
+                    }
+                    while (hit) { // completed from the inputs two at a time: their loads are independent
+                        const uint32_t p0 = __ffs(hit) - 1;
+                        hit &= hit - 1;
+                        const uint32_t p1 = hit ? __ffs(hit) - 1 : p0;
+                        hit &= hit - 1; // (0 stays 0)
+                        const float v0 = dd.at(e0 + p0), v1 = dd.at(e0 + p1);
+                        f |= visit(key_of(v0));
+                        if (p1 != p0) f |= visit(key_of(v1));
                     }
                 }
             } else if (e0 < cv.len) { // ragged first or last unit of the chunk
@@ -179,7 +185,7 @@ __device__ __forceinline__ void sel_count_chunk(const DSource& dbuf, const Chunk
     __syncthreads();
 }
 
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 6)
 k_sel_count(DSource dbuf, const Chunk* __restrict__ chunks, uint32_t n_chunks, uint64_t dstride,
             uint32_t L, const Sel* __restrict__ sel, const LayerDesc* __restrict__ layers, ChunkSel* __restrict__ csel,
             uint32_t* __restrict__ low_hist, uint32_t* __restrict__ recount_n, uint2* __restrict__ recount_list,
