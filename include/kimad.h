@@ -22,6 +22,9 @@
  * Conventions
  *   - L layers of sizes n_l, concatenated in list order into one flat vector of N elements.
  *     Worker w's vector starts at element w * worker_stride of `grads` and of `state`.
+ *     The sweeps use 128-bit loads when grads, state (and est / x on the receiving side) are 16-byte aligned
+ *     and worker_stride is a multiple of 4 elements; otherwise they read element by element (same results,
+ *     the sweep over the gradients takes about twice as long): pad worker_stride rather than pass an odd N.
  *   - "device" pointers are CUDA device memory of the current device; "host" pointers are
  *     ordinary host memory.  The library never allocates or frees device memory: scratch is
  *     the caller's (kimad_set_workspace).  All kernels are ordered on the caller's stream (some of them
@@ -68,7 +71,8 @@ typedef struct {
     uint32_t check_finite;      /* != 0: a non-finite d makes that worker's step fail with NONFINITE */
     uint32_t infeasible_policy; /* 0: take candidate 0 everywhere and report KIMAD_STATUS_INFEASIBLE */
     uint64_t max_packed_elems;  /* capacity (entries) of each worker's idx/val buffer; 0 -> N        */
-    uint64_t worker_stride;     /* elements between consecutive workers in grads/state; 0 -> N       */
+    uint64_t worker_stride;     /* elements between consecutive workers in grads/state; 0 -> N; a multiple
+                                   of 4 keeps the 128-bit loads (see Conventions)                     */
     uint32_t curve_mode;        /* 0: error curves from one sweep over sampled bands; a candidate whose certified
                                    bound is too loose is refined, a layer whose threshold fell outside its band
                                    takes the exact radix select; 1: exact radix select everywhere          */
