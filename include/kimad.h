@@ -24,7 +24,7 @@
  *     Worker w's vector starts at element w * worker_stride of `grads` and of `state`.
  *     The sweeps use 128-bit loads when grads, state (and est / x on the receiving side) are 16-byte aligned
  *     and worker_stride is a multiple of 4 elements; otherwise they read element by element (same results,
- *     the sweep over the gradients takes about twice as long): pad worker_stride rather than pass an odd N.
+ *     the sweep over the gradients takes about a third longer): pad worker_stride rather than pass an odd N.
  *   - "device" pointers are CUDA device memory of the current device; "host" pointers are
  *     ordinary host memory.  The library never allocates or frees device memory: scratch is
  *     the caller's (kimad_set_workspace).  All kernels are ordered on the caller's stream (some of them

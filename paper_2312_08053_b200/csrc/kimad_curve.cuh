@@ -548,15 +548,26 @@ k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, uint8
         const bool active = wr != 0xffffffffu;
         const ChunkView cv(ch);
         uint8_t* dc = dc0 + cv.a0;
-        if (VEC) {
-            const float4* gr4 = reinterpret_cast<const float4*>(gr0 + cv.a0);
-            const float4* st4 = reinterpret_cast<const float4*>(st0 + cv.a0);
+        {
             const uint32_t q_lo = (cv.first + 3) >> 2, q_hi = cv.len >> 2; // whole quads [q_lo, q_hi)
             // One quad per thread and round; the loads of the round three rounds ahead are issued before the current
             // round is processed (four register sets, taken in turn), so that a round's memory latency lies behind
-            // the work of the rounds before it
+            // the work of the rounds before it.  VEC: both inputs are 16-byte aligned at every worker's start and a
+            // quad is one 128-bit load per input; otherwise four 32-bit loads, served from L1 after the first.
+            const float4* gr4 = reinterpret_cast<const float4*>(gr0 + cv.a0); // (only dereferenced as float4 when VEC)
+            const float4* st4 = reinterpret_cast<const float4*>(st0 + cv.a0);
             auto fetch = [&](float4& a, float4& b, uint32_t q) {
-                if (q < q_hi) { a = __ldcg(gr4 + q); b = __ldcg(st4 + q); }
+                if (q < q_hi) {
+                    if (VEC) {
+                        a = __ldcg(gr4 + q);
+                        b = __ldcg(st4 + q);
+                    } else {
+                        const float* g = reinterpret_cast<const float*>(gr4 + q);
+                        const float* t = reinterpret_cast<const float*>(st4 + q);
+                        a = make_float4(__ldg(g), __ldg(g + 1), __ldg(g + 2), __ldg(g + 3));
+                        b = make_float4(__ldg(t), __ldg(t + 1), __ldg(t + 2), __ldg(t + 3));
+                    }
+                }
             };
             auto work = [&](const float4& a, const float4& b, uint32_t q, auto skip) {
                 const uint32_t k[4] = {key_of(__fsub_rn(a.x, b.x)), key_of(__fsub_rn(a.y, b.y)),
@@ -587,11 +598,6 @@ k_pass_a(const float* __restrict__ grads, const float* __restrict__ state, uint8
                     const uint32_t key = key_of(__fsub_rn(gr0[cv.a0 + e], st0[cv.a0 + e]));
                     dc[e] = (uint8_t)(active ? acc(key) : code_of_key(key));
                 }
-            }
-        } else {
-            for (uint32_t e = cv.first + threadIdx.x; e < cv.len; e += kBigThreads) {
-                const uint32_t key = key_of(__fsub_rn(gr0[cv.a0 + e], st0[cv.a0 + e]));
-                dc[e] = (uint8_t)(active ? acc(key) : code_of_key(key));
             }
         }
         if (active) dirty = true;
